@@ -1,0 +1,121 @@
+/*
+ * sdwino -- stride-1, pad-1, 3x3 2-D convolution by the Winograd algorithm on one
+ * NVIDIA B200 (sm_100a).  C ABI; every pointer is a DEVICE pointer unless stated;
+ * `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *
+ * The operation is the one the paper accelerates: the 3x3 `ggml_conv_2d` of Stable
+ * Diffusion's UNet and VAE (Abstract; Section "Techniques"), split, as that section
+ * lists, into (i) a preprocess of the filter and of the activation, (ii) an
+ * element-wise multiplication of the preprocessed tensors and (iii) a postprocess of
+ * the intermediate result.  Tensor layouts are those of the header of Table 1
+ * (Filter = [KW,KH,IC,OC], Activation = [IW,IH,IC,N], fastest dimension first), i.e.
+ * contiguous w[K][C][3][3] and x[N][C][H][W].
+ *
+ * Semantics: cross-correlation (no filter flip), zero padding 1, stride 1, dilation 1,
+ * groups 1; fp16 storage, fp32 arithmetic and accumulation, one round-to-nearest-even
+ * to fp16 per stored value.  `tile` is the output tile edge m of F(m x m, 3 x 3):
+ * 2 or 4.  All calls are asynchronous on `stream`: SDWINO_OK means "enqueued".
+ * The library never allocates device memory except where a function says so, keeps no
+ * reference to caller buffers after a call except the registered workspace, and has no
+ * CPU fallback: without a CUDA device every compute call returns SDWINO_ERR_CUDA.
+ */
+#ifndef SDWINO_H
+#define SDWINO_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SDWINO_OK = 0,
+    SDWINO_ERR_INVALID_ARG = 1, /* NULL required pointer, dimension <= 0, size overflow       */
+    SDWINO_ERR_UNSUPPORTED = 2, /* tile not in {2,4}                                          */
+    SDWINO_ERR_MISALIGNED = 3,  /* x, w, bias or y not 2-byte aligned; wT / workspace not 1024-byte aligned */
+    SDWINO_ERR_WORKSPACE = 4,   /* no workspace registered / passed, or it is too small       */
+    SDWINO_ERR_CUDA = 5,        /* a CUDA runtime or driver call failed (see cudaGetLastError) */
+    SDWINO_ERR_TIMEOUT = 6      /* a bounded device-side wait gave up (sdwino_last_device_status) */
+} sdwino_status;
+
+/* Library version: major*10000 + minor*100 + patch. */
+int sdwino_version(void);
+
+/* Static, human-readable name of a status code. */
+const char *sdwino_status_string(int status);
+
+/*
+ * Filter preprocess, step (i) of Section "Techniques": U[k][c] = G w[k][c] G^T.
+ *
+ * sdwino_filter_bytes: bytes the caller must allocate for wT (0 on bad arguments).
+ * sdwino_filter_transform: w is fp16 [K][C][3][3]; wT receives fp16 U laid out as
+ *   [a*a][Kp][Cp] with a = tile+2, Kp = K rounded up to 128, Cp = C rounded up to 64,
+ *   position index xi*a+nu, zero in the padding.  wT must be 1024-byte aligned (any
+ *   cudaMalloc / torch allocation is).  wT depends on `tile`; pass the same tile to
+ *   sdwino_conv3x3.  Done once per weight; the caller owns both buffers.
+ */
+size_t sdwino_filter_bytes(int K, int C, int tile);
+int sdwino_filter_transform(const void *w, void *wT, int K, int C, int tile, void *stream);
+
+/*
+ * Scratch for the transformed activation V and the per-position products M (steps (i)
+ * and (ii)).  sdwino_workspace_bytes returns the size that lets the call run in the
+ * fewest passes while keeping V and M of one pass resident in the L2 cache (0 on bad
+ * arguments); any workspace of at least sdwino_workspace_min_bytes is accepted and only
+ * changes how many passes over the tile list are made.  The workspace is caller-owned,
+ * must be 1024-byte aligned, is overwritten by every call, and may be shared by calls
+ * that are ordered on one stream; calls on different streams need different workspaces.
+ * sdwino_set_workspace registers the scratch that sdwino_conv3x3 uses (NULL, 0 clears).
+ */
+size_t sdwino_workspace_bytes(int N, int C, int H, int W, int K, int tile);
+size_t sdwino_workspace_min_bytes(int N, int C, int H, int W, int K, int tile);
+int sdwino_set_workspace(void *workspace, size_t bytes);
+
+/*
+ * The convolution, steps (i) activation preprocess V = B^T d B on overlapping
+ * (tile+2)^2 windows, (ii) M = sum_c U (.) V per transform position (a batched GEMM on
+ * the tensor cores) and (iii) postprocess Y = A^T M A, plus bias, cast and store.
+ *
+ *   x    fp16 [N][C][H][W]   (read only)         bias fp16 [K] or NULL (= 0)
+ *   wT   from sdwino_filter_transform(K, C, tile)
+ *   y    fp16 [N][K][H][W]   (written; must not overlap x or the workspace)
+ *
+ * H and W need not be multiples of tile: windows are zero-extended past every edge and
+ * outputs outside the image are not stored.  sdwino_conv3x3 uses the registered
+ * workspace; sdwino_conv3x3_ws takes it explicitly.
+ */
+int sdwino_conv3x3(const void *x, const void *wT, const void *bias, void *y,
+                   int N, int C, int H, int W, int K, int tile, void *stream);
+int sdwino_conv3x3_ws(const void *x, const void *wT, const void *bias, void *y,
+                      int N, int C, int H, int W, int K, int tile,
+                      void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * The same convolution for callers whose tensors live in HOST memory (pageable or pinned):
+ * x_host, bias_host and y_host are host pointers, wT stays a device pointer.  On `stream`
+ * the call copies x (and bias) to the device, runs the three steps, copies y back and then
+ * synchronises the stream, so y_host is complete on return.  It allocates nothing: the
+ * device-side copies of x, bias and y are carved from the front of `workspace`, which must
+ * therefore hold sdwino_host_staging_bytes(...) in addition to a scratch accepted by
+ * sdwino_conv3x3_ws (at least sdwino_workspace_min_bytes).  Used for end-to-end timing.
+ */
+size_t sdwino_host_staging_bytes(int N, int C, int H, int W, int K, int tile);
+int sdwino_conv3x3_host(const void *x_host, const void *wT, const void *bias_host, void *y_host,
+                        int N, int C, int H, int W, int K, int tile,
+                        void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Device-side waits (on TMA / tensor-core completion barriers) are bounded; a wait that
+ * gives up records SDWINO_ERR_TIMEOUT in a device status word and the kernel returns
+ * normally.  This call synchronises `stream`, returns that word (SDWINO_OK if nothing
+ * was recorded) and clears it.
+ */
+int sdwino_last_device_status(void *stream);
+
+/* Kernel launches made by this library in the calling process so far (all entry points). */
+unsigned long long sdwino_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SDWINO_H */

@@ -1,0 +1,178 @@
+"""ctypes binding of the sdwino C ABI (include/sdwino.h).
+
+Argument marshalling only: every step of the convolution runs in the CUDA kernels of
+libsdwino.so.  torch is used for device memory and streams.  There is no fallback: if the
+shared library is missing the import of this module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+from .build import LIB_PATH
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_MISALIGNED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(7)
+
+EXPORTS = [
+    "sdwino_version", "sdwino_status_string", "sdwino_filter_bytes", "sdwino_filter_transform",
+    "sdwino_workspace_bytes", "sdwino_workspace_min_bytes", "sdwino_set_workspace", "sdwino_conv3x3",
+    "sdwino_conv3x3_ws", "sdwino_host_staging_bytes", "sdwino_conv3x3_host",
+    "sdwino_last_device_status", "sdwino_launch_count",
+]
+
+
+class SdwinoError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} ({status})")
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2412_05781_b200.build` "
+            "(there is no non-CUDA fallback)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+    lib.sdwino_version.restype = i
+    lib.sdwino_status_string.restype = ctypes.c_char_p
+    lib.sdwino_status_string.argtypes = [i]
+    lib.sdwino_filter_bytes.restype = sz
+    lib.sdwino_filter_bytes.argtypes = [i, i, i]
+    lib.sdwino_filter_transform.restype = i
+    lib.sdwino_filter_transform.argtypes = [vp, vp, i, i, i, vp]
+    for name in ("sdwino_workspace_bytes", "sdwino_workspace_min_bytes", "sdwino_host_staging_bytes"):
+        getattr(lib, name).restype = sz
+        getattr(lib, name).argtypes = [i] * 6
+    lib.sdwino_set_workspace.restype = i
+    lib.sdwino_set_workspace.argtypes = [vp, sz]
+    lib.sdwino_conv3x3.restype = i
+    lib.sdwino_conv3x3.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, vp]
+    lib.sdwino_conv3x3_ws.restype = i
+    lib.sdwino_conv3x3_ws.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, vp, sz, vp]
+    lib.sdwino_conv3x3_host.restype = i
+    lib.sdwino_conv3x3_host.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, vp, sz, vp]
+    lib.sdwino_last_device_status.restype = i
+    lib.sdwino_last_device_status.argtypes = [vp]
+    lib.sdwino_launch_count.restype = ctypes.c_ulonglong
+    return lib
+
+
+lib = _load()
+
+
+def status_string(status: int) -> str:
+    return lib.sdwino_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != OK:
+        raise SdwinoError(status, where)
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return s.cuda_stream
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def sdwino_version() -> int:
+    return int(lib.sdwino_version())
+
+
+def sdwino_filter_bytes(K: int, C: int, tile: int) -> int:
+    return int(lib.sdwino_filter_bytes(K, C, tile))
+
+
+def sdwino_workspace_bytes(N: int, C: int, H: int, W: int, K: int, tile: int) -> int:
+    return int(lib.sdwino_workspace_bytes(N, C, H, W, K, tile))
+
+
+def sdwino_workspace_min_bytes(N: int, C: int, H: int, W: int, K: int, tile: int) -> int:
+    return int(lib.sdwino_workspace_min_bytes(N, C, H, W, K, tile))
+
+
+def sdwino_host_staging_bytes(N: int, C: int, H: int, W: int, K: int, tile: int) -> int:
+    return int(lib.sdwino_host_staging_bytes(N, C, H, W, K, tile))
+
+
+def sdwino_launch_count() -> int:
+    return int(lib.sdwino_launch_count())
+
+
+def sdwino_last_device_status(stream: Optional[torch.cuda.Stream] = None) -> int:
+    return int(lib.sdwino_last_device_status(_stream_ptr(stream)))
+
+
+def alloc_workspace(nbytes: int, device="cuda") -> torch.Tensor:
+    """Device scratch of `nbytes` bytes (torch allocations are at least 512-byte aligned;
+    the returned view starts on a 1024-byte boundary)."""
+    buf = torch.empty(nbytes + 1024, dtype=torch.uint8, device=device)
+    off = (-buf.data_ptr()) % 1024
+    return buf[off:off + nbytes]
+
+
+def sdwino_filter_transform(w: torch.Tensor, tile: int, stream=None) -> torch.Tensor:
+    """w: fp16 CUDA [K, C, 3, 3] contiguous -> wT (opaque uint8 CUDA tensor, tile-specific)."""
+    assert w.is_cuda and w.dtype == torch.float16 and w.is_contiguous() and w.dim() == 4
+    K, C = int(w.shape[0]), int(w.shape[1])
+    assert tuple(w.shape[2:]) == (3, 3)
+    nbytes = sdwino_filter_bytes(K, C, tile)
+    if nbytes == 0:
+        raise SdwinoError(ERR_UNSUPPORTED if tile not in (2, 4) else ERR_INVALID_ARG, "sdwino_filter_bytes")
+    wT = alloc_workspace(nbytes, w.device)
+    _check(lib.sdwino_filter_transform(w.data_ptr(), wT.data_ptr(), K, C, tile, _stream_ptr(stream)),
+           "sdwino_filter_transform")
+    return wT
+
+
+def sdwino_set_workspace(workspace: Optional[torch.Tensor]) -> None:
+    if workspace is None:
+        _check(lib.sdwino_set_workspace(None, 0), "sdwino_set_workspace")
+    else:
+        _check(lib.sdwino_set_workspace(workspace.data_ptr(), workspace.numel() * workspace.element_size()),
+               "sdwino_set_workspace")
+
+
+def sdwino_conv3x3(x: torch.Tensor, wT: torch.Tensor, bias: Optional[torch.Tensor], K: int, tile: int,
+                   y: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                   stream=None) -> torch.Tensor:
+    """x: fp16 CUDA [N, C, H, W]; returns y fp16 [N, K, H, W].  With `workspace=None` the scratch
+    registered by sdwino_set_workspace is used."""
+    assert x.is_cuda and x.dtype == torch.float16 and x.is_contiguous() and x.dim() == 4
+    N, C, H, W = (int(v) for v in x.shape)
+    if y is None:
+        y = torch.empty((N, K, H, W), dtype=torch.float16, device=x.device)
+    assert y.is_contiguous() and y.dtype == torch.float16 and tuple(y.shape) == (N, K, H, W)
+    if bias is not None:
+        assert bias.is_cuda and bias.dtype == torch.float16 and bias.numel() == K and bias.is_contiguous()
+    if workspace is None:
+        rc = lib.sdwino_conv3x3(x.data_ptr(), wT.data_ptr(), _ptr(bias), y.data_ptr(), N, C, H, W, K, tile,
+                                _stream_ptr(stream))
+    else:
+        rc = lib.sdwino_conv3x3_ws(x.data_ptr(), wT.data_ptr(), _ptr(bias), y.data_ptr(), N, C, H, W, K, tile,
+                                   workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                                   _stream_ptr(stream))
+    _check(rc, "sdwino_conv3x3")
+    return y
+
+
+def sdwino_conv3x3_host(x: torch.Tensor, wT: torch.Tensor, bias: Optional[torch.Tensor], y: torch.Tensor,
+                        tile: int, workspace: torch.Tensor, stream=None) -> torch.Tensor:
+    """x, bias, y: fp16 CPU tensors (ideally pinned); wT and workspace on the device.  Returns y
+    after the stream has been synchronised."""
+    assert not x.is_cuda and not y.is_cuda and x.dtype == torch.float16 and y.dtype == torch.float16
+    assert x.is_contiguous() and y.is_contiguous()
+    N, C, H, W = (int(v) for v in x.shape)
+    K = int(y.shape[1])
+    rc = lib.sdwino_conv3x3_host(x.data_ptr(), wT.data_ptr(), _ptr(bias), y.data_ptr(), N, C, H, W, K, tile,
+                                 workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                                 _stream_ptr(stream))
+    _check(rc, "sdwino_conv3x3_host")
+    return y

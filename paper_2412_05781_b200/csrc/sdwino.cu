@@ -1,0 +1,346 @@
+// Host side of the sdwino C ABI: argument checks, workspace planning, tensor-map
+// construction and kernel launches.  See include/sdwino.h for the contract.
+#include "../../include/sdwino.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <atomic>
+#include <mutex>
+#include <unordered_map>
+
+#include "transforms.cuh"
+#include "wino_gemm.cuh"
+
+namespace {
+
+using namespace sdw;
+
+__device__ int g_status_word = 0;
+
+std::atomic<unsigned long long> g_launches{0};
+std::mutex g_mutex;
+void* g_workspace = nullptr;
+size_t g_workspace_bytes = 0;
+
+constexpr int GEMM_BLOCK_N = 128;
+constexpr int GEMM_STAGES = 5;
+// V and M of one pass over the tile list should stay in the 126 MB L2 together with the
+// operands being streamed; this is the budget for the two of them.
+constexpr size_t L2_PASS_BUDGET = 64ull << 20;
+constexpr size_t WS_ALIGN = 1024;
+
+inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
+inline long long round_up_ll(long long v, long long m) { return (v + m - 1) / m * m; }
+
+struct Plan {
+    int a2;            // transform positions
+    int Kp, Cp;        // padded filter dims
+    int TH, TW;
+    long long P;       // tiles in the whole batch
+    long long P128;    // P rounded up to the GEMM tile
+    size_t per_tile;   // workspace bytes per tile column (V + M)
+};
+
+bool make_plan(int N, int C, int H, int W, int K, int tile, Plan* pl) {
+    if (N <= 0 || C <= 0 || H <= 0 || W <= 0 || K <= 0) return false;
+    if (tile != 2 && tile != 4) return false;
+    const int a = tile + 2;
+    pl->a2 = a * a;
+    pl->Kp = round_up(K, GEMM_BLOCK_M);
+    pl->Cp = round_up(C, GEMM_BLOCK_K);
+    pl->TH = (H + tile - 1) / tile;
+    pl->TW = (W + tile - 1) / tile;
+    pl->P = static_cast<long long>(N) * pl->TH * pl->TW;
+    pl->P128 = round_up_ll(pl->P, GEMM_BLOCK_N);
+    pl->per_tile = static_cast<size_t>(pl->a2) * (static_cast<size_t>(C) + pl->Kp) * sizeof(__half);
+    // element counts must stay far inside int64
+    const long double big = 9.0e18L;
+    if (static_cast<long double>(N) * C * H * W > big || static_cast<long double>(N) * K * H * W > big) return false;
+    if (pl->P128 > (1ll << 40)) return false;
+    return true;
+}
+
+// Tiles per pass for a workspace of `bytes` (0 = not even one GEMM tile fits).
+long long tiles_per_pass(const Plan& pl, size_t bytes) {
+    long long fit = static_cast<long long>(bytes / pl.per_tile) / GEMM_BLOCK_N * GEMM_BLOCK_N;
+    long long want = static_cast<long long>(L2_PASS_BUDGET / pl.per_tile) / GEMM_BLOCK_N * GEMM_BLOCK_N;
+    if (want < 4 * GEMM_BLOCK_N) want = 4 * GEMM_BLOCK_N;
+    long long pc = fit < want ? fit : want;
+    if (pc > pl.P128) pc = pl.P128;
+    return pc;
+}
+
+// ---- driver entry point for tensor maps (no link-time dependency on libcuda) ----
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    });
+    return fn;
+}
+
+// fp16 tensor [d2][d1][d0] (d0 contiguous, row pitch `pitch0` elements, plane pitch `pitch1`
+// elements) with a {b0, b1, 1} box and the 128-byte swizzle.
+bool encode_map(CUtensorMap* m, const void* base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t pitch0,
+                uint64_t pitch1, uint32_t b0, uint32_t b1) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {d0, d1, d2};
+    cuuint64_t strides[2] = {pitch0 * sizeof(__half), pitch1 * sizeof(__half)};
+    cuuint32_t box[3] = {b0, b1, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+int sm_count() {
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n = 0;
+    }
+    return n;
+}
+
+template <int M>
+int launch_filter(const __half* w, __half* U, int K, int C, int Kp, int Cp, cudaStream_t st) {
+    dim3 grid((Cp + 255) / 256, Kp);
+    filter_transform_kernel<M><<<grid, 256, 0, st>>>(w, U, K, C, Kp, Cp);
+    g_launches.fetch_add(1);
+    return cudaGetLastError() == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
+}
+
+template <int M>
+int launch_input(const __half* x, __half* V, const TileGeom& geo, int C, long long p_begin, int p_count,
+                 long long Pstride, cudaStream_t st) {
+    dim3 grid((p_count + 127) / 128, C);
+    input_transform_kernel<M><<<grid, 128, 0, st>>>(x, V, geo, C, p_begin, p_count, Pstride);
+    g_launches.fetch_add(1);
+    return cudaGetLastError() == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
+}
+
+template <int M>
+int launch_output(const __half* Mws, const __half* bias, __half* y, const TileGeom& geo, int K, int Kp,
+                  long long p_begin, int p_count, long long Pstride, cudaStream_t st) {
+    dim3 grid((p_count + 127) / 128, K);
+    output_transform_kernel<M><<<grid, 128, 0, st>>>(Mws, bias, y, geo, K, Kp, p_begin, p_count, Pstride);
+    g_launches.fetch_add(1);
+    return cudaGetLastError() == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
+}
+
+int launch_gemm(const CUtensorMap& tmU, const CUtensorMap& tmV, const CUtensorMap& tmM, int num_k_tiles,
+                int num_p_tiles, int num_pos, int num_c_blocks, cudaStream_t st) {
+    using L = GemmSmem<GEMM_BLOCK_N, GEMM_STAGES>;
+    auto kern = wino_gemm_kernel<GEMM_BLOCK_N, GEMM_STAGES>;
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [&] {
+        attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES);
+    });
+    if (attr_err != cudaSuccess) return SDWINO_ERR_CUDA;
+    const int sms = sm_count();
+    if (sms <= 0) return SDWINO_ERR_CUDA;
+    const long long tiles = static_cast<long long>(num_k_tiles) * num_p_tiles * num_pos;
+    const int grid = static_cast<int>(tiles < sms ? tiles : sms);
+    int* status = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&status), g_status_word) != cudaSuccess) return SDWINO_ERR_CUDA;
+    kern<<<grid, GEMM_THREADS, L::DYN_BYTES, st>>>(tmU, tmV, tmM, num_k_tiles, num_p_tiles, num_pos, num_c_blocks,
+                                                   status);
+    g_launches.fetch_add(1);
+    return cudaGetLastError() == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
+}
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, int C, int H, int W, int K, int tile,
+              void* ws, size_t ws_bytes, cudaStream_t st) {
+    if (tile != 2 && tile != 4) {
+        return (N <= 0 || C <= 0 || H <= 0 || W <= 0 || K <= 0 || !x || !wT || !y) ? SDWINO_ERR_INVALID_ARG
+                                                                                     : SDWINO_ERR_UNSUPPORTED;
+    }
+    Plan pl;
+    if (!x || !wT || !y || !make_plan(N, C, H, W, K, tile, &pl)) return SDWINO_ERR_INVALID_ARG;
+    if (!aligned(x, 2) || !aligned(y, 2) || (bias && !aligned(bias, 2)) || !aligned(wT, WS_ALIGN))
+        return SDWINO_ERR_MISALIGNED;
+    if (!ws || ws_bytes == 0) return SDWINO_ERR_WORKSPACE;
+    if (!aligned(ws, WS_ALIGN)) return SDWINO_ERR_MISALIGNED;
+    const long long pc = tiles_per_pass(pl, ws_bytes);
+    if (pc < GEMM_BLOCK_N) return SDWINO_ERR_WORKSPACE;
+
+    // workspace: V[a2][C][pc] then M[a2][Kp][pc]; both start on 1024-byte boundaries because pc is a
+    // multiple of 128 elements and the counts of rows are integers (pc * 2 bytes = multiple of 256).
+    __half* V = static_cast<__half*>(ws);
+    size_t v_bytes = static_cast<size_t>(pl.a2) * C * pc * sizeof(__half);
+    v_bytes = (v_bytes + WS_ALIGN - 1) / WS_ALIGN * WS_ALIGN;
+    __half* Mws = reinterpret_cast<__half*>(static_cast<uint8_t*>(ws) + v_bytes);
+    const size_t m_bytes = static_cast<size_t>(pl.a2) * pl.Kp * pc * sizeof(__half);
+    if (v_bytes + m_bytes > ws_bytes) return SDWINO_ERR_WORKSPACE;
+
+    CUtensorMap tmU, tmV, tmM;
+    if (!encode_map(&tmU, wT, pl.Cp, pl.Kp, pl.a2, pl.Cp, static_cast<uint64_t>(pl.Kp) * pl.Cp, 64, GEMM_BLOCK_M) ||
+        !encode_map(&tmV, V, pc, C, pl.a2, pc, static_cast<uint64_t>(C) * pc, 64, GEMM_BLOCK_K) ||
+        !encode_map(&tmM, Mws, pc, pl.Kp, pl.a2, pc, static_cast<uint64_t>(pl.Kp) * pc, 64, GEMM_BLOCK_M))
+        return SDWINO_ERR_CUDA;
+
+    TileGeom geo{H, W, pl.TH, pl.TW, pl.P};
+    const __half* xh = static_cast<const __half*>(x);
+    const __half* bh = static_cast<const __half*>(bias);
+    __half* yh = static_cast<__half*>(y);
+    for (long long p0 = 0; p0 < pl.P; p0 += pc) {
+        long long remaining = pl.P128 - p0;
+        const int count = static_cast<int>(remaining < pc ? remaining : pc);  // multiple of 128
+        int rc;
+        if (tile == 2) rc = launch_input<2>(xh, V, geo, C, p0, count, pc, st);
+        else rc = launch_input<4>(xh, V, geo, C, p0, count, pc, st);
+        if (rc != SDWINO_OK) return rc;
+        rc = launch_gemm(tmU, tmV, tmM, pl.Kp / GEMM_BLOCK_M, count / GEMM_BLOCK_N, pl.a2, pl.Cp / GEMM_BLOCK_K, st);
+        if (rc != SDWINO_OK) return rc;
+        if (tile == 2) rc = launch_output<2>(Mws, bh, yh, geo, K, pl.Kp, p0, count, pc, st);
+        else rc = launch_output<4>(Mws, bh, yh, geo, K, pl.Kp, p0, count, pc, st);
+        if (rc != SDWINO_OK) return rc;
+    }
+    return SDWINO_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int sdwino_version(void) { return 100; }
+
+const char* sdwino_status_string(int status) {
+    switch (status) {
+        case SDWINO_OK: return "ok";
+        case SDWINO_ERR_INVALID_ARG: return "invalid argument";
+        case SDWINO_ERR_UNSUPPORTED: return "unsupported tile size";
+        case SDWINO_ERR_MISALIGNED: return "misaligned pointer";
+        case SDWINO_ERR_WORKSPACE: return "workspace missing or too small";
+        case SDWINO_ERR_CUDA: return "CUDA error";
+        case SDWINO_ERR_TIMEOUT: return "device-side wait timed out";
+        default: return "unknown status";
+    }
+}
+
+size_t sdwino_filter_bytes(int K, int C, int tile) {
+    if (K <= 0 || C <= 0 || (tile != 2 && tile != 4)) return 0;
+    const size_t a = tile + 2;
+    return a * a * static_cast<size_t>(round_up(K, GEMM_BLOCK_M)) * round_up(C, GEMM_BLOCK_K) * sizeof(__half);
+}
+
+int sdwino_filter_transform(const void* w, void* wT, int K, int C, int tile, void* stream) {
+    if (!w || !wT || K <= 0 || C <= 0) return SDWINO_ERR_INVALID_ARG;
+    if (tile != 2 && tile != 4) return SDWINO_ERR_UNSUPPORTED;
+    if (!aligned(w, 2) || !aligned(wT, WS_ALIGN)) return SDWINO_ERR_MISALIGNED;
+    if (static_cast<long double>(K) * C > 4.0e15L) return SDWINO_ERR_INVALID_ARG;
+    const int Kp = round_up(K, GEMM_BLOCK_M), Cp = round_up(C, GEMM_BLOCK_K);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (tile == 2) return launch_filter<2>(static_cast<const __half*>(w), static_cast<__half*>(wT), K, C, Kp, Cp, st);
+    return launch_filter<4>(static_cast<const __half*>(w), static_cast<__half*>(wT), K, C, Kp, Cp, st);
+}
+
+size_t sdwino_workspace_bytes(int N, int C, int H, int W, int K, int tile) {
+    Plan pl;
+    if (!make_plan(N, C, H, W, K, tile, &pl)) return 0;
+    const long long pc = tiles_per_pass(pl, static_cast<size_t>(-1) / 2);
+    return static_cast<size_t>(pc) * pl.per_tile + WS_ALIGN;
+}
+
+size_t sdwino_workspace_min_bytes(int N, int C, int H, int W, int K, int tile) {
+    Plan pl;
+    if (!make_plan(N, C, H, W, K, tile, &pl)) return 0;
+    return static_cast<size_t>(GEMM_BLOCK_N) * pl.per_tile + WS_ALIGN;
+}
+
+int sdwino_set_workspace(void* workspace, size_t bytes) {
+    if ((workspace == nullptr) != (bytes == 0)) return SDWINO_ERR_INVALID_ARG;
+    if (workspace && !aligned(workspace, WS_ALIGN)) return SDWINO_ERR_MISALIGNED;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    g_workspace = workspace;
+    g_workspace_bytes = bytes;
+    return SDWINO_OK;
+}
+
+int sdwino_conv3x3_ws(const void* x, const void* wT, const void* bias, void* y, int N, int C, int H, int W, int K,
+                      int tile, void* workspace, size_t workspace_bytes, void* stream) {
+    return conv_impl(x, wT, bias, y, N, C, H, W, K, tile, workspace, workspace_bytes,
+                     static_cast<cudaStream_t>(stream));
+}
+
+int sdwino_conv3x3(const void* x, const void* wT, const void* bias, void* y, int N, int C, int H, int W, int K,
+                   int tile, void* stream) {
+    void* ws;
+    size_t bytes;
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        ws = g_workspace;
+        bytes = g_workspace_bytes;
+    }
+    return conv_impl(x, wT, bias, y, N, C, H, W, K, tile, ws, bytes, static_cast<cudaStream_t>(stream));
+}
+
+size_t sdwino_host_staging_bytes(int N, int C, int H, int W, int K, int tile) {
+    Plan pl;
+    if (!make_plan(N, C, H, W, K, tile, &pl)) return 0;
+    auto up = [](size_t v) { return (v + WS_ALIGN - 1) / WS_ALIGN * WS_ALIGN; };
+    const size_t xb = up(static_cast<size_t>(N) * C * H * W * sizeof(__half));
+    const size_t yb = up(static_cast<size_t>(N) * K * H * W * sizeof(__half));
+    const size_t bb = up(static_cast<size_t>(K) * sizeof(__half));
+    return xb + yb + bb;
+}
+
+int sdwino_conv3x3_host(const void* x_host, const void* wT, const void* bias_host, void* y_host, int N, int C, int H,
+                        int W, int K, int tile, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!x_host || !y_host || !wT) return SDWINO_ERR_INVALID_ARG;
+    if (tile != 2 && tile != 4) return SDWINO_ERR_UNSUPPORTED;
+    const size_t staging = sdwino_host_staging_bytes(N, C, H, W, K, tile);
+    if (staging == 0) return SDWINO_ERR_INVALID_ARG;
+    if (!workspace || workspace_bytes <= staging) return SDWINO_ERR_WORKSPACE;
+    if (!aligned(workspace, WS_ALIGN)) return SDWINO_ERR_MISALIGNED;
+    auto up = [](size_t v) { return (v + WS_ALIGN - 1) / WS_ALIGN * WS_ALIGN; };
+    const size_t xbytes = static_cast<size_t>(N) * C * H * W * sizeof(__half);
+    const size_t ybytes = static_cast<size_t>(N) * K * H * W * sizeof(__half);
+    uint8_t* base = static_cast<uint8_t*>(workspace);
+    uint8_t* xd = base;
+    uint8_t* yd = xd + up(xbytes);
+    uint8_t* bd = yd + up(ybytes);
+    uint8_t* ws = base + staging;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(xd, x_host, xbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return SDWINO_ERR_CUDA;
+    if (bias_host &&
+        cudaMemcpyAsync(bd, bias_host, static_cast<size_t>(K) * sizeof(__half), cudaMemcpyHostToDevice, st) !=
+            cudaSuccess)
+        return SDWINO_ERR_CUDA;
+    int rc = conv_impl(xd, wT, bias_host ? bd : nullptr, yd, N, C, H, W, K, tile, ws, workspace_bytes - staging, st);
+    if (rc != SDWINO_OK) return rc;
+    if (cudaMemcpyAsync(y_host, yd, ybytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return SDWINO_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return SDWINO_ERR_CUDA;
+    return SDWINO_OK;
+}
+
+int sdwino_last_device_status(void* stream) {
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return SDWINO_ERR_CUDA;
+    int v = 0;
+    if (cudaMemcpyFromSymbol(&v, g_status_word, sizeof(int)) != cudaSuccess) return SDWINO_ERR_CUDA;
+    if (v != 0) {
+        int zero = 0;
+        if (cudaMemcpyToSymbol(g_status_word, &zero, sizeof(int)) != cudaSuccess) return SDWINO_ERR_CUDA;
+    }
+    return v;
+}
+
+unsigned long long sdwino_launch_count(void) { return g_launches.load(); }
+
+}  // extern "C"

@@ -1,0 +1,259 @@
+// Steps (i) and (iii) of Section "Techniques": filter preprocess U = G g G^T, activation
+// preprocess V = B^T d B on overlapping (m+2)x(m+2) windows, and postprocess
+// Y = A^T M A followed by bias add, rounding to fp16 and a store masked at the image edge.
+// These kernels are bandwidth-bound: one thread per (channel, tile), consecutive threads on
+// consecutive tiles so that every global access of a warp is contiguous.
+//
+// The paper prints no matrices; these are the Toom-Cook matrices of the construction it cites.
+// F(2x2,3x3) uses the points {0, 1, -1, inf}; F(4x4,3x3) uses {0, 3/4, -3/4, 3/2, -3/2, inf},
+// whose B^T and A^T entries are dyadic and whose fp16 error is about a third of that of the
+// integer points {0, +-1, +-2, inf}.
+#pragma once
+#include <cuda_fp16.h>
+#include <stdint.h>
+
+namespace sdw {
+
+template <int M> struct Wino;
+
+template <> struct Wino<2> {
+    static constexpr int A = 4;
+    struct Bt {
+        __host__ __device__ constexpr float operator()(int i, int j) const {
+            constexpr float m[4][4] = {{1, 0, -1, 0}, {0, 1, 1, 0}, {0, -1, 1, 0}, {0, 1, 0, -1}};
+            return m[i][j];
+        }
+    };
+    struct G {
+        __host__ __device__ constexpr float operator()(int i, int j) const {
+            constexpr float m[4][3] = {{1, 0, 0}, {0.5f, 0.5f, 0.5f}, {0.5f, -0.5f, 0.5f}, {0, 0, 1}};
+            return m[i][j];
+        }
+    };
+    struct At {
+        __host__ __device__ constexpr float operator()(int i, int j) const {
+            constexpr float m[2][4] = {{1, 1, 1, 0}, {0, 1, -1, -1}};
+            return m[i][j];
+        }
+    };
+};
+
+template <> struct Wino<4> {
+    static constexpr int A = 6;
+    struct Bt {
+        __host__ __device__ constexpr float operator()(int i, int j) const {
+            constexpr float m[6][6] = {{1.265625f, 0, -2.8125f, 0, 1, 0},    {0, -1.6875f, -2.25f, 0.75f, 1, 0},
+                                       {0, 1.6875f, -2.25f, -0.75f, 1, 0},   {0, -0.84375f, -0.5625f, 1.5f, 1, 0},
+                                       {0, 0.84375f, -0.5625f, -1.5f, 1, 0}, {0, 1.265625f, 0, -2.8125f, 0, 1}};
+            return m[i][j];
+        }
+    };
+    struct G {
+        __host__ __device__ constexpr float operator()(int i, int j) const {
+            constexpr float m[6][3] = {{64.f / 81.f, 0, 0},
+                                       {-128.f / 243.f, -32.f / 81.f, -8.f / 27.f},
+                                       {-128.f / 243.f, 32.f / 81.f, -8.f / 27.f},
+                                       {32.f / 243.f, 16.f / 81.f, 8.f / 27.f},
+                                       {32.f / 243.f, -16.f / 81.f, 8.f / 27.f},
+                                       {0, 0, 1}};
+            return m[i][j];
+        }
+    };
+    struct At {
+        __host__ __device__ constexpr float operator()(int i, int j) const {
+            constexpr float m[4][6] = {{1, 1, 1, 1, 1, 0},
+                                       {0, 0.75f, -0.75f, 1.5f, -1.5f, 0},
+                                       {0, 0.5625f, 0.5625f, 2.25f, 2.25f, 0},
+                                       {0, 0.421875f, -0.421875f, 3.375f, -3.375f, 1}};
+            return m[i][j];
+        }
+    };
+};
+
+// out[i] = sum_j coef[i][j] * in[j] with compile-time coefficients: zero terms vanish and
+// unit terms become adds once the loops are unrolled.
+template <int R, int Cn, typename MatT>
+__device__ __forceinline__ void mat_apply(MatT coef, const float (&in)[Cn], float (&out)[R]) {
+#pragma unroll
+    for (int i = 0; i < R; ++i) {
+        float acc = 0.f;
+        bool first = true;
+#pragma unroll
+        for (int j = 0; j < Cn; ++j) {
+            const float cf = coef(i, j);
+            if (cf != 0.f) {
+                if (first) { acc = cf * in[j]; first = false; }
+                else acc = fmaf(cf, in[j], acc);
+            }
+        }
+        out[i] = acc;
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Filter preprocess.  One thread per (k, c) of the padded [Kp][Cp] plane; writes all a*a
+// positions (zeros in the padding).  U layout: [a*a][Kp][Cp], c contiguous.
+// ---------------------------------------------------------------------------------------
+template <int M>
+__global__ void __launch_bounds__(256)
+filter_transform_kernel(const __half* __restrict__ w, __half* __restrict__ U, int K, int C, int Kp, int Cp) {
+    using Wm = Wino<M>;
+    constexpr int A = Wm::A;
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    const int k = blockIdx.y;
+    if (c >= Cp) return;
+    float g[3][3];
+    const bool live = (k < K) && (c < C);
+#pragma unroll
+    for (int r = 0; r < 3; ++r)
+#pragma unroll
+        for (int s = 0; s < 3; ++s)
+            g[r][s] = live ? __half2float(w[(static_cast<size_t>(k) * C + c) * 9 + r * 3 + s]) : 0.f;
+    // t = G g  (A x 3), u = t G^T (A x A)
+    float t[A][3];
+#pragma unroll
+    for (int s = 0; s < 3; ++s) {
+        float col[3] = {g[0][s], g[1][s], g[2][s]};
+        float o[A];
+        mat_apply<A, 3>(typename Wm::G{}, col, o);
+#pragma unroll
+        for (int i = 0; i < A; ++i) t[i][s] = o[i];
+    }
+    const size_t plane = static_cast<size_t>(Kp) * Cp;
+    __half* dst = U + static_cast<size_t>(k) * Cp + c;
+#pragma unroll
+    for (int i = 0; i < A; ++i) {
+        float o[A];
+        mat_apply<A, 3>(typename Wm::G{}, t[i], o);
+#pragma unroll
+        for (int j = 0; j < A; ++j) dst[(i * A + j) * plane] = __float2half_rn(o[j]);
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Tile index arithmetic shared by both activation-side kernels.  Tile p (global index over
+// the whole batch) belongs to image n = p / (TH*TW), tile row th and tile column tw; its
+// input window starts at pixel (m*th - 1, m*tw - 1) and its outputs at (m*th, m*tw).
+// ---------------------------------------------------------------------------------------
+struct TileGeom {
+    int H, W, TH, TW;
+    long long P;  // N*TH*TW
+};
+
+// Activation preprocess.  V layout: [a*a][C][Pstride] with the chunk-local tile index
+// (p - p_begin) contiguous.  Threads past the last tile write zeros so that the GEMM reads
+// defined data.
+template <int M>
+__global__ void __launch_bounds__(128)
+input_transform_kernel(const __half* __restrict__ x, __half* __restrict__ V, TileGeom geo, int C, long long p_begin,
+                       int p_count, long long Pstride) {
+    using Wm = Wino<M>;
+    constexpr int A = Wm::A;
+    const int pl = blockIdx.x * blockDim.x + threadIdx.x;  // chunk-local tile
+    const int c = blockIdx.y;
+    if (pl >= p_count) return;
+    const long long p = p_begin + pl;
+    float d[A][A];
+    if (p < geo.P) {
+        const int tw = static_cast<int>(p % geo.TW);
+        const int th = static_cast<int>((p / geo.TW) % geo.TH);
+        const long long n = p / (static_cast<long long>(geo.TW) * geo.TH);
+        const __half* img = x + (n * C + c) * static_cast<long long>(geo.H) * geo.W;
+        const int i0 = M * th - 1, j0 = M * tw - 1;
+#pragma unroll
+        for (int r = 0; r < A; ++r) {
+            const int i = i0 + r;
+            const bool rin = (i >= 0) && (i < geo.H);
+#pragma unroll
+            for (int s = 0; s < A; ++s) {
+                const int j = j0 + s;
+                d[r][s] = (rin && j >= 0 && j < geo.W) ? __half2float(__ldg(img + static_cast<long long>(i) * geo.W + j))
+                                                        : 0.f;
+            }
+        }
+    } else {
+#pragma unroll
+        for (int r = 0; r < A; ++r)
+#pragma unroll
+            for (int s = 0; s < A; ++s) d[r][s] = 0.f;
+    }
+    // t = B^T d (column by column), v = t B (row by row)
+    float t[A][A];
+#pragma unroll
+    for (int s = 0; s < A; ++s) {
+        float col[A], o[A];
+#pragma unroll
+        for (int r = 0; r < A; ++r) col[r] = d[r][s];
+        mat_apply<A, A>(typename Wm::Bt{}, col, o);
+#pragma unroll
+        for (int r = 0; r < A; ++r) t[r][s] = o[r];
+    }
+    const long long plane = static_cast<long long>(C) * Pstride;
+    __half* dst = V + static_cast<long long>(c) * Pstride + pl;
+#pragma unroll
+    for (int r = 0; r < A; ++r) {
+        float o[A];
+        mat_apply<A, A>(typename Wm::Bt{}, t[r], o);
+#pragma unroll
+        for (int s = 0; s < A; ++s) dst[(r * A + s) * plane] = __float2half_rn(o[s]);
+    }
+}
+
+// Postprocess + bias + cast + masked store.  Mws layout: [a*a][Kp][Pstride]; y is NCHW.
+template <int M>
+__global__ void __launch_bounds__(128)
+output_transform_kernel(const __half* __restrict__ Mws, const __half* __restrict__ bias, __half* __restrict__ y,
+                        TileGeom geo, int K, int Kp, long long p_begin, int p_count, long long Pstride) {
+    using Wm = Wino<M>;
+    constexpr int A = Wm::A;
+    const int pl = blockIdx.x * blockDim.x + threadIdx.x;
+    const int k = blockIdx.y;
+    if (pl >= p_count) return;
+    const long long p = p_begin + pl;
+    if (p >= geo.P) return;
+    const long long plane = static_cast<long long>(Kp) * Pstride;
+    const __half* src = Mws + static_cast<long long>(k) * Pstride + pl;
+    float mm[A][A];
+#pragma unroll
+    for (int r = 0; r < A; ++r)
+#pragma unroll
+        for (int s = 0; s < A; ++s) mm[r][s] = __half2float(__ldg(src + (r * A + s) * plane));
+    // t = A^T mm (M x A), Y = t A (M x M)
+    float t[M][A];
+#pragma unroll
+    for (int s = 0; s < A; ++s) {
+        float col[A], o[M];
+#pragma unroll
+        for (int r = 0; r < A; ++r) col[r] = mm[r][s];
+        mat_apply<M, A>(typename Wm::At{}, col, o);
+#pragma unroll
+        for (int i = 0; i < M; ++i) t[i][s] = o[i];
+    }
+    const int tw = static_cast<int>(p % geo.TW);
+    const int th = static_cast<int>((p / geo.TW) % geo.TH);
+    const long long n = p / (static_cast<long long>(geo.TW) * geo.TH);
+    const float b = bias ? __half2float(__ldg(bias + k)) : 0.f;
+    __half* img = y + (n * K + k) * static_cast<long long>(geo.H) * geo.W;
+    const int i0 = M * th, j0 = M * tw;
+    const bool vec_ok = ((geo.W & 1) == 0) && ((reinterpret_cast<uintptr_t>(y) & 3) == 0);
+#pragma unroll
+    for (int i = 0; i < M; ++i) {
+        float o[M];
+        mat_apply<M, A>(typename Wm::At{}, t[i], o);
+        const int oi = i0 + i;
+        if (oi >= geo.H) continue;
+        __half* rowp = img + static_cast<long long>(oi) * geo.W + j0;
+#pragma unroll
+        for (int j = 0; j < M; j += 2) {
+            const __half h0 = __float2half_rn(o[j] + b), h1 = __float2half_rn(o[j + 1] + b);
+            if (vec_ok && (j0 + j + 1 < geo.W)) {
+                *reinterpret_cast<__half2*>(rowp + j) = __halves2half2(h0, h1);
+            } else {
+                if (j0 + j < geo.W) rowp[j] = h0;
+                if (j0 + j + 1 < geo.W) rowp[j + 1] = h1;
+            }
+        }
+    }
+}
+
+}  // namespace sdw

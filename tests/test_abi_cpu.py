@@ -1,0 +1,97 @@
+"""Host-only checks of the C-ABI boundary: the library builds, loads and exports every symbol the
+header declares, and argument validation answers without a GPU."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_2412_05781_b200 import build_library
+    build_library()
+    from paper_2412_05781_b200 import binding as b
+    return b
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "sdwino.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(sdwino_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(binding):
+    names = _declared_symbols()
+    assert "sdwino_conv3x3" in names and "sdwino_filter_transform" in names
+    for n in names:
+        assert hasattr(binding.lib, n), n
+    assert sorted(binding.EXPORTS) == names
+
+
+def test_version_and_status_strings(binding):
+    assert binding.sdwino_version() >= 100
+    seen = {binding.status_string(s) for s in range(7)}
+    assert len(seen) == 7 and "ok" in seen
+    assert binding.status_string(99) == "unknown status"
+
+
+def test_size_queries(binding):
+    # wT = a*a planes of [K rounded to 128][C rounded to 64] fp16
+    assert binding.sdwino_filter_bytes(320, 320, 2) == 16 * 384 * 320 * 2
+    assert binding.sdwino_filter_bytes(3, 4, 4) == 36 * 128 * 64 * 2
+    assert binding.sdwino_filter_bytes(0, 4, 2) == 0
+    assert binding.sdwino_filter_bytes(4, 4, 3) == 0
+    full = binding.sdwino_workspace_bytes(2, 320, 64, 64, 320, 2)
+    small = binding.sdwino_workspace_min_bytes(2, 320, 64, 64, 320, 2)
+    # P = 2*32*32 = 2048 tiles, (C + Kp) = 704 fp16 per position and tile
+    assert full == 2048 * 16 * 704 * 2 + 1024
+    assert small == 128 * 16 * 704 * 2 + 1024
+    assert binding.sdwino_workspace_bytes(1, 1, 1, 1, 1, 5) == 0
+    assert binding.sdwino_workspace_bytes(1, 0, 1, 1, 1, 2) == 0
+    assert binding.sdwino_host_staging_bytes(1, 4, 8, 8, 4, 2) == 1024 * 3
+
+
+def test_argument_validation_without_gpu(binding):
+    lib = binding.lib
+    buf = ctypes.create_string_buffer(4096)
+    p = (ctypes.addressof(buf) + 1023) // 1024 * 1024
+    assert lib.sdwino_filter_transform(None, p, 4, 4, 2, None) == binding.ERR_INVALID_ARG
+    assert lib.sdwino_filter_transform(p, p, 4, 4, 3, None) == binding.ERR_UNSUPPORTED
+    assert lib.sdwino_filter_transform(p + 1, p, 4, 4, 2, None) == binding.ERR_MISALIGNED
+    assert lib.sdwino_filter_transform(p, p + 16, 4, 4, 2, None) == binding.ERR_MISALIGNED
+    assert lib.sdwino_conv3x3_ws(None, p, None, p, 1, 4, 8, 8, 4, 2, p, 1 << 20, None) == binding.ERR_INVALID_ARG
+    assert lib.sdwino_conv3x3_ws(p, p, None, p, 1, 4, 8, 0, 4, 2, p, 1 << 20, None) == binding.ERR_INVALID_ARG
+    assert lib.sdwino_conv3x3_ws(p, p, None, p, 1, 4, 8, 8, 4, 6, p, 1 << 20, None) == binding.ERR_UNSUPPORTED
+    assert lib.sdwino_conv3x3_ws(p, p, None, p + 1, 1, 4, 8, 8, 4, 2, p, 1 << 20, None) == binding.ERR_MISALIGNED
+    assert lib.sdwino_conv3x3_ws(p, p, None, p, 1, 4, 8, 8, 4, 2, None, 0, None) == binding.ERR_WORKSPACE
+    assert lib.sdwino_conv3x3_ws(p, p, None, p, 1, 4, 8, 8, 4, 2, p, 4096, None) == binding.ERR_WORKSPACE
+    assert lib.sdwino_conv3x3_ws(p, p, None, p, 1, 4, 8, 8, 4, 2, p + 8, 1 << 20, None) == binding.ERR_MISALIGNED
+    # no workspace registered
+    assert lib.sdwino_set_workspace(None, 0) == binding.OK
+    assert lib.sdwino_conv3x3(p, p, None, p, 1, 4, 8, 8, 4, 2, None) == binding.ERR_WORKSPACE
+    assert lib.sdwino_set_workspace(p, 0) == binding.ERR_INVALID_ARG
+    assert lib.sdwino_set_workspace(p + 4, 64) == binding.ERR_MISALIGNED
+    assert lib.sdwino_conv3x3_host(None, p, None, p, 1, 4, 8, 8, 4, 2, p, 1 << 20, None) == binding.ERR_INVALID_ARG
+    assert lib.sdwino_conv3x3_host(p, p, None, p, 1, 4, 8, 8, 4, 2, p, 1024, None) == binding.ERR_WORKSPACE
+
+
+def test_missing_library_fails_loudly(monkeypatch, binding):
+    import importlib
+    from paper_2412_05781_b200 import build as bmod
+    monkeypatch.setattr(bmod, "LIB_PATH", "/nonexistent/libsdwino.so")
+    import paper_2412_05781_b200.binding as bind
+    monkeypatch.setattr(bind, "LIB_PATH", "/nonexistent/libsdwino.so")
+    with pytest.raises(ImportError):
+        bind._load()
+
+
+def test_product_package_does_not_import_oracle():
+    pkg = os.path.join(ROOT, "paper_2412_05781_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                src = open(os.path.join(dirpath, f)).read()
+                assert "import oracle" not in src and "from oracle" not in src and "conv_oracle" not in src, f
