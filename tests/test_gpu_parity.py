@@ -1,0 +1,245 @@
+"""Parity of the CUDA path (through the C ABI) with the fp64 oracle on seeded synthetic inputs.
+
+Bar: max|gpu - ref| <= 1e-2 * max|ref| per layer, ref = fp64 direct convolution of the fp16 inputs
+(fp16 storage, fp32 accumulation).  The same bound is evaluated separately on the edge tiles.  A tighter
+regression bound is asserted for F(2x2,3x3), whose error is dominated by the fp16 rounding of V and M
+(about 7e-4 measured; 2.5e-3 leaves a 3x margin).
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2412_05781_b200 import workloads
+from paper_2412_05781_b200.workloads import ConvLayer
+
+pytestmark = pytest.mark.gpu
+
+TOL = 1e-2
+TOL_F2_REGRESSION = 2.5e-3
+F4_POINTS = (0, 0.75, -0.75, 1.5, -1.5)
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2412_05781_b200 import build_library
+    build_library()
+    from paper_2412_05781_b200 import binding
+    assert torch.cuda.is_available()
+    return binding
+
+
+def _run(B, layer, tile, seed=0, with_bias=True, ws_bytes=None, x=None, w=None, b=None):
+    if x is None:
+        x, w, b = workloads.make_inputs(layer, seed=seed, with_bias=with_bias)
+    wT = B.sdwino_filter_transform(w.cuda(), tile)
+    if ws_bytes is None:
+        ws_bytes = B.sdwino_workspace_bytes(layer.N, layer.C, layer.H, layer.W, layer.K, tile)
+    ws = B.alloc_workspace(ws_bytes)
+    y = B.sdwino_conv3x3(x.cuda(), wT, None if b is None else b.cuda(), layer.K, tile, workspace=ws)
+    assert B.sdwino_last_device_status() == B.OK
+    return x, w, b, y.cpu()
+
+
+def _rel_err(y, ref):
+    return float(np.abs(y.double().numpy() - ref).max() / np.abs(ref).max())
+
+
+def _edge_mask(H, W, m):
+    """Pixels belonging to the first/last tile row or column."""
+    TH, TW = -(-H // m), -(-W // m)
+    mask = np.zeros((H, W), dtype=bool)
+    mask[:m, :] = True
+    mask[:, :m] = True
+    mask[(TH - 1) * m:, :] = True
+    mask[:, (TW - 1) * m:] = True
+    return mask
+
+
+SMALL = [
+    # C, K, H, W, N   -- several GEMM tiles in every direction plus ragged tails
+    (1, 1, 4, 4, 1), (3, 4, 5, 7, 2), (4, 7, 1, 1, 3), (7, 33, 2, 9, 1), (33, 3, 13, 1, 2),
+    (64, 128, 16, 16, 1), (65, 129, 17, 19, 1), (96, 160, 18, 21, 2), (130, 257, 33, 35, 1),
+    (16, 16, 40, 56, 3), (200, 64, 23, 46, 1),
+]
+
+
+@pytest.mark.parametrize("tile", [2, 4])
+@pytest.mark.parametrize("shape", SMALL)
+def test_small_shapes_elementwise(B, shape, tile):
+    C, K, H, W, N = shape
+    layer = ConvLayer(C=C, K=K, H=H, W=W, N=N)
+    x, w, b, y = _run(B, layer, tile, seed=sum(shape))
+    ref = oracle.direct_conv3x3(x.numpy(), w.numpy(), b.numpy())
+    err = _rel_err(y, ref)
+    assert err <= (TOL_F2_REGRESSION if tile == 2 else TOL), err
+    # the same bound on the edge tiles alone (padding and tile-index logic)
+    mask = _edge_mask(H, W, tile)
+    d = np.abs(y.double().numpy() - ref)[:, :, mask].max()
+    assert d <= TOL * np.abs(ref).max()
+    # and against the three-step fp64 Winograd route with the same interpolation points
+    wino = oracle.winograd_conv3x3(x.numpy(), w.numpy(), b.numpy(), m=tile, points=None if tile == 2 else F4_POINTS)
+    assert _rel_err(y, wino) <= TOL
+
+
+@pytest.mark.parametrize("tile", [2, 4])
+def test_no_bias_and_zero_input(B, tile):
+    layer = ConvLayer(C=20, K=24, H=11, W=10, N=2)
+    x, w, b, y = _run(B, layer, tile, with_bias=False)
+    ref = oracle.direct_conv3x3(x.numpy(), w.numpy(), None)
+    assert _rel_err(y, ref) <= TOL
+    # x = 0  =>  y = bias exactly (every transform of zero is zero)
+    x0, w0, b0 = workloads.make_inputs(layer, seed=3)
+    x0.zero_()
+    _, _, _, y0 = _run(B, layer, tile, x=x0, w=w0, b=b0)
+    assert torch.equal(y0, b0.view(1, -1, 1, 1).expand_as(y0))
+
+
+@pytest.mark.parametrize("tile", [2, 4])
+def test_delta_filter_copies_input(B, tile):
+    # centre tap 1 on the diagonal: y = x.  F(2x2) reproduces it exactly (all transforms are sums of
+    # fp16 values that stay representable for |x| <= 2); F(4x4) within tolerance.
+    layer = ConvLayer(C=8, K=8, H=12, W=14, N=1)
+    x, w, b = workloads.make_inputs(layer, seed=5, with_bias=False)
+    x = (x * 8).round() / 8
+    x.clamp_(-2, 2)
+    w.zero_()
+    for c in range(8):
+        w[c, c, 1, 1] = 1
+    _, _, _, y = _run(B, layer, tile, x=x, w=w, b=None)
+    if tile == 2:
+        assert torch.equal(y, x)
+    else:
+        assert (y.float() - x.float()).abs().max() <= TOL * x.float().abs().max()
+
+
+@pytest.mark.parametrize("tile", [2, 4])
+@pytest.mark.parametrize("KC", [(320, 320), (3, 128), (130, 7)])
+def test_filter_transform_matches_oracle(B, KC, tile):
+    K, C = KC
+    a = tile + 2
+    g = torch.Generator().manual_seed(K + C)
+    w = (torch.randn(K, C, 3, 3, generator=g) / (9 * C) ** 0.5).half()
+    wT = B.sdwino_filter_transform(w.cuda(), tile)
+    Kp, Cp = -(-K // 128) * 128, -(-C // 64) * 64
+    U = wT.view(torch.float16).view(a * a, Kp, Cp).cpu()
+    Uo = oracle.filter_transform(w.numpy(), tile, points=None if tile == 2 else F4_POINTS)
+    Uo = torch.from_numpy(Uo.reshape(K, C, a * a).transpose(2, 0, 1).copy())
+    got = U[:, :K, :C].double()
+    # |U - fp16(U64)| <= 1 ulp(fp16): compare with the two fp16 neighbours of the exact value
+    ref16 = Uo.half()
+    ulp = torch.maximum((torch.nextafter(ref16, torch.full_like(ref16, float("inf"))) - ref16).double().abs(),
+                        (ref16 - torch.nextafter(ref16, torch.full_like(ref16, -float("inf")))).double().abs())
+    assert bool(((got - ref16.double()).abs() <= ulp).all())
+    # padding rows / columns are zero
+    assert float(U[:, K:, :].abs().max() if Kp > K else 0) == 0
+    assert float(U[:, :, C:].abs().max() if Cp > C else 0) == 0
+
+
+def test_single_layer_config_full(B):
+    # the small single-layer configuration, every output element
+    layer = workloads.single_layer()[0]
+    x, w, b, y = _run(B, layer, 2)
+    ref = oracle.direct_conv3x3(x.numpy(), w.numpy(), b.numpy())
+    assert _rel_err(y, ref) <= TOL_F2_REGRESSION
+
+
+def _sampled_check(B, layer, tile, nch, seed=0):
+    x, w, b, y = _run(B, layer, tile, seed=seed)
+    rng = np.random.default_rng(seed + layer.K)
+    ks = np.sort(rng.choice(layer.K, size=min(nch, layer.K), replace=False))
+    ref = oracle.direct_conv3x3(x.numpy(), w.numpy(), b.numpy(), channels=ks.tolist())
+    got = y[:, torch.from_numpy(ks)].double().numpy()
+    scale = np.abs(ref).max()
+    err = np.abs(got - ref).max() / scale
+    mask = _edge_mask(layer.H, layer.W, tile)
+    edge = np.abs(got - ref)[:, :, mask].max() / scale
+    return err, edge
+
+
+@pytest.mark.parametrize("idx", range(16))
+def test_sd15_unet_layers_sampled_channels(B, idx):
+    # the benchmarked workload at full size: 16 seeded output channels, all spatial positions
+    layer = workloads.sd15_unet()[idx]
+    err, edge = _sampled_check(B, layer, 2, 16)
+    assert err <= TOL_F2_REGRESSION and edge <= TOL, (layer.name, err, edge)
+
+
+@pytest.mark.parametrize("idx", [0, 1, 2, 5, 9])
+def test_vae_layers_sampled_channels(B, idx):
+    layer = workloads.sd_vae_decoder_512()[idx]
+    nch = 16 if layer.direct_flops < 1e11 else 4
+    err, edge = _sampled_check(B, layer, 2, nch)
+    assert err <= TOL_F2_REGRESSION and edge <= TOL, (layer.name, err, edge)
+
+
+@pytest.mark.parametrize("idx,N", [(1, 1), (3, 2), (6, 4), (7, 1), (15, 8)])
+@pytest.mark.parametrize("tile", [2, 4])
+def test_sd21_unet_layers_both_tiles(B, idx, N, tile):
+    layer = workloads.sd21_unet(N)[idx]
+    err, edge = _sampled_check(B, layer, tile, 8)
+    assert err <= TOL and edge <= TOL, (layer.name, tile, err, edge)
+
+
+def test_multi_pass_equals_single_pass_bitwise(B):
+    layer = ConvLayer(C=48, K=72, H=50, W=46, N=2)      # 1150 tiles -> 9 GEMM tiles of 128
+    x, w, b = workloads.make_inputs(layer, seed=9)
+    _, _, _, y_full = _run(B, layer, 2, x=x, w=w, b=b)
+    small = B.sdwino_workspace_min_bytes(layer.N, layer.C, layer.H, layer.W, layer.K, 2)
+    _, _, _, y_min = _run(B, layer, 2, x=x, w=w, b=b, ws_bytes=small)            # 128 tiles per pass
+    _, _, _, y_mid = _run(B, layer, 2, x=x, w=w, b=b, ws_bytes=small * 3 + 5000)  # 384 tiles per pass
+    assert torch.equal(y_full, y_min) and torch.equal(y_full, y_mid)
+
+
+def test_run_to_run_determinism_and_canaries(B):
+    layer = ConvLayer(C=40, K=36, H=21, W=27, N=2)
+    x, w, b = workloads.make_inputs(layer, seed=11)
+    wT = B.sdwino_filter_transform(w.cuda(), 2)
+    ws = B.alloc_workspace(B.sdwino_workspace_bytes(layer.N, layer.C, layer.H, layer.W, layer.K, 2))
+    n = layer.N * layer.K * layer.H * layer.W
+    pad = 4096
+    canary = torch.full((n + 2 * pad,), 1234.0, dtype=torch.float16, device="cuda")
+    y = canary[pad:pad + n].view(layer.N, layer.K, layer.H, layer.W)
+    B.sdwino_conv3x3(x.cuda(), wT, b.cuda(), layer.K, 2, y=y, workspace=ws)
+    first = y.clone()
+    B.sdwino_conv3x3(x.cuda(), wT, b.cuda(), layer.K, 2, y=y, workspace=ws)
+    assert B.sdwino_last_device_status() == B.OK
+    assert torch.equal(first, y)
+    assert bool((canary[:pad] == 1234.0).all()) and bool((canary[pad + n:] == 1234.0).all())
+
+
+def test_registered_workspace_and_host_entry_match_device_entry(B):
+    layer = ConvLayer(C=24, K=40, H=19, W=16, N=2)
+    x, w, b = workloads.make_inputs(layer, seed=13)
+    _, _, _, y_dev = _run(B, layer, 2, x=x, w=w, b=b)
+    wT = B.sdwino_filter_transform(w.cuda(), 2)
+    ws = B.alloc_workspace(B.sdwino_workspace_bytes(layer.N, layer.C, layer.H, layer.W, layer.K, 2))
+    B.sdwino_set_workspace(ws)
+    try:
+        y_reg = B.sdwino_conv3x3(x.cuda(), wT, b.cuda(), layer.K, 2)
+        assert torch.equal(y_reg.cpu(), y_dev)
+    finally:
+        B.sdwino_set_workspace(None)
+    with pytest.raises(B.SdwinoError) as e:
+        B.sdwino_conv3x3(x.cuda(), wT, b.cuda(), layer.K, 2)
+    assert e.value.status == B.ERR_WORKSPACE
+    args = (layer.N, layer.C, layer.H, layer.W, layer.K, 2)
+    hws = B.alloc_workspace(B.sdwino_host_staging_bytes(*args) + B.sdwino_workspace_bytes(*args))
+    y_host = torch.empty(layer.N, layer.K, layer.H, layer.W, dtype=torch.float16).pin_memory()
+    B.sdwino_conv3x3_host(x.pin_memory(), wT, b.pin_memory(), y_host, 2, hws)
+    assert torch.equal(y_host, y_dev)
+
+
+def test_non_default_stream_and_launch_counter(B):
+    layer = ConvLayer(C=16, K=16, H=8, W=8, N=1)
+    x, w, b = workloads.make_inputs(layer, seed=17)
+    _, _, _, y_ref = _run(B, layer, 2, x=x, w=w, b=b)
+    s = torch.cuda.Stream()
+    before = B.sdwino_launch_count()
+    with torch.cuda.stream(s):
+        wT = B.sdwino_filter_transform(w.cuda(), 2)
+        ws = B.alloc_workspace(B.sdwino_workspace_bytes(1, 16, 8, 8, 16, 2))
+        y = B.sdwino_conv3x3(x.cuda(), wT, b.cuda(), 16, 2, workspace=ws)
+    s.synchronize()
+    assert B.sdwino_launch_count() - before == 4      # filter + input + GEMM + output
+    assert torch.equal(y.cpu(), y_ref)
