@@ -115,6 +115,18 @@ int sdwino_last_device_status(void *stream);
 /* Kernel launches made by this library in the calling process so far (all entry points). */
 unsigned long long sdwino_launch_count(void);
 
+/*
+ * Per-kernel timing for benchmarks.  While enabled, every kernel launch of the library is
+ * bracketed by two CUDA events recorded on the launch's stream (this adds a little idle time
+ * between kernels, so whole-call timings should be taken with profiling disabled).
+ * sdwino_profile_collect waits for the recorded events, adds the elapsed milliseconds and
+ * the launch counts per kernel kind into the two caller arrays of 4 entries (0 filter
+ * transform, 1 activation transform, 2 batched GEMM, 3 output transform; either may be NULL)
+ * and forgets the records.  Host arrays; not thread-safe against concurrent compute calls.
+ */
+int sdwino_profile_enable(int enable);
+int sdwino_profile_collect(double *ms_by_kind, unsigned long long *launches_by_kind);
+
 #ifdef __cplusplus
 }
 #endif

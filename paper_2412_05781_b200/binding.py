@@ -20,8 +20,10 @@ EXPORTS = [
     "sdwino_version", "sdwino_status_string", "sdwino_filter_bytes", "sdwino_filter_transform",
     "sdwino_workspace_bytes", "sdwino_workspace_min_bytes", "sdwino_set_workspace", "sdwino_conv3x3",
     "sdwino_conv3x3_ws", "sdwino_host_staging_bytes", "sdwino_conv3x3_host",
-    "sdwino_last_device_status", "sdwino_launch_count",
+    "sdwino_last_device_status", "sdwino_launch_count", "sdwino_profile_enable", "sdwino_profile_collect",
 ]
+
+KERNEL_KINDS = ("filter_transform", "input_transform", "wino_gemm", "output_transform")
 
 
 class SdwinoError(RuntimeError):
@@ -58,6 +60,10 @@ def _load() -> ctypes.CDLL:
     lib.sdwino_last_device_status.restype = i
     lib.sdwino_last_device_status.argtypes = [vp]
     lib.sdwino_launch_count.restype = ctypes.c_ulonglong
+    lib.sdwino_profile_enable.restype = i
+    lib.sdwino_profile_enable.argtypes = [i]
+    lib.sdwino_profile_collect.restype = i
+    lib.sdwino_profile_collect.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_ulonglong)]
     return lib
 
 
@@ -108,6 +114,18 @@ def sdwino_launch_count() -> int:
 
 def sdwino_last_device_status(stream: Optional[torch.cuda.Stream] = None) -> int:
     return int(lib.sdwino_last_device_status(_stream_ptr(stream)))
+
+
+def sdwino_profile_enable(enable: bool) -> None:
+    _check(lib.sdwino_profile_enable(1 if enable else 0), "sdwino_profile_enable")
+
+
+def sdwino_profile_collect():
+    """-> {kernel kind: (total milliseconds, launches)} since the last collect."""
+    ms = (ctypes.c_double * 4)()
+    n = (ctypes.c_ulonglong * 4)()
+    _check(lib.sdwino_profile_collect(ms, n), "sdwino_profile_collect")
+    return {k: (float(ms[i]), int(n[i])) for i, k in enumerate(KERNEL_KINDS)}
 
 
 def alloc_workspace(nbytes: int, device="cuda") -> torch.Tensor:

@@ -8,7 +8,7 @@
 
 #include <atomic>
 #include <mutex>
-#include <unordered_map>
+#include <vector>
 
 #include "transforms.cuh"
 #include "wino_gemm.cuh"
@@ -23,6 +23,33 @@ std::atomic<unsigned long long> g_launches{0};
 std::mutex g_mutex;
 void* g_workspace = nullptr;
 size_t g_workspace_bytes = 0;
+
+// Optional per-kernel timing: when enabled every launch is bracketed by CUDA events on its stream.
+enum KernelKind { KIND_FILTER = 0, KIND_INPUT = 1, KIND_GEMM = 2, KIND_OUTPUT = 3, KIND_COUNT = 4 };
+struct ProfRecord { int kind; cudaEvent_t beg, end; };
+bool g_profile = false;
+std::vector<ProfRecord> g_prof_records;
+std::vector<cudaEvent_t> g_event_pool;
+
+cudaEvent_t prof_event() {
+    cudaEvent_t e = nullptr;
+    if (!g_event_pool.empty()) { e = g_event_pool.back(); g_event_pool.pop_back(); return e; }
+    if (cudaEventCreate(&e) != cudaSuccess) return nullptr;
+    return e;
+}
+struct ProfScope {
+    cudaStream_t st; int kind; cudaEvent_t beg = nullptr;
+    ProfScope(int k, cudaStream_t s) : st(s), kind(k) {
+        if (g_profile) { beg = prof_event(); if (beg) cudaEventRecord(beg, st); }
+    }
+    ~ProfScope() {
+        if (beg) {
+            cudaEvent_t end = prof_event();
+            if (end) { cudaEventRecord(end, st); g_prof_records.push_back({kind, beg, end}); }
+            else g_event_pool.push_back(beg);
+        }
+    }
+};
 
 constexpr int GEMM_BLOCK_N = 128;
 constexpr int GEMM_STAGES = 5;
@@ -118,6 +145,7 @@ int sm_count() {
 template <int M>
 int launch_filter(const __half* w, __half* U, int K, int C, int Kp, int Cp, cudaStream_t st) {
     dim3 grid((Cp + 255) / 256, Kp);
+    ProfScope prof(KIND_FILTER, st);
     filter_transform_kernel<M><<<grid, 256, 0, st>>>(w, U, K, C, Kp, Cp);
     g_launches.fetch_add(1);
     return cudaGetLastError() == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
@@ -127,6 +155,7 @@ template <int M>
 int launch_input(const __half* x, __half* V, const TileGeom& geo, int C, long long p_begin, int p_count,
                  long long Pstride, cudaStream_t st) {
     dim3 grid((p_count + 127) / 128, C);
+    ProfScope prof(KIND_INPUT, st);
     input_transform_kernel<M><<<grid, 128, 0, st>>>(x, V, geo, C, p_begin, p_count, Pstride);
     g_launches.fetch_add(1);
     return cudaGetLastError() == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
@@ -136,6 +165,7 @@ template <int M>
 int launch_output(const __half* Mws, const __half* bias, __half* y, const TileGeom& geo, int K, int Kp,
                   long long p_begin, int p_count, long long Pstride, cudaStream_t st) {
     dim3 grid((p_count + 127) / 128, K);
+    ProfScope prof(KIND_OUTPUT, st);
     output_transform_kernel<M><<<grid, 128, 0, st>>>(Mws, bias, y, geo, K, Kp, p_begin, p_count, Pstride);
     g_launches.fetch_add(1);
     return cudaGetLastError() == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
@@ -157,6 +187,7 @@ int launch_gemm(const CUtensorMap& tmU, const CUtensorMap& tmV, const CUtensorMa
     const int grid = static_cast<int>(tiles < sms ? tiles : sms);
     int* status = nullptr;
     if (cudaGetSymbolAddress(reinterpret_cast<void**>(&status), g_status_word) != cudaSuccess) return SDWINO_ERR_CUDA;
+    ProfScope prof(KIND_GEMM, st);
     kern<<<grid, GEMM_THREADS, L::DYN_BYTES, st>>>(tmU, tmV, tmM, num_k_tiles, num_p_tiles, num_pos, num_c_blocks,
                                                    status);
     g_launches.fetch_add(1);
@@ -342,5 +373,33 @@ int sdwino_last_device_status(void* stream) {
 }
 
 unsigned long long sdwino_launch_count(void) { return g_launches.load(); }
+
+int sdwino_profile_enable(int enable) {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    g_profile = enable != 0;
+    return SDWINO_OK;
+}
+
+int sdwino_profile_collect(double* ms_by_kind, unsigned long long* launches_by_kind) {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    int rc = SDWINO_OK;
+    for (int k = 0; k < KIND_COUNT; ++k) {
+        if (ms_by_kind) ms_by_kind[k] = 0.0;
+        if (launches_by_kind) launches_by_kind[k] = 0;
+    }
+    for (const ProfRecord& r : g_prof_records) {
+        float ms = 0.f;
+        if (cudaEventSynchronize(r.end) != cudaSuccess || cudaEventElapsedTime(&ms, r.beg, r.end) != cudaSuccess) {
+            rc = SDWINO_ERR_CUDA;
+        } else {
+            if (ms_by_kind) ms_by_kind[r.kind] += ms;
+            if (launches_by_kind) launches_by_kind[r.kind] += 1;
+        }
+        g_event_pool.push_back(r.beg);
+        g_event_pool.push_back(r.end);
+    }
+    g_prof_records.clear();
+    return rc;
+}
 
 }  // extern "C"
