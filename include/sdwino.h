@@ -49,10 +49,10 @@ const char *sdwino_status_string(int status);
  *
  * sdwino_filter_bytes: bytes the caller must allocate for wT (0 on bad arguments).
  * sdwino_filter_transform: w is fp16 [K][C][3][3]; wT receives fp16 U laid out as
- *   [a*a][Kp][Cp] with a = tile+2, Kp = K rounded up to 128, Cp = C rounded up to 64,
- *   position index xi*a+nu, zero in the padding.  wT must be 1024-byte aligned (any
- *   cudaMalloc / torch allocation is).  wT depends on `tile`; pass the same tile to
- *   sdwino_conv3x3.  Done once per weight; the caller owns both buffers.
+ *   [a*a][K][C8] with a = tile+2, C8 = C rounded up to 8 (16-byte rows), position index
+ *   xi*a+nu, zero in the padding columns.  wT must be 1024-byte aligned (a cudaMalloc
+ *   base is).  wT depends on `tile`; pass the same tile to sdwino_conv3x3.  Done once
+ *   per weight; the caller owns both buffers.
  */
 size_t sdwino_filter_bytes(int K, int C, int tile);
 int sdwino_filter_transform(const void *w, void *wT, int K, int C, int tile, void *stream);
@@ -114,6 +114,16 @@ int sdwino_last_device_status(void *stream);
 
 /* Kernel launches made by this library in the calling process so far (all entry points). */
 unsigned long long sdwino_launch_count(void);
+
+/*
+ * Tuning and test hook for the batched GEMM of step (ii).  By default the library picks, per
+ * call, between single-CTA tiles (128 tiles x n output channels) and CTA-pair tiles (256 tiles x
+ * n output channels, tcgen05 cta_group::2) and the n that fits the layer.  ctas in {1, 2} and/or
+ * n_tile (a multiple of 16 in [16, 256]) force that choice for later calls of this process; 0
+ * restores the automatic choice for that field.  Results do not depend on the choice beyond
+ * the fp32 summation order inside the tensor core.  Returns SDWINO_ERR_INVALID_ARG otherwise.
+ */
+int sdwino_set_gemm_shape(int ctas, int n_tile);
 
 /*
  * Per-kernel timing for benchmarks.  While enabled, every kernel launch of the library is

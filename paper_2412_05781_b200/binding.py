@@ -21,6 +21,7 @@ EXPORTS = [
     "sdwino_workspace_bytes", "sdwino_workspace_min_bytes", "sdwino_set_workspace", "sdwino_conv3x3",
     "sdwino_conv3x3_ws", "sdwino_host_staging_bytes", "sdwino_conv3x3_host",
     "sdwino_last_device_status", "sdwino_launch_count", "sdwino_profile_enable", "sdwino_profile_collect",
+    "sdwino_set_gemm_shape",
 ]
 
 KERNEL_KINDS = ("filter_transform", "input_transform", "wino_gemm", "output_transform")
@@ -60,6 +61,8 @@ def _load() -> ctypes.CDLL:
     lib.sdwino_last_device_status.restype = i
     lib.sdwino_last_device_status.argtypes = [vp]
     lib.sdwino_launch_count.restype = ctypes.c_ulonglong
+    lib.sdwino_set_gemm_shape.restype = i
+    lib.sdwino_set_gemm_shape.argtypes = [i, i]
     lib.sdwino_profile_enable.restype = i
     lib.sdwino_profile_enable.argtypes = [i]
     lib.sdwino_profile_collect.restype = i
@@ -114,6 +117,11 @@ def sdwino_launch_count() -> int:
 
 def sdwino_last_device_status(stream: Optional[torch.cuda.Stream] = None) -> int:
     return int(lib.sdwino_last_device_status(_stream_ptr(stream)))
+
+
+def sdwino_set_gemm_shape(ctas: int = 0, n_tile: int = 0) -> None:
+    """Force single-CTA (1) or CTA-pair (2) GEMM tiles and/or the channels per tile; 0 = automatic."""
+    _check(lib.sdwino_set_gemm_shape(ctas, n_tile), "sdwino_set_gemm_shape")
 
 
 def sdwino_profile_enable(enable: bool) -> None:

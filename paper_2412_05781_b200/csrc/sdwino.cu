@@ -6,6 +6,9 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <stdio.h>
+#include <stdlib.h>
+
 #include <atomic>
 #include <mutex>
 #include <vector>
@@ -21,6 +24,9 @@ __device__ int g_status_word = 0;
 
 std::atomic<unsigned long long> g_launches{0};
 std::mutex g_mutex;
+// test / tuning overrides of the GEMM launch shape (0 = choose automatically)
+int g_force_ctas = 0;
+int g_force_n_tile = 0;
 void* g_workspace = nullptr;
 size_t g_workspace_bytes = 0;
 
@@ -51,8 +57,7 @@ struct ProfScope {
     }
 };
 
-constexpr int GEMM_BLOCK_N = 128;
-constexpr int GEMM_STAGES = 5;
+constexpr int MAX_DYN_SMEM = 232448;  // 227 KB opt-in limit per CTA on sm_100
 // V and M of one pass over the tile list should stay in the 126 MB L2 together with the
 // operands being streamed; this is the budget for the two of them.
 constexpr size_t L2_PASS_BUDGET = 64ull << 20;
@@ -63,7 +68,7 @@ inline long long round_up_ll(long long v, long long m) { return (v + m - 1) / m 
 
 struct Plan {
     int a2;            // transform positions
-    int Kp, Cp;        // padded filter dims
+    int C8;            // row pitch of U in elements (C rounded up to 8: 16-byte rows for TMA)
     int TH, TW;
     long long P;       // tiles in the whole batch
     long long P128;    // P rounded up to the GEMM tile
@@ -75,13 +80,12 @@ bool make_plan(int N, int C, int H, int W, int K, int tile, Plan* pl) {
     if (tile != 2 && tile != 4) return false;
     const int a = tile + 2;
     pl->a2 = a * a;
-    pl->Kp = round_up(K, GEMM_BLOCK_M);
-    pl->Cp = round_up(C, GEMM_BLOCK_K);
+    pl->C8 = round_up(C, 8);
     pl->TH = (H + tile - 1) / tile;
     pl->TW = (W + tile - 1) / tile;
     pl->P = static_cast<long long>(N) * pl->TH * pl->TW;
-    pl->P128 = round_up_ll(pl->P, GEMM_BLOCK_N);
-    pl->per_tile = static_cast<size_t>(pl->a2) * (static_cast<size_t>(C) + pl->Kp) * sizeof(__half);
+    pl->P128 = round_up_ll(pl->P, GEMM_BLOCK_P);
+    pl->per_tile = static_cast<size_t>(pl->a2) * (static_cast<size_t>(C) + K) * sizeof(__half);
     // element counts must stay far inside int64
     const long double big = 9.0e18L;
     if (static_cast<long double>(N) * C * H * W > big || static_cast<long double>(N) * K * H * W > big) return false;
@@ -91,9 +95,9 @@ bool make_plan(int N, int C, int H, int W, int K, int tile, Plan* pl) {
 
 // Tiles per pass for a workspace of `bytes` (0 = not even one GEMM tile fits).
 long long tiles_per_pass(const Plan& pl, size_t bytes) {
-    long long fit = static_cast<long long>(bytes / pl.per_tile) / GEMM_BLOCK_N * GEMM_BLOCK_N;
-    long long want = static_cast<long long>(L2_PASS_BUDGET / pl.per_tile) / GEMM_BLOCK_N * GEMM_BLOCK_N;
-    if (want < 4 * GEMM_BLOCK_N) want = 4 * GEMM_BLOCK_N;
+    long long fit = static_cast<long long>(bytes / pl.per_tile) / GEMM_BLOCK_P * GEMM_BLOCK_P;
+    long long want = static_cast<long long>(L2_PASS_BUDGET / pl.per_tile) / GEMM_BLOCK_P * GEMM_BLOCK_P;
+    if (want < 4 * GEMM_BLOCK_P) want = 4 * GEMM_BLOCK_P;
     long long pc = fit < want ? fit : want;
     if (pc > pl.P128) pc = pl.P128;
     return pc;
@@ -117,9 +121,9 @@ EncodeTiledFn get_encode_fn() {
 }
 
 // fp16 tensor [d2][d1][d0] (d0 contiguous, row pitch `pitch0` elements, plane pitch `pitch1`
-// elements) with a {b0, b1, 1} box and the 128-byte swizzle.
+// elements) with a {b0, b1, 1} box, with the 128-byte swizzle or none.
 bool encode_map(CUtensorMap* m, const void* base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t pitch0,
-                uint64_t pitch1, uint32_t b0, uint32_t b1) {
+                uint64_t pitch1, uint32_t b0, uint32_t b1, bool swizzle128) {
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return false;
     cuuint64_t dims[3] = {d0, d1, d2};
@@ -127,7 +131,8 @@ bool encode_map(CUtensorMap* m, const void* base, uint64_t d0, uint64_t d1, uint
     cuuint32_t box[3] = {b0, b1, 1};
     cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
 }
@@ -143,10 +148,10 @@ int sm_count() {
 }
 
 template <int M>
-int launch_filter(const __half* w, __half* U, int K, int C, int Kp, int Cp, cudaStream_t st) {
-    dim3 grid((Cp + 255) / 256, Kp);
+int launch_filter(const __half* w, __half* U, int K, int C, int C8, cudaStream_t st) {
+    dim3 grid((C8 + 127) / 128, K);
     ProfScope prof(KIND_FILTER, st);
-    filter_transform_kernel<M><<<grid, 256, 0, st>>>(w, U, K, C, Kp, Cp);
+    filter_transform_kernel<M><<<grid, 128, 0, st>>>(w, U, K, C, C8);
     g_launches.fetch_add(1);
     return cudaGetLastError() == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
 }
@@ -162,36 +167,86 @@ int launch_input(const __half* x, __half* V, const TileGeom& geo, int C, long lo
 }
 
 template <int M>
-int launch_output(const __half* Mws, const __half* bias, __half* y, const TileGeom& geo, int K, int Kp,
+int launch_output(const __half* Mws, const __half* bias, __half* y, const TileGeom& geo, int K,
                   long long p_begin, int p_count, long long Pstride, cudaStream_t st) {
     dim3 grid((p_count + 127) / 128, K);
     ProfScope prof(KIND_OUTPUT, st);
-    output_transform_kernel<M><<<grid, 128, 0, st>>>(Mws, bias, y, geo, K, Kp, p_begin, p_count, Pstride);
+    output_transform_kernel<M><<<grid, 128, 0, st>>>(Mws, bias, y, geo, K, p_begin, p_count, Pstride);
     g_launches.fetch_add(1);
     return cudaGetLastError() == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
 }
 
-int launch_gemm(const CUtensorMap& tmU, const CUtensorMap& tmV, const CUtensorMap& tmM, int num_k_tiles,
-                int num_p_tiles, int num_pos, int num_c_blocks, cudaStream_t st) {
-    using L = GemmSmem<GEMM_BLOCK_N, GEMM_STAGES>;
-    auto kern = wino_gemm_kernel<GEMM_BLOCK_N, GEMM_STAGES>;
+// Shape of the GEMM launch: CTA pairs or single CTAs, and the output channels per tile (UMMA N, a
+// multiple of 16 up to 256).  The candidate with the smallest modelled time wins: a tile costs its
+// pipeline stages, each limited by the tensor pipe (2 n cycles per stage) or by the bytes the CTA must
+// fetch from L2 per stage (about 40 bytes per cycle per SM were measured), plus an epilogue that is
+// hidden unless the tile is short; tiles run in waves over the SMs.
+struct GemmShape { int ctas; int n_tile; };
+GemmShape choose_gemm_shape(int K, int C, long long p_tiles128, int a2, int sms) {
+    const long long cblocks = (C + GEMM_BLOCK_C - 1) / GEMM_BLOCK_C;
+    GemmShape best{1, 16};
+    double best_cost = 1e300;
+    for (int ctas = 1; ctas <= 2; ++ctas) {
+        if (ctas == 2 && p_tiles128 < 2) continue;
+        const long long p_tiles = (p_tiles128 + ctas - 1) / ctas;
+        const long long workers = sms / ctas;
+        for (int n = 16; n <= GEMM_MAX_N; n += 16) {
+            const long long ktiles = (K + n - 1) / n;
+            if (n > 16 && (ktiles == (K + n - 17) / (n - 16))) continue;  // a smaller n needs as many tiles
+            const long long tiles = ktiles * p_tiles * a2;
+            const long long waves = (tiles + workers - 1) / workers;
+            const double mma = 2.0 * n;
+            const double load = (GemmSmemLayout::A_BYTES + 128.0 * n / ctas) / 40.0;
+            const double main = cblocks * (mma > load ? mma : load);
+            const double epi = 300.0 + 14.0 * n;
+            const double per_tile = (main > epi ? main : epi) + 200.0;
+            const double cost = waves * per_tile + epi;
+            if (cost < best_cost) { best_cost = cost; best = GemmShape{ctas, n}; }
+        }
+    }
+    return best;
+}
+
+template <int CTAS>
+int launch_gemm_shape(const CUtensorMap& tmU, const CUtensorMap& tmV, const CUtensorMap& tmM, const GemmParams& prm,
+                      int sms, int* status, cudaStream_t st) {
+    using L = GemmSmemLayout;
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [&] {
-        attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES);
+        attr_err =
+            cudaFuncSetAttribute(wino_gemm_kernel<CTAS>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_DYN_SMEM);
     });
     if (attr_err != cudaSuccess) return SDWINO_ERR_CUDA;
+    const long long tiles = static_cast<long long>(prm.num_k_tiles) * prm.num_p_tiles * prm.num_pos;
+    const long long workers = sms / CTAS;
+    const int grid = static_cast<int>(tiles < workers ? tiles : workers) * CTAS;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(GEMM_THREADS);
+    cfg.dynamicSmemBytes = L::dyn_bytes(prm.n_tile / CTAS, prm.stages);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = CTAS;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    ProfScope prof(KIND_GEMM, st);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, wino_gemm_kernel<CTAS>, tmU, tmV, tmM, prm, status);
+    g_launches.fetch_add(1);
+    return e == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
+}
+
+int launch_gemm(const CUtensorMap& tmU, const CUtensorMap& tmV, const CUtensorMap& tmM, const GemmParams& prm,
+                int ctas, cudaStream_t st) {
     const int sms = sm_count();
     if (sms <= 0) return SDWINO_ERR_CUDA;
-    const long long tiles = static_cast<long long>(num_k_tiles) * num_p_tiles * num_pos;
-    const int grid = static_cast<int>(tiles < sms ? tiles : sms);
     int* status = nullptr;
     if (cudaGetSymbolAddress(reinterpret_cast<void**>(&status), g_status_word) != cudaSuccess) return SDWINO_ERR_CUDA;
-    ProfScope prof(KIND_GEMM, st);
-    kern<<<grid, GEMM_THREADS, L::DYN_BYTES, st>>>(tmU, tmV, tmM, num_k_tiles, num_p_tiles, num_pos, num_c_blocks,
-                                                   status);
-    g_launches.fetch_add(1);
-    return cudaGetLastError() == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
+    if (ctas == 2) return launch_gemm_shape<2>(tmU, tmV, tmM, prm, sms, status, st);
+    return launch_gemm_shape<1>(tmU, tmV, tmM, prm, sms, status, st);
 }
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
@@ -209,21 +264,36 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
     if (!ws || ws_bytes == 0) return SDWINO_ERR_WORKSPACE;
     if (!aligned(ws, WS_ALIGN)) return SDWINO_ERR_MISALIGNED;
     const long long pc = tiles_per_pass(pl, ws_bytes);
-    if (pc < GEMM_BLOCK_N) return SDWINO_ERR_WORKSPACE;
+    if (pc < GEMM_BLOCK_P) return SDWINO_ERR_WORKSPACE;
 
-    // workspace: V[a2][C][pc] then M[a2][Kp][pc]; both start on 1024-byte boundaries because pc is a
-    // multiple of 128 elements and the counts of rows are integers (pc * 2 bytes = multiple of 256).
+    // workspace: V[a2][C][pc] then M[a2][K][pc]; pc is a multiple of 128 elements, so every row starts
+    // on a 256-byte boundary.
     __half* V = static_cast<__half*>(ws);
     size_t v_bytes = static_cast<size_t>(pl.a2) * C * pc * sizeof(__half);
     v_bytes = (v_bytes + WS_ALIGN - 1) / WS_ALIGN * WS_ALIGN;
     __half* Mws = reinterpret_cast<__half*>(static_cast<uint8_t*>(ws) + v_bytes);
-    const size_t m_bytes = static_cast<size_t>(pl.a2) * pl.Kp * pc * sizeof(__half);
+    const size_t m_bytes = static_cast<size_t>(pl.a2) * K * pc * sizeof(__half);
     if (v_bytes + m_bytes > ws_bytes) return SDWINO_ERR_WORKSPACE;
 
+    const int sms = sm_count();
+    if (sms <= 0) return SDWINO_ERR_CUDA;
+    GemmParams prm;
+    GemmShape shape = choose_gemm_shape(K, C, pc / GEMM_BLOCK_P, pl.a2, sms);
+    if (g_force_ctas == 1 || g_force_ctas == 2) shape.ctas = (pc / GEMM_BLOCK_P < 2) ? 1 : g_force_ctas;
+    if (g_force_n_tile >= 16 && g_force_n_tile <= GEMM_MAX_N && g_force_n_tile % 16 == 0) shape.n_tile = g_force_n_tile;
+    prm.n_tile = shape.n_tile;
+    prm.num_k_tiles = (K + prm.n_tile - 1) / prm.n_tile;
+    prm.num_pos = pl.a2;
+    prm.num_c_blocks = (C + GEMM_BLOCK_C - 1) / GEMM_BLOCK_C;
+    prm.C = C;
+    const int b_rows = prm.n_tile / shape.ctas;
+    prm.stages = (MAX_DYN_SMEM - GemmSmemLayout::dyn_bytes(b_rows, 0)) / GemmSmemLayout::stage_bytes(b_rows);
+    if (prm.stages > GEMM_MAX_STAGES) prm.stages = GEMM_MAX_STAGES;
+
     CUtensorMap tmU, tmV, tmM;
-    if (!encode_map(&tmU, wT, pl.Cp, pl.Kp, pl.a2, pl.Cp, static_cast<uint64_t>(pl.Kp) * pl.Cp, 64, GEMM_BLOCK_M) ||
-        !encode_map(&tmV, V, pc, C, pl.a2, pc, static_cast<uint64_t>(C) * pc, 64, GEMM_BLOCK_K) ||
-        !encode_map(&tmM, Mws, pc, pl.Kp, pl.a2, pc, static_cast<uint64_t>(pl.Kp) * pc, 64, GEMM_BLOCK_M))
+    if (!encode_map(&tmU, wT, C, K, pl.a2, pl.C8, static_cast<uint64_t>(K) * pl.C8, 64, b_rows, true) ||
+        !encode_map(&tmV, V, pc, C, pl.a2, pc, static_cast<uint64_t>(C) * pc, 64, GEMM_BLOCK_C, true) ||
+        !encode_map(&tmM, Mws, pc, K, pl.a2, pc, static_cast<uint64_t>(K) * pc, 32, 16, false))
         return SDWINO_ERR_CUDA;
 
     TileGeom geo{H, W, pl.TH, pl.TW, pl.P};
@@ -237,10 +307,11 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
         if (tile == 2) rc = launch_input<2>(xh, V, geo, C, p0, count, pc, st);
         else rc = launch_input<4>(xh, V, geo, C, p0, count, pc, st);
         if (rc != SDWINO_OK) return rc;
-        rc = launch_gemm(tmU, tmV, tmM, pl.Kp / GEMM_BLOCK_M, count / GEMM_BLOCK_N, pl.a2, pl.Cp / GEMM_BLOCK_K, st);
+        prm.num_p_tiles = (count / GEMM_BLOCK_P + shape.ctas - 1) / shape.ctas;
+        rc = launch_gemm(tmU, tmV, tmM, prm, shape.ctas, st);
         if (rc != SDWINO_OK) return rc;
-        if (tile == 2) rc = launch_output<2>(Mws, bh, yh, geo, K, pl.Kp, p0, count, pc, st);
-        else rc = launch_output<4>(Mws, bh, yh, geo, K, pl.Kp, p0, count, pc, st);
+        if (tile == 2) rc = launch_output<2>(Mws, bh, yh, geo, K, p0, count, pc, st);
+        else rc = launch_output<4>(Mws, bh, yh, geo, K, p0, count, pc, st);
         if (rc != SDWINO_OK) return rc;
     }
     return SDWINO_OK;
@@ -251,6 +322,13 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
 extern "C" {
 
 int sdwino_version(void) { return 100; }
+
+int sdwino_set_gemm_shape(int ctas, int n_tile) {
+    if (ctas < 0 || ctas > 2 || n_tile < 0 || n_tile > GEMM_MAX_N || n_tile % 16 != 0) return SDWINO_ERR_INVALID_ARG;
+    g_force_ctas = ctas;
+    g_force_n_tile = n_tile;
+    return SDWINO_OK;
+}
 
 const char* sdwino_status_string(int status) {
     switch (status) {
@@ -268,7 +346,8 @@ const char* sdwino_status_string(int status) {
 size_t sdwino_filter_bytes(int K, int C, int tile) {
     if (K <= 0 || C <= 0 || (tile != 2 && tile != 4)) return 0;
     const size_t a = tile + 2;
-    return a * a * static_cast<size_t>(round_up(K, GEMM_BLOCK_M)) * round_up(C, GEMM_BLOCK_K) * sizeof(__half);
+    const size_t bytes = a * a * static_cast<size_t>(K) * round_up(C, 8) * sizeof(__half);
+    return (bytes + WS_ALIGN - 1) / WS_ALIGN * WS_ALIGN;
 }
 
 int sdwino_filter_transform(const void* w, void* wT, int K, int C, int tile, void* stream) {
@@ -276,10 +355,10 @@ int sdwino_filter_transform(const void* w, void* wT, int K, int C, int tile, voi
     if (tile != 2 && tile != 4) return SDWINO_ERR_UNSUPPORTED;
     if (!aligned(w, 2) || !aligned(wT, WS_ALIGN)) return SDWINO_ERR_MISALIGNED;
     if (static_cast<long double>(K) * C > 4.0e15L) return SDWINO_ERR_INVALID_ARG;
-    const int Kp = round_up(K, GEMM_BLOCK_M), Cp = round_up(C, GEMM_BLOCK_K);
+    const int C8 = round_up(C, 8);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (tile == 2) return launch_filter<2>(static_cast<const __half*>(w), static_cast<__half*>(wT), K, C, Kp, Cp, st);
-    return launch_filter<4>(static_cast<const __half*>(w), static_cast<__half*>(wT), K, C, Kp, Cp, st);
+    if (tile == 2) return launch_filter<2>(static_cast<const __half*>(w), static_cast<__half*>(wT), K, C, C8, st);
+    return launch_filter<4>(static_cast<const __half*>(w), static_cast<__half*>(wT), K, C, C8, st);
 }
 
 size_t sdwino_workspace_bytes(int N, int C, int H, int W, int K, int tile) {
@@ -292,7 +371,7 @@ size_t sdwino_workspace_bytes(int N, int C, int H, int W, int K, int tile) {
 size_t sdwino_workspace_min_bytes(int N, int C, int H, int W, int K, int tile) {
     Plan pl;
     if (!make_plan(N, C, H, W, K, tile, &pl)) return 0;
-    return static_cast<size_t>(GEMM_BLOCK_N) * pl.per_tile + WS_ALIGN;
+    return static_cast<size_t>(GEMM_BLOCK_P) * pl.per_tile + WS_ALIGN;
 }
 
 int sdwino_set_workspace(void* workspace, size_t bytes) {
@@ -368,8 +447,9 @@ int sdwino_last_device_status(void* stream) {
     if (v != 0) {
         int zero = 0;
         if (cudaMemcpyToSymbol(g_status_word, &zero, sizeof(int)) != cudaSuccess) return SDWINO_ERR_CUDA;
+        if (getenv("SDWINO_LOG")) fprintf(stderr, "sdwino: device status word 0x%x\n", v);
     }
-    return v;
+    return v & 0xFF;
 }
 
 unsigned long long sdwino_launch_count(void) { return g_launches.load(); }

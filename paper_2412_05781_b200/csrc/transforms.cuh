@@ -91,19 +91,20 @@ __device__ __forceinline__ void mat_apply(MatT coef, const float (&in)[Cn], floa
 }
 
 // ---------------------------------------------------------------------------------------
-// Filter preprocess.  One thread per (k, c) of the padded [Kp][Cp] plane; writes all a*a
-// positions (zeros in the padding).  U layout: [a*a][Kp][Cp], c contiguous.
+// Filter preprocess.  One thread per (k, c) of the [K][C8] plane (C8 = C rounded up to 8 so that
+// rows are 16-byte multiples); writes all a*a positions (zeros in the padding columns).
+// U layout: [a*a][K][C8], c contiguous.
 // ---------------------------------------------------------------------------------------
 template <int M>
-__global__ void __launch_bounds__(256)
-filter_transform_kernel(const __half* __restrict__ w, __half* __restrict__ U, int K, int C, int Kp, int Cp) {
+__global__ void __launch_bounds__(128)
+filter_transform_kernel(const __half* __restrict__ w, __half* __restrict__ U, int K, int C, int C8) {
     using Wm = Wino<M>;
     constexpr int A = Wm::A;
     const int c = blockIdx.x * blockDim.x + threadIdx.x;
     const int k = blockIdx.y;
-    if (c >= Cp) return;
+    if (c >= C8) return;
     float g[3][3];
-    const bool live = (k < K) && (c < C);
+    const bool live = c < C;
 #pragma unroll
     for (int r = 0; r < 3; ++r)
 #pragma unroll
@@ -119,8 +120,8 @@ filter_transform_kernel(const __half* __restrict__ w, __half* __restrict__ U, in
 #pragma unroll
         for (int i = 0; i < A; ++i) t[i][s] = o[i];
     }
-    const size_t plane = static_cast<size_t>(Kp) * Cp;
-    __half* dst = U + static_cast<size_t>(k) * Cp + c;
+    const size_t plane = static_cast<size_t>(K) * C8;
+    __half* dst = U + static_cast<size_t>(k) * C8 + c;
 #pragma unroll
     for (int i = 0; i < A; ++i) {
         float o[A];
@@ -199,11 +200,11 @@ input_transform_kernel(const __half* __restrict__ x, __half* __restrict__ V, Til
     }
 }
 
-// Postprocess + bias + cast + masked store.  Mws layout: [a*a][Kp][Pstride]; y is NCHW.
+// Postprocess + bias + cast + masked store.  Mws layout: [a*a][K][Pstride]; y is NCHW.
 template <int M>
 __global__ void __launch_bounds__(128)
 output_transform_kernel(const __half* __restrict__ Mws, const __half* __restrict__ bias, __half* __restrict__ y,
-                        TileGeom geo, int K, int Kp, long long p_begin, int p_count, long long Pstride) {
+                        TileGeom geo, int K, long long p_begin, int p_count, long long Pstride) {
     using Wm = Wino<M>;
     constexpr int A = Wm::A;
     const int pl = blockIdx.x * blockDim.x + threadIdx.x;
@@ -211,7 +212,7 @@ output_transform_kernel(const __half* __restrict__ Mws, const __half* __restrict
     if (pl >= p_count) return;
     const long long p = p_begin + pl;
     if (p >= geo.P) return;
-    const long long plane = static_cast<long long>(Kp) * Pstride;
+    const long long plane = static_cast<long long>(K) * Pstride;
     const __half* src = Mws + static_cast<long long>(k) * Pstride + pl;
     float mm[A][A];
 #pragma unroll

@@ -3,13 +3,25 @@
 // positions, the dense contraction  M[pos][k][p] = sum_c U[pos][k][c] * V[pos][c][p],
 // i.e. a batched GEMM.  It runs on the tcgen05 tensor cores: operands are brought into
 // shared memory by TMA (128-byte swizzle), accumulated in fp32 in tensor memory, and the
-// result is rounded once to fp16 and written back by a TMA store.
+// result is rounded once to fp16 and written back by TMA stores.
 //
-// One persistent CTA per SM walks the list of (pos, k-tile, p-tile) output tiles.
+// Orientation: the 128 TMEM lanes hold 128 consecutive tiles p (operand A = V, M-major), the
+// TMEM columns hold n_tile output channels k (operand B = U, K-major), n_tile any multiple of
+// 16 up to 256, so that channel counts such as 320 = 2 x 160 waste nothing.
+//
+// Two launch shapes share the code.  CTAS == 1: one persistent CTA per SM, 128 p x n_tile k per
+// tile.  CTAS == 2: persistent CTA pairs (a 2-CTA cluster) drive one 256-row MMA (cta_group::2);
+// each CTA loads its own 128 p rows of V but only half of the n_tile rows of U, which cuts the
+// bytes fetched from L2 per MMA cycle -- the measured limit of the single-CTA shape.  The leader
+// (even rank) issues the MMAs; completion is signalled to the barriers of both CTAs.
+//
+// One persistent CTA (pair) per SM (pair) walks the list of (pos, k-tile, p-tile) output tiles.
 //   warp 0   : TMA producer        (one lane)
 //   warp 1   : TMEM owner + MMA issuer (one lane)
 //   warps 2-5: epilogue, one TMEM lane quarter each; TMEM accumulators are double-buffered so
-//              the epilogue of tile i overlaps the MMAs of tile i+1.
+//              the epilogue of tile i overlaps the MMAs of tile i+1.  Each epilogue warp stages
+//              its own [16 k][32 p] fp16 blocks in a private ring and stores them by TMA, so the
+//              epilogue needs no CTA-wide barrier.
 #pragma once
 #include <cuda_fp16.h>
 
@@ -17,59 +29,84 @@
 
 namespace sdw {
 
-constexpr int GEMM_BLOCK_M = 128;  // output channels per tile (TMEM lanes)
-constexpr int GEMM_BLOCK_K = 64;   // input channels per pipeline stage (one 128-byte swizzle row of U)
+// first device-side failure wins: low byte = status code (6 = timeout), next byte = which wait gave up
+__device__ __forceinline__ void report_timeout(int* status_word, int where, uint32_t rank) {
+    atomicCAS(status_word, 0, 6 | ((where | (static_cast<int>(rank) << 4)) << 8));
+}
+
+constexpr int GEMM_BLOCK_P = 128;  // tiles per output tile (TMEM lanes, UMMA M)
+constexpr int GEMM_BLOCK_C = 64;   // input channels per pipeline stage (one 128-byte swizzle row of U)
+constexpr int GEMM_MAX_N = 256;    // output channels per output tile (UMMA N), multiple of 16
 constexpr int GEMM_THREADS = 192;
+constexpr int GEMM_MAX_STAGES = 8;
+constexpr int GEMM_EPI_RING = 8;   // staging slots per epilogue warp
 constexpr uint64_t GEMM_WAIT_LIMIT_NS = 2000000000ull;  // a wait longer than 2 s is reported, not spun on
 
-template <int BLOCK_N, int STAGES>
-struct GemmSmem {
-    static constexpr int A_BYTES = GEMM_BLOCK_M * GEMM_BLOCK_K * 2;
-    static constexpr int B_BOX_BYTES = 64 * GEMM_BLOCK_K * 2;  // one [64 p] x [64 c] box
-    static constexpr int B_BYTES = (BLOCK_N / 64) * B_BOX_BYTES;
-    static constexpr int C_BOX_BYTES = GEMM_BLOCK_M * 64 * 2;  // one [64 p] x [128 k] box
-    static constexpr int C_BYTES = (BLOCK_N / 64) * C_BOX_BYTES;
-    static constexpr int OFF_A = 0;
-    static constexpr int OFF_B = OFF_A + STAGES * A_BYTES;
-    static constexpr int OFF_C = OFF_B + STAGES * B_BYTES;
-    static constexpr int OFF_BAR = OFF_C + C_BYTES;
-    static constexpr int NUM_BARS = 2 * STAGES + 4;
-    static constexpr int OFF_MISC = OFF_BAR + NUM_BARS * 8;
-    static constexpr int TOTAL = OFF_MISC + 16;
-    static constexpr int DYN_BYTES = TOTAL + 1024;  // slack to align the base to 1024 bytes
+struct GemmSmemLayout {
+    static constexpr int A_BYTES = GEMM_BLOCK_P * GEMM_BLOCK_C * 2;          // two [64 p][64 c] boxes
+    static constexpr int A_BOX_BYTES = 64 * GEMM_BLOCK_C * 2;
+    static constexpr int EPI_SLOT_BYTES = 16 * 32 * 2;                       // [16 k][32 p] fp16
+    static constexpr int EPI_BYTES = 4 * GEMM_EPI_RING * EPI_SLOT_BYTES;
+    static constexpr int BAR_BYTES = (2 * GEMM_MAX_STAGES + 4) * 8 + 16;
+    // `rows` = rows of U this CTA loads per stage: n_tile (single CTA) or n_tile / 2 (CTA pair)
+    __host__ __device__ static constexpr int b_bytes(int rows) { return rows * GEMM_BLOCK_C * 2; }
+    __host__ __device__ static constexpr int stage_bytes(int rows) {
+        return (A_BYTES + b_bytes(rows) + 1023) / 1024 * 1024;
+    }
+    // dynamic shared memory for `stages` stages, including slack to align the base to 1024 bytes
+    __host__ __device__ static constexpr int dyn_bytes(int rows, int stages) {
+        return stages * stage_bytes(rows) + EPI_BYTES + BAR_BYTES + 1024;
+    }
 };
 
-// tmU: fp16 [pos][Kp][Cp]      box {64 c, 128 k, 1}, 128B swizzle  (A operand, K-major)
-// tmV: fp16 [pos][C][Pstride]  box {64 p,  64 c, 1}, 128B swizzle  (B operand, MN-major; rows c >= C read as 0)
-// tmM: fp16 [pos][Kp][Pstride] box {64 p, 128 k, 1}, 128B swizzle  (result)
-template <int BLOCK_N, int STAGES>
+struct GemmParams {
+    int num_k_tiles;   // ceil(K / n_tile)
+    int num_p_tiles;   // tiles of 128 p (single CTA) or 256 p (CTA pair) in this pass
+    int num_pos;       // a*a
+    int num_c_blocks;  // ceil(C / 64)
+    int C;             // input channels (for the k-steps of the last block)
+    int n_tile;        // UMMA N
+    int stages;
+};
+
+// tmV: fp16 [pos][C][Pstride]   box {64 p, 64 c, 1},      128B swizzle  (A operand; rows c >= C read as 0)
+// tmU: fp16 [pos][K][C8]        box {64 c, n_tile k, 1},  128B swizzle  (B operand; rows k >= K read as 0)
+// tmM: fp16 [pos][K][Pstride]   box {32 p, 16 k, 1},      no swizzle    (result; rows k >= K are clipped)
+template <int CTAS>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant__ CUtensorMap tmV,
-                 const __grid_constant__ CUtensorMap tmM, int num_k_tiles, int num_p_tiles, int num_pos,
-                 int num_c_blocks, int* __restrict__ status_word) {
-    using L = GemmSmem<BLOCK_N, STAGES>;
+                 const __grid_constant__ CUtensorMap tmM, const GemmParams prm, int* __restrict__ status_word) {
+    using L = GemmSmemLayout;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + L::OFF_BAR);
-    uint64_t* empty_bar = full_bar + STAGES;
-    uint64_t* acc_full_bar = empty_bar + STAGES;
+    const int b_rows = prm.n_tile / CTAS;            // rows of U this CTA loads per stage
+    const int stage_bytes = L::stage_bytes(b_rows);
+    const int stages = prm.stages;
+    const uint32_t cta_rank = CTAS == 2 ? cluster_ctarank() : 0u;
+    const bool leader = cta_rank == 0;
+    const int worker = blockIdx.x / CTAS;            // index of this CTA (pair) among the persistent workers
+    const int num_workers = gridDim.x / CTAS;
+    uint8_t* epi_base = smem + stages * stage_bytes;
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(epi_base + L::EPI_BYTES);
+    uint64_t* empty_bar = full_bar + GEMM_MAX_STAGES;
+    uint64_t* acc_full_bar = empty_bar + GEMM_MAX_STAGES;
     uint64_t* acc_empty_bar = acc_full_bar + 2;
-    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(smem + L::OFF_MISC);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::OFF_MISC + 4);
+    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(acc_empty_bar + 2);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_base_slot + 1);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const int num_tiles = num_k_tiles * num_p_tiles * num_pos;
-    constexpr uint32_t TMEM_COLS = 2 * BLOCK_N;
+    const int num_tiles = prm.num_k_tiles * prm.num_p_tiles * prm.num_pos;
+    constexpr uint32_t TMEM_COLS = 2 * GEMM_MAX_N;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) {
+        for (int s = 0; s < stages; ++s) {
             mbar_init(&full_bar[s], 1);
             mbar_init(&empty_bar[s], 1);
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(&acc_full_bar[b], 1);
-            mbar_init(&acc_empty_bar[b], 4);
+            mbar_init(&acc_empty_bar[b], 4 * CTAS);   // one arrival per epilogue warp of every CTA
         }
         *abort_flag = 0;
         fence_barrier_init();
@@ -78,135 +115,149 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
         prefetch_tmap(&tmM);
     }
     if (warp == 1) {
-        tmem_alloc(tmem_base_slot, TMEM_COLS);
-        tmem_relinquish();
+        if constexpr (CTAS == 2) { tmem_alloc_pair(tmem_base_slot, TMEM_COLS); tmem_relinquish_pair(); }
+        else { tmem_alloc(tmem_base_slot, TMEM_COLS); tmem_relinquish(); }
     }
     tc_fence_before_sync();
     __syncthreads();
+    if constexpr (CTAS == 2) cluster_sync_all();   // the peer's barriers are initialised before anyone signals them
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_base_slot;
 
     if (warp == 0) {
         // ------------------------------ TMA producer ------------------------------
         if (lane == 0) {
+            // the full barrier of a pair lives in the leader and counts the bytes of both CTAs
+            const uint32_t tx_bytes = CTAS * (L::A_BYTES + L::b_bytes(b_rows));
+            const uint32_t leader_full0 = CTAS == 2 ? map_to_cta(smem_u32(&full_bar[0]), 0) : 0u;
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-                const int pt = tile % num_p_tiles;
-                const int kt = (tile / num_p_tiles) % num_k_tiles;
-                const int pos = tile / (num_p_tiles * num_k_tiles);
-                for (int cb = 0; cb < num_c_blocks; ++cb) {
+            for (int tile = worker; tile < num_tiles && ok; tile += num_workers) {
+                const int pt = tile % prm.num_p_tiles;
+                const int kt = (tile / prm.num_p_tiles) % prm.num_k_tiles;
+                const int pos = tile / (prm.num_p_tiles * prm.num_k_tiles);
+                const int p0 = (pt * CTAS + static_cast<int>(cta_rank)) * GEMM_BLOCK_P;
+                const int k0 = kt * prm.n_tile + static_cast<int>(cta_rank) * b_rows;
+                for (int cb = 0; cb < prm.num_c_blocks; ++cb) {
                     ok = mbar_wait_bounded(&empty_bar[stage], phase ^ 1u, abort_flag, GEMM_WAIT_LIMIT_NS);
-                    if (!ok) break;
-                    mbar_arrive_expect_tx(&full_bar[stage], L::A_BYTES + L::B_BYTES);
-                    tma_load_3d(smem + L::OFF_A + stage * L::A_BYTES, &tmU, &full_bar[stage], cb * GEMM_BLOCK_K,
-                                kt * GEMM_BLOCK_M, pos);
-#pragma unroll
-                    for (int j = 0; j < BLOCK_N / 64; ++j)
-                        tma_load_3d(smem + L::OFF_B + stage * L::B_BYTES + j * L::B_BOX_BYTES, &tmV, &full_bar[stage],
-                                    pt * BLOCK_N + j * 64, cb * GEMM_BLOCK_K, pos);
-                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                    if (!ok) { if (*abort_flag == 0) report_timeout(status_word, 1, cta_rank); break; }
+                    uint8_t* sa = smem + stage * stage_bytes;
+                    if constexpr (CTAS == 2) {
+                        if (leader) mbar_arrive_expect_tx(&full_bar[stage], tx_bytes);
+                        const uint32_t fb = leader_full0 + static_cast<uint32_t>(stage) * 8u;
+                        tma_load_3d_pair(sa, &tmV, fb, p0, cb * GEMM_BLOCK_C, pos);
+                        tma_load_3d_pair(sa + L::A_BOX_BYTES, &tmV, fb, p0 + 64, cb * GEMM_BLOCK_C, pos);
+                        tma_load_3d_pair(sa + L::A_BYTES, &tmU, fb, cb * GEMM_BLOCK_C, k0, pos);
+                    } else {
+                        mbar_arrive_expect_tx(&full_bar[stage], tx_bytes);
+                        tma_load_3d(sa, &tmV, &full_bar[stage], p0, cb * GEMM_BLOCK_C, pos);
+                        tma_load_3d(sa + L::A_BOX_BYTES, &tmV, &full_bar[stage], p0 + 64, cb * GEMM_BLOCK_C, pos);
+                        tma_load_3d(sa + L::A_BYTES, &tmU, &full_bar[stage], cb * GEMM_BLOCK_C, k0, pos);
+                    }
+                    if (++stage == stages) { stage = 0; phase ^= 1u; }
                 }
             }
-            if (!ok) { *abort_flag = 1; atomicExch(status_word, 6); }
+            if (!ok) *abort_flag = 1;
         }
     } else if (warp == 1) {
         // ------------------------------ MMA issuer ------------------------------
-        if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc_f16_f32(GEMM_BLOCK_M, BLOCK_N, false, true);
+        if (lane == 0 && leader) {
+            const uint32_t idesc = make_idesc_f16_f32(GEMM_BLOCK_P * CTAS, prm.n_tile, true, false);
             int stage = 0;
             uint32_t phase = 0;
             int buf = 0;
             uint32_t acc_phase = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+            for (int tile = worker; tile < num_tiles && ok; tile += num_workers) {
                 ok = mbar_wait_bounded(&acc_empty_bar[buf], acc_phase ^ 1u, abort_flag, GEMM_WAIT_LIMIT_NS);
-                if (!ok) break;
+                if (!ok) { if (*abort_flag == 0) report_timeout(status_word, 2, cta_rank); break; }
                 tc_fence_after_sync();
-                const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(buf * BLOCK_N);
-                for (int cb = 0; cb < num_c_blocks; ++cb) {
+                const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(buf * GEMM_MAX_N);
+                for (int cb = 0; cb < prm.num_c_blocks; ++cb) {
                     ok = mbar_wait_bounded(&full_bar[stage], phase, abort_flag, GEMM_WAIT_LIMIT_NS);
-                    if (!ok) break;
+                    if (!ok) { if (*abort_flag == 0) report_timeout(status_word, 3, cta_rank); break; }
                     tc_fence_after_sync();
-                    const uint32_t a_addr = smem_u32(smem + L::OFF_A + stage * L::A_BYTES);
-                    const uint32_t b_addr = smem_u32(smem + L::OFF_B + stage * L::B_BYTES);
-#pragma unroll
-                    for (int s = 0; s < GEMM_BLOCK_K / 16; ++s) {
-                        // A (K-major): 16 channels = 32 bytes further along the swizzled 128-byte row.
-                        // B (MN-major): 16 channels = 16 rows of 128 bytes; 64-wide p blocks are B_BOX_BYTES apart.
-                        const uint64_t adesc = make_smem_desc_sw128(a_addr + s * 32, 16, 1024);
-                        const uint64_t bdesc = make_smem_desc_sw128(b_addr + s * 2048, L::B_BOX_BYTES, 1024);
-                        umma_f16(d_tmem, adesc, bdesc, idesc, (cb > 0 || s > 0) ? 1u : 0u);
+                    const uint32_t a_addr = smem_u32(smem + stage * stage_bytes);
+                    const uint32_t b_addr = a_addr + L::A_BYTES;
+                    const int c_left = prm.C - cb * GEMM_BLOCK_C;
+                    const int ksteps = c_left >= GEMM_BLOCK_C ? GEMM_BLOCK_C / 16 : (c_left + 15) / 16;
+                    for (int s = 0; s < ksteps; ++s) {
+                        // A (M-major): 16 channels = 16 rows of 128 bytes; the two 64-wide p blocks are
+                        // A_BOX_BYTES apart.  B (K-major): 16 channels = 32 bytes along the swizzled row.
+                        const uint64_t adesc = make_smem_desc_sw128(a_addr + s * 2048, L::A_BOX_BYTES, 1024);
+                        const uint64_t bdesc = make_smem_desc_sw128(b_addr + s * 32, 16, 1024);
+                        if constexpr (CTAS == 2) umma_f16_pair(d_tmem, adesc, bdesc, idesc, (cb > 0 || s > 0) ? 1u : 0u);
+                        else umma_f16(d_tmem, adesc, bdesc, idesc, (cb > 0 || s > 0) ? 1u : 0u);
                     }
-                    umma_commit(&empty_bar[stage]);
-                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                    if constexpr (CTAS == 2) umma_commit_pair(&empty_bar[stage]);
+                    else umma_commit(&empty_bar[stage]);
+                    if (++stage == stages) { stage = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
-                umma_commit(&acc_full_bar[buf]);
+                if constexpr (CTAS == 2) umma_commit_pair(&acc_full_bar[buf]);
+                else umma_commit(&acc_full_bar[buf]);
                 buf ^= 1;
                 if (buf == 0) acc_phase ^= 1u;
             }
-            if (!ok) { *abort_flag = 1; atomicExch(status_word, 6); }
+            if (!ok) *abort_flag = 1;
         }
     } else {
         // ------------------------------ epilogue ------------------------------
-        const int quarter = warp & 3;               // TMEM lanes this warp may read: 32*quarter ..
-        const int row = quarter * 32 + lane;        // output channel within the tile
-        const int epi_tid = threadIdx.x - 64;
-        uint8_t* stage_c = smem + L::OFF_C;
+        const int quarter = warp & 3;          // TMEM lanes this warp may read: 32*quarter .. +31
+        uint8_t* ring = epi_base + quarter * (GEMM_EPI_RING * L::EPI_SLOT_BYTES);
+        int slot = 0;
         int buf = 0;
         uint32_t acc_phase = 0;
-        for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
-            const int pt = tile % num_p_tiles;
-            const int kt = (tile / num_p_tiles) % num_k_tiles;
-            const int pos = tile / (num_p_tiles * num_k_tiles);
+        // the accumulator-empty barrier of a pair lives in the leader
+        const uint32_t acc_empty_addr0 = CTAS == 2 ? map_to_cta(smem_u32(&acc_empty_bar[0]), 0) : 0u;
+        for (int tile = worker; tile < num_tiles; tile += num_workers) {
+            const int pt = tile % prm.num_p_tiles;
+            const int kt = (tile / prm.num_p_tiles) % prm.num_k_tiles;
+            const int pos = tile / (prm.num_p_tiles * prm.num_k_tiles);
             bool ok = mbar_wait_bounded(&acc_full_bar[buf], acc_phase, abort_flag, GEMM_WAIT_LIMIT_NS);
-            if (!ok) { *abort_flag = 1; atomicExch(status_word, 6); }
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            if (*abort_flag != 0) break;
-            tc_fence_after_sync();
-#pragma unroll 1
-            for (int chunk = 0; chunk < BLOCK_N / 32; ++chunk) {
-                uint32_t r[32];
-                tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
-                                  static_cast<uint32_t>(buf * BLOCK_N + chunk * 32), r);
-                tmem_ld_wait();
-                uint8_t* box = stage_c + (chunk >> 1) * L::C_BOX_BYTES + row * 128;
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    uint4 v;
-                    __half2 h;
-                    h = __floats2half2_rn(__uint_as_float(r[8 * i + 0]), __uint_as_float(r[8 * i + 1]));
-                    v.x = *reinterpret_cast<uint32_t*>(&h);
-                    h = __floats2half2_rn(__uint_as_float(r[8 * i + 2]), __uint_as_float(r[8 * i + 3]));
-                    v.y = *reinterpret_cast<uint32_t*>(&h);
-                    h = __floats2half2_rn(__uint_as_float(r[8 * i + 4]), __uint_as_float(r[8 * i + 5]));
-                    v.z = *reinterpret_cast<uint32_t*>(&h);
-                    h = __floats2half2_rn(__uint_as_float(r[8 * i + 6]), __uint_as_float(r[8 * i + 7]));
-                    v.w = *reinterpret_cast<uint32_t*>(&h);
-                    const int c16 = ((chunk & 1) * 4 + i) ^ (row & 7);  // 128-byte swizzle of the 16-byte chunk
-                    *reinterpret_cast<uint4*>(box + c16 * 16) = v;
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) {
+                if (lane == 0) {
+                    if (*abort_flag == 0) report_timeout(status_word, 4, cta_rank);
+                    *abort_flag = 1;
                 }
+                break;
+            }
+            tc_fence_after_sync();
+            const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
+                                    static_cast<uint32_t>(buf * GEMM_MAX_N);
+            const int p0 = (pt * CTAS + static_cast<int>(cta_rank)) * GEMM_BLOCK_P + quarter * 32;
+            const int k0 = kt * prm.n_tile;
+            for (int col = 0; col < prm.n_tile; col += 16) {
+                uint32_t r[16];
+                tmem_ld_32x16_sync(t_addr + col, r);
+                // the slot about to be overwritten must have been read by its TMA store
+                if (lane == 0) tma_store_wait_read_pending<GEMM_EPI_RING - 1>();
+                __syncwarp();
+                uint8_t* sl = ring + slot * L::EPI_SLOT_BYTES;   // [16 k][32 p] fp16, lane = p
+#pragma unroll
+                for (int i = 0; i < 16; ++i)
+                    *reinterpret_cast<__half*>(sl + i * 64 + lane * 2) = __float2half_rn(__uint_as_float(r[i]));
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    tma_store_3d(&tmM, sl, p0, k0 + col, pos);
+                    tma_store_commit();
+                }
+                if (++slot == GEMM_EPI_RING) slot = 0;
             }
             // accumulator drained: hand the TMEM buffer back to the MMA warp
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&acc_empty_bar[buf]);
-            fence_proxy_async_smem();
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            if (epi_tid == 0) {
-#pragma unroll
-                for (int j = 0; j < BLOCK_N / 64; ++j)
-                    tma_store_3d(&tmM, stage_c + j * L::C_BOX_BYTES, pt * BLOCK_N + j * 64, kt * GEMM_BLOCK_M, pos);
-                tma_store_commit();
-                tma_store_wait_read();
+            if (lane == 0) {
+                if constexpr (CTAS == 2) mbar_arrive_cluster(acc_empty_addr0 + static_cast<uint32_t>(buf) * 8u);
+                else mbar_arrive(&acc_empty_bar[buf]);
             }
-            asm volatile("bar.sync 1, 128;" ::: "memory");
             buf ^= 1;
             if (buf == 0) acc_phase ^= 1u;
         }
-        if (epi_tid == 0) tma_store_wait_all();
+        if (lane == 0) tma_store_wait_all();
     }
 
     __syncwarp();
@@ -218,9 +269,11 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
         while (global_timer_ns() - t0 < 200000ull) __nanosleep(1000);
         __syncthreads();
     }
+    if constexpr (CTAS == 2) cluster_sync_all();   // no CTA leaves while its peer may still signal it
     if (warp == 1) {
         tc_fence_after_sync();
-        tmem_dealloc(tmem_base, TMEM_COLS);
+        if constexpr (CTAS == 2) tmem_dealloc_pair(tmem_base, TMEM_COLS);
+        else tmem_dealloc(tmem_base, TMEM_COLS);
     }
 }
 

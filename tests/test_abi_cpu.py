@@ -39,16 +39,16 @@ def test_version_and_status_strings(binding):
 
 
 def test_size_queries(binding):
-    # wT = a*a planes of [K rounded to 128][C rounded to 64] fp16
-    assert binding.sdwino_filter_bytes(320, 320, 2) == 16 * 384 * 320 * 2
-    assert binding.sdwino_filter_bytes(3, 4, 4) == 36 * 128 * 64 * 2
+    # wT = a*a planes of [K][C rounded to 8] fp16, the total rounded up to 1024 bytes
+    assert binding.sdwino_filter_bytes(320, 320, 2) == 16 * 320 * 320 * 2
+    assert binding.sdwino_filter_bytes(3, 4, 4) == 2048        # 36 * 3 * 8 * 2 = 1728 -> 2048
     assert binding.sdwino_filter_bytes(0, 4, 2) == 0
     assert binding.sdwino_filter_bytes(4, 4, 3) == 0
     full = binding.sdwino_workspace_bytes(2, 320, 64, 64, 320, 2)
     small = binding.sdwino_workspace_min_bytes(2, 320, 64, 64, 320, 2)
-    # P = 2*32*32 = 2048 tiles, (C + Kp) = 704 fp16 per position and tile
-    assert full == 2048 * 16 * 704 * 2 + 1024
-    assert small == 128 * 16 * 704 * 2 + 1024
+    # P = 2*32*32 = 2048 tiles, (C + K) = 640 fp16 per position and tile
+    assert full == 2048 * 16 * 640 * 2 + 1024
+    assert small == 128 * 16 * 640 * 2 + 1024
     assert binding.sdwino_workspace_bytes(1, 1, 1, 1, 1, 5) == 0
     assert binding.sdwino_workspace_bytes(1, 0, 1, 1, 1, 2) == 0
     assert binding.sdwino_host_staging_bytes(1, 4, 8, 8, 4, 2) == 1024 * 3

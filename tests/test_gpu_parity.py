@@ -82,6 +82,30 @@ def test_small_shapes_elementwise(B, shape, tile):
     assert _rel_err(y, wino) <= TOL
 
 
+@pytest.mark.parametrize("ctas,n_tile", [(1, 16), (1, 32), (1, 48), (1, 160), (1, 256), (2, 16), (2, 32), (2, 80),
+                                          (2, 160), (2, 256)])
+def test_forced_gemm_shapes(B, ctas, n_tile):
+    # every GEMM launch shape (single CTA / CTA pair, channels per tile) must give the same convolution;
+    # 1150 tiles = 9 blocks of 128 (an odd count, so the last CTA pair is half empty), K = 200 is ragged
+    # for every n_tile, C = 72 leaves a partial channel block
+    layer = ConvLayer(C=72, K=200, H=50, W=46, N=2)
+    x, w, b = workloads.make_inputs(layer, seed=21)
+    ref = oracle.direct_conv3x3(x.numpy(), w.numpy(), b.numpy())
+    B.sdwino_set_gemm_shape(ctas, n_tile)
+    try:
+        _, _, _, y = _run(B, layer, 2, x=x, w=w, b=b)
+    finally:
+        B.sdwino_set_gemm_shape(0, 0)
+    assert _rel_err(y, ref) <= TOL_F2_REGRESSION
+
+
+def test_set_gemm_shape_rejects_bad_values(B):
+    for ctas, n in [(3, 0), (-1, 0), (0, 8), (0, 272), (1, 100)]:
+        with pytest.raises(B.SdwinoError):
+            B.sdwino_set_gemm_shape(ctas, n)
+    B.sdwino_set_gemm_shape(0, 0)
+
+
 @pytest.mark.parametrize("tile", [2, 4])
 def test_no_bias_and_zero_input(B, tile):
     layer = ConvLayer(C=20, K=24, H=11, W=10, N=2)
@@ -121,8 +145,8 @@ def test_filter_transform_matches_oracle(B, KC, tile):
     g = torch.Generator().manual_seed(K + C)
     w = (torch.randn(K, C, 3, 3, generator=g) / (9 * C) ** 0.5).half()
     wT = B.sdwino_filter_transform(w.cuda(), tile)
-    Kp, Cp = -(-K // 128) * 128, -(-C // 64) * 64
-    U = wT.view(torch.float16).view(a * a, Kp, Cp).cpu()
+    C8 = -(-C // 8) * 8
+    U = wT.view(torch.float16)[:a * a * K * C8].view(a * a, K, C8).cpu()
     Uo = oracle.filter_transform(w.numpy(), tile, points=None if tile == 2 else F4_POINTS)
     Uo = torch.from_numpy(Uo.reshape(K, C, a * a).transpose(2, 0, 1).copy())
     got = U[:, :K, :C].double()
@@ -131,9 +155,8 @@ def test_filter_transform_matches_oracle(B, KC, tile):
     ulp = torch.maximum((torch.nextafter(ref16, torch.full_like(ref16, float("inf"))) - ref16).double().abs(),
                         (ref16 - torch.nextafter(ref16, torch.full_like(ref16, -float("inf")))).double().abs())
     assert bool(((got - ref16.double()).abs() <= ulp).all())
-    # padding rows / columns are zero
-    assert float(U[:, K:, :].abs().max() if Kp > K else 0) == 0
-    assert float(U[:, :, C:].abs().max() if Cp > C else 0) == 0
+    # padding columns are zero
+    assert float(U[:, :, C:].abs().max() if C8 > C else 0) == 0
 
 
 def test_single_layer_config_full(B):
