@@ -45,20 +45,22 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 
-// Wait for the phase with the given parity to complete.  Gives up after `limit_ns`
-// (checked every 256 polls) or as soon as *abort_flag becomes non-zero; returns false then.
+// Wait for the phase with the given parity to complete.  Gives up after `limit_ns` or as soon as
+// *abort_flag becomes non-zero; returns false then.  The hot path is a bare try_wait loop: the
+// global timer is slow to read, so it (and the abort flag) are only consulted every 4096 failed polls.
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
                                                   uint64_t limit_ns) {
-    if (mbar_try_wait(bar, parity)) return true;
-    uint64_t t0 = global_timer_ns();
     uint32_t polls = 0;
-    while (true) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((++polls & 255u) == 0u) {
+    uint64_t t0 = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++polls & 4095u) == 0u) {
             if (*abort_flag != 0) return false;
-            if (global_timer_ns() - t0 > limit_ns) return false;
+            const uint64_t now = global_timer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > limit_ns) return false;
         }
     }
+    return true;
 }
 
 // ---- TMA --------------------------------------------------------------------

@@ -224,7 +224,7 @@ int launch_gemm_shape(const CUtensorMap& tmU, const CUtensorMap& tmV, const CUte
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(GEMM_THREADS);
-    cfg.dynamicSmemBytes = L::dyn_bytes(prm.n_tile / CTAS, prm.stages);
+    cfg.dynamicSmemBytes = L::dyn_bytes(prm.n_tile / CTAS, prm.stages, prm.epi_rows, prm.epi_bufs);
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -287,13 +287,22 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
     prm.num_c_blocks = (C + GEMM_BLOCK_C - 1) / GEMM_BLOCK_C;
     prm.C = C;
     const int b_rows = prm.n_tile / shape.ctas;
-    prm.stages = (MAX_DYN_SMEM - GemmSmemLayout::dyn_bytes(b_rows, 0)) / GemmSmemLayout::stage_bytes(b_rows);
+    // epilogue staging: half a tile per TMA store when that is a multiple of 16 channels, two buffers when at
+    // least four pipeline stages still fit beside them
+    prm.epi_rows = (prm.n_tile > 64 && (prm.n_tile / 2) % 16 == 0) ? prm.n_tile / 2 : prm.n_tile;
+    prm.epi_bufs = 2;
+    prm.stages = (MAX_DYN_SMEM - GemmSmemLayout::dyn_bytes(b_rows, 0, prm.epi_rows, 2)) / GemmSmemLayout::stage_bytes(b_rows);
+    if (prm.stages < 4) {
+        prm.epi_bufs = 1;
+        prm.stages = (MAX_DYN_SMEM - GemmSmemLayout::dyn_bytes(b_rows, 0, prm.epi_rows, 1)) / GemmSmemLayout::stage_bytes(b_rows);
+    }
     if (prm.stages > GEMM_MAX_STAGES) prm.stages = GEMM_MAX_STAGES;
 
+    prm.p_stride = pc;
     CUtensorMap tmU, tmV, tmM;
     if (!encode_map(&tmU, wT, C, K, pl.a2, pl.C8, static_cast<uint64_t>(K) * pl.C8, 64, b_rows, true) ||
         !encode_map(&tmV, V, pc, C, pl.a2, pc, static_cast<uint64_t>(C) * pc, 64, GEMM_BLOCK_C, true) ||
-        !encode_map(&tmM, Mws, pc, K, pl.a2, pc, static_cast<uint64_t>(K) * pc, 32, 16, false))
+        !encode_map(&tmM, Mws, pc, K, pl.a2, pc, static_cast<uint64_t>(K) * pc, GEMM_BLOCK_P, prm.epi_rows, false))
         return SDWINO_ERR_CUDA;
 
     TileGeom geo{H, W, pl.TH, pl.TW, pl.P};

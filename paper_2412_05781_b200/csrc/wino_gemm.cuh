@@ -19,9 +19,10 @@
 //   warp 0   : TMA producer        (one lane)
 //   warp 1   : TMEM owner + MMA issuer (one lane)
 //   warps 2-5: epilogue, one TMEM lane quarter each; TMEM accumulators are double-buffered so
-//              the epilogue of tile i overlaps the MMAs of tile i+1.  Each epilogue warp stages
-//              its own [16 k][32 p] fp16 blocks in a private ring and stores them by TMA, so the
-//              epilogue needs no CTA-wide barrier.
+//              the epilogue of tile i overlaps the MMAs of tile i+1.  A thread owns one tile p and
+//              reads its channels from TMEM; the fp16 results are transposed through a shared-memory
+//              staging buffer [k][128 p] and leave with one TMA store per epi_rows channels, so M is
+//              written in full 256-byte rows.
 #pragma once
 #include <cuda_fp16.h>
 
@@ -39,23 +40,25 @@ constexpr int GEMM_BLOCK_C = 64;   // input channels per pipeline stage (one 128
 constexpr int GEMM_MAX_N = 256;    // output channels per output tile (UMMA N), multiple of 16
 constexpr int GEMM_THREADS = 192;
 constexpr int GEMM_MAX_STAGES = 8;
-constexpr int GEMM_EPI_RING = 8;   // staging slots per epilogue warp
 constexpr uint64_t GEMM_WAIT_LIMIT_NS = 2000000000ull;  // a wait longer than 2 s is reported, not spun on
 
 struct GemmSmemLayout {
     static constexpr int A_BYTES = GEMM_BLOCK_P * GEMM_BLOCK_C * 2;          // two [64 p][64 c] boxes
     static constexpr int A_BOX_BYTES = 64 * GEMM_BLOCK_C * 2;
-    static constexpr int EPI_SLOT_BYTES = 16 * 32 * 2;                       // [16 k][32 p] fp16
-    static constexpr int EPI_BYTES = 4 * GEMM_EPI_RING * EPI_SLOT_BYTES;
+    static constexpr int EPI_ROW_BYTES = GEMM_BLOCK_P * 2;                   // one staged row: 128 p fp16
     static constexpr int BAR_BYTES = (2 * GEMM_MAX_STAGES + 4) * 8 + 16;
     // `rows` = rows of U this CTA loads per stage: n_tile (single CTA) or n_tile / 2 (CTA pair)
     __host__ __device__ static constexpr int b_bytes(int rows) { return rows * GEMM_BLOCK_C * 2; }
     __host__ __device__ static constexpr int stage_bytes(int rows) {
         return (A_BYTES + b_bytes(rows) + 1023) / 1024 * 1024;
     }
+    // epilogue staging: `bufs` buffers of [epi_rows k][128 p] fp16
+    __host__ __device__ static constexpr int epi_bytes(int epi_rows, int bufs) {
+        return bufs * epi_rows * EPI_ROW_BYTES;
+    }
     // dynamic shared memory for `stages` stages, including slack to align the base to 1024 bytes
-    __host__ __device__ static constexpr int dyn_bytes(int rows, int stages) {
-        return stages * stage_bytes(rows) + EPI_BYTES + BAR_BYTES + 1024;
+    __host__ __device__ static constexpr int dyn_bytes(int rows, int stages, int epi_rows, int bufs) {
+        return stages * stage_bytes(rows) + epi_bytes(epi_rows, bufs) + BAR_BYTES + 1024;
     }
 };
 
@@ -67,11 +70,14 @@ struct GemmParams {
     int C;             // input channels (for the k-steps of the last block)
     int n_tile;        // UMMA N
     int stages;
+    int epi_rows;      // channels staged per TMA store: divides n_tile, multiple of 16
+    int epi_bufs;      // staging buffers (1 or 2)
+    long long p_stride;  // tiles per pass (row pitch of V and M)
 };
 
 // tmV: fp16 [pos][C][Pstride]   box {64 p, 64 c, 1},      128B swizzle  (A operand; rows c >= C read as 0)
 // tmU: fp16 [pos][K][C8]        box {64 c, n_tile k, 1},  128B swizzle  (B operand; rows k >= K read as 0)
-// tmM: fp16 [pos][K][Pstride]   box {32 p, 16 k, 1},      no swizzle    (result; rows k >= K are clipped)
+// tmM: fp16 [pos][K][Pstride]   box {128 p, epi_rows k, 1}, no swizzle  (result; rows k >= K are clipped)
 template <int CTAS>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant__ CUtensorMap tmV,
@@ -87,7 +93,7 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
     const int worker = blockIdx.x / CTAS;            // index of this CTA (pair) among the persistent workers
     const int num_workers = gridDim.x / CTAS;
     uint8_t* epi_base = smem + stages * stage_bytes;
-    uint64_t* full_bar = reinterpret_cast<uint64_t*>(epi_base + L::EPI_BYTES);
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(epi_base + L::epi_bytes(prm.epi_rows, prm.epi_bufs));
     uint64_t* empty_bar = full_bar + GEMM_MAX_STAGES;
     uint64_t* acc_full_bar = empty_bar + GEMM_MAX_STAGES;
     uint64_t* acc_empty_bar = acc_full_bar + 2;
@@ -205,9 +211,8 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
     } else {
         // ------------------------------ epilogue ------------------------------
         const int quarter = warp & 3;          // TMEM lanes this warp may read: 32*quarter .. +31
-        uint8_t* ring = epi_base + quarter * (GEMM_EPI_RING * L::EPI_SLOT_BYTES);
-        int slot = 0;
         int buf = 0;
+        int sbuf = 0;
         uint32_t acc_phase = 0;
         // the accumulator-empty barrier of a pair lives in the leader
         const uint32_t acc_empty_addr0 = CTAS == 2 ? map_to_cta(smem_u32(&acc_empty_bar[0]), 0) : 0u;
@@ -229,23 +234,33 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
                                     static_cast<uint32_t>(buf * GEMM_MAX_N);
             const int p0 = (pt * CTAS + static_cast<int>(cta_rank)) * GEMM_BLOCK_P + quarter * 32;
             const int k0 = kt * prm.n_tile;
-            for (int col = 0; col < prm.n_tile; col += 16) {
-                uint32_t r[16];
-                tmem_ld_32x16_sync(t_addr + col, r);
-                // the slot about to be overwritten must have been read by its TMA store
-                if (lane == 0) tma_store_wait_read_pending<GEMM_EPI_RING - 1>();
-                __syncwarp();
-                uint8_t* sl = ring + slot * L::EPI_SLOT_BYTES;   // [16 k][32 p] fp16, lane = p
+            const bool p_ok = p0 < prm.p_stride;   // the second CTA of the last pair may hang over the pass
+            const int epi_tid = threadIdx.x - 64;
+            // lane = tile p, registers = output channels: staging row k receives 32 consecutive p from
+            // each warp (64 contiguous bytes, no bank conflict)
+            for (int row0 = 0; row0 < prm.n_tile; row0 += prm.epi_rows) {
+                uint8_t* stg = epi_base + sbuf * prm.epi_rows * L::EPI_ROW_BYTES;
+                // the buffer about to be overwritten must have been read by its TMA store
+                if (epi_tid == 0) {
+                    if (prm.epi_bufs == 2) tma_store_wait_read_pending<1>();
+                    else tma_store_wait_read_pending<0>();
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                __half* dst = reinterpret_cast<__half*>(stg) + quarter * 32 + lane;
+                for (int col = 0; col < prm.epi_rows; col += 16) {
+                    uint32_t r[16];
+                    tmem_ld_32x16_sync(t_addr + row0 + col, r);
 #pragma unroll
-                for (int i = 0; i < 16; ++i)
-                    *reinterpret_cast<__half*>(sl + i * 64 + lane * 2) = __float2half_rn(__uint_as_float(r[i]));
+                    for (int i = 0; i < 16; ++i)
+                        dst[(col + i) * GEMM_BLOCK_P] = __float2half_rn(__uint_as_float(r[i]));
+                }
                 fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) {
-                    tma_store_3d(&tmM, sl, p0, k0 + col, pos);
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (epi_tid == 0) {
+                    if (p_ok) tma_store_3d(&tmM, stg, p0 - quarter * 32, k0 + row0, pos);
                     tma_store_commit();
                 }
-                if (++slot == GEMM_EPI_RING) slot = 0;
+                if (prm.epi_bufs == 2) sbuf ^= 1;
             }
             // accumulator drained: hand the TMEM buffer back to the MMA warp
             tc_fence_before_sync();
@@ -257,7 +272,7 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
             buf ^= 1;
             if (buf == 0) acc_phase ^= 1u;
         }
-        if (lane == 0) tma_store_wait_all();
+        if (threadIdx.x == 64) tma_store_wait_all();
     }
 
     __syncwarp();
