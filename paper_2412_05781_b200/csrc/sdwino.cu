@@ -137,6 +137,8 @@ bool encode_map(CUtensorMap* m, const void* base, uint64_t d0, uint64_t d1, uint
     return r == CUDA_SUCCESS;
 }
 
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
 int sm_count() {
     static int n = 0;
     if (n == 0) {
@@ -159,9 +161,15 @@ int launch_filter(const __half* w, __half* U, int K, int C, int C8, cudaStream_t
 template <int M>
 int launch_input(const __half* x, __half* V, const TileGeom& geo, int C, long long p_begin, int p_count,
                  long long Pstride, cudaStream_t st) {
-    dim3 grid((p_count + 127) / 128, C);
     ProfScope prof(KIND_INPUT, st);
-    input_transform_kernel<M><<<grid, 128, 0, st>>>(x, V, geo, C, p_begin, p_count, Pstride);
+    constexpr int TPT = 8 / M;
+    if (geo.W % 8 == 0 && aligned(x, 16)) {
+        dim3 grid((p_count / TPT + 127) / 128, C);
+        input_transform_vec_kernel<M, TPT><<<grid, 128, 0, st>>>(x, V, geo, C, p_begin, p_count, Pstride);
+    } else {
+        dim3 grid((p_count + 127) / 128, C);
+        input_transform_kernel<M><<<grid, 128, 0, st>>>(x, V, geo, C, p_begin, p_count, Pstride);
+    }
     g_launches.fetch_add(1);
     return cudaGetLastError() == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
 }
@@ -169,9 +177,15 @@ int launch_input(const __half* x, __half* V, const TileGeom& geo, int C, long lo
 template <int M>
 int launch_output(const __half* Mws, const __half* bias, __half* y, const TileGeom& geo, int K,
                   long long p_begin, int p_count, long long Pstride, cudaStream_t st) {
-    dim3 grid((p_count + 127) / 128, K);
     ProfScope prof(KIND_OUTPUT, st);
-    output_transform_kernel<M><<<grid, 128, 0, st>>>(Mws, bias, y, geo, K, p_begin, p_count, Pstride);
+    constexpr int TPT = 8 / M;
+    if (geo.W % 8 == 0 && aligned(y, 16)) {
+        dim3 grid((p_count / TPT + 127) / 128, K);
+        output_transform_vec_kernel<M, TPT><<<grid, 128, 0, st>>>(Mws, bias, y, geo, K, p_begin, p_count, Pstride);
+    } else {
+        dim3 grid((p_count + 127) / 128, K);
+        output_transform_kernel<M><<<grid, 128, 0, st>>>(Mws, bias, y, geo, K, p_begin, p_count, Pstride);
+    }
     g_launches.fetch_add(1);
     return cudaGetLastError() == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
 }
@@ -249,7 +263,6 @@ int launch_gemm(const CUtensorMap& tmU, const CUtensorMap& tmV, const CUtensorMa
     return launch_gemm_shape<1>(tmU, tmV, tmM, prm, sms, status, st);
 }
 
-bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
 int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, int C, int H, int W, int K, int tile,
               void* ws, size_t ws_bytes, cudaStream_t st) {

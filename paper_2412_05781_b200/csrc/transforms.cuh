@@ -257,4 +257,177 @@ output_transform_kernel(const __half* __restrict__ Mws, const __half* __restrict
     }
 }
 
+
+// ---------------------------------------------------------------------------------------
+// Vector variants for image widths that are multiples of 8 (every SD layer of 16 pixels or more):
+// a thread owns TPT consecutive tiles of one tile row (m * TPT = 8 pixels), so each input or
+// output row segment is one aligned 16-byte access, the halo pixels left and right of it are two
+// scalar loads, and each transform position is stored / loaded as TPT packed fp16 values.
+// Arithmetic is fp32 as in the scalar kernels (the row and column passes run in the other order).
+// Requirements (checked by the host): W % 8 == 0, x / y 16-byte aligned, m * TPT == 8.
+// ---------------------------------------------------------------------------------------
+template <int N> struct PackedHalf;
+template <> struct PackedHalf<2> { using type = uint32_t; };
+template <> struct PackedHalf<4> { using type = uint2; };
+
+__device__ __forceinline__ uint32_t pack2(float a, float b) {
+    __half2 h = __floats2half2_rn(a, b);
+    return *reinterpret_cast<uint32_t*>(&h);
+}
+__device__ __forceinline__ void unpack2(uint32_t v, float& a, float& b) {
+    const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&v));
+    a = f.x;
+    b = f.y;
+}
+
+template <int M, int TPT>
+__global__ void __launch_bounds__(128)
+input_transform_vec_kernel(const __half* __restrict__ x, __half* __restrict__ V, TileGeom geo, int C,
+                           long long p_begin, int p_count, long long Pstride) {
+    using Wm = Wino<M>;
+    constexpr int A = Wm::A;
+    static_assert(M * TPT == 8, "one 16-byte row segment per thread");
+    const int pl = (blockIdx.x * blockDim.x + threadIdx.x) * TPT;  // first chunk-local tile of this thread
+    const int c = blockIdx.y;
+    if (pl >= p_count) return;
+    const long long p = p_begin + pl;
+    float e[A][TPT][A];  // rows transformed along the columns: e[r][t][nu] = sum_s Bt[nu][s] d[r][s]
+    if (p < geo.P) {
+        const int tw = static_cast<int>(p % geo.TW);
+        const int th = static_cast<int>((p / geo.TW) % geo.TH);
+        const long long n = p / (static_cast<long long>(geo.TW) * geo.TH);
+        const __half* img = x + (n * C + c) * static_cast<long long>(geo.H) * geo.W;
+        const int i0 = M * th - 1, j0 = M * tw;
+#pragma unroll
+        for (int r = 0; r < A; ++r) {
+            const int i = i0 + r;
+            float row[10];
+            if (i >= 0 && i < geo.H) {
+                const __half* rp = img + static_cast<long long>(i) * geo.W + j0;
+                const uint4 v = __ldg(reinterpret_cast<const uint4*>(rp));
+                unpack2(v.x, row[1], row[2]);
+                unpack2(v.y, row[3], row[4]);
+                unpack2(v.z, row[5], row[6]);
+                unpack2(v.w, row[7], row[8]);
+                row[0] = j0 > 0 ? __half2float(__ldg(rp - 1)) : 0.f;
+                row[9] = j0 + 8 < geo.W ? __half2float(__ldg(rp + 8)) : 0.f;
+            } else {
+#pragma unroll
+                for (int s = 0; s < 10; ++s) row[s] = 0.f;
+            }
+#pragma unroll
+            for (int t = 0; t < TPT; ++t) {
+                float d[A], o[A];
+#pragma unroll
+                for (int s = 0; s < A; ++s) d[s] = row[M * t + s];
+                mat_apply<A, A>(typename Wm::Bt{}, d, o);
+#pragma unroll
+                for (int s = 0; s < A; ++s) e[r][t][s] = o[s];
+            }
+        }
+    } else {
+#pragma unroll
+        for (int r = 0; r < A; ++r)
+#pragma unroll
+            for (int t = 0; t < TPT; ++t)
+#pragma unroll
+                for (int s = 0; s < A; ++s) e[r][t][s] = 0.f;
+    }
+    const long long plane = static_cast<long long>(C) * Pstride;
+    __half* dst = V + static_cast<long long>(c) * Pstride + pl;
+#pragma unroll
+    for (int nu = 0; nu < A; ++nu) {
+        float v[A][TPT];  // v[xi][t]
+#pragma unroll
+        for (int t = 0; t < TPT; ++t) {
+            float col[A], o[A];
+#pragma unroll
+            for (int r = 0; r < A; ++r) col[r] = e[r][t][nu];
+            mat_apply<A, A>(typename Wm::Bt{}, col, o);
+#pragma unroll
+            for (int xi = 0; xi < A; ++xi) v[xi][t] = o[xi];
+        }
+#pragma unroll
+        for (int xi = 0; xi < A; ++xi) {
+            __half* q = dst + (xi * A + nu) * plane;
+            if constexpr (TPT == 4) {
+                uint2 w;
+                w.x = pack2(v[xi][0], v[xi][1]);
+                w.y = pack2(v[xi][2], v[xi][3]);
+                *reinterpret_cast<uint2*>(q) = w;
+            } else {
+                *reinterpret_cast<uint32_t*>(q) = pack2(v[xi][0], v[xi][1]);
+            }
+        }
+    }
+}
+
+template <int M, int TPT>
+__global__ void __launch_bounds__(128)
+output_transform_vec_kernel(const __half* __restrict__ Mws, const __half* __restrict__ bias, __half* __restrict__ y,
+                            TileGeom geo, int K, long long p_begin, int p_count, long long Pstride) {
+    using Wm = Wino<M>;
+    constexpr int A = Wm::A;
+    static_assert(M * TPT == 8, "one 16-byte row segment per thread");
+    const int pl = (blockIdx.x * blockDim.x + threadIdx.x) * TPT;
+    const int k = blockIdx.y;
+    if (pl >= p_count) return;
+    const long long p = p_begin + pl;
+    if (p >= geo.P) return;
+    const long long plane = static_cast<long long>(K) * Pstride;
+    const __half* src = Mws + static_cast<long long>(k) * Pstride + pl;
+    float mm[A][A][TPT];
+#pragma unroll
+    for (int r = 0; r < A; ++r)
+#pragma unroll
+        for (int s = 0; s < A; ++s) {
+            const __half* q = src + (r * A + s) * plane;
+            if constexpr (TPT == 4) {
+                const uint2 w = __ldg(reinterpret_cast<const uint2*>(q));
+                unpack2(w.x, mm[r][s][0], mm[r][s][1]);
+                unpack2(w.y, mm[r][s][2], mm[r][s][3]);
+            } else {
+                const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(q));
+                unpack2(w, mm[r][s][0], mm[r][s][1]);
+            }
+        }
+    const int tw = static_cast<int>(p % geo.TW);
+    const int th = static_cast<int>((p / geo.TW) % geo.TH);
+    const long long n = p / (static_cast<long long>(geo.TW) * geo.TH);
+    const float b = bias ? __half2float(__ldg(bias + k)) : 0.f;
+    __half* img = y + (n * K + k) * static_cast<long long>(geo.H) * geo.W;
+    const int i0 = M * th, j0 = M * tw;
+    float out[M][8];  // M output rows of 8 pixels
+#pragma unroll
+    for (int t = 0; t < TPT; ++t) {
+        float tt[M][A];  // A^T mm (M x A)
+#pragma unroll
+        for (int s = 0; s < A; ++s) {
+            float col[A], o[M];
+#pragma unroll
+            for (int r = 0; r < A; ++r) col[r] = mm[r][s][t];
+            mat_apply<M, A>(typename Wm::At{}, col, o);
+#pragma unroll
+            for (int i = 0; i < M; ++i) tt[i][s] = o[i];
+        }
+#pragma unroll
+        for (int i = 0; i < M; ++i) {
+            float o[M];
+            mat_apply<M, A>(typename Wm::At{}, tt[i], o);
+#pragma unroll
+            for (int j = 0; j < M; ++j) out[i][M * t + j] = o[j] + b;
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < M; ++i) {
+        if (i0 + i >= geo.H) continue;
+        uint4 w;
+        w.x = pack2(out[i][0], out[i][1]);
+        w.y = pack2(out[i][2], out[i][3]);
+        w.z = pack2(out[i][4], out[i][5]);
+        w.w = pack2(out[i][6], out[i][7]);
+        *reinterpret_cast<uint4*>(img + static_cast<long long>(i0 + i) * geo.W + j0) = w;
+    }
+}
+
 }  // namespace sdw
