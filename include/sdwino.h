@@ -136,6 +136,12 @@ int sdwino_set_gemm_shape(int ctas, int n_tile);
  */
 int sdwino_profile_enable(int enable);
 int sdwino_profile_collect(double *ms_by_kind, unsigned long long *launches_by_kind);
+/* The same records one by one, in launch order: fills kinds[i] and ms[i] (host arrays of `capacity`
+ * entries, either may be NULL; ms < 0 marks an event error) for the first `capacity` launches since
+ * the last collect and returns how many there were.  keep == 0 forgets the records; keep != 0
+ * leaves them in place, which is how launches captured into a CUDA graph while profiling was
+ * enabled are read again after every replay of that graph (the events are then graph nodes). */
+int sdwino_profile_records(int *kinds, float *ms, int capacity, int keep);
 
 #ifdef __cplusplus
 }

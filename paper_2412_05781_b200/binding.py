@@ -21,7 +21,7 @@ EXPORTS = [
     "sdwino_workspace_bytes", "sdwino_workspace_min_bytes", "sdwino_set_workspace", "sdwino_conv3x3",
     "sdwino_conv3x3_ws", "sdwino_host_staging_bytes", "sdwino_conv3x3_host",
     "sdwino_last_device_status", "sdwino_launch_count", "sdwino_profile_enable", "sdwino_profile_collect",
-    "sdwino_set_gemm_shape",
+    "sdwino_profile_records", "sdwino_set_gemm_shape",
 ]
 
 KERNEL_KINDS = ("filter_transform", "input_transform", "wino_gemm", "output_transform")
@@ -61,6 +61,8 @@ def _load() -> ctypes.CDLL:
     lib.sdwino_last_device_status.restype = i
     lib.sdwino_last_device_status.argtypes = [vp]
     lib.sdwino_launch_count.restype = ctypes.c_ulonglong
+    lib.sdwino_profile_records.restype = i
+    lib.sdwino_profile_records.argtypes = [ctypes.POINTER(i), ctypes.POINTER(ctypes.c_float), i, i]
     lib.sdwino_set_gemm_shape.restype = i
     lib.sdwino_set_gemm_shape.argtypes = [i, i]
     lib.sdwino_profile_enable.restype = i
@@ -134,6 +136,17 @@ def sdwino_profile_collect():
     n = (ctypes.c_ulonglong * 4)()
     _check(lib.sdwino_profile_collect(ms, n), "sdwino_profile_collect")
     return {k: (float(ms[i]), int(n[i])) for i, k in enumerate(KERNEL_KINDS)}
+
+
+def sdwino_profile_records(capacity: int = 1 << 16, keep: bool = False):
+    """-> [(kernel kind, milliseconds)] in launch order since the last collect; keep=True leaves the
+    records in place (launches captured in a CUDA graph, read again after every replay)."""
+    kinds = (ctypes.c_int * capacity)()
+    ms = (ctypes.c_float * capacity)()
+    n = int(lib.sdwino_profile_records(kinds, ms, capacity, 1 if keep else 0))
+    if n > capacity:
+        raise RuntimeError(f"{n} profile records, capacity {capacity}")
+    return [(KERNEL_KINDS[kinds[i]], float(ms[i])) for i in range(n)]
 
 
 def alloc_workspace(nbytes: int, device="cuda") -> torch.Tensor:

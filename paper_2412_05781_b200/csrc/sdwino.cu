@@ -43,15 +43,24 @@ cudaEvent_t prof_event() {
     if (cudaEventCreate(&e) != cudaSuccess) return nullptr;
     return e;
 }
+// While the stream is being captured into a CUDA graph the records must be external event nodes,
+// otherwise their elapsed time cannot be queried after a replay.
+void prof_record(cudaEvent_t e, cudaStream_t st) {
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cs) == cudaSuccess && cs == cudaStreamCaptureStatusActive)
+        cudaEventRecordWithFlags(e, st, cudaEventRecordExternal);
+    else
+        cudaEventRecord(e, st);
+}
 struct ProfScope {
     cudaStream_t st; int kind; cudaEvent_t beg = nullptr;
     ProfScope(int k, cudaStream_t s) : st(s), kind(k) {
-        if (g_profile) { beg = prof_event(); if (beg) cudaEventRecord(beg, st); }
+        if (g_profile) { beg = prof_event(); if (beg) prof_record(beg, st); }
     }
     ~ProfScope() {
         if (beg) {
             cudaEvent_t end = prof_event();
-            if (end) { cudaEventRecord(end, st); g_prof_records.push_back({kind, beg, end}); }
+            if (end) { prof_record(end, st); g_prof_records.push_back({kind, beg, end}); }
             else g_event_pool.push_back(beg);
         }
     }
@@ -121,9 +130,40 @@ EncodeTiledFn get_encode_fn() {
 }
 
 // fp16 tensor [d2][d1][d0] (d0 contiguous, row pitch `pitch0` elements, plane pitch `pitch1`
-// elements) with a {b0, b1, 1} box, with the 128-byte swizzle or none.
+// elements) with a {b0, b1, 1} box, with the 128-byte swizzle or none.  Encoding costs about a
+// microsecond of host time, so the last few maps are kept (a map depends only on these arguments).
+struct MapKey {
+    const void* base; uint64_t d0, d1, d2, pitch0, pitch1; uint32_t b0, b1; bool sw;
+    bool operator==(const MapKey& o) const {
+        return base == o.base && d0 == o.d0 && d1 == o.d1 && d2 == o.d2 && pitch0 == o.pitch0 && pitch1 == o.pitch1 &&
+               b0 == o.b0 && b1 == o.b1 && sw == o.sw;
+    }
+};
+struct MapSlot { MapKey key; CUtensorMap map; bool used = false; };
+constexpr int MAP_CACHE_SLOTS = 256;
+MapSlot g_map_cache[MAP_CACHE_SLOTS];
+std::mutex g_map_mutex;
+
+bool encode_map_uncached(CUtensorMap* m, const void* base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t pitch0,
+                         uint64_t pitch1, uint32_t b0, uint32_t b1, bool swizzle128);
+
 bool encode_map(CUtensorMap* m, const void* base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t pitch0,
                 uint64_t pitch1, uint32_t b0, uint32_t b1, bool swizzle128) {
+    const MapKey key{base, d0, d1, d2, pitch0, pitch1, b0, b1, swizzle128};
+    uint64_t h = reinterpret_cast<uintptr_t>(base) >> 8;
+    h = h * 1000003u ^ d0 * 31u ^ d1 * 131u ^ pitch0 * 7u ^ (static_cast<uint64_t>(b1) << 20) ^ (b0 << 3) ^ swizzle128;
+    MapSlot& slot = g_map_cache[h % MAP_CACHE_SLOTS];
+    std::lock_guard<std::mutex> lock(g_map_mutex);
+    if (slot.used && slot.key == key) { *m = slot.map; return true; }
+    if (!encode_map_uncached(m, base, d0, d1, d2, pitch0, pitch1, b0, b1, swizzle128)) return false;
+    slot.key = key;
+    slot.map = *m;
+    slot.used = true;
+    return true;
+}
+
+bool encode_map_uncached(CUtensorMap* m, const void* base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t pitch0,
+                         uint64_t pitch1, uint32_t b0, uint32_t b1, bool swizzle128) {
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return false;
     cuuint64_t dims[3] = {d0, d1, d2};
@@ -257,8 +297,9 @@ int launch_gemm(const CUtensorMap& tmU, const CUtensorMap& tmV, const CUtensorMa
                 int ctas, cudaStream_t st) {
     const int sms = sm_count();
     if (sms <= 0) return SDWINO_ERR_CUDA;
-    int* status = nullptr;
-    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&status), g_status_word) != cudaSuccess) return SDWINO_ERR_CUDA;
+    static int* status = nullptr;   // device address of the status word (one device per process)
+    if (!status && cudaGetSymbolAddress(reinterpret_cast<void**>(&status), g_status_word) != cudaSuccess)
+        return SDWINO_ERR_CUDA;
     if (ctas == 2) return launch_gemm_shape<2>(tmU, tmV, tmM, prm, sms, status, st);
     return launch_gemm_shape<1>(tmU, tmV, tmM, prm, sms, status, st);
 }
@@ -300,15 +341,12 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
     prm.num_c_blocks = (C + GEMM_BLOCK_C - 1) / GEMM_BLOCK_C;
     prm.C = C;
     const int b_rows = prm.n_tile / shape.ctas;
-    // epilogue staging: half a tile per TMA store when that is a multiple of 16 channels, two buffers when at
-    // least four pipeline stages still fit beside them
-    prm.epi_rows = (prm.n_tile > 64 && (prm.n_tile / 2) % 16 == 0) ? prm.n_tile / 2 : prm.n_tile;
-    prm.epi_bufs = 2;
-    prm.stages = (MAX_DYN_SMEM - GemmSmemLayout::dyn_bytes(b_rows, 0, prm.epi_rows, 2)) / GemmSmemLayout::stage_bytes(b_rows);
-    if (prm.stages < 4) {
-        prm.epi_bufs = 1;
-        prm.stages = (MAX_DYN_SMEM - GemmSmemLayout::dyn_bytes(b_rows, 0, prm.epi_rows, 1)) / GemmSmemLayout::stage_bytes(b_rows);
-    }
+    // epilogue staging: two groups of epilogue warps each take half a tile when that is a multiple of 16 channels
+    const bool split = (prm.n_tile / 2) % 16 == 0;
+    prm.epi_rows = split ? prm.n_tile / 2 : prm.n_tile;
+    prm.epi_bufs = split ? 2 : 1;
+    prm.stages = (MAX_DYN_SMEM - GemmSmemLayout::dyn_bytes(b_rows, 0, prm.epi_rows, prm.epi_bufs)) /
+                 GemmSmemLayout::stage_bytes(b_rows);
     if (prm.stages > GEMM_MAX_STAGES) prm.stages = GEMM_MAX_STAGES;
 
     prm.p_stride = pc;
@@ -480,6 +518,26 @@ int sdwino_profile_enable(int enable) {
     std::lock_guard<std::mutex> lock(g_mutex);
     g_profile = enable != 0;
     return SDWINO_OK;
+}
+
+int sdwino_profile_records(int* kinds, float* ms, int capacity, int keep) {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    int n = 0;
+    for (const ProfRecord& r : g_prof_records) {
+        float t = 0.f;
+        if (cudaEventSynchronize(r.end) != cudaSuccess || cudaEventElapsedTime(&t, r.beg, r.end) != cudaSuccess) t = -1.f;
+        if (n < capacity) {
+            if (kinds) kinds[n] = r.kind;
+            if (ms) ms[n] = t;
+        }
+        ++n;
+        if (!keep) {
+            g_event_pool.push_back(r.beg);
+            g_event_pool.push_back(r.end);
+        }
+    }
+    if (!keep) g_prof_records.clear();
+    return n;
 }
 
 int sdwino_profile_collect(double* ms_by_kind, unsigned long long* launches_by_kind) {

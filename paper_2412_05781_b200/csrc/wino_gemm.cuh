@@ -18,7 +18,8 @@
 // One persistent CTA (pair) per SM (pair) walks the list of (pos, k-tile, p-tile) output tiles.
 //   warp 0   : TMA producer        (one lane)
 //   warp 1   : TMEM owner + MMA issuer (one lane)
-//   warps 2-5: epilogue, one TMEM lane quarter each; TMEM accumulators are double-buffered so
+//   warps 2-9: epilogue in two groups of four warps (one TMEM lane quarter per warp); group g drains
+//              channels [g * epi_rows, (g + 1) * epi_rows) of the tile; TMEM accumulators are double-buffered so
 //              the epilogue of tile i overlaps the MMAs of tile i+1.  A thread owns one tile p and
 //              reads its channels from TMEM; the fp16 results are transposed through a shared-memory
 //              staging buffer [k][128 p] and leave with one TMA store per epi_rows channels, so M is
@@ -38,7 +39,7 @@ __device__ __forceinline__ void report_timeout(int* status_word, int where, uint
 constexpr int GEMM_BLOCK_P = 128;  // tiles per output tile (TMEM lanes, UMMA M)
 constexpr int GEMM_BLOCK_C = 64;   // input channels per pipeline stage (one 128-byte swizzle row of U)
 constexpr int GEMM_MAX_N = 256;    // output channels per output tile (UMMA N), multiple of 16
-constexpr int GEMM_THREADS = 192;
+constexpr int GEMM_THREADS = 320;  // warp 0 producer, warp 1 MMA, warps 2-9 epilogue (two groups of four)
 constexpr int GEMM_MAX_STAGES = 8;
 constexpr uint64_t GEMM_WAIT_LIMIT_NS = 2000000000ull;  // a wait longer than 2 s is reported, not spun on
 
@@ -70,8 +71,8 @@ struct GemmParams {
     int C;             // input channels (for the k-steps of the last block)
     int n_tile;        // UMMA N
     int stages;
-    int epi_rows;      // channels staged per TMA store: divides n_tile, multiple of 16
-    int epi_bufs;      // staging buffers (1 or 2)
+    int epi_rows;      // channels staged per TMA store and epilogue group: n_tile or n_tile / 2, multiple of 16
+    int epi_bufs;      // staging buffers = epilogue groups with work (1 or 2)
     long long p_stride;  // tiles per pass (row pitch of V and M)
 };
 
@@ -112,7 +113,7 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(&acc_full_bar[b], 1);
-            mbar_init(&acc_empty_bar[b], 4 * CTAS);   // one arrival per epilogue warp of every CTA
+            mbar_init(&acc_empty_bar[b], 8 * CTAS);   // one arrival per epilogue warp of every CTA
         }
         *abort_flag = 0;
         fence_barrier_init();
@@ -135,7 +136,11 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
         if (lane == 0) {
             // the full barrier of a pair lives in the leader and counts the bytes of both CTAs
             const uint32_t tx_bytes = CTAS * (L::A_BYTES + L::b_bytes(b_rows));
-            const uint32_t leader_full0 = CTAS == 2 ? map_to_cta(smem_u32(&full_bar[0]), 0) : 0u;
+            // single-thread loop: shared-memory and barrier addresses are running 32-bit values
+            const uint32_t smem_base = smem_u32(smem);
+            const uint32_t full0_local = smem_u32(&full_bar[0]);
+            const uint32_t full0 = CTAS == 2 ? map_to_cta(full0_local, 0) : full0_local;
+            uint32_t sa = smem_base, fb = full0, fb_local = full0_local;
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
@@ -145,23 +150,24 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
                 const int pos = tile / (prm.num_p_tiles * prm.num_k_tiles);
                 const int p0 = (pt * CTAS + static_cast<int>(cta_rank)) * GEMM_BLOCK_P;
                 const int k0 = kt * prm.n_tile + static_cast<int>(cta_rank) * b_rows;
-                for (int cb = 0; cb < prm.num_c_blocks; ++cb) {
+                for (int c0 = 0; c0 < prm.C; c0 += GEMM_BLOCK_C) {
                     ok = mbar_wait_bounded(&empty_bar[stage], phase ^ 1u, abort_flag, GEMM_WAIT_LIMIT_NS);
                     if (!ok) { if (*abort_flag == 0) report_timeout(status_word, 1, cta_rank); break; }
-                    uint8_t* sa = smem + stage * stage_bytes;
                     if constexpr (CTAS == 2) {
-                        if (leader) mbar_arrive_expect_tx(&full_bar[stage], tx_bytes);
-                        const uint32_t fb = leader_full0 + static_cast<uint32_t>(stage) * 8u;
-                        tma_load_3d_pair(sa, &tmV, fb, p0, cb * GEMM_BLOCK_C, pos);
-                        tma_load_3d_pair(sa + L::A_BOX_BYTES, &tmV, fb, p0 + 64, cb * GEMM_BLOCK_C, pos);
-                        tma_load_3d_pair(sa + L::A_BYTES, &tmU, fb, cb * GEMM_BLOCK_C, k0, pos);
+                        if (leader) mbar_arrive_expect_tx_a32(fb_local, tx_bytes);
+                        tma_load_3d_pair(sa, &tmV, fb, p0, c0, pos);
+                        tma_load_3d_pair(sa + L::A_BOX_BYTES, &tmV, fb, p0 + 64, c0, pos);
+                        tma_load_3d_pair(sa + L::A_BYTES, &tmU, fb, c0, k0, pos);
                     } else {
-                        mbar_arrive_expect_tx(&full_bar[stage], tx_bytes);
-                        tma_load_3d(sa, &tmV, &full_bar[stage], p0, cb * GEMM_BLOCK_C, pos);
-                        tma_load_3d(sa + L::A_BOX_BYTES, &tmV, &full_bar[stage], p0 + 64, cb * GEMM_BLOCK_C, pos);
-                        tma_load_3d(sa + L::A_BYTES, &tmU, &full_bar[stage], cb * GEMM_BLOCK_C, k0, pos);
+                        mbar_arrive_expect_tx_a32(fb, tx_bytes);
+                        tma_load_3d_a32(sa, &tmV, fb, p0, c0, pos);
+                        tma_load_3d_a32(sa + L::A_BOX_BYTES, &tmV, fb, p0 + 64, c0, pos);
+                        tma_load_3d_a32(sa + L::A_BYTES, &tmU, fb, c0, k0, pos);
                     }
-                    if (++stage == stages) { stage = 0; phase ^= 1u; }
+                    sa += stage_bytes;
+                    fb += 8;
+                    fb_local += 8;
+                    if (++stage == stages) { stage = 0; phase ^= 1u; sa = smem_base; fb = full0; fb_local = full0_local; }
                 }
             }
             if (!ok) *abort_flag = 1;
@@ -170,6 +176,17 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
         // ------------------------------ MMA issuer ------------------------------
         if (lane == 0 && leader) {
             const uint32_t idesc = make_idesc_f16_f32(GEMM_BLOCK_P * CTAS, prm.n_tile, true, false);
+            // This loop is executed by ONE thread, so every instruction in it costs its full latency: the
+            // descriptors of stage 0 are built once and then only advanced by additions (the 14-bit
+            // address field cannot overflow inside 227 KB of shared memory).
+            //   A (M-major): 16 channels = 16 rows of 128 bytes = +2048 bytes; the two 64-wide p blocks are
+            //   A_BOX_BYTES apart.  B (K-major): 16 channels = +32 bytes along the swizzled 128-byte row.
+            const uint32_t smem_base = smem_u32(smem);
+            const uint64_t adesc0 = make_smem_desc_sw128(smem_base, L::A_BOX_BYTES, 1024);
+            const uint64_t bdesc0 = make_smem_desc_sw128(smem_base + L::A_BYTES, 16, 1024);
+            const uint64_t stage_step = static_cast<uint64_t>(stage_bytes >> 4);
+            uint64_t adesc = adesc0, bdesc = bdesc0;
+            const int last_ksteps = ((prm.C - (prm.num_c_blocks - 1) * GEMM_BLOCK_C) + 15) / 16;  // 1..4
             int stage = 0;
             uint32_t phase = 0;
             int buf = 0;
@@ -184,21 +201,31 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
                     ok = mbar_wait_bounded(&full_bar[stage], phase, abort_flag, GEMM_WAIT_LIMIT_NS);
                     if (!ok) { if (*abort_flag == 0) report_timeout(status_word, 3, cta_rank); break; }
                     tc_fence_after_sync();
-                    const uint32_t a_addr = smem_u32(smem + stage * stage_bytes);
-                    const uint32_t b_addr = a_addr + L::A_BYTES;
-                    const int c_left = prm.C - cb * GEMM_BLOCK_C;
-                    const int ksteps = c_left >= GEMM_BLOCK_C ? GEMM_BLOCK_C / 16 : (c_left + 15) / 16;
-                    for (int s = 0; s < ksteps; ++s) {
-                        // A (M-major): 16 channels = 16 rows of 128 bytes; the two 64-wide p blocks are
-                        // A_BOX_BYTES apart.  B (K-major): 16 channels = 32 bytes along the swizzled row.
-                        const uint64_t adesc = make_smem_desc_sw128(a_addr + s * 2048, L::A_BOX_BYTES, 1024);
-                        const uint64_t bdesc = make_smem_desc_sw128(b_addr + s * 32, 16, 1024);
-                        if constexpr (CTAS == 2) umma_f16_pair(d_tmem, adesc, bdesc, idesc, (cb > 0 || s > 0) ? 1u : 0u);
-                        else umma_f16(d_tmem, adesc, bdesc, idesc, (cb > 0 || s > 0) ? 1u : 0u);
+                    if (cb + 1 < prm.num_c_blocks || last_ksteps == 4) {
+                        if constexpr (CTAS == 2) {
+                            umma_f16_pair(d_tmem, adesc, bdesc, idesc, cb > 0 ? 1u : 0u);
+                            umma_f16_pair_acc(d_tmem, adesc + 128, bdesc + 2, idesc);
+                            umma_f16_pair_acc(d_tmem, adesc + 256, bdesc + 4, idesc);
+                            umma_f16_pair_acc(d_tmem, adesc + 384, bdesc + 6, idesc);
+                        } else {
+                            umma_f16(d_tmem, adesc, bdesc, idesc, cb > 0 ? 1u : 0u);
+                            umma_f16_acc(d_tmem, adesc + 128, bdesc + 2, idesc);
+                            umma_f16_acc(d_tmem, adesc + 256, bdesc + 4, idesc);
+                            umma_f16_acc(d_tmem, adesc + 384, bdesc + 6, idesc);
+                        }
+                    } else {
+                        for (int s = 0; s < last_ksteps; ++s) {
+                            if constexpr (CTAS == 2)
+                                umma_f16_pair(d_tmem, adesc + 128 * s, bdesc + 2 * s, idesc, (cb > 0 || s > 0) ? 1u : 0u);
+                            else
+                                umma_f16(d_tmem, adesc + 128 * s, bdesc + 2 * s, idesc, (cb > 0 || s > 0) ? 1u : 0u);
+                        }
                     }
                     if constexpr (CTAS == 2) umma_commit_pair(&empty_bar[stage]);
                     else umma_commit(&empty_bar[stage]);
-                    if (++stage == stages) { stage = 0; phase ^= 1u; }
+                    adesc += stage_step;
+                    bdesc += stage_step;
+                    if (++stage == stages) { stage = 0; phase ^= 1u; adesc = adesc0; bdesc = bdesc0; }
                 }
                 if (!ok) break;
                 if constexpr (CTAS == 2) umma_commit_pair(&acc_full_bar[buf]);
@@ -211,8 +238,9 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
     } else {
         // ------------------------------ epilogue ------------------------------
         const int quarter = warp & 3;          // TMEM lanes this warp may read: 32*quarter .. +31
+        const int group = (warp - 2) >> 2;           // 0: warps 2-5, 1: warps 6-9
+        const int group_tid = threadIdx.x - 64 - group * 128;
         int buf = 0;
-        int sbuf = 0;
         uint32_t acc_phase = 0;
         // the accumulator-empty barrier of a pair lives in the leader
         const uint32_t acc_empty_addr0 = CTAS == 2 ? map_to_cta(smem_u32(&acc_empty_bar[0]), 0) : 0u;
@@ -235,19 +263,25 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
             const int p0 = (pt * CTAS + static_cast<int>(cta_rank)) * GEMM_BLOCK_P + quarter * 32;
             const int k0 = kt * prm.n_tile;
             const bool p_ok = p0 < prm.p_stride;   // the second CTA of the last pair may hang over the pass
-            const int epi_tid = threadIdx.x - 64;
             // lane = tile p, registers = output channels: staging row k receives 32 consecutive p from
-            // each warp (64 contiguous bytes, no bank conflict)
-            for (int row0 = 0; row0 < prm.n_tile; row0 += prm.epi_rows) {
-                uint8_t* stg = epi_base + sbuf * prm.epi_rows * L::EPI_ROW_BYTES;
-                // the buffer about to be overwritten must have been read by its TMA store
-                if (epi_tid == 0) {
-                    if (prm.epi_bufs == 2) tma_store_wait_read_pending<1>();
-                    else tma_store_wait_read_pending<0>();
-                }
-                asm volatile("bar.sync 1, 128;" ::: "memory");
+            // each warp (64 contiguous bytes, no bank conflict).  Group g owns staging buffer g.
+            const int row0 = group * prm.epi_rows;
+            if (row0 < prm.n_tile) {
+                uint8_t* stg = epi_base + group * prm.epi_rows * L::EPI_ROW_BYTES;
+                // the buffer about to be overwritten must have been read by the group's previous TMA store
+                if (group_tid == 0) tma_store_wait_read_pending<0>();
+                if (group == 0) asm volatile("bar.sync 1, 128;" ::: "memory");
+                else asm volatile("bar.sync 2, 128;" ::: "memory");
                 __half* dst = reinterpret_cast<__half*>(stg) + quarter * 32 + lane;
-                for (int col = 0; col < prm.epi_rows; col += 16) {
+                int col = 0;
+                for (; col + 32 <= prm.epi_rows; col += 32) {
+                    uint32_t r[32];
+                    tmem_ld_32x32_sync(t_addr + row0 + col, r);
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        dst[(col + i) * GEMM_BLOCK_P] = __float2half_rn(__uint_as_float(r[i]));
+                }
+                if (col < prm.epi_rows) {
                     uint32_t r[16];
                     tmem_ld_32x16_sync(t_addr + row0 + col, r);
 #pragma unroll
@@ -255,12 +289,12 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
                         dst[(col + i) * GEMM_BLOCK_P] = __float2half_rn(__uint_as_float(r[i]));
                 }
                 fence_proxy_async_smem();
-                asm volatile("bar.sync 1, 128;" ::: "memory");
-                if (epi_tid == 0) {
+                if (group == 0) asm volatile("bar.sync 1, 128;" ::: "memory");
+                else asm volatile("bar.sync 2, 128;" ::: "memory");
+                if (group_tid == 0) {
                     if (p_ok) tma_store_3d(&tmM, stg, p0 - quarter * 32, k0 + row0, pos);
                     tma_store_commit();
                 }
-                if (prm.epi_bufs == 2) sbuf ^= 1;
             }
             // accumulator drained: hand the TMEM buffer back to the MMA warp
             tc_fence_before_sync();
@@ -272,7 +306,7 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
             buf ^= 1;
             if (buf == 0) acc_phase ^= 1u;
         }
-        if (threadIdx.x == 64) tma_store_wait_all();
+        if (group_tid == 0) tma_store_wait_all();
     }
 
     __syncwarp();
