@@ -91,6 +91,29 @@ int sdwino_conv3x3_ws(const void *x, const void *wT, const void *bias, void *y,
                       void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * The convolution for callers that must not allocate device memory.  (The paper has no
+ * counterpart; this entry point exists for the embedding of the library.)  Some callers cannot
+ * call cudaMalloc or any allocator at all: code that runs inside a CUDA-graph capture or another
+ * region where allocation is forbidden, plug-ins whose host hands them fixed buffers and bans
+ * further allocation, and processes whose memory budget is fixed at start-up.  They still pass x,
+ * wT, bias and y exactly as to sdwino_conv3x3, but the scratch for V and M is a file-scope device
+ * array of SDWINO_STATIC_SCRATCH_BYTES inside the library image, so every GPU that loads the library
+ * holds that much memory until the process exits, and no allocation call is made on this path.
+ *
+ *   - Limit: a layer is accepted when one pass of 128 tiles fits, i.e. when
+ *     128 * (tile+2)^2 * (C + K) * 2 bytes + 2 KiB <= SDWINO_STATIC_SCRATCH_BYTES (for tile 2,
+ *     C + K <= 4095); larger layers return SDWINO_ERR_WORKSPACE.  Large images simply take more passes.
+ *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
+ *     that device current).  Make that first call outside any stream capture.
+ *   - All calls share the one array and it keeps the contents of the last call.  Nothing in it has to
+ *     start at zero: every pass overwrites all elements it later reads.  Calls that may overlap on the
+ *     GPU (different streams, or graphs replayed concurrently) race on the array; order them.
+ */
+#define SDWINO_STATIC_SCRATCH_BYTES (32u << 20)
+int sdwino_conv3x3_static(const void *x, const void *wT, const void *bias, void *y,
+                          int N, int C, int H, int W, int K, int tile, void *stream);
+
+/*
  * The same convolution for callers whose tensors live in HOST memory (pageable or pinned):
  * x_host, bias_host and y_host are host pointers, wT stays a device pointer.  On `stream`
  * the call copies x (and bias) to the device, runs the three steps, copies y back and then

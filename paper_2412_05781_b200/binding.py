@@ -21,7 +21,7 @@ EXPORTS = [
     "sdwino_workspace_bytes", "sdwino_workspace_min_bytes", "sdwino_set_workspace", "sdwino_conv3x3",
     "sdwino_conv3x3_ws", "sdwino_host_staging_bytes", "sdwino_conv3x3_host",
     "sdwino_last_device_status", "sdwino_launch_count", "sdwino_profile_enable", "sdwino_profile_collect",
-    "sdwino_profile_records", "sdwino_set_gemm_shape",
+    "sdwino_profile_records", "sdwino_set_gemm_shape", "sdwino_conv3x3_static",
 ]
 
 KERNEL_KINDS = ("filter_transform", "input_transform", "wino_gemm", "output_transform")
@@ -54,6 +54,8 @@ def _load() -> ctypes.CDLL:
     lib.sdwino_set_workspace.argtypes = [vp, sz]
     lib.sdwino_conv3x3.restype = i
     lib.sdwino_conv3x3.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, vp]
+    lib.sdwino_conv3x3_static.restype = i
+    lib.sdwino_conv3x3_static.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, vp]
     lib.sdwino_conv3x3_ws.restype = i
     lib.sdwino_conv3x3_ws.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, vp, sz, vp]
     lib.sdwino_conv3x3_host.restype = i
@@ -199,6 +201,24 @@ def sdwino_conv3x3(x: torch.Tensor, wT: torch.Tensor, bias: Optional[torch.Tenso
                                    workspace.data_ptr(), workspace.numel() * workspace.element_size(),
                                    _stream_ptr(stream))
     _check(rc, "sdwino_conv3x3")
+    return y
+
+
+STATIC_SCRATCH_BYTES = 32 << 20
+
+
+def sdwino_conv3x3_static(x: torch.Tensor, wT: torch.Tensor, bias: Optional[torch.Tensor], K: int, tile: int,
+                          y: torch.Tensor, stream=None) -> torch.Tensor:
+    """The convolution with the library's built-in scratch array: for callers that may not allocate
+    device memory.  x, wT, bias and the output y are all supplied by the caller; this wrapper allocates
+    nothing either.  Layers whose smallest pass does not fit the STATIC_SCRATCH_BYTES array raise
+    SdwinoError(ERR_WORKSPACE).  Calls share the array, so do not let two of them overlap on the GPU."""
+    assert x.is_cuda and x.dtype == torch.float16 and x.is_contiguous() and x.dim() == 4
+    N, C, H, W = (int(v) for v in x.shape)
+    assert y.is_cuda and y.is_contiguous() and y.dtype == torch.float16 and tuple(y.shape) == (N, K, H, W)
+    rc = lib.sdwino_conv3x3_static(x.data_ptr(), wT.data_ptr(), _ptr(bias), y.data_ptr(), N, C, H, W, K, tile,
+                                   _stream_ptr(stream))
+    _check(rc, "sdwino_conv3x3_static")
     return y
 
 

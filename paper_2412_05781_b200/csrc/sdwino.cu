@@ -514,6 +514,52 @@ int sdwino_last_device_status(void* stream) {
 
 unsigned long long sdwino_launch_count(void) { return g_launches.load(); }
 
+}  // extern "C"
+
+namespace {
+// Scratch for sdwino_conv3x3_static: lives in the library's device image, so no allocation call is ever
+// made for it.  In host code this name is only a stand-in for the device object (it is not a device
+// address); the address kernels can use comes from cudaGetSymbolAddress, once per device.
+static __device__ __align__(256) unsigned char g_static_scratch[SDWINO_STATIC_SCRATCH_BYTES];
+constexpr int STATIC_MAX_DEVICES = 64;
+void* g_static_scratch_ptr[STATIC_MAX_DEVICES] = {};
+std::mutex g_static_mutex;
+}  // namespace
+
+extern "C" {
+
+int sdwino_conv3x3_static(const void* x, const void* wT, const void* bias, void* y, int N, int C, int H, int W,
+                          int K, int tile, void* stream) {
+    if (tile != 2 && tile != 4) {
+        return (N <= 0 || C <= 0 || H <= 0 || W <= 0 || K <= 0 || !x || !wT || !y) ? SDWINO_ERR_INVALID_ARG
+                                                                                     : SDWINO_ERR_UNSUPPORTED;
+    }
+    Plan pl;
+    if (!x || !wT || !y || !make_plan(N, C, H, W, K, tile, &pl)) return SDWINO_ERR_INVALID_ARG;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return SDWINO_ERR_CUDA;
+    if (dev < 0 || dev >= STATIC_MAX_DEVICES) return SDWINO_ERR_UNSUPPORTED;
+    void* base = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        if (!g_static_scratch_ptr[dev]) {
+            // set-up, once per device, with that device current
+            void* p = nullptr;
+            if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return SDWINO_ERR_CUDA;
+            g_static_scratch_ptr[dev] = p;
+        }
+        base = g_static_scratch_ptr[dev];
+    }
+    // the convolution wants its scratch on a 1024-byte boundary; the array is only promised 256
+    const uintptr_t raw = reinterpret_cast<uintptr_t>(base);
+    const uintptr_t up = (raw + WS_ALIGN - 1) / WS_ALIGN * WS_ALIGN;
+    const size_t usable = SDWINO_STATIC_SCRATCH_BYTES - static_cast<size_t>(up - raw);
+    // sizes beyond the maximum: even one pass of 128 tiles would not fit
+    if (static_cast<size_t>(GEMM_BLOCK_P) * pl.per_tile + WS_ALIGN > usable) return SDWINO_ERR_WORKSPACE;
+    return conv_impl(x, wT, bias, y, N, C, H, W, K, tile, reinterpret_cast<void*>(up), usable,
+                     static_cast<cudaStream_t>(stream));
+}
+
 int sdwino_profile_enable(int enable) {
     std::lock_guard<std::mutex> lock(g_mutex);
     g_profile = enable != 0;
