@@ -18,6 +18,15 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
     return t;
 }
 
+// ---- programmatic dependent launch -------------------------------------------------------
+// The kernels of the library (all but the CTA-pair GEMM) are launched with programmatic stream
+// serialization: such a kernel may be scheduled
+// while its predecessor in the stream is still running.  pdl_wait() blocks until the predecessor has
+// completed and its memory is visible; it must come before the first global read or write of the kernel.
+// pdl_launch_dependents() lets the successor be scheduled early (its own pdl_wait keeps it correct).
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---- mbarrier -------------------------------------------------------------
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
@@ -45,6 +54,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 
+__device__ __forceinline__ bool mbar_try_wait_a32(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
 // Slow path of the bounded wait: polls, and every 4096 failed polls looks at the abort flag and at
 // the (slow to read) global timer.  Kept out of line so that the hot path stays a handful of
 // instructions: the waiting roles are single threads, whose instruction latency is the pipeline's.
@@ -198,6 +216,16 @@ __device__ __forceinline__ void umma_f16_acc(uint32_t tmem_d, uint64_t adesc, ui
         "{\n .reg .pred p;\n setp.eq.b32 p, 0, 0;\n"
         " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}" ::"r"(tmem_d),
         "l"(adesc), "l"(bdesc), "r"(idesc)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit_a32(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void umma_commit_pair_a32(uint32_t bar) {
+    const uint16_t mask = 3;
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
+        "h"(mask)
         : "memory");
 }
 // Arrive on an mbarrier once every MMA issued so far by this thread has completed.

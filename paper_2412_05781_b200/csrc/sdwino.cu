@@ -10,6 +10,7 @@
 #include <stdlib.h>
 
 #include <atomic>
+#include <utility>
 #include <mutex>
 #include <vector>
 
@@ -189,13 +190,44 @@ int sm_count() {
     return n;
 }
 
+// Kernels are launched with programmatic stream serialization (see pdl_wait in ptx.cuh); cluster_x: 0 for
+// the transform kernels, 1 or 2 CTAs per cluster for the GEMM.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, int cluster_x,
+                       Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    int n = 0;
+    // Cluster launches do not get the attribute: CTA-pair GEMMs launched with it stalled the stream
+    // intermittently (two-pass convolutions with few output channels), single-CTA launches never did.
+    if (cluster_x <= 1) {
+        attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n].val.programmaticStreamSerializationAllowed = 1;
+        ++n;
+    }
+    if (cluster_x > 1) {
+        attr[n].id = cudaLaunchAttributeClusterDimension;
+        attr[n].val.clusterDim.x = cluster_x;
+        attr[n].val.clusterDim.y = 1;
+        attr[n].val.clusterDim.z = 1;
+        ++n;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = n;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
 template <int M>
 int launch_filter(const __half* w, __half* U, int K, int C, int C8, cudaStream_t st) {
     dim3 grid((C8 + 127) / 128, K);
     ProfScope prof(KIND_FILTER, st);
-    filter_transform_kernel<M><<<grid, 128, 0, st>>>(w, U, K, C, C8);
+    const cudaError_t e = launch_pdl(filter_transform_kernel<M>, grid, dim3(128), 0, st, 0, w, U, K, C, C8);
     g_launches.fetch_add(1);
-    return cudaGetLastError() == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
+    return e == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
 }
 
 template <int M>
@@ -203,15 +235,17 @@ int launch_input(const __half* x, __half* V, const TileGeom& geo, int C, long lo
                  long long Pstride, cudaStream_t st) {
     ProfScope prof(KIND_INPUT, st);
     constexpr int TPT = 8 / M;
+    cudaError_t e;
     if (geo.W % 8 == 0 && aligned(x, 16)) {
         dim3 grid((p_count / TPT + 127) / 128, C);
-        input_transform_vec_kernel<M, TPT><<<grid, 128, 0, st>>>(x, V, geo, C, p_begin, p_count, Pstride);
+        e = launch_pdl(input_transform_vec_kernel<M, TPT>, grid, dim3(128), 0, st, 0, x, V, geo, C, p_begin, p_count,
+                       Pstride);
     } else {
         dim3 grid((p_count + 127) / 128, C);
-        input_transform_kernel<M><<<grid, 128, 0, st>>>(x, V, geo, C, p_begin, p_count, Pstride);
+        e = launch_pdl(input_transform_kernel<M>, grid, dim3(128), 0, st, 0, x, V, geo, C, p_begin, p_count, Pstride);
     }
     g_launches.fetch_add(1);
-    return cudaGetLastError() == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
+    return e == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
 }
 
 template <int M>
@@ -219,15 +253,18 @@ int launch_output(const __half* Mws, const __half* bias, __half* y, const TileGe
                   long long p_begin, int p_count, long long Pstride, cudaStream_t st) {
     ProfScope prof(KIND_OUTPUT, st);
     constexpr int TPT = 8 / M;
+    cudaError_t e;
     if (geo.W % 8 == 0 && aligned(y, 16)) {
         dim3 grid((p_count / TPT + 127) / 128, K);
-        output_transform_vec_kernel<M, TPT><<<grid, 128, 0, st>>>(Mws, bias, y, geo, K, p_begin, p_count, Pstride);
+        e = launch_pdl(output_transform_vec_kernel<M, TPT>, grid, dim3(128), 0, st, 0, Mws, bias, y, geo, K, p_begin,
+                       p_count, Pstride);
     } else {
         dim3 grid((p_count + 127) / 128, K);
-        output_transform_kernel<M><<<grid, 128, 0, st>>>(Mws, bias, y, geo, K, p_begin, p_count, Pstride);
+        e = launch_pdl(output_transform_kernel<M>, grid, dim3(128), 0, st, 0, Mws, bias, y, geo, K, p_begin, p_count,
+                       Pstride);
     }
     g_launches.fetch_add(1);
-    return cudaGetLastError() == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
+    return e == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
 }
 
 // Shape of the GEMM launch: CTA pairs or single CTAs, and the output channels per tile (UMMA N, a
@@ -254,7 +291,7 @@ GemmShape choose_gemm_shape(int K, int C, long long p_tiles128, int a2, int sms)
             const double main = cblocks * (mma > load ? mma : load);
             const double epi = 300.0 + 14.0 * n;
             const double per_tile = (main > epi ? main : epi) + 200.0;
-            const double cost = waves * per_tile + epi;
+            const double cost = (waves * per_tile + epi) * (ctas == 2 ? 1.05 : 1.0);  // pairs must win clearly
             if (cost < best_cost) { best_cost = cost; best = GemmShape{ctas, n}; }
         }
     }
@@ -275,20 +312,11 @@ int launch_gemm_shape(const CUtensorMap& tmU, const CUtensorMap& tmV, const CUte
     const long long tiles = static_cast<long long>(prm.num_k_tiles) * prm.num_p_tiles * prm.num_pos;
     const long long workers = sms / CTAS;
     const int grid = static_cast<int>(tiles < workers ? tiles : workers) * CTAS;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(GEMM_THREADS);
-    cfg.dynamicSmemBytes = L::dyn_bytes(prm.n_tile / CTAS, prm.stages, prm.epi_rows, prm.epi_bufs);
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = CTAS;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
     ProfScope prof(KIND_GEMM, st);
-    cudaError_t e = cudaLaunchKernelEx(&cfg, wino_gemm_kernel<CTAS>, tmU, tmV, tmM, prm, status);
+    const cudaError_t e =
+        launch_pdl(wino_gemm_kernel<CTAS>, dim3(grid), dim3(GEMM_THREADS),
+                   static_cast<size_t>(L::dyn_bytes(prm.n_tile / CTAS, prm.stages, prm.epi_rows, prm.epi_bufs)), st, CTAS,
+                   tmU, tmV, tmM, prm, status);
     g_launches.fetch_add(1);
     return e == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
 }

@@ -12,6 +12,8 @@
 #include <cuda_fp16.h>
 #include <stdint.h>
 
+#include "ptx.cuh"
+
 namespace sdw {
 
 template <int M> struct Wino;
@@ -100,6 +102,8 @@ __global__ void __launch_bounds__(128)
 filter_transform_kernel(const __half* __restrict__ w, __half* __restrict__ U, int K, int C, int C8) {
     using Wm = Wino<M>;
     constexpr int A = Wm::A;
+    pdl_launch_dependents();
+    pdl_wait();
     const int c = blockIdx.x * blockDim.x + threadIdx.x;
     const int k = blockIdx.y;
     if (c >= C8) return;
@@ -150,6 +154,8 @@ input_transform_kernel(const __half* __restrict__ x, __half* __restrict__ V, Til
                        int p_count, long long Pstride) {
     using Wm = Wino<M>;
     constexpr int A = Wm::A;
+    pdl_launch_dependents();
+    pdl_wait();
     const int pl = blockIdx.x * blockDim.x + threadIdx.x;  // chunk-local tile
     const int c = blockIdx.y;
     if (pl >= p_count) return;
@@ -207,6 +213,8 @@ output_transform_kernel(const __half* __restrict__ Mws, const __half* __restrict
                         TileGeom geo, int K, long long p_begin, int p_count, long long Pstride) {
     using Wm = Wino<M>;
     constexpr int A = Wm::A;
+    pdl_launch_dependents();
+    pdl_wait();
     const int pl = blockIdx.x * blockDim.x + threadIdx.x;
     const int k = blockIdx.y;
     if (pl >= p_count) return;
@@ -286,6 +294,8 @@ input_transform_vec_kernel(const __half* __restrict__ x, __half* __restrict__ V,
                            long long p_begin, int p_count, long long Pstride) {
     using Wm = Wino<M>;
     constexpr int A = Wm::A;
+    pdl_launch_dependents();
+    pdl_wait();
     static_assert(M * TPT == 8, "one 16-byte row segment per thread");
     const int pl = (blockIdx.x * blockDim.x + threadIdx.x) * TPT;  // first chunk-local tile of this thread
     const int c = blockIdx.y;
@@ -368,6 +378,8 @@ output_transform_vec_kernel(const __half* __restrict__ Mws, const __half* __rest
                             TileGeom geo, int K, long long p_begin, int p_count, long long Pstride) {
     using Wm = Wino<M>;
     constexpr int A = Wm::A;
+    pdl_launch_dependents();
+    pdl_wait();
     static_assert(M * TPT == 8, "one 16-byte row segment per thread");
     const int pl = (blockIdx.x * blockDim.x + threadIdx.x) * TPT;
     const int k = blockIdx.y;

@@ -125,6 +125,7 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
         if constexpr (CTAS == 2) { tmem_alloc_pair(tmem_base_slot, TMEM_COLS); tmem_relinquish_pair(); }
         else { tmem_alloc(tmem_base_slot, TMEM_COLS); tmem_relinquish(); }
     }
+    pdl_launch_dependents();
     tc_fence_before_sync();
     __syncthreads();
     if constexpr (CTAS == 2) cluster_sync_all();   // the peer's barriers are initialised before anyone signals them
@@ -141,6 +142,7 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
             const uint32_t full0_local = smem_u32(&full_bar[0]);
             const uint32_t full0 = CTAS == 2 ? map_to_cta(full0_local, 0) : full0_local;
             uint32_t sa = smem_base, fb = full0, fb_local = full0_local;
+            pdl_wait();   // V is written by the preceding kernel
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
@@ -186,7 +188,10 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
             const uint64_t bdesc0 = make_smem_desc_sw128(smem_base + L::A_BYTES, 16, 1024);
             const uint64_t stage_step = static_cast<uint64_t>(stage_bytes >> 4);
             uint64_t adesc = adesc0, bdesc = bdesc0;
+            const uint32_t full0_a = smem_u32(&full_bar[0]), empty0_a = smem_u32(&empty_bar[0]);
+            uint32_t full_a = full0_a, empty_a = empty0_a;
             const int last_ksteps = ((prm.C - (prm.num_c_blocks - 1) * GEMM_BLOCK_C) + 15) / 16;  // 1..4
+            const int full_blocks = last_ksteps == 4 ? prm.num_c_blocks : prm.num_c_blocks - 1;
             int stage = 0;
             uint32_t phase = 0;
             int buf = 0;
@@ -198,17 +203,19 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(buf * GEMM_MAX_N);
                 for (int cb = 0; cb < prm.num_c_blocks; ++cb) {
-                    ok = mbar_wait_bounded(&full_bar[stage], phase, abort_flag, GEMM_WAIT_LIMIT_NS);
-                    if (!ok) { if (*abort_flag == 0) report_timeout(status_word, 3, cta_rank); break; }
+                    if (!mbar_try_wait_a32(full_a, phase)) {
+                        ok = mbar_wait_slow(&full_bar[stage], phase, abort_flag, GEMM_WAIT_LIMIT_NS);
+                        if (!ok) { if (*abort_flag == 0) report_timeout(status_word, 3, cta_rank); break; }
+                    }
                     tc_fence_after_sync();
-                    if (cb + 1 < prm.num_c_blocks || last_ksteps == 4) {
+                    if (cb < full_blocks) {
                         if constexpr (CTAS == 2) {
-                            umma_f16_pair(d_tmem, adesc, bdesc, idesc, cb > 0 ? 1u : 0u);
+                            umma_f16_pair(d_tmem, adesc, bdesc, idesc, static_cast<uint32_t>(cb));
                             umma_f16_pair_acc(d_tmem, adesc + 128, bdesc + 2, idesc);
                             umma_f16_pair_acc(d_tmem, adesc + 256, bdesc + 4, idesc);
                             umma_f16_pair_acc(d_tmem, adesc + 384, bdesc + 6, idesc);
                         } else {
-                            umma_f16(d_tmem, adesc, bdesc, idesc, cb > 0 ? 1u : 0u);
+                            umma_f16(d_tmem, adesc, bdesc, idesc, static_cast<uint32_t>(cb));
                             umma_f16_acc(d_tmem, adesc + 128, bdesc + 2, idesc);
                             umma_f16_acc(d_tmem, adesc + 256, bdesc + 4, idesc);
                             umma_f16_acc(d_tmem, adesc + 384, bdesc + 6, idesc);
@@ -221,11 +228,15 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
                                 umma_f16(d_tmem, adesc + 128 * s, bdesc + 2 * s, idesc, (cb > 0 || s > 0) ? 1u : 0u);
                         }
                     }
-                    if constexpr (CTAS == 2) umma_commit_pair(&empty_bar[stage]);
-                    else umma_commit(&empty_bar[stage]);
+                    if constexpr (CTAS == 2) umma_commit_pair_a32(empty_a);
+                    else umma_commit_a32(empty_a);
                     adesc += stage_step;
                     bdesc += stage_step;
-                    if (++stage == stages) { stage = 0; phase ^= 1u; adesc = adesc0; bdesc = bdesc0; }
+                    full_a += 8;
+                    empty_a += 8;
+                    if (++stage == stages) {
+                        stage = 0; phase ^= 1u; adesc = adesc0; bdesc = bdesc0; full_a = full0_a; empty_a = empty0_a;
+                    }
                 }
                 if (!ok) break;
                 if constexpr (CTAS == 2) umma_commit_pair(&acc_full_bar[buf]);
@@ -238,6 +249,7 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
     } else {
         // ------------------------------ epilogue ------------------------------
         const int quarter = warp & 3;          // TMEM lanes this warp may read: 32*quarter .. +31
+        pdl_wait();   // nothing is written to global memory before the predecessor has completed
         const int group = (warp - 2) >> 2;           // 0: warps 2-5, 1: warps 6-9
         const int group_tid = threadIdx.x - 64 - group * 128;
         int buf = 0;
