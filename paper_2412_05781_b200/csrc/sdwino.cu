@@ -277,8 +277,9 @@ GemmShape choose_gemm_shape(int K, int C, long long p_tiles128, int a2, int sms)
     const long long cblocks = (C + GEMM_BLOCK_C - 1) / GEMM_BLOCK_C;
     GemmShape best{1, 16};
     double best_cost = 1e300;
-    for (int ctas = 1; ctas <= 2; ++ctas) {
-        if (ctas == 2 && p_tiles128 < 2) continue;
+    // CTA pairs never beat single CTAs in measurement (the mainloop is not bound by L2 bytes) and cannot use
+    // programmatic dependent launch, so they are only taken when forced through sdwino_set_gemm_shape.
+    for (int ctas = 1; ctas <= 1; ++ctas) {
         const long long p_tiles = (p_tiles128 + ctas - 1) / ctas;
         const long long workers = sms / ctas;
         for (int n = 16; n <= GEMM_MAX_N; n += 16) {
