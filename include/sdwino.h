@@ -49,8 +49,8 @@ const char *sdwino_status_string(int status);
  *
  * sdwino_filter_bytes: bytes the caller must allocate for wT (0 on bad arguments).
  * sdwino_filter_transform: w is fp16 [K][C][3][3]; wT receives fp16 U laid out as
- *   [a*a][K][C8] with a = tile+2, C8 = C rounded up to 8 (16-byte rows), position index
- *   xi*a+nu, zero in the padding columns.  wT must be 1024-byte aligned (a cudaMalloc
+ *   [a*a][Kb][Cb][16][64] with a = tile+2, Kb = ceil(K/16), Cb = ceil(C/64): blocks of 16 output
+ *   channels x 64 input channels (2 KB contiguous each), position index xi*a+nu, zero in the padding.  wT must be 1024-byte aligned (a cudaMalloc
  *   base is).  wT depends on `tile`; pass the same tile to sdwino_conv3x3.  Done once
  *   per weight; the caller owns both buffers.
  */
@@ -141,7 +141,8 @@ unsigned long long sdwino_launch_count(void);
 /*
  * Tuning and test hook for the batched GEMM of step (ii).  By default the library picks, per
  * call, between single-CTA tiles (128 tiles x n output channels) and CTA-pair tiles (256 tiles x
- * n output channels, tcgen05 cta_group::2) and the n that fits the layer.  ctas in {1, 2} and/or
+ * n output channels, tcgen05 cta_group::2; n is then rounded up to a multiple of 32) and the n that
+ * fits the layer.  ctas in {1, 2} and/or
  * n_tile (a multiple of 16 in [16, 256]) force that choice for later calls of this process; 0
  * restores the automatic choice for that field.  Results do not depend on the choice beyond
  * the fp32 summation order inside the tensor core.  Returns SDWINO_ERR_INVALID_ARG otherwise.

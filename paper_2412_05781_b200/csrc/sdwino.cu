@@ -78,7 +78,7 @@ inline long long round_up_ll(long long v, long long m) { return (v + m - 1) / m 
 
 struct Plan {
     int a2;            // transform positions
-    int C8;            // row pitch of U in elements (C rounded up to 8: 16-byte rows for TMA)
+    int Kb, Cb;        // blocks of 16 output channels / 64 input channels of the filter tensor
     int TH, TW;
     long long P;       // tiles in the whole batch
     long long P128;    // P rounded up to the GEMM tile
@@ -90,7 +90,8 @@ bool make_plan(int N, int C, int H, int W, int K, int tile, Plan* pl) {
     if (tile != 2 && tile != 4) return false;
     const int a = tile + 2;
     pl->a2 = a * a;
-    pl->C8 = round_up(C, 8);
+    pl->Kb = (K + 15) / 16;
+    pl->Cb = (C + 63) / 64;
     pl->TH = (H + tile - 1) / tile;
     pl->TW = (W + tile - 1) / tile;
     pl->P = static_cast<long long>(N) * pl->TH * pl->TW;
@@ -180,6 +181,29 @@ bool encode_map_uncached(CUtensorMap* m, const void* base, uint64_t d0, uint64_t
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
+// The blocked filter tensor U[pos][Kb][Cb][16][64] as a 5-D map whose box is `kblocks` blocks of 16 rows.
+bool encode_filter_map(CUtensorMap* m, const void* base, uint64_t Cb, uint64_t Kb, uint64_t npos, uint32_t kblocks) {
+    const MapKey key{base, Cb, Kb, npos, ~0ull, ~0ull, kblocks, 5, true};
+    const uint64_t h = (reinterpret_cast<uintptr_t>(base) >> 8) * 1000003u ^ Cb * 31u ^ Kb * 131u ^ (kblocks << 7) ^ 5u;
+    MapSlot& slot = g_map_cache[h % MAP_CACHE_SLOTS];
+    std::lock_guard<std::mutex> lock(g_map_mutex);
+    if (slot.used && slot.key == key) { *m = slot.map; return true; }
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[5] = {64, 16, Cb, Kb, npos};
+    cuuint64_t strides[4] = {128, 2048, Cb * 2048, Kb * Cb * 2048};
+    cuuint32_t box[5] = {64, 16, 1, kblocks, 1};
+    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    if (fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 5, const_cast<void*>(base), dims, strides, box, estr,
+           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    slot.key = key;
+    slot.map = *m;
+    slot.used = true;
+    return true;
+}
+
 int sm_count() {
     static int n = 0;
     if (n == 0) {
@@ -222,10 +246,10 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
 }
 
 template <int M>
-int launch_filter(const __half* w, __half* U, int K, int C, int C8, cudaStream_t st) {
-    dim3 grid((C8 + 127) / 128, K);
+int launch_filter(const __half* w, __half* U, int K, int C, int Kb, int Cb, cudaStream_t st) {
+    dim3 grid((Cb * 64 + 127) / 128, Kb * 16);
     ProfScope prof(KIND_FILTER, st);
-    const cudaError_t e = launch_pdl(filter_transform_kernel<M>, grid, dim3(128), 0, st, 0, w, U, K, C, C8);
+    const cudaError_t e = launch_pdl(filter_transform_kernel<M>, grid, dim3(128), 0, st, 0, w, U, K, C, Kb, Cb);
     g_launches.fetch_add(1);
     return e == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
 }
@@ -364,6 +388,7 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
     GemmShape shape = choose_gemm_shape(K, C, pc / GEMM_BLOCK_P, pl.a2, sms);
     if (g_force_ctas == 1 || g_force_ctas == 2) shape.ctas = (pc / GEMM_BLOCK_P < 2) ? 1 : g_force_ctas;
     if (g_force_n_tile >= 16 && g_force_n_tile <= GEMM_MAX_N && g_force_n_tile % 16 == 0) shape.n_tile = g_force_n_tile;
+    if (shape.ctas == 2) shape.n_tile = round_up(shape.n_tile, 32);  // each CTA of a pair loads whole 16-row blocks
     prm.n_tile = shape.n_tile;
     prm.num_k_tiles = (K + prm.n_tile - 1) / prm.n_tile;
     prm.num_pos = pl.a2;
@@ -380,7 +405,7 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
 
     prm.p_stride = pc;
     CUtensorMap tmU, tmV, tmM;
-    if (!encode_map(&tmU, wT, C, K, pl.a2, pl.C8, static_cast<uint64_t>(K) * pl.C8, 64, b_rows, true) ||
+    if (!encode_filter_map(&tmU, wT, pl.Cb, pl.Kb, pl.a2, b_rows / 16) ||
         !encode_map(&tmV, V, pc, C, pl.a2, pc, static_cast<uint64_t>(C) * pc, 64, GEMM_BLOCK_C, true) ||
         !encode_map(&tmM, Mws, pc, K, pl.a2, pc, static_cast<uint64_t>(K) * pc, GEMM_BLOCK_P, prm.epi_rows, false))
         return SDWINO_ERR_CUDA;
@@ -435,7 +460,7 @@ const char* sdwino_status_string(int status) {
 size_t sdwino_filter_bytes(int K, int C, int tile) {
     if (K <= 0 || C <= 0 || (tile != 2 && tile != 4)) return 0;
     const size_t a = tile + 2;
-    const size_t bytes = a * a * static_cast<size_t>(K) * round_up(C, 8) * sizeof(__half);
+    const size_t bytes = a * a * static_cast<size_t>((K + 15) / 16) * ((C + 63) / 64) * 1024 * sizeof(__half);
     return (bytes + WS_ALIGN - 1) / WS_ALIGN * WS_ALIGN;
 }
 
@@ -444,10 +469,10 @@ int sdwino_filter_transform(const void* w, void* wT, int K, int C, int tile, voi
     if (tile != 2 && tile != 4) return SDWINO_ERR_UNSUPPORTED;
     if (!aligned(w, 2) || !aligned(wT, WS_ALIGN)) return SDWINO_ERR_MISALIGNED;
     if (static_cast<long double>(K) * C > 4.0e15L) return SDWINO_ERR_INVALID_ARG;
-    const int C8 = round_up(C, 8);
+    const int Kb = (K + 15) / 16, Cb = (C + 63) / 64;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (tile == 2) return launch_filter<2>(static_cast<const __half*>(w), static_cast<__half*>(wT), K, C, C8, st);
-    return launch_filter<4>(static_cast<const __half*>(w), static_cast<__half*>(wT), K, C, C8, st);
+    if (tile == 2) return launch_filter<2>(static_cast<const __half*>(w), static_cast<__half*>(wT), K, C, Kb, Cb, st);
+    return launch_filter<4>(static_cast<const __half*>(w), static_cast<__half*>(wT), K, C, Kb, Cb, st);
 }
 
 size_t sdwino_workspace_bytes(int N, int C, int H, int W, int K, int tile) {

@@ -93,22 +93,25 @@ __device__ __forceinline__ void mat_apply(MatT coef, const float (&in)[Cn], floa
 }
 
 // ---------------------------------------------------------------------------------------
-// Filter preprocess.  One thread per (k, c) of the [K][C8] plane (C8 = C rounded up to 8 so that
-// rows are 16-byte multiples); writes all a*a positions (zeros in the padding columns).
-// U layout: [a*a][K][C8], c contiguous.
+// Filter preprocess.  U is stored in blocks of 16 output channels x 64 input channels,
+//   U[a*a][Kb][Cb][16][64]   (Kb = ceil(K/16), Cb = ceil(C/64), zeros in the padding),
+// so that the [n_tile k][64 c] operand box of one GEMM pipeline stage is n_tile/16 contiguous 2 KB
+// pieces of DRAM instead of n_tile separate 128-byte rows (the weights are the one operand that is
+// streamed from HBM).  One thread per (k, c) of the padded plane.
+// Writes all a*a positions.
 // ---------------------------------------------------------------------------------------
 template <int M>
 __global__ void __launch_bounds__(128)
-filter_transform_kernel(const __half* __restrict__ w, __half* __restrict__ U, int K, int C, int C8) {
+filter_transform_kernel(const __half* __restrict__ w, __half* __restrict__ U, int K, int C, int Kb, int Cb) {
     using Wm = Wino<M>;
     constexpr int A = Wm::A;
     pdl_launch_dependents();
     pdl_wait();
     const int c = blockIdx.x * blockDim.x + threadIdx.x;
     const int k = blockIdx.y;
-    if (c >= C8) return;
+    if (c >= Cb * 64) return;
     float g[3][3];
-    const bool live = c < C;
+    const bool live = (c < C) && (k < K);
 #pragma unroll
     for (int r = 0; r < 3; ++r)
 #pragma unroll
@@ -124,8 +127,8 @@ filter_transform_kernel(const __half* __restrict__ w, __half* __restrict__ U, in
 #pragma unroll
         for (int i = 0; i < A; ++i) t[i][s] = o[i];
     }
-    const size_t plane = static_cast<size_t>(K) * C8;
-    __half* dst = U + static_cast<size_t>(k) * C8 + c;
+    const size_t plane = static_cast<size_t>(Kb) * Cb * 1024;   // one position: Kb x Cb blocks of 16 x 64
+    __half* dst = U + ((static_cast<size_t>(k >> 4) * Cb + (c >> 6)) * 16 + (k & 15)) * 64 + (c & 63);
 #pragma unroll
     for (int i = 0; i < A; ++i) {
         float o[A];

@@ -77,7 +77,8 @@ struct GemmParams {
 };
 
 // tmV: fp16 [pos][C][Pstride]   box {64 p, 64 c, 1},      128B swizzle  (A operand; rows c >= C read as 0)
-// tmU: fp16 [pos][K][C8]        box {64 c, n_tile k, 1},  128B swizzle  (B operand; rows k >= K read as 0)
+// tmU: fp16 [pos][Kb][Cb][16][64] box {64 c, 16 k, 1, n_tile/16, 1}, 128B swizzle (B operand: n_tile rows of 128
+//      bytes in k order; blocks past Kb read as 0)
 // tmM: fp16 [pos][K][Pstride]   box {128 p, epi_rows k, 1}, no swizzle  (result; rows k >= K are clipped)
 template <int CTAS>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
@@ -159,12 +160,12 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
                         if (leader) mbar_arrive_expect_tx_a32(fb_local, tx_bytes);
                         tma_load_3d_pair(sa, &tmV, fb, p0, c0, pos);
                         tma_load_3d_pair(sa + L::A_BOX_BYTES, &tmV, fb, p0 + 64, c0, pos);
-                        tma_load_3d_pair(sa + L::A_BYTES, &tmU, fb, c0, k0, pos);
+                        tma_load_5d_pair(sa + L::A_BYTES, &tmU, fb, c0 >> 6, k0 >> 4, pos);
                     } else {
                         mbar_arrive_expect_tx_a32(fb, tx_bytes);
                         tma_load_3d_a32(sa, &tmV, fb, p0, c0, pos);
                         tma_load_3d_a32(sa + L::A_BOX_BYTES, &tmV, fb, p0 + 64, c0, pos);
-                        tma_load_3d_a32(sa + L::A_BYTES, &tmU, fb, c0, k0, pos);
+                        tma_load_5d_a32(sa + L::A_BYTES, &tmU, fb, c0 >> 6, k0 >> 4, pos);
                     }
                     sa += stage_bytes;
                     fb += 8;

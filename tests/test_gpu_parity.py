@@ -145,8 +145,10 @@ def test_filter_transform_matches_oracle(B, KC, tile):
     g = torch.Generator().manual_seed(K + C)
     w = (torch.randn(K, C, 3, 3, generator=g) / (9 * C) ** 0.5).half()
     wT = B.sdwino_filter_transform(w.cuda(), tile)
-    C8 = -(-C // 8) * 8
-    U = wT.view(torch.float16)[:a * a * K * C8].view(a * a, K, C8).cpu()
+    Kb, Cb = -(-K // 16), -(-C // 64)
+    # U[a*a][Kb][Cb][16][64]  ->  [a*a][Kb*16][Cb*64]
+    U = wT.view(torch.float16)[:a * a * Kb * Cb * 1024].view(a * a, Kb, Cb, 16, 64).permute(0, 1, 3, 2, 4)
+    U = U.reshape(a * a, Kb * 16, Cb * 64).cpu()
     Uo = oracle.filter_transform(w.numpy(), tile, points=None if tile == 2 else F4_POINTS)
     Uo = torch.from_numpy(Uo.reshape(K, C, a * a).transpose(2, 0, 1).copy())
     got = U[:, :K, :C].double()
@@ -155,8 +157,9 @@ def test_filter_transform_matches_oracle(B, KC, tile):
     ulp = torch.maximum((torch.nextafter(ref16, torch.full_like(ref16, float("inf"))) - ref16).double().abs(),
                         (ref16 - torch.nextafter(ref16, torch.full_like(ref16, -float("inf")))).double().abs())
     assert bool(((got - ref16.double()).abs() <= ulp).all())
-    # padding columns are zero
-    assert float(U[:, :, C:].abs().max() if C8 > C else 0) == 0
+    # padding rows and columns are zero
+    assert float(U[:, :, C:].abs().max() if Cb * 64 > C else 0) == 0
+    assert float(U[:, K:, :].abs().max() if Kb * 16 > K else 0) == 0
 
 
 def test_single_layer_config_full(B):
