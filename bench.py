@@ -30,6 +30,10 @@ UNIT = "TFLOP/s"
 WORKLOAD = "sd15_unet"
 TILE = 2
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# dram__bytes_read.sum + dram__bytes_write.sum of the 17 GEMM launches of one SD v1.5 step, from one ncu
+# capture (profiles/launch_list_sd15_unet_sweep.md): 691.3 MB, i.e. 40.7 MB per launch.  Only valid for the
+# default workload with all layers.
+GEMM_DRAM_BYTES_PER_LAUNCH_SD15 = 40.66e6
 PAPER_CONTEXT = {"per_layer_speedup_vs_sdcpp_m1pro": 2.76, "end_to_end_speedup_vs_sdcpp_m1pro": 4.79}
 
 
@@ -96,6 +100,22 @@ class ClockSampler:
         loaded = [m for m, u in self.samples if u > 0] or [m for m, _ in self.samples]
         return {"sm_mhz": int(statistics.median(loaded)), "sm_max_mhz": self.max_mhz,
                 "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def max_over_ranks(value: float, dist=None, device=None) -> float:
+    """The slowest rank's figure: every multi-GPU number is the max over ranks of a device-side time."""
+    if dist is None:
+        return float(value)
+    import torch
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_value(flops_per_replica: float, world: int, ms_per_step: float) -> float:
+    """Whole-job throughput in TFLOP/s of `world` independent replicas that each do
+    `flops_per_replica` per step, the step taking `ms_per_step` on the slowest rank."""
+    return world * flops_per_replica / (ms_per_step * 1e-3) / 1e12
 
 
 def visible_to_nvml_index(local_rank: int) -> int:
@@ -278,14 +298,11 @@ def run_ours(args):
     barrier()
     launches = launches_per_step * args.steps
     ms_total = e0.elapsed_time(e1)
-    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_step = float(t.item()) / args.steps
+    ms_step = max_over_ranks(ms_total, dist, dev) / args.steps
     assert B.sdwino_last_device_status(stream) == B.OK, "a device-side wait timed out"
 
     flops_step = sum(L.direct_flops for L in layers)
-    value = world * flops_step / (ms_step * 1e-3) / 1e12
+    value = aggregate_value(flops_step, world, ms_step)
 
     # ---- end to end: host buffers in, host buffers out, through sdwino_conv3x3_host ----
     e2e_steps = max(3, min(args.steps, 30))
@@ -302,10 +319,7 @@ def run_ours(args):
         e2e_step()
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
-    te = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(te, op=dist.ReduceOp.MAX)
-    e2e_value = world * flops_step / (float(te.item()) / e2e_steps) / 1e12
+    e2e_value = aggregate_value(flops_step, world, max_over_ranks(e2e_s, dist, dev) / e2e_steps * 1e3)
     h2d = sum(x.numel() * 2 + b.numel() * 2 for (x, w, b, y) in host)
     d2h = sum(y.numel() * 2 for (x, w, b, y) in host)
 
@@ -319,7 +333,8 @@ def run_ours(args):
             B.sdwino_conv3x3(xd, wT, bd, L.K, TILE, y=yd, workspace=ws, stream=stream)
             records_per_layer.append(len(B.sdwino_profile_records()))
     prof_steps = max(3, min(args.steps, 20))
-    per_layer = [dict(input_transform=0.0, wino_gemm=0.0, output_transform=0.0, launches=0) for _ in layers]
+    per_layer = [dict(input_transform=0.0, wino_gemm=0.0, output_transform=0.0, fused_small_c=0.0, launches=0)
+                 for _ in layers]
 
     def account(recs):
         assert len(recs) == sum(records_per_layer) and all(ms >= 0 for _, ms in recs)
@@ -359,6 +374,7 @@ def run_ours(args):
     gemm_flops = gemm_ms = 0.0
     in_ms = out_ms = 0.0
     in_bytes = out_bytes = 0.0
+    fused_ms = 0.0
     for L, pl in zip(layers, per_layer):
         P = L.tiles(TILE)
         wino_flops = 2.0 * a2 * L.K * L.C * P
@@ -366,32 +382,38 @@ def run_ours(args):
         xb, yb = 2.0 * L.N * L.C * L.H * L.W, 2.0 * L.N * L.K * L.H * L.W
         t_tensor = wino_flops / (tpeak * 1e12) * 1e6
         t_hbm = (xb + 2.0 * a2 * L.K * L.C + yb + 2 * L.K) / (hpeak * 1e9) * 1e6
-        total_us = (pl["input_transform"] + pl["wino_gemm"] + pl["output_transform"]) * 1e3
+        total_us = (pl["input_transform"] + pl["wino_gemm"] + pl["output_transform"] + pl["fused_small_c"]) * 1e3
         layer_rows.append({
             "layer": L.name, "us": round(total_us, 2),
             "us_input": round(pl["input_transform"] * 1e3, 2), "us_gemm": round(pl["wino_gemm"] * 1e3, 2),
-            "us_output": round(pl["output_transform"] * 1e3, 2),
+            "us_output": round(pl["output_transform"] * 1e3, 2), "us_fused": round(pl["fused_small_c"] * 1e3, 2),
             "eq_tflops": round(L.direct_flops / (total_us * 1e-6) / 1e12, 1),
             "bound": "tensor" if t_tensor >= t_hbm else "hbm",
             "roof_us": round(max(t_tensor, t_hbm), 2),
             "frac_of_roof": round(max(t_tensor, t_hbm) / total_us, 3),
-            "gemm_tensor_frac": round(wino_flops / (pl["wino_gemm"] * 1e-3) / 1e12 / tpeak, 3),
+            "gemm_tensor_frac": (round(wino_flops / (pl["wino_gemm"] * 1e-3) / 1e12 / tpeak, 3)
+                                 if pl["wino_gemm"] > 0 else None),
         })
-        gemm_flops += wino_flops
-        gemm_ms += pl["wino_gemm"]
-        in_ms += pl["input_transform"]
-        out_ms += pl["output_transform"]
-        in_bytes += xb + 2.0 * a2 * L.C * P      # read x, write V
-        out_bytes += 2.0 * a2 * L.K * P + yb     # read M, write y
+        if pl["wino_gemm"] > 0:                  # layers on the fused few-channel kernel have no GEMM launch
+            gemm_flops += wino_flops
+            gemm_ms += pl["wino_gemm"]
+            in_ms += pl["input_transform"]
+            out_ms += pl["output_transform"]
+            in_bytes += xb + 2.0 * a2 * L.C * P      # read x, write V
+            out_bytes += 2.0 * a2 * L.K * P + yb     # read M, write y
+        fused_ms += pl["fused_small_c"]
     gemm_launches = sum(pl["launches"] for pl in per_layer) / prof_steps
     achieved = gemm_flops / (gemm_ms * 1e-3) / 1e12
     roofline = {
         "kernel": "wino_gemm_kernel", "bound": "tensor", "achieved": round(achieved, 1), "peak": tpeak,
-        "unit": "TFLOP/s", "frac": round(achieved / tpeak, 4), "traffic": None,
+        "unit": "TFLOP/s", "frac": round(achieved / tpeak, 4),
+        "traffic": (GEMM_DRAM_BYTES_PER_LAUNCH_SD15 if (args.workload == WORKLOAD and not args.layers and TILE == 2)
+                    else None),
+        "traffic_unit": "bytes per launch (ncu dram read + write, L2 left warm)",
         "peak_source": f"{peak_kind} (cuBLAS bf16 burst; fp16 has the same nominal rate)",
         "launches_per_step": gemm_launches, "avg_launch_us": round(gemm_ms * 1e3 / gemm_launches, 2),
         "algorithmic_flops_per_step": gemm_flops,
-        "share_of_step": round(gemm_ms / (gemm_ms + in_ms + out_ms), 3),
+        "share_of_step": round(gemm_ms / (gemm_ms + in_ms + out_ms + fused_ms), 3),
     }
     transforms = {
         "input_transform": {"gbs": round(in_bytes / (in_ms * 1e-3) / 1e9, 1), "frac_of_hbm_peak":

@@ -154,8 +154,9 @@ int sdwino_set_gemm_shape(int ctas, int n_tile);
  * bracketed by two CUDA events recorded on the launch's stream (this adds a little idle time
  * between kernels, so whole-call timings should be taken with profiling disabled).
  * sdwino_profile_collect waits for the recorded events, adds the elapsed milliseconds and
- * the launch counts per kernel kind into the two caller arrays of 4 entries (0 filter
- * transform, 1 activation transform, 2 batched GEMM, 3 output transform; either may be NULL)
+ * the launch counts per kernel kind into the two caller arrays of 5 entries (0 filter
+ * transform, 1 activation transform, 2 batched GEMM, 3 output transform, 4 the fused
+ * few-input-channel kernel; either may be NULL)
  * and forgets the records.  Host arrays; not thread-safe against concurrent compute calls.
  */
 int sdwino_profile_enable(int enable);

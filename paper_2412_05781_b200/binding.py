@@ -24,7 +24,7 @@ EXPORTS = [
     "sdwino_profile_records", "sdwino_set_gemm_shape", "sdwino_conv3x3_static",
 ]
 
-KERNEL_KINDS = ("filter_transform", "input_transform", "wino_gemm", "output_transform")
+KERNEL_KINDS = ("filter_transform", "input_transform", "wino_gemm", "output_transform", "fused_small_c")
 
 
 class SdwinoError(RuntimeError):
@@ -134,8 +134,8 @@ def sdwino_profile_enable(enable: bool) -> None:
 
 def sdwino_profile_collect():
     """-> {kernel kind: (total milliseconds, launches)} since the last collect."""
-    ms = (ctypes.c_double * 4)()
-    n = (ctypes.c_ulonglong * 4)()
+    ms = (ctypes.c_double * 5)()
+    n = (ctypes.c_ulonglong * 5)()
     _check(lib.sdwino_profile_collect(ms, n), "sdwino_profile_collect")
     return {k: (float(ms[i]), int(n[i])) for i, k in enumerate(KERNEL_KINDS)}
 

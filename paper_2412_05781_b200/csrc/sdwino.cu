@@ -27,12 +27,13 @@ std::atomic<unsigned long long> g_launches{0};
 std::mutex g_mutex;
 // test / tuning overrides of the GEMM launch shape (0 = choose automatically)
 int g_force_ctas = 0;
+bool g_disable_fused = false;  // forcing a GEMM shape also forces the GEMM path for few-channel layers
 int g_force_n_tile = 0;
 void* g_workspace = nullptr;
 size_t g_workspace_bytes = 0;
 
 // Optional per-kernel timing: when enabled every launch is bracketed by CUDA events on its stream.
-enum KernelKind { KIND_FILTER = 0, KIND_INPUT = 1, KIND_GEMM = 2, KIND_OUTPUT = 3, KIND_COUNT = 4 };
+enum KernelKind { KIND_FILTER = 0, KIND_INPUT = 1, KIND_GEMM = 2, KIND_OUTPUT = 3, KIND_FUSED = 4, KIND_COUNT = 5 };
 struct ProfRecord { int kind; cudaEvent_t beg, end; };
 bool g_profile = false;
 std::vector<ProfRecord> g_prof_records;
@@ -291,6 +292,20 @@ int launch_output(const __half* Mws, const __half* bias, __half* y, const TileGe
     return e == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
 }
 
+// Layers with at most 8 (tile 2) or 4 (tile 4) input channels run as one fused kernel without a workspace.
+bool use_fused_small_c(int C, int tile) { return tile == 2 ? C <= 8 : C <= 4; }
+
+template <int M, int CP>
+int launch_fused_small_c(const __half* x, const __half* U, const __half* bias, __half* y, const TileGeom& geo, int C,
+                         int K, int Kb, int Cb, cudaStream_t st) {
+    dim3 grid(static_cast<unsigned>((geo.P + 127) / 128), (K + FUSED_KC - 1) / FUSED_KC);
+    ProfScope prof(KIND_FUSED, st);
+    const cudaError_t e = launch_pdl(fused_small_c_kernel<M, CP>, grid, dim3(128), 0, st, 0, x, U, bias, y, geo, C, K,
+                                     Kb, Cb);
+    g_launches.fetch_add(1);
+    return e == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
+}
+
 // Shape of the GEMM launch: CTA pairs or single CTAs, and the output channels per tile (UMMA N, a
 // multiple of 16 up to 256).  The candidate with the smallest modelled time wins: a tile costs its
 // pipeline stages, each limited by the tensor pipe (2 n cycles per stage) or by the bytes the CTA must
@@ -372,6 +387,16 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
     if (!aligned(ws, WS_ALIGN)) return SDWINO_ERR_MISALIGNED;
     const long long pc = tiles_per_pass(pl, ws_bytes);
     if (pc < GEMM_BLOCK_P) return SDWINO_ERR_WORKSPACE;
+    if (use_fused_small_c(C, tile) && !g_disable_fused) {
+        TileGeom geo{H, W, pl.TH, pl.TW, pl.P};
+        const __half* xh = static_cast<const __half*>(x);
+        const __half* uh = static_cast<const __half*>(wT);
+        const __half* bh = static_cast<const __half*>(bias);
+        __half* yh = static_cast<__half*>(y);
+        if (tile == 4) return launch_fused_small_c<4, 4>(xh, uh, bh, yh, geo, C, K, pl.Kb, pl.Cb, st);
+        if (C <= 4) return launch_fused_small_c<2, 4>(xh, uh, bh, yh, geo, C, K, pl.Kb, pl.Cb, st);
+        return launch_fused_small_c<2, 8>(xh, uh, bh, yh, geo, C, K, pl.Kb, pl.Cb, st);
+    }
 
     // workspace: V[a2][C][pc] then M[a2][K][pc]; pc is a multiple of 128 elements, so every row starts
     // on a 256-byte boundary.
@@ -441,6 +466,7 @@ int sdwino_set_gemm_shape(int ctas, int n_tile) {
     if (ctas < 0 || ctas > 2 || n_tile < 0 || n_tile > GEMM_MAX_N || n_tile % 16 != 0) return SDWINO_ERR_INVALID_ARG;
     g_force_ctas = ctas;
     g_force_n_tile = n_tile;
+    g_disable_fused = (ctas != 0 || n_tile != 0);
     return SDWINO_OK;
 }
 

@@ -445,4 +445,125 @@ output_transform_vec_kernel(const __half* __restrict__ Mws, const __half* __rest
     }
 }
 
+
+// ---------------------------------------------------------------------------------------
+// All three steps in one kernel for layers with very few input channels (the 4 -> 320 / 4 -> 512
+// input convolutions of the UNet and the VAE decoder).  With C <= 8 the contraction over channels is
+// too short for the tensor cores and V, M would only be round trips through L2: a thread owns one
+// tile, keeps V[c][a*a] in registers (fp32, not rounded), and for every output channel of the
+// block's chunk forms M = sum_c U (.) V from the filter chunk staged in shared memory, applies
+// A^T M A, adds the bias and stores.  Consecutive threads own consecutive tiles, so stores coalesce.
+// CP = channel count padded to 4 or 8; KC output channels per block.
+// ---------------------------------------------------------------------------------------
+constexpr int FUSED_KC = 8;
+
+template <int M, int CP>
+__global__ void __launch_bounds__(128)
+fused_small_c_kernel(const __half* __restrict__ x, const __half* __restrict__ U, const __half* __restrict__ bias,
+                     __half* __restrict__ y, TileGeom geo, int C, int K, int Kb, int Cb) {
+    using Wm = Wino<M>;
+    constexpr int A = Wm::A;
+    constexpr int A2 = A * A;
+    __shared__ __align__(16) float Us[FUSED_KC][CP][A2];
+    pdl_launch_dependents();
+    pdl_wait();
+    const int k0 = blockIdx.y * FUSED_KC;
+    // stage the filter chunk: U[pos][Kb][Cb][16][64], this layer has Cb == 1
+    const size_t plane = static_cast<size_t>(Kb) * Cb * 1024;
+    for (int i = threadIdx.x; i < FUSED_KC * CP * A2; i += blockDim.x) {
+        const int pos = i % A2;
+        const int c = (i / A2) % CP;
+        const int kk = i / (A2 * CP);
+        const int k = k0 + kk;
+        float v = 0.f;
+        if (k < K && c < C)
+            v = __half2float(U[pos * plane + (static_cast<size_t>(k >> 4) * Cb * 16 + (k & 15)) * 64 + c]);
+        Us[kk][c][pos] = v;
+    }
+    __syncthreads();
+    const long long p = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (p >= geo.P) return;
+    const int tw = static_cast<int>(p % geo.TW);
+    const int th = static_cast<int>((p / geo.TW) % geo.TH);
+    const long long n = p / (static_cast<long long>(geo.TW) * geo.TH);
+    float v[CP][A2];
+#pragma unroll
+    for (int c = 0; c < CP; ++c) {
+        float d[A][A];
+        const __half* img = x + (n * C + (c < C ? c : 0)) * static_cast<long long>(geo.H) * geo.W;
+        const int i0 = M * th - 1, j0 = M * tw - 1;
+#pragma unroll
+        for (int r = 0; r < A; ++r) {
+            const int i = i0 + r;
+            const bool rin = (c < C) && (i >= 0) && (i < geo.H);
+#pragma unroll
+            for (int s2 = 0; s2 < A; ++s2) {
+                const int j = j0 + s2;
+                d[r][s2] = (rin && j >= 0 && j < geo.W)
+                               ? __half2float(__ldg(img + static_cast<long long>(i) * geo.W + j)) : 0.f;
+            }
+        }
+        float t[A][A];
+#pragma unroll
+        for (int s2 = 0; s2 < A; ++s2) {
+            float col[A], o[A];
+#pragma unroll
+            for (int r = 0; r < A; ++r) col[r] = d[r][s2];
+            mat_apply<A, A>(typename Wm::Bt{}, col, o);
+#pragma unroll
+            for (int r = 0; r < A; ++r) t[r][s2] = o[r];
+        }
+#pragma unroll
+        for (int r = 0; r < A; ++r) {
+            float o[A];
+            mat_apply<A, A>(typename Wm::Bt{}, t[r], o);
+#pragma unroll
+            for (int s2 = 0; s2 < A; ++s2) v[c][r * A + s2] = o[s2];
+        }
+    }
+    const int oi0 = M * th, oj0 = M * tw;
+    const bool vec_ok = ((geo.W & 1) == 0) && ((reinterpret_cast<uintptr_t>(y) & 3) == 0);
+    const int kend = (K - k0) < FUSED_KC ? (K - k0) : FUSED_KC;
+    for (int kk = 0; kk < kend; ++kk) {
+        float mm[A][A];
+#pragma unroll
+        for (int e = 0; e < A2; ++e) {
+            float acc = 0.f;
+#pragma unroll
+            for (int c = 0; c < CP; ++c) acc = fmaf(Us[kk][c][e], v[c][e], acc);
+            mm[e / A][e % A] = acc;
+        }
+        float tt[M][A];
+#pragma unroll
+        for (int s2 = 0; s2 < A; ++s2) {
+            float col[A], o[M];
+#pragma unroll
+            for (int r = 0; r < A; ++r) col[r] = mm[r][s2];
+            mat_apply<M, A>(typename Wm::At{}, col, o);
+#pragma unroll
+            for (int i = 0; i < M; ++i) tt[i][s2] = o[i];
+        }
+        const int k = k0 + kk;
+        const float b = bias ? __half2float(__ldg(bias + k)) : 0.f;
+        __half* img = y + (n * K + k) * static_cast<long long>(geo.H) * geo.W;
+#pragma unroll
+        for (int i = 0; i < M; ++i) {
+            float o[M];
+            mat_apply<M, A>(typename Wm::At{}, tt[i], o);
+            if (oi0 + i >= geo.H) continue;
+            __half* rowp = img + static_cast<long long>(oi0 + i) * geo.W + oj0;
+#pragma unroll
+            for (int j = 0; j < M; j += 2) {
+                const __half h0 = __float2half_rn(o[j] + b), h1 = __float2half_rn(o[j + 1] + b);
+                if (vec_ok && (oj0 + j + 1 < geo.W)) {
+                    *reinterpret_cast<__half2*>(rowp + j) = __halves2half2(h0, h1);
+                } else {
+                    if (oj0 + j < geo.W) rowp[j] = h0;
+                    if (oj0 + j + 1 < geo.W) rowp[j + 1] = h1;
+                }
+            }
+        }
+    }
+}
+
 }  // namespace sdw
