@@ -262,7 +262,7 @@ int launch_input(const __half* x, __half* V, const TileGeom& geo, int C, long lo
     constexpr int TPT = 8 / M;
     cudaError_t e;
     if (geo.W % 8 == 0 && aligned(x, 16)) {
-        dim3 grid((p_count / TPT + 127) / 128, C);
+        dim3 grid(static_cast<unsigned>((static_cast<long long>(p_count / TPT) * C + 127) / 128));
         e = launch_pdl(input_transform_vec_kernel<M, TPT>, grid, dim3(128), 0, st, 0, x, V, geo, C, p_begin, p_count,
                        Pstride);
     } else {
@@ -280,7 +280,7 @@ int launch_output(const __half* Mws, const __half* bias, __half* y, const TileGe
     constexpr int TPT = 8 / M;
     cudaError_t e;
     if (geo.W % 8 == 0 && aligned(y, 16)) {
-        dim3 grid((p_count / TPT + 127) / 128, K);
+        dim3 grid(static_cast<unsigned>((static_cast<long long>(p_count / TPT) * K + 127) / 128));
         e = launch_pdl(output_transform_vec_kernel<M, TPT>, grid, dim3(128), 0, st, 0, Mws, bias, y, geo, K, p_begin,
                        p_count, Pstride);
     } else {

@@ -300,9 +300,12 @@ input_transform_vec_kernel(const __half* __restrict__ x, __half* __restrict__ V,
     pdl_launch_dependents();
     pdl_wait();
     static_assert(M * TPT == 8, "one 16-byte row segment per thread");
-    const int pl = (blockIdx.x * blockDim.x + threadIdx.x) * TPT;  // first chunk-local tile of this thread
-    const int c = blockIdx.y;
-    if (pl >= p_count) return;
+    // flat index over (channel, group of TPT tiles): blocks stay full when a pass has few tiles
+    const int groups = p_count / TPT;
+    const long long idx = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    const int c = static_cast<int>(idx / groups);
+    if (c >= C) return;
+    const int pl = static_cast<int>(idx % groups) * TPT;  // first chunk-local tile of this thread
     const long long p = p_begin + pl;
     float e[A][TPT][A];  // rows transformed along the columns: e[r][t][nu] = sum_s Bt[nu][s] d[r][s]
     if (p < geo.P) {
@@ -384,9 +387,11 @@ output_transform_vec_kernel(const __half* __restrict__ Mws, const __half* __rest
     pdl_launch_dependents();
     pdl_wait();
     static_assert(M * TPT == 8, "one 16-byte row segment per thread");
-    const int pl = (blockIdx.x * blockDim.x + threadIdx.x) * TPT;
-    const int k = blockIdx.y;
-    if (pl >= p_count) return;
+    const int groups = p_count / TPT;
+    const long long idx = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    const int k = static_cast<int>(idx / groups);
+    if (k >= K) return;
+    const int pl = static_cast<int>(idx % groups) * TPT;
     const long long p = p_begin + pl;
     if (p >= geo.P) return;
     const long long plane = static_cast<long long>(K) * Pstride;
