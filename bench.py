@@ -333,7 +333,7 @@ def run_ours(args):
             B.sdwino_conv3x3(xd, wT, bd, L.K, TILE, y=yd, workspace=ws, stream=stream)
             records_per_layer.append(len(B.sdwino_profile_records()))
     prof_steps = max(3, min(args.steps, 20))
-    per_layer = [dict(input_transform=0.0, wino_gemm=0.0, output_transform=0.0, fused_small_c=0.0, launches=0)
+    per_layer = [dict(input_transform=0.0, wino_gemm=0.0, output_transform=0.0, fused=0.0, launches=0)
                  for _ in layers]
 
     def account(recs):
@@ -382,11 +382,11 @@ def run_ours(args):
         xb, yb = 2.0 * L.N * L.C * L.H * L.W, 2.0 * L.N * L.K * L.H * L.W
         t_tensor = wino_flops / (tpeak * 1e12) * 1e6
         t_hbm = (xb + 2.0 * a2 * L.K * L.C + yb + 2 * L.K) / (hpeak * 1e9) * 1e6
-        total_us = (pl["input_transform"] + pl["wino_gemm"] + pl["output_transform"] + pl["fused_small_c"]) * 1e3
+        total_us = (pl["input_transform"] + pl["wino_gemm"] + pl["output_transform"] + pl["fused"]) * 1e3
         layer_rows.append({
             "layer": L.name, "us": round(total_us, 2),
             "us_input": round(pl["input_transform"] * 1e3, 2), "us_gemm": round(pl["wino_gemm"] * 1e3, 2),
-            "us_output": round(pl["output_transform"] * 1e3, 2), "us_fused": round(pl["fused_small_c"] * 1e3, 2),
+            "us_output": round(pl["output_transform"] * 1e3, 2), "us_fused": round(pl["fused"] * 1e3, 2),
             "eq_tflops": round(L.direct_flops / (total_us * 1e-6) / 1e12, 1),
             "bound": "tensor" if t_tensor >= t_hbm else "hbm",
             "roof_us": round(max(t_tensor, t_hbm), 2),
@@ -401,7 +401,7 @@ def run_ours(args):
             out_ms += pl["output_transform"]
             in_bytes += xb + 2.0 * a2 * L.C * P      # read x, write V
             out_bytes += 2.0 * a2 * L.K * P + yb     # read M, write y
-        fused_ms += pl["fused_small_c"]
+        fused_ms += pl["fused"]
     gemm_launches = sum(pl["launches"] for pl in per_layer) / prof_steps
     achieved = gemm_flops / (gemm_ms * 1e-3) / 1e12
     roofline = {

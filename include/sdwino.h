@@ -150,13 +150,24 @@ unsigned long long sdwino_launch_count(void);
 int sdwino_set_gemm_shape(int ctas, int n_tile);
 
 /*
+ * Tuning and test knob.  F(2x2,3x3) layers with at most 8 output channels (the 320 -> 4 and 128 -> 3
+ * output convolutions) run as ONE kernel that keeps V and M on chip (input transform into shared memory,
+ * tcgen05 MMAs into TMEM, output transform from TMEM) when the batch has at least `p_tiles` blocks of 128
+ * tiles (default 48: below that too few SMs get work and the three-kernel path is faster), W % 8 == 0,
+ * x is 16-byte and y 4-byte aligned.  p_tiles = 0 restores the default; 1 sends every eligible layer
+ * through the kernel (used by the tests).  Forcing a GEMM shape with sdwino_set_gemm_shape disables it.
+ * Returns SDWINO_ERR_INVALID_ARG for a negative value.  Not thread-safe against concurrent compute calls.
+ */
+int sdwino_set_fused_min_tiles(long long p_tiles);
+
+/*
  * Per-kernel timing for benchmarks.  While enabled, every kernel launch of the library is
  * bracketed by two CUDA events recorded on the launch's stream (this adds a little idle time
  * between kernels, so whole-call timings should be taken with profiling disabled).
  * sdwino_profile_collect waits for the recorded events, adds the elapsed milliseconds and
  * the launch counts per kernel kind into the two caller arrays of 5 entries (0 filter
- * transform, 1 activation transform, 2 batched GEMM, 3 output transform, 4 the fused
- * few-input-channel kernel; either may be NULL)
+ * transform, 1 activation transform, 2 batched GEMM, 3 output transform, 4 the single-kernel
+ * paths for layers with few input or few output channels; either may be NULL)
  * and forgets the records.  Host arrays; not thread-safe against concurrent compute calls.
  */
 int sdwino_profile_enable(int enable);

@@ -21,10 +21,10 @@ EXPORTS = [
     "sdwino_workspace_bytes", "sdwino_workspace_min_bytes", "sdwino_set_workspace", "sdwino_conv3x3",
     "sdwino_conv3x3_ws", "sdwino_host_staging_bytes", "sdwino_conv3x3_host",
     "sdwino_last_device_status", "sdwino_launch_count", "sdwino_profile_enable", "sdwino_profile_collect",
-    "sdwino_profile_records", "sdwino_set_gemm_shape", "sdwino_conv3x3_static",
+    "sdwino_profile_records", "sdwino_set_gemm_shape", "sdwino_conv3x3_static", "sdwino_set_fused_min_tiles",
 ]
 
-KERNEL_KINDS = ("filter_transform", "input_transform", "wino_gemm", "output_transform", "fused_small_c")
+KERNEL_KINDS = ("filter_transform", "input_transform", "wino_gemm", "output_transform", "fused")
 
 
 class SdwinoError(RuntimeError):
@@ -67,6 +67,8 @@ def _load() -> ctypes.CDLL:
     lib.sdwino_profile_records.argtypes = [ctypes.POINTER(i), ctypes.POINTER(ctypes.c_float), i, i]
     lib.sdwino_set_gemm_shape.restype = i
     lib.sdwino_set_gemm_shape.argtypes = [i, i]
+    lib.sdwino_set_fused_min_tiles.restype = i
+    lib.sdwino_set_fused_min_tiles.argtypes = [ctypes.c_longlong]
     lib.sdwino_profile_enable.restype = i
     lib.sdwino_profile_enable.argtypes = [i]
     lib.sdwino_profile_collect.restype = i
@@ -126,6 +128,11 @@ def sdwino_last_device_status(stream: Optional[torch.cuda.Stream] = None) -> int
 def sdwino_set_gemm_shape(ctas: int = 0, n_tile: int = 0) -> None:
     """Force single-CTA (1) or CTA-pair (2) GEMM tiles and/or the channels per tile; 0 = automatic."""
     _check(lib.sdwino_set_gemm_shape(ctas, n_tile), "sdwino_set_gemm_shape")
+
+
+def sdwino_set_fused_min_tiles(p_tiles: int = 0) -> None:
+    """Blocks of 128 tiles from which few-output-channel layers take the single fused kernel; 0 = default."""
+    _check(lib.sdwino_set_fused_min_tiles(p_tiles), "sdwino_set_fused_min_tiles")
 
 
 def sdwino_profile_enable(enable: bool) -> None:

@@ -117,6 +117,15 @@ __device__ __forceinline__ void tma_load_5d_a32(uint32_t smem_dst, const CUtenso
         "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(0), "r"(c2), "r"(c3), "r"(c4)
         : "memory");
 }
+// The same with a row offset inside the 16-row block (coordinate 1): {0, k row, c-block, k-block, position}.
+__device__ __forceinline__ void tma_load_5d_k_a32(uint32_t smem_dst, const CUtensorMap* m, uint32_t bar, int c1, int c2,
+                                                  int c3, int c4) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%3, %4, %5, %6, %7}], [%2];" ::"r"(smem_dst),
+        "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+        : "memory");
+}
 __device__ __forceinline__ void mbar_arrive_expect_tx_a32(uint32_t bar, uint32_t bytes) {
     asm volatile("{\n .reg .b64 st;\n mbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n}" ::"r"(bar),
                  "r"(bytes)
@@ -172,6 +181,22 @@ __device__ __forceinline__ void tmem_ld_32x16_sync(uint32_t taddr, uint32_t (&r)
         : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
           "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
         : "r"(taddr)
+        : "memory");
+}
+
+// Four loads of 4 columns each (from four column addresses) and one wait: the accumulators of four
+// transform positions for the same 4 output channels.
+__device__ __forceinline__ void tmem_ld_4x_32x4_sync(uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                                     uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0, %1, %2, %3}, [%16];\n"
+        "tcgen05.ld.sync.aligned.32x32b.x4.b32 {%4, %5, %6, %7}, [%17];\n"
+        "tcgen05.ld.sync.aligned.32x32b.x4.b32 {%8, %9, %10, %11}, [%18];\n"
+        "tcgen05.ld.sync.aligned.32x32b.x4.b32 {%12, %13, %14, %15}, [%19];\n"
+        "tcgen05.wait::ld.sync.aligned;"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3)
         : "memory");
 }
 

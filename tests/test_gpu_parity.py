@@ -99,6 +99,83 @@ def test_forced_gemm_shapes(B, ctas, n_tile):
     assert _rel_err(y, ref) <= TOL_F2_REGRESSION
 
 
+@pytest.mark.parametrize("tile", [2, 4])
+@pytest.mark.parametrize("C,K", [(4, 40), (3, 17), (8, 8), (1, 5)])
+def test_few_input_channels_fused_kernel_matches_gemm_path(B, C, K, tile):
+    # layers with at most 8 (F2) / 4 (F4) input channels take the single fused kernel; forcing a GEMM shape
+    # sends the same layer through the three-kernel path: both must agree with the oracle and with each other
+    layer = ConvLayer(C=C, K=K, H=21, W=26, N=2)
+    x, w, b = workloads.make_inputs(layer, seed=5 + C)
+    ref = oracle.direct_conv3x3(x.numpy(), w.numpy(), b.numpy())
+    n0 = B.sdwino_launch_count()
+    _, _, _, y_auto = _run(B, layer, tile, x=x, w=w, b=b)
+    launches_auto = B.sdwino_launch_count() - n0
+    B.sdwino_set_gemm_shape(1, 16)
+    try:
+        n1 = B.sdwino_launch_count()
+        _, _, _, y_gemm = _run(B, layer, tile, x=x, w=w, b=b)
+        launches_gemm = B.sdwino_launch_count() - n1
+    finally:
+        B.sdwino_set_gemm_shape(0, 0)
+    assert _rel_err(y_auto, ref) <= TOL and _rel_err(y_gemm, ref) <= TOL
+    assert _rel_err(y_auto, y_gemm.double().numpy()) <= TOL
+    assert launches_gemm == 4                       # filter transform + three kernels of one pass
+    fused_expected = C <= (8 if tile == 2 else 4)
+    assert launches_auto == (2 if fused_expected else 4)
+
+
+FEW_K = [
+    # C, K, H, W, N: W % 8 == 0; ragged channel blocks (C % 16, C % 64), odd H, several images, more than
+    # two 64-channel filter blocks (ring instead of resident filters), a last block of tiles that is partial
+    (16, 4, 8, 8, 1), (70, 3, 10, 16, 2), (128, 3, 32, 32, 1), (130, 8, 17, 24, 2), (320, 4, 64, 64, 2),
+    (200, 7, 33, 40, 1), (300, 5, 7, 8, 3), (129, 1, 9, 48, 1), (64, 2, 130, 136, 1),
+]
+
+
+@pytest.mark.parametrize("shape", FEW_K)
+def test_few_output_channels_fused_kernel(B, shape):
+    # F2 layers with at most 8 output channels: one kernel (input transform -> tcgen05 -> output transform on
+    # chip) once the layer is large enough; the threshold is lowered so that small ragged shapes take it too
+    C, K, H, W, N = shape
+    layer = ConvLayer(C=C, K=K, H=H, W=W, N=N)
+    x, w, b = workloads.make_inputs(layer, seed=sum(shape))
+    ref = oracle.direct_conv3x3(x.numpy(), w.numpy(), b.numpy())
+    B.sdwino_set_fused_min_tiles(1)
+    try:
+        n0 = B.sdwino_launch_count()
+        _, _, _, y = _run(B, layer, 2, x=x, w=w, b=b)
+        assert B.sdwino_launch_count() - n0 == 2          # filter transform + the fused kernel
+        _, _, _, y2 = _run(B, layer, 2, x=x, w=w, b=b)
+    finally:
+        B.sdwino_set_fused_min_tiles(0)
+    assert torch.equal(y, y2)                              # deterministic
+    assert _rel_err(y, ref) <= TOL_F2_REGRESSION
+    mask = _edge_mask(H, W, 2)
+    assert np.abs(y.double().numpy() - ref)[:, :, mask].max() <= TOL * np.abs(ref).max()
+    # the three-kernel path on the same inputs
+    B.sdwino_set_gemm_shape(1, 16)
+    try:
+        _, _, _, y_gemm = _run(B, layer, 2, x=x, w=w, b=b)
+    finally:
+        B.sdwino_set_gemm_shape(0, 0)
+    assert _rel_err(y, y_gemm.double().numpy()) <= TOL_F2_REGRESSION
+
+
+def test_few_output_channels_default_threshold_and_no_bias(B):
+    # 6272 tiles = 49 blocks: above the default threshold without touching the knob; no bias
+    layer = ConvLayer(C=48, K=3, H=112, W=112, N=2)
+    x, w, _ = workloads.make_inputs(layer, seed=11, with_bias=False)
+    n0 = B.sdwino_launch_count()
+    _, _, _, y = _run(B, layer, 2, x=x, w=w, b=None)
+    assert B.sdwino_launch_count() - n0 == 2
+    ks = [0, 2]
+    ref = oracle.direct_conv3x3(x.numpy(), w.numpy(), None, channels=ks)
+    d = np.abs(y[:, ks].double().numpy() - ref).max()
+    assert d <= TOL_F2_REGRESSION * np.abs(ref).max()
+    with pytest.raises(B.SdwinoError):
+        B.sdwino_set_fused_min_tiles(-1)
+
+
 def test_set_gemm_shape_rejects_bad_values(B):
     for ctas, n in [(3, 0), (-1, 0), (0, 8), (0, 272), (1, 100)]:
         with pytest.raises(B.SdwinoError):
