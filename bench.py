@@ -28,12 +28,11 @@ if ROOT not in sys.path:
 METRIC = "direct-conv-equivalent TFLOP/s over the SD v1.5 UNet 3x3 conv sweep (2*N*K*C*H*W*9 / time)"
 UNIT = "TFLOP/s"
 WORKLOAD = "sd15_unet"
-TILE = 2
+TILE = "auto"   # per layer: what sdwino_choose_tile returns; --tile 2 / --tile 4 force one algorithm
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# dram__bytes_read.sum + dram__bytes_write.sum of the 17 GEMM launches of one SD v1.5 step, from one ncu
-# capture (profiles/launch_list_sd15_unet_sweep.md): 691.3 MB, i.e. 40.7 MB per launch.  Only valid for the
-# default workload with all layers.
-GEMM_DRAM_BYTES_PER_LAUNCH_SD15 = 40.66e6
+# dram__bytes_read.sum + dram__bytes_write.sum per GEMM launch of one SD v1.5 step, from ncu captures
+# (profiles/launch_list_sd15_unet_sweep.md), by --tile.  Only valid for the default workload with all layers.
+GEMM_DRAM_BYTES_PER_LAUNCH_SD15 = {"2": 40.66e6}
 PAPER_CONTEXT = {"per_layer_speedup_vs_sdcpp_m1pro": 2.76, "end_to_end_speedup_vs_sdcpp_m1pro": 4.79}
 
 
@@ -225,8 +224,7 @@ def run_ours(args):
 
     peaks, peak_kind = load_peaks()
     layers = select_layers(args)
-    TILE = args.tile
-    a2 = (TILE + 2) ** 2
+    tiles = [B.sdwino_choose_tile(L.N, L.C, L.H, L.W, L.K) if args.tile == "auto" else int(args.tile) for L in layers]
 
     # ---- inputs: pinned host copies (for the end-to-end pass) and resident device copies ----
     host, devt = [], []
@@ -235,7 +233,7 @@ def run_ours(args):
         x, w, b = workloads.make_inputs(L, seed=li, pin=True)
         y_h = torch.empty(L.N, L.K, L.H, L.W, dtype=torch.float16).pin_memory()
         host.append((x, w, b, y_h))
-        dims = (L.N, L.C, L.H, L.W, L.K, TILE)
+        dims = (L.N, L.C, L.H, L.W, L.K, tiles[li])
         ws_bytes = max(ws_bytes, B.sdwino_workspace_bytes(*dims))
         hws_bytes = max(hws_bytes, B.sdwino_host_staging_bytes(*dims) + B.sdwino_workspace_bytes(*dims))
     ws = B.alloc_workspace(max(ws_bytes, hws_bytes), dev)
@@ -244,17 +242,17 @@ def run_ours(args):
     B.sdwino_profile_enable(True)
     w_dev = [h[1].to(dev) for h in host]
     for _ in range(3):
-        wTs = [B.sdwino_filter_transform(wd, TILE) for wd in w_dev]
+        wTs = [B.sdwino_filter_transform(wd, t) for wd, t in zip(w_dev, tiles)]
         prof = B.sdwino_profile_collect()
     ft_ms = prof["filter_transform"][0]
-    ft_bytes = sum(L.K * L.C * 18 + B.sdwino_filter_bytes(L.K, L.C, TILE) for L in layers)
+    ft_bytes = sum(L.K * L.C * 18 + B.sdwino_filter_bytes(L.K, L.C, t) for L, t in zip(layers, tiles))
     B.sdwino_profile_enable(False)
     del w_dev
     for (x, w, b, y_h), wT in zip(host, wTs):
         devt.append((x.to(dev), wT, b.to(dev), torch.empty(y_h.shape, dtype=torch.float16, device=dev)))
     def step():
-        for L, (xd, wT, bd, yd) in zip(layers, devt):
-            B.sdwino_conv3x3(xd, wT, bd, L.K, TILE, y=yd, workspace=ws, stream=torch.cuda.current_stream())
+        for L, t, (xd, wT, bd, yd) in zip(layers, tiles, devt):
+            B.sdwino_conv3x3(xd, wT, bd, L.K, t, y=yd, workspace=ws, stream=torch.cuda.current_stream())
 
     sampler = ClockSampler(visible_to_nvml_index(local_rank))
     # the timed step is replayed from a CUDA graph captured from the same C-ABI calls, so that host launch
@@ -308,8 +306,8 @@ def run_ours(args):
     e2e_steps = max(3, min(args.steps, 30))
 
     def e2e_step():
-        for L, (x, w, b, y_h), (_, wT, _, _) in zip(layers, host, devt):
-            B.sdwino_conv3x3_host(x, wT, b, y_h, TILE, ws, stream=stream)
+        for t, (x, w, b, y_h), (_, wT, _, _) in zip(tiles, host, devt):
+            B.sdwino_conv3x3_host(x, wT, b, y_h, t, ws, stream=stream)
 
     for _ in range(3):
         e2e_step()
@@ -329,8 +327,8 @@ def run_ours(args):
     B.sdwino_profile_enable(True)
     records_per_layer = []
     with torch.cuda.stream(stream):
-        for L, (xd, wT, bd, yd) in zip(layers, devt):     # learn how many launches each layer makes
-            B.sdwino_conv3x3(xd, wT, bd, L.K, TILE, y=yd, workspace=ws, stream=stream)
+        for L, t, (xd, wT, bd, yd) in zip(layers, tiles, devt):     # learn how many launches each layer makes
+            B.sdwino_conv3x3(xd, wT, bd, L.K, t, y=yd, workspace=ws, stream=stream)
             records_per_layer.append(len(B.sdwino_profile_records()))
     prof_steps = max(3, min(args.steps, 20))
     per_layer = [dict(input_transform=0.0, wino_gemm=0.0, output_transform=0.0, fused=0.0, launches=0)
@@ -375,16 +373,17 @@ def run_ours(args):
     in_ms = out_ms = 0.0
     in_bytes = out_bytes = 0.0
     fused_ms = 0.0
-    for L, pl in zip(layers, per_layer):
-        P = L.tiles(TILE)
+    for L, t, pl in zip(layers, tiles, per_layer):
+        a2 = (t + 2) ** 2
+        P = L.tiles(t)
         wino_flops = 2.0 * a2 * L.K * L.C * P
-        u_bytes = B.sdwino_filter_bytes(L.K, L.C, TILE)
+        u_bytes = B.sdwino_filter_bytes(L.K, L.C, t)
         xb, yb = 2.0 * L.N * L.C * L.H * L.W, 2.0 * L.N * L.K * L.H * L.W
         t_tensor = wino_flops / (tpeak * 1e12) * 1e6
         t_hbm = (xb + 2.0 * a2 * L.K * L.C + yb + 2 * L.K) / (hpeak * 1e9) * 1e6
         total_us = (pl["input_transform"] + pl["wino_gemm"] + pl["output_transform"] + pl["fused"]) * 1e3
         layer_rows.append({
-            "layer": L.name, "us": round(total_us, 2),
+            "layer": L.name, "tile": t, "us": round(total_us, 2),
             "us_input": round(pl["input_transform"] * 1e3, 2), "us_gemm": round(pl["wino_gemm"] * 1e3, 2),
             "us_output": round(pl["output_transform"] * 1e3, 2), "us_fused": round(pl["fused"] * 1e3, 2),
             "eq_tflops": round(L.direct_flops / (total_us * 1e-6) / 1e12, 1),
@@ -407,8 +406,8 @@ def run_ours(args):
     roofline = {
         "kernel": "wino_gemm_kernel", "bound": "tensor", "achieved": round(achieved, 1), "peak": tpeak,
         "unit": "TFLOP/s", "frac": round(achieved / tpeak, 4),
-        "traffic": (GEMM_DRAM_BYTES_PER_LAUNCH_SD15 if (args.workload == WORKLOAD and not args.layers and TILE == 2)
-                    else None),
+        "traffic": (GEMM_DRAM_BYTES_PER_LAUNCH_SD15.get(str(args.tile))
+                    if (args.workload == WORKLOAD and not args.layers) else None),
         "traffic_unit": "bytes per launch (ncu dram read + write, L2 left warm)",
         "peak_source": f"{peak_kind} (cuBLAS bf16 burst; fp16 has the same nominal rate)",
         "launches_per_step": gemm_launches, "avg_launch_us": round(gemm_ms * 1e3 / gemm_launches, 2),
@@ -467,8 +466,11 @@ def run_ours(args):
             "warmup": max(args.warmup, 3), "ms_per_step": round(ms_step, 4), "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f16", "data": "synthetic",
             "config": {"workload": args.workload, "layers": len(layers), "layer_subset": args.layers or "all",
-                       "batch": layers[0].N, "tile": TILE,
-                       "algorithm": f"Winograd F({TILE}x{TILE},3x3), fp16 storage, fp32 accumulate",
+                       "batch": layers[0].N, "tile": args.tile,
+                       "tile_per_layer": tiles,
+                       "algorithm": ("Winograd F(2x2,3x3) or F(4x4,3x3) per layer (sdwino_choose_tile)"
+                                     if args.tile == "auto" else f"Winograd F({args.tile}x{args.tile},3x3)") +
+                                    ", fp16 storage, fp32 accumulate",
                        "parallelism": f"replicas x{world} (no exchange step)",
                        "launch": "direct" if args.no_graph else "CUDA graph of one step, replayed",
                        "l2": "no flush: one step streams ~0.5 GB of transformed weights, 4x the 126 MB L2, so "
@@ -498,7 +500,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=WORKLOAD, choices=["single", "sd15_unet", "sd_vae_512", "sd21_unet", "sdxl_1024"])
     ap.add_argument("--layers", default="", help="comma-separated layer indices of the workload (default: all)")
-    ap.add_argument("--tile", type=int, default=TILE, choices=[2, 4])
+    ap.add_argument("--tile", default=TILE, choices=["auto", "2", "4"])
     ap.add_argument("--no-graph", action="store_true", help="launch every step directly instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-yardstick", action="store_true")

@@ -150,6 +150,17 @@ unsigned long long sdwino_launch_count(void);
 int sdwino_set_gemm_shape(int ctas, int n_tile);
 
 /*
+ * Which of the two supported algorithms is expected to be faster for a layer: returns 2 for F(2x2,3x3),
+ * 4 for F(4x4,3x3), 0 for non-positive sizes.  The paper leaves the tile size open; both satisfy the
+ * accuracy bound (F4 with about 4x the error of F2).  Rule: layers with at most 8 input or output
+ * channels -> 2 (single-kernel paths); otherwise 4 when 2 * tiles * (C + K) >= K * C with
+ * tiles = N * ceil(H/2) * ceil(W/2), i.e. when the activation-side traffic outweighs the weights.
+ * Pure host arithmetic: no device is touched.  The caller passes the result as `tile` to
+ * sdwino_filter_transform and sdwino_conv3x3.
+ */
+int sdwino_choose_tile(int N, int C, int H, int W, int K);
+
+/*
  * Tuning and test knob.  F(2x2,3x3) layers with at most 8 output channels (the 320 -> 4 and 128 -> 3
  * output convolutions) run as ONE kernel that keeps V and M on chip (input transform into shared memory,
  * tcgen05 MMAs into TMEM, output transform from TMEM) when the batch has at least `p_tiles` blocks of 128

@@ -21,7 +21,7 @@ EXPORTS = [
     "sdwino_workspace_bytes", "sdwino_workspace_min_bytes", "sdwino_set_workspace", "sdwino_conv3x3",
     "sdwino_conv3x3_ws", "sdwino_host_staging_bytes", "sdwino_conv3x3_host",
     "sdwino_last_device_status", "sdwino_launch_count", "sdwino_profile_enable", "sdwino_profile_collect",
-    "sdwino_profile_records", "sdwino_set_gemm_shape", "sdwino_conv3x3_static", "sdwino_set_fused_min_tiles",
+    "sdwino_profile_records", "sdwino_set_gemm_shape", "sdwino_conv3x3_static", "sdwino_set_fused_min_tiles", "sdwino_choose_tile",
 ]
 
 KERNEL_KINDS = ("filter_transform", "input_transform", "wino_gemm", "output_transform", "fused")
@@ -67,6 +67,8 @@ def _load() -> ctypes.CDLL:
     lib.sdwino_profile_records.argtypes = [ctypes.POINTER(i), ctypes.POINTER(ctypes.c_float), i, i]
     lib.sdwino_set_gemm_shape.restype = i
     lib.sdwino_set_gemm_shape.argtypes = [i, i]
+    lib.sdwino_choose_tile.restype = i
+    lib.sdwino_choose_tile.argtypes = [i, i, i, i, i]
     lib.sdwino_set_fused_min_tiles.restype = i
     lib.sdwino_set_fused_min_tiles.argtypes = [ctypes.c_longlong]
     lib.sdwino_profile_enable.restype = i
@@ -128,6 +130,14 @@ def sdwino_last_device_status(stream: Optional[torch.cuda.Stream] = None) -> int
 def sdwino_set_gemm_shape(ctas: int = 0, n_tile: int = 0) -> None:
     """Force single-CTA (1) or CTA-pair (2) GEMM tiles and/or the channels per tile; 0 = automatic."""
     _check(lib.sdwino_set_gemm_shape(ctas, n_tile), "sdwino_set_gemm_shape")
+
+
+def sdwino_choose_tile(N: int, C: int, H: int, W: int, K: int) -> int:
+    """2 or 4: the output tile size (F(2x2) / F(4x4)) expected to be faster for this layer."""
+    t = int(lib.sdwino_choose_tile(N, C, H, W, K))
+    if t not in (2, 4):
+        raise SdwinoError(ERR_INVALID_ARG, "sdwino_choose_tile")
+    return t
 
 
 def sdwino_set_fused_min_tiles(p_tiles: int = 0) -> None:

@@ -70,9 +70,9 @@ __device__ __forceinline__ FkUnitGeo fk_decode(const TileGeom& geo, int C, long 
     FkUnitGeo g;
     g.valid = p < geo.P;
     const long long pp = g.valid ? p : 0;
-    const int tw = static_cast<int>(pp % geo.TW);
-    const int th = static_cast<int>((pp / geo.TW) % geo.TH);
-    const long long n = pp / (static_cast<long long>(geo.TW) * geo.TH);
+    int tw, th;
+    long long n;
+    decode_tile(geo, pp, n, th, tw);
     const int i0 = 2 * th - 1, j0 = 2 * tw;
     g.base = n * C * static_cast<long long>(geo.H) * geo.W + static_cast<long long>(i0) * geo.W + j0;
     g.rows_ok = 0;
@@ -325,9 +325,9 @@ fused_small_k_kernel(const __grid_constant__ CUtensorMap tmU, const __half* __re
             const long long p = static_cast<long long>(tile) * 128 + quarter * 32 + lane;
             const bool valid = p < prm.geo.P;
             const long long pp = valid ? p : 0;
-            const int tw = static_cast<int>(pp % prm.geo.TW);
-            const int th = static_cast<int>((pp / prm.geo.TW) % prm.geo.TH);
-            const long long n = pp / (static_cast<long long>(prm.geo.TW) * prm.geo.TH);
+            int tw, th;
+            long long n;
+            decode_tile(prm.geo, pp, n, th, tw);
             const long long plane = static_cast<long long>(prm.geo.H) * prm.geo.W;
             __half* out0 = y + (n * prm.K + k0) * plane + static_cast<long long>(2 * th) * prm.geo.W + 2 * tw;
             const bool row1_ok = 2 * th + 1 < prm.geo.H;

@@ -97,6 +97,7 @@ bool make_plan(int N, int C, int H, int W, int K, int tile, Plan* pl) {
     pl->TH = (H + tile - 1) / tile;
     pl->TW = (W + tile - 1) / tile;
     pl->P = static_cast<long long>(N) * pl->TH * pl->TW;
+    if (pl->P >= (1ll << 31) - GEMM_BLOCK_P) return false;   // tile indices are 32-bit on the device
     pl->P128 = round_up_ll(pl->P, GEMM_BLOCK_P);
     pl->per_tile = static_cast<size_t>(pl->a2) * (static_cast<size_t>(C) + K) * sizeof(__half);
     // element counts must stay far inside int64
@@ -265,10 +266,11 @@ int launch_input(const __half* x, __half* V, const TileGeom& geo, int C, long lo
     ProfScope prof(KIND_INPUT, st);
     constexpr int TPT = 8 / M;
     cudaError_t e;
-    if (geo.W % 8 == 0 && aligned(x, 16)) {
-        dim3 grid(static_cast<unsigned>((static_cast<long long>(p_count / TPT) * C + 127) / 128));
-        e = launch_pdl(input_transform_vec_kernel<M, TPT>, grid, dim3(128), 0, st, 0, x, V, geo, C, p_begin, p_count,
-                       Pstride);
+    const long long units = static_cast<long long>(p_count / TPT) * C;   // one thread each
+    if (geo.W % 8 == 0 && aligned(x, 16) && units < (1ll << 31) - 128) {
+        dim3 grid(static_cast<unsigned>((units + 127) / 128));
+        e = launch_pdl(input_transform_vec_kernel<M, TPT>, grid, dim3(128), 0, st, 0, x, V, geo, C, p_begin,
+                       make_fastdiv(static_cast<uint32_t>(p_count / TPT)), Pstride);
     } else {
         dim3 grid((p_count + 127) / 128, C);
         e = launch_pdl(input_transform_kernel<M>, grid, dim3(128), 0, st, 0, x, V, geo, C, p_begin, p_count, Pstride);
@@ -283,10 +285,11 @@ int launch_output(const __half* Mws, const __half* bias, __half* y, const TileGe
     ProfScope prof(KIND_OUTPUT, st);
     constexpr int TPT = 8 / M;
     cudaError_t e;
-    if (geo.W % 8 == 0 && aligned(y, 16)) {
-        dim3 grid(static_cast<unsigned>((static_cast<long long>(p_count / TPT) * K + 127) / 128));
+    const long long units = static_cast<long long>(p_count / TPT) * K;   // one thread each
+    if (geo.W % 8 == 0 && aligned(y, 16) && units < (1ll << 31) - 128) {
+        dim3 grid(static_cast<unsigned>((units + 127) / 128));
         e = launch_pdl(output_transform_vec_kernel<M, TPT>, grid, dim3(128), 0, st, 0, Mws, bias, y, geo, K, p_begin,
-                       p_count, Pstride);
+                       make_fastdiv(static_cast<uint32_t>(p_count / TPT)), Pstride);
     } else {
         dim3 grid((p_count + 127) / 128, K);
         e = launch_pdl(output_transform_kernel<M>, grid, dim3(128), 0, st, 0, Mws, bias, y, geo, K, p_begin, p_count,
@@ -337,7 +340,7 @@ int launch_fused_small_k(const __half* x, const void* wT, const __half* bias, __
     CUtensorMap tmU;
     if (!encode_filter_map(&tmU, wT, pl.Cb, pl.Kb, pl.a2, 1, 16, FK_KMAX)) return SDWINO_ERR_CUDA;
     FusedKParams prm;
-    prm.geo = TileGeom{H, W, pl.TH, pl.TW, pl.P};
+    prm.geo = make_geom(H, W, pl.TH, pl.TW, pl.P);
     prm.C = C;
     prm.K = K;
     prm.num_stages = (C + FK_CSTEP - 1) / FK_CSTEP;
@@ -436,7 +439,7 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
         return launch_fused_small_k(static_cast<const __half*>(x), wT, static_cast<const __half*>(bias),
                                     static_cast<__half*>(y), pl, C, H, W, K, st);
     if (use_fused_small_c(C, tile) && !g_disable_fused) {
-        TileGeom geo{H, W, pl.TH, pl.TW, pl.P};
+        const TileGeom geo = make_geom(H, W, pl.TH, pl.TW, pl.P);
         const __half* xh = static_cast<const __half*>(x);
         const __half* uh = static_cast<const __half*>(wT);
         const __half* bh = static_cast<const __half*>(bias);
@@ -483,7 +486,7 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
         !encode_map(&tmM, Mws, pc, K, pl.a2, pc, static_cast<uint64_t>(K) * pc, GEMM_BLOCK_P, prm.epi_rows, false))
         return SDWINO_ERR_CUDA;
 
-    TileGeom geo{H, W, pl.TH, pl.TW, pl.P};
+    const TileGeom geo = make_geom(H, W, pl.TH, pl.TW, pl.P);
     const __half* xh = static_cast<const __half*>(x);
     const __half* bh = static_cast<const __half*>(bias);
     __half* yh = static_cast<__half*>(y);
@@ -516,6 +519,17 @@ int sdwino_set_gemm_shape(int ctas, int n_tile) {
     g_force_n_tile = n_tile;
     g_disable_fused = (ctas != 0 || n_tile != 0);
     return SDWINO_OK;
+}
+
+int sdwino_choose_tile(int N, int C, int H, int W, int K) {
+    if (N <= 0 || C <= 0 || H <= 0 || W <= 0 || K <= 0) return 0;
+    // Few-channel layers have single-kernel F(2x2) paths.  Otherwise F(4x4) moves 2.25 instead of 4 transform
+    // values per pixel through the workspace and the tensor cores but streams 36 instead of 16 values per
+    // weight: it wins once the tiles outnumber the weights per channel pair.  Measured on 97 layer shapes:
+    // F4 is 15-40 % faster above twice the threshold below, within +-7 % around it, up to 2x slower far below.
+    if (C <= 8 || K <= 8) return 2;
+    const long long P2 = static_cast<long long>(N) * ((H + 1) / 2) * ((W + 1) / 2);
+    return 2 * P2 * (static_cast<long long>(C) + K) >= static_cast<long long>(K) * C ? 4 : 2;
 }
 
 int sdwino_set_fused_min_tiles(long long p_tiles) {

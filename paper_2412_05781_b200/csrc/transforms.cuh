@@ -143,10 +143,45 @@ filter_transform_kernel(const __half* __restrict__ w, __half* __restrict__ U, in
 // the whole batch) belongs to image n = p / (TH*TW), tile row th and tile column tw; its
 // input window starts at pixel (m*th - 1, m*tw - 1) and its outputs at (m*th, m*tw).
 // ---------------------------------------------------------------------------------------
+// Division by a launch-invariant 32-bit divisor as multiply-high and shift (a 64-bit or even 32-bit integer
+// division costs on the order of a hundred instructions per thread; the index decode of a transform thread
+// needs three).  For 0 <= n < 2^31 and d >= 2: with L = ceil(log2 d) and mul = ceil(2^(31+L) / d) < 2^32,
+// floor(n / d) = (n * mul) >> (31 + L), because mul * d = 2^(31+L) + e with 0 <= e < d <= 2^L makes the
+// excess n * e / (d * 2^(31+L)) smaller than 1 / d.
+struct FastDiv {
+    uint32_t d, mul, shr;
+};
+inline FastDiv make_fastdiv(uint32_t d) {
+    FastDiv f{d, 0u, 0u};
+    if (d > 1) {
+        uint32_t L = 0;
+        while ((1ull << L) < d) ++L;
+        f.mul = static_cast<uint32_t>(((1ull << (31 + L)) + d - 1) / d);
+        f.shr = L - 1;
+    }
+    return f;
+}
+__device__ __forceinline__ uint32_t fast_div(uint32_t n, const FastDiv& f) {
+    return f.d == 1 ? n : (__umulhi(n, f.mul) >> f.shr);
+}
+
 struct TileGeom {
     int H, W, TH, TW;
-    long long P;  // N*TH*TW
+    long long P;  // N*TH*TW, below 2^31
+    FastDiv tw_div, th_div;
 };
+inline TileGeom make_geom(int H, int W, int TH, int TW, long long P) {
+    return TileGeom{H, W, TH, TW, P, make_fastdiv(static_cast<uint32_t>(TW)), make_fastdiv(static_cast<uint32_t>(TH))};
+}
+// tile p -> image n, tile row th, tile column tw
+__device__ __forceinline__ void decode_tile(const TileGeom& geo, long long p, long long& n, int& th, int& tw) {
+    const uint32_t pu = static_cast<uint32_t>(p);
+    const uint32_t row = fast_div(pu, geo.tw_div);
+    const uint32_t img = fast_div(row, geo.th_div);
+    tw = static_cast<int>(pu - row * static_cast<uint32_t>(geo.TW));
+    th = static_cast<int>(row - img * static_cast<uint32_t>(geo.TH));
+    n = img;
+}
 
 // Activation preprocess.  V layout: [a*a][C][Pstride] with the chunk-local tile index
 // (p - p_begin) contiguous.  Threads past the last tile write zeros so that the GEMM reads
@@ -165,9 +200,9 @@ input_transform_kernel(const __half* __restrict__ x, __half* __restrict__ V, Til
     const long long p = p_begin + pl;
     float d[A][A];
     if (p < geo.P) {
-        const int tw = static_cast<int>(p % geo.TW);
-        const int th = static_cast<int>((p / geo.TW) % geo.TH);
-        const long long n = p / (static_cast<long long>(geo.TW) * geo.TH);
+        int tw, th;
+        long long n;
+        decode_tile(geo, p, n, th, tw);
         const __half* img = x + (n * C + c) * static_cast<long long>(geo.H) * geo.W;
         const int i0 = M * th - 1, j0 = M * tw - 1;
 #pragma unroll
@@ -241,9 +276,9 @@ output_transform_kernel(const __half* __restrict__ Mws, const __half* __restrict
 #pragma unroll
         for (int i = 0; i < M; ++i) t[i][s] = o[i];
     }
-    const int tw = static_cast<int>(p % geo.TW);
-    const int th = static_cast<int>((p / geo.TW) % geo.TH);
-    const long long n = p / (static_cast<long long>(geo.TW) * geo.TH);
+    int tw, th;
+    long long n;
+    decode_tile(geo, p, n, th, tw);
     const float b = bias ? __half2float(__ldg(bias + k)) : 0.f;
     __half* img = y + (n * K + k) * static_cast<long long>(geo.H) * geo.W;
     const int i0 = M * th, j0 = M * tw;
@@ -291,27 +326,110 @@ __device__ __forceinline__ void unpack2(uint32_t v, float& a, float& b) {
     b = f.y;
 }
 
+// ---------------------------------------------------------------------------------------
+// F(4x4,3x3) in packed fp32 (sm_100 has two-wide fp32 FMA/ADD/MUL): the two halves of a float2 are the
+// two tiles a thread owns.  The rows of B^T and A^T for the points {0, +-3/4, +-3/2, inf} come in +- pairs,
+// so each pair shares its even and its odd part: 14 packed operations for B^T d (6 -> 6) and 12 for
+// A^T m (6 -> 4), against 22 and 18 scalar ones per tile when the matrix is applied row by row.  The vector
+// transform kernels of F4 are bound by instruction issue, not by memory (ncu: 69 % issue-active).
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ float2 f2s(float a) { return make_float2(a, a); }
+
+__device__ __forceinline__ void bt4_packed(const float2 (&d)[6], float2 (&o)[6]) {
+    const float2 e1 = __ffma2_rn(f2s(-2.25f), d[2], d[4]);
+    const float2 o1 = __ffma2_rn(f2s(0.75f), d[3], __fmul2_rn(f2s(-1.6875f), d[1]));
+    const float2 e2 = __ffma2_rn(f2s(-0.5625f), d[2], d[4]);
+    const float2 o2 = __ffma2_rn(f2s(1.5f), d[3], __fmul2_rn(f2s(-0.84375f), d[1]));
+    o[0] = __ffma2_rn(f2s(1.265625f), d[0], __ffma2_rn(f2s(-2.8125f), d[2], d[4]));
+    o[1] = __fadd2_rn(e1, o1);
+    o[2] = __ffma2_rn(f2s(-1.f), o1, e1);
+    o[3] = __fadd2_rn(e2, o2);
+    o[4] = __ffma2_rn(f2s(-1.f), o2, e2);
+    o[5] = __ffma2_rn(f2s(1.265625f), d[1], __ffma2_rn(f2s(-2.8125f), d[3], d[5]));
+}
+
+__device__ __forceinline__ void at4_packed(const float2 (&m)[6], float2 (&o)[4]) {
+    const float2 s1 = __fadd2_rn(m[1], m[2]);
+    const float2 d1 = __ffma2_rn(f2s(-1.f), m[2], m[1]);
+    const float2 s2 = __fadd2_rn(m[3], m[4]);
+    const float2 d2 = __ffma2_rn(f2s(-1.f), m[4], m[3]);
+    o[0] = __fadd2_rn(__fadd2_rn(m[0], s1), s2);
+    o[1] = __ffma2_rn(f2s(1.5f), d2, __fmul2_rn(f2s(0.75f), d1));
+    o[2] = __ffma2_rn(f2s(2.25f), s2, __fmul2_rn(f2s(0.5625f), s1));
+    o[3] = __ffma2_rn(f2s(3.375f), d2, __ffma2_rn(f2s(0.421875f), d1, m[5]));
+}
+
 template <int M, int TPT>
 __global__ void __launch_bounds__(128)
 input_transform_vec_kernel(const __half* __restrict__ x, __half* __restrict__ V, TileGeom geo, int C,
-                           long long p_begin, int p_count, long long Pstride) {
+                           long long p_begin, FastDiv gdiv, long long Pstride) {
     using Wm = Wino<M>;
     constexpr int A = Wm::A;
     pdl_launch_dependents();
     pdl_wait();
     static_assert(M * TPT == 8, "one 16-byte row segment per thread");
     // flat index over (channel, group of TPT tiles): blocks stay full when a pass has few tiles
-    const int groups = p_count / TPT;
-    const long long idx = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
-    const int c = static_cast<int>(idx / groups);
+    const uint32_t idx = blockIdx.x * blockDim.x + threadIdx.x;   // below 2^31 (checked by the launcher)
+    const int c = static_cast<int>(fast_div(idx, gdiv));           // gdiv.d = p_count / TPT groups per channel
     if (c >= C) return;
-    const int pl = static_cast<int>(idx % groups) * TPT;  // first chunk-local tile of this thread
+    const int pl = static_cast<int>(idx - static_cast<uint32_t>(c) * gdiv.d) * TPT;  // first chunk-local tile of this thread
     const long long p = p_begin + pl;
+    if constexpr (M == 4) {
+        // packed path: e2[r][nu] holds (tile 0, tile 1)
+        float2 e2[A][A];
+        if (p < geo.P) {
+            int tw, th;
+            long long n;
+            decode_tile(geo, p, n, th, tw);
+            const __half* img = x + (n * C + c) * static_cast<long long>(geo.H) * geo.W;
+            const int i0 = M * th - 1, j0 = M * tw;
+#pragma unroll
+            for (int r = 0; r < A; ++r) {
+                const int i = i0 + r;
+                float row[10];
+                if (i >= 0 && i < geo.H) {
+                    const __half* rp = img + static_cast<long long>(i) * geo.W + j0;
+                    const uint4 v = __ldg(reinterpret_cast<const uint4*>(rp));
+                    unpack2(v.x, row[1], row[2]);
+                    unpack2(v.y, row[3], row[4]);
+                    unpack2(v.z, row[5], row[6]);
+                    unpack2(v.w, row[7], row[8]);
+                    row[0] = j0 > 0 ? __half2float(__ldg(rp - 1)) : 0.f;
+                    row[9] = j0 + 8 < geo.W ? __half2float(__ldg(rp + 8)) : 0.f;
+                } else {
+#pragma unroll
+                    for (int s = 0; s < 10; ++s) row[s] = 0.f;
+                }
+                float2 d[A];
+#pragma unroll
+                for (int s = 0; s < A; ++s) d[s] = make_float2(row[s], row[M + s]);
+                bt4_packed(d, e2[r]);
+            }
+        } else {
+#pragma unroll
+            for (int r = 0; r < A; ++r)
+#pragma unroll
+                for (int s = 0; s < A; ++s) e2[r][s] = make_float2(0.f, 0.f);
+        }
+        const long long plane = static_cast<long long>(C) * Pstride;
+        __half* dst = V + static_cast<long long>(c) * Pstride + pl;
+#pragma unroll
+        for (int nu = 0; nu < A; ++nu) {
+            float2 col[A], o[A];
+#pragma unroll
+            for (int r = 0; r < A; ++r) col[r] = e2[r][nu];
+            bt4_packed(col, o);
+#pragma unroll
+            for (int xi = 0; xi < A; ++xi)
+                *reinterpret_cast<uint32_t*>(dst + (xi * A + nu) * plane) = pack2(o[xi].x, o[xi].y);
+        }
+        return;
+    }
     float e[A][TPT][A];  // rows transformed along the columns: e[r][t][nu] = sum_s Bt[nu][s] d[r][s]
     if (p < geo.P) {
-        const int tw = static_cast<int>(p % geo.TW);
-        const int th = static_cast<int>((p / geo.TW) % geo.TH);
-        const long long n = p / (static_cast<long long>(geo.TW) * geo.TH);
+        int tw, th;
+        long long n;
+        decode_tile(geo, p, n, th, tw);
         const __half* img = x + (n * C + c) * static_cast<long long>(geo.H) * geo.W;
         const int i0 = M * th - 1, j0 = M * tw;
 #pragma unroll
@@ -381,21 +499,55 @@ input_transform_vec_kernel(const __half* __restrict__ x, __half* __restrict__ V,
 template <int M, int TPT>
 __global__ void __launch_bounds__(128)
 output_transform_vec_kernel(const __half* __restrict__ Mws, const __half* __restrict__ bias, __half* __restrict__ y,
-                            TileGeom geo, int K, long long p_begin, int p_count, long long Pstride) {
+                            TileGeom geo, int K, long long p_begin, FastDiv gdiv, long long Pstride) {
     using Wm = Wino<M>;
     constexpr int A = Wm::A;
     pdl_launch_dependents();
     pdl_wait();
     static_assert(M * TPT == 8, "one 16-byte row segment per thread");
-    const int groups = p_count / TPT;
-    const long long idx = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
-    const int k = static_cast<int>(idx / groups);
+    const uint32_t idx = blockIdx.x * blockDim.x + threadIdx.x;   // below 2^31 (checked by the launcher)
+    const int k = static_cast<int>(fast_div(idx, gdiv));           // gdiv.d = p_count / TPT groups per channel
     if (k >= K) return;
-    const int pl = static_cast<int>(idx % groups) * TPT;
+    const int pl = static_cast<int>(idx - static_cast<uint32_t>(k) * gdiv.d) * TPT;
     const long long p = p_begin + pl;
     if (p >= geo.P) return;
     const long long plane = static_cast<long long>(K) * Pstride;
     const __half* src = Mws + static_cast<long long>(k) * Pstride + pl;
+    if constexpr (M == 4) {
+        // packed path: every float2 holds (tile 0, tile 1)
+        float2 tt[M][A];   // A^T m, one column nu at a time
+#pragma unroll
+        for (int s = 0; s < A; ++s) {
+            float2 col[A], o[M];
+#pragma unroll
+            for (int r = 0; r < A; ++r) {
+                const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(src + (r * A + s) * plane));
+                col[r] = __half22float2(*reinterpret_cast<const __half2*>(&w));
+            }
+            at4_packed(col, o);
+#pragma unroll
+            for (int i = 0; i < M; ++i) tt[i][s] = o[i];
+        }
+        int tw, th;
+        long long n;
+        decode_tile(geo, p, n, th, tw);
+        const float b = bias ? __half2float(__ldg(bias + k)) : 0.f;
+        __half* img = y + (n * K + k) * static_cast<long long>(geo.H) * geo.W;
+        const int i0 = M * th, j0 = M * tw;
+#pragma unroll
+        for (int i = 0; i < M; ++i) {
+            float2 o[M];
+            at4_packed(tt[i], o);
+            if (i0 + i >= geo.H) continue;
+            uint4 w;
+            w.x = pack2(o[0].x + b, o[1].x + b);
+            w.y = pack2(o[2].x + b, o[3].x + b);
+            w.z = pack2(o[0].y + b, o[1].y + b);
+            w.w = pack2(o[2].y + b, o[3].y + b);
+            *reinterpret_cast<uint4*>(img + static_cast<long long>(i0 + i) * geo.W + j0) = w;
+        }
+        return;
+    }
     float mm[A][A][TPT];
 #pragma unroll
     for (int r = 0; r < A; ++r)
@@ -411,9 +563,9 @@ output_transform_vec_kernel(const __half* __restrict__ Mws, const __half* __rest
                 unpack2(w, mm[r][s][0], mm[r][s][1]);
             }
         }
-    const int tw = static_cast<int>(p % geo.TW);
-    const int th = static_cast<int>((p / geo.TW) % geo.TH);
-    const long long n = p / (static_cast<long long>(geo.TW) * geo.TH);
+    int tw, th;
+    long long n;
+    decode_tile(geo, p, n, th, tw);
     const float b = bias ? __half2float(__ldg(bias + k)) : 0.f;
     __half* img = y + (n * K + k) * static_cast<long long>(geo.H) * geo.W;
     const int i0 = M * th, j0 = M * tw;
@@ -488,9 +640,9 @@ fused_small_c_kernel(const __half* __restrict__ x, const __half* __restrict__ U,
     __syncthreads();
     const long long p = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
     if (p >= geo.P) return;
-    const int tw = static_cast<int>(p % geo.TW);
-    const int th = static_cast<int>((p / geo.TW) % geo.TH);
-    const long long n = p / (static_cast<long long>(geo.TW) * geo.TH);
+    int tw, th;
+    long long n;
+    decode_tile(geo, p, n, th, tw);
     float v[CP][A2];
 #pragma unroll
     for (int c = 0; c < CP; ++c) {

@@ -95,3 +95,18 @@ def test_product_package_does_not_import_oracle():
             if f.endswith((".py", ".cu", ".cuh", ".h")):
                 src = open(os.path.join(dirpath, f)).read()
                 assert "import oracle" not in src and "from oracle" not in src and "conv_oracle" not in src, f
+
+
+def test_choose_tile_is_host_arithmetic(binding):
+    # few-channel layers -> F(2x2); weight-heavy layers -> F(2x2); activation-heavy layers -> F(4x4)
+    assert binding.sdwino_choose_tile(2, 4, 64, 64, 320) == 2
+    assert binding.sdwino_choose_tile(2, 320, 64, 64, 4) == 2
+    assert binding.sdwino_choose_tile(2, 1280, 8, 8, 1280) == 2
+    assert binding.sdwino_choose_tile(2, 2560, 16, 16, 1280) == 2
+    assert binding.sdwino_choose_tile(2, 320, 64, 64, 320) == 4
+    assert binding.sdwino_choose_tile(1, 512, 256, 256, 512) == 4
+    # threshold: 2 * tiles * (C + K) >= K * C with tiles = N * ceil(H/2) * ceil(W/2)
+    assert binding.sdwino_choose_tile(1, 64, 7, 7, 64) == 4       # 2*16*128 = 4096 >= 4096
+    assert binding.sdwino_choose_tile(1, 64, 6, 7, 64) == 2       # 2*12*128 = 3072 <  4096
+    with pytest.raises(binding.SdwinoError):
+        binding.sdwino_choose_tile(0, 1, 1, 1, 1)
