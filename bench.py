@@ -402,7 +402,7 @@ def run_ours(args):
             out_bytes += 2.0 * a2 * L.K * P + yb     # read M, write y
         fused_ms += pl["fused"]
     gemm_launches = sum(pl["launches"] for pl in per_layer) / prof_steps
-    achieved = gemm_flops / (gemm_ms * 1e-3) / 1e12
+    achieved = gemm_flops / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0   # a subset of fused-kernel layers
     roofline = {
         "kernel": "wino_gemm_kernel", "bound": "tensor", "achieved": round(achieved, 1), "peak": tpeak,
         "unit": "TFLOP/s", "frac": round(achieved / tpeak, 4),
@@ -410,15 +410,19 @@ def run_ours(args):
                     if (args.workload == WORKLOAD and not args.layers) else None),
         "traffic_unit": "bytes per launch (ncu dram read + write, L2 left warm)",
         "peak_source": f"{peak_kind} (cuBLAS bf16 burst; fp16 has the same nominal rate)",
-        "launches_per_step": gemm_launches, "avg_launch_us": round(gemm_ms * 1e3 / gemm_launches, 2),
+        "launches_per_step": gemm_launches,
+        "avg_launch_us": round(gemm_ms * 1e3 / gemm_launches, 2) if gemm_launches else None,
         "algorithmic_flops_per_step": gemm_flops,
-        "share_of_step": round(gemm_ms / (gemm_ms + in_ms + out_ms + fused_ms), 3),
+        "share_of_step": round(gemm_ms / max(gemm_ms + in_ms + out_ms + fused_ms, 1e-12), 3),
     }
+    def gbs(nbytes, ms):
+        return nbytes / (ms * 1e-3) / 1e9 if ms > 0 else 0.0
+
     transforms = {
-        "input_transform": {"gbs": round(in_bytes / (in_ms * 1e-3) / 1e9, 1), "frac_of_hbm_peak":
-                            round(in_bytes / (in_ms * 1e-3) / 1e9 / hpeak, 3), "ms_per_step": round(in_ms, 4)},
-        "output_transform": {"gbs": round(out_bytes / (out_ms * 1e-3) / 1e9, 1), "frac_of_hbm_peak":
-                             round(out_bytes / (out_ms * 1e-3) / 1e9 / hpeak, 3), "ms_per_step": round(out_ms, 4)},
+        "input_transform": {"gbs": round(gbs(in_bytes, in_ms), 1), "frac_of_hbm_peak":
+                            round(gbs(in_bytes, in_ms) / hpeak, 3), "ms_per_step": round(in_ms, 4)},
+        "output_transform": {"gbs": round(gbs(out_bytes, out_ms), 1), "frac_of_hbm_peak":
+                             round(gbs(out_bytes, out_ms) / hpeak, 3), "ms_per_step": round(out_ms, 4)},
         "filter_transform_once_per_weight": {"ms": round(ft_ms, 4), "gbs": round(ft_bytes / (ft_ms * 1e-3) / 1e9, 1),
                                              "frac_of_hbm_peak": round(ft_bytes / (ft_ms * 1e-3) / 1e9 / hpeak, 3)},
         "hbm_peak_gbs": hpeak, "peak_source": peak_kind,

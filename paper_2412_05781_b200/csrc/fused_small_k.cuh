@@ -360,7 +360,7 @@ fused_small_k_kernel(const __grid_constant__ CUtensorMap tmU, const __half* __re
                         t[0][nu] = o[0];
                         t[1][nu] = o[1];
                     }
-                    const float b = bias ? __half2float(__ldg(bias + k0 + kc + kk)) : 0.f;
+                    const float b = load_bias(bias, k0 + kc + kk);
                     float o0[2], o1[2];
                     mat_apply<2, 4>(typename Wm::At{}, t[0], o0);
                     mat_apply<2, 4>(typename Wm::At{}, t[1], o1);

@@ -354,6 +354,25 @@ int launch_fused_small_k(const __half* x, const void* wT, const __half* bias, __
     return e == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
 }
 
+// F(2x2,3x3) layers with at most 8 input channels: one warp-MMA kernel (see fused_small_c_mma_kernel).
+int launch_fused_small_c_mma(const __half* x, const __half* U, const __half* bias, __half* y, const TileGeom& geo, int C,
+                             int K, int Kb, cudaStream_t st) {
+    const int sms = sm_count();
+    if (sms <= 0) return SDWINO_ERR_CUDA;
+    const long long groups = (geo.P + 7) / 8;
+    const long long blocks_x = (groups + 3) / 4;
+    // about four blocks per SM: split the output-channel blocks over grid.y until there are enough
+    long long ksplit = (static_cast<long long>(sms) * 4 + blocks_x - 1) / blocks_x;
+    ksplit = ksplit < 1 ? 1 : (ksplit > Kb ? Kb : ksplit);
+    const int kb_per_block = static_cast<int>((Kb + ksplit - 1) / ksplit);
+    dim3 grid(static_cast<unsigned>(blocks_x), static_cast<unsigned>((Kb + kb_per_block - 1) / kb_per_block));
+    ProfScope prof(KIND_FUSED, st);
+    const cudaError_t e = launch_pdl(fused_small_c_mma_kernel, grid, dim3(128), 0, st, 0, x, U, bias, y, geo, C, K, Kb,
+                                     kb_per_block);
+    g_launches.fetch_add(1);
+    return e == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
+}
+
 // Shape of the GEMM launch: CTA pairs or single CTAs, and the output channels per tile (UMMA N, a
 // multiple of 16 up to 256).  The candidate with the smallest modelled time wins: a tile costs its
 // pipeline stages, each limited by the tensor pipe (2 n cycles per stage) or by the bytes the CTA must
@@ -445,8 +464,7 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
         const __half* bh = static_cast<const __half*>(bias);
         __half* yh = static_cast<__half*>(y);
         if (tile == 4) return launch_fused_small_c<4, 4>(xh, uh, bh, yh, geo, C, K, pl.Kb, pl.Cb, st);
-        if (C <= 4) return launch_fused_small_c<2, 4>(xh, uh, bh, yh, geo, C, K, pl.Kb, pl.Cb, st);
-        return launch_fused_small_c<2, 8>(xh, uh, bh, yh, geo, C, K, pl.Kb, pl.Cb, st);
+        return launch_fused_small_c_mma(xh, uh, bh, yh, geo, C, K, pl.Kb, st);
     }
 
     // workspace: V[a2][C][pc] then M[a2][K][pc]; pc is a multiple of 128 elements, so every row starts

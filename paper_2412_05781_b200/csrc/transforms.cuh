@@ -72,6 +72,14 @@ template <> struct Wino<4> {
     };
 };
 
+// Optional bias (NULL = 0).  A plain load under the null check: a read-only-path load (__ldg) may be
+// hoisted above the check by the compiler, and then faults on the null pointer.
+__device__ __forceinline__ float load_bias(const __half* bias, int k) {
+    float b = 0.f;
+    if (bias != nullptr) b = __half2float(bias[k]);
+    return b;
+}
+
 // out[i] = sum_j coef[i][j] * in[j] with compile-time coefficients: zero terms vanish and
 // unit terms become adds once the loops are unrolled.
 template <int R, int Cn, typename MatT>
@@ -279,7 +287,7 @@ output_transform_kernel(const __half* __restrict__ Mws, const __half* __restrict
     int tw, th;
     long long n;
     decode_tile(geo, p, n, th, tw);
-    const float b = bias ? __half2float(__ldg(bias + k)) : 0.f;
+    const float b = load_bias(bias, k);
     __half* img = y + (n * K + k) * static_cast<long long>(geo.H) * geo.W;
     const int i0 = M * th, j0 = M * tw;
     const bool vec_ok = ((geo.W & 1) == 0) && ((reinterpret_cast<uintptr_t>(y) & 3) == 0);
@@ -423,8 +431,7 @@ input_transform_vec_kernel(const __half* __restrict__ x, __half* __restrict__ V,
             for (int xi = 0; xi < A; ++xi)
                 *reinterpret_cast<uint32_t*>(dst + (xi * A + nu) * plane) = pack2(o[xi].x, o[xi].y);
         }
-        return;
-    }
+    } else {
     float e[A][TPT][A];  // rows transformed along the columns: e[r][t][nu] = sum_s Bt[nu][s] d[r][s]
     if (p < geo.P) {
         int tw, th;
@@ -494,6 +501,7 @@ input_transform_vec_kernel(const __half* __restrict__ x, __half* __restrict__ V,
             }
         }
     }
+    }   // M != 4
 }
 
 template <int M, int TPT>
@@ -531,7 +539,7 @@ output_transform_vec_kernel(const __half* __restrict__ Mws, const __half* __rest
         int tw, th;
         long long n;
         decode_tile(geo, p, n, th, tw);
-        const float b = bias ? __half2float(__ldg(bias + k)) : 0.f;
+        const float b = load_bias(bias, k);
         __half* img = y + (n * K + k) * static_cast<long long>(geo.H) * geo.W;
         const int i0 = M * th, j0 = M * tw;
 #pragma unroll
@@ -546,8 +554,7 @@ output_transform_vec_kernel(const __half* __restrict__ Mws, const __half* __rest
             w.w = pack2(o[2].y + b, o[3].y + b);
             *reinterpret_cast<uint4*>(img + static_cast<long long>(i0 + i) * geo.W + j0) = w;
         }
-        return;
-    }
+    } else {
     float mm[A][A][TPT];
 #pragma unroll
     for (int r = 0; r < A; ++r)
@@ -566,7 +573,7 @@ output_transform_vec_kernel(const __half* __restrict__ Mws, const __half* __rest
     int tw, th;
     long long n;
     decode_tile(geo, p, n, th, tw);
-    const float b = bias ? __half2float(__ldg(bias + k)) : 0.f;
+    const float b = load_bias(bias, k);
     __half* img = y + (n * K + k) * static_cast<long long>(geo.H) * geo.W;
     const int i0 = M * th, j0 = M * tw;
     float out[M][8];  // M output rows of 8 pixels
@@ -600,6 +607,7 @@ output_transform_vec_kernel(const __half* __restrict__ Mws, const __half* __rest
         w.w = pack2(out[i][6], out[i][7]);
         *reinterpret_cast<uint4*>(img + static_cast<long long>(i0 + i) * geo.W + j0) = w;
     }
+    }   // M != 4
 }
 
 
@@ -701,7 +709,7 @@ fused_small_c_kernel(const __half* __restrict__ x, const __half* __restrict__ U,
             for (int i = 0; i < M; ++i) tt[i][s2] = o[i];
         }
         const int k = k0 + kk;
-        const float b = bias ? __half2float(__ldg(bias + k)) : 0.f;
+        const float b = load_bias(bias, k);
         __half* img = y + (n * K + k) * static_cast<long long>(geo.H) * geo.W;
 #pragma unroll
         for (int i = 0; i < M; ++i) {
@@ -717,6 +725,193 @@ fused_small_c_kernel(const __half* __restrict__ x, const __half* __restrict__ U,
                 } else {
                     if (oj0 + j < geo.W) rowp[j] = h0;
                     if (oj0 + j + 1 < geo.W) rowp[j + 1] = h1;
+                }
+            }
+        }
+    }
+}
+
+
+// ---------------------------------------------------------------------------------------
+// The same for F(2x2,3x3) on the warp-level tensor-core path: with C <= 8 the contraction per position
+// is exactly one m16n8k8 MMA (16 output channels x 8 tiles x 8 input channels), and its fragment layout
+// needs no data exchange at all.  A warp owns 16 output channels and groups of 8 consecutive tiles:
+//   * lane (g = lane / 4, t = lane % 4) transforms tile g of the group for channels 2t and 2t+1 and packs
+//     the pair as fp16 -- for every position that IS its B fragment (rows 2t, 2t+1 of column g);
+//   * its A fragment per position is two 32-bit loads of the transformed filter (rows g and g+8, channels
+//     2t, 2t+1 of the 16 x 64 block; channels past C and rows past K are stored as zeros);
+//   * after the 16 MMAs it holds all 16 positions of output channels g, g+8 for tiles 2t, 2t+1, so the
+//     output transform, bias and store stay in the lane.
+// About 2 instructions per output value against 90 for the scalar kernel above (which stays for F(4x4):
+// 36 positions x 4 accumulators would not fit the registers).  tcgen05 is not used here: its smallest tile
+// (64 x 8 x 16 per instruction, operands staged in shared memory) does not pay for a contraction of 4.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ void mma_m16n8k8_f16f32(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t b0) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k8.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5}, {%6}, {%0, %1, %2, %3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(b0));
+}
+
+constexpr int FUSED_C_MAX = 8;
+
+// Grid: x = groups of 8 tiles, four per block (one per warp); y = chunks of `kb_per_block` blocks of 16 output
+// channels.  A warp transforms its 8 tiles once and then walks the chunk's output-channel blocks.
+__global__ void __launch_bounds__(128)
+fused_small_c_mma_kernel(const __half* __restrict__ x, const __half* __restrict__ U, const __half* __restrict__ bias,
+                         __half* __restrict__ y, TileGeom geo, int C, int K, int Kb, int kb_per_block) {
+    using Wm = Wino<2>;
+    pdl_launch_dependents();
+    pdl_wait();
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const int g = lane >> 2, t = lane & 3;
+    const long long hw = static_cast<long long>(geo.H) * geo.W;
+    const long long num_groups = (geo.P + 7) / 8;
+    const long long grp = static_cast<long long>(blockIdx.x) * 4 + warp;
+    if (grp >= num_groups) return;   // warp-uniform; the kernel has no block-wide barrier
+
+    // ---- input transform: lane (g, t) transforms tile g of the group for channel t (and t + 4 if C > 4) ----
+    uint32_t bfrag[16];
+    {
+        const long long p = grp * 8 + g;
+        int tw = 0, th = 0;
+        long long n = 0;
+        const bool p_ok = p < geo.P;
+        if (p_ok) decode_tile(geo, p, n, th, tw);
+        const int i0 = 2 * th - 1, j0 = 2 * tw - 1;
+        uint32_t packed[2][16];   // per round: (V[c even], V[c odd]) of tile g, valid in the even-channel lanes
+#pragma unroll
+        for (int round = 0; round < 2; ++round) {
+            const int c = 4 * round + t;
+            float d[4][4];
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+#pragma unroll
+                for (int s2 = 0; s2 < 4; ++s2) d[r][s2] = 0.f;
+            if (p_ok && c < C) {       // round 1 is skipped by every lane when C <= 4
+                const __half* img = x + (n * C + c) * hw;
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    const int i = i0 + r;
+                    if (i < 0 || i >= geo.H) continue;
+                    const __half* rowp = img + static_cast<long long>(i) * geo.W;
+#pragma unroll
+                    for (int s2 = 0; s2 < 4; ++s2) {
+                        const int j = j0 + s2;
+                        if (j >= 0 && j < geo.W) d[r][s2] = __half2float(rowp[j]);
+                    }
+                }
+            }
+            float e[4][4];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) mat_apply<4, 4>(typename Wm::Bt{}, d[r], e[r]);   // along the columns
+#pragma unroll
+            for (int nu = 0; nu < 4; ++nu) {
+                float col[4], o[4];
+#pragma unroll
+                for (int r = 0; r < 4; ++r) col[r] = e[r][nu];
+                mat_apply<4, 4>(typename Wm::Bt{}, col, o);
+#pragma unroll
+                for (int xi = 0; xi < 4; ++xi) {
+                    const float mine = o[xi];
+                    const float other = __shfl_xor_sync(0xffffffffu, mine, 1);   // channel c ^ 1 of the same tile
+                    packed[round][xi * 4 + nu] = pack2(mine, other);            // meaningful where c is even
+                }
+            }
+            if (C <= 4) break;   // uniform
+        }
+        // B fragment of lane (g, t): channels 2t, 2t+1 of tile g = the packed pair of lane (g, (2t) & 3), round t >> 1
+        const int src = (g << 2) | ((2 * t) & 3);
+#pragma unroll
+        for (int pos = 0; pos < 16; ++pos) {
+            const uint32_t r0 = __shfl_sync(0xffffffffu, packed[0][pos], src);
+            uint32_t r1 = 0u;
+            if (C > 4) r1 = __shfl_sync(0xffffffffu, packed[1][pos], src);      // uniform branch
+            bfrag[pos] = t < 2 ? r0 : r1;
+        }
+    }
+
+    // ---- this lane's output tiles: tiles 2t and 2t+1 of the group ----
+    long long out_off[2];       // element offset of (n, k = 0, 2*th, 2*tw); -1 = tile past the end
+    bool row1_ok[2], col1_ok[2];
+#pragma unroll
+    for (int jt = 0; jt < 2; ++jt) {
+        const long long p = grp * 8 + 2 * t + jt;
+        out_off[jt] = -1;
+        row1_ok[jt] = col1_ok[jt] = false;
+        if (p < geo.P) {
+            int tw, th;
+            long long n;
+            decode_tile(geo, p, n, th, tw);
+            out_off[jt] = n * K * hw + static_cast<long long>(2 * th) * geo.W + 2 * tw;
+            row1_ok[jt] = 2 * th + 1 < geo.H;
+            col1_ok[jt] = 2 * tw + 1 < geo.W;
+        }
+    }
+    const bool vec_ok = ((geo.W & 1) == 0) && ((reinterpret_cast<uintptr_t>(y) & 3) == 0);
+    // W % 4 == 0 makes TW even, so tiles 2t and 2t+1 of a group always share a tile row
+    const bool pair_ok = ((geo.W & 3) == 0) && ((reinterpret_cast<uintptr_t>(y) & 7) == 0) && out_off[1] >= 0;
+
+    const int kb_end = min(Kb, static_cast<int>(blockIdx.y + 1) * kb_per_block);
+    const size_t plane_w = static_cast<size_t>(Kb) * 512;   // one position of U, in 32-bit words
+    for (int kb = blockIdx.y * kb_per_block; kb < kb_end; ++kb) {
+        // A fragments: U[pos][kb][0][row][c], rows g and g+8, channels 2t, 2t+1 (zeros past K and C)
+        const uint32_t* Uw = reinterpret_cast<const uint32_t*>(U + (static_cast<size_t>(kb) * 16 + g) * 64 + 2 * t);
+        float acc[16][4];   // acc[pos] = {M[g][2t], M[g][2t+1], M[g+8][2t], M[g+8][2t+1]}
+#pragma unroll
+        for (int pos = 0; pos < 16; ++pos) {
+            acc[pos][0] = acc[pos][1] = acc[pos][2] = acc[pos][3] = 0.f;
+            const uint32_t a0 = __ldg(Uw + pos * plane_w);
+            const uint32_t a1 = __ldg(Uw + pos * plane_w + 8 * 32);
+            mma_m16n8k8_f16f32(acc[pos], a0, a1, bfrag[pos]);
+        }
+#pragma unroll
+        for (int hk = 0; hk < 2; ++hk) {
+            const int k = kb * 16 + g + 8 * hk;
+            if (k >= K) continue;
+            const float b = load_bias(bias, k);
+            uint32_t row0[2], row1[2];   // packed output pixels of the two tiles: first and second output row
+            float o0[2][2], o1[2][2];
+#pragma unroll
+            for (int jt = 0; jt < 2; ++jt) {
+                float tt[2][4];
+#pragma unroll
+                for (int nu = 0; nu < 4; ++nu) {
+                    float col[4], o[2];
+#pragma unroll
+                    for (int xi = 0; xi < 4; ++xi) col[xi] = acc[xi * 4 + nu][2 * hk + jt];
+                    mat_apply<2, 4>(typename Wm::At{}, col, o);
+                    tt[0][nu] = o[0];
+                    tt[1][nu] = o[1];
+                }
+                mat_apply<2, 4>(typename Wm::At{}, tt[0], o0[jt]);
+                mat_apply<2, 4>(typename Wm::At{}, tt[1], o1[jt]);
+                row0[jt] = pack2(o0[jt][0] + b, o0[jt][1] + b);
+                row1[jt] = pack2(o1[jt][0] + b, o1[jt][1] + b);
+            }
+            if (pair_ok) {
+                // the lane's two tiles are neighbours in one tile row: 4 pixels = one 8-byte store per output row,
+                // and the four lanes of an output channel complete a 32-byte sector
+                __half* q = y + out_off[0] + k * hw;
+                *reinterpret_cast<uint2*>(q) = make_uint2(row0[0], row0[1]);
+                if (row1_ok[0]) *reinterpret_cast<uint2*>(q + geo.W) = make_uint2(row1[0], row1[1]);
+                continue;
+            }
+#pragma unroll
+            for (int jt = 0; jt < 2; ++jt) {
+                if (out_off[jt] < 0) continue;
+                __half* q = y + out_off[jt] + k * hw;
+                if (vec_ok) {           // W even: both columns exist and q is 4-byte aligned
+                    *reinterpret_cast<uint32_t*>(q) = row0[jt];
+                    if (row1_ok[jt]) *reinterpret_cast<uint32_t*>(q + geo.W) = row1[jt];
+                } else {
+                    q[0] = __float2half_rn(o0[jt][0] + b);
+                    if (col1_ok[jt]) q[1] = __float2half_rn(o0[jt][1] + b);
+                    if (row1_ok[jt]) {
+                        q[geo.W] = __float2half_rn(o1[jt][0] + b);
+                        if (col1_ok[jt]) q[geo.W + 1] = __float2half_rn(o1[jt][1] + b);
+                    }
                 }
             }
         }
