@@ -418,6 +418,14 @@ def run_ours(args):
     def gbs(nbytes, ms):
         return nbytes / (ms * 1e-3) / 1e9 if ms > 0 else 0.0
 
+    # the whole step against the per-layer roofline max(tensor time, mandatory HBM bytes / bandwidth), both at
+    # the measured peaks: what an ideal implementation of each layer would need, summed over the sweep
+    roof_us_sum = sum(r["roof_us"] for r in layer_rows)
+    roofline["step_vs_layer_rooflines"] = {
+        "sum_of_layer_rooflines_us": round(roof_us_sum, 1), "step_us": round(ms_step * 1e3, 1),
+        "frac": round(roof_us_sum / (ms_step * 1e3), 3),
+        "hbm_bound_layers": sum(1 for r in layer_rows if r["bound"] == "hbm"), "layers": len(layer_rows)}
+
     transforms = {
         "input_transform": {"gbs": round(gbs(in_bytes, in_ms), 1), "frac_of_hbm_peak":
                             round(gbs(in_bytes, in_ms) / hpeak, 3), "ms_per_step": round(in_ms, 4)},

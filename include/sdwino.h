@@ -49,8 +49,9 @@ const char *sdwino_status_string(int status);
  *
  * sdwino_filter_bytes: bytes the caller must allocate for wT (0 on bad arguments).
  * sdwino_filter_transform: w is fp16 [K][C][3][3]; wT receives fp16 U laid out as
- *   [a*a][Kb][Cb][16][64] with a = tile+2, Kb = ceil(K/16), Cb = ceil(C/64): blocks of 16 output
- *   channels x 64 input channels (2 KB contiguous each), position index xi*a+nu, zero in the padding.  wT must be 1024-byte aligned (a cudaMalloc
+ *   [a*a][Cb][Kb][16][64] with a = tile+2, Kb = ceil(K/16), Cb = ceil(C/64): blocks of 16 output
+ *   channels x 64 input channels (2 KB contiguous each; the blocks of consecutive output channels are
+ *   adjacent), position index xi*a+nu, zero in the padding.  wT must be 1024-byte aligned (a cudaMalloc
  *   base is).  wT depends on `tile`; pass the same tile to sdwino_conv3x3.  Done once
  *   per weight; the caller owns both buffers.
  */

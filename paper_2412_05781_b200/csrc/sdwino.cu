@@ -184,7 +184,7 @@ bool encode_map_uncached(CUtensorMap* m, const void* base, uint64_t d0, uint64_t
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
-// The blocked filter tensor U[pos][Kb][Cb][16][64] as a 5-D map whose box is `kblocks` blocks of 16 rows
+// The blocked filter tensor U[pos][Cb][Kb][16][64] as a 5-D map (dimension order {c, k, c-block, k-block, pos}) whose box is `kblocks` blocks of 16 rows
 // of `posbox` consecutive transform positions (`krows` < 16: only the first rows of a block).
 bool encode_filter_map(CUtensorMap* m, const void* base, uint64_t Cb, uint64_t Kb, uint64_t npos, uint32_t kblocks,
                        uint32_t posbox = 1, uint32_t krows = 16) {
@@ -197,7 +197,7 @@ bool encode_filter_map(CUtensorMap* m, const void* base, uint64_t Cb, uint64_t K
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return false;
     cuuint64_t dims[5] = {64, 16, Cb, Kb, npos};
-    cuuint64_t strides[4] = {128, 2048, Cb * 2048, Kb * Cb * 2048};
+    cuuint64_t strides[4] = {128, 2048 * Kb, 2048, Kb * Cb * 2048};   // memory order [pos][Cb][Kb][16][64]
     cuuint32_t box[5] = {64, krows, 1, kblocks, posbox};
     cuuint32_t estr[5] = {1, 1, 1, 1, 1};
     if (fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 5, const_cast<void*>(base), dims, strides, box, estr,

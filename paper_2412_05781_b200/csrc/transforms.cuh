@@ -102,10 +102,10 @@ __device__ __forceinline__ void mat_apply(MatT coef, const float (&in)[Cn], floa
 
 // ---------------------------------------------------------------------------------------
 // Filter preprocess.  U is stored in blocks of 16 output channels x 64 input channels,
-//   U[a*a][Kb][Cb][16][64]   (Kb = ceil(K/16), Cb = ceil(C/64), zeros in the padding),
-// so that the [n_tile k][64 c] operand box of one GEMM pipeline stage is n_tile/16 contiguous 2 KB
-// pieces of DRAM instead of n_tile separate 128-byte rows (the weights are the one operand that is
-// streamed from HBM).  One thread per (k, c) of the padded plane.
+//   U[a*a][Cb][Kb][16][64]   (Kb = ceil(K/16), Cb = ceil(C/64), zeros in the padding),
+// with the blocks of consecutive output channels next to each other, so that the [n_tile k][64 c]
+// operand box of one GEMM pipeline stage is ONE contiguous piece of n_tile/16 x 2 KB of DRAM instead of
+// n_tile separate 128-byte rows (the weights are the one operand that is streamed from HBM).  One thread per (k, c) of the padded plane.
 // Writes all a*a positions.
 // ---------------------------------------------------------------------------------------
 template <int M>
@@ -136,7 +136,7 @@ filter_transform_kernel(const __half* __restrict__ w, __half* __restrict__ U, in
         for (int i = 0; i < A; ++i) t[i][s] = o[i];
     }
     const size_t plane = static_cast<size_t>(Kb) * Cb * 1024;   // one position: Kb x Cb blocks of 16 x 64
-    __half* dst = U + ((static_cast<size_t>(k >> 4) * Cb + (c >> 6)) * 16 + (k & 15)) * 64 + (c & 63);
+    __half* dst = U + ((static_cast<size_t>(c >> 6) * Kb + (k >> 4)) * 16 + (k & 15)) * 64 + (c & 63);
 #pragma unroll
     for (int i = 0; i < A; ++i) {
         float o[A];
@@ -633,7 +633,7 @@ fused_small_c_kernel(const __half* __restrict__ x, const __half* __restrict__ U,
     pdl_launch_dependents();
     pdl_wait();
     const int k0 = blockIdx.y * FUSED_KC;
-    // stage the filter chunk: U[pos][Kb][Cb][16][64], this layer has Cb == 1
+    // stage the filter chunk: U[pos][Cb][Kb][16][64], this layer has Cb == 1
     const size_t plane = static_cast<size_t>(Kb) * Cb * 1024;
     for (int i = threadIdx.x; i < FUSED_KC * CP * A2; i += blockDim.x) {
         const int pos = i % A2;

@@ -77,7 +77,7 @@ struct GemmParams {
 };
 
 // tmV: fp16 [pos][C][Pstride]   box {64 p, 64 c, 1},      128B swizzle  (A operand; rows c >= C read as 0)
-// tmU: fp16 [pos][Kb][Cb][16][64] box {64 c, 16 k, 1, n_tile/16, 1}, 128B swizzle (B operand: n_tile rows of 128
+// tmU: fp16 [pos][Cb][Kb][16][64] box {64 c, 16 k, 1, n_tile/16, 1}, 128B swizzle (B operand: n_tile rows of 128
 //      bytes in k order; blocks past Kb read as 0)
 // tmM: fp16 [pos][K][Pstride]   box {128 p, epi_rows k, 1}, no swizzle  (result; rows k >= K are clipped)
 template <int CTAS>

@@ -223,8 +223,8 @@ def test_filter_transform_matches_oracle(B, KC, tile):
     w = (torch.randn(K, C, 3, 3, generator=g) / (9 * C) ** 0.5).half()
     wT = B.sdwino_filter_transform(w.cuda(), tile)
     Kb, Cb = -(-K // 16), -(-C // 64)
-    # U[a*a][Kb][Cb][16][64]  ->  [a*a][Kb*16][Cb*64]
-    U = wT.view(torch.float16)[:a * a * Kb * Cb * 1024].view(a * a, Kb, Cb, 16, 64).permute(0, 1, 3, 2, 4)
+    # U[a*a][Cb][Kb][16][64]  ->  [a*a][Kb*16][Cb*64]
+    U = wT.view(torch.float16)[:a * a * Kb * Cb * 1024].view(a * a, Cb, Kb, 16, 64).permute(0, 2, 3, 1, 4)
     U = U.reshape(a * a, Kb * 16, Cb * 64).cpu()
     Uo = oracle.filter_transform(w.numpy(), tile, points=None if tile == 2 else F4_POINTS)
     Uo = torch.from_numpy(Uo.reshape(K, C, a * a).transpose(2, 0, 1).copy())
