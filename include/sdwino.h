@@ -136,6 +136,15 @@ int sdwino_conv3x3_host(const void *x_host, const void *wT, const void *bias_hos
  */
 int sdwino_last_device_status(void *stream);
 
+/*
+ * Self-test of that mechanism: launches one thread that waits on a barrier nothing signals, with the
+ * given limit (1 ns .. 10 ms, else SDWINO_ERR_INVALID_ARG).  The kernel returns normally after about
+ * the limit (the timer is sampled every few thousand polls, so up to ~1 ms later) and
+ * sdwino_last_device_status then reports SDWINO_ERR_TIMEOUT once.  Nothing else is touched: the
+ * context stays usable and later calls are unaffected.
+ */
+int sdwino_selftest_wait_timeout(unsigned long long limit_ns, void *stream);
+
 /* Kernel launches made by this library in the calling process so far (all entry points). */
 unsigned long long sdwino_launch_count(void);
 

@@ -22,6 +22,7 @@ EXPORTS = [
     "sdwino_conv3x3_ws", "sdwino_host_staging_bytes", "sdwino_conv3x3_host",
     "sdwino_last_device_status", "sdwino_launch_count", "sdwino_profile_enable", "sdwino_profile_collect",
     "sdwino_profile_records", "sdwino_set_gemm_shape", "sdwino_conv3x3_static", "sdwino_set_fused_min_tiles", "sdwino_choose_tile",
+    "sdwino_selftest_wait_timeout",
 ]
 
 KERNEL_KINDS = ("filter_transform", "input_transform", "wino_gemm", "output_transform", "fused")
@@ -67,6 +68,8 @@ def _load() -> ctypes.CDLL:
     lib.sdwino_profile_records.argtypes = [ctypes.POINTER(i), ctypes.POINTER(ctypes.c_float), i, i]
     lib.sdwino_set_gemm_shape.restype = i
     lib.sdwino_set_gemm_shape.argtypes = [i, i]
+    lib.sdwino_selftest_wait_timeout.restype = i
+    lib.sdwino_selftest_wait_timeout.argtypes = [ctypes.c_ulonglong, vp]
     lib.sdwino_choose_tile.restype = i
     lib.sdwino_choose_tile.argtypes = [i, i, i, i, i]
     lib.sdwino_set_fused_min_tiles.restype = i
@@ -125,6 +128,11 @@ def sdwino_launch_count() -> int:
 
 def sdwino_last_device_status(stream: Optional[torch.cuda.Stream] = None) -> int:
     return int(lib.sdwino_last_device_status(_stream_ptr(stream)))
+
+
+def sdwino_selftest_wait_timeout(limit_ns: int, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Launch the bounded-wait self-test; sdwino_last_device_status() reports ERR_TIMEOUT afterwards."""
+    _check(lib.sdwino_selftest_wait_timeout(limit_ns, _stream_ptr(stream)), "sdwino_selftest_wait_timeout")
 
 
 def sdwino_set_gemm_shape(ctas: int = 0, n_tile: int = 0) -> None:

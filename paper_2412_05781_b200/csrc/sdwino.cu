@@ -680,6 +680,15 @@ int sdwino_last_device_status(void* stream) {
 
 unsigned long long sdwino_launch_count(void) { return g_launches.load(); }
 
+int sdwino_selftest_wait_timeout(unsigned long long limit_ns, void* stream) {
+    if (limit_ns == 0 || limit_ns > 10000000ull) return SDWINO_ERR_INVALID_ARG;   // at most 10 ms
+    int* status = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&status), g_status_word) != cudaSuccess) return SDWINO_ERR_CUDA;
+    wait_timeout_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(status, limit_ns);
+    g_launches.fetch_add(1);
+    return cudaGetLastError() == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
+}
+
 }  // extern "C"
 
 namespace {

@@ -339,4 +339,18 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
     }
 }
 
+
+// Exercises the bounded wait and the status word without disturbing anything: one thread waits on a barrier
+// that nothing ever signals, gives up after `limit_ns`, records the timeout (where = 7) and returns.
+__global__ void wait_timeout_selftest_kernel(int* status_word, unsigned long long limit_ns) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(&bar, 1);
+        fence_barrier_init();
+        if (!mbar_wait_bounded(&bar, 0u, &abort_flag, limit_ns)) report_timeout(status_word, 7, 0);
+    }
+}
+
 }  // namespace sdw

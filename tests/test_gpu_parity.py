@@ -357,3 +357,27 @@ def test_non_default_stream_and_launch_counter(B):
     s.synchronize()
     assert B.sdwino_launch_count() - before == 4      # filter + input + GEMM + output
     assert torch.equal(y.cpu(), y_ref)
+
+
+def test_bounded_wait_reports_timeout_and_context_stays_usable(B):
+    # a wait that nothing satisfies gives up after its limit, the kernel returns normally, the host reads the
+    # status once, and the next convolution is unaffected
+    assert B.sdwino_last_device_status() == B.OK
+    B.sdwino_selftest_wait_timeout(1_000_000)            # 1 ms
+    assert B.sdwino_last_device_status() == B.ERR_TIMEOUT
+    assert B.sdwino_last_device_status() == B.OK          # cleared by the read
+    with pytest.raises(B.SdwinoError):
+        B.sdwino_selftest_wait_timeout(0)
+    with pytest.raises(B.SdwinoError):
+        B.sdwino_selftest_wait_timeout(20_000_000)        # more than 10 ms is refused
+    layer = ConvLayer(C=32, K=48, H=10, W=12, N=1)
+    x, w, b, y = _run(B, layer, 2, seed=2)
+    assert _rel_err(y, oracle.direct_conv3x3(x.numpy(), w.numpy(), b.numpy())) <= TOL_F2_REGRESSION
+
+
+@pytest.mark.parametrize("idx,tile", [(5, 2), (6, 4), (8, 4), (15, 2), (16, 2), (25, 2)])
+def test_sdxl_layers_sampled_channels(B, idx, tile):
+    # SDXL at 1024x1024: weight-streaming UNet layers, a large F4 layer, the few-channel layers at full size
+    layer = workloads.sdxl_1024()[idx]
+    err, edge = _sampled_check(B, layer, tile, nch=3, seed=idx)
+    assert err <= TOL and edge <= TOL, (layer.name, err, edge)
