@@ -200,8 +200,10 @@ input_transform_kernel(const __half* __restrict__ x, __half* __restrict__ V, Til
                        int p_count, long long Pstride) {
     using Wm = Wino<M>;
     constexpr int A = Wm::A;
-    pdl_launch_dependents();
+    // Wait first, release the GEMM second: once the GEMM runs, everything before this kernel has completed,
+    // which is what lets it fetch its filters (written at the latest by the kernel before this one) early.
     pdl_wait();
+    pdl_launch_dependents();
     const int pl = blockIdx.x * blockDim.x + threadIdx.x;  // chunk-local tile
     const int c = blockIdx.y;
     if (pl >= p_count) return;
@@ -373,8 +375,10 @@ input_transform_vec_kernel(const __half* __restrict__ x, __half* __restrict__ V,
                            long long p_begin, FastDiv gdiv, long long Pstride) {
     using Wm = Wino<M>;
     constexpr int A = Wm::A;
-    pdl_launch_dependents();
+    // Wait first, release the GEMM second: once the GEMM runs, everything before this kernel has completed,
+    // which is what lets it fetch its filters (written at the latest by the kernel before this one) early.
     pdl_wait();
+    pdl_launch_dependents();
     static_assert(M * TPT == 8, "one 16-byte row segment per thread");
     // flat index over (channel, group of TPT tiles): blocks stay full when a pass has few tiles
     const uint32_t idx = blockIdx.x * blockDim.x + threadIdx.x;   // below 2^31 (checked by the launcher)

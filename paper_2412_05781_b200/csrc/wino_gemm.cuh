@@ -143,8 +143,29 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
             const uint32_t full0_local = smem_u32(&full_bar[0]);
             const uint32_t full0 = CTAS == 2 ? map_to_cta(full0_local, 0) : full0_local;
             uint32_t sa = smem_base, fb = full0, fb_local = full0_local;
+            // The filters do not depend on the preceding kernel (the activation transform), and the kernel
+            // before that has completed by the time this one runs (the filter transform never releases its
+            // dependents early): the filter loads of the first ring-full of stages go out before the wait, so
+            // the weight stream from HBM starts while the activation transform is still running.
+            int pre = 0;
+            if constexpr (CTAS == 1) {
+                uint32_t sa_u = smem_base + L::A_BYTES, fb_u = full0;
+                for (int tile = worker; tile < num_tiles && pre < stages; tile += num_workers) {
+                    const int kt = (tile / prm.num_p_tiles) % prm.num_k_tiles;
+                    const int pos = tile / (prm.num_p_tiles * prm.num_k_tiles);
+                    const int k0 = kt * prm.n_tile;
+                    for (int c0 = 0; c0 < prm.C && pre < stages; c0 += GEMM_BLOCK_C) {
+                        mbar_arrive_expect_tx_a32(fb_u, tx_bytes);
+                        tma_load_5d_a32(sa_u, &tmU, fb_u, c0 >> 6, k0 >> 4, pos);
+                        sa_u += stage_bytes;
+                        fb_u += 8;
+                        ++pre;
+                    }
+                }
+            }
             pdl_wait();   // V is written by the preceding kernel
             int stage = 0;
+            int issued = 0;
             uint32_t phase = 0;
             bool ok = true;
             for (int tile = worker; tile < num_tiles && ok; tile += num_workers) {
@@ -154,6 +175,17 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
                 const int p0 = (pt * CTAS + static_cast<int>(cta_rank)) * GEMM_BLOCK_P;
                 const int k0 = kt * prm.n_tile + static_cast<int>(cta_rank) * b_rows;
                 for (int c0 = 0; c0 < prm.C; c0 += GEMM_BLOCK_C) {
+                    if (issued < pre) {
+                        // the barrier is armed and the filter box is on its way: add the two boxes of V
+                        tma_load_3d_a32(sa, &tmV, fb, p0, c0, pos);
+                        tma_load_3d_a32(sa + L::A_BOX_BYTES, &tmV, fb, p0 + 64, c0, pos);
+                        ++issued;
+                        sa += stage_bytes;
+                        fb += 8;
+                        fb_local += 8;
+                        if (++stage == stages) { stage = 0; phase ^= 1u; sa = smem_base; fb = full0; fb_local = full0_local; }
+                        continue;
+                    }
                     ok = mbar_wait_bounded(&empty_bar[stage], phase ^ 1u, abort_flag, GEMM_WAIT_LIMIT_NS);
                     if (!ok) { if (*abort_flag == 0) report_timeout(status_word, 1, cta_rank); break; }
                     if constexpr (CTAS == 2) {
