@@ -268,9 +268,17 @@ int launch_input(const __half* x, __half* V, const TileGeom& geo, int C, long lo
     cudaError_t e;
     const long long units = static_cast<long long>(p_count / TPT) * C;   // one thread each
     if (geo.W % 8 == 0 && aligned(x, 16) && units < (1ll << 31) - 128) {
-        dim3 grid(static_cast<unsigned>((units + 127) / 128));
-        e = launch_pdl(input_transform_vec_kernel<M, TPT>, grid, dim3(128), 0, st, 0, x, V, geo, C, p_begin,
-                       make_fastdiv(static_cast<uint32_t>(p_count / TPT)), Pstride);
+        if constexpr (M == 4) {
+            constexpr int CH = 1;   // channels per thread
+            const long long threads = static_cast<long long>(p_count / TPT) * ((C + CH - 1) / CH);
+            dim3 grid(static_cast<unsigned>((threads + 127) / 128));
+            e = launch_pdl(input_transform_f4_kernel<CH>, grid, dim3(128), 0, st, 0, x, V, geo, C, p_begin,
+                           make_fastdiv(static_cast<uint32_t>(p_count / TPT)), Pstride);
+        } else {
+            dim3 grid(static_cast<unsigned>((units + 127) / 128));
+            e = launch_pdl(input_transform_vec_kernel<M, TPT>, grid, dim3(128), 0, st, 0, x, V, geo, C, p_begin,
+                           make_fastdiv(static_cast<uint32_t>(p_count / TPT)), Pstride);
+        }
     } else {
         dim3 grid((p_count + 127) / 128, C);
         e = launch_pdl(input_transform_kernel<M>, grid, dim3(128), 0, st, 0, x, V, geo, C, p_begin, p_count, Pstride);

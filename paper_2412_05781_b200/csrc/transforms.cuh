@@ -508,6 +508,85 @@ input_transform_vec_kernel(const __half* __restrict__ x, __half* __restrict__ V,
     }   // M != 4
 }
 
+// F(4x4,3x3) activation transform, vector path: a thread owns 2 tiles (8 pixels of a tile row) and CH consecutive
+// channels.  Loads go into zero-initialised registers under precomputed border masks (no selects), and the
+// (tile 0, tile 1) operand pairs of the packed arithmetic are cut straight out of the loaded halves with byte
+// permutes.  The kernel is bound by instruction issue, so this is where its time goes: 3-10 % per layer over
+// the generic vector kernel.  CH = 1 is what runs: with 2 or 4 channels per thread the per-thread set-up is
+// amortised, but the serial load -> compute chain per channel and the lower thread count cost more (measured).
+template <int CH>
+__global__ void __launch_bounds__(128, 5)
+input_transform_f4_kernel(const __half* __restrict__ x, __half* __restrict__ V, TileGeom geo, int C, long long p_begin,
+                          FastDiv gdiv, long long Pstride) {
+    constexpr int A = 6;
+    pdl_wait();                 // see input_transform_vec_kernel: wait first, release the GEMM second
+    pdl_launch_dependents();
+    const uint32_t idx = blockIdx.x * blockDim.x + threadIdx.x;   // below 2^31 (checked by the launcher)
+    const int cg = static_cast<int>(fast_div(idx, gdiv));          // gdiv.d = groups of 2 tiles in this pass
+    const int c0 = cg * CH;
+    if (c0 >= C) return;
+    const int pl = static_cast<int>(idx - static_cast<uint32_t>(cg) * gdiv.d) * 2;
+    const long long p = p_begin + pl;
+    const long long hw = static_cast<long long>(geo.H) * geo.W;
+    const bool valid = p < geo.P;
+    int rowmask = 0;
+    bool left_ok = false, right_ok = false;
+    const __half* xp = x;
+    if (valid) {
+        int tw, th;
+        long long n;
+        decode_tile(geo, p, n, th, tw);
+        const int i0 = 4 * th - 1, j0 = 4 * tw;
+#pragma unroll
+        for (int r = 0; r < A; ++r)
+            if (i0 + r >= 0 && i0 + r < geo.H) rowmask |= 1 << r;
+        left_ok = j0 > 0;
+        right_ok = j0 + 8 < geo.W;
+        xp = x + (n * C + c0) * hw + static_cast<long long>(i0) * geo.W + j0;
+    }
+    const long long plane = static_cast<long long>(C) * Pstride;
+    __half* vp = V + static_cast<long long>(c0) * Pstride + pl;
+    const int cend = (C - c0) < CH ? (C - c0) : CH;
+    for (int cc = 0; cc < cend; ++cc) {
+        float2 e2[A][A];   // e2[r][nu]: rows transformed along the columns, (tile 0, tile 1)
+#pragma unroll
+        for (int r = 0; r < A; ++r) {
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+            uint32_t lw = 0u, rw = 0u;   // aligned words before / after the segment
+            if ((rowmask >> r) & 1) {
+                const __half* rp = xp + r * geo.W;
+                v = __ldg(reinterpret_cast<const uint4*>(rp));
+                if (left_ok) lw = __ldg(reinterpret_cast<const uint32_t*>(rp - 2));
+                if (right_ok) rw = __ldg(reinterpret_cast<const uint32_t*>(rp + 8));
+            }
+            // pixels: L = lw.hi, px0..px7 = v.x.lo, v.x.hi, ..., v.w.hi, R = rw.lo; tile 0 uses L..px4, tile 1 px3..R
+            uint32_t h[A];
+            h[0] = __byte_perm(lw, v.y, 0x7632);    // (L,   px3)
+            h[1] = __byte_perm(v.x, v.z, 0x5410);   // (px0, px4)
+            h[2] = __byte_perm(v.x, v.z, 0x7632);   // (px1, px5)
+            h[3] = __byte_perm(v.y, v.w, 0x5410);   // (px2, px6)
+            h[4] = __byte_perm(v.y, v.w, 0x7632);   // (px3, px7)
+            h[5] = __byte_perm(v.z, rw, 0x5410);    // (px4, R)
+            float2 d[A];
+#pragma unroll
+            for (int s2 = 0; s2 < A; ++s2) d[s2] = __half22float2(*reinterpret_cast<const __half2*>(&h[s2]));
+            bt4_packed(d, e2[r]);
+        }
+#pragma unroll
+        for (int nu = 0; nu < A; ++nu) {
+            float2 col[A], o[A];
+#pragma unroll
+            for (int r = 0; r < A; ++r) col[r] = e2[r][nu];
+            bt4_packed(col, o);
+#pragma unroll
+            for (int xi = 0; xi < A; ++xi)
+                *reinterpret_cast<uint32_t*>(vp + (xi * A + nu) * plane) = pack2(o[xi].x, o[xi].y);
+        }
+        xp += hw;
+        vp += Pstride;
+    }
+}
+
 template <int M, int TPT>
 __global__ void __launch_bounds__(128)
 output_transform_vec_kernel(const __half* __restrict__ Mws, const __half* __restrict__ bias, __half* __restrict__ y,
