@@ -386,56 +386,8 @@ input_transform_vec_kernel(const __half* __restrict__ x, __half* __restrict__ V,
     if (c >= C) return;
     const int pl = static_cast<int>(idx - static_cast<uint32_t>(c) * gdiv.d) * TPT;  // first chunk-local tile of this thread
     const long long p = p_begin + pl;
-    if constexpr (M == 4) {
-        // packed path: e2[r][nu] holds (tile 0, tile 1)
-        float2 e2[A][A];
-        if (p < geo.P) {
-            int tw, th;
-            long long n;
-            decode_tile(geo, p, n, th, tw);
-            const __half* img = x + (n * C + c) * static_cast<long long>(geo.H) * geo.W;
-            const int i0 = M * th - 1, j0 = M * tw;
-#pragma unroll
-            for (int r = 0; r < A; ++r) {
-                const int i = i0 + r;
-                float row[10];
-                if (i >= 0 && i < geo.H) {
-                    const __half* rp = img + static_cast<long long>(i) * geo.W + j0;
-                    const uint4 v = __ldg(reinterpret_cast<const uint4*>(rp));
-                    unpack2(v.x, row[1], row[2]);
-                    unpack2(v.y, row[3], row[4]);
-                    unpack2(v.z, row[5], row[6]);
-                    unpack2(v.w, row[7], row[8]);
-                    row[0] = j0 > 0 ? __half2float(__ldg(rp - 1)) : 0.f;
-                    row[9] = j0 + 8 < geo.W ? __half2float(__ldg(rp + 8)) : 0.f;
-                } else {
-#pragma unroll
-                    for (int s = 0; s < 10; ++s) row[s] = 0.f;
-                }
-                float2 d[A];
-#pragma unroll
-                for (int s = 0; s < A; ++s) d[s] = make_float2(row[s], row[M + s]);
-                bt4_packed(d, e2[r]);
-            }
-        } else {
-#pragma unroll
-            for (int r = 0; r < A; ++r)
-#pragma unroll
-                for (int s = 0; s < A; ++s) e2[r][s] = make_float2(0.f, 0.f);
-        }
-        const long long plane = static_cast<long long>(C) * Pstride;
-        __half* dst = V + static_cast<long long>(c) * Pstride + pl;
-#pragma unroll
-        for (int nu = 0; nu < A; ++nu) {
-            float2 col[A], o[A];
-#pragma unroll
-            for (int r = 0; r < A; ++r) col[r] = e2[r][nu];
-            bt4_packed(col, o);
-#pragma unroll
-            for (int xi = 0; xi < A; ++xi)
-                *reinterpret_cast<uint32_t*>(dst + (xi * A + nu) * plane) = pack2(o[xi].x, o[xi].y);
-        }
-    } else {
+    static_assert(M == 2, "F(4x4) has its own vector kernel (input_transform_f4_kernel)");
+    {
     float e[A][TPT][A];  // rows transformed along the columns: e[r][t][nu] = sum_s Bt[nu][s] d[r][s]
     if (p < geo.P) {
         int tw, th;
