@@ -117,6 +117,21 @@ __device__ __forceinline__ void tma_load_5d_a32(uint32_t smem_dst, const CUtenso
         "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(0), "r"(c2), "r"(c3), "r"(c4)
         : "memory");
 }
+// The same with an L2 eviction-priority hint.  The filters are streamed once per call: marking their lines
+// evict-first keeps them from pushing the L2-resident V and M of the pass out to DRAM.
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ void tma_load_5d_hint_a32(uint32_t smem_dst, const CUtensorMap* m, uint32_t bar, int c2, int c3,
+                                                     int c4, uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+        "[%0], [%1, {%3, %3, %4, %5, %6}], [%2], %7;" ::"r"(smem_dst),
+        "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(0), "r"(c2), "r"(c3), "r"(c4), "l"(policy)
+        : "memory");
+}
 // The same with a row offset inside the 16-row block (coordinate 1): {0, k row, c-block, k-block, position}.
 __device__ __forceinline__ void tma_load_5d_k_a32(uint32_t smem_dst, const CUtensorMap* m, uint32_t bar, int c1, int c2,
                                                   int c3, int c4) {

@@ -147,6 +147,7 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
             // before that has completed by the time this one runs (the filter transform never releases its
             // dependents early): the filter loads of the first ring-full of stages go out before the wait, so
             // the weight stream from HBM starts while the activation transform is still running.
+            const uint64_t u_policy = l2_policy_evict_first();
             int pre = 0;
             if constexpr (CTAS == 1) {
                 uint32_t sa_u = smem_base + L::A_BYTES, fb_u = full0;
@@ -156,7 +157,7 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
                     const int k0 = kt * prm.n_tile;
                     for (int c0 = 0; c0 < prm.C && pre < stages; c0 += GEMM_BLOCK_C) {
                         mbar_arrive_expect_tx_a32(fb_u, tx_bytes);
-                        tma_load_5d_a32(sa_u, &tmU, fb_u, c0 >> 6, k0 >> 4, pos);
+                        tma_load_5d_hint_a32(sa_u, &tmU, fb_u, c0 >> 6, k0 >> 4, pos, u_policy);
                         sa_u += stage_bytes;
                         fb_u += 8;
                         ++pre;
@@ -197,7 +198,7 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
                         mbar_arrive_expect_tx_a32(fb, tx_bytes);
                         tma_load_3d_a32(sa, &tmV, fb, p0, c0, pos);
                         tma_load_3d_a32(sa + L::A_BOX_BYTES, &tmV, fb, p0 + 64, c0, pos);
-                        tma_load_5d_a32(sa + L::A_BYTES, &tmU, fb, c0 >> 6, k0 >> 4, pos);
+                        tma_load_5d_hint_a32(sa + L::A_BYTES, &tmU, fb, c0 >> 6, k0 >> 4, pos, u_policy);
                     }
                     sa += stage_bytes;
                     fb += 8;
