@@ -338,7 +338,7 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
                 if (group == 0) asm volatile("bar.sync 1, 128;" ::: "memory");
                 else asm volatile("bar.sync 2, 128;" ::: "memory");
                 if (group_tid == 0) {
-                    if (p_ok) tma_store_3d(&tmM, stg, p0 - quarter * 32, k0 + row0, pos);
+                    if (p_ok) tma_store_3d_hint(&tmM, stg, p0 - quarter * 32, k0 + row0, pos, l2_policy_evict_last());
                     tma_store_commit();
                 }
             }
