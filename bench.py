@@ -32,7 +32,7 @@ TILE = "auto"   # per layer: what sdwino_choose_tile returns; --tile 2 / --tile 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum per GEMM launch of one SD v1.5 step, from ncu captures
 # (profiles/launch_list_sd15_unet_sweep.md), by --tile.  Only valid for the default workload with all layers.
-GEMM_DRAM_BYTES_PER_LAUNCH_SD15 = {"auto": 53.92e6, "2": 40.66e6}
+GEMM_DRAM_BYTES_PER_LAUNCH_SD15 = {"auto": 49.89e6, "2": 40.66e6}
 PAPER_CONTEXT = {"per_layer_speedup_vs_sdcpp_m1pro": 2.76, "end_to_end_speedup_vs_sdcpp_m1pro": 4.79}
 
 
