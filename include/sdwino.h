@@ -162,9 +162,10 @@ int sdwino_set_gemm_shape(int ctas, int n_tile);
 /*
  * Which of the two supported algorithms is expected to be faster for a layer: returns 2 for F(2x2,3x3),
  * 4 for F(4x4,3x3), 0 for non-positive sizes.  The paper leaves the tile size open; both satisfy the
- * accuracy bound (F4 with about 4x the error of F2).  Rule: layers with at most 8 input or output
- * channels -> 2 (single-kernel paths); otherwise 4 when 2 * tiles * (C + K) >= K * C with
- * tiles = N * ceil(H/2) * ceil(W/2), i.e. when the activation-side traffic outweighs the weights.
+ * accuracy bound (F4 with about 4x the error of F2).  Rule, with tiles = N * ceil(H/2) * ceil(W/2):
+ * at most 8 input channels -> 2 (single-kernel path); at most 8 output channels -> 2 from 12288 tiles
+ * (single-kernel path), 4 below; otherwise 4 when 2 * tiles * (C + K) >= K * C, i.e. when the
+ * activation-side traffic outweighs the weights.
  * Pure host arithmetic: no device is touched.  The caller passes the result as `tile` to
  * sdwino_filter_transform and sdwino_conv3x3.
  */

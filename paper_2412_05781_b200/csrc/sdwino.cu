@@ -551,12 +551,15 @@ int sdwino_set_gemm_shape(int ctas, int n_tile) {
 
 int sdwino_choose_tile(int N, int C, int H, int W, int K) {
     if (N <= 0 || C <= 0 || H <= 0 || W <= 0 || K <= 0) return 0;
-    // Few-channel layers have single-kernel F(2x2) paths.  Otherwise F(4x4) moves 2.25 instead of 4 transform
+    // Layers with few input channels have a single-kernel F(2x2) path.  Otherwise F(4x4) moves 2.25 instead of 4 transform
     // values per pixel through the workspace and the tensor cores but streams 36 instead of 16 values per
     // weight: it wins once the tiles outnumber the weights per channel pair.  Measured on 97 layer shapes:
     // F4 is 15-40 % faster above twice the threshold below, within +-7 % around it, up to 2x slower far below.
-    if (C <= 8 || K <= 8) return 2;
     const long long P2 = static_cast<long long>(N) * ((H + 1) / 2) * ((W + 1) / 2);
+    if (C <= 8) return 2;
+    // few output channels: the single-kernel F(2x2) path needs many blocks of tiles to fill the SMs; below about
+    // a hundred of them the three-kernel F(4x4) path is 5-20 % faster (320->4 at 64x64: 12.2 against 14.7 us)
+    if (K <= 8) return P2 >= 12288 ? 2 : 4;
     return 2 * P2 * (static_cast<long long>(C) + K) >= static_cast<long long>(K) * C ? 4 : 2;
 }
 

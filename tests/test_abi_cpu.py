@@ -100,7 +100,8 @@ def test_product_package_does_not_import_oracle():
 def test_choose_tile_is_host_arithmetic(binding):
     # few-channel layers -> F(2x2); weight-heavy layers -> F(2x2); activation-heavy layers -> F(4x4)
     assert binding.sdwino_choose_tile(2, 4, 64, 64, 320) == 2
-    assert binding.sdwino_choose_tile(2, 320, 64, 64, 4) == 2
+    assert binding.sdwino_choose_tile(2, 320, 64, 64, 4) == 4      # few output channels, 2048 tiles
+    assert binding.sdwino_choose_tile(1, 128, 512, 512, 3) == 2    # few output channels, 65536 tiles
     assert binding.sdwino_choose_tile(2, 1280, 8, 8, 1280) == 2
     assert binding.sdwino_choose_tile(2, 2560, 16, 16, 1280) == 2
     assert binding.sdwino_choose_tile(2, 320, 64, 64, 320) == 4
