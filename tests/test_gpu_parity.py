@@ -381,3 +381,33 @@ def test_sdxl_layers_sampled_channels(B, idx, tile):
     layer = workloads.sdxl_1024()[idx]
     err, edge = _sampled_check(B, layer, tile, nch=3, seed=idx)
     assert err <= TOL and edge <= TOL, (layer.name, err, edge)
+
+
+def _random_shapes(count, seed):
+    rng = np.random.default_rng(seed)
+    shapes = []
+    for _ in range(count):
+        C = int(rng.choice([1, 2, 5, 8, 9, 17, 40, 64, 70, 130, 200]))
+        K = int(rng.choice([1, 3, 8, 9, 16, 31, 48, 100, 160, 260]))
+        H = int(rng.integers(1, 41))
+        W = int(rng.choice([int(rng.integers(1, 41)), 8 * int(rng.integers(1, 6))]))   # half of them W % 8 == 0
+        N = int(rng.integers(1, 4))
+        shapes.append((C, K, H, W, N))
+    return shapes
+
+
+@pytest.mark.parametrize("shape", _random_shapes(24, seed=2412))
+def test_seeded_random_shapes_both_tiles(B, shape):
+    # a seeded draw over channel counts (few / ragged / several blocks), odd and even sizes, scalar and vector
+    # transform paths, small batches: every path of the dispatcher must agree with the oracle
+    C, K, H, W, N = shape
+    layer = ConvLayer(C=C, K=K, H=H, W=W, N=N)
+    x, w, b = workloads.make_inputs(layer, seed=sum(shape))
+    ref = oracle.direct_conv3x3(x.numpy(), w.numpy(), b.numpy())
+    scale = np.abs(ref).max()
+    for tile in (2, 4):
+        _, _, _, y = _run(B, layer, tile, x=x, w=w, b=b)
+        d = np.abs(y.double().numpy() - ref)
+        assert d.max() <= (TOL_F2_REGRESSION if tile == 2 else TOL) * scale, (shape, tile, d.max() / scale)
+        mask = _edge_mask(H, W, tile)
+        assert d[:, :, mask].max() <= TOL * scale
