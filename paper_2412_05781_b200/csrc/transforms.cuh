@@ -788,8 +788,6 @@ __device__ __forceinline__ void mma_m16n8k8_f16f32(float (&d)[4], uint32_t a0, u
         : "r"(a0), "r"(a1), "r"(b0));
 }
 
-constexpr int FUSED_C_MAX = 8;
-
 // Grid: x = groups of 8 tiles, four per block (one per warp); y = chunks of `kb_per_block` blocks of 16 output
 // channels.  A warp transforms its 8 tiles once and then walks the chunk's output-channel blocks.
 __global__ void __launch_bounds__(128)
