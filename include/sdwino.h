@@ -122,11 +122,25 @@ int sdwino_conv3x3_static(const void *x, const void *wT, const void *bias, void 
  * device-side copies of x, bias and y are carved from the front of `workspace`, which must
  * therefore hold sdwino_host_staging_bytes(...) in addition to a scratch accepted by
  * sdwino_conv3x3_ws (at least sdwino_workspace_min_bytes).  Used for end-to-end timing.
+ *
+ * sdwino_conv3x3_host_async is the same without the final synchronisation: it returns once the work is
+ * enqueued.  Uploads and downloads run on two copy streams owned by the library and alternate between two
+ * slots of the staging area, so the upload of the next call and the download of the previous one overlap the
+ * kernels of this one (PCIe is full duplex); the kernels stay on `stream`, in call order.  y_host of every
+ * earlier call is complete once sdwino_host_join(stream) has been called (it makes `stream` wait for the
+ * outstanding downloads) and `stream` has then been synchronised; x_host and bias_host must not change until
+ * then.  While such calls are in flight the staging part of the workspace belongs to them: do not hand the
+ * same workspace to other entry points before the join.  The first call on a device creates the two streams
+ * and eight events (make it outside any stream capture); not thread-safe.
  */
 size_t sdwino_host_staging_bytes(int N, int C, int H, int W, int K, int tile);
 int sdwino_conv3x3_host(const void *x_host, const void *wT, const void *bias_host, void *y_host,
                         int N, int C, int H, int W, int K, int tile,
                         void *workspace, size_t workspace_bytes, void *stream);
+int sdwino_conv3x3_host_async(const void *x_host, const void *wT, const void *bias_host, void *y_host,
+                              int N, int C, int H, int W, int K, int tile,
+                              void *workspace, size_t workspace_bytes, void *stream);
+int sdwino_host_join(void *stream);
 
 /*
  * Device-side waits (on TMA / tensor-core completion barriers) are bounded; a wait that

@@ -22,7 +22,7 @@ EXPORTS = [
     "sdwino_conv3x3_ws", "sdwino_host_staging_bytes", "sdwino_conv3x3_host",
     "sdwino_last_device_status", "sdwino_launch_count", "sdwino_profile_enable", "sdwino_profile_collect",
     "sdwino_profile_records", "sdwino_set_gemm_shape", "sdwino_conv3x3_static", "sdwino_set_fused_min_tiles", "sdwino_choose_tile",
-    "sdwino_selftest_wait_timeout",
+    "sdwino_selftest_wait_timeout", "sdwino_conv3x3_host_async", "sdwino_host_join",
 ]
 
 KERNEL_KINDS = ("filter_transform", "input_transform", "wino_gemm", "output_transform", "fused")
@@ -61,6 +61,10 @@ def _load() -> ctypes.CDLL:
     lib.sdwino_conv3x3_ws.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, vp, sz, vp]
     lib.sdwino_conv3x3_host.restype = i
     lib.sdwino_conv3x3_host.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, vp, sz, vp]
+    lib.sdwino_host_join.restype = i
+    lib.sdwino_host_join.argtypes = [vp]
+    lib.sdwino_conv3x3_host_async.restype = i
+    lib.sdwino_conv3x3_host_async.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, vp, sz, vp]
     lib.sdwino_last_device_status.restype = i
     lib.sdwino_last_device_status.argtypes = [vp]
     lib.sdwino_launch_count.restype = ctypes.c_ulonglong
@@ -247,16 +251,22 @@ def sdwino_conv3x3_static(x: torch.Tensor, wT: torch.Tensor, bias: Optional[torc
     return y
 
 
+def sdwino_host_join(stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Make `stream` wait for the downloads of all earlier sdwino_conv3x3_host(..., wait=False) calls."""
+    _check(lib.sdwino_host_join(_stream_ptr(stream)), "sdwino_host_join")
+
+
 def sdwino_conv3x3_host(x: torch.Tensor, wT: torch.Tensor, bias: Optional[torch.Tensor], y: torch.Tensor,
-                        tile: int, workspace: torch.Tensor, stream=None) -> torch.Tensor:
-    """x, bias, y: fp16 CPU tensors (ideally pinned); wT and workspace on the device.  Returns y
-    after the stream has been synchronised."""
+                        tile: int, workspace: torch.Tensor, stream=None, wait: bool = True) -> torch.Tensor:
+    """x, bias, y: fp16 CPU tensors (ideally pinned); wT and workspace on the device.  wait=True returns y
+    after the stream has been synchronised; wait=False (sdwino_conv3x3_host_async) returns once the work is
+    enqueued: y is complete after sdwino_host_join(stream) and a synchronisation of the stream."""
     assert not x.is_cuda and not y.is_cuda and x.dtype == torch.float16 and y.dtype == torch.float16
     assert x.is_contiguous() and y.is_contiguous()
     N, C, H, W = (int(v) for v in x.shape)
     K = int(y.shape[1])
-    rc = lib.sdwino_conv3x3_host(x.data_ptr(), wT.data_ptr(), _ptr(bias), y.data_ptr(), N, C, H, W, K, tile,
-                                 workspace.data_ptr(), workspace.numel() * workspace.element_size(),
-                                 _stream_ptr(stream))
-    _check(rc, "sdwino_conv3x3_host")
+    fn = lib.sdwino_conv3x3_host if wait else lib.sdwino_conv3x3_host_async
+    rc = fn(x.data_ptr(), wT.data_ptr(), _ptr(bias), y.data_ptr(), N, C, H, W, K, tile,
+            workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    _check(rc, "sdwino_conv3x3_host" if wait else "sdwino_conv3x3_host_async")
     return y

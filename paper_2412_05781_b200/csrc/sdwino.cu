@@ -76,6 +76,7 @@ constexpr int MAX_DYN_SMEM = 232448;  // 227 KB opt-in limit per CTA on sm_100
 // with 64 MB passes, 216 us with 128 MB, 202 us in a single pass).  The cap only bounds the memory asked for.
 constexpr size_t PASS_BUDGET = 1024ull << 20;
 constexpr size_t WS_ALIGN = 1024;
+constexpr int STATIC_MAX_DEVICES_HOST = 64;
 
 inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
 inline long long round_up_ll(long long v, long long m) { return (v + m - 1) / m * m; }
@@ -647,35 +648,102 @@ size_t sdwino_host_staging_bytes(int N, int C, int H, int W, int K, int tile) {
     const size_t xb = up(static_cast<size_t>(N) * C * H * W * sizeof(__half));
     const size_t yb = up(static_cast<size_t>(N) * K * H * W * sizeof(__half));
     const size_t bb = up(static_cast<size_t>(K) * sizeof(__half));
-    return xb + yb + bb;
+    return 2 * (xb + bb + yb);   // two slots: uploads, kernels and downloads of consecutive calls overlap
 }
 
-int sdwino_conv3x3_host(const void* x_host, const void* wT, const void* bias_host, void* y_host, int N, int C, int H,
-                        int W, int K, int tile, void* workspace, size_t workspace_bytes, void* stream) {
+namespace {
+// Per-device state of the asynchronous host path: one copy stream per direction and four events per staging
+// slot.  Created on first use; one device per process is the common case.
+struct HostPipe {
+    bool ready = false;
+    cudaStream_t s_in = nullptr, s_out = nullptr;
+    cudaEvent_t uploaded[2] = {nullptr, nullptr};    // on s_in: x (and bias) of slot i are on the device
+    cudaEvent_t consumed[2] = {nullptr, nullptr};    // on the caller's stream: the kernels have read slot i
+    cudaEvent_t computed[2] = {nullptr, nullptr};    // on the caller's stream: y of slot i is complete on the device
+    cudaEvent_t downloaded[2] = {nullptr, nullptr};  // on s_out: y of slot i has reached host memory
+    bool slot_used[2] = {false, false};
+    unsigned long long calls = 0;
+};
+HostPipe g_host_pipe[STATIC_MAX_DEVICES_HOST];
+
+HostPipe* host_pipe() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= STATIC_MAX_DEVICES_HOST) return nullptr;
+    HostPipe& hp = g_host_pipe[dev];
+    if (!hp.ready) {
+        if (cudaStreamCreateWithFlags(&hp.s_in, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+        if (cudaStreamCreateWithFlags(&hp.s_out, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+        for (int i = 0; i < 2; ++i) {
+            if (cudaEventCreateWithFlags(&hp.uploaded[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+            if (cudaEventCreateWithFlags(&hp.consumed[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+            if (cudaEventCreateWithFlags(&hp.computed[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+            if (cudaEventCreateWithFlags(&hp.downloaded[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        }
+        hp.ready = true;
+    }
+    return &hp;
+}
+}  // namespace
+
+int sdwino_conv3x3_host_async(const void* x_host, const void* wT, const void* bias_host, void* y_host, int N, int C,
+                              int H, int W, int K, int tile, void* workspace, size_t workspace_bytes, void* stream) {
     if (!x_host || !y_host || !wT) return SDWINO_ERR_INVALID_ARG;
     if (tile != 2 && tile != 4) return SDWINO_ERR_UNSUPPORTED;
     const size_t staging = sdwino_host_staging_bytes(N, C, H, W, K, tile);
     if (staging == 0) return SDWINO_ERR_INVALID_ARG;
     if (!workspace || workspace_bytes <= staging) return SDWINO_ERR_WORKSPACE;
     if (!aligned(workspace, WS_ALIGN)) return SDWINO_ERR_MISALIGNED;
+    HostPipe* hp = host_pipe();
+    if (!hp) return SDWINO_ERR_CUDA;
     auto up = [](size_t v) { return (v + WS_ALIGN - 1) / WS_ALIGN * WS_ALIGN; };
     const size_t xbytes = static_cast<size_t>(N) * C * H * W * sizeof(__half);
     const size_t ybytes = static_cast<size_t>(N) * K * H * W * sizeof(__half);
+    const size_t bbytes = static_cast<size_t>(K) * sizeof(__half);
+    const int slot = static_cast<int>(hp->calls++ & 1ull);
     uint8_t* base = static_cast<uint8_t*>(workspace);
-    uint8_t* xd = base;
-    uint8_t* yd = xd + up(xbytes);
-    uint8_t* bd = yd + up(ybytes);
+    uint8_t* xd = base + slot * up(xbytes);
+    uint8_t* bd = base + 2 * up(xbytes) + slot * up(bbytes);
+    uint8_t* yd = base + 2 * (up(xbytes) + up(bbytes)) + slot * up(ybytes);
     uint8_t* ws = base + staging;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (cudaMemcpyAsync(xd, x_host, xbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return SDWINO_ERR_CUDA;
-    if (bias_host &&
-        cudaMemcpyAsync(bd, bias_host, static_cast<size_t>(K) * sizeof(__half), cudaMemcpyHostToDevice, st) !=
-            cudaSuccess)
+    // upload on the copy stream, as soon as the kernels of the call before last have finished reading this slot
+    if (hp->slot_used[slot] && cudaStreamWaitEvent(hp->s_in, hp->consumed[slot], 0) != cudaSuccess) return SDWINO_ERR_CUDA;
+    if (cudaMemcpyAsync(xd, x_host, xbytes, cudaMemcpyHostToDevice, hp->s_in) != cudaSuccess) return SDWINO_ERR_CUDA;
+    if (bias_host && cudaMemcpyAsync(bd, bias_host, bbytes, cudaMemcpyHostToDevice, hp->s_in) != cudaSuccess)
         return SDWINO_ERR_CUDA;
-    int rc = conv_impl(xd, wT, bias_host ? bd : nullptr, yd, N, C, H, W, K, tile, ws, workspace_bytes - staging, st);
+    if (cudaEventRecord(hp->uploaded[slot], hp->s_in) != cudaSuccess) return SDWINO_ERR_CUDA;
+    // kernels on the caller's stream, once the upload is there and the download of the call before last has
+    // left this slot's output buffer
+    if (cudaStreamWaitEvent(st, hp->uploaded[slot], 0) != cudaSuccess) return SDWINO_ERR_CUDA;
+    if (hp->slot_used[slot] && cudaStreamWaitEvent(st, hp->downloaded[slot], 0) != cudaSuccess) return SDWINO_ERR_CUDA;
+    const int rc = conv_impl(xd, wT, bias_host ? bd : nullptr, yd, N, C, H, W, K, tile, ws, workspace_bytes - staging, st);
     if (rc != SDWINO_OK) return rc;
-    if (cudaMemcpyAsync(y_host, yd, ybytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return SDWINO_ERR_CUDA;
-    if (cudaStreamSynchronize(st) != cudaSuccess) return SDWINO_ERR_CUDA;
+    if (cudaEventRecord(hp->consumed[slot], st) != cudaSuccess) return SDWINO_ERR_CUDA;
+    if (cudaEventRecord(hp->computed[slot], st) != cudaSuccess) return SDWINO_ERR_CUDA;
+    // download on the second copy stream
+    if (cudaStreamWaitEvent(hp->s_out, hp->computed[slot], 0) != cudaSuccess) return SDWINO_ERR_CUDA;
+    if (cudaMemcpyAsync(y_host, yd, ybytes, cudaMemcpyDeviceToHost, hp->s_out) != cudaSuccess) return SDWINO_ERR_CUDA;
+    if (cudaEventRecord(hp->downloaded[slot], hp->s_out) != cudaSuccess) return SDWINO_ERR_CUDA;
+    hp->slot_used[slot] = true;
+    return SDWINO_OK;
+}
+
+int sdwino_host_join(void* stream) {
+    HostPipe* hp = host_pipe();
+    if (!hp) return SDWINO_ERR_CUDA;
+    for (int i = 0; i < 2; ++i)
+        if (hp->slot_used[i] && cudaStreamWaitEvent(static_cast<cudaStream_t>(stream), hp->downloaded[i], 0) != cudaSuccess)
+            return SDWINO_ERR_CUDA;
+    return SDWINO_OK;
+}
+
+int sdwino_conv3x3_host(const void* x_host, const void* wT, const void* bias_host, void* y_host, int N, int C, int H,
+                        int W, int K, int tile, void* workspace, size_t workspace_bytes, void* stream) {
+    const int rc = sdwino_conv3x3_host_async(x_host, wT, bias_host, y_host, N, C, H, W, K, tile, workspace,
+                                             workspace_bytes, stream);
+    if (rc != SDWINO_OK) return rc;
+    if (sdwino_host_join(stream) != SDWINO_OK) return SDWINO_ERR_CUDA;
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return SDWINO_ERR_CUDA;
     return SDWINO_OK;
 }
 

@@ -51,7 +51,8 @@ def test_size_queries(binding):
     assert small == 128 * 16 * 640 * 2 + 1024
     assert binding.sdwino_workspace_bytes(1, 1, 1, 1, 1, 5) == 0
     assert binding.sdwino_workspace_bytes(1, 0, 1, 1, 1, 2) == 0
-    assert binding.sdwino_host_staging_bytes(1, 4, 8, 8, 4, 2) == 1024 * 3
+    # two slots of x, bias and y, each rounded up to 1 KB
+    assert binding.sdwino_host_staging_bytes(1, 4, 8, 8, 4, 2) == 1024 * 6
 
 
 def test_argument_validation_without_gpu(binding):

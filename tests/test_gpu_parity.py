@@ -411,3 +411,34 @@ def test_seeded_random_shapes_both_tiles(B, shape):
         assert d.max() <= (TOL_F2_REGRESSION if tile == 2 else TOL) * scale, (shape, tile, d.max() / scale)
         mask = _edge_mask(H, W, tile)
         assert d[:, :, mask].max() <= TOL * scale
+
+
+def test_async_host_entry_pipelines_calls_and_matches_device_entry(B):
+    # several layers enqueued back to back through the asynchronous host entry (uploads on the library's copy
+    # stream, alternating input slots), one synchronisation at the end: every result equals the device entry
+    shapes = [(24, 40, 20, 24, 2), (40, 16, 12, 16, 1), (8, 24, 16, 16, 2), (64, 64, 9, 11, 1), (24, 40, 20, 24, 2)]
+    stream = torch.cuda.Stream()
+    jobs = []
+    ws_bytes = 0
+    for i, (C, K, H, W, N) in enumerate(shapes):
+        layer = ConvLayer(C=C, K=K, H=H, W=W, N=N)
+        x, w, b = workloads.make_inputs(layer, seed=40 + i, pin=True)
+        tile = 2 if i % 2 == 0 else 4
+        wT = B.sdwino_filter_transform(w.cuda(), tile)
+        y = torch.empty(N, K, H, W, dtype=torch.float16).pin_memory()
+        args = (N, C, H, W, K, tile)
+        ws_bytes = max(ws_bytes, B.sdwino_host_staging_bytes(*args) + B.sdwino_workspace_bytes(*args))
+        jobs.append((layer, tile, x, w, b, wT, y))
+    ws = B.alloc_workspace(ws_bytes)
+    torch.cuda.synchronize()
+    for rep in range(2):                       # the second round reuses both slots
+        for layer, tile, x, w, b, wT, y in jobs:
+            y.zero_()
+            B.sdwino_conv3x3_host(x, wT, b, y, tile, ws, stream=stream, wait=False)
+        B.sdwino_host_join(stream)
+        stream.synchronize()
+        assert B.sdwino_last_device_status(stream) == B.OK
+        for layer, tile, x, w, b, wT, y in jobs:
+            ws2 = B.alloc_workspace(B.sdwino_workspace_bytes(layer.N, layer.C, layer.H, layer.W, layer.K, tile))
+            y_dev = B.sdwino_conv3x3(x.cuda(), wT, b.cuda(), layer.K, tile, workspace=ws2)
+            assert torch.equal(y, y_dev.cpu()), (layer.name, tile, rep)
