@@ -369,19 +369,16 @@ __device__ __forceinline__ void at4_packed(const float2 (&m)[6], float2 (&o)[4])
     o[3] = __ffma2_rn(f2s(3.375f), d2, __ffma2_rn(f2s(0.421875f), d1, m[5]));
 }
 
+// One unit of the vector activation transform: channel c = idx / groups, TPT tiles of one tile row.  The flat
+// index over (channel, group of TPT tiles) keeps blocks full when a pass has few tiles.  Called by the kernel
+// below (one unit per thread) and by the single-launch layer kernel (a grid-stride loop).
 template <int M, int TPT>
-__global__ void __launch_bounds__(128)
-input_transform_vec_kernel(const __half* __restrict__ x, __half* __restrict__ V, TileGeom geo, int C,
-                           long long p_begin, FastDiv gdiv, long long Pstride) {
+__device__ __forceinline__ void input_unit_vec(const __half* __restrict__ x, __half* __restrict__ V, const TileGeom& geo,
+                                               int C, long long p_begin, const FastDiv& gdiv, long long Pstride,
+                                               uint32_t idx) {
     using Wm = Wino<M>;
     constexpr int A = Wm::A;
-    // Wait first, release the GEMM second: once the GEMM runs, everything before this kernel has completed,
-    // which is what lets it fetch its filters (written at the latest by the kernel before this one) early.
-    pdl_wait();
-    pdl_launch_dependents();
     static_assert(M * TPT == 8, "one 16-byte row segment per thread");
-    // flat index over (channel, group of TPT tiles): blocks stay full when a pass has few tiles
-    const uint32_t idx = blockIdx.x * blockDim.x + threadIdx.x;   // below 2^31 (checked by the launcher)
     const int c = static_cast<int>(fast_div(idx, gdiv));           // gdiv.d = p_count / TPT groups per channel
     if (c >= C) return;
     const int pl = static_cast<int>(idx - static_cast<uint32_t>(c) * gdiv.d) * TPT;  // first chunk-local tile of this thread
@@ -460,6 +457,17 @@ input_transform_vec_kernel(const __half* __restrict__ x, __half* __restrict__ V,
     }   // M != 4
 }
 
+template <int M, int TPT>
+__global__ void __launch_bounds__(128)
+input_transform_vec_kernel(const __half* __restrict__ x, __half* __restrict__ V, TileGeom geo, int C,
+                           long long p_begin, FastDiv gdiv, long long Pstride) {
+    // Wait first, release the GEMM second: once the GEMM runs, everything before this kernel has completed,
+    // which is what lets it fetch its filters (written at the latest by the kernel before this one) early.
+    pdl_wait();
+    pdl_launch_dependents();
+    input_unit_vec<M, TPT>(x, V, geo, C, p_begin, gdiv, Pstride, blockIdx.x * blockDim.x + threadIdx.x);   // < 2^31
+}
+
 // F(4x4,3x3) activation transform, vector path: a thread owns 2 tiles (8 pixels of a tile row) and CH consecutive
 // channels.  Loads go into zero-initialised registers under precomputed border masks (no selects), and the
 // (tile 0, tile 1) operand pairs of the packed arithmetic are cut straight out of the loaded halves with byte
@@ -467,13 +475,10 @@ input_transform_vec_kernel(const __half* __restrict__ x, __half* __restrict__ V,
 // the generic vector kernel.  CH = 1 is what runs: with 2 or 4 channels per thread the per-thread set-up is
 // amortised, but the serial load -> compute chain per channel and the lower thread count cost more (measured).
 template <int CH>
-__global__ void __launch_bounds__(128, 5)
-input_transform_f4_kernel(const __half* __restrict__ x, __half* __restrict__ V, TileGeom geo, int C, long long p_begin,
-                          FastDiv gdiv, long long Pstride) {
+__device__ __forceinline__ void input_unit_f4(const __half* __restrict__ x, __half* __restrict__ V, const TileGeom& geo,
+                                              int C, long long p_begin, const FastDiv& gdiv, long long Pstride,
+                                              uint32_t idx) {
     constexpr int A = 6;
-    pdl_wait();                 // see input_transform_vec_kernel: wait first, release the GEMM second
-    pdl_launch_dependents();
-    const uint32_t idx = blockIdx.x * blockDim.x + threadIdx.x;   // below 2^31 (checked by the launcher)
     const int cg = static_cast<int>(fast_div(idx, gdiv));          // gdiv.d = groups of 2 tiles in this pass
     const int c0 = cg * CH;
     if (c0 >= C) return;
@@ -539,16 +544,45 @@ input_transform_f4_kernel(const __half* __restrict__ x, __half* __restrict__ V, 
     }
 }
 
-template <int M, int TPT>
-__global__ void __launch_bounds__(128)
-output_transform_vec_kernel(const __half* __restrict__ Mws, const __half* __restrict__ bias, __half* __restrict__ y,
-                            TileGeom geo, int K, long long p_begin, FastDiv gdiv, long long Pstride) {
+template <int CH>
+__global__ void __launch_bounds__(128, 5)
+input_transform_f4_kernel(const __half* __restrict__ x, __half* __restrict__ V, TileGeom geo, int C, long long p_begin,
+                          FastDiv gdiv, long long Pstride) {
+    pdl_wait();                 // see input_transform_vec_kernel: wait first, release the GEMM second
+    pdl_launch_dependents();
+    input_unit_f4<CH>(x, V, geo, C, p_begin, gdiv, Pstride, blockIdx.x * blockDim.x + threadIdx.x);   // < 2^31
+}
+
+// Loads of M: through the read-only path when M was written by an earlier kernel, with a plain L2 load when it
+// was written earlier in the SAME kernel by other CTAs (the read-only path is not coherent within a kernel).
+template <bool SAME_KERNEL>
+__device__ __forceinline__ uint32_t load_m_u32(const __half* q) {
+    if constexpr (SAME_KERNEL) {
+        uint32_t v;
+        asm volatile("ld.global.cg.u32 %0, [%1];" : "=r"(v) : "l"(q) : "memory");
+        return v;
+    } else {
+        return __ldg(reinterpret_cast<const uint32_t*>(q));
+    }
+}
+template <bool SAME_KERNEL>
+__device__ __forceinline__ uint2 load_m_u64(const __half* q) {
+    if constexpr (SAME_KERNEL) {
+        uint2 v;
+        asm volatile("ld.global.cg.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(q) : "memory");
+        return v;
+    } else {
+        return __ldg(reinterpret_cast<const uint2*>(q));
+    }
+}
+
+template <int M, int TPT, bool SAME_KERNEL>
+__device__ __forceinline__ void output_unit_vec(const __half* __restrict__ Mws, const __half* __restrict__ bias,
+                                                __half* __restrict__ y, const TileGeom& geo, int K, long long p_begin,
+                                                const FastDiv& gdiv, long long Pstride, uint32_t idx) {
     using Wm = Wino<M>;
     constexpr int A = Wm::A;
-    pdl_launch_dependents();
-    pdl_wait();
     static_assert(M * TPT == 8, "one 16-byte row segment per thread");
-    const uint32_t idx = blockIdx.x * blockDim.x + threadIdx.x;   // below 2^31 (checked by the launcher)
     const int k = static_cast<int>(fast_div(idx, gdiv));           // gdiv.d = p_count / TPT groups per channel
     if (k >= K) return;
     const int pl = static_cast<int>(idx - static_cast<uint32_t>(k) * gdiv.d) * TPT;
@@ -564,7 +598,7 @@ output_transform_vec_kernel(const __half* __restrict__ Mws, const __half* __rest
             float2 col[A], o[M];
 #pragma unroll
             for (int r = 0; r < A; ++r) {
-                const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(src + (r * A + s) * plane));
+                const uint32_t w = load_m_u32<SAME_KERNEL>(src + (r * A + s) * plane);
                 col[r] = __half22float2(*reinterpret_cast<const __half2*>(&w));
             }
             at4_packed(col, o);
@@ -597,11 +631,11 @@ output_transform_vec_kernel(const __half* __restrict__ Mws, const __half* __rest
         for (int s = 0; s < A; ++s) {
             const __half* q = src + (r * A + s) * plane;
             if constexpr (TPT == 4) {
-                const uint2 w = __ldg(reinterpret_cast<const uint2*>(q));
+                const uint2 w = load_m_u64<SAME_KERNEL>(q);
                 unpack2(w.x, mm[r][s][0], mm[r][s][1]);
                 unpack2(w.y, mm[r][s][2], mm[r][s][3]);
             } else {
-                const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(q));
+                const uint32_t w = load_m_u32<SAME_KERNEL>(q);
                 unpack2(w, mm[r][s][0], mm[r][s][1]);
             }
         }
@@ -643,6 +677,15 @@ output_transform_vec_kernel(const __half* __restrict__ Mws, const __half* __rest
         *reinterpret_cast<uint4*>(img + static_cast<long long>(i0 + i) * geo.W + j0) = w;
     }
     }   // M != 4
+}
+
+template <int M, int TPT>
+__global__ void __launch_bounds__(128)
+output_transform_vec_kernel(const __half* __restrict__ Mws, const __half* __restrict__ bias, __half* __restrict__ y,
+                            TileGeom geo, int K, long long p_begin, FastDiv gdiv, long long Pstride) {
+    pdl_launch_dependents();
+    pdl_wait();
+    output_unit_vec<M, TPT, false>(Mws, bias, y, geo, K, p_begin, gdiv, Pstride, blockIdx.x * blockDim.x + threadIdx.x);
 }
 
 
