@@ -442,3 +442,20 @@ def test_async_host_entry_pipelines_calls_and_matches_device_entry(B):
             ws2 = B.alloc_workspace(B.sdwino_workspace_bytes(layer.N, layer.C, layer.H, layer.W, layer.K, tile))
             y_dev = B.sdwino_conv3x3(x.cuda(), wT, b.cuda(), layer.K, tile, workspace=ws2)
             assert torch.equal(y, y_dev.cpu()), (layer.name, tile, rep)
+
+
+@pytest.mark.parametrize("tile", [2, 4])
+@pytest.mark.parametrize("scale", [2.0 ** -10, 64.0])
+def test_relative_error_is_scale_invariant_within_fp16_range(B, tile, scale):
+    # V and M are stored in fp16: powers of two well inside its range only shift exponents, so the relative
+    # error must not change (overflow of V needs |x| of a few thousand, underflow |x| below about 1e-5)
+    layer = ConvLayer(C=96, K=64, H=24, W=32, N=1)
+    x, w, b = workloads.make_inputs(layer, seed=9)
+    xs = (x.float() * scale).half()
+    bs = (b.float() * scale).half()
+    _, _, _, y = _run(B, layer, tile, x=x, w=w, b=b)
+    _, _, _, ysc = _run(B, layer, tile, x=xs, w=w, b=bs)
+    ref = oracle.direct_conv3x3(xs.numpy(), w.numpy(), bs.numpy())
+    assert _rel_err(ysc, ref) <= (TOL_F2_REGRESSION if tile == 2 else TOL)
+    if scale > 1:      # exact power-of-two scaling without subnormals: bit-identical up to the exponent shift
+        assert torch.equal((y.float() * scale).half(), ysc)
