@@ -371,7 +371,7 @@ __device__ __forceinline__ void at4_packed(const float2 (&m)[6], float2 (&o)[4])
 
 // One unit of the vector activation transform: channel c = idx / groups, TPT tiles of one tile row.  The flat
 // index over (channel, group of TPT tiles) keeps blocks full when a pass has few tiles.  Called by the kernel
-// below (one unit per thread) and by the single-launch layer kernel (a grid-stride loop).
+// below with one unit per thread.
 template <int M, int TPT>
 __device__ __forceinline__ void input_unit_vec(const __half* __restrict__ x, __half* __restrict__ V, const TileGeom& geo,
                                                int C, long long p_begin, const FastDiv& gdiv, long long Pstride,
@@ -553,30 +553,7 @@ input_transform_f4_kernel(const __half* __restrict__ x, __half* __restrict__ V, 
     input_unit_f4<CH>(x, V, geo, C, p_begin, gdiv, Pstride, blockIdx.x * blockDim.x + threadIdx.x);   // < 2^31
 }
 
-// Loads of M: through the read-only path when M was written by an earlier kernel, with a plain L2 load when it
-// was written earlier in the SAME kernel by other CTAs (the read-only path is not coherent within a kernel).
-template <bool SAME_KERNEL>
-__device__ __forceinline__ uint32_t load_m_u32(const __half* q) {
-    if constexpr (SAME_KERNEL) {
-        uint32_t v;
-        asm volatile("ld.global.cg.u32 %0, [%1];" : "=r"(v) : "l"(q) : "memory");
-        return v;
-    } else {
-        return __ldg(reinterpret_cast<const uint32_t*>(q));
-    }
-}
-template <bool SAME_KERNEL>
-__device__ __forceinline__ uint2 load_m_u64(const __half* q) {
-    if constexpr (SAME_KERNEL) {
-        uint2 v;
-        asm volatile("ld.global.cg.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(q) : "memory");
-        return v;
-    } else {
-        return __ldg(reinterpret_cast<const uint2*>(q));
-    }
-}
-
-template <int M, int TPT, bool SAME_KERNEL>
+template <int M, int TPT>
 __device__ __forceinline__ void output_unit_vec(const __half* __restrict__ Mws, const __half* __restrict__ bias,
                                                 __half* __restrict__ y, const TileGeom& geo, int K, long long p_begin,
                                                 const FastDiv& gdiv, long long Pstride, uint32_t idx) {
@@ -598,7 +575,7 @@ __device__ __forceinline__ void output_unit_vec(const __half* __restrict__ Mws, 
             float2 col[A], o[M];
 #pragma unroll
             for (int r = 0; r < A; ++r) {
-                const uint32_t w = load_m_u32<SAME_KERNEL>(src + (r * A + s) * plane);
+                const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(src + (r * A + s) * plane));
                 col[r] = __half22float2(*reinterpret_cast<const __half2*>(&w));
             }
             at4_packed(col, o);
@@ -631,11 +608,11 @@ __device__ __forceinline__ void output_unit_vec(const __half* __restrict__ Mws, 
         for (int s = 0; s < A; ++s) {
             const __half* q = src + (r * A + s) * plane;
             if constexpr (TPT == 4) {
-                const uint2 w = load_m_u64<SAME_KERNEL>(q);
+                const uint2 w = __ldg(reinterpret_cast<const uint2*>(q));
                 unpack2(w.x, mm[r][s][0], mm[r][s][1]);
                 unpack2(w.y, mm[r][s][2], mm[r][s][3]);
             } else {
-                const uint32_t w = load_m_u32<SAME_KERNEL>(q);
+                const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(q));
                 unpack2(w, mm[r][s][0], mm[r][s][1]);
             }
         }
@@ -685,7 +662,7 @@ output_transform_vec_kernel(const __half* __restrict__ Mws, const __half* __rest
                             TileGeom geo, int K, long long p_begin, FastDiv gdiv, long long Pstride) {
     pdl_launch_dependents();
     pdl_wait();
-    output_unit_vec<M, TPT, false>(Mws, bias, y, geo, K, p_begin, gdiv, Pstride, blockIdx.x * blockDim.x + threadIdx.x);
+    output_unit_vec<M, TPT>(Mws, bias, y, geo, K, p_begin, gdiv, Pstride, blockIdx.x * blockDim.x + threadIdx.x);
 }
 
 
