@@ -48,7 +48,9 @@ const char *sdwino_status_string(int status);
  * Filter preprocess, step (i) of Section "Techniques": U[k][c] = G w[k][c] G^T.
  *
  * sdwino_filter_bytes: bytes the caller must allocate for wT (0 on bad arguments).
- * sdwino_filter_transform: w is fp16 [K][C][3][3]; wT receives fp16 U laid out as
+ * sdwino_filter_transform: w is fp16 [K][C][3][3]; wT receives a 1024-byte header (magic, K, C, tile: the
+ *   kernels of sdwino_conv3x3 compare it with their arguments before they read the filters, and a
+ *   mismatch is reported as SDWINO_ERR_INVALID_ARG by sdwino_last_device_status) followed by fp16 U laid out as
  *   [a*a][Cb][Kb][16][64] with a = tile+2, Kb = ceil(K/16), Cb = ceil(C/64): blocks of 16 output
  *   channels x 64 input channels (2 KB contiguous each; the blocks of consecutive output channels are
  *   adjacent), position index xi*a+nu, zero in the padding.  wT must be 1024-byte aligned (a cudaMalloc

@@ -45,6 +45,7 @@ constexpr int FK_ACC_COLS = 16 * FK_N;         // 256 TMEM columns per accumulat
 constexpr int FK_DYN_SMEM = FK_V_STAGES * FK_V_STAGE_BYTES + FK_U_BUFS * FK_U_BUF_BYTES + 1024 + 256;
 
 struct FusedKParams {
+    const uint32_t* wt_header;   // header of the transformed filter (see wt_header_ok)
     TileGeom geo;
     int C, K;
     int num_stages;     // ceil(C / 16)
@@ -160,6 +161,10 @@ __device__ __forceinline__ void fk_transform_store(const FkRaw& raw, uint8_t* st
 __global__ void __launch_bounds__(FK_THREADS, 1)
 fused_small_k_kernel(const __grid_constant__ CUtensorMap tmU, const __half* __restrict__ x,
                      const __half* __restrict__ bias, __half* __restrict__ y, FusedKParams prm, int* status_word) {
+    // The header may have been written by the kernel right before this one: wait for it before anything else.
+    // (Uniform early return: no barrier or TMEM has been set up yet.)
+    pdl_wait();
+    if (!wt_header_ok(prm.wt_header, prm.K, prm.C, 2, status_word)) return;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     // The filter buffers come first: the MMA reads 16 rows of B where only 8 are loaded, i.e. up to 1 KB past

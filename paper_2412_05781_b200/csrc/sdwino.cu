@@ -223,6 +223,15 @@ int sm_count() {
     return n;
 }
 
+// Device address of the status word (one device per process is the common case; looked up once).
+int* status_word_ptr() {
+    static int* status = nullptr;
+    if (!status && cudaGetSymbolAddress(reinterpret_cast<void**>(&status), g_status_word) != cudaSuccess) status = nullptr;
+    return status;
+}
+inline const uint32_t* wt_header_of(const void* wT) { return static_cast<const uint32_t*>(wT); }
+inline const void* wt_filters_of(const void* wT) { return static_cast<const uint8_t*>(wT) + WT_HEADER_BYTES; }
+
 // Kernels are launched with programmatic stream serialization (see pdl_wait in ptx.cuh); cluster_x: 0 for
 // the transform kernels, 1 or 2 CTAs per cluster for the GEMM.
 template <typename... KArgs, typename... Args>
@@ -255,10 +264,12 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
 }
 
 template <int M>
-int launch_filter(const __half* w, __half* U, int K, int C, int Kb, int Cb, cudaStream_t st) {
+int launch_filter(const __half* w, void* wT, int K, int C, int Kb, int Cb, cudaStream_t st) {
     dim3 grid((Cb * 64 + 127) / 128, Kb * 16);
     ProfScope prof(KIND_FILTER, st);
-    const cudaError_t e = launch_pdl(filter_transform_kernel<M>, grid, dim3(128), 0, st, 0, w, U, K, C, Kb, Cb);
+    uint32_t* header = static_cast<uint32_t*>(wT);
+    __half* U = reinterpret_cast<__half*>(static_cast<uint8_t*>(wT) + WT_HEADER_BYTES);
+    const cudaError_t e = launch_pdl(filter_transform_kernel<M>, grid, dim3(128), 0, st, 0, w, header, U, K, C, Kb, Cb);
     g_launches.fetch_add(1);
     return e == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
 }
@@ -292,7 +303,7 @@ int launch_input(const __half* x, __half* V, const TileGeom& geo, int C, long lo
 
 template <int M>
 int launch_output(const __half* Mws, const __half* bias, __half* y, const TileGeom& geo, int K,
-                  long long p_begin, int p_count, long long Pstride, cudaStream_t st) {
+                  long long p_begin, int p_count, long long Pstride, const WtCheck& chk, cudaStream_t st) {
     ProfScope prof(KIND_OUTPUT, st);
     constexpr int TPT = 8 / M;
     cudaError_t e;
@@ -300,11 +311,11 @@ int launch_output(const __half* Mws, const __half* bias, __half* y, const TileGe
     if (geo.W % 8 == 0 && aligned(y, 16) && units < (1ll << 31) - 128) {
         dim3 grid(static_cast<unsigned>((units + 127) / 128));
         e = launch_pdl(output_transform_vec_kernel<M, TPT>, grid, dim3(128), 0, st, 0, Mws, bias, y, geo, K, p_begin,
-                       make_fastdiv(static_cast<uint32_t>(p_count / TPT)), Pstride);
+                       make_fastdiv(static_cast<uint32_t>(p_count / TPT)), Pstride, chk);
     } else {
         dim3 grid((p_count + 127) / 128, K);
         e = launch_pdl(output_transform_kernel<M>, grid, dim3(128), 0, st, 0, Mws, bias, y, geo, K, p_begin, p_count,
-                       Pstride);
+                       Pstride, chk);
     }
     g_launches.fetch_add(1);
     return e == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
@@ -314,12 +325,14 @@ int launch_output(const __half* Mws, const __half* bias, __half* y, const TileGe
 bool use_fused_small_c(int C, int tile) { return tile == 2 ? C <= 8 : C <= 4; }
 
 template <int M, int CP>
-int launch_fused_small_c(const __half* x, const __half* U, const __half* bias, __half* y, const TileGeom& geo, int C,
+int launch_fused_small_c(const __half* x, const void* wT, const __half* bias, __half* y, const TileGeom& geo, int C,
                          int K, int Kb, int Cb, cudaStream_t st) {
+    int* status = status_word_ptr();
+    if (!status) return SDWINO_ERR_CUDA;
     dim3 grid(static_cast<unsigned>((geo.P + 127) / 128), (K + FUSED_KC - 1) / FUSED_KC);
     ProfScope prof(KIND_FUSED, st);
-    const cudaError_t e = launch_pdl(fused_small_c_kernel<M, CP>, grid, dim3(128), 0, st, 0, x, U, bias, y, geo, C, K,
-                                     Kb, Cb);
+    const cudaError_t e = launch_pdl(fused_small_c_kernel<M, CP>, grid, dim3(128), 0, st, 0, x, wt_header_of(wT),
+                                     static_cast<const __half*>(wt_filters_of(wT)), bias, y, geo, C, K, Kb, Cb, status);
     g_launches.fetch_add(1);
     return e == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
 }
@@ -349,8 +362,9 @@ int launch_fused_small_k(const __half* x, const void* wT, const __half* bias, __
     });
     if (attr_err != cudaSuccess) return SDWINO_ERR_CUDA;
     CUtensorMap tmU;
-    if (!encode_filter_map(&tmU, wT, pl.Cb, pl.Kb, pl.a2, 1, 16, FK_KMAX)) return SDWINO_ERR_CUDA;
+    if (!encode_filter_map(&tmU, wt_filters_of(wT), pl.Cb, pl.Kb, pl.a2, 1, 16, FK_KMAX)) return SDWINO_ERR_CUDA;
     FusedKParams prm;
+    prm.wt_header = wt_header_of(wT);
     prm.geo = make_geom(H, W, pl.TH, pl.TW, pl.P);
     prm.C = C;
     prm.K = K;
@@ -366,10 +380,11 @@ int launch_fused_small_k(const __half* x, const void* wT, const __half* bias, __
 }
 
 // F(2x2,3x3) layers with at most 8 input channels: one warp-MMA kernel (see fused_small_c_mma_kernel).
-int launch_fused_small_c_mma(const __half* x, const __half* U, const __half* bias, __half* y, const TileGeom& geo, int C,
+int launch_fused_small_c_mma(const __half* x, const void* wT, const __half* bias, __half* y, const TileGeom& geo, int C,
                              int K, int Kb, cudaStream_t st) {
     const int sms = sm_count();
-    if (sms <= 0) return SDWINO_ERR_CUDA;
+    int* status = status_word_ptr();
+    if (sms <= 0 || !status) return SDWINO_ERR_CUDA;
     const long long groups = (geo.P + 7) / 8;
     const long long blocks_x = (groups + 3) / 4;
     // about four blocks per SM: split the output-channel blocks over grid.y until there are enough
@@ -378,8 +393,9 @@ int launch_fused_small_c_mma(const __half* x, const __half* U, const __half* bia
     const int kb_per_block = static_cast<int>((Kb + ksplit - 1) / ksplit);
     dim3 grid(static_cast<unsigned>(blocks_x), static_cast<unsigned>((Kb + kb_per_block - 1) / kb_per_block));
     ProfScope prof(KIND_FUSED, st);
-    const cudaError_t e = launch_pdl(fused_small_c_mma_kernel, grid, dim3(128), 0, st, 0, x, U, bias, y, geo, C, K, Kb,
-                                     kb_per_block);
+    const cudaError_t e = launch_pdl(fused_small_c_mma_kernel, grid, dim3(128), 0, st, 0, x, wt_header_of(wT),
+                                     static_cast<const __half*>(wt_filters_of(wT)), bias, y, geo, C, K, Kb, kb_per_block,
+                                     status);
     g_launches.fetch_add(1);
     return e == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
 }
@@ -471,11 +487,10 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
     if (use_fused_small_c(C, tile) && !g_disable_fused) {
         const TileGeom geo = make_geom(H, W, pl.TH, pl.TW, pl.P);
         const __half* xh = static_cast<const __half*>(x);
-        const __half* uh = static_cast<const __half*>(wT);
         const __half* bh = static_cast<const __half*>(bias);
         __half* yh = static_cast<__half*>(y);
-        if (tile == 4) return launch_fused_small_c<4, 4>(xh, uh, bh, yh, geo, C, K, pl.Kb, pl.Cb, st);
-        return launch_fused_small_c_mma(xh, uh, bh, yh, geo, C, K, pl.Kb, st);
+        if (tile == 4) return launch_fused_small_c<4, 4>(xh, wT, bh, yh, geo, C, K, pl.Kb, pl.Cb, st);
+        return launch_fused_small_c_mma(xh, wT, bh, yh, geo, C, K, pl.Kb, st);
     }
 
     // workspace: V[a2][C][pc] then M[a2][K][pc]; pc is a multiple of 128 elements, so every row starts
@@ -490,6 +505,9 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
     const int sms = sm_count();
     if (sms <= 0) return SDWINO_ERR_CUDA;
     GemmParams prm;
+    prm.wt_header = wt_header_of(wT);
+    prm.K = K;
+    prm.tile = tile;
     GemmShape shape = choose_gemm_shape(K, C, pc / GEMM_BLOCK_P, pl.a2, sms);
     if (g_force_ctas == 1 || g_force_ctas == 2) shape.ctas = (pc / GEMM_BLOCK_P < 2) ? 1 : g_force_ctas;
     if (g_force_n_tile >= 16 && g_force_n_tile <= GEMM_MAX_N && g_force_n_tile % 16 == 0) shape.n_tile = g_force_n_tile;
@@ -510,7 +528,7 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
 
     prm.p_stride = pc;
     CUtensorMap tmU, tmV, tmM;
-    if (!encode_filter_map(&tmU, wT, pl.Cb, pl.Kb, pl.a2, b_rows / 16) ||
+    if (!encode_filter_map(&tmU, wt_filters_of(wT), pl.Cb, pl.Kb, pl.a2, b_rows / 16) ||
         !encode_map(&tmV, V, pc, C, pl.a2, pc, static_cast<uint64_t>(C) * pc, 64, GEMM_BLOCK_C, true) ||
         !encode_map(&tmM, Mws, pc, K, pl.a2, pc, static_cast<uint64_t>(K) * pc, GEMM_BLOCK_P, prm.epi_rows, false))
         return SDWINO_ERR_CUDA;
@@ -519,6 +537,8 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
     const __half* xh = static_cast<const __half*>(x);
     const __half* bh = static_cast<const __half*>(bias);
     __half* yh = static_cast<__half*>(y);
+    const WtCheck chk{wt_header_of(wT), K, C, tile, status_word_ptr()};
+    if (!chk.status_word) return SDWINO_ERR_CUDA;
     for (long long p0 = 0; p0 < pl.P; p0 += pc) {
         long long remaining = pl.P128 - p0;
         const int count = static_cast<int>(remaining < pc ? remaining : pc);  // multiple of 128
@@ -529,8 +549,8 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
         prm.num_p_tiles = (count / GEMM_BLOCK_P + shape.ctas - 1) / shape.ctas;
         rc = launch_gemm(tmU, tmV, tmM, prm, shape.ctas, st);
         if (rc != SDWINO_OK) return rc;
-        if (tile == 2) rc = launch_output<2>(Mws, bh, yh, geo, K, p0, count, pc, st);
-        else rc = launch_output<4>(Mws, bh, yh, geo, K, p0, count, pc, st);
+        if (tile == 2) rc = launch_output<2>(Mws, bh, yh, geo, K, p0, count, pc, chk, st);
+        else rc = launch_output<4>(Mws, bh, yh, geo, K, p0, count, pc, chk, st);
         if (rc != SDWINO_OK) return rc;
     }
     return SDWINO_OK;
@@ -587,7 +607,7 @@ size_t sdwino_filter_bytes(int K, int C, int tile) {
     if (K <= 0 || C <= 0 || (tile != 2 && tile != 4)) return 0;
     const size_t a = tile + 2;
     const size_t bytes = a * a * static_cast<size_t>((K + 15) / 16) * ((C + 63) / 64) * 1024 * sizeof(__half);
-    return (bytes + WS_ALIGN - 1) / WS_ALIGN * WS_ALIGN;
+    return WT_HEADER_BYTES + (bytes + WS_ALIGN - 1) / WS_ALIGN * WS_ALIGN;   // header + U
 }
 
 int sdwino_filter_transform(const void* w, void* wT, int K, int C, int tile, void* stream) {
@@ -597,8 +617,8 @@ int sdwino_filter_transform(const void* w, void* wT, int K, int C, int tile, voi
     if (static_cast<long double>(K) * C > 4.0e15L) return SDWINO_ERR_INVALID_ARG;
     const int Kb = (K + 15) / 16, Cb = (C + 63) / 64;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (tile == 2) return launch_filter<2>(static_cast<const __half*>(w), static_cast<__half*>(wT), K, C, Kb, Cb, st);
-    return launch_filter<4>(static_cast<const __half*>(w), static_cast<__half*>(wT), K, C, Kb, Cb, st);
+    if (tile == 2) return launch_filter<2>(static_cast<const __half*>(w), wT, K, C, Kb, Cb, st);
+    return launch_filter<4>(static_cast<const __half*>(w), wT, K, C, Kb, Cb, st);
 }
 
 size_t sdwino_workspace_bytes(int N, int C, int H, int W, int K, int tile) {

@@ -101,6 +101,33 @@ __device__ __forceinline__ void mat_apply(MatT coef, const float (&in)[Cn], floa
 }
 
 // ---------------------------------------------------------------------------------------
+// Header of a transformed filter: the first 1024 bytes of wT, written by the filter transform.  Every kernel
+// that reads U first compares it with the layer it was launched for: a buffer that was transformed for another
+// tile size or other channel counts (it may be SMALLER than the one expected) is never read: the kernel records
+// SDWINO_ERR_INVALID_ARG in the device status word and returns.
+// ---------------------------------------------------------------------------------------
+constexpr uint32_t WT_MAGIC = 0x55574453u;   // "SDWU"
+constexpr int WT_HEADER_BYTES = 1024;
+__device__ __forceinline__ bool wt_header_ok(const uint32_t* __restrict__ header, int K, int C, int tile,
+                                             int* status_word) {
+    const uint4 h = *reinterpret_cast<const uint4*>(header);   // plain load: written by an earlier kernel
+    const bool ok = h.x == WT_MAGIC && h.y == static_cast<uint32_t>(K) && h.z == static_cast<uint32_t>(C) &&
+                    h.w == static_cast<uint32_t>(tile);
+    if (!ok && threadIdx.x == 0) atomicCAS(status_word, 0, 1 | (9 << 8));   // 1 = SDWINO_ERR_INVALID_ARG
+    return ok;
+}
+// The same check as one kernel argument (the output transform reads no filters, but leaves y alone when the GEMM
+// before it refused to run).
+struct WtCheck {
+    const uint32_t* header;
+    int K, C, tile;
+    int* status_word;
+};
+__device__ __forceinline__ bool wt_check(const WtCheck& c) {
+    return wt_header_ok(c.header, c.K, c.C, c.tile, c.status_word);
+}
+
+// ---------------------------------------------------------------------------------------
 // Filter preprocess.  U is stored in blocks of 16 output channels x 64 input channels,
 //   U[a*a][Cb][Kb][16][64]   (Kb = ceil(K/16), Cb = ceil(C/64), zeros in the padding),
 // with the blocks of consecutive output channels next to each other, so that the [n_tile k][64 c]
@@ -110,13 +137,17 @@ __device__ __forceinline__ void mat_apply(MatT coef, const float (&in)[Cn], floa
 // ---------------------------------------------------------------------------------------
 template <int M>
 __global__ void __launch_bounds__(128)
-filter_transform_kernel(const __half* __restrict__ w, __half* __restrict__ U, int K, int C, int Kb, int Cb) {
+filter_transform_kernel(const __half* __restrict__ w, uint32_t* __restrict__ header, __half* __restrict__ U, int K,
+                        int C, int Kb, int Cb) {
     using Wm = Wino<M>;
     constexpr int A = Wm::A;
     pdl_launch_dependents();
     pdl_wait();
     const int c = blockIdx.x * blockDim.x + threadIdx.x;
     const int k = blockIdx.y;
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0)
+        *reinterpret_cast<uint4*>(header) = make_uint4(WT_MAGIC, static_cast<uint32_t>(K), static_cast<uint32_t>(C),
+                                                       static_cast<uint32_t>(M));
     if (c >= Cb * 64) return;
     float g[3][3];
     const bool live = (c < C) && (k < K);
@@ -258,11 +289,15 @@ input_transform_kernel(const __half* __restrict__ x, __half* __restrict__ V, Til
 template <int M>
 __global__ void __launch_bounds__(128)
 output_transform_kernel(const __half* __restrict__ Mws, const __half* __restrict__ bias, __half* __restrict__ y,
-                        TileGeom geo, int K, long long p_begin, int p_count, long long Pstride) {
+                        TileGeom geo, int K, long long p_begin, int p_count, long long Pstride, WtCheck chk) {
     using Wm = Wino<M>;
     constexpr int A = Wm::A;
     pdl_launch_dependents();
+    // the header is older than the activation transform two kernels back, which waited for everything before
+    // it: reading it before this kernel's own wait takes the load off the critical path
+    const bool wt_ok = wt_check(chk);
     pdl_wait();
+    if (!wt_ok) return;
     const int pl = blockIdx.x * blockDim.x + threadIdx.x;
     const int k = blockIdx.y;
     if (pl >= p_count) return;
@@ -659,9 +694,11 @@ __device__ __forceinline__ void output_unit_vec(const __half* __restrict__ Mws, 
 template <int M, int TPT>
 __global__ void __launch_bounds__(128)
 output_transform_vec_kernel(const __half* __restrict__ Mws, const __half* __restrict__ bias, __half* __restrict__ y,
-                            TileGeom geo, int K, long long p_begin, FastDiv gdiv, long long Pstride) {
+                            TileGeom geo, int K, long long p_begin, FastDiv gdiv, long long Pstride, WtCheck chk) {
     pdl_launch_dependents();
+    const bool wt_ok = wt_check(chk);   // before the wait: see output_transform_kernel
     pdl_wait();
+    if (!wt_ok) return;
     output_unit_vec<M, TPT>(Mws, bias, y, geo, K, p_begin, gdiv, Pstride, blockIdx.x * blockDim.x + threadIdx.x);
 }
 
@@ -679,14 +716,16 @@ constexpr int FUSED_KC = 8;
 
 template <int M, int CP>
 __global__ void __launch_bounds__(128)
-fused_small_c_kernel(const __half* __restrict__ x, const __half* __restrict__ U, const __half* __restrict__ bias,
-                     __half* __restrict__ y, TileGeom geo, int C, int K, int Kb, int Cb) {
+fused_small_c_kernel(const __half* __restrict__ x, const uint32_t* __restrict__ wt_header,
+                     const __half* __restrict__ U, const __half* __restrict__ bias, __half* __restrict__ y, TileGeom geo,
+                     int C, int K, int Kb, int Cb, int* status_word) {
     using Wm = Wino<M>;
     constexpr int A = Wm::A;
     constexpr int A2 = A * A;
     __shared__ __align__(16) float Us[FUSED_KC][CP][A2];
     pdl_launch_dependents();
     pdl_wait();
+    if (!wt_header_ok(wt_header, K, C, M, status_word)) return;
     const int k0 = blockIdx.y * FUSED_KC;
     // stage the filter chunk: U[pos][Cb][Kb][16][64], this layer has Cb == 1
     const size_t plane = static_cast<size_t>(Kb) * Cb * 1024;
@@ -811,11 +850,13 @@ __device__ __forceinline__ void mma_m16n8k8_f16f32(float (&d)[4], uint32_t a0, u
 // Grid: x = groups of 8 tiles, four per block (one per warp); y = chunks of `kb_per_block` blocks of 16 output
 // channels.  A warp transforms its 8 tiles once and then walks the chunk's output-channel blocks.
 __global__ void __launch_bounds__(128)
-fused_small_c_mma_kernel(const __half* __restrict__ x, const __half* __restrict__ U, const __half* __restrict__ bias,
-                         __half* __restrict__ y, TileGeom geo, int C, int K, int Kb, int kb_per_block) {
+fused_small_c_mma_kernel(const __half* __restrict__ x, const uint32_t* __restrict__ wt_header,
+                         const __half* __restrict__ U, const __half* __restrict__ bias, __half* __restrict__ y,
+                         TileGeom geo, int C, int K, int Kb, int kb_per_block, int* status_word) {
     using Wm = Wino<2>;
     pdl_launch_dependents();
     pdl_wait();
+    if (!wt_header_ok(wt_header, K, C, 2, status_word)) return;
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     const int g = lane >> 2, t = lane & 3;

@@ -64,6 +64,8 @@ struct GemmSmemLayout {
 };
 
 struct GemmParams {
+    const uint32_t* wt_header;   // header of the transformed filter (see wt_header_ok)
+    int K, tile;                 // what the header must say (C is below)
     int num_k_tiles;   // ceil(K / n_tile)
     int num_p_tiles;   // tiles of 128 p (single CTA) or 256 p (CTA pair) in this pass
     int num_pos;       // a*a
@@ -85,6 +87,9 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
 wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant__ CUtensorMap tmV,
                  const __grid_constant__ CUtensorMap tmM, const GemmParams prm, int* __restrict__ status_word) {
     using L = GemmSmemLayout;
+    // The activation transform before this kernel has waited for everything before it, so the filter header is
+    // final: its load is issued first and looked at after the set-up below (uniform over the CTA).
+    const uint4 wt_hdr = *reinterpret_cast<const uint4*>(prm.wt_header);
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int b_rows = prm.n_tile / CTAS;            // rows of U this CTA loads per stage
@@ -133,7 +138,12 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_base_slot;
 
-    if (warp == 0) {
+    const bool wt_ok = wt_hdr.x == WT_MAGIC && wt_hdr.y == static_cast<uint32_t>(prm.K) &&
+                       wt_hdr.z == static_cast<uint32_t>(prm.C) && wt_hdr.w == static_cast<uint32_t>(prm.tile);
+    if (!wt_ok) {
+        // a filter buffer made for another layer: nothing is read from it, nothing is computed
+        if (threadIdx.x == 0) atomicCAS(status_word, 0, 1 | (9 << 8));   // 1 = SDWINO_ERR_INVALID_ARG
+    } else if (warp == 0) {
         // ------------------------------ TMA producer ------------------------------
         if (lane == 0) {
             // the full barrier of a pair lives in the leader and counts the bytes of both CTAs

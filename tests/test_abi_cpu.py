@@ -40,8 +40,9 @@ def test_version_and_status_strings(binding):
 
 def test_size_queries(binding):
     # wT = a*a planes of ceil(K/16) x ceil(C/64) blocks of 16 x 64 fp16
-    assert binding.sdwino_filter_bytes(320, 320, 2) == 16 * 20 * 5 * 1024 * 2
-    assert binding.sdwino_filter_bytes(3, 4, 4) == 36 * 1 * 1 * 1024 * 2
+    # 1 KB header + blocks of 16 x 64 fp16
+    assert binding.sdwino_filter_bytes(320, 320, 2) == 1024 + 16 * 20 * 5 * 1024 * 2
+    assert binding.sdwino_filter_bytes(3, 4, 4) == 1024 + 36 * 1 * 1 * 1024 * 2
     assert binding.sdwino_filter_bytes(0, 4, 2) == 0
     assert binding.sdwino_filter_bytes(4, 4, 3) == 0
     full = binding.sdwino_workspace_bytes(2, 320, 64, 64, 320, 2)

@@ -223,8 +223,10 @@ def test_filter_transform_matches_oracle(B, KC, tile):
     w = (torch.randn(K, C, 3, 3, generator=g) / (9 * C) ** 0.5).half()
     wT = B.sdwino_filter_transform(w.cuda(), tile)
     Kb, Cb = -(-K // 16), -(-C // 64)
-    # U[a*a][Cb][Kb][16][64]  ->  [a*a][Kb*16][Cb*64]
-    U = wT.view(torch.float16)[:a * a * Kb * Cb * 1024].view(a * a, Cb, Kb, 16, 64).permute(0, 2, 3, 1, 4)
+    # header, then U[a*a][Cb][Kb][16][64]  ->  [a*a][Kb*16][Cb*64]
+    hdr = wT[:16].view(torch.int32).cpu().tolist()          # 1 KB header: magic 'SDWU', K, C, tile
+    assert hdr == [0x55574453, K, C, tile]
+    U = wT[1024:].view(torch.float16)[:a * a * Kb * Cb * 1024].view(a * a, Cb, Kb, 16, 64).permute(0, 2, 3, 1, 4)
     U = U.reshape(a * a, Kb * 16, Cb * 64).cpu()
     Uo = oracle.filter_transform(w.numpy(), tile, points=None if tile == 2 else F4_POINTS)
     Uo = torch.from_numpy(Uo.reshape(K, C, a * a).transpose(2, 0, 1).copy())
@@ -459,3 +461,36 @@ def test_relative_error_is_scale_invariant_within_fp16_range(B, tile, scale):
     assert _rel_err(ysc, ref) <= (TOL_F2_REGRESSION if tile == 2 else TOL)
     if scale > 1:      # exact power-of-two scaling without subnormals: bit-identical up to the exponent shift
         assert torch.equal((y.float() * scale).half(), ysc)
+
+
+@pytest.mark.parametrize("case", ["tile", "channels_gemm", "few_in", "few_out"])
+def test_mismatched_filter_buffer_is_reported_and_never_read(B, case):
+    # wT carries a header (tile, K, C); every kernel that reads U checks it first.  A buffer transformed for
+    # another tile size or other channel counts -- possibly much smaller than the one the call expects -- must give
+    # SDWINO_ERR_INVALID_ARG through the device status word, leave the context usable and not touch memory
+    # behind the buffer.
+    if case == "tile":
+        made, used, tile_made, tile_used = (64, 64), (64, 64), 2, 4
+    elif case == "channels_gemm":
+        made, used, tile_made, tile_used = (16, 16), (320, 320), 2, 2          # 50x smaller than expected
+    elif case == "few_in":
+        made, used, tile_made, tile_used = (8, 4), (64, 4), 2, 2               # (K, C): fused few-input-channel kernel
+    else:
+        made, used, tile_made, tile_used = (3, 32), (3, 64), 2, 2              # fused few-output-channel kernel
+    g = torch.Generator().manual_seed(3)
+    w = (torch.randn(made[0], made[1], 3, 3, generator=g) * 0.1).half()
+    wT = B.sdwino_filter_transform(w.cuda(), tile_made)
+    K, C = used
+    H = W = 112 if case == "few_out" else 16
+    N = 2 if case == "few_out" else 1
+    x = torch.randn(N, C, H, W, generator=g).half().cuda()
+    ws = B.alloc_workspace(B.sdwino_workspace_bytes(N, C, H, W, K, tile_used))
+    y = torch.full((N, K, H, W), 7.0, dtype=torch.float16, device="cuda")
+    B.sdwino_conv3x3(x, wT, None, K, tile_used, y=y, workspace=ws)
+    assert B.sdwino_last_device_status() == B.ERR_INVALID_ARG
+    assert B.sdwino_last_device_status() == B.OK
+    assert bool((y == 7.0).all())                           # nothing was computed from the wrong filters
+    # the context is fine: a correct call right after
+    layer = ConvLayer(C=32, K=48, H=10, W=12, N=1)
+    xx, ww, bb, yy = _run(B, layer, 2, seed=2)
+    assert _rel_err(yy, oracle.direct_conv3x3(xx.numpy(), ww.numpy(), bb.numpy())) <= TOL_F2_REGRESSION
