@@ -874,16 +874,16 @@ fused_small_c_mma_kernel(const __half* __restrict__ x, const uint32_t* __restric
         const bool p_ok = p < geo.P;
         if (p_ok) decode_tile(geo, p, n, th, tw);
         const int i0 = 2 * th - 1, j0 = 2 * tw - 1;
-        uint32_t packed[2][16];   // per round: (V[c even], V[c odd]) of tile g, valid in the even-channel lanes
+        uint32_t packed[2][16];   // per channel quad: (V[c even], V[c odd]) of tile g, valid in the even-channel lanes
 #pragma unroll
-        for (int round = 0; round < 2; ++round) {
-            const int c = 4 * round + t;
+        for (int quad = 0; quad < 2; ++quad) {
+            const int c = 4 * quad + t;
             float d[4][4];
 #pragma unroll
             for (int r = 0; r < 4; ++r)
 #pragma unroll
                 for (int s2 = 0; s2 < 4; ++s2) d[r][s2] = 0.f;
-            if (p_ok && c < C) {       // round 1 is skipped by every lane when C <= 4
+            if (p_ok && c < C) {       // the second quad is skipped by every lane when C <= 4
                 const __half* img = x + (n * C + c) * hw;
 #pragma unroll
                 for (int r = 0; r < 4; ++r) {
@@ -910,12 +910,12 @@ fused_small_c_mma_kernel(const __half* __restrict__ x, const uint32_t* __restric
                 for (int xi = 0; xi < 4; ++xi) {
                     const float mine = o[xi];
                     const float other = __shfl_xor_sync(0xffffffffu, mine, 1);   // channel c ^ 1 of the same tile
-                    packed[round][xi * 4 + nu] = pack2(mine, other);            // meaningful where c is even
+                    packed[quad][xi * 4 + nu] = pack2(mine, other);            // meaningful where c is even
                 }
             }
             if (C <= 4) break;   // uniform
         }
-        // B fragment of lane (g, t): channels 2t, 2t+1 of tile g = the packed pair of lane (g, (2t) & 3), round t >> 1
+        // B fragment of lane (g, t): channels 2t, 2t+1 of tile g = the packed pair of lane (g, (2t) & 3), quad t >> 1
         const int src = (g << 2) | ((2 * t) & 3);
 #pragma unroll
         for (int pos = 0; pos < 16; ++pos) {
