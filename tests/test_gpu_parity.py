@@ -494,3 +494,31 @@ def test_mismatched_filter_buffer_is_reported_and_never_read(B, case):
     layer = ConvLayer(C=32, K=48, H=10, W=12, N=1)
     xx, ww, bb, yy = _run(B, layer, 2, seed=2)
     assert _rel_err(yy, oracle.direct_conv3x3(xx.numpy(), ww.numpy(), bb.numpy())) <= TOL_F2_REGRESSION
+
+
+@pytest.mark.parametrize("force_gemm", [False, True])
+def test_hand_worked_example_bit_exact(B, force_gemm):
+    # tests/golden/hand_worked_4x4.txt: every value of the example is representable in fp16 and every partial sum
+    # exact, so F(2x2) must reproduce the hand-computed y bit for bit -- through the few-channel kernel and
+    # through the three-kernel path
+    import os
+    rows, on = [], False
+    with open(os.path.join(os.path.dirname(__file__), "golden", "hand_worked_4x4.txt")) as f:
+        for line in f:
+            line = line.strip()
+            if line.startswith("["):
+                on = line == "[y]"
+            elif on and line and not line.startswith("#"):
+                rows.append([float(v) for v in line.split()])
+    want = torch.tensor(rows, dtype=torch.float16)
+    x = torch.arange(1, 17, dtype=torch.float16).reshape(1, 1, 4, 4)
+    w = torch.arange(1, 10, dtype=torch.float16).reshape(1, 1, 3, 3)
+    b = torch.tensor([0.5], dtype=torch.float16)
+    layer = ConvLayer(C=1, K=1, H=4, W=4, N=1)
+    if force_gemm:
+        B.sdwino_set_gemm_shape(1, 16)
+    try:
+        _, _, _, y = _run(B, layer, 2, x=x, w=w, b=b)
+    finally:
+        B.sdwino_set_gemm_shape(0, 0)
+    assert torch.equal(y[0, 0], want)

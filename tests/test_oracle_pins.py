@@ -78,6 +78,32 @@ HAND_Y = np.array([[111.5, 178.5, 217.5, 145.5], [231.5, 348.5, 393.5, 252.5],
                    [363.5, 528.5, 573.5, 360.5], [197.5, 274.5, 295.5, 175.5]])
 
 
+def _load_golden(name):
+    """Sections of a text fixture under tests/golden/ as float64 matrices ('#' lines are the citation)."""
+    import os
+    out, cur = {}, None
+    with open(os.path.join(os.path.dirname(__file__), "golden", name)) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            if line.startswith("["):
+                cur = line.strip("[]")
+                out[cur] = []
+            else:
+                out[cur].append([float(v) for v in line.split()])
+    return {k: np.array(v) for k, v in out.items()}
+
+
+def test_golden_fixture_matches_the_inline_hand_values():
+    g = _load_golden("hand_worked_4x4.txt")
+    assert np.array_equal(g["y"], HAND_Y)
+    x, w, b = _hand_inputs()
+    assert np.array_equal(oracle.direct_conv3x3(x, w, b)[0, 0], g["y"])
+    assert np.array_equal(oracle.filter_transform(w, 2)[0, 0], g["U"])
+    assert np.array_equal(oracle.input_tile_transform(x, 0, 0, 0, 2)[0], g["V_tile00"])
+
+
 def _hand_inputs():
     x = np.arange(1, 17, dtype=np.float64).reshape(1, 1, 4, 4)
     w = np.arange(1, 10, dtype=np.float64).reshape(1, 1, 3, 3)
