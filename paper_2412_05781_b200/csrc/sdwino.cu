@@ -405,27 +405,40 @@ int launch_fused_small_c_mma(const __half* x, const void* wT, const __half* bias
 // pipeline stages, each limited by the tensor pipe (2 n cycles per stage) or by the bytes the CTA must
 // fetch from L2 per stage (about 40 bytes per cycle per SM were measured), plus an epilogue that is
 // hidden unless the tile is short; tiles run in waves over the SMs.
+//
+// A CTA pair fetches half of the filter rows per CTA.  Measured over the layers of all workloads it is 4-10 % faster
+// for the layer where the mainloop dominates (C >= 512, several waves of 256-channel tiles), and slower where
+// tiles are short (its epilogue hand-off crosses two CTAs), where an odd number of 128-tile blocks leaves half a
+// pair idle, and for short launches (it runs without programmatic dependent launch, see launch_gemm_shape).  The
+// constants below reproduce that: 35 bytes per cycle per CTA of a pair (on the scale where a single CTA gets 40),
+// epilogue x 1.35 and a fixed charge for the lost overlap.
 struct GemmShape { int ctas; int n_tile; };
-GemmShape choose_gemm_shape(int K, int C, long long p_tiles128, int a2, int sms) {
+GemmShape choose_gemm_shape(int K, int C, long long p_tiles128, int a2, int sms, int force_ctas) {
     const long long cblocks = (C + GEMM_BLOCK_C - 1) / GEMM_BLOCK_C;
     GemmShape best{1, 16};
     double best_cost = 1e300;
-    // CTA pairs never beat single CTAs in measurement (the mainloop is not bound by L2 bytes) and cannot use
-    // programmatic dependent launch, so they are only taken when forced through sdwino_set_gemm_shape.
-    for (int ctas = 1; ctas <= 1; ++ctas) {
+    // a pair needs two blocks of 128 tiles; with fewer than 8 stages per tile it measured 4-35 % slower
+    const int max_ctas = p_tiles128 >= 2 && (cblocks >= 8 || force_ctas == 2) ? 2 : 1;
+    for (int ctas = 1; ctas <= max_ctas; ++ctas) {
+        if (force_ctas != 0 && ctas != (force_ctas < max_ctas ? force_ctas : max_ctas)) continue;
         const long long p_tiles = (p_tiles128 + ctas - 1) / ctas;
         const long long workers = sms / ctas;
-        for (int n = 16; n <= GEMM_MAX_N; n += 16) {
+        const int step = 16 * ctas;   // each CTA of a pair loads whole 16-row blocks
+        for (int n = step; n <= GEMM_MAX_N; n += step) {
             const long long ktiles = (K + n - 1) / n;
-            if (n > 16 && (ktiles == (K + n - 17) / (n - 16))) continue;  // a smaller n needs as many tiles
+            if (n > step && (ktiles == (K + n - step - 1) / (n - step))) continue;  // a smaller n needs as many tiles
             const long long tiles = ktiles * p_tiles * a2;
             const long long waves = (tiles + workers - 1) / workers;
+            // with one or two tiles per pair the fixed cost of a pair is not paid back (measured 9-12 % slower)
+            if (ctas == 2 && force_ctas != 2 && waves < 3) continue;
             const double mma = 2.0 * n;
-            const double load = (GemmSmemLayout::A_BYTES + 128.0 * n / ctas) / 40.0;
+            const double load = ctas == 1 ? (GemmSmemLayout::A_BYTES + 128.0 * n) / 40.0
+                                          : (GemmSmemLayout::A_BYTES + 64.0 * n) / 35.0;
             const double main = cblocks * (mma > load ? mma : load);
-            const double epi = 300.0 + 14.0 * n;
-            const double per_tile = (main > epi ? main : epi) + 200.0;
-            const double cost = (waves * per_tile + epi) * (ctas == 2 ? 1.05 : 1.0);  // pairs must win clearly
+            const double epi = (300.0 + 14.0 * n) * (ctas == 2 ? 1.35 : 1.0);
+            const double per_tile = (main > epi ? main : epi) + (ctas == 2 ? 400.0 : 200.0);
+            const double fixed = ctas == 2 ? 7000.0 : 0.0;
+            const double cost = waves * per_tile + epi + fixed;
             if (cost < best_cost) { best_cost = cost; best = GemmShape{ctas, n}; }
         }
     }
@@ -508,8 +521,7 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
     prm.wt_header = wt_header_of(wT);
     prm.K = K;
     prm.tile = tile;
-    GemmShape shape = choose_gemm_shape(K, C, pc / GEMM_BLOCK_P, pl.a2, sms);
-    if (g_force_ctas == 1 || g_force_ctas == 2) shape.ctas = (pc / GEMM_BLOCK_P < 2) ? 1 : g_force_ctas;
+    GemmShape shape = choose_gemm_shape(K, C, pc / GEMM_BLOCK_P, pl.a2, sms, g_force_ctas);
     if (g_force_n_tile >= 16 && g_force_n_tile <= GEMM_MAX_N && g_force_n_tile % 16 == 0) shape.n_tile = g_force_n_tile;
     if (shape.ctas == 2) shape.n_tile = round_up(shape.n_tile, 32);  // each CTA of a pair loads whole 16-row blocks
     prm.n_tile = shape.n_tile;
