@@ -387,10 +387,14 @@ int launch_fused_small_c_mma(const __half* x, const void* wT, const __half* bias
     if (sms <= 0 || !status) return SDWINO_ERR_CUDA;
     const long long groups = (geo.P + 7) / 8;
     const long long blocks_x = (groups + 3) / 4;
-    // about four blocks per SM: split the output-channel blocks over grid.y until there are enough
-    long long ksplit = (static_cast<long long>(sms) * 4 + blocks_x - 1) / blocks_x;
-    ksplit = ksplit < 1 ? 1 : (ksplit > Kb ? Kb : ksplit);
-    const int kb_per_block = static_cast<int>((Kb + ksplit - 1) / ksplit);
+    // The kernel is a latency chain per warp (load, transform, then per block of output channels MMAs, output
+    // transform, store): it runs best with 12-14 warps per SM.  Fewer output-channel blocks per CTA shorten the
+    // chain but repeat the input transform and the filter staging; more than 3.5 CTAs per SM measured slower
+    // again (4->320 at 64x64, batch 2: 10.2 / 9.0 / 7.6 / 8.9 / 11.7 us with 1 / 2 / 3 / 4 / 7 blocks per CTA).
+    int kb_per_block = Kb;
+    for (int cand = 1; cand <= Kb; ++cand) {
+        if (blocks_x * ((Kb + cand - 1) / cand) * 2 <= static_cast<long long>(sms) * 7) { kb_per_block = cand; break; }
+    }
     dim3 grid(static_cast<unsigned>(blocks_x), static_cast<unsigned>((Kb + kb_per_block - 1) / kb_per_block));
     ProfScope prof(KIND_FUSED, st);
     const cudaError_t e = launch_pdl(fused_small_c_mma_kernel, grid, dim3(128), 0, st, 0, x, wt_header_of(wT),

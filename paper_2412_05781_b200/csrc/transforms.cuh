@@ -840,6 +840,15 @@ fused_small_c_kernel(const __half* __restrict__ x, const uint32_t* __restrict__ 
 // 36 positions x 4 accumulators would not fit the registers).  tcgen05 is not used here: its smallest tile
 // (64 x 8 x 16 per instruction, operands staged in shared memory) does not pay for a contraction of 4.
 // ---------------------------------------------------------------------------------------
+// 16-byte asynchronous copy global -> shared memory (no register staging) and the wait for all copies of the thread
+__device__ __forceinline__ void cp_async_16(void* smem_dst, const void* gmem_src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst))),
+                 "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
+constexpr int FC_KB_CHUNK = 4;   // blocks of 16 output channels staged in shared memory at a time (16 KB)
+
 __device__ __forceinline__ void mma_m16n8k8_f16f32(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t b0) {
     asm volatile(
         "mma.sync.aligned.m16n8k8.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5}, {%6}, {%0, %1, %2, %3};"
@@ -863,11 +872,25 @@ fused_small_c_mma_kernel(const __half* __restrict__ x, const uint32_t* __restric
     const long long hw = static_cast<long long>(geo.H) * geo.W;
     const long long num_groups = (geo.P + 7) / 8;
     const long long grp = static_cast<long long>(blockIdx.x) * 4 + warp;
-    if (grp >= num_groups) return;   // warp-uniform; the kernel has no block-wide barrier
+    const bool active = grp < num_groups;   // warp-uniform; idle warps still help to stage the filters
+    // The used part of a filter block (16 rows x 8 channels = 16 bytes of every 128-byte row) is staged in shared
+    // memory once per block of four warps: fragment loads straight from global memory touch eight 128-byte
+    // lines per instruction and kept the L1 at 77 % of its peak, which bounded the kernel.
+    __shared__ uint4 sU[FC_KB_CHUNK][16][16];   // [block of 16 output channels][position][row]: channels 0..7
+    const int kb_begin = blockIdx.y * kb_per_block;
+    const int kb_end = min(Kb, kb_begin + kb_per_block);
+    const size_t plane = static_cast<size_t>(Kb) * 1024;   // one position of U, in elements
+    auto stage_filters = [&](int kb0, int chunk) {
+        for (int i = threadIdx.x; i < chunk * 256; i += 128) {
+            const int row = i & 15, pos = (i >> 4) & 15, kbi = i >> 8;
+            cp_async_16(&sU[kbi][pos][row], U + pos * plane + (static_cast<size_t>(kb0 + kbi) * 16 + row) * 64);
+        }
+    };
+    stage_filters(kb_begin, min(FC_KB_CHUNK, kb_end - kb_begin));   // in flight during the input transform
 
     // ---- input transform: lane (g, t) transforms tile g of the group for channel t (and t + 4 if C > 4) ----
     uint32_t bfrag[16];
-    {
+    if (active) {
         const long long p = grp * 8 + g;
         int tw = 0, th = 0;
         long long n = 0;
@@ -947,17 +970,23 @@ fused_small_c_mma_kernel(const __half* __restrict__ x, const uint32_t* __restric
     // W % 4 == 0 makes TW even, so tiles 2t and 2t+1 of a group always share a tile row
     const bool pair_ok = ((geo.W & 3) == 0) && ((reinterpret_cast<uintptr_t>(y) & 7) == 0) && out_off[1] >= 0;
 
-    const int kb_end = min(Kb, static_cast<int>(blockIdx.y + 1) * kb_per_block);
-    const size_t plane_w = static_cast<size_t>(Kb) * 512;   // one position of U, in 32-bit words
-    for (int kb = blockIdx.y * kb_per_block; kb < kb_end; ++kb) {
+    for (int kb0 = kb_begin; kb0 < kb_end; kb0 += FC_KB_CHUNK) {
+    const int chunk = min(FC_KB_CHUNK, kb_end - kb0);
+    if (kb0 != kb_begin) {
+        __syncthreads();   // the previous chunk has been read
+        stage_filters(kb0, chunk);
+    }
+    cp_async_wait_all();
+    __syncthreads();
+    if (!active) continue;
+    for (int kb = kb0; kb < kb0 + chunk; ++kb) {
         // A fragments: U[pos][kb][0][row][c], rows g and g+8, channels 2t, 2t+1 (zeros past K and C)
-        const uint32_t* Uw = reinterpret_cast<const uint32_t*>(U + (static_cast<size_t>(kb) * 16 + g) * 64 + 2 * t);
         float acc[16][4];   // acc[pos] = {M[g][2t], M[g][2t+1], M[g+8][2t], M[g+8][2t+1]}
 #pragma unroll
         for (int pos = 0; pos < 16; ++pos) {
             acc[pos][0] = acc[pos][1] = acc[pos][2] = acc[pos][3] = 0.f;
-            const uint32_t a0 = __ldg(Uw + pos * plane_w);
-            const uint32_t a1 = __ldg(Uw + pos * plane_w + 8 * 32);
+            const uint32_t a0 = reinterpret_cast<const uint32_t*>(&sU[kb - kb0][pos][g])[t];
+            const uint32_t a1 = reinterpret_cast<const uint32_t*>(&sU[kb - kb0][pos][g + 8])[t];
             mma_m16n8k8_f16f32(acc[pos], a0, a1, bfrag[pos]);
         }
 #pragma unroll
@@ -1010,6 +1039,7 @@ fused_small_c_mma_kernel(const __half* __restrict__ x, const uint32_t* __restric
             }
         }
     }
+    }   // chunks of output-channel blocks
 }
 
 }  // namespace sdw
