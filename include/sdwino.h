@@ -176,6 +176,15 @@ unsigned long long sdwino_launch_count(void);
 int sdwino_set_gemm_shape(int ctas, int n_tile);
 
 /*
+ * Test hook for the activation transform of step (i) with tile = 4.  A layer that is done in one pass, with
+ * W % 8 == 0 and a 16-byte aligned x, can stage the overlapping input tiles in shared memory by TMA instead of
+ * loading them into registers; both kernels produce the same bits.  mode 1 (the default) stages where that
+ * measured faster (W % 64 == 0), mode 2 wherever it is possible, mode 0 never.  Returns SDWINO_ERR_INVALID_ARG
+ * for any other value.  Not thread-safe against concurrent compute calls.
+ */
+int sdwino_set_input_staging(int mode);
+
+/*
  * Which of the two supported algorithms is expected to be faster for a layer: returns 2 for F(2x2,3x3),
  * 4 for F(4x4,3x3), 0 for non-positive sizes.  The paper leaves the tile size open; both satisfy the
  * accuracy bound (F4 with about 4x the error of F2).  Rule, with tiles = N * ceil(H/2) * ceil(W/2):

@@ -22,7 +22,7 @@ EXPORTS = [
     "sdwino_conv3x3_ws", "sdwino_host_staging_bytes", "sdwino_conv3x3_host",
     "sdwino_last_device_status", "sdwino_launch_count", "sdwino_profile_enable", "sdwino_profile_collect",
     "sdwino_profile_records", "sdwino_set_gemm_shape", "sdwino_conv3x3_static", "sdwino_set_fused_min_tiles", "sdwino_choose_tile",
-    "sdwino_selftest_wait_timeout", "sdwino_conv3x3_host_async", "sdwino_host_join",
+    "sdwino_selftest_wait_timeout", "sdwino_conv3x3_host_async", "sdwino_host_join", "sdwino_set_input_staging",
 ]
 
 KERNEL_KINDS = ("filter_transform", "input_transform", "wino_gemm", "output_transform", "fused")
@@ -72,6 +72,8 @@ def _load() -> ctypes.CDLL:
     lib.sdwino_profile_records.argtypes = [ctypes.POINTER(i), ctypes.POINTER(ctypes.c_float), i, i]
     lib.sdwino_set_gemm_shape.restype = i
     lib.sdwino_set_gemm_shape.argtypes = [i, i]
+    lib.sdwino_set_input_staging.restype = i
+    lib.sdwino_set_input_staging.argtypes = [i]
     lib.sdwino_selftest_wait_timeout.restype = i
     lib.sdwino_selftest_wait_timeout.argtypes = [ctypes.c_ulonglong, vp]
     lib.sdwino_choose_tile.restype = i
@@ -142,6 +144,12 @@ def sdwino_selftest_wait_timeout(limit_ns: int, stream: Optional[torch.cuda.Stre
 def sdwino_set_gemm_shape(ctas: int = 0, n_tile: int = 0) -> None:
     """Force single-CTA (1) or CTA-pair (2) GEMM tiles and/or the channels per tile; 0 = automatic."""
     _check(lib.sdwino_set_gemm_shape(ctas, n_tile), "sdwino_set_gemm_shape")
+
+
+def sdwino_set_input_staging(mode: int = 1) -> None:
+    """Test hook for the F(4x4) activation transform: 0 register-only kernel, 1 automatic, 2 TMA-staged kernel
+    wherever it applies."""
+    _check(lib.sdwino_set_input_staging(int(mode)), "sdwino_set_input_staging")
 
 
 def sdwino_choose_tile(N: int, C: int, H: int, W: int, K: int) -> int:

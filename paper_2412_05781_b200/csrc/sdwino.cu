@@ -9,6 +9,7 @@
 #include <stdio.h>
 #include <stdlib.h>
 
+#include <algorithm>
 #include <atomic>
 #include <utility>
 #include <mutex>
@@ -17,6 +18,7 @@
 #include "transforms.cuh"
 #include "wino_gemm.cuh"
 #include "fused_small_k.cuh"
+#include "input_tma.cuh"
 
 namespace {
 
@@ -28,6 +30,7 @@ std::atomic<unsigned long long> g_launches{0};
 std::mutex g_mutex;
 // test / tuning overrides of the GEMM launch shape (0 = choose automatically)
 int g_force_ctas = 0;
+int g_input_staging = 1;  // 0 never, 1 where it is faster, 2 wherever possible (sdwino_set_input_staging)
 bool g_disable_fused = false;  // forcing a GEMM shape also forces the GEMM path for few-channel layers
 int g_force_n_tile = 0;
 void* g_workspace = nullptr;
@@ -232,6 +235,31 @@ int* status_word_ptr() {
 inline const uint32_t* wt_header_of(const void* wT) { return static_cast<const uint32_t*>(wT); }
 inline const void* wt_filters_of(const void* wT) { return static_cast<const uint8_t*>(wT) + WT_HEADER_BYTES; }
 
+// x as a 3-D tensor [N * C][H][W] with a box of bw x bh pixels of cpb channel images (no swizzle, zeros outside).
+bool encode_image_map(CUtensorMap* m, const void* base, uint64_t W, uint64_t H, uint64_t NC, uint32_t bw, uint32_t bh,
+                      uint32_t cpb) {
+    const MapKey key{base, W, H, NC, ~1ull, cpb, bw, bh, false};
+    const uint64_t h = (reinterpret_cast<uintptr_t>(base) >> 8) * 1000003u ^ W * 31u ^ H * 131u ^ NC * 7u ^ (bw << 9) ^
+                       (bh << 17) ^ (cpb << 25) ^ 3u;
+    MapSlot& slot = g_map_cache[h % MAP_CACHE_SLOTS];
+    std::lock_guard<std::mutex> lock(g_map_mutex);
+    if (slot.used && slot.key == key) { *m = slot.map; return true; }
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {W, H, NC};
+    cuuint64_t strides[2] = {W * sizeof(__half), H * W * sizeof(__half)};
+    cuuint32_t box[3] = {bw, bh, cpb};
+    cuuint32_t estr[3] = {1, 1, 1};
+    if (fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    slot.key = key;
+    slot.map = *m;
+    slot.used = true;
+    return true;
+}
+
 // Kernels are launched with programmatic stream serialization (see pdl_wait in ptx.cuh); cluster_x: 0 for
 // the transform kernels, 1 or 2 CTAs per cluster for the GEMM.
 template <typename... KArgs, typename... Args>
@@ -297,6 +325,86 @@ int launch_input(const __half* x, __half* V, const TileGeom& geo, int C, long lo
         dim3 grid((p_count + 127) / 128, C);
         e = launch_pdl(input_transform_kernel<M>, grid, dim3(128), 0, st, 0, x, V, geo, C, p_begin, p_count, Pstride);
     }
+    g_launches.fetch_add(1);
+    return e == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
+}
+
+
+// The TMA-staged F(4x4) activation transform covers a layer done in one pass whose rows TMA can address.
+bool use_input_tma(const TileGeom& geo, int N, int C, const void* x, long long p_begin, long long p_count,
+                   long long P128) {
+    const bool possible = p_begin == 0 && p_count == P128 && geo.W % 8 == 0 && aligned(x, 16) &&
+                          static_cast<long long>(N) * C < (1ll << 31) && geo.TH < (1 << 20);
+    if (!possible || g_input_staging == 0) return false;
+    // Faster where a block row is a whole number of 32-byte sectors of V (W % 64 == 0: 15.8 against 17.0 us on
+    // 960->320 at 64x64, 45.6 against 60.5 us on 512->512 at 256x256).  Image widths of 32 (8 tiles per row,
+    // four channel images per step) come out even, widths of 24, 48 and 96 up to 2x slower: their rows of 6, 12
+    // and 24 tiles leave runs of V that start and end inside sectors, where the register-only kernel, whose
+    // threads follow the tile index, always stores whole 128-byte lines.
+    return g_input_staging == 2 || geo.TW % 16 == 0;
+}
+
+int launch_input_tma(const __half* x, __half* V, const TileGeom& geo, int N, int C, long long Pstride, cudaStream_t st) {
+    ProfScope prof(KIND_INPUT, st);
+    const int sms = sm_count();
+    int* status = status_word_ptr();
+    if (sms <= 0 || !status) return SDWINO_ERR_CUDA;
+    InTmaParams q;
+    q.C = C; q.TH = geo.TH; q.TW = geo.TW; q.P = geo.P; q.Pstride = Pstride;
+    // A block of up to 256 tiles (128 threads).  Blocks span the full width of the image when it has at most 60
+    // tiles per row, otherwise at least 32 tiles: the tiles of a block row (of the whole block, at full width) are
+    // then consecutive in V, and a warp stores runs of at least 64 bytes (narrower blocks measured 2-3x slower:
+    // 8-byte pieces per store).  Among those, the shape that leaves the fewest threads without a tile -- over the
+    // tiles that hang over the right and bottom edges and the threads that no channel image fills --, and among
+    // equals the one that fetches the smallest halo.
+    int best_half = 1, best_trb = 1;
+    double best_score = -1e30;
+    const int half_full = geo.TW / 2;   // W % 8 == 0: TW is even
+    for (int half = (half_full <= 30 ? half_full : 16); half <= (half_full <= 30 ? half_full : 30); ++half) {
+        const int sbc = (geo.TW + 2 * half - 1) / (2 * half);
+        for (int trb = 1; trb <= 32 && half * trb <= 128; ++trb) {
+            const int sbr = (geo.TH + trb - 1) / trb;
+            const int cpb = std::min(16, 128 / (half * trb));
+            double used = static_cast<double>(geo.TW) * geo.TH / (static_cast<double>(sbc) * 2 * half * sbr * trb) *
+                          (half * trb * cpb / 128.0);
+            const int run = half_full <= 30 ? std::min(trb, geo.TH) * geo.TW : 2 * half;   // consecutive tiles in V
+            if (run < 32) used *= run / 32.0;
+            const double halo = (8.0 * half + 16) * (4.0 * trb + 2) / (32.0 * half * trb);
+            const double score = used - 0.02 * halo;
+            if (score > best_score) { best_score = score; best_half = half; best_trb = trb; }
+        }
+    }
+    const int tcb = 2 * best_half;
+    q.tcb_half = best_half;
+    q.trb = best_trb;
+    q.cpb = std::min(16, 128 / (best_half * best_trb));
+    q.bw = 4 * tcb + 16;
+    q.bh = 4 * q.trb + 2;
+    q.sb_c = (geo.TW + tcb - 1) / tcb;
+    q.sb_r = (geo.TH + q.trb - 1) / q.trb;
+    q.stage_bytes = (q.bw * q.bh * q.cpb * 2 + 127) / 128 * 128;
+    const long long blocks = static_cast<long long>(N) * q.sb_c * q.sb_r;
+    const long long csteps = (C + q.cpb - 1) / q.cpb;
+    // enough CTAs for four per SM, at most 16 steps each
+    long long steps = blocks * csteps / (4ll * sms);
+    steps = steps < 1 ? 1 : (steps > 16 ? 16 : steps);
+    steps = steps > csteps ? csteps : steps;
+    q.steps = static_cast<int>(steps);
+    const long long grid_y = (csteps + steps - 1) / steps;
+    if (blocks >= (1ll << 31) || grid_y > 65535) return SDWINO_ERR_UNSUPPORTED;
+    CUtensorMap tmX;
+    if (!encode_image_map(&tmX, x, geo.W, geo.H, static_cast<uint64_t>(N) * C, q.bw, q.bh, q.cpb)) return SDWINO_ERR_CUDA;
+    const size_t smem = static_cast<size_t>(IN_TMA_STAGES) * q.stage_bytes + 128;
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [&] {
+        attr_err = cudaFuncSetAttribute(input_transform_f4_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        IN_TMA_STAGES * 32 * 1024 + 128);
+    });
+    if (attr_err != cudaSuccess || smem > IN_TMA_STAGES * 32 * 1024 + 128) return SDWINO_ERR_CUDA;
+    dim3 grid(static_cast<unsigned>(blocks), static_cast<unsigned>(grid_y));
+    const cudaError_t e = launch_pdl(input_transform_f4_tma_kernel, grid, dim3(IN_TMA_THREADS), smem, st, 0, tmX, V, q,
+                                     status);
     g_launches.fetch_add(1);
     return e == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
 }
@@ -560,6 +668,7 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
         const int count = static_cast<int>(remaining < pc ? remaining : pc);  // multiple of 128
         int rc;
         if (tile == 2) rc = launch_input<2>(xh, V, geo, C, p0, count, pc, st);
+        else if (use_input_tma(geo, N, C, x, p0, count, pl.P128)) rc = launch_input_tma(xh, V, geo, N, C, pc, st);
         else rc = launch_input<4>(xh, V, geo, C, p0, count, pc, st);
         if (rc != SDWINO_OK) return rc;
         prm.num_p_tiles = (count / GEMM_BLOCK_P + shape.ctas - 1) / shape.ctas;
@@ -583,6 +692,12 @@ int sdwino_set_gemm_shape(int ctas, int n_tile) {
     g_force_ctas = ctas;
     g_force_n_tile = n_tile;
     g_disable_fused = (ctas != 0 || n_tile != 0);
+    return SDWINO_OK;
+}
+
+int sdwino_set_input_staging(int mode) {
+    if (mode < 0 || mode > 2) return SDWINO_ERR_INVALID_ARG;
+    g_input_staging = mode;
     return SDWINO_OK;
 }
 

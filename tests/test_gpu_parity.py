@@ -522,3 +522,24 @@ def test_hand_worked_example_bit_exact(B, force_gemm):
     finally:
         B.sdwino_set_gemm_shape(0, 0)
     assert torch.equal(y[0, 0], want)
+
+
+@pytest.mark.parametrize("shape", [(64, 48, 64, 64, 2), (40, 16, 32, 32, 1), (24, 32, 16, 16, 3), (16, 16, 8, 8, 2),
+                                   (9, 16, 20, 40, 1), (130, 16, 37, 24, 1), (12, 16, 140, 136, 1), (10, 16, 5, 8, 5),
+                                   (33, 16, 260, 8, 1), (20, 16, 3, 264, 1), (6, 16, 248, 248, 1), (70, 16, 96, 96, 2)])
+def test_staged_activation_transform_matches_register_kernel_bitwise(B, shape):
+    # F(4x4), one pass, W % 8 == 0: the activation transform stages its input tiles in shared memory by TMA.  It
+    # must produce the bits of the register-only kernel (same arithmetic) for whole-image blocks, blocks that
+    # hang over the right and bottom edges, several channel images per step, and ragged channel counts.
+    C, K, H, W, N = shape
+    layer = ConvLayer(C=C, K=K, H=H, W=W, N=N)
+    B.sdwino_set_input_staging(2)
+    try:
+        x, w, b, y_staged = _run(B, layer, 4, seed=7)
+        B.sdwino_set_input_staging(0)
+        _, _, _, y_regs = _run(B, layer, 4, x=x, w=w, b=b)
+    finally:
+        B.sdwino_set_input_staging(1)
+    assert torch.equal(y_staged, y_regs)
+    ref = oracle.direct_conv3x3(x.numpy(), w.numpy(), b.numpy())
+    assert _rel_err(y_staged, ref) <= TOL
