@@ -12,8 +12,8 @@
 // shared memory (one 16-byte and two 4-byte reads per row), releases the stage and applies B^T . B in packed
 // two-wide fp32 exactly like the register-only kernel, so both produce the same bits.
 //
-// Used when a layer is one pass (p_begin = 0, every tile of the layer in this launch) with W % 8 == 0 and a
-// 16-byte aligned x; other cases keep the register-only kernels.
+// A launch covers a pass of whole tile rows (the passes of a large layer are cut at multiples of the tiles per
+// row).  Needs W % 8 == 0 and a 16-byte aligned x; other cases keep the register-only kernels.
 #pragma once
 #include <cuda_fp16.h>
 
@@ -35,8 +35,11 @@ struct InTmaParams {
     int sb_c, sb_r;      // blocks per image along the columns / rows
     int steps;           // steps (groups of cpb channels) per CTA
     int stage_bytes;     // bw * bh * cpb * 2, rounded up to 128
-    long long P;         // tiles of the layer
-    long long Pstride;   // tiles per row of V (a multiple of 128, >= P)
+    long long Pstride;   // tiles per row of V (a multiple of 128)
+    long long p_begin;   // first tile of this pass (a multiple of TW)
+    long long g_begin, g_end;   // this pass covers the tile rows g = n * TH + th in [g_begin, g_end)
+    long long tail_begin, tail_end;   // tiles (relative to p_begin) past the last one of the pass: stored as zeros
+    int tail_block;      // the block (blockIdx.x) that stores them
 };
 
 // tmX: fp16 [N * C][H][W], box {bw, bh, cpb}, no swizzle, zero fill outside
@@ -57,6 +60,12 @@ input_transform_f4_tma_kernel(const __grid_constant__ CUtensorMap tmX, __half* _
     const int bc = blockIdx.x - n * sb - br * prm.sb_c;
     const int tcb = prm.tcb_half * 2;
     const int th0 = br * prm.trb, tw0 = bc * tcb;
+    // a block none of whose tile rows belong to this pass has nothing to do (a layer done in several passes)
+    {
+        const long long g_lo = static_cast<long long>(n) * prm.TH + th0;
+        const long long g_hi = static_cast<long long>(n) * prm.TH + (th0 + prm.trb < prm.TH ? th0 + prm.trb : prm.TH);
+        if (g_hi <= prm.g_begin || g_lo >= prm.g_end) return;
+    }
     const int c_first = blockIdx.y * prm.steps * prm.cpb;
     int steps = (prm.C - c_first + prm.cpb - 1) / prm.cpb;
     steps = steps < prm.steps ? steps : prm.steps;
@@ -87,9 +96,11 @@ input_transform_f4_tma_kernel(const __grid_constant__ CUtensorMap tmX, __half* _
     const int r = rest % prm.trb;
     const int cl = rest / prm.trb;
     const int th = th0 + r, tw = tw0 + 2 * j;
-    const bool tile_ok = cl < prm.cpb && th < prm.TH && tw < prm.TW;   // W % 8 == 0: TW is even, tw + 1 < TW as well
+    const long long g = static_cast<long long>(n) * prm.TH + th;   // tile row over all images
+    // W % 8 == 0: TW is even, so tile tw + 1 exists whenever tile tw does
+    const bool tile_ok = cl < prm.cpb && th < prm.TH && tw < prm.TW && g >= prm.g_begin && g < prm.g_end;
     const long long plane = static_cast<long long>(prm.C) * prm.Pstride;
-    const long long p = (static_cast<long long>(n) * prm.TH + th) * prm.TW + tw;
+    const long long p = g * prm.TW + tw - prm.p_begin;   // tile index inside the pass
     // first of the six window rows of this thread inside a stage; the 16-byte segment starts at column 8 j + 8
     const uint32_t win = (static_cast<uint32_t>(cl * prm.bh + 4 * r) * prm.bw + 8 * j + 8) * 2u;
     const uint32_t row_pitch = static_cast<uint32_t>(prm.bw) * 2u;
@@ -151,16 +162,17 @@ input_transform_f4_tma_kernel(const __grid_constant__ CUtensorMap tmX, __half* _
         }
     }
 
-    // tiles P .. Pstride - 1 of every row of V (the padding of the last block of 128) are zero, as the
+    // the tiles between the last one of the pass and the end of its last block of 128 are zero, as the
     // register-only kernels leave them
-    if (blockIdx.x == 0) {
-        const int tail2 = static_cast<int>((prm.Pstride - prm.P) / 2);   // P and Pstride are even
+    if (static_cast<int>(blockIdx.x) == prm.tail_block) {
+        const int tail2 = static_cast<int>((prm.tail_end - prm.tail_begin) / 2);   // both are even
         const int chans = steps * prm.cpb < prm.C - c_first ? steps * prm.cpb : prm.C - c_first;
         for (int i = tid; i < chans * tail2 * A * A; i += IN_TMA_THREADS) {
             const int t2 = i % tail2;
             const int rest2 = i / tail2;
             const int pos = rest2 % (A * A), c = c_first + rest2 / (A * A);
-            *reinterpret_cast<uint32_t*>(V + pos * plane + static_cast<long long>(c) * prm.Pstride + prm.P + 2 * t2) = 0u;
+            *reinterpret_cast<uint32_t*>(V + pos * plane + static_cast<long long>(c) * prm.Pstride + prm.tail_begin +
+                                         2 * t2) = 0u;
         }
     }
     if (abort_flag != 0) {

@@ -331,10 +331,15 @@ int launch_input(const __half* x, __half* V, const TileGeom& geo, int C, long lo
 
 
 // The TMA-staged F(4x4) activation transform covers a layer done in one pass whose rows TMA can address.
-bool use_input_tma(const TileGeom& geo, int N, int C, const void* x, long long p_begin, long long p_count,
-                   long long P128) {
-    const bool possible = p_begin == 0 && p_count == P128 && geo.W % 8 == 0 && aligned(x, 16) &&
-                          static_cast<long long>(N) * C < (1ll << 31) && geo.TH < (1 << 20);
+bool input_tma_possible(const TileGeom& geo, int N, int C, const void* x) {
+    return geo.W % 8 == 0 && aligned(x, 16) && static_cast<long long>(N) * C < (1ll << 31) && geo.TH < (1 << 20) &&
+           static_cast<long long>(N) * geo.TH < (1ll << 31);
+}
+
+bool use_input_tma(const TileGeom& geo, int N, int C, const void* x, long long p_begin, long long p_count) {
+    // a pass of whole tile rows (the last one may end with the layer)
+    const bool possible = input_tma_possible(geo, N, C, x) && p_begin % geo.TW == 0 &&
+                          (p_count % geo.TW == 0 || p_begin + p_count >= geo.P);
     if (!possible || g_input_staging == 0) return false;
     // Faster where a block row is a whole number of 32-byte sectors of V (W % 64 == 0: 15.8 against 17.0 us on
     // 960->320 at 64x64, 45.6 against 60.5 us on 512->512 at 256x256).  Image widths of 32 (8 tiles per row,
@@ -344,13 +349,20 @@ bool use_input_tma(const TileGeom& geo, int N, int C, const void* x, long long p
     return g_input_staging == 2 || geo.TW % 16 == 0;
 }
 
-int launch_input_tma(const __half* x, __half* V, const TileGeom& geo, int N, int C, long long Pstride, cudaStream_t st) {
+int launch_input_tma(const __half* x, __half* V, const TileGeom& geo, int N, int C, long long p_begin, long long p_count,
+                     long long Pstride, cudaStream_t st) {
     ProfScope prof(KIND_INPUT, st);
     const int sms = sm_count();
     int* status = status_word_ptr();
     if (sms <= 0 || !status) return SDWINO_ERR_CUDA;
     InTmaParams q;
-    q.C = C; q.TH = geo.TH; q.TW = geo.TW; q.P = geo.P; q.Pstride = Pstride;
+    q.C = C; q.TH = geo.TH; q.TW = geo.TW; q.Pstride = Pstride;
+    q.p_begin = p_begin;
+    const long long p_end = std::min(p_begin + p_count, geo.P);   // one past the last tile of the pass
+    q.g_begin = p_begin / geo.TW;
+    q.g_end = p_end / geo.TW;                                      // P = N * TH * TW: whole rows
+    q.tail_begin = p_end - p_begin;
+    q.tail_end = p_count;                                          // a multiple of 128
     // A block of up to 256 tiles (128 threads).  Blocks span the full width of the image when it has at most 60
     // tiles per row, otherwise at least 32 tiles: the tiles of a block row (of the whole block, at full width) are
     // then consecutive in V, and a warp stores runs of at least 64 bytes (narrower blocks measured 2-3x slower:
@@ -383,12 +395,23 @@ int launch_input_tma(const __half* x, __half* V, const TileGeom& geo, int N, int
     q.sb_c = (geo.TW + tcb - 1) / tcb;
     q.sb_r = (geo.TH + q.trb - 1) / q.trb;
     q.stage_bytes = (q.bw * q.bh * q.cpb * 2 + 127) / 128 * 128;
+    {
+        const long long g_last = q.g_end - 1;
+        q.tail_block = static_cast<int>((g_last / geo.TH) * q.sb_c * q.sb_r + ((g_last % geo.TH) / q.trb) * q.sb_c);
+    }
     const long long blocks = static_cast<long long>(N) * q.sb_c * q.sb_r;
     const long long csteps = (C + q.cpb - 1) / q.cpb;
-    // enough CTAs for four per SM, at most 16 steps each
-    long long steps = blocks * csteps / (4ll * sms);
-    steps = steps < 1 ? 1 : (steps > 16 ? 16 : steps);
-    steps = steps > csteps ? csteps : steps;
+    // Steps per CTA (at most 16): five CTAs are resident per SM and an SM needs about four of them to keep its
+    // issue slots busy; the time follows the SM with the most CTA-steps (one more step per CTA for the fill).
+    long long steps = 1;
+    double best_cost = 1e300;
+    for (long long cand = 1; cand <= 16 && cand <= csteps; ++cand) {
+        const long long ctas = blocks * ((csteps + cand - 1) / cand);
+        const long long per_sm = (ctas + sms - 1) / sms;
+        const double cost = per_sm <= 5 ? per_sm * (cand + 1.0) * std::max(1.0, 4.0 / per_sm)
+                                        : static_cast<double>((ctas + 5ll * sms - 1) / (5ll * sms)) * 5.0 * (cand + 1.0);
+        if (cost <= best_cost) { best_cost = cost; steps = cand; }
+    }
     q.steps = static_cast<int>(steps);
     const long long grid_y = (csteps + steps - 1) / steps;
     if (blocks >= (1ll << 31) || grid_y > 65535) return SDWINO_ERR_UNSUPPORTED;
@@ -604,8 +627,16 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
         return SDWINO_ERR_MISALIGNED;
     if (!ws || ws_bytes == 0) return SDWINO_ERR_WORKSPACE;
     if (!aligned(ws, WS_ALIGN)) return SDWINO_ERR_MISALIGNED;
-    const long long pc = tiles_per_pass(pl, ws_bytes);
+    long long pc = tiles_per_pass(pl, ws_bytes);
     if (pc < GEMM_BLOCK_P) return SDWINO_ERR_WORKSPACE;
+    if (tile == 4 && pc < pl.P128) {
+        // several passes: cut them at whole tile rows where that keeps the TMA-staged activation transform usable
+        const TileGeom g0 = make_geom(H, W, pl.TH, pl.TW, pl.P);
+        long long a = pl.TW, b = GEMM_BLOCK_P;
+        while (b != 0) { const long long t = a % b; a = b; b = t; }
+        const long long lcm = static_cast<long long>(pl.TW) / a * GEMM_BLOCK_P;
+        if (pc >= lcm && use_input_tma(g0, N, C, x, 0, lcm)) pc = pc / lcm * lcm;
+    }
     if (use_fused_small_k(K, W, tile, pl.P128 / 128, x, y) && !use_fused_small_c(C, tile) && !g_disable_fused)
         return launch_fused_small_k(static_cast<const __half*>(x), wT, static_cast<const __half*>(bias),
                                     static_cast<__half*>(y), pl, C, H, W, K, st);
@@ -668,7 +699,7 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
         const int count = static_cast<int>(remaining < pc ? remaining : pc);  // multiple of 128
         int rc;
         if (tile == 2) rc = launch_input<2>(xh, V, geo, C, p0, count, pc, st);
-        else if (use_input_tma(geo, N, C, x, p0, count, pl.P128)) rc = launch_input_tma(xh, V, geo, N, C, pc, st);
+        else if (use_input_tma(geo, N, C, x, p0, count)) rc = launch_input_tma(xh, V, geo, N, C, p0, count, pc, st);
         else rc = launch_input<4>(xh, V, geo, C, p0, count, pc, st);
         if (rc != SDWINO_OK) return rc;
         prm.num_p_tiles = (count / GEMM_BLOCK_P + shape.ctas - 1) / shape.ctas;

@@ -543,3 +543,25 @@ def test_staged_activation_transform_matches_register_kernel_bitwise(B, shape):
     assert torch.equal(y_staged, y_regs)
     ref = oracle.direct_conv3x3(x.numpy(), w.numpy(), b.numpy())
     assert _rel_err(y_staged, ref) <= TOL
+
+
+@pytest.mark.parametrize("shape,passes", [((24, 32, 100, 64, 3), 2), ((16, 16, 96, 96, 2), 3), ((8, 16, 64, 256, 1), 4),
+                                          ((20, 16, 40, 128, 2), 5)])
+def test_staged_activation_transform_over_several_passes(B, shape, passes):
+    # F(4x4) with a workspace for a fraction of the tiles: the passes are cut at whole tile rows, each runs the
+    # TMA-staged transform on its rows (blocks that straddle a cut are visited by both passes), the last one
+    # zero-fills the padding of its last block of 128 tiles.  Same bits as one pass and as the register kernel.
+    C, K, H, W, N = shape
+    layer = ConvLayer(C=C, K=K, H=H, W=W, N=N)
+    x, w, b = workloads.make_inputs(layer, seed=13)
+    full = B.sdwino_workspace_bytes(N, C, H, W, K, 4)
+    B.sdwino_set_input_staging(2)
+    try:
+        _, _, _, y_one = _run(B, layer, 4, x=x, w=w, b=b)
+        _, _, _, y_cut = _run(B, layer, 4, x=x, w=w, b=b, ws_bytes=full // passes + 4096)
+        B.sdwino_set_input_staging(0)
+        _, _, _, y_regs = _run(B, layer, 4, x=x, w=w, b=b, ws_bytes=full // passes + 4096)
+    finally:
+        B.sdwino_set_input_staging(1)
+    assert torch.equal(y_one, y_cut) and torch.equal(y_one, y_regs)
+    assert _rel_err(y_one, oracle.direct_conv3x3(x.numpy(), w.numpy(), b.numpy())) <= TOL
