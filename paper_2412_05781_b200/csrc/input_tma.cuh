@@ -2,8 +2,8 @@
 // tiles staged in shared memory by TMA.
 //
 // A CTA owns a block of TRb x TCb tiles of CPB channel images (TRb * TCb * CPB <= 256 tiles, two per thread) and
-// walks `steps` consecutive groups of CPB channels.  Per step one thread issues one 3-D TMA load of the pixel
-// window of the block, rows 4 th0 - 1 .. 4 (th0 + TRb) and columns 4 tw0 - 8 .. 4 (tw0 + TCb) + 7 (the column
+// walks `steps` consecutive groups of CPB channels.  Per step one thread issues one 3-D TMA load (two, side by
+// side, where the image is wide enough for block rows of 64 tiles) of the pixel window of the block, rows 4 th0 - 1 .. 4 (th0 + TRb) and columns 4 tw0 - 8 .. 4 (tw0 + TCb) + 7 (the column
 // origin is rounded down to a 16-byte boundary, as TMA requires; the rows and columns outside the image are the
 // zero padding of the convolution and come back as zeros from the TMA unit, so the kernel has no border code at
 // all).  Loads run up to IN_TMA_STAGES steps ahead of the arithmetic, which is what the register-only kernel
@@ -28,13 +28,15 @@ constexpr uint64_t IN_TMA_WAIT_LIMIT_NS = 2000000000ull;
 
 struct InTmaParams {
     int C, TH, TW;
-    int tcb_half;        // threads per tile row of a block = TCb / 2
+    int tcb_half;        // threads per tile row of a box = TCb / 2
+    int nb;              // boxes side by side per block (1 or 2): a block row is nb * TCb tiles
+    int box_bytes;       // bw * bh * cpb * 2, rounded up to 128
     int trb;             // tile rows per block
     int cpb;             // channel images per step
     int bw, bh;          // box of the TMA load in pixels: 4 TCb + 16 columns, 4 TRb + 2 rows
     int sb_c, sb_r;      // blocks per image along the columns / rows
     int steps;           // steps (groups of cpb channels) per CTA
-    int stage_bytes;     // bw * bh * cpb * 2, rounded up to 128
+    int stage_bytes;     // nb * box_bytes
     long long Pstride;   // tiles per row of V (a multiple of 128)
     long long p_begin;   // first tile of this pass (a multiple of TW)
     long long g_begin, g_end;   // this pass covers the tile rows g = n * TH + th in [g_begin, g_end)
@@ -59,7 +61,7 @@ input_transform_f4_tma_kernel(const __grid_constant__ CUtensorMap tmX, __half* _
     const int br = (blockIdx.x - n * sb) / prm.sb_c;
     const int bc = blockIdx.x - n * sb - br * prm.sb_c;
     const int tcb = prm.tcb_half * 2;
-    const int th0 = br * prm.trb, tw0 = bc * tcb;
+    const int th0 = br * prm.trb, tw0 = bc * tcb * prm.nb;
     // a block none of whose tile rows belong to this pass has nothing to do (a layer done in several passes)
     {
         const long long g_lo = static_cast<long long>(n) * prm.TH + th0;
@@ -81,28 +83,33 @@ input_transform_f4_tma_kernel(const __grid_constant__ CUtensorMap tmX, __half* _
     pdl_launch_dependents();
 
     const int x0 = 4 * tw0 - 8, y0 = 4 * th0 - 1;
-    const uint32_t tx_bytes = static_cast<uint32_t>(prm.bw) * prm.bh * prm.cpb * 2u;
+    const uint32_t tx_bytes = static_cast<uint32_t>(prm.bw) * prm.bh * prm.cpb * 2u * prm.nb;
     if (tid == 0) {
         const int pre = steps < IN_TMA_STAGES ? steps : IN_TMA_STAGES;
         for (int s = 0; s < pre; ++s) {
             mbar_arrive_expect_tx(&full_bar[s], tx_bytes);
-            tma_load_3d(smem + s * prm.stage_bytes, &tmX, &full_bar[s], x0, y0, n * prm.C + c_first + s * prm.cpb);
+            for (int sub = 0; sub < prm.nb; ++sub)
+                tma_load_3d(smem + s * prm.stage_bytes + sub * prm.box_bytes, &tmX, &full_bar[s], x0 + sub * 4 * tcb, y0,
+                            n * prm.C + c_first + s * prm.cpb);
         }
     }
 
     // thread -> (channel within the step, tile row within the block, pair of tiles within the row)
-    const int rest = tid / prm.tcb_half;
-    const int j = tid - rest * prm.tcb_half;
+    const int row_threads = prm.tcb_half * prm.nb;
+    const int rest = tid / row_threads;
+    const int jf = tid - rest * row_threads;          // pair of tiles within the block row
+    const int sub = jf >= prm.tcb_half ? 1 : 0;       // which box
+    const int j = jf - sub * prm.tcb_half;
     const int r = rest % prm.trb;
     const int cl = rest / prm.trb;
-    const int th = th0 + r, tw = tw0 + 2 * j;
+    const int th = th0 + r, tw = tw0 + 2 * jf;
     const long long g = static_cast<long long>(n) * prm.TH + th;   // tile row over all images
     // W % 8 == 0: TW is even, so tile tw + 1 exists whenever tile tw does
     const bool tile_ok = cl < prm.cpb && th < prm.TH && tw < prm.TW && g >= prm.g_begin && g < prm.g_end;
     const long long plane = static_cast<long long>(prm.C) * prm.Pstride;
     const long long p = g * prm.TW + tw - prm.p_begin;   // tile index inside the pass
     // first of the six window rows of this thread inside a stage; the 16-byte segment starts at column 8 j + 8
-    const uint32_t win = (static_cast<uint32_t>(cl * prm.bh + 4 * r) * prm.bw + 8 * j + 8) * 2u;
+    const uint32_t win = sub * prm.box_bytes + (static_cast<uint32_t>(cl * prm.bh + 4 * r) * prm.bw + 8 * j + 8) * 2u;
     const uint32_t row_pitch = static_cast<uint32_t>(prm.bw) * 2u;
 
     for (int it = 0; it < steps; ++it) {
@@ -144,8 +151,9 @@ input_transform_f4_tma_kernel(const __grid_constant__ CUtensorMap tmX, __half* _
         }
         if (tid == 0 && it + IN_TMA_STAGES < steps) {
             mbar_arrive_expect_tx(&full_bar[s], tx_bytes);
-            tma_load_3d(smem + s * prm.stage_bytes, &tmX, &full_bar[s], x0, y0,
-                        n * prm.C + c_first + (it + IN_TMA_STAGES) * prm.cpb);
+            for (int sub = 0; sub < prm.nb; ++sub)
+                tma_load_3d(smem + s * prm.stage_bytes + sub * prm.box_bytes, &tmX, &full_bar[s], x0 + sub * 4 * tcb, y0,
+                            n * prm.C + c_first + (it + IN_TMA_STAGES) * prm.cpb);
         }
         const int c = c_first + it * prm.cpb + cl;
         if (!tile_ok || c >= prm.C) continue;
