@@ -132,8 +132,11 @@ int sdwino_conv3x3_static(const void *x, const void *wT, const void *bias, void 
  * earlier call is complete once sdwino_host_join(stream) has been called (it makes `stream` wait for the
  * outstanding downloads) and `stream` has then been synchronised; x_host and bias_host must not change until
  * then.  While such calls are in flight the staging part of the workspace belongs to them: do not hand the
- * same workspace to other entry points before the join.  The first call on a device creates the two streams
- * and eight events (make it outside any stream capture); not thread-safe.
+ * same workspace to other entry points before the join.  Calls with the same sizes may share a workspace and
+ * still overlap (they alternate between the two slots); a call whose sizes differ from those of an in-flight
+ * call on overlapping memory is ordered after that call's kernels and download, so give every layer of a
+ * network its own workspace if their copies are to overlap.  The first call on a device creates the two streams
+ * and 96 events (make it outside any stream capture); not thread-safe.
  */
 size_t sdwino_host_staging_bytes(int N, int C, int H, int W, int K, int tile);
 int sdwino_conv3x3_host(const void *x_host, const void *wT, const void *bias_host, void *y_host,

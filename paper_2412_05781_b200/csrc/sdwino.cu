@@ -838,16 +838,25 @@ size_t sdwino_host_staging_bytes(int N, int C, int H, int W, int K, int tile) {
 }
 
 namespace {
-// Per-device state of the asynchronous host path: one copy stream per direction and four events per staging
-// slot.  Created on first use; one device per process is the common case.
+// Per-device state of the asynchronous host path: one copy stream per direction and a ring of the most recent
+// calls (what memory each used, with which sizes and staging slot, and its three events).  A new call is ordered
+// only after earlier calls that touch the same memory, so the copies of layers with workspaces of their own run
+// ahead of the kernels as far as the copy streams allow.  Created on first use.
+constexpr int HOST_RING = 32;
+struct HostCall {
+    bool used = false;
+    const uint8_t* begin = nullptr;   // workspace of the call
+    const uint8_t* end = nullptr;
+    size_t sizes[3] = {0, 0, 0};      // bytes of x, bias, y
+    int slot = 0;                     // half of the staging area
+    cudaEvent_t uploaded = nullptr;   // on s_in: x (and bias) are on the device
+    cudaEvent_t computed = nullptr;   // on the caller's stream: the kernels have read x and written y
+    cudaEvent_t downloaded = nullptr; // on s_out: y has reached host memory
+};
 struct HostPipe {
     bool ready = false;
     cudaStream_t s_in = nullptr, s_out = nullptr;
-    cudaEvent_t uploaded[2] = {nullptr, nullptr};    // on s_in: x (and bias) of slot i are on the device
-    cudaEvent_t consumed[2] = {nullptr, nullptr};    // on the caller's stream: the kernels have read slot i
-    cudaEvent_t computed[2] = {nullptr, nullptr};    // on the caller's stream: y of slot i is complete on the device
-    cudaEvent_t downloaded[2] = {nullptr, nullptr};  // on s_out: y of slot i has reached host memory
-    bool slot_used[2] = {false, false};
+    HostCall ring[HOST_RING];
     unsigned long long calls = 0;
 };
 HostPipe g_host_pipe[STATIC_MAX_DEVICES_HOST];
@@ -859,11 +868,10 @@ HostPipe* host_pipe() {
     if (!hp.ready) {
         if (cudaStreamCreateWithFlags(&hp.s_in, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
         if (cudaStreamCreateWithFlags(&hp.s_out, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
-        for (int i = 0; i < 2; ++i) {
-            if (cudaEventCreateWithFlags(&hp.uploaded[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
-            if (cudaEventCreateWithFlags(&hp.consumed[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
-            if (cudaEventCreateWithFlags(&hp.computed[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
-            if (cudaEventCreateWithFlags(&hp.downloaded[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        for (int i = 0; i < HOST_RING; ++i) {
+            if (cudaEventCreateWithFlags(&hp.ring[i].uploaded, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+            if (cudaEventCreateWithFlags(&hp.ring[i].computed, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+            if (cudaEventCreateWithFlags(&hp.ring[i].downloaded, cudaEventDisableTiming) != cudaSuccess) return nullptr;
         }
         hp.ready = true;
     }
@@ -885,41 +893,85 @@ int sdwino_conv3x3_host_async(const void* x_host, const void* wT, const void* bi
     const size_t xbytes = static_cast<size_t>(N) * C * H * W * sizeof(__half);
     const size_t ybytes = static_cast<size_t>(N) * K * H * W * sizeof(__half);
     const size_t bbytes = static_cast<size_t>(K) * sizeof(__half);
-    const int slot = static_cast<int>(hp->calls++ & 1ull);
     uint8_t* base = static_cast<uint8_t*>(workspace);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+    // Earlier calls, newest first.  One with the same workspace and sizes owns one half (slot) of the staging area:
+    // this call takes the other half and waits only for the newest call that had its own half (its kernels before
+    // the upload, its download before the kernels).  One that overlaps this workspace with other sizes laid its
+    // copies and its scratch out differently: everything of it, download included, comes first.
+    int slot = -1;
+    bool waited_same_slot = false;
+    const unsigned long long first = hp->calls > HOST_RING ? hp->calls - HOST_RING : 0;
+    for (unsigned long long c = hp->calls; c-- > first;) {
+        const HostCall& e = hp->ring[c % HOST_RING];
+        if (!e.used || !(base < e.end && e.begin < base + workspace_bytes)) continue;
+        const bool same = e.begin == base && e.end == base + workspace_bytes && e.sizes[0] == xbytes &&
+                          e.sizes[1] == bbytes && e.sizes[2] == ybytes;
+        if (same) {
+            if (slot < 0) slot = 1 - e.slot;          // the newest one decides
+            if (e.slot == slot && !waited_same_slot) {
+                // (a wait for an event that has completed would still cost the copy stream a semaphore)
+                if (cudaEventQuery(e.downloaded) != cudaSuccess &&
+                    (cudaStreamWaitEvent(hp->s_in, e.computed, 0) != cudaSuccess ||
+                     cudaStreamWaitEvent(st, e.downloaded, 0) != cudaSuccess))
+                    return SDWINO_ERR_CUDA;
+                waited_same_slot = true;
+            }
+        } else {
+            if (cudaStreamWaitEvent(hp->s_in, e.computed, 0) != cudaSuccess ||
+                cudaStreamWaitEvent(hp->s_in, e.downloaded, 0) != cudaSuccess ||
+                cudaStreamWaitEvent(st, e.downloaded, 0) != cudaSuccess)
+                return SDWINO_ERR_CUDA;
+        }
+    }
+    if (slot < 0) slot = 0;
+    // the ring entry this call takes over belongs to a call of HOST_RING calls ago: it is forgotten only once it
+    // has completed
+    HostCall& me = hp->ring[hp->calls % HOST_RING];
+    if (me.used && cudaEventQuery(me.downloaded) != cudaSuccess &&   // its download is its last operation
+        (cudaStreamWaitEvent(hp->s_in, me.downloaded, 0) != cudaSuccess ||
+         cudaStreamWaitEvent(st, me.downloaded, 0) != cudaSuccess))
+        return SDWINO_ERR_CUDA;
+    me.used = false;
+
     uint8_t* xd = base + slot * up(xbytes);
     uint8_t* bd = base + 2 * up(xbytes) + slot * up(bbytes);
     uint8_t* yd = base + 2 * (up(xbytes) + up(bbytes)) + slot * up(ybytes);
     uint8_t* ws = base + staging;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    // upload on the copy stream, as soon as the kernels of the call before last have finished reading this slot
-    if (hp->slot_used[slot] && cudaStreamWaitEvent(hp->s_in, hp->consumed[slot], 0) != cudaSuccess) return SDWINO_ERR_CUDA;
+    // upload on the first copy stream
     if (cudaMemcpyAsync(xd, x_host, xbytes, cudaMemcpyHostToDevice, hp->s_in) != cudaSuccess) return SDWINO_ERR_CUDA;
     if (bias_host && cudaMemcpyAsync(bd, bias_host, bbytes, cudaMemcpyHostToDevice, hp->s_in) != cudaSuccess)
         return SDWINO_ERR_CUDA;
-    if (cudaEventRecord(hp->uploaded[slot], hp->s_in) != cudaSuccess) return SDWINO_ERR_CUDA;
-    // kernels on the caller's stream, once the upload is there and the download of the call before last has
-    // left this slot's output buffer
-    if (cudaStreamWaitEvent(st, hp->uploaded[slot], 0) != cudaSuccess) return SDWINO_ERR_CUDA;
-    if (hp->slot_used[slot] && cudaStreamWaitEvent(st, hp->downloaded[slot], 0) != cudaSuccess) return SDWINO_ERR_CUDA;
+    if (cudaEventRecord(me.uploaded, hp->s_in) != cudaSuccess) return SDWINO_ERR_CUDA;
+    // kernels on the caller's stream
+    if (cudaStreamWaitEvent(st, me.uploaded, 0) != cudaSuccess) return SDWINO_ERR_CUDA;
     const int rc = conv_impl(xd, wT, bias_host ? bd : nullptr, yd, N, C, H, W, K, tile, ws, workspace_bytes - staging, st);
     if (rc != SDWINO_OK) return rc;
-    if (cudaEventRecord(hp->consumed[slot], st) != cudaSuccess) return SDWINO_ERR_CUDA;
-    if (cudaEventRecord(hp->computed[slot], st) != cudaSuccess) return SDWINO_ERR_CUDA;
+    if (cudaEventRecord(me.computed, st) != cudaSuccess) return SDWINO_ERR_CUDA;
     // download on the second copy stream
-    if (cudaStreamWaitEvent(hp->s_out, hp->computed[slot], 0) != cudaSuccess) return SDWINO_ERR_CUDA;
+    if (cudaStreamWaitEvent(hp->s_out, me.computed, 0) != cudaSuccess) return SDWINO_ERR_CUDA;
     if (cudaMemcpyAsync(y_host, yd, ybytes, cudaMemcpyDeviceToHost, hp->s_out) != cudaSuccess) return SDWINO_ERR_CUDA;
-    if (cudaEventRecord(hp->downloaded[slot], hp->s_out) != cudaSuccess) return SDWINO_ERR_CUDA;
-    hp->slot_used[slot] = true;
+    if (cudaEventRecord(me.downloaded, hp->s_out) != cudaSuccess) return SDWINO_ERR_CUDA;
+    me.used = true;
+    me.begin = base;
+    me.end = base + workspace_bytes;
+    me.sizes[0] = xbytes;
+    me.sizes[1] = bbytes;
+    me.sizes[2] = ybytes;
+    me.slot = slot;
+    ++hp->calls;
     return SDWINO_OK;
 }
 
 int sdwino_host_join(void* stream) {
     HostPipe* hp = host_pipe();
     if (!hp) return SDWINO_ERR_CUDA;
-    for (int i = 0; i < 2; ++i)
-        if (hp->slot_used[i] && cudaStreamWaitEvent(static_cast<cudaStream_t>(stream), hp->downloaded[i], 0) != cudaSuccess)
-            return SDWINO_ERR_CUDA;
+    if (hp->calls == 0) return SDWINO_OK;
+    // the download stream works in order: the newest download is the last one to finish
+    const HostCall& last = hp->ring[(hp->calls - 1) % HOST_RING];
+    if (last.used && cudaStreamWaitEvent(static_cast<cudaStream_t>(stream), last.downloaded, 0) != cudaSuccess)
+        return SDWINO_ERR_CUDA;
     return SDWINO_OK;
 }
 

@@ -565,3 +565,43 @@ def test_staged_activation_transform_over_several_passes(B, shape, passes):
         B.sdwino_set_input_staging(1)
     assert torch.equal(y_one, y_cut) and torch.equal(y_one, y_regs)
     assert _rel_err(y_one, oracle.direct_conv3x3(x.numpy(), w.numpy(), b.numpy())) <= TOL
+
+
+@pytest.mark.parametrize("shared", [True, False])
+def test_async_host_entry_with_layers_of_different_sizes(B, shared):
+    # Layers of very different sizes enqueued back to back through the asynchronous host entry.  With one shared
+    # workspace their staging layouts overlap, so the library must order each call after the copies and kernels of
+    # the calls still in flight (a 60 MB upload would otherwise land in memory that the previous layer's kernels
+    # are still reading); with a workspace per layer the copies are free to overlap.  Either way every result
+    # equals the device entry.
+    shapes = [(64, 32, 96, 96, 2), (1200, 16, 64, 64, 4), (16, 256, 32, 32, 1), (320, 320, 64, 64, 2), (8, 16, 256, 256, 2),
+              (256, 64, 16, 16, 1), (64, 32, 96, 96, 2)]
+    stream = torch.cuda.Stream()
+    jobs = []
+    for i, (C, K, H, W, N) in enumerate(shapes):
+        layer = ConvLayer(C=C, K=K, H=H, W=W, N=N)
+        x, w, b = workloads.make_inputs(layer, seed=70 + i, pin=True)
+        tile = B.sdwino_choose_tile(N, C, H, W, K)
+        wT = B.sdwino_filter_transform(w.cuda(), tile)
+        y = torch.empty(N, K, H, W, dtype=torch.float16).pin_memory()
+        nbytes = B.sdwino_host_staging_bytes(N, C, H, W, K, tile) + B.sdwino_workspace_bytes(N, C, H, W, K, tile)
+        jobs.append([layer, tile, x, b, wT, y, nbytes])
+    if shared:
+        ws_all = B.alloc_workspace(max(j[6] for j in jobs))
+        spaces = [ws_all] * len(jobs)
+    else:
+        spaces = [B.alloc_workspace(j[6]) for j in jobs]
+    expect = []
+    for (layer, tile, x, b, wT, y, _) in jobs:
+        ws2 = B.alloc_workspace(B.sdwino_workspace_bytes(layer.N, layer.C, layer.H, layer.W, layer.K, tile))
+        expect.append(B.sdwino_conv3x3(x.cuda(), wT, b.cuda(), layer.K, tile, workspace=ws2).cpu())
+    torch.cuda.synchronize()
+    for rep in range(3):
+        for (layer, tile, x, b, wT, y, _), wsl in zip(jobs, spaces):
+            y.zero_()
+            B.sdwino_conv3x3_host(x, wT, b, y, tile, wsl, stream=stream, wait=False)
+        B.sdwino_host_join(stream)
+        stream.synchronize()
+        assert B.sdwino_last_device_status(stream) == B.OK
+        for (layer, tile, x, b, wT, y, _), want in zip(jobs, expect):
+            assert torch.equal(y, want), (layer.name, tile, rep, shared)
