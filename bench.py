@@ -349,6 +349,9 @@ def run_ours(args):
     e2e_value = aggregate_value(flops_step, world, max_over_ranks(e2e_s, dist, dev) / e2e_steps * 1e3)
     h2d = sum(x.numel() * 2 + b.numel() * 2 for (x, w, b, y) in host)
     d2h = sum(y.numel() * 2 for (x, w, b, y) in host)
+    # what came back through the host path is what the device-resident step computed (same kernels: same bits)
+    e2e_matches = all(torch.equal(y_h, yd.cpu()) for (_, _, _, y_h), (_, _, _, yd) in zip(host, devt))
+    assert e2e_matches, "the host path returned something else than the device path"
 
     # ---- per-kernel and per-layer times: a second timed pass with CUDA events around every launch (recorded
     #      by the library on the launch stream).  The sweeps run back to back without host syncs, so the device
@@ -531,7 +534,7 @@ def run_ours(args):
                                "cold")),
                        "filter_transform": "once per weight, before the timed region (reported separately)"},
             "e2e": {"value": round(e2e_value, 2), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "steps": e2e_steps, "api": "sdwino_conv3x3_host_async per layer (pinned host x, bias, y; " +
+                    "steps": e2e_steps, "matches_device_path": bool(e2e_matches), "api": "sdwino_conv3x3_host_async per layer (pinned host x, bias, y; " +
                            ("a workspace per layer: uploads and downloads overlap the neighbouring layers" if per_layer_ws
                             else "one shared workspace: the copies of differently sized layers are ordered one after the other") +
                            "), one join + stream synchronisation per step"},
