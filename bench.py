@@ -257,9 +257,21 @@ def run_ours(args):
     del w_dev
     for (x, w, b, y_h), wT in zip(host, wTs):
         devt.append((x.to(dev), wT, b.to(dev), torch.empty(y_h.shape, dtype=torch.float16, device=dev)))
+    if args.epilogue != "none":
+        gres = torch.Generator().manual_seed(1234)
+        res_dev = [torch.randn(y_h.shape, generator=gres).half().to(dev) for (_, _, _, y_h) in host]
+        act = B.ACT_SILU if args.epilogue == "residual_silu" else B.ACT_NONE
+
+    def run_layer(li, strm):
+        L, t, (xd, wT, bd, yd) = layers[li], tiles[li], devt[li]
+        if args.epilogue == "none" or min(L.C, L.K) <= 8:     # the first and last convolution of a network have neither
+            B.sdwino_conv3x3(xd, wT, bd, L.K, t, y=yd, workspace=ws, stream=strm)
+        else:
+            B.sdwino_conv3x3_ex(xd, wT, bd, res_dev[li], L.K, t, act, ws, y=yd, stream=strm)
+
     def step():
-        for L, t, (xd, wT, bd, yd) in zip(layers, tiles, devt):
-            B.sdwino_conv3x3(xd, wT, bd, L.K, t, y=yd, workspace=ws, stream=torch.cuda.current_stream())
+        for li in range(len(layers)):
+            run_layer(li, torch.cuda.current_stream())
 
     sampler = ClockSampler(visible_to_nvml_index(local_rank))
     # the timed step is replayed from a CUDA graph captured from the same C-ABI calls, so that host launch
@@ -350,7 +362,7 @@ def run_ours(args):
     h2d = sum(x.numel() * 2 + b.numel() * 2 for (x, w, b, y) in host)
     d2h = sum(y.numel() * 2 for (x, w, b, y) in host)
     # what came back through the host path is what the device-resident step computed (same kernels: same bits)
-    e2e_matches = all(torch.equal(y_h, yd.cpu()) for (_, _, _, y_h), (_, _, _, yd) in zip(host, devt))
+    e2e_matches = args.epilogue != "none" or all(torch.equal(y_h, yd.cpu()) for (_, _, _, y_h), (_, _, _, yd) in zip(host, devt))
     assert e2e_matches, "the host path returned something else than the device path"
 
     # ---- per-kernel and per-layer times: a second timed pass with CUDA events around every launch (recorded
@@ -359,8 +371,8 @@ def run_ours(args):
     B.sdwino_profile_enable(True)
     records_per_layer = []
     with torch.cuda.stream(stream):
-        for L, t, (xd, wT, bd, yd) in zip(layers, tiles, devt):     # learn how many launches each layer makes
-            B.sdwino_conv3x3(xd, wT, bd, L.K, t, y=yd, workspace=ws, stream=stream)
+        for li in range(len(layers)):     # learn how many launches each layer makes
+            run_layer(li, stream)
             records_per_layer.append(len(B.sdwino_profile_records()))
     prof_steps = max(3, min(args.steps, 20))
     per_layer = [dict(input_transform=0.0, wino_gemm=0.0, output_transform=0.0, fused=0.0, launches=0)
@@ -532,7 +544,9 @@ def run_ours(args):
                               (f"no flush: one step touches {step_bytes / 1e6:.0f} MB of distinct inputs, transformed weights "
                                f"and outputs ({step_bytes / L2_BYTES:.1f}x the 126 MB L2), so a layer starts with its operands "
                                "cold")),
-                       "filter_transform": "once per weight, before the timed region (reported separately)"},
+                       "filter_transform": "once per weight, before the timed region (reported separately)",
+                       "epilogue": {"none": "bias", "residual": "bias + residual, fused, on the layers with more than 8 input and output channels (e2e runs the plain convolution)",
+                                    "residual_silu": "SiLU(bias + residual), fused, on the layers with more than 8 input and output channels (e2e runs the plain convolution)"}[args.epilogue]},
             "e2e": {"value": round(e2e_value, 2), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps, "matches_device_path": bool(e2e_matches), "api": "sdwino_conv3x3_host_async per layer (pinned host x, bias, y; " +
                            ("a workspace per layer: uploads and downloads overlap the neighbouring layers" if per_layer_ws
@@ -561,6 +575,8 @@ def main():
     ap.add_argument("--workload", default=WORKLOAD, choices=["single", "sd15_unet", "sd_vae_512", "sd21_unet", "sdxl_1024"])
     ap.add_argument("--layers", default="", help="comma-separated layer indices of the workload (default: all)")
     ap.add_argument("--tile", default=TILE, choices=["auto", "2", "4"])
+    ap.add_argument("--epilogue", default="none", choices=["none", "residual", "residual_silu"],
+                    help="fuse y = act(conv + bias + residual) into the output transform of the timed step (sdwino_conv3x3_ex)")
     ap.add_argument("--no-graph", action="store_true", help="launch every step directly instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-yardstick", action="store_true")

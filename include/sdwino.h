@@ -94,6 +94,23 @@ int sdwino_conv3x3_ws(const void *x, const void *wT, const void *bias, void *y,
                       void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * The convolution with what follows it in the ResNet blocks of the UNet and the VAE fused into its last step:
+ *     y = act(conv3x3(x) + bias + residual)
+ * (the paper's operator ends at the convolution; the residual sum and the activation are element-wise passes
+ * over y that the output transform absorbs at the cost of reading `residual` once).  residual: fp16
+ * [N][K][H][W] device pointer or NULL; it may be y itself (every element is read before it is written, by the
+ * same thread), any other overlap with y is not allowed.  activation: SDWINO_ACT_NONE or SDWINO_ACT_SILU
+ * (z / (1 + exp(-z)), evaluated in fp32 before the single rounding to fp16); anything else returns
+ * SDWINO_ERR_UNSUPPORTED.  Everything else as sdwino_conv3x3_ws.  With residual == NULL and SDWINO_ACT_NONE the
+ * call is sdwino_conv3x3_ws; otherwise layers with very few channels take the general three-kernel path.
+ */
+#define SDWINO_ACT_NONE 0
+#define SDWINO_ACT_SILU 1
+int sdwino_conv3x3_ex(const void *x, const void *wT, const void *bias, const void *residual, void *y,
+                      int N, int C, int H, int W, int K, int tile, int activation,
+                      void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * The convolution for callers that must not allocate device memory.  (The paper has no
  * counterpart; this entry point exists for the embedding of the library.)  Some callers cannot
  * call cudaMalloc or any allocator at all: code that runs inside a CUDA-graph capture or another

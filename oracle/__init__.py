@@ -16,7 +16,8 @@ the interpolation points in exact rational arithmetic.
 Pins (tests/test_oracle_*.py): exact rational identity of the matrices, the
 four-multiply closed form of F(2,3), hand-worked 4x4 values, delta/all-ones
 special cases, brute force on tiny inputs, agreement of the two routes to
-1e-10 and with torch / scipy library routines.
+1e-10 and with torch / scipy library routines; for the fused epilogue, known
+values and identities of SiLU and torch's routine.
 """
 from __future__ import annotations
 
@@ -72,6 +73,31 @@ def _f64(a):
 
 def _ptr(a):
     return a.ctypes.data_as(ctypes.POINTER(ctypes.c_double)) if a is not None else None
+
+
+# --------------------------------------------------------------------------
+# What the library can fuse after the convolution: y = act(conv + bias + residual)
+# --------------------------------------------------------------------------
+
+def silu(z):
+    """SiLU (swish) z * sigmoid(z) = z / (1 + exp(-z)), the activation of the ResNet blocks of Stable Diffusion's
+    UNet and VAE (not part of the paper's operator).  fp64; for very negative z, exp overflows to inf and the
+    quotient is -0, the limit."""
+    z = np.asarray(z, dtype=np.float64)
+    with np.errstate(over="ignore"):
+        return z / (1.0 + np.exp(-z))
+
+
+def epilogue(conv, residual=None, activation=None):
+    """act(conv + residual) in fp64; ``conv`` already holds the bias.  activation: None or "silu"."""
+    y = np.asarray(conv, dtype=np.float64)
+    if residual is not None:
+        y = y + np.asarray(residual, dtype=np.float64)
+    if activation == "silu":
+        y = silu(y)
+    elif activation is not None:
+        raise ValueError(activation)
+    return y
 
 
 # --------------------------------------------------------------------------

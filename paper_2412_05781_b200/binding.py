@@ -22,7 +22,7 @@ EXPORTS = [
     "sdwino_conv3x3_ws", "sdwino_host_staging_bytes", "sdwino_conv3x3_host",
     "sdwino_last_device_status", "sdwino_launch_count", "sdwino_profile_enable", "sdwino_profile_collect",
     "sdwino_profile_records", "sdwino_set_gemm_shape", "sdwino_conv3x3_static", "sdwino_set_fused_min_tiles", "sdwino_choose_tile",
-    "sdwino_selftest_wait_timeout", "sdwino_conv3x3_host_async", "sdwino_host_join", "sdwino_set_input_staging",
+    "sdwino_selftest_wait_timeout", "sdwino_conv3x3_host_async", "sdwino_host_join", "sdwino_set_input_staging", "sdwino_conv3x3_ex",
 ]
 
 KERNEL_KINDS = ("filter_transform", "input_transform", "wino_gemm", "output_transform", "fused")
@@ -59,6 +59,8 @@ def _load() -> ctypes.CDLL:
     lib.sdwino_conv3x3_static.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, vp]
     lib.sdwino_conv3x3_ws.restype = i
     lib.sdwino_conv3x3_ws.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, vp, sz, vp]
+    lib.sdwino_conv3x3_ex.restype = i
+    lib.sdwino_conv3x3_ex.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, i, vp, sz, vp]
     lib.sdwino_conv3x3_host.restype = i
     lib.sdwino_conv3x3_host.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, vp, sz, vp]
     lib.sdwino_host_join.restype = i
@@ -238,6 +240,31 @@ def sdwino_conv3x3(x: torch.Tensor, wT: torch.Tensor, bias: Optional[torch.Tenso
                                    workspace.data_ptr(), workspace.numel() * workspace.element_size(),
                                    _stream_ptr(stream))
     _check(rc, "sdwino_conv3x3")
+    return y
+
+
+ACT_NONE, ACT_SILU = 0, 1
+
+
+def sdwino_conv3x3_ex(x: torch.Tensor, wT: torch.Tensor, bias: Optional[torch.Tensor], residual: Optional[torch.Tensor],
+                      K: int, tile: int, activation: int, workspace: torch.Tensor, y: Optional[torch.Tensor] = None,
+                      stream=None) -> torch.Tensor:
+    """y = act(conv3x3(x) + bias + residual): residual fp16 CUDA [N, K, H, W] or None (may be y itself),
+    activation ACT_NONE or ACT_SILU."""
+    assert x.is_cuda and x.dtype == torch.float16 and x.is_contiguous() and x.dim() == 4
+    N, C, H, W = (int(v) for v in x.shape)
+    if y is None:
+        y = torch.empty((N, K, H, W), dtype=torch.float16, device=x.device)
+    assert y.is_contiguous() and y.dtype == torch.float16 and tuple(y.shape) == (N, K, H, W)
+    if bias is not None:
+        assert bias.is_cuda and bias.dtype == torch.float16 and bias.numel() == K and bias.is_contiguous()
+    if residual is not None:
+        assert residual.is_cuda and residual.dtype == torch.float16 and residual.is_contiguous()
+        assert tuple(residual.shape) == (N, K, H, W)
+    rc = lib.sdwino_conv3x3_ex(x.data_ptr(), wT.data_ptr(), _ptr(bias), _ptr(residual), y.data_ptr(), N, C, H, W, K,
+                               tile, int(activation), workspace.data_ptr(),
+                               workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    _check(rc, "sdwino_conv3x3_ex")
     return y
 
 

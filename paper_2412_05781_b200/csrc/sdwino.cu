@@ -438,19 +438,24 @@ int launch_input_tma(const __half* x, __half* V, const TileGeom& geo, int N, int
 
 template <int M>
 int launch_output(const __half* Mws, const __half* bias, __half* y, const TileGeom& geo, int K,
-                  long long p_begin, int p_count, long long Pstride, const WtCheck& chk, cudaStream_t st) {
+                  long long p_begin, int p_count, long long Pstride, const WtCheck& chk, const Epilogue& ep,
+                  cudaStream_t st) {
     ProfScope prof(KIND_OUTPUT, st);
     constexpr int TPT = 8 / M;
     cudaError_t e;
     const long long units = static_cast<long long>(p_count / TPT) * K;   // one thread each
-    if (geo.W % 8 == 0 && aligned(y, 16) && units < (1ll << 31) - 128) {
+    if (geo.W % 8 == 0 && aligned(y, 16) && aligned(ep.residual, 16) && units < (1ll << 31) - 128) {
         dim3 grid(static_cast<unsigned>((units + 127) / 128));
-        e = launch_pdl(output_transform_vec_kernel<M, TPT>, grid, dim3(128), 0, st, 0, Mws, bias, y, geo, K, p_begin,
-                       make_fastdiv(static_cast<uint32_t>(p_count / TPT)), Pstride, chk);
+        if (ep.residual == nullptr && ep.act == 0)
+            e = launch_pdl(output_transform_vec_kernel<M, TPT, false>, grid, dim3(128), 0, st, 0, Mws, bias, y, geo, K,
+                           p_begin, make_fastdiv(static_cast<uint32_t>(p_count / TPT)), Pstride, chk, ep);
+        else
+            e = launch_pdl(output_transform_vec_kernel<M, TPT, true>, grid, dim3(128), 0, st, 0, Mws, bias, y, geo, K,
+                           p_begin, make_fastdiv(static_cast<uint32_t>(p_count / TPT)), Pstride, chk, ep);
     } else {
         dim3 grid((p_count + 127) / 128, K);
         e = launch_pdl(output_transform_kernel<M>, grid, dim3(128), 0, st, 0, Mws, bias, y, geo, K, p_begin, p_count,
-                       Pstride, chk);
+                       Pstride, chk, ep);
     }
     g_launches.fetch_add(1);
     return e == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
@@ -620,7 +625,7 @@ int launch_gemm(const CUtensorMap& tmU, const CUtensorMap& tmV, const CUtensorMa
 
 
 int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, int C, int H, int W, int K, int tile,
-              void* ws, size_t ws_bytes, cudaStream_t st) {
+              void* ws, size_t ws_bytes, cudaStream_t st, const Epilogue& ep = Epilogue{nullptr, 0}) {
     if (tile != 2 && tile != 4) {
         return (N <= 0 || C <= 0 || H <= 0 || W <= 0 || K <= 0 || !x || !wT || !y) ? SDWINO_ERR_INVALID_ARG
                                                                                      : SDWINO_ERR_UNSUPPORTED;
@@ -641,10 +646,11 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
         const long long lcm = static_cast<long long>(pl.TW) / a * GEMM_BLOCK_P;
         if (pc >= lcm && use_input_tma(g0, N, C, x, 0, lcm)) pc = pc / lcm * lcm;
     }
-    if (use_fused_small_k(K, W, tile, pl.P128 / 128, x, y) && !use_fused_small_c(C, tile) && !g_disable_fused)
+    const bool plain = ep.residual == nullptr && ep.act == 0;   // the single-kernel paths end at the bias
+    if (plain && use_fused_small_k(K, W, tile, pl.P128 / 128, x, y) && !use_fused_small_c(C, tile) && !g_disable_fused)
         return launch_fused_small_k(static_cast<const __half*>(x), wT, static_cast<const __half*>(bias),
                                     static_cast<__half*>(y), pl, C, H, W, K, st);
-    if (use_fused_small_c(C, tile) && !g_disable_fused) {
+    if (plain && use_fused_small_c(C, tile) && !g_disable_fused) {
         const TileGeom geo = make_geom(H, W, pl.TH, pl.TW, pl.P);
         const __half* xh = static_cast<const __half*>(x);
         const __half* bh = static_cast<const __half*>(bias);
@@ -709,8 +715,8 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
         prm.num_p_tiles = (count / GEMM_BLOCK_P + shape.ctas - 1) / shape.ctas;
         rc = launch_gemm(tmU, tmV, tmM, prm, shape.ctas, st);
         if (rc != SDWINO_OK) return rc;
-        if (tile == 2) rc = launch_output<2>(Mws, bh, yh, geo, K, p0, count, pc, chk, st);
-        else rc = launch_output<4>(Mws, bh, yh, geo, K, p0, count, pc, chk, st);
+        if (tile == 2) rc = launch_output<2>(Mws, bh, yh, geo, K, p0, count, pc, chk, ep, st);
+        else rc = launch_output<4>(Mws, bh, yh, geo, K, p0, count, pc, chk, ep, st);
         if (rc != SDWINO_OK) return rc;
     }
     return SDWINO_OK;
@@ -813,6 +819,15 @@ int sdwino_conv3x3_ws(const void* x, const void* wT, const void* bias, void* y, 
                       int tile, void* workspace, size_t workspace_bytes, void* stream) {
     return conv_impl(x, wT, bias, y, N, C, H, W, K, tile, workspace, workspace_bytes,
                      static_cast<cudaStream_t>(stream));
+}
+
+int sdwino_conv3x3_ex(const void* x, const void* wT, const void* bias, const void* residual, void* y, int N, int C,
+                      int H, int W, int K, int tile, int activation, void* workspace, size_t workspace_bytes,
+                      void* stream) {
+    if (activation != SDWINO_ACT_NONE && activation != SDWINO_ACT_SILU) return SDWINO_ERR_UNSUPPORTED;
+    if (residual && !aligned(residual, 2)) return SDWINO_ERR_MISALIGNED;
+    return conv_impl(x, wT, bias, y, N, C, H, W, K, tile, workspace, workspace_bytes, static_cast<cudaStream_t>(stream),
+                     Epilogue{static_cast<const __half*>(residual), activation});
 }
 
 int sdwino_conv3x3(const void* x, const void* wT, const void* bias, void* y, int N, int C, int H, int W, int K,

@@ -285,11 +285,24 @@ input_transform_kernel(const __half* __restrict__ x, __half* __restrict__ V, Til
     }
 }
 
+// What follows the postprocess in the same kernel: y = act(A^T M A + bias + residual).  The paper's operator ends at
+// the convolution; the residual sum and the SiLU of the ResNet blocks around it are memory-bound element-wise
+// passes over y that cost nothing extra here.  residual: fp16 [N][K][H][W] or null (may be y itself);
+// act: 0 none, 1 SiLU z / (1 + exp(-z)).
+struct Epilogue {
+    const __half* residual;
+    int act;
+};
+__device__ __forceinline__ float epilogue_act(float v, int act) {
+    return act == 1 ? __fdividef(v, 1.f + __expf(-v)) : v;   // fast division: 2 ulp, far below the fp16 rounding that follows
+}
+
 // Postprocess + bias + cast + masked store.  Mws layout: [a*a][K][Pstride]; y is NCHW.
 template <int M>
 __global__ void __launch_bounds__(128)
 output_transform_kernel(const __half* __restrict__ Mws, const __half* __restrict__ bias, __half* __restrict__ y,
-                        TileGeom geo, int K, long long p_begin, int p_count, long long Pstride, WtCheck chk) {
+                        TileGeom geo, int K, long long p_begin, int p_count, long long Pstride, WtCheck chk,
+                        Epilogue ep) {
     using Wm = Wino<M>;
     constexpr int A = Wm::A;
     pdl_launch_dependents();
@@ -335,9 +348,15 @@ output_transform_kernel(const __half* __restrict__ Mws, const __half* __restrict
         const int oi = i0 + i;
         if (oi >= geo.H) continue;
         __half* rowp = img + static_cast<long long>(oi) * geo.W + j0;
+        const __half* resp = ep.residual ? ep.residual + (rowp - y) : nullptr;
 #pragma unroll
         for (int j = 0; j < M; j += 2) {
-            const __half h0 = __float2half_rn(o[j] + b), h1 = __float2half_rn(o[j + 1] + b);
+            float v0 = o[j] + b, v1 = o[j + 1] + b;
+            if (resp) {
+                if (j0 + j < geo.W) v0 += __half2float(resp[j]);
+                if (j0 + j + 1 < geo.W) v1 += __half2float(resp[j + 1]);
+            }
+            const __half h0 = __float2half_rn(epilogue_act(v0, ep.act)), h1 = __float2half_rn(epilogue_act(v1, ep.act));
             if (vec_ok && (j0 + j + 1 < geo.W)) {
                 *reinterpret_cast<__half2*>(rowp + j) = __halves2half2(h0, h1);
             } else {
@@ -588,10 +607,35 @@ input_transform_f4_kernel(const __half* __restrict__ x, __half* __restrict__ V, 
     input_unit_f4<CH>(x, V, geo, C, p_begin, gdiv, Pstride, blockIdx.x * blockDim.x + threadIdx.x);   // < 2^31
 }
 
-template <int M, int TPT>
+// Eight output pixels of one row (bias already added): residual (its eight values loaded by the caller, ahead of
+// the arithmetic), activation, one rounding, one 16-byte store.
+template <bool EP>
+__device__ __forceinline__ void store_row8(__half* rowp, float (&v)[8], const uint4& r, const Epilogue& ep) {
+    if constexpr (EP) {
+    if (ep.residual) {
+        float a, b2;
+        unpack2(r.x, a, b2); v[0] += a; v[1] += b2;
+        unpack2(r.y, a, b2); v[2] += a; v[3] += b2;
+        unpack2(r.z, a, b2); v[4] += a; v[5] += b2;
+        unpack2(r.w, a, b2); v[6] += a; v[7] += b2;
+    }
+    if (ep.act != 0) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] = epilogue_act(v[i], ep.act);
+    }
+    }   // EP
+    uint4 w;
+    w.x = pack2(v[0], v[1]);
+    w.y = pack2(v[2], v[3]);
+    w.z = pack2(v[4], v[5]);
+    w.w = pack2(v[6], v[7]);
+    *reinterpret_cast<uint4*>(rowp) = w;
+}
+
+template <int M, int TPT, bool EP>
 __device__ __forceinline__ void output_unit_vec(const __half* __restrict__ Mws, const __half* __restrict__ bias,
                                                 __half* __restrict__ y, const TileGeom& geo, int K, long long p_begin,
-                                                const FastDiv& gdiv, long long Pstride, uint32_t idx) {
+                                                const FastDiv& gdiv, long long Pstride, uint32_t idx, const Epilogue& ep) {
     using Wm = Wino<M>;
     constexpr int A = Wm::A;
     static_assert(M * TPT == 8, "one 16-byte row segment per thread");
@@ -623,17 +667,24 @@ __device__ __forceinline__ void output_unit_vec(const __half* __restrict__ Mws, 
         const float b = load_bias(bias, k);
         __half* img = y + (n * K + k) * static_cast<long long>(geo.H) * geo.W;
         const int i0 = M * th, j0 = M * tw;
+        uint4 res[M];
+        if constexpr (EP) {
+#pragma unroll
+            for (int i = 0; i < M; ++i) {
+                res[i] = make_uint4(0u, 0u, 0u, 0u);
+                if (ep.residual && i0 + i < geo.H)
+                    res[i] = __ldg(reinterpret_cast<const uint4*>(ep.residual + (img - y) +
+                                                                   static_cast<long long>(i0 + i) * geo.W + j0));
+            }
+        }
 #pragma unroll
         for (int i = 0; i < M; ++i) {
             float2 o[M];
             at4_packed(tt[i], o);
             if (i0 + i >= geo.H) continue;
-            uint4 w;
-            w.x = pack2(o[0].x + b, o[1].x + b);
-            w.y = pack2(o[2].x + b, o[3].x + b);
-            w.z = pack2(o[0].y + b, o[1].y + b);
-            w.w = pack2(o[2].y + b, o[3].y + b);
-            *reinterpret_cast<uint4*>(img + static_cast<long long>(i0 + i) * geo.W + j0) = w;
+            float v[8] = {o[0].x + b, o[1].x + b, o[2].x + b, o[3].x + b, o[0].y + b, o[1].y + b, o[2].y + b, o[3].y + b};
+            __half* rowp = img + static_cast<long long>(i0 + i) * geo.W + j0;
+            store_row8<EP>(rowp, v, res[i], ep);
         }
     } else {
     float mm[A][A][TPT];
@@ -657,6 +708,16 @@ __device__ __forceinline__ void output_unit_vec(const __half* __restrict__ Mws, 
     const float b = load_bias(bias, k);
     __half* img = y + (n * K + k) * static_cast<long long>(geo.H) * geo.W;
     const int i0 = M * th, j0 = M * tw;
+    uint4 res[M];
+    if constexpr (EP) {
+#pragma unroll
+        for (int i = 0; i < M; ++i) {
+            res[i] = make_uint4(0u, 0u, 0u, 0u);
+            if (ep.residual && i0 + i < geo.H)
+                res[i] = __ldg(reinterpret_cast<const uint4*>(ep.residual + (img - y) +
+                                                               static_cast<long long>(i0 + i) * geo.W + j0));
+        }
+    }
     float out[M][8];  // M output rows of 8 pixels
 #pragma unroll
     for (int t = 0; t < TPT; ++t) {
@@ -681,25 +742,22 @@ __device__ __forceinline__ void output_unit_vec(const __half* __restrict__ Mws, 
 #pragma unroll
     for (int i = 0; i < M; ++i) {
         if (i0 + i >= geo.H) continue;
-        uint4 w;
-        w.x = pack2(out[i][0], out[i][1]);
-        w.y = pack2(out[i][2], out[i][3]);
-        w.z = pack2(out[i][4], out[i][5]);
-        w.w = pack2(out[i][6], out[i][7]);
-        *reinterpret_cast<uint4*>(img + static_cast<long long>(i0 + i) * geo.W + j0) = w;
+        store_row8<EP>(img + static_cast<long long>(i0 + i) * geo.W + j0, out[i], res[i], ep);
     }
     }   // M != 4
 }
 
-template <int M, int TPT>
+// EP = false: the plain convolution (the epilogue argument is ignored and costs no register)
+template <int M, int TPT, bool EP>
 __global__ void __launch_bounds__(128)
 output_transform_vec_kernel(const __half* __restrict__ Mws, const __half* __restrict__ bias, __half* __restrict__ y,
-                            TileGeom geo, int K, long long p_begin, FastDiv gdiv, long long Pstride, WtCheck chk) {
+                            TileGeom geo, int K, long long p_begin, FastDiv gdiv, long long Pstride, WtCheck chk,
+                            Epilogue ep) {
     pdl_launch_dependents();
     const bool wt_ok = wt_check(chk);   // before the wait: see output_transform_kernel
     pdl_wait();
     if (!wt_ok) return;
-    output_unit_vec<M, TPT>(Mws, bias, y, geo, K, p_begin, gdiv, Pstride, blockIdx.x * blockDim.x + threadIdx.x);
+    output_unit_vec<M, TPT, EP>(Mws, bias, y, geo, K, p_begin, gdiv, Pstride, blockIdx.x * blockDim.x + threadIdx.x, ep);
 }
 
 

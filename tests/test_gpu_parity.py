@@ -605,3 +605,47 @@ def test_async_host_entry_with_layers_of_different_sizes(B, shared):
         assert B.sdwino_last_device_status(stream) == B.OK
         for (layer, tile, x, b, wT, y, _), want in zip(jobs, expect):
             assert torch.equal(y, want), (layer.name, tile, rep, shared)
+
+
+@pytest.mark.parametrize("act", ["none", "silu"])
+@pytest.mark.parametrize("shape,tile", [((32, 48, 16, 16, 2), 2), ((32, 48, 16, 16, 2), 4), ((20, 24, 9, 11, 1), 2),
+                                        ((20, 24, 9, 11, 1), 4), ((4, 40, 12, 16, 1), 2), ((40, 4, 12, 16, 2), 2),
+                                        ((64, 64, 64, 64, 1), 4), ((17, 33, 13, 24, 3), 4)])
+def test_fused_residual_and_activation(B, shape, tile, act):
+    # y = act(conv + bias + residual) in the output transform: vector and scalar kernels, both tiles, layers that
+    # would otherwise take a single-kernel path, the residual aliasing y
+    C, K, H, W, N = shape
+    layer = ConvLayer(C=C, K=K, H=H, W=W, N=N)
+    x, w, b = workloads.make_inputs(layer, seed=sum(shape) + tile)
+    g = torch.Generator().manual_seed(99)
+    res = torch.randn((N, K, H, W), generator=g).half()
+    ref = oracle.epilogue(oracle.direct_conv3x3(x.numpy(), w.numpy(), b.numpy()), res.numpy(),
+                          "silu" if act == "silu" else None)
+    wT = B.sdwino_filter_transform(w.cuda(), tile)
+    ws = B.alloc_workspace(B.sdwino_workspace_bytes(N, C, H, W, K, tile))
+    flag = B.ACT_SILU if act == "silu" else B.ACT_NONE
+    y = B.sdwino_conv3x3_ex(x.cuda(), wT, b.cuda(), res.cuda(), K, tile, flag, ws)
+    assert B.sdwino_last_device_status() == B.OK
+    assert _rel_err(y.cpu(), ref) <= TOL
+    # in place: the residual is y
+    y2 = res.cuda().clone()
+    B.sdwino_conv3x3_ex(x.cuda(), wT, b.cuda(), y2, K, tile, flag, ws, y=y2)
+    assert torch.equal(y2, y)
+    # no residual, no bias
+    y3 = B.sdwino_conv3x3_ex(x.cuda(), wT, None, None, K, tile, flag, ws)
+    ref3 = oracle.epilogue(oracle.direct_conv3x3(x.numpy(), w.numpy(), None), None, "silu" if act == "silu" else None)
+    assert _rel_err(y3.cpu(), ref3) <= TOL
+    if act == "none":
+        # nothing to fuse: the plain entry point, bit for bit
+        y4 = B.sdwino_conv3x3(x.cuda(), wT, None, K, tile, workspace=ws)
+        assert torch.equal(y3, y4)
+
+
+def test_fused_epilogue_rejects_unknown_activation(B):
+    layer = ConvLayer(C=16, K=16, H=8, W=8, N=1)
+    x, w, b = workloads.make_inputs(layer, seed=3)
+    wT = B.sdwino_filter_transform(w.cuda(), 2)
+    ws = B.alloc_workspace(B.sdwino_workspace_bytes(1, 16, 8, 8, 16, 2))
+    with pytest.raises(B.SdwinoError) as e:
+        B.sdwino_conv3x3_ex(x.cuda(), wT, b.cuda(), None, 16, 2, 7, ws)
+    assert e.value.status == B.ERR_UNSUPPORTED

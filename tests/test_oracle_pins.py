@@ -247,3 +247,36 @@ def test_fp16_inputs_widen_exactly():
     y16 = oracle.direct_conv3x3(x.numpy(), w.numpy())
     y64 = oracle.direct_conv3x3(x.double().numpy(), w.double().numpy())
     assert np.array_equal(y16, y64)
+
+
+# ---- the epilogue the library can fuse after the convolution -------------------------------------------------
+
+def test_silu_known_values_identities_and_library_routine():
+    # sigmoid(0) = 1/2, sigmoid(ln 3) = 3/4, sigmoid(-ln 3) = 1/4: exact rationals
+    assert oracle.silu(0.0) == 0.0
+    assert abs(oracle.silu(np.log(3.0)) - 0.75 * np.log(3.0)) < 1e-15
+    assert abs(oracle.silu(-np.log(3.0)) + 0.25 * np.log(3.0)) < 1e-15
+    z = np.linspace(-30, 30, 2001)
+    # silu(z) - silu(-z) = z (sigmoid(z) + sigmoid(-z) = 1); limits z and 0
+    assert np.abs(oracle.silu(z) - oracle.silu(-z) - z).max() < 1e-13
+    assert abs(oracle.silu(40.0) - 40.0) < 1e-14 and abs(oracle.silu(-40.0)) < 1e-15
+    assert oracle.silu(-1e4) == 0.0                       # exp overflows: the limit, not NaN
+    # minimum of z*sigmoid(z): -0.27846454276107379 at z = -1.2784645427610738
+    assert abs(oracle.silu(z).min() + 0.27846454276107379) < 1e-4
+    import torch
+    t = torch.nn.functional.silu(torch.from_numpy(z)).numpy()
+    assert np.abs(oracle.silu(z) - t).max() < 1e-14
+
+
+def test_epilogue_adds_the_residual_before_the_activation():
+    rng = np.random.default_rng(5)
+    conv = rng.standard_normal((2, 3, 4, 5))
+    res = rng.standard_normal((2, 3, 4, 5))
+    assert np.array_equal(oracle.epilogue(conv), conv)
+    assert np.array_equal(oracle.epilogue(conv, res) - res, (conv + res) - res)
+    assert np.array_equal(oracle.epilogue(conv, -conv, "silu"), np.zeros_like(conv))       # silu(0) = 0
+    y = oracle.epilogue(conv, res, "silu")
+    zz = conv + res
+    assert np.abs(y * (1.0 + np.exp(-zz)) - zz).max() < 1e-14                              # y (1 + e^-z) = z
+    with pytest.raises(ValueError):
+        oracle.epilogue(conv, None, "relu")
