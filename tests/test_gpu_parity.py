@@ -649,3 +649,35 @@ def test_fused_epilogue_rejects_unknown_activation(B):
     with pytest.raises(B.SdwinoError) as e:
         B.sdwino_conv3x3_ex(x.cuda(), wT, b.cuda(), None, 16, 2, 7, ws)
     assert e.value.status == B.ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("tile", [2, 4])
+def test_more_than_2_to_31_elements(B, tile):
+    # x and y of 2.15e9 elements each (4.3 GB): element offsets no longer fit 32 bits, the layer takes about twenty
+    # passes, and with F(4x4) the passes are cut at whole tile rows for the TMA-staged transform.  Checked on
+    # patches that the oracle computes from crops of x: the two corners that see the zero padding and a patch
+    # whose offsets lie beyond 2^31 and 2^32 bytes.
+    C, K, H, W = 16, 16, 11600, 11584
+    assert C * H * W > 2 ** 31
+    free, _ = torch.cuda.mem_get_info()
+    if free < (24 << 30):
+        pytest.skip("needs 24 GB of free device memory")
+    g = torch.Generator(device="cuda").manual_seed(5)
+    x = torch.empty((1, C, H, W), dtype=torch.float16, device="cuda")
+    for c in range(C):
+        x[0, c] = torch.randn((H, W), generator=g, device="cuda", dtype=torch.float32).half()
+    layer = ConvLayer(C=C, K=K, H=16, W=16, N=1)
+    _, w, b = workloads.make_inputs(layer, seed=21)
+    wT = B.sdwino_filter_transform(w.cuda(), tile)
+    ws = B.alloc_workspace(B.sdwino_workspace_bytes(1, C, H, W, K, tile))
+    y = B.sdwino_conv3x3(x, wT, b.cuda(), K, tile, workspace=ws)
+    assert B.sdwino_last_device_status() == B.OK
+    S = 40
+    for (i0, j0) in [(0, 0), (H - S, W - S), (H // 2 + 3, W // 2 - 5), (H - 2 * S, 8)]:
+        # crop with one extra row / column where the image continues; the oracle pads the crop with zeros, so its
+        # outermost rows and columns are only right where they coincide with the image border
+        r0, r1, c0, c1 = max(i0 - 1, 0), min(i0 + S + 1, H), max(j0 - 1, 0), min(j0 + S + 1, W)
+        crop = x[:, :, r0:r1, c0:c1].cpu().numpy()
+        ref = oracle.direct_conv3x3(crop, w.numpy(), b.numpy())[:, :, i0 - r0:i0 - r0 + S, j0 - c0:j0 - c0 + S]
+        got = y[:, :, i0:i0 + S, j0:j0 + S].cpu().double().numpy()
+        assert np.abs(got - ref).max() <= TOL * np.abs(ref).max(), (tile, i0, j0)
