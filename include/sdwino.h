@@ -210,7 +210,8 @@ int sdwino_set_input_staging(int mode);
  * accuracy bound (F4 with about 4x the error of F2).  Rule, with tiles = N * ceil(H/2) * ceil(W/2):
  * at most 8 input channels -> 2 (single-kernel path); at most 8 output channels -> 2 from 12288 tiles
  * (single-kernel path), 4 below; otherwise 4 when 2 * tiles * (C + K) >= K * C, i.e. when the
- * activation-side traffic outweighs the weights.
+ * activation-side traffic outweighs the weights, and also from 0.65 of that threshold when there are at least
+ * 256 tiles.
  * Pure host arithmetic: no device is touched.  The caller passes the result as `tile` to
  * sdwino_filter_transform and sdwino_conv3x3.
  */

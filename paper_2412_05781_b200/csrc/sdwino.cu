@@ -753,7 +753,11 @@ int sdwino_choose_tile(int N, int C, int H, int W, int K) {
     // few output channels: the single-kernel F(2x2) path needs many blocks of tiles to fill the SMs; below about
     // a hundred of them the three-kernel F(4x4) path is 5-20 % faster (320->4 at 64x64: 12.2 against 14.7 us)
     if (K <= 8) return P2 >= 12288 ? 2 : 4;
-    return 2 * P2 * (static_cast<long long>(C) + K) >= static_cast<long long>(K) * C ? 4 : 2;
+    const long long act = 2 * P2 * (static_cast<long long>(C) + K), wgt = static_cast<long long>(K) * C;
+    if (act >= wgt) return 4;
+    // between 0.65 and 1 of the threshold F4 is still 7-10 % faster once there are 256 tiles or more (2560->1280 at
+    // 24x24, batch 2: 53 against 59 us), and 4-35 % slower with fewer (640->1280 at 24x24, batch 1)
+    return (20 * act >= 13 * wgt && P2 >= 256) ? 4 : 2;
 }
 
 int sdwino_set_fused_min_tiles(long long p_tiles) {

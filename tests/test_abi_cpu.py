@@ -111,5 +111,9 @@ def test_choose_tile_is_host_arithmetic(binding):
     # threshold: 2 * tiles * (C + K) >= K * C with tiles = N * ceil(H/2) * ceil(W/2)
     assert binding.sdwino_choose_tile(1, 64, 7, 7, 64) == 4       # 2*16*128 = 4096 >= 4096
     assert binding.sdwino_choose_tile(1, 64, 6, 7, 64) == 2       # 2*12*128 = 3072 <  4096
+    # between 0.65 and 1 of the threshold: F(4x4) only with at least 256 tiles
+    assert binding.sdwino_choose_tile(2, 2560, 24, 24, 1280) == 4  # 288 tiles, ratio 0.68
+    assert binding.sdwino_choose_tile(1, 640, 24, 24, 1280) == 2   # 144 tiles, ratio 0.68
+    assert binding.sdwino_choose_tile(2, 640, 16, 16, 1280) == 2   # 128 tiles, ratio 0.60
     with pytest.raises(binding.SdwinoError):
         binding.sdwino_choose_tile(0, 1, 1, 1, 1)
