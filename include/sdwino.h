@@ -196,11 +196,13 @@ unsigned long long sdwino_launch_count(void);
 int sdwino_set_gemm_shape(int ctas, int n_tile);
 
 /*
- * Test hook for the activation transform of step (i) with tile = 4.  A layer that is done in one pass, with
- * W % 8 == 0 and a 16-byte aligned x, can stage the overlapping input tiles in shared memory by TMA instead of
- * loading them into registers; both kernels produce the same bits.  mode 1 (the default) stages where that
- * measured faster (W % 64 == 0), mode 2 wherever it is possible, mode 0 never.  Returns SDWINO_ERR_INVALID_ARG
- * for any other value.  Not thread-safe against concurrent compute calls.
+ * Test hook for the transforms of steps (i) and (iii) with tile = 4.  With W % 8 == 0 and 16-byte aligned x / y
+ * they can stage their operands in shared memory by TMA, several channels ahead of the arithmetic (the
+ * overlapping input tiles of a block; the 36 transform positions of a block of tiles), instead of loading them
+ * into registers; both forms produce the same bits.  mode 1 (the default) stages where that measured faster
+ * (activation transform: W % 64 == 0; output transform: passes of 512 tiles or more), mode 2 wherever it is
+ * possible, mode 0 never.  Returns SDWINO_ERR_INVALID_ARG for any other value.  Not thread-safe against
+ * concurrent compute calls.
  */
 int sdwino_set_input_staging(int mode);
 

@@ -19,6 +19,7 @@
 #include "wino_gemm.cuh"
 #include "fused_small_k.cuh"
 #include "input_tma.cuh"
+#include "output_tma.cuh"
 
 namespace {
 
@@ -436,6 +437,59 @@ int launch_input_tma(const __half* x, __half* V, const TileGeom& geo, int N, int
     return e == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
 }
 
+// The TMA-staged F(4x4) output transform: see output_tma.cuh.
+bool use_output_tma(const TileGeom& geo, int K, const void* y, const Epilogue& ep, int p_count) {
+    const bool possible = geo.W % 8 == 0 && aligned(y, 16) && aligned(ep.residual, 16) && K <= 65535 * 16;
+    if (!possible || g_input_staging == 0) return false;
+    // 7-13 % faster on layers of thousands of tiles (256->256 at 512x512: 73.5 -> 65.9 us), even at 512, a few
+    // percent slower on the 128-tile passes of the 32x32 layers
+    return g_input_staging == 2 || p_count >= 512;
+}
+
+int launch_output_tma(const __half* Mws, const __half* bias, __half* y, const TileGeom& geo, int K, long long p_begin,
+                      int p_count, long long Pstride, const WtCheck& chk, const Epilogue& ep, cudaStream_t st) {
+    ProfScope prof(KIND_OUTPUT, st);
+    const int sms = sm_count();
+    int* status = status_word_ptr();
+    if (sms <= 0 || !status) return SDWINO_ERR_CUDA;
+    CUtensorMap tmM;
+    if (!encode_image_map(&tmM, Mws, static_cast<uint64_t>(Pstride), static_cast<uint64_t>(K), 36, OUT_TMA_TILES, 1, 36))
+        return SDWINO_ERR_CUDA;
+    const long long blocks = (p_count + OUT_TMA_TILES - 1) / OUT_TMA_TILES;
+    // channels per CTA (at most 16): three CTAs are resident per SM; the time follows the SM with the most
+    // CTA-steps (one more step per CTA for the fill)
+    long long steps = 1;
+    double best_cost = 1e300;
+    for (long long cand = 1; cand <= 16 && cand <= K; ++cand) {
+        const long long ctas = blocks * ((K + cand - 1) / cand);
+        const long long per_sm = (ctas + sms - 1) / sms;
+        const double cost = per_sm <= 3 ? per_sm * (cand + 1.0) * std::max(1.0, 3.0 / per_sm)
+                                        : static_cast<double>((ctas + 3ll * sms - 1) / (3ll * sms)) * 3.0 * (cand + 1.0);
+        if (cost <= best_cost) { best_cost = cost; steps = cand; }
+    }
+    const size_t smem = static_cast<size_t>(OUT_TMA_STAGES) * OUT_TMA_STAGE_BYTES + 128;
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [&] {
+        attr_err = cudaFuncSetAttribute(output_transform_f4_tma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        static_cast<int>(smem));
+        if (attr_err == cudaSuccess)
+            attr_err = cudaFuncSetAttribute(output_transform_f4_tma_kernel<true>,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    });
+    if (attr_err != cudaSuccess || blocks >= (1ll << 31)) return SDWINO_ERR_CUDA;
+    dim3 grid(static_cast<unsigned>(blocks), static_cast<unsigned>((K + steps - 1) / steps));
+    cudaError_t e;
+    if (ep.residual == nullptr && ep.act == 0)
+        e = launch_pdl(output_transform_f4_tma_kernel<false>, grid, dim3(OUT_TMA_THREADS), smem, st, 0, tmM, bias, y, geo, K,
+                       p_begin, static_cast<int>(steps), chk, ep, status);
+    else
+        e = launch_pdl(output_transform_f4_tma_kernel<true>, grid, dim3(OUT_TMA_THREADS), smem, st, 0, tmM, bias, y, geo, K,
+                       p_begin, static_cast<int>(steps), chk, ep, status);
+    g_launches.fetch_add(1);
+    return e == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
+}
+
 template <int M>
 int launch_output(const __half* Mws, const __half* bias, __half* y, const TileGeom& geo, int K,
                   long long p_begin, int p_count, long long Pstride, const WtCheck& chk, const Epilogue& ep,
@@ -716,6 +770,7 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
         rc = launch_gemm(tmU, tmV, tmM, prm, shape.ctas, st);
         if (rc != SDWINO_OK) return rc;
         if (tile == 2) rc = launch_output<2>(Mws, bh, yh, geo, K, p0, count, pc, chk, ep, st);
+        else if (use_output_tma(geo, K, y, ep, count)) rc = launch_output_tma(Mws, bh, yh, geo, K, p0, count, pc, chk, ep, st);
         else rc = launch_output<4>(Mws, bh, yh, geo, K, p0, count, pc, chk, ep, st);
         if (rc != SDWINO_OK) return rc;
     }
