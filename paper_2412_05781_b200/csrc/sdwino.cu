@@ -643,15 +643,15 @@ GemmShape choose_gemm_shape(int K, int C, long long p_tiles128, int a2, int sms,
     return best;
 }
 
-template <int CTAS>
+template <int CTAS, bool RES>
 int launch_gemm_shape(const CUtensorMap& tmU, const CUtensorMap& tmV, const CUtensorMap& tmM, const GemmParams& prm,
                       int sms, int* status, cudaStream_t st) {
     using L = GemmSmemLayout;
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [&] {
-        attr_err =
-            cudaFuncSetAttribute(wino_gemm_kernel<CTAS>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_DYN_SMEM);
+        attr_err = cudaFuncSetAttribute(wino_gemm_kernel<CTAS, RES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        MAX_DYN_SMEM);
     });
     if (attr_err != cudaSuccess) return SDWINO_ERR_CUDA;
     const long long tiles = static_cast<long long>(prm.num_k_tiles) * prm.num_p_tiles * prm.num_pos;
@@ -659,9 +659,10 @@ int launch_gemm_shape(const CUtensorMap& tmU, const CUtensorMap& tmV, const CUte
     const int grid = static_cast<int>(tiles < workers ? tiles : workers) * CTAS;
     ProfScope prof(KIND_GEMM, st);
     const cudaError_t e =
-        launch_pdl(wino_gemm_kernel<CTAS>, dim3(grid), dim3(GEMM_THREADS),
-                   static_cast<size_t>(L::dyn_bytes(prm.n_tile / CTAS, prm.stages, prm.epi_rows, prm.epi_bufs)), st, CTAS,
-                   tmU, tmV, tmM, prm, status);
+        launch_pdl(wino_gemm_kernel<CTAS, RES>, dim3(grid), dim3(GEMM_THREADS),
+                   static_cast<size_t>(L::dyn_bytes(RES ? 0 : prm.n_tile / CTAS, prm.stages, prm.epi_rows, prm.epi_bufs,
+                                                    RES ? prm.num_c_blocks * L::b_bytes(prm.n_tile) : 0)),
+                   st, CTAS, tmU, tmV, tmM, prm, status);
     g_launches.fetch_add(1);
     return e == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
 }
@@ -673,8 +674,9 @@ int launch_gemm(const CUtensorMap& tmU, const CUtensorMap& tmV, const CUtensorMa
     static int* status = nullptr;   // device address of the status word (one device per process)
     if (!status && cudaGetSymbolAddress(reinterpret_cast<void**>(&status), g_status_word) != cudaSuccess)
         return SDWINO_ERR_CUDA;
-    if (ctas == 2) return launch_gemm_shape<2>(tmU, tmV, tmM, prm, sms, status, st);
-    return launch_gemm_shape<1>(tmU, tmV, tmM, prm, sms, status, st);
+    if (ctas == 2) return launch_gemm_shape<2, false>(tmU, tmV, tmM, prm, sms, status, st);
+    if (prm.resident) return launch_gemm_shape<1, true>(tmU, tmV, tmM, prm, sms, status, st);
+    return launch_gemm_shape<1, false>(tmU, tmV, tmM, prm, sms, status, st);
 }
 
 
@@ -741,9 +743,50 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
     const bool split = (prm.n_tile / 2) % 16 == 0;
     prm.epi_rows = split ? prm.n_tile / 2 : prm.n_tile;
     prm.epi_bufs = split ? 2 : 1;
+    prm.epi_chunks = 1;
+    prm.resident = 0;
+    prm.group = 1;
     prm.stages = (MAX_DYN_SMEM - GemmSmemLayout::dyn_bytes(b_rows, 0, prm.epi_rows, prm.epi_bufs)) /
                  GemmSmemLayout::stage_bytes(b_rows);
     if (prm.stages > GEMM_MAX_STAGES) prm.stages = GEMM_MAX_STAGES;
+    {
+        // Filter-resident mode (see wino_gemm.cuh): single CTAs, many tiles per CTA and long runs of tiles per
+        // (position, k-tile), the filter block two thirds of a stage (n_tile 224-256), and room for it beside a ring
+        // of at least four V stages once the epilogue stages 64 channels at a time.  Measured: 256->256 at 512x512
+        // GEMM 146 -> 120 us, at 1024x1024 570 -> 472 us; with n_tile 128-160 (filters half of a stage or less, the
+        // layer close to the HBM roof already) the pause at every change of filter block costs more than the
+        // re-reads: 128->128 at 512x512 57 -> 74 us.
+        const long long p_tiles = pc / GEMM_BLOCK_P;
+        const long long tiles = p_tiles * ((K + prm.n_tile - 1) / prm.n_tile) * pl.a2;
+        const int ures = prm.num_c_blocks * GemmSmemLayout::b_bytes(prm.n_tile);
+        const int grp = prm.epi_rows;
+        const int rows = (grp > 64 && grp % 64 == 0) ? 64 : grp;
+        const int stages = (MAX_DYN_SMEM - GemmSmemLayout::dyn_bytes(0, 0, rows, prm.epi_bufs, ures)) / GemmSmemLayout::A_BYTES;
+        if (shape.ctas == 1 && g_force_ctas == 0 && g_force_n_tile == 0 && p_tiles >= 16 && tiles >= 4ll * sms &&
+            prm.n_tile >= 224 && stages >= 4) {
+            prm.resident = 1;
+            // CTAs per (position, k-tile) pair: as many as leave every CTA a run of at least 8 tiles (so that its
+            // filter block is re-used), the largest group among the splits of pairs over groups and of tiles over a group that
+            // are within 3 % of the most even one (the CTAs of a group read neighbouring pieces of V at the same time)
+            const long long keys = ((K + prm.n_tile - 1) / prm.n_tile) * static_cast<long long>(pl.a2);
+            auto efficiency = [&](int g) {
+                const long long ng = sms / g;
+                const long long rounds = (keys + ng - 1) / ng;
+                const long long run = (p_tiles + g - 1) / g;
+                return static_cast<double>(keys * p_tiles) / (static_cast<double>(rounds) * run * sms);
+            };
+            const int g_max = static_cast<int>(std::min<long long>(sms, p_tiles / 8));
+            double best_eff = 0.0;
+            for (int g = 1; g <= g_max; ++g) best_eff = std::max(best_eff, efficiency(g));
+            int best_g = 1;
+            for (int g = 1; g <= g_max; ++g)
+                if (efficiency(g) >= best_eff - 0.03) best_g = g;     // the largest group within 3 % of the best split
+            prm.group = best_g;
+            prm.epi_chunks = grp / rows;
+            prm.epi_rows = rows;
+            prm.stages = stages > GEMM_MAX_STAGES ? GEMM_MAX_STAGES : stages;
+        }
+    }
 
     prm.p_stride = pc;
     CUtensorMap tmU, tmV, tmM;

@@ -15,6 +15,12 @@
 // bytes fetched from L2 per MMA cycle -- the measured limit of the single-CTA shape.  The leader
 // (even rank) issues the MMAs; completion is signalled to the barriers of both CTAs.
 //
+// Filter-resident mode (single CTAs, layers whose filter block n_tile x C fits beside the ring): a layer with few
+// channels and many tiles re-reads the same n_tile x C filter block for every tile p, and at C = K = 256 those
+// re-reads are two thirds of the bytes that cross from L2 to the SMs, which is what bounds the kernel there.  The CTAs
+// then work in groups: a group takes whole (pos, k-tile) pairs, its CTAs share out the tiles p of a pair, load the
+// pair's filter block once into a resident buffer and stream only V through the ring.
+//
 // One persistent CTA (pair) per SM (pair) walks the list of (pos, k-tile, p-tile) output tiles.
 //   warp 0   : TMA producer        (one lane)
 //   warp 1   : TMEM owner + MMA issuer (one lane)
@@ -47,7 +53,7 @@ struct GemmSmemLayout {
     static constexpr int A_BYTES = GEMM_BLOCK_P * GEMM_BLOCK_C * 2;          // two [64 p][64 c] boxes
     static constexpr int A_BOX_BYTES = 64 * GEMM_BLOCK_C * 2;
     static constexpr int EPI_ROW_BYTES = GEMM_BLOCK_P * 2;                   // one staged row: 128 p fp16
-    static constexpr int BAR_BYTES = (2 * GEMM_MAX_STAGES + 4) * 8 + 16;
+    static constexpr int BAR_BYTES = (2 * GEMM_MAX_STAGES + 6) * 8 + 16;
     // `rows` = rows of U this CTA loads per stage: n_tile (single CTA) or n_tile / 2 (CTA pair)
     __host__ __device__ static constexpr int b_bytes(int rows) { return rows * GEMM_BLOCK_C * 2; }
     __host__ __device__ static constexpr int stage_bytes(int rows) {
@@ -57,9 +63,10 @@ struct GemmSmemLayout {
     __host__ __device__ static constexpr int epi_bytes(int epi_rows, int bufs) {
         return bufs * epi_rows * EPI_ROW_BYTES;
     }
-    // dynamic shared memory for `stages` stages, including slack to align the base to 1024 bytes
-    __host__ __device__ static constexpr int dyn_bytes(int rows, int stages, int epi_rows, int bufs) {
-        return stages * stage_bytes(rows) + epi_bytes(epi_rows, bufs) + BAR_BYTES + 1024;
+    // dynamic shared memory for `stages` stages, including slack to align the base to 1024 bytes; `resident` =
+    // bytes of filter blocks kept in shared memory across tiles (0 when the filters travel with the stages)
+    __host__ __device__ static constexpr int dyn_bytes(int rows, int stages, int epi_rows, int bufs, int resident = 0) {
+        return stages * stage_bytes(rows) + resident + epi_bytes(epi_rows, bufs) + BAR_BYTES + 1024;
     }
 };
 
@@ -75,6 +82,10 @@ struct GemmParams {
     int stages;
     int epi_rows;      // channels staged per TMA store and epilogue group: n_tile or n_tile / 2, multiple of 16
     int epi_bufs;      // staging buffers = epilogue groups with work (1 or 2)
+    int epi_chunks;    // TMA stores per group and tile: a group drains epi_rows * epi_chunks channels
+    int resident;      // 1: the filter blocks of a (position, k-tile) stay in shared memory while the CTA walks the
+                       // tiles p of that pair (stages then hold V only)
+    int group;         // filter-resident mode: CTAs that share out the tiles of one (position, k-tile) pair
     long long p_stride;  // tiles per pass (row pitch of V and M)
 };
 
@@ -82,7 +93,8 @@ struct GemmParams {
 // tmU: fp16 [pos][Cb][Kb][16][64] box {64 c, 16 k, 1, n_tile/16, 1}, 128B swizzle (B operand: n_tile rows of 128
 //      bytes in k order; blocks past Kb read as 0)
 // tmM: fp16 [pos][K][Pstride]   box {128 p, epi_rows k, 1}, no swizzle  (result; rows k >= K are clipped)
-template <int CTAS>
+// RES: the filter-resident mode as a separate instantiation, so that the streaming kernel pays nothing for it.
+template <int CTAS, bool RES = false>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant__ CUtensorMap tmV,
                  const __grid_constant__ CUtensorMap tmM, const GemmParams prm, int* __restrict__ status_word) {
@@ -93,24 +105,56 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int b_rows = prm.n_tile / CTAS;            // rows of U this CTA loads per stage
-    const int stage_bytes = L::stage_bytes(b_rows);
+    static_assert(!RES || CTAS == 1, "filter-resident mode is for single CTAs");
+    constexpr bool resident = RES;
+    const int stage_bytes = resident ? L::A_BYTES : L::stage_bytes(b_rows);
+    const int ures_cb_bytes = L::b_bytes(prm.n_tile);                       // one 64-channel block of the resident filters
+    const int ures_bytes = resident ? prm.num_c_blocks * ures_cb_bytes : 0;
     const int stages = prm.stages;
     const uint32_t cta_rank = CTAS == 2 ? cluster_ctarank() : 0u;
     const bool leader = cta_rank == 0;
     const int worker = blockIdx.x / CTAS;            // index of this CTA (pair) among the persistent workers
     const int num_workers = gridDim.x / CTAS;
-    uint8_t* epi_base = smem + stages * stage_bytes;
+    uint8_t* ures_base = smem + stages * stage_bytes;
+    uint8_t* epi_base = ures_base + ures_bytes;
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(epi_base + L::epi_bytes(prm.epi_rows, prm.epi_bufs));
     uint64_t* empty_bar = full_bar + GEMM_MAX_STAGES;
     uint64_t* acc_full_bar = empty_bar + GEMM_MAX_STAGES;
     uint64_t* acc_empty_bar = acc_full_bar + 2;
-    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(acc_empty_bar + 2);
+    uint64_t* ures_full_bar = acc_empty_bar + 2;     // the resident filter block has arrived
+    uint64_t* ures_empty_bar = ures_full_bar + 1;    // the MMAs that read it have completed
+    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(ures_empty_bar + 1);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_base_slot + 1);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const int num_tiles = prm.num_k_tiles * prm.num_p_tiles * prm.num_pos;
     constexpr uint32_t TMEM_COLS = 2 * GEMM_MAX_N;
+    // The tiles of this worker, numbered i = 0 .. my_count - 1.  Streaming mode: every num_workers-th tile of the
+    // list.  Filter-resident mode: the workers form groups of `group` CTAs; a group takes every num_groups-th
+    // (position, k-tile) pair and its CTAs share out the tiles p of the pair round-robin, so that a CTA stays with
+    // one filter block for many tiles while the CTAs of a group read neighbouring pieces of V at the same time.
+    const int grp_size = resident ? prm.group : 1;
+    const int num_groups = num_workers / grp_size;
+    const int grp_id = worker / grp_size, grp_lane = worker - grp_id * grp_size;
+    int run_len = 0;      // tiles per (position, k-tile) pair for this CTA
+    int my_count;
+    if constexpr (resident) {
+        const int num_keys = prm.num_k_tiles * prm.num_pos;
+        run_len = grp_lane < prm.num_p_tiles ? (prm.num_p_tiles - grp_lane + grp_size - 1) / grp_size : 0;
+        my_count = grp_id < num_groups ? run_len * ((num_keys - grp_id + num_groups - 1) / num_groups) : 0;
+        if (grp_id >= num_keys) my_count = 0;
+    } else {
+        my_count = worker < num_tiles ? (num_tiles - worker + num_workers - 1) / num_workers : 0;
+    }
+    auto tile_of = [&](int i) -> int {
+        if constexpr (!resident) {
+            return worker + i * num_workers;
+        } else {
+            const int r = i / run_len;
+            return (grp_id + r * num_groups) * prm.num_p_tiles + grp_lane + (i - r * run_len) * grp_size;
+        }
+    };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) {
@@ -121,6 +165,8 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
             mbar_init(&acc_full_bar[b], 1);
             mbar_init(&acc_empty_bar[b], 8 * CTAS);   // one arrival per epilogue warp of every CTA
         }
+        mbar_init(ures_full_bar, 1);
+        mbar_init(ures_empty_bar, 1);
         *abort_flag = 0;
         fence_barrier_init();
         prefetch_tmap(&tmU);
@@ -145,7 +191,59 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
         if (threadIdx.x == 0) atomicCAS(status_word, 0, 1 | (9 << 8));   // 1 = SDWINO_ERR_INVALID_ARG
     } else if (warp == 0) {
         // ------------------------------ TMA producer ------------------------------
-        if (lane == 0) {
+        if (resident && lane == 0) {
+            // filter-resident mode: the filter block of a (position, k-tile) is loaded once, V streams through the ring
+            const uint32_t smem_base = smem_u32(smem);
+            const uint32_t ures_a = smem_u32(ures_base);
+            const uint32_t ures_full_a = smem_u32(ures_full_bar);
+            const uint32_t full0 = smem_u32(&full_bar[0]);
+            auto load_filters = [&](int pos, int kt) {
+                mbar_arrive_expect_tx_a32(ures_full_a, static_cast<uint32_t>(ures_bytes));
+                for (int cb = 0; cb < prm.num_c_blocks; ++cb)
+                    tma_load_5d_a32(ures_a + cb * ures_cb_bytes, &tmU, ures_full_a, cb, (kt * prm.n_tile) >> 4, pos);
+            };
+            int cur_key = -1;
+            uint32_t reloads = 0;
+            if (my_count > 0) {
+                // the filters do not depend on the preceding kernel: the first block goes out before the wait
+                const int t0 = tile_of(0);
+                const int kt = (t0 / prm.num_p_tiles) % prm.num_k_tiles;
+                const int pos = t0 / (prm.num_p_tiles * prm.num_k_tiles);
+                load_filters(pos, kt);
+                cur_key = pos * prm.num_k_tiles + kt;
+            }
+            pdl_wait();   // V is written by the preceding kernel
+            int stage = 0;
+            uint32_t phase = 0;
+            uint32_t sa = smem_base, fb = full0;
+            bool ok = true;
+            for (int i = 0; i < my_count && ok; ++i) {
+                const int tile = tile_of(i);
+                const int pt = tile % prm.num_p_tiles;
+                const int kt = (tile / prm.num_p_tiles) % prm.num_k_tiles;
+                const int pos = tile / (prm.num_p_tiles * prm.num_k_tiles);
+                if (pos * prm.num_k_tiles + kt != cur_key) {
+                    // the MMAs of the previous run of tiles have finished reading the resident block
+                    ok = mbar_wait_bounded(ures_empty_bar, reloads & 1u, abort_flag, GEMM_WAIT_LIMIT_NS);
+                    if (!ok) { if (*abort_flag == 0) report_timeout(status_word, 5, cta_rank); break; }
+                    ++reloads;
+                    load_filters(pos, kt);
+                    cur_key = pos * prm.num_k_tiles + kt;
+                }
+                const int p0 = pt * GEMM_BLOCK_P;
+                for (int c0 = 0; c0 < prm.C; c0 += GEMM_BLOCK_C) {
+                    ok = mbar_wait_bounded(&empty_bar[stage], phase ^ 1u, abort_flag, GEMM_WAIT_LIMIT_NS);
+                    if (!ok) { if (*abort_flag == 0) report_timeout(status_word, 1, cta_rank); break; }
+                    mbar_arrive_expect_tx_a32(fb, L::A_BYTES);
+                    tma_load_3d_a32(sa, &tmV, fb, p0, c0, pos);
+                    tma_load_3d_a32(sa + L::A_BOX_BYTES, &tmV, fb, p0 + 64, c0, pos);
+                    sa += stage_bytes;
+                    fb += 8;
+                    if (++stage == stages) { stage = 0; phase ^= 1u; sa = smem_base; fb = full0; }
+                }
+            }
+            if (!ok) *abort_flag = 1;
+        } else if (!resident && lane == 0) {
             // the full barrier of a pair lives in the leader and counts the bytes of both CTAs
             const uint32_t tx_bytes = CTAS * (L::A_BYTES + L::b_bytes(b_rows));
             // single-thread loop: shared-memory and barrier addresses are running 32-bit values
@@ -161,7 +259,8 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
             int pre = 0;
             if constexpr (CTAS == 1) {
                 uint32_t sa_u = smem_base + L::A_BYTES, fb_u = full0;
-                for (int tile = worker; tile < num_tiles && pre < stages; tile += num_workers) {
+                for (int i = 0; i < my_count && pre < stages; ++i) {
+                    const int tile = tile_of(i);
                     const int kt = (tile / prm.num_p_tiles) % prm.num_k_tiles;
                     const int pos = tile / (prm.num_p_tiles * prm.num_k_tiles);
                     const int k0 = kt * prm.n_tile;
@@ -179,7 +278,8 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
             int issued = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int tile = worker; tile < num_tiles && ok; tile += num_workers) {
+            for (int i = 0; i < my_count && ok; ++i) {
+                const int tile = tile_of(i);
                 const int pt = tile % prm.num_p_tiles;
                 const int kt = (tile / prm.num_p_tiles) % prm.num_k_tiles;
                 const int pos = tile / (prm.num_p_tiles * prm.num_k_tiles);
@@ -231,6 +331,10 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
             const uint64_t adesc0 = make_smem_desc_sw128(smem_base, L::A_BOX_BYTES, 1024);
             const uint64_t bdesc0 = make_smem_desc_sw128(smem_base + L::A_BYTES, 16, 1024);
             const uint64_t stage_step = static_cast<uint64_t>(stage_bytes >> 4);
+            const uint64_t ures_desc0 = make_smem_desc_sw128(smem_u32(ures_base), 16, 1024);
+            const uint64_t ures_step = static_cast<uint64_t>(ures_cb_bytes >> 4);
+            int cur_key = -1;          // filter-resident mode: the (position, k-tile) whose filters are in shared memory
+            uint32_t loads_seen = 0;
             uint64_t adesc = adesc0, bdesc = bdesc0;
             const uint32_t full0_a = smem_u32(&full_bar[0]), empty0_a = smem_u32(&empty_bar[0]);
             uint32_t full_a = full0_a, empty_a = empty0_a;
@@ -241,7 +345,18 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
             int buf = 0;
             uint32_t acc_phase = 0;
             bool ok = true;
-            for (int tile = worker; tile < num_tiles && ok; tile += num_workers) {
+            for (int i = 0; i < my_count && ok; ++i) {
+                const int tile = tile_of(i);
+                int key = 0;
+                if (resident) {
+                    key = tile / prm.num_p_tiles;      // pos * num_k_tiles + kt
+                    if (key != cur_key) {
+                        ok = mbar_wait_bounded(ures_full_bar, loads_seen & 1u, abort_flag, GEMM_WAIT_LIMIT_NS);
+                        if (!ok) { if (*abort_flag == 0) report_timeout(status_word, 6, cta_rank); break; }
+                        ++loads_seen;
+                        cur_key = key;
+                    }
+                }
                 ok = mbar_wait_bounded(&acc_empty_bar[buf], acc_phase ^ 1u, abort_flag, GEMM_WAIT_LIMIT_NS);
                 if (!ok) { if (*abort_flag == 0) report_timeout(status_word, 2, cta_rank); break; }
                 tc_fence_after_sync();
@@ -252,6 +367,7 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
                         if (!ok) { if (*abort_flag == 0) report_timeout(status_word, 3, cta_rank); break; }
                     }
                     tc_fence_after_sync();
+                    const uint64_t bd = resident ? ures_desc0 + static_cast<uint64_t>(cb) * ures_step : bdesc;
                     if (cb < full_blocks) {
                         if constexpr (CTAS == 2) {
                             umma_f16_pair(d_tmem, adesc, bdesc, idesc, static_cast<uint32_t>(cb));
@@ -259,17 +375,17 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
                             umma_f16_pair_acc(d_tmem, adesc + 256, bdesc + 4, idesc);
                             umma_f16_pair_acc(d_tmem, adesc + 384, bdesc + 6, idesc);
                         } else {
-                            umma_f16(d_tmem, adesc, bdesc, idesc, static_cast<uint32_t>(cb));
-                            umma_f16_acc(d_tmem, adesc + 128, bdesc + 2, idesc);
-                            umma_f16_acc(d_tmem, adesc + 256, bdesc + 4, idesc);
-                            umma_f16_acc(d_tmem, adesc + 384, bdesc + 6, idesc);
+                            umma_f16(d_tmem, adesc, bd, idesc, static_cast<uint32_t>(cb));
+                            umma_f16_acc(d_tmem, adesc + 128, bd + 2, idesc);
+                            umma_f16_acc(d_tmem, adesc + 256, bd + 4, idesc);
+                            umma_f16_acc(d_tmem, adesc + 384, bd + 6, idesc);
                         }
                     } else {
                         for (int s = 0; s < last_ksteps; ++s) {
                             if constexpr (CTAS == 2)
                                 umma_f16_pair(d_tmem, adesc + 128 * s, bdesc + 2 * s, idesc, (cb > 0 || s > 0) ? 1u : 0u);
                             else
-                                umma_f16(d_tmem, adesc + 128 * s, bdesc + 2 * s, idesc, (cb > 0 || s > 0) ? 1u : 0u);
+                                umma_f16(d_tmem, adesc + 128 * s, bd + 2 * s, idesc, (cb > 0 || s > 0) ? 1u : 0u);
                         }
                     }
                     if constexpr (CTAS == 2) umma_commit_pair_a32(empty_a);
@@ -285,6 +401,8 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
                 if (!ok) break;
                 if constexpr (CTAS == 2) umma_commit_pair(&acc_full_bar[buf]);
                 else umma_commit(&acc_full_bar[buf]);
+                // the last tile of a run: once its MMAs have completed the resident filters may be replaced
+                if (resident && i + 1 < my_count && tile_of(i + 1) / prm.num_p_tiles != key) umma_commit(ures_empty_bar);
                 buf ^= 1;
                 if (buf == 0) acc_phase ^= 1u;
             }
@@ -300,7 +418,8 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
         uint32_t acc_phase = 0;
         // the accumulator-empty barrier of a pair lives in the leader
         const uint32_t acc_empty_addr0 = CTAS == 2 ? map_to_cta(smem_u32(&acc_empty_bar[0]), 0) : 0u;
-        for (int tile = worker; tile < num_tiles; tile += num_workers) {
+        for (int i = 0; i < my_count; ++i) {
+            const int tile = tile_of(i);
             const int pt = tile % prm.num_p_tiles;
             const int kt = (tile / prm.num_p_tiles) % prm.num_k_tiles;
             const int pos = tile / (prm.num_p_tiles * prm.num_k_tiles);
@@ -321,7 +440,10 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
             const bool p_ok = p0 < prm.p_stride;   // the second CTA of the last pair may hang over the pass
             // lane = tile p, registers = output channels: staging row k receives 32 consecutive p from
             // each warp (64 contiguous bytes, no bank conflict).  Group g owns staging buffer g.
-            const int row0 = group * prm.epi_rows;
+            // a group drains its channels in epi_chunks pieces of epi_rows, one TMA store each
+            const int chunks = resident ? prm.epi_chunks : 1;
+            for (int ch = 0; ch < chunks; ++ch) {
+            const int row0 = (group * chunks + ch) * prm.epi_rows;
             if (row0 < prm.n_tile) {
                 uint8_t* stg = epi_base + group * prm.epi_rows * L::EPI_ROW_BYTES;
                 // the buffer about to be overwritten must have been read by the group's previous TMA store
@@ -352,6 +474,7 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
                     tma_store_commit();
                 }
             }
+            }   // chunks
             // accumulator drained: hand the TMEM buffer back to the MMA warp
             tc_fence_before_sync();
             __syncwarp();

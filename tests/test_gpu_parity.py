@@ -681,3 +681,29 @@ def test_more_than_2_to_31_elements(B, tile):
         ref = oracle.direct_conv3x3(crop, w.numpy(), b.numpy())[:, :, i0 - r0:i0 - r0 + S, j0 - c0:j0 - c0 + S]
         got = y[:, :, i0:i0 + S, j0:j0 + S].cpu().double().numpy()
         assert np.abs(got - ref).max() <= TOL * np.abs(ref).max(), (tile, i0, j0)
+
+
+@pytest.mark.parametrize("shape,tile", [((128, 128, 128, 128, 3), 4), ((256, 256, 128, 128, 2), 4), ((256, 256, 96, 96, 1), 2),
+                                        ((320, 320, 128, 128, 1), 4), ((192, 200, 100, 104, 2), 4), ((64, 96, 160, 160, 2), 4),
+                                        ((256, 128, 256, 256, 1), 4)])
+def test_filter_resident_gemm_matches_streaming_gemm_bitwise(B, shape, tile):
+    # Layers with few channels and thousands of tiles keep the filter block of a (position, k-tile) in shared memory
+    # and give every CTA a contiguous run of tiles; forcing the same GEMM shape by hand switches that off.  Same MMAs
+    # in the same order: same bits.  Ragged K and C, runs that end inside a CTA's range, both tiles.
+    C, K, H, W, N = shape
+    layer = ConvLayer(C=C, K=K, H=H, W=W, N=N)
+    x, w, b, y_res = _run(B, layer, tile, seed=31)
+    n_auto = min(256, -(-K // 16) * 16)
+    outs = []
+    for n_tile in sorted({n_auto, 128, 64}):
+        B.sdwino_set_gemm_shape(1, n_tile)
+        try:
+            outs.append(_run(B, layer, tile, x=x, w=w, b=b)[3])
+        finally:
+            B.sdwino_set_gemm_shape(0, 0)
+    for y_str in outs:
+        assert torch.equal(y_res, y_str)
+    nch = 8
+    ks = sorted(np.random.default_rng(3).choice(K, nch, replace=False).tolist())
+    ref = oracle.direct_conv3x3(x.numpy(), w.numpy(), b.numpy(), channels=ks)
+    assert np.abs(y_res[:, ks].double().numpy() - ref).max() <= TOL * np.abs(ref).max()
