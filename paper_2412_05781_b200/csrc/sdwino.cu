@@ -663,6 +663,9 @@ int launch_gemm_shape(const CUtensorMap& tmU, const CUtensorMap& tmV, const CUte
                    static_cast<size_t>(L::dyn_bytes(RES ? 0 : prm.n_tile / CTAS, prm.stages, prm.epi_rows, prm.epi_bufs,
                                                     RES ? prm.num_c_blocks * L::b_bytes(prm.n_tile) : 0)),
                    st, CTAS, tmU, tmV, tmM, prm, status);
+    if (e != cudaSuccess && getenv("SDWINO_LOG"))
+        fprintf(stderr, "sdwino: GEMM launch failed: %s (grid %d, stages %d, n_tile %d, resident %d)\n", cudaGetErrorString(e),
+                grid, prm.stages, prm.n_tile, prm.resident);
     g_launches.fetch_add(1);
     return e == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
 }
@@ -756,31 +759,32 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
         // GEMM 146 -> 120 us, at 1024x1024 570 -> 472 us; with n_tile 128-160 (filters half of a stage or less, the
         // layer close to the HBM roof already) the pause at every change of filter block costs more than the
         // re-reads: 128->128 at 512x512 57 -> 74 us.
-        const long long p_tiles = pc / GEMM_BLOCK_P;
-        const long long tiles = p_tiles * ((K + prm.n_tile - 1) / prm.n_tile) * pl.a2;
-        const int ures = prm.num_c_blocks * GemmSmemLayout::b_bytes(prm.n_tile);
+        const long long workers = sms / shape.ctas;
+        const long long p_tiles = (pc / GEMM_BLOCK_P + shape.ctas - 1) / shape.ctas;     // tiles of 128 (256) tiles p
+        const long long keys = ((K + prm.n_tile - 1) / prm.n_tile) * static_cast<long long>(pl.a2);
+        const int ures = prm.num_c_blocks * GemmSmemLayout::b_bytes(b_rows);
         const int grp = prm.epi_rows;
         const int rows = (grp > 64 && grp % 64 == 0) ? 64 : grp;
         const int stages = (MAX_DYN_SMEM - GemmSmemLayout::dyn_bytes(0, 0, rows, prm.epi_bufs, ures)) / GemmSmemLayout::A_BYTES;
-        if (shape.ctas == 1 && g_force_ctas == 0 && g_force_n_tile == 0 && p_tiles >= 16 && tiles >= 4ll * sms &&
+        // (CTA pairs gain nothing from it: with their half of a 512-channel block resident only four 16 KB stages
+        // of V remain, too few bytes in flight: 512->512 at 256x256 99 against 94 us)
+        if (shape.ctas == 1 && g_force_ctas == 0 && g_force_n_tile == 0 && p_tiles >= 16 && keys * p_tiles >= 4 * workers &&
             prm.n_tile >= 224 && stages >= 4) {
             prm.resident = 1;
-            // CTAs per (position, k-tile) pair: as many as leave every CTA a run of at least 8 tiles (so that its
-            // filter block is re-used), the largest group among the splits of pairs over groups and of tiles over a group that
-            // are within 3 % of the most even one (the CTAs of a group read neighbouring pieces of V at the same time)
-            const long long keys = ((K + prm.n_tile - 1) / prm.n_tile) * static_cast<long long>(pl.a2);
-            auto efficiency = [&](int g) {
-                const long long ng = sms / g;
+            // CTAs per (position, k-tile) pair.  A group walks `rounds` pairs, each CTA `run` tiles per pair,
+            // and every change of pair costs about a tile and a half (the MMAs that read the old filter block drain,
+            // the new block arrives): the group size with the smallest rounds * (run + 1.5) wins, larger groups on
+            // ties (their CTAs read neighbouring pieces of V at the same time); runs of at least 8 tiles.
+            auto cost = [&](int g) {
+                const long long ng = workers / g;
                 const long long rounds = (keys + ng - 1) / ng;
                 const long long run = (p_tiles + g - 1) / g;
-                return static_cast<double>(keys * p_tiles) / (static_cast<double>(rounds) * run * sms);
+                return static_cast<double>(rounds) * (static_cast<double>(run) + 1.5);
             };
-            const int g_max = static_cast<int>(std::min<long long>(sms, p_tiles / 8));
-            double best_eff = 0.0;
-            for (int g = 1; g <= g_max; ++g) best_eff = std::max(best_eff, efficiency(g));
+            const int g_max = static_cast<int>(std::min<long long>(workers, p_tiles / 8));
             int best_g = 1;
-            for (int g = 1; g <= g_max; ++g)
-                if (efficiency(g) >= best_eff - 0.03) best_g = g;     // the largest group within 3 % of the best split
+            for (int g = 2; g <= g_max; ++g)
+                if (cost(g) <= cost(best_g) + 1e-9) best_g = g;
             prm.group = best_g;
             prm.epi_chunks = grp / rows;
             prm.epi_rows = rows;

@@ -687,6 +687,16 @@ def test_more_than_2_to_31_elements(B, tile):
                                         ((320, 320, 128, 128, 1), 4), ((192, 200, 100, 104, 2), 4), ((64, 96, 160, 160, 2), 4),
                                         ((256, 128, 256, 256, 1), 4)])
 def test_filter_resident_gemm_matches_streaming_gemm_bitwise(B, shape, tile):
+    _check_resident_against_forced_shapes(B, shape, tile, [(1, None), (1, 128), (1, 64)])
+
+
+@pytest.mark.parametrize("shape,tile", [((512, 512, 256, 256, 1), 4), ((512, 512, 128, 128, 1), 2), ((576, 500, 192, 192, 2), 4)])
+def test_automatic_gemm_shape_on_large_layers_matches_forced_shapes_bitwise(B, shape, tile):
+    # 512-channel layers with thousands of tiles (the automatic choice is CTA pairs): same bits as either shape forced
+    _check_resident_against_forced_shapes(B, shape, tile, [(2, 256), (1, 256)])
+
+
+def _check_resident_against_forced_shapes(B, shape, tile, forced):
     # Layers with few channels and thousands of tiles keep the filter block of a (position, k-tile) in shared memory
     # and give every CTA a contiguous run of tiles; forcing the same GEMM shape by hand switches that off.  Same MMAs
     # in the same order: same bits.  Ragged K and C, runs that end inside a CTA's range, both tiles.
@@ -695,8 +705,8 @@ def test_filter_resident_gemm_matches_streaming_gemm_bitwise(B, shape, tile):
     x, w, b, y_res = _run(B, layer, tile, seed=31)
     n_auto = min(256, -(-K // 16) * 16)
     outs = []
-    for n_tile in sorted({n_auto, 128, 64}):
-        B.sdwino_set_gemm_shape(1, n_tile)
+    for ctas, n_tile in forced:
+        B.sdwino_set_gemm_shape(ctas, n_auto if n_tile is None else n_tile)
         try:
             outs.append(_run(B, layer, tile, x=x, w=w, b=b)[3])
         finally:
