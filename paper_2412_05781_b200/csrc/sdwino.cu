@@ -764,7 +764,7 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
         const long long keys = ((K + prm.n_tile - 1) / prm.n_tile) * static_cast<long long>(pl.a2);
         const int ures = prm.num_c_blocks * GemmSmemLayout::b_bytes(b_rows);
         const int grp = prm.epi_rows;
-        const int rows = (grp > 64 && grp % 64 == 0) ? 64 : grp;
+        const int rows = (grp > 64 && grp % 64 == 0) ? 64 : grp;   // (32 at a time for a fifth stage measured 2-10 % slower)
         const int stages = (MAX_DYN_SMEM - GemmSmemLayout::dyn_bytes(0, 0, rows, prm.epi_bufs, ures)) / GemmSmemLayout::A_BYTES;
         // (CTA pairs gain nothing from it: with their half of a 512-channel block resident only four 16 KB stages
         // of V remain, too few bytes in flight: 512->512 at 256x256 99 against 94 us)
