@@ -467,6 +467,7 @@ int launch_output_tma(const __half* Mws, const __half* bias, __half* y, const Ti
                                         : static_cast<double>((ctas + 3ll * sms - 1) / (3ll * sms)) * 3.0 * (cand + 1.0);
         if (cost <= best_cost) { best_cost = cost; steps = cand; }
     }
+    if ((K + steps - 1) / steps > 65535) steps = (K + 65534) / 65535;   // grid limit; K <= 65535 * 16 was checked
     const size_t smem = static_cast<size_t>(OUT_TMA_STAGES) * OUT_TMA_STAGE_BYTES + 128;
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
@@ -810,8 +811,11 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
         const int count = static_cast<int>(remaining < pc ? remaining : pc);  // multiple of 128
         int rc;
         if (tile == 2) rc = launch_input<2>(xh, V, geo, C, p0, count, pc, st);
-        else if (use_input_tma(geo, N, C, x, p0, count)) rc = launch_input_tma(xh, V, geo, N, C, p0, count, pc, st);
-        else rc = launch_input<4>(xh, V, geo, C, p0, count, pc, st);
+        else {
+            rc = use_input_tma(geo, N, C, x, p0, count) ? launch_input_tma(xh, V, geo, N, C, p0, count, pc, st)
+                                                        : SDWINO_ERR_UNSUPPORTED;
+            if (rc == SDWINO_ERR_UNSUPPORTED) rc = launch_input<4>(xh, V, geo, C, p0, count, pc, st);   // grid limits
+        }
         if (rc != SDWINO_OK) return rc;
         prm.num_p_tiles = (count / GEMM_BLOCK_P + shape.ctas - 1) / shape.ctas;
         rc = launch_gemm(tmU, tmV, tmM, prm, shape.ctas, st);
