@@ -611,10 +611,10 @@ int launch_fused_small_c_mma(const __half* x, const void* wT, const __half* bias
 // pair idle, and for short launches (it runs without programmatic dependent launch, see launch_gemm_shape).  The
 // constants below reproduce that: 35 bytes per cycle per CTA of a pair (on the scale where a single CTA gets 40),
 // epilogue x 1.35 and a fixed charge for the lost overlap.
-struct GemmShape { int ctas; int n_tile; };
+struct GemmShape { int ctas; int n_tile; int dual; };   // dual: two blocks of 128 tiles per CTA tile (single CTAs)
 GemmShape choose_gemm_shape(int K, int C, long long p_tiles128, int a2, int sms, int force_ctas) {
     const long long cblocks = (C + GEMM_BLOCK_C - 1) / GEMM_BLOCK_C;
-    GemmShape best{1, 16};
+    GemmShape best{1, 16, 0};
     double best_cost = 1e300;
     // a pair needs two blocks of 128 tiles; with fewer than 8 stages per tile it measured 4-35 % slower
     const int max_ctas = p_tiles128 >= 2 && (cblocks >= 8 || force_ctas == 2) ? 2 : 1;
@@ -638,20 +638,39 @@ GemmShape choose_gemm_shape(int K, int C, long long p_tiles128, int a2, int sms,
             const double per_tile = (main > epi ? main : epi) + (ctas == 2 ? 400.0 : 200.0);
             const double fixed = ctas == 2 ? 7000.0 : 0.0;
             const double cost = waves * per_tile + epi + fixed;
-            if (cost < best_cost) { best_cost = cost; best = GemmShape{ctas, n}; }
+            if (cost < best_cost) { best_cost = cost; best = GemmShape{ctas, n, 0}; }
+        }
+    }
+    // Single CTAs with two blocks of 128 tiles per CTA tile (see wino_gemm.cuh): the filter box is fetched once per
+    // 256 tiles and there are half as many CTA tiles, but the accumulators are not double-buffered across tiles, so
+    // the epilogues of a tile are added to its mainloop.  n_tile up to 192 leaves room for three stages.
+    // Taken for layers of 2 to 15 blocks of tiles (larger ones have the filter-resident mode and CTA pairs).
+    if (force_ctas == 0 && p_tiles128 >= 2 && p_tiles128 < 16) {
+        const long long p_tiles = (p_tiles128 + 1) / 2;
+        for (int n = 16; n <= 192; n += 16) {
+            const long long ktiles = (K + n - 1) / n;
+            if (n > 16 && (ktiles == (K + n - 17) / (n - 16))) continue;
+            const long long tiles = ktiles * p_tiles * a2;
+            const long long waves = (tiles + sms - 1) / sms;
+            const double mma = 4.0 * n;
+            const double load = (2.0 * GemmSmemLayout::A_BYTES + 128.0 * n) / 40.0;
+            const double main = cblocks * (mma > load ? mma : load);
+            const double epi = 300.0 + 14.0 * n;
+            const double cost = 1.08 * waves * (main + 2.0 * epi + 200.0);   // measured gains are 5-10 %, not the modelled 20
+            if (cost < best_cost) { best_cost = cost; best = GemmShape{1, n, 1}; }
         }
     }
     return best;
 }
 
-template <int CTAS, bool RES>
+template <int CTAS, bool RES, bool DUAL = false>
 int launch_gemm_shape(const CUtensorMap& tmU, const CUtensorMap& tmV, const CUtensorMap& tmM, const GemmParams& prm,
                       int sms, int* status, cudaStream_t st) {
     using L = GemmSmemLayout;
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [&] {
-        attr_err = cudaFuncSetAttribute(wino_gemm_kernel<CTAS, RES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        attr_err = cudaFuncSetAttribute(wino_gemm_kernel<CTAS, RES, DUAL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         MAX_DYN_SMEM);
     });
     if (attr_err != cudaSuccess) return SDWINO_ERR_CUDA;
@@ -660,9 +679,10 @@ int launch_gemm_shape(const CUtensorMap& tmU, const CUtensorMap& tmV, const CUte
     const int grid = static_cast<int>(tiles < workers ? tiles : workers) * CTAS;
     ProfScope prof(KIND_GEMM, st);
     const cudaError_t e =
-        launch_pdl(wino_gemm_kernel<CTAS, RES>, dim3(grid), dim3(GEMM_THREADS),
+        launch_pdl(wino_gemm_kernel<CTAS, RES, DUAL>, dim3(grid), dim3(GEMM_THREADS),
                    static_cast<size_t>(L::dyn_bytes(RES ? 0 : prm.n_tile / CTAS, prm.stages, prm.epi_rows, prm.epi_bufs,
-                                                    RES ? prm.num_c_blocks * L::b_bytes(prm.n_tile) : 0)),
+                                                    RES ? prm.num_c_blocks * L::b_bytes(prm.n_tile)
+                                                        : (DUAL ? prm.stages * L::A_BYTES : 0))),
                    st, CTAS, tmU, tmV, tmM, prm, status);
     if (e != cudaSuccess && getenv("SDWINO_LOG"))
         fprintf(stderr, "sdwino: GEMM launch failed: %s (grid %d, stages %d, n_tile %d, resident %d)\n", cudaGetErrorString(e),
@@ -680,6 +700,7 @@ int launch_gemm(const CUtensorMap& tmU, const CUtensorMap& tmV, const CUtensorMa
         return SDWINO_ERR_CUDA;
     if (ctas == 2) return launch_gemm_shape<2, false>(tmU, tmV, tmM, prm, sms, status, st);
     if (prm.resident) return launch_gemm_shape<1, true>(tmU, tmV, tmM, prm, sms, status, st);
+    if (prm.dual) return launch_gemm_shape<1, false, true>(tmU, tmV, tmM, prm, sms, status, st);
     return launch_gemm_shape<1, false>(tmU, tmV, tmM, prm, sms, status, st);
 }
 
@@ -743,6 +764,8 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
     prm.num_c_blocks = (C + GEMM_BLOCK_C - 1) / GEMM_BLOCK_C;
     prm.C = C;
     const int b_rows = prm.n_tile / shape.ctas;
+    if (g_force_n_tile != 0) shape.dual = 0;
+    prm.dual = shape.dual;
     // epilogue staging: two groups of epilogue warps each take half a tile when that is a multiple of 16 channels
     const bool split = (prm.n_tile / 2) % 16 == 0;
     prm.epi_rows = split ? prm.n_tile / 2 : prm.n_tile;
@@ -751,7 +774,7 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
     prm.resident = 0;
     prm.group = 1;
     prm.stages = (MAX_DYN_SMEM - GemmSmemLayout::dyn_bytes(b_rows, 0, prm.epi_rows, prm.epi_bufs)) /
-                 GemmSmemLayout::stage_bytes(b_rows);
+                 (GemmSmemLayout::stage_bytes(b_rows) + (shape.dual ? GemmSmemLayout::A_BYTES : 0));
     if (prm.stages > GEMM_MAX_STAGES) prm.stages = GEMM_MAX_STAGES;
     {
         // Filter-resident mode (see wino_gemm.cuh): single CTAs, many tiles per CTA and long runs of tiles per
@@ -769,7 +792,7 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
         const int stages = (MAX_DYN_SMEM - GemmSmemLayout::dyn_bytes(0, 0, rows, prm.epi_bufs, ures)) / GemmSmemLayout::A_BYTES;
         // (CTA pairs gain nothing from it: with their half of a 512-channel block resident only four 16 KB stages
         // of V remain, too few bytes in flight: 512->512 at 256x256 99 against 94 us)
-        if (shape.ctas == 1 && g_force_ctas == 0 && g_force_n_tile == 0 && p_tiles >= 16 && keys * p_tiles >= 4 * workers &&
+        if (shape.ctas == 1 && !shape.dual && g_force_ctas == 0 && g_force_n_tile == 0 && p_tiles >= 16 && keys * p_tiles >= 4 * workers &&
             prm.n_tile >= 224 && stages >= 4) {
             prm.resident = 1;
             // CTAs per (position, k-tile) pair.  A group walks `rounds` pairs, each CTA `run` tiles per pair,
@@ -817,7 +840,8 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
             if (rc == SDWINO_ERR_UNSUPPORTED) rc = launch_input<4>(xh, V, geo, C, p0, count, pc, st);   // grid limits
         }
         if (rc != SDWINO_OK) return rc;
-        prm.num_p_tiles = (count / GEMM_BLOCK_P + shape.ctas - 1) / shape.ctas;
+        const int p_blocks = shape.ctas * (shape.dual ? 2 : 1);      // blocks of 128 tiles per CTA tile / pair tile
+        prm.num_p_tiles = (count / GEMM_BLOCK_P + p_blocks - 1) / p_blocks;
         rc = launch_gemm(tmU, tmV, tmM, prm, shape.ctas, st);
         if (rc != SDWINO_OK) return rc;
         if (tile == 2) rc = launch_output<2>(Mws, bh, yh, geo, K, p0, count, pc, chk, ep, st);

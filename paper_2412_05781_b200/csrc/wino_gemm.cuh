@@ -21,6 +21,13 @@
 // then work in groups: a group takes whole (pos, k-tile) pairs, its CTAs share out the tiles p of a pair, load the
 // pair's filter block once into a resident buffer and stream only V through the ring.
 //
+// Two blocks of tiles per CTA tile (DUAL, single CTAs): a stage holds V of 256 tiles and one filter box, every k-step
+// issues one MMA per block of 128 tiles into the two accumulator buffers, which the epilogue then drains one after
+// the other.  The filter box is fetched once per 256 instead of once per 128 tiles (like a CTA pair, but on one SM
+// and with programmatic dependent launch), and a layer of 2 j blocks of tiles makes half as many CTA tiles, which
+// turns two waves into one where the tiles number about twice the SMs.  The accumulators are no longer
+// double-buffered across tiles, so this pays where a CTA has one or two tiles or many stages per tile.
+//
 // One persistent CTA (pair) per SM (pair) walks the list of (pos, k-tile, p-tile) output tiles.
 //   warp 0   : TMA producer        (one lane)
 //   warp 1   : TMEM owner + MMA issuer (one lane)
@@ -86,6 +93,7 @@ struct GemmParams {
     int resident;      // 1: the filter blocks of a (position, k-tile) stay in shared memory while the CTA walks the
                        // tiles p of that pair (stages then hold V only)
     int group;         // filter-resident mode: CTAs that share out the tiles of one (position, k-tile) pair
+    int dual;          // 1: the kernel instantiation with two blocks of 128 tiles per CTA tile (host side only)
     long long p_stride;  // tiles per pass (row pitch of V and M)
 };
 
@@ -93,8 +101,9 @@ struct GemmParams {
 // tmU: fp16 [pos][Cb][Kb][16][64] box {64 c, 16 k, 1, n_tile/16, 1}, 128B swizzle (B operand: n_tile rows of 128
 //      bytes in k order; blocks past Kb read as 0)
 // tmM: fp16 [pos][K][Pstride]   box {128 p, epi_rows k, 1}, no swizzle  (result; rows k >= K are clipped)
-// RES: the filter-resident mode as a separate instantiation, so that the streaming kernel pays nothing for it.
-template <int CTAS, bool RES = false>
+// RES: the filter-resident mode, DUAL: two blocks of 128 tiles per CTA tile; separate instantiations, so that the
+// plain streaming kernel pays nothing for them.
+template <int CTAS, bool RES = false, bool DUAL = false>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant__ CUtensorMap tmV,
                  const __grid_constant__ CUtensorMap tmM, const GemmParams prm, int* __restrict__ status_word) {
@@ -106,8 +115,11 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int b_rows = prm.n_tile / CTAS;            // rows of U this CTA loads per stage
     static_assert(!RES || CTAS == 1, "filter-resident mode is for single CTAs");
+    static_assert(!DUAL || (CTAS == 1 && !RES), "two blocks of tiles per CTA: single CTAs, streaming mode");
     constexpr bool resident = RES;
-    const int stage_bytes = resident ? L::A_BYTES : L::stage_bytes(b_rows);
+    constexpr int PT = DUAL ? 2 : 1;                 // blocks of 128 tiles p per CTA tile (one accumulator each)
+    constexpr int a_bytes = PT * L::A_BYTES;         // V part of a stage
+    const int stage_bytes = resident ? L::A_BYTES : (PT - 1) * L::A_BYTES + L::stage_bytes(b_rows);
     const int ures_cb_bytes = L::b_bytes(prm.n_tile);                       // one 64-channel block of the resident filters
     const int ures_bytes = resident ? prm.num_c_blocks * ures_cb_bytes : 0;
     const int stages = prm.stages;
@@ -245,7 +257,7 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
             if (!ok) *abort_flag = 1;
         } else if (!resident && lane == 0) {
             // the full barrier of a pair lives in the leader and counts the bytes of both CTAs
-            const uint32_t tx_bytes = CTAS * (L::A_BYTES + L::b_bytes(b_rows));
+            const uint32_t tx_bytes = CTAS * (a_bytes + L::b_bytes(b_rows));
             // single-thread loop: shared-memory and barrier addresses are running 32-bit values
             const uint32_t smem_base = smem_u32(smem);
             const uint32_t full0_local = smem_u32(&full_bar[0]);
@@ -258,7 +270,7 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
             const uint64_t u_policy = l2_policy_evict_first();
             int pre = 0;
             if constexpr (CTAS == 1) {
-                uint32_t sa_u = smem_base + L::A_BYTES, fb_u = full0;
+                uint32_t sa_u = smem_base + a_bytes, fb_u = full0;
                 for (int i = 0; i < my_count && pre < stages; ++i) {
                     const int tile = tile_of(i);
                     const int kt = (tile / prm.num_p_tiles) % prm.num_k_tiles;
@@ -283,13 +295,16 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
                 const int pt = tile % prm.num_p_tiles;
                 const int kt = (tile / prm.num_p_tiles) % prm.num_k_tiles;
                 const int pos = tile / (prm.num_p_tiles * prm.num_k_tiles);
-                const int p0 = (pt * CTAS + static_cast<int>(cta_rank)) * GEMM_BLOCK_P;
+                const int p0 = (pt * CTAS * PT + static_cast<int>(cta_rank)) * GEMM_BLOCK_P;
                 const int k0 = kt * prm.n_tile + static_cast<int>(cta_rank) * b_rows;
                 for (int c0 = 0; c0 < prm.C; c0 += GEMM_BLOCK_C) {
                     if (issued < pre) {
-                        // the barrier is armed and the filter box is on its way: add the two boxes of V
-                        tma_load_3d_a32(sa, &tmV, fb, p0, c0, pos);
-                        tma_load_3d_a32(sa + L::A_BOX_BYTES, &tmV, fb, p0 + 64, c0, pos);
+                        // the barrier is armed and the filter box is on its way: add the boxes of V
+#pragma unroll
+                        for (int sub = 0; sub < PT; ++sub) {
+                            tma_load_3d_a32(sa + sub * L::A_BYTES, &tmV, fb, p0 + sub * GEMM_BLOCK_P, c0, pos);
+                            tma_load_3d_a32(sa + sub * L::A_BYTES + L::A_BOX_BYTES, &tmV, fb, p0 + sub * GEMM_BLOCK_P + 64, c0, pos);
+                        }
                         ++issued;
                         sa += stage_bytes;
                         fb += 8;
@@ -306,9 +321,12 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
                         tma_load_5d_pair(sa + L::A_BYTES, &tmU, fb, c0 >> 6, k0 >> 4, pos);
                     } else {
                         mbar_arrive_expect_tx_a32(fb, tx_bytes);
-                        tma_load_3d_a32(sa, &tmV, fb, p0, c0, pos);
-                        tma_load_3d_a32(sa + L::A_BOX_BYTES, &tmV, fb, p0 + 64, c0, pos);
-                        tma_load_5d_hint_a32(sa + L::A_BYTES, &tmU, fb, c0 >> 6, k0 >> 4, pos, u_policy);
+#pragma unroll
+                        for (int sub = 0; sub < PT; ++sub) {
+                            tma_load_3d_a32(sa + sub * L::A_BYTES, &tmV, fb, p0 + sub * GEMM_BLOCK_P, c0, pos);
+                            tma_load_3d_a32(sa + sub * L::A_BYTES + L::A_BOX_BYTES, &tmV, fb, p0 + sub * GEMM_BLOCK_P + 64, c0, pos);
+                        }
+                        tma_load_5d_hint_a32(sa + a_bytes, &tmU, fb, c0 >> 6, k0 >> 4, pos, u_policy);
                     }
                     sa += stage_bytes;
                     fb += 8;
@@ -329,7 +347,7 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
             //   A_BOX_BYTES apart.  B (K-major): 16 channels = +32 bytes along the swizzled 128-byte row.
             const uint32_t smem_base = smem_u32(smem);
             const uint64_t adesc0 = make_smem_desc_sw128(smem_base, L::A_BOX_BYTES, 1024);
-            const uint64_t bdesc0 = make_smem_desc_sw128(smem_base + L::A_BYTES, 16, 1024);
+            const uint64_t bdesc0 = make_smem_desc_sw128(smem_base + a_bytes, 16, 1024);
             const uint64_t stage_step = static_cast<uint64_t>(stage_bytes >> 4);
             const uint64_t ures_desc0 = make_smem_desc_sw128(smem_u32(ures_base), 16, 1024);
             const uint64_t ures_step = static_cast<uint64_t>(ures_cb_bytes >> 4);
@@ -358,9 +376,14 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
                     }
                 }
                 ok = mbar_wait_bounded(&acc_empty_bar[buf], acc_phase ^ 1u, abort_flag, GEMM_WAIT_LIMIT_NS);
+                if constexpr (DUAL) {   // this tile fills both accumulator buffers
+                    if (ok) ok = mbar_wait_bounded(&acc_empty_bar[1], acc_phase ^ 1u, abort_flag, GEMM_WAIT_LIMIT_NS);
+                }
                 if (!ok) { if (*abort_flag == 0) report_timeout(status_word, 2, cta_rank); break; }
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(buf * GEMM_MAX_N);
+                [[maybe_unused]] const uint32_t d_tmem1 = tmem_base + static_cast<uint32_t>(GEMM_MAX_N);
+                [[maybe_unused]] constexpr uint64_t a_sub = static_cast<uint64_t>(L::A_BYTES >> 4);   // second block of tiles
                 for (int cb = 0; cb < prm.num_c_blocks; ++cb) {
                     if (!mbar_try_wait_a32(full_a, phase)) {
                         ok = mbar_wait_slow(&full_bar[stage], phase, abort_flag, GEMM_WAIT_LIMIT_NS);
@@ -379,6 +402,12 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
                             umma_f16_acc(d_tmem, adesc + 128, bd + 2, idesc);
                             umma_f16_acc(d_tmem, adesc + 256, bd + 4, idesc);
                             umma_f16_acc(d_tmem, adesc + 384, bd + 6, idesc);
+                            if constexpr (DUAL) {
+                                umma_f16(d_tmem1, adesc + a_sub, bd, idesc, static_cast<uint32_t>(cb));
+                                umma_f16_acc(d_tmem1, adesc + a_sub + 128, bd + 2, idesc);
+                                umma_f16_acc(d_tmem1, adesc + a_sub + 256, bd + 4, idesc);
+                                umma_f16_acc(d_tmem1, adesc + a_sub + 384, bd + 6, idesc);
+                            }
                         }
                     } else {
                         for (int s = 0; s < last_ksteps; ++s) {
@@ -386,6 +415,8 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
                                 umma_f16_pair(d_tmem, adesc + 128 * s, bdesc + 2 * s, idesc, (cb > 0 || s > 0) ? 1u : 0u);
                             else
                                 umma_f16(d_tmem, adesc + 128 * s, bd + 2 * s, idesc, (cb > 0 || s > 0) ? 1u : 0u);
+                            if constexpr (DUAL)
+                                umma_f16(d_tmem1, adesc + a_sub + 128 * s, bd + 2 * s, idesc, (cb > 0 || s > 0) ? 1u : 0u);
                         }
                     }
                     if constexpr (CTAS == 2) umma_commit_pair_a32(empty_a);
@@ -401,10 +432,15 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
                 if (!ok) break;
                 if constexpr (CTAS == 2) umma_commit_pair(&acc_full_bar[buf]);
                 else umma_commit(&acc_full_bar[buf]);
+                if constexpr (DUAL) umma_commit(&acc_full_bar[1]);
                 // the last tile of a run: once its MMAs have completed the resident filters may be replaced
                 if (resident && i + 1 < my_count && tile_of(i + 1) / prm.num_p_tiles != key) umma_commit(ures_empty_bar);
-                buf ^= 1;
-                if (buf == 0) acc_phase ^= 1u;
+                if constexpr (DUAL) {
+                    acc_phase ^= 1u;          // both buffers were used: buf stays 0
+                } else {
+                    buf ^= 1;
+                    if (buf == 0) acc_phase ^= 1u;
+                }
             }
             if (!ok) *abort_flag = 1;
         }
@@ -418,9 +454,11 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
         uint32_t acc_phase = 0;
         // the accumulator-empty barrier of a pair lives in the leader
         const uint32_t acc_empty_addr0 = CTAS == 2 ? map_to_cta(smem_u32(&acc_empty_bar[0]), 0) : 0u;
-        for (int i = 0; i < my_count; ++i) {
-            const int tile = tile_of(i);
-            const int pt = tile % prm.num_p_tiles;
+        // one iteration per accumulator: a tile of two blocks of 128 tiles p (DUAL) fills both buffers, which are
+        // drained in turn exactly as two consecutive tiles would be
+        for (int i2 = 0; i2 < my_count * PT; ++i2) {
+            const int tile = tile_of(i2 / PT);
+            const int pt = (tile % prm.num_p_tiles) * PT + (i2 % PT);
             const int kt = (tile / prm.num_p_tiles) % prm.num_k_tiles;
             const int pos = tile / (prm.num_p_tiles * prm.num_k_tiles);
             bool ok = mbar_wait_bounded(&acc_full_bar[buf], acc_phase, abort_flag, GEMM_WAIT_LIMIT_NS);

@@ -696,6 +696,14 @@ def test_automatic_gemm_shape_on_large_layers_matches_forced_shapes_bitwise(B, s
     _check_resident_against_forced_shapes(B, shape, tile, [(2, 256), (1, 256)])
 
 
+@pytest.mark.parametrize("shape,tile", [((960, 320, 64, 64, 2), 4), ((640, 640, 48, 48, 1), 4), ((320, 320, 96, 96, 1), 4),
+                                        ((200, 150, 40, 48, 3), 2), ((640, 320, 40, 40, 1), 4)])
+def test_two_blocks_of_tiles_per_cta_match_forced_shapes_bitwise(B, shape, tile):
+    # layers of 2 to 15 blocks of 128 tiles: a CTA tile covers two blocks (two accumulators, one filter box per
+    # stage); an odd number of blocks leaves the last tile half empty.  Forcing a shape switches that off.
+    _check_resident_against_forced_shapes(B, shape, tile, [(1, None), (1, 64)])
+
+
 def _check_resident_against_forced_shapes(B, shape, tile, forced):
     # Layers with few channels and thousands of tiles keep the filter block of a (position, k-tile) in shared memory
     # and give every CTA a contiguous run of tiles; forcing the same GEMM shape by hand switches that off.  Same MMAs
