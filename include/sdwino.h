@@ -186,9 +186,10 @@ unsigned long long sdwino_launch_count(void);
 
 /*
  * Tuning and test hook for the batched GEMM of step (ii).  By default the library picks, per
- * call, between single-CTA tiles (128 tiles x n output channels) and CTA-pair tiles (256 tiles x
+ * call, between single-CTA tiles (128 tiles x n output channels; also with two blocks of 128 tiles per
+ * CTA tile, or with the filter block of a position resident in shared memory) and CTA-pair tiles (256 tiles x
  * n output channels, tcgen05 cta_group::2; n is then rounded up to a multiple of 32) and the n that
- * fits the layer.  ctas in {1, 2} and/or
+ * fits the layer.  Forcing either field selects the plain kernel of that shape.  ctas in {1, 2} and/or
  * n_tile (a multiple of 16 in [16, 256]) force that choice for later calls of this process; 0
  * restores the automatic choice for that field.  Results do not depend on the choice beyond
  * the fp32 summation order inside the tensor core.  Returns SDWINO_ERR_INVALID_ARG otherwise.
