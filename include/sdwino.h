@@ -63,7 +63,7 @@ int sdwino_filter_transform(const void *w, void *wT, int K, int C, int tile, voi
 /*
  * Scratch for the transformed activation V and the per-position products M (steps (i)
  * and (ii)).  sdwino_workspace_bytes returns the size that lets the call run in one pass
- * over the tile list, capped at 1 GiB (0 on bad arguments); any workspace of at least
+ * over the tile list, capped at 4 GiB (0 on bad arguments); any workspace of at least
  * sdwino_workspace_min_bytes is accepted and only changes how many passes are made (fewer,
  * longer passes are faster).  The workspace is caller-owned,
  * must be 1024-byte aligned, is overwritten by every call, and may be shared by calls

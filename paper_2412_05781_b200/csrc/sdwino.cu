@@ -78,7 +78,7 @@ constexpr int MAX_DYN_SMEM = 232448;  // 227 KB opt-in limit per CTA on sm_100
 // the first design; with the filter stream marked evict-first, one long pass that streams V and M through HBM
 // beats many short L2-resident ones, whose kernels are mostly ramp and tail (512->512 at 256x256, F4: 236 us
 // with 64 MB passes, 216 us with 128 MB, 202 us in a single pass).  The cap only bounds the memory asked for.
-constexpr size_t PASS_BUDGET = 1024ull << 20;
+constexpr size_t PASS_BUDGET = 4096ull << 20;
 constexpr size_t WS_ALIGN = 1024;
 constexpr int STATIC_MAX_DEVICES_HOST = 64;
 
