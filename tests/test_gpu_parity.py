@@ -725,3 +725,54 @@ def _check_resident_against_forced_shapes(B, shape, tile, forced):
     ks = sorted(np.random.default_rng(3).choice(K, nch, replace=False).tolist())
     ref = oracle.direct_conv3x3(x.numpy(), w.numpy(), b.numpy(), channels=ks)
     assert np.abs(y_res[:, ks].double().numpy() - ref).max() <= TOL * np.abs(ref).max()
+
+
+def _random_large_shapes(count, seed):
+    rng = np.random.default_rng(seed)
+    shapes = []
+    while len(shapes) < count:
+        W = int(rng.choice([8, 16, 24, 32, 40, 48, 64, 64, 96, 128, 128, 192, 256, 320, 512]))
+        H = int(rng.choice([W, max(1, W // 2), W + int(rng.integers(0, 9)), int(rng.integers(1, 70))]))
+        C = int(rng.choice([9, 16, 40, 64, 96, 128, 192, 200, 256, 256, 320, 384, 512, 640]))
+        K = int(rng.choice([9, 16, 48, 64, 100, 128, 160, 200, 256, 256, 320, 512, 640]))
+        N = int(rng.choice([1, 1, 2, 3]))
+        tile = int(rng.choice([2, 4, 4]))
+        if N * C * H * W > 1.5e8 or N * K * H * W > 1.5e8 or 2.0 * N * K * C * H * W * 9 > 1.5e12:
+            continue
+        shapes.append((C, K, H, W, N, tile))
+    return shapes
+
+
+@pytest.mark.parametrize("shape", _random_large_shapes(40, seed=5781))
+def test_seeded_random_layers_against_plain_kernels_and_oracle(B, shape):
+    # A seeded draw over layer sizes up to a few hundred MB: whatever the dispatcher picks (staged transforms, CTA
+    # pairs, two blocks of tiles per CTA tile, resident filters, one pass) must give the bits of the plain kernels
+    # (register-only transforms, single-CTA streaming GEMM of a forced shape), also when the layer is cut into
+    # about three passes with staging forced on, and must agree with the oracle on sampled channels.
+    C, K, H, W, N, tile = shape
+    layer = ConvLayer(C=C, K=K, H=H, W=W, N=N)
+    rng = np.random.default_rng(sum(shape))
+    x, w, b = workloads.make_inputs(layer, seed=sum(shape))
+    xd, bd = x.cuda(), b.cuda()
+    wT = B.sdwino_filter_transform(w.cuda(), tile)
+    ws = B.alloc_workspace(B.sdwino_workspace_bytes(N, C, H, W, K, tile))
+    y_auto = B.sdwino_conv3x3(xd, wT, bd, K, tile, workspace=ws)
+    assert B.sdwino_last_device_status() == B.OK
+    n_auto = min(256, -(-K // 16) * 16)
+    B.sdwino_set_input_staging(0)
+    B.sdwino_set_gemm_shape(1, int(rng.choice([n_auto, 64, 16])))
+    try:
+        y_plain = B.sdwino_conv3x3(xd, wT, bd, K, tile, workspace=ws)
+    finally:
+        B.sdwino_set_gemm_shape(0, 0)
+        B.sdwino_set_input_staging(1)
+    B.sdwino_set_input_staging(2)
+    try:
+        small = max(B.sdwino_workspace_min_bytes(N, C, H, W, K, tile) * 3, B.sdwino_workspace_bytes(N, C, H, W, K, tile) // 3)
+        y_cut = B.sdwino_conv3x3(xd, wT, bd, K, tile, workspace=B.alloc_workspace(small))
+    finally:
+        B.sdwino_set_input_staging(1)
+    assert torch.equal(y_auto, y_plain) and torch.equal(y_auto, y_cut)
+    ks = sorted(rng.choice(K, min(K, 4), replace=False).tolist())
+    ref = oracle.direct_conv3x3(x.numpy(), w.numpy(), b.numpy(), channels=ks)
+    assert np.abs(y_auto[:, ks].cpu().double().numpy() - ref).max() <= TOL * np.abs(ref).max()
