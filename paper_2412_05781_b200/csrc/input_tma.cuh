@@ -144,7 +144,7 @@ input_transform_f4_tma_kernel(const __grid_constant__ CUtensorMap tmX, __half* _
         // every thread has read the stage (or nobody uses it): it can be refilled
         if (!__syncthreads_and(ok)) {
             if (tid == 0 && abort_flag == 0) {
-                atomicCAS(status_word, 0, 6 | (5 << 8));   // 6 = timeout, where = 5: the input staging
+                atomicCAS(status_word, 0, 6 | (10 << 8));   // 6 = timeout, where = 10: the input staging
                 abort_flag = 1;
             }
             break;

@@ -90,7 +90,7 @@ output_transform_f4_tma_kernel(const __grid_constant__ CUtensorMap tmM, const __
         }
         if (!__syncthreads_and(ok)) {
             if (tid == 0 && abort_flag == 0) {
-                atomicCAS(status_word, 0, 6 | (8 << 8));   // 6 = timeout, where = 8: the staging of M
+                atomicCAS(status_word, 0, 6 | (11 << 8));   // 6 = timeout, where = 11: the staging of M
                 abort_flag = 1;
             }
             break;

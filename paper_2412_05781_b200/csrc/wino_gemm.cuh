@@ -9,7 +9,7 @@
 // TMEM columns hold n_tile output channels k (operand B = U, K-major), n_tile any multiple of
 // 16 up to 256, so that channel counts such as 320 = 2 x 160 waste nothing.
 //
-// Two launch shapes share the code.  CTAS == 1: one persistent CTA per SM, 128 p x n_tile k per
+// The instantiations share the code.  CTAS == 1: one persistent CTA per SM, 128 p x n_tile k per
 // tile.  CTAS == 2: persistent CTA pairs (a 2-CTA cluster) drive one 256-row MMA (cta_group::2);
 // each CTA loads its own 128 p rows of V but only half of the n_tile rows of U, which cuts the
 // bytes fetched from L2 per MMA cycle -- the measured limit of the single-CTA shape.  The leader
