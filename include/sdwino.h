@@ -18,6 +18,10 @@
  * The library never allocates device memory except where a function says so, keeps no
  * reference to caller buffers after a call except the registered workspace, and has no
  * CPU fallback: without a CUDA device every compute call returns SDWINO_ERR_CUDA.
+ * Every call works on the calling thread's current CUDA device (cudaSetDevice); what the library keeps per
+ * device (SM count, status word, kernel attributes, copy streams of the host path, the built-in scratch of
+ * sdwino_conv3x3_static) is set up on first use there, for up to 64 devices per process.  The workspace
+ * registered with sdwino_set_workspace and the test hooks are per process.
  */
 #ifndef SDWINO_H
 #define SDWINO_H

@@ -217,21 +217,50 @@ bool encode_filter_map(CUtensorMap* m, const void* base, uint64_t Cb, uint64_t K
     return true;
 }
 
-int sm_count() {
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess) return 0;
-        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n = 0;
-    }
-    return n;
+// Per-device facts, looked up once per device (a process may drive several GPUs: everything that belongs to a
+// device -- the SM count, the address of the status word, the shared-memory limit of a kernel -- is kept per device).
+int current_device() {
+    int dev = -1;
+    return (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < STATIC_MAX_DEVICES_HOST) ? dev : -1;
 }
 
-// Device address of the status word (one device per process is the common case; looked up once).
+int sm_count() {
+    static std::atomic<int> n[STATIC_MAX_DEVICES_HOST];
+    const int dev = current_device();
+    if (dev < 0) return 0;
+    int v = n[dev].load(std::memory_order_relaxed);
+    if (v == 0) {
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) v = 0;
+        n[dev].store(v, std::memory_order_relaxed);
+    }
+    return v;
+}
+
+// Device address of the status word on the current device.
 int* status_word_ptr() {
-    static int* status = nullptr;
-    if (!status && cudaGetSymbolAddress(reinterpret_cast<void**>(&status), g_status_word) != cudaSuccess) status = nullptr;
-    return status;
+    static std::atomic<int*> ptr[STATIC_MAX_DEVICES_HOST];
+    const int dev = current_device();
+    if (dev < 0) return nullptr;
+    int* v = ptr[dev].load(std::memory_order_relaxed);
+    if (!v) {
+        if (cudaGetSymbolAddress(reinterpret_cast<void**>(&v), g_status_word) != cudaSuccess) v = nullptr;
+        ptr[dev].store(v, std::memory_order_relaxed);
+    }
+    return v;
+}
+
+// Raises the dynamic shared-memory limit of a kernel, once per kernel and device.
+bool ensure_dyn_smem(const void* kernel, int bytes) {
+    static std::mutex mutex;
+    static std::vector<std::pair<const void*, int>> done;
+    const int dev = current_device();
+    if (dev < 0) return false;
+    std::lock_guard<std::mutex> lock(mutex);
+    for (const auto& e : done)
+        if (e.first == kernel && e.second == dev) return true;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return false;
+    done.emplace_back(kernel, dev);
+    return true;
 }
 inline const uint32_t* wt_header_of(const void* wT) { return static_cast<const uint32_t*>(wT); }
 inline const void* wt_filters_of(const void* wT) { return static_cast<const uint8_t*>(wT) + WT_HEADER_BYTES; }
@@ -423,13 +452,9 @@ int launch_input_tma(const __half* x, __half* V, const TileGeom& geo, int N, int
     CUtensorMap tmX;
     if (!encode_image_map(&tmX, x, geo.W, geo.H, static_cast<uint64_t>(N) * C, q.bw, q.bh, q.cpb)) return SDWINO_ERR_CUDA;
     const size_t smem = static_cast<size_t>(IN_TMA_STAGES) * q.stage_bytes + 128;
-    static std::once_flag once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(once, [&] {
-        attr_err = cudaFuncSetAttribute(input_transform_f4_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        IN_TMA_STAGES * 32 * 1024 + 128);
-    });
-    if (attr_err != cudaSuccess || smem > IN_TMA_STAGES * 32 * 1024 + 128) return SDWINO_ERR_CUDA;
+    if (smem > IN_TMA_STAGES * 32 * 1024 + 128 ||
+        !ensure_dyn_smem(reinterpret_cast<const void*>(input_transform_f4_tma_kernel), IN_TMA_STAGES * 32 * 1024 + 128))
+        return SDWINO_ERR_CUDA;
     dim3 grid(static_cast<unsigned>(blocks), static_cast<unsigned>(grid_y));
     const cudaError_t e = launch_pdl(input_transform_f4_tma_kernel, grid, dim3(IN_TMA_THREADS), smem, st, 0, tmX, V, q,
                                      status);
@@ -469,16 +494,10 @@ int launch_output_tma(const __half* Mws, const __half* bias, __half* y, const Ti
     }
     if ((K + steps - 1) / steps > 65535) steps = (K + 65534) / 65535;   // grid limit; K <= 65535 * 16 was checked
     const size_t smem = static_cast<size_t>(OUT_TMA_STAGES) * OUT_TMA_STAGE_BYTES + 128;
-    static std::once_flag once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(once, [&] {
-        attr_err = cudaFuncSetAttribute(output_transform_f4_tma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        static_cast<int>(smem));
-        if (attr_err == cudaSuccess)
-            attr_err = cudaFuncSetAttribute(output_transform_f4_tma_kernel<true>,
-                                            cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-    });
-    if (attr_err != cudaSuccess || blocks >= (1ll << 31)) return SDWINO_ERR_CUDA;
+    if (blocks >= (1ll << 31) ||
+        !ensure_dyn_smem(reinterpret_cast<const void*>(output_transform_f4_tma_kernel<false>), static_cast<int>(smem)) ||
+        !ensure_dyn_smem(reinterpret_cast<const void*>(output_transform_f4_tma_kernel<true>), static_cast<int>(smem)))
+        return SDWINO_ERR_CUDA;
     dim3 grid(static_cast<unsigned>(blocks), static_cast<unsigned>((K + steps - 1) / steps));
     cudaError_t e;
     if (ep.residual == nullptr && ep.act == 0)
@@ -547,15 +566,8 @@ int launch_fused_small_k(const __half* x, const void* wT, const __half* bias, __
                          int W, int K, cudaStream_t st) {
     const int sms = sm_count();
     if (sms <= 0) return SDWINO_ERR_CUDA;
-    static int* status = nullptr;
-    if (!status && cudaGetSymbolAddress(reinterpret_cast<void**>(&status), g_status_word) != cudaSuccess)
-        return SDWINO_ERR_CUDA;
-    static std::once_flag once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(once, [&] {
-        attr_err = cudaFuncSetAttribute(fused_small_k_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FK_DYN_SMEM);
-    });
-    if (attr_err != cudaSuccess) return SDWINO_ERR_CUDA;
+    int* status = status_word_ptr();
+    if (!status || !ensure_dyn_smem(reinterpret_cast<const void*>(fused_small_k_kernel), FK_DYN_SMEM)) return SDWINO_ERR_CUDA;
     CUtensorMap tmU;
     if (!encode_filter_map(&tmU, wt_filters_of(wT), pl.Cb, pl.Kb, pl.a2, 1, 16, FK_KMAX)) return SDWINO_ERR_CUDA;
     FusedKParams prm;
@@ -667,13 +679,7 @@ template <int CTAS, bool RES, bool DUAL = false>
 int launch_gemm_shape(const CUtensorMap& tmU, const CUtensorMap& tmV, const CUtensorMap& tmM, const GemmParams& prm,
                       int sms, int* status, cudaStream_t st) {
     using L = GemmSmemLayout;
-    static std::once_flag once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(once, [&] {
-        attr_err = cudaFuncSetAttribute(wino_gemm_kernel<CTAS, RES, DUAL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        MAX_DYN_SMEM);
-    });
-    if (attr_err != cudaSuccess) return SDWINO_ERR_CUDA;
+    if (!ensure_dyn_smem(reinterpret_cast<const void*>(wino_gemm_kernel<CTAS, RES, DUAL>), MAX_DYN_SMEM)) return SDWINO_ERR_CUDA;
     const long long tiles = static_cast<long long>(prm.num_k_tiles) * prm.num_p_tiles * prm.num_pos;
     const long long workers = sms / CTAS;
     const int grid = static_cast<int>(tiles < workers ? tiles : workers) * CTAS;
@@ -695,9 +701,8 @@ int launch_gemm(const CUtensorMap& tmU, const CUtensorMap& tmV, const CUtensorMa
                 int ctas, cudaStream_t st) {
     const int sms = sm_count();
     if (sms <= 0) return SDWINO_ERR_CUDA;
-    static int* status = nullptr;   // device address of the status word (one device per process)
-    if (!status && cudaGetSymbolAddress(reinterpret_cast<void**>(&status), g_status_word) != cudaSuccess)
-        return SDWINO_ERR_CUDA;
+    int* status = status_word_ptr();
+    if (!status) return SDWINO_ERR_CUDA;
     if (ctas == 2) return launch_gemm_shape<2, false>(tmU, tmV, tmM, prm, sms, status, st);
     if (prm.resident) return launch_gemm_shape<1, true>(tmU, tmV, tmM, prm, sms, status, st);
     if (prm.dual) return launch_gemm_shape<1, false, true>(tmU, tmV, tmM, prm, sms, status, st);
