@@ -78,6 +78,16 @@ def test_argument_validation_without_gpu(binding):
     assert lib.sdwino_set_workspace(p + 4, 64) == binding.ERR_MISALIGNED
     assert lib.sdwino_conv3x3_host(None, p, None, p, 1, 4, 8, 8, 4, 2, p, 1 << 20, None) == binding.ERR_INVALID_ARG
     assert lib.sdwino_conv3x3_host(p, p, None, p, 1, 4, 8, 8, 4, 2, p, 1024, None) == binding.ERR_WORKSPACE
+    # fused epilogue: unknown activation, odd residual pointer, then the checks of the plain call
+    assert lib.sdwino_conv3x3_ex(p, p, None, None, p, 1, 4, 8, 8, 4, 2, 7, p, 1 << 20, None) == binding.ERR_UNSUPPORTED
+    assert lib.sdwino_conv3x3_ex(p, p, None, p + 1, p, 1, 4, 8, 8, 4, 2, 1, p, 1 << 20, None) == binding.ERR_MISALIGNED
+    assert lib.sdwino_conv3x3_ex(None, p, None, None, p, 1, 4, 8, 8, 4, 2, 1, p, 1 << 20, None) == binding.ERR_INVALID_ARG
+    assert lib.sdwino_conv3x3_ex(p, p, None, None, p, 1, 4, 8, 8, 4, 2, 0, None, 0, None) == binding.ERR_WORKSPACE
+    # test hooks reject values outside their range and accept the defaults
+    assert lib.sdwino_set_input_staging(3) == binding.ERR_INVALID_ARG
+    assert lib.sdwino_set_input_staging(-1) == binding.ERR_INVALID_ARG
+    assert lib.sdwino_set_input_staging(1) == binding.OK
+    assert lib.sdwino_set_gemm_shape(0, 0) == binding.OK
 
 
 def test_missing_library_fails_loudly(monkeypatch, binding):
