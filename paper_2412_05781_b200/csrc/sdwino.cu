@@ -323,7 +323,7 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
 
 template <int M>
 int launch_filter(const __half* w, void* wT, int K, int C, int Kb, int Cb, cudaStream_t st) {
-    dim3 grid((Cb * 64 + 127) / 128, Kb * 16);
+    dim3 grid((Cb * 32 + 127) / 128, Kb * 16);   // a thread transforms two neighbouring input channels
     ProfScope prof(KIND_FILTER, st);
     uint32_t* header = static_cast<uint32_t*>(wT);
     __half* U = reinterpret_cast<__half*>(static_cast<uint8_t*>(wT) + WT_HEADER_BYTES);
