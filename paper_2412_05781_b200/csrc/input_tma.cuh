@@ -79,21 +79,6 @@ input_transform_f4_tma_kernel(const __grid_constant__ CUtensorMap tmX, __half* _
         prefetch_tmap(&tmX);
     }
     __syncthreads();
-    pdl_wait();                 // x may be the output of the preceding kernel: wait first, release the GEMM second
-    pdl_launch_dependents();
-
-    const int x0 = 4 * tw0 - 8, y0 = 4 * th0 - 1;
-    const uint32_t tx_bytes = static_cast<uint32_t>(prm.bw) * prm.bh * prm.cpb * 2u * prm.nb;
-    if (tid == 0) {
-        const int pre = steps < IN_TMA_STAGES ? steps : IN_TMA_STAGES;
-        for (int s = 0; s < pre; ++s) {
-            mbar_arrive_expect_tx(&full_bar[s], tx_bytes);
-            for (int sub = 0; sub < prm.nb; ++sub)
-                tma_load_3d(smem + s * prm.stage_bytes + sub * prm.box_bytes, &tmX, &full_bar[s], x0 + sub * 4 * tcb, y0,
-                            n * prm.C + c_first + s * prm.cpb);
-        }
-    }
-
     // thread -> (channel within the step, tile row within the block, pair of tiles within the row)
     const int row_threads = prm.tcb_half * prm.nb;
     const int rest = tid / row_threads;
@@ -111,6 +96,22 @@ input_transform_f4_tma_kernel(const __grid_constant__ CUtensorMap tmX, __half* _
     // first of the six window rows of this thread inside a stage; the 16-byte segment starts at column 8 j + 8
     const uint32_t win = sub * prm.box_bytes + (static_cast<uint32_t>(cl * prm.bh + 4 * r) * prm.bw + 8 * j + 8) * 2u;
     const uint32_t row_pitch = static_cast<uint32_t>(prm.bw) * 2u;
+
+    // the index arithmetic above runs while the preceding kernel drains
+    pdl_wait();                 // x may be the output of the preceding kernel: wait first, release the GEMM second
+    pdl_launch_dependents();
+
+    const int x0 = 4 * tw0 - 8, y0 = 4 * th0 - 1;
+    const uint32_t tx_bytes = static_cast<uint32_t>(prm.bw) * prm.bh * prm.cpb * 2u * prm.nb;
+    if (tid == 0) {
+        const int pre = steps < IN_TMA_STAGES ? steps : IN_TMA_STAGES;
+        for (int s = 0; s < pre; ++s) {
+            mbar_arrive_expect_tx(&full_bar[s], tx_bytes);
+            for (int bx = 0; bx < prm.nb; ++bx)
+                tma_load_3d(smem + s * prm.stage_bytes + bx * prm.box_bytes, &tmX, &full_bar[s], x0 + bx * 4 * tcb, y0,
+                            n * prm.C + c_first + s * prm.cpb);
+        }
+    }
 
     for (int it = 0; it < steps; ++it) {
         const int s = it % IN_TMA_STAGES;
@@ -151,8 +152,8 @@ input_transform_f4_tma_kernel(const __grid_constant__ CUtensorMap tmX, __half* _
         }
         if (tid == 0 && it + IN_TMA_STAGES < steps) {
             mbar_arrive_expect_tx(&full_bar[s], tx_bytes);
-            for (int sub = 0; sub < prm.nb; ++sub)
-                tma_load_3d(smem + s * prm.stage_bytes + sub * prm.box_bytes, &tmX, &full_bar[s], x0 + sub * 4 * tcb, y0,
+            for (int bx = 0; bx < prm.nb; ++bx)
+                tma_load_3d(smem + s * prm.stage_bytes + bx * prm.box_bytes, &tmX, &full_bar[s], x0 + bx * 4 * tcb, y0,
                             n * prm.C + c_first + (it + IN_TMA_STAGES) * prm.cpb);
         }
         const int c = c_first + it * prm.cpb + cl;

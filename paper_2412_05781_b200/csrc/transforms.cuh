@@ -444,10 +444,15 @@ __device__ __forceinline__ void input_unit_vec(const __half* __restrict__ x, __h
     static_assert(M == 2, "F(4x4) has its own vector kernel (input_transform_f4_kernel)");
     {
     float e[A][TPT][A];  // rows transformed along the columns: e[r][t][nu] = sum_s Bt[nu][s] d[r][s]
+    int tw = 0, th = 0;
+    long long n = 0;
+    if (p < geo.P) decode_tile(geo, p, n, th, tw);
+    // The index arithmetic above needs nothing from memory and runs while the preceding kernel drains.  Wait
+    // first, release the GEMM second: once the GEMM runs, everything before this kernel has completed, which is
+    // what lets it fetch its filters (written at the latest by the kernel before this one) early.
+    pdl_wait();
+    pdl_launch_dependents();
     if (p < geo.P) {
-        int tw, th;
-        long long n;
-        decode_tile(geo, p, n, th, tw);
         const __half* img = x + (n * C + c) * static_cast<long long>(geo.H) * geo.W;
         const int i0 = M * th - 1, j0 = M * tw;
 #pragma unroll
@@ -519,10 +524,6 @@ template <int M, int TPT>
 __global__ void __launch_bounds__(128)
 input_transform_vec_kernel(const __half* __restrict__ x, __half* __restrict__ V, TileGeom geo, int C,
                            long long p_begin, FastDiv gdiv, long long Pstride) {
-    // Wait first, release the GEMM second: once the GEMM runs, everything before this kernel has completed,
-    // which is what lets it fetch its filters (written at the latest by the kernel before this one) early.
-    pdl_wait();
-    pdl_launch_dependents();
     input_unit_vec<M, TPT>(x, V, geo, C, p_begin, gdiv, Pstride, blockIdx.x * blockDim.x + threadIdx.x);   // < 2^31
 }
 
@@ -562,6 +563,11 @@ __device__ __forceinline__ void input_unit_f4(const __half* __restrict__ x, __ha
     const long long plane = static_cast<long long>(C) * Pstride;
     __half* vp = V + static_cast<long long>(c0) * Pstride + pl;
     const int cend = (C - c0) < CH ? (C - c0) : CH;
+    // The index arithmetic above needs nothing from memory and runs while the preceding kernel drains.  Wait
+    // first, release the GEMM second: once the GEMM runs, everything before this kernel has completed, which is
+    // what lets it fetch its filters (written at the latest by the kernel before this one) early.
+    pdl_wait();
+    pdl_launch_dependents();
     for (int cc = 0; cc < cend; ++cc) {
         float2 e2[A][A];   // e2[r][nu]: rows transformed along the columns, (tile 0, tile 1)
 #pragma unroll
@@ -606,8 +612,6 @@ template <int CH>
 __global__ void __launch_bounds__(128, 5)
 input_transform_f4_kernel(const __half* __restrict__ x, __half* __restrict__ V, TileGeom geo, int C, long long p_begin,
                           FastDiv gdiv, long long Pstride) {
-    pdl_wait();                 // see input_transform_vec_kernel: wait first, release the GEMM second
-    pdl_launch_dependents();
     input_unit_f4<CH>(x, V, geo, C, p_begin, gdiv, Pstride, blockIdx.x * blockDim.x + threadIdx.x);   // < 2^31
 }
 
