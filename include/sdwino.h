@@ -115,6 +115,27 @@ int sdwino_conv3x3_ex(const void *x, const void *wT, const void *bias, const voi
                       void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * The fp32 interface: the same path for models kept in fp32 (the paper reports its largest end-to-end gains
+ * for them, Tables 2 and 3 "Type F32").  w, x, bias and y are fp32 device tensors with the layouts of the fp16
+ * calls; the transformed filters U, the transformed activations V and the products M stay fp16 -- the 11-bit
+ * significand of the TF32 tensor-core format at half its bytes, on a path bound by those bytes -- with fp32
+ * accumulation, an fp32 output transform and bias sum, and no rounding of y.  Same tolerance as the fp16 calls,
+ * max|y - ref| <= 1e-2 max|ref| against the fp64 direct convolution of the fp32 inputs, and the same value
+ * range (|x| <= 1e3 for tile 2, 1e2 for tile 4: V is fp16).
+ *
+ * sdwino_filter_transform_f32 writes the same wT as sdwino_filter_transform (size sdwino_filter_bytes; U is
+ * computed in fp32 from the fp32 weights and rounded once), so the buffer serves either convolution call.
+ * sdwino_conv3x3_f32 takes its workspace explicitly (sdwino_workspace_bytes, as for the fp16 calls); layers
+ * with very few channels take the general three-kernel path.  Pointers must be 4-byte aligned
+ * (SDWINO_ERR_MISALIGNED); 16-byte aligned x and y with W % 8 == 0 take the vector kernels.  Arguments, errors
+ * and asynchrony otherwise as sdwino_filter_transform / sdwino_conv3x3_ws.
+ */
+int sdwino_filter_transform_f32(const float *w, void *wT, int K, int C, int tile, void *stream);
+int sdwino_conv3x3_f32(const float *x, const void *wT, const float *bias, float *y,
+                       int N, int C, int H, int W, int K, int tile,
+                       void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * The convolution for callers that must not allocate device memory.  (The paper has no
  * counterpart; this entry point exists for the embedding of the library.)  Some callers cannot
  * call cudaMalloc or any allocator at all: code that runs inside a CUDA-graph capture or another

@@ -23,6 +23,7 @@ EXPORTS = [
     "sdwino_last_device_status", "sdwino_launch_count", "sdwino_profile_enable", "sdwino_profile_collect",
     "sdwino_profile_records", "sdwino_set_gemm_shape", "sdwino_conv3x3_static", "sdwino_set_fused_min_tiles", "sdwino_choose_tile",
     "sdwino_selftest_wait_timeout", "sdwino_conv3x3_host_async", "sdwino_host_join", "sdwino_set_input_staging", "sdwino_conv3x3_ex",
+    "sdwino_filter_transform_f32", "sdwino_conv3x3_f32",
 ]
 
 KERNEL_KINDS = ("filter_transform", "input_transform", "wino_gemm", "output_transform", "fused")
@@ -61,6 +62,10 @@ def _load() -> ctypes.CDLL:
     lib.sdwino_conv3x3_ws.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, vp, sz, vp]
     lib.sdwino_conv3x3_ex.restype = i
     lib.sdwino_conv3x3_ex.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, i, vp, sz, vp]
+    lib.sdwino_filter_transform_f32.restype = i
+    lib.sdwino_filter_transform_f32.argtypes = [vp, vp, i, i, i, vp]
+    lib.sdwino_conv3x3_f32.restype = i
+    lib.sdwino_conv3x3_f32.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, vp, sz, vp]
     lib.sdwino_conv3x3_host.restype = i
     lib.sdwino_conv3x3_host.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, vp, sz, vp]
     lib.sdwino_host_join.restype = i
@@ -265,6 +270,37 @@ def sdwino_conv3x3_ex(x: torch.Tensor, wT: torch.Tensor, bias: Optional[torch.Te
                                tile, int(activation), workspace.data_ptr(),
                                workspace.numel() * workspace.element_size(), _stream_ptr(stream))
     _check(rc, "sdwino_conv3x3_ex")
+    return y
+
+
+def sdwino_filter_transform_f32(w: torch.Tensor, tile: int, stream=None) -> torch.Tensor:
+    """w: fp32 CUDA [K, C, 3, 3] contiguous -> wT (the same opaque buffer sdwino_filter_transform makes)."""
+    assert w.is_cuda and w.dtype == torch.float32 and w.is_contiguous() and w.dim() == 4
+    K, C = int(w.shape[0]), int(w.shape[1])
+    assert tuple(w.shape[2:]) == (3, 3)
+    nbytes = sdwino_filter_bytes(K, C, tile)
+    if nbytes == 0:
+        raise SdwinoError(ERR_UNSUPPORTED if tile not in (2, 4) else ERR_INVALID_ARG, "sdwino_filter_bytes")
+    wT = alloc_workspace(nbytes, w.device)
+    _check(lib.sdwino_filter_transform_f32(w.data_ptr(), wT.data_ptr(), K, C, tile, _stream_ptr(stream)),
+           "sdwino_filter_transform_f32")
+    return wT
+
+
+def sdwino_conv3x3_f32(x: torch.Tensor, wT: torch.Tensor, bias: Optional[torch.Tensor], K: int, tile: int,
+                       workspace: torch.Tensor, y: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """The convolution with fp32 x [N, C, H, W], bias [K] (or None) and y [N, K, H, W]."""
+    assert x.is_cuda and x.dtype == torch.float32 and x.is_contiguous() and x.dim() == 4
+    N, C, H, W = (int(v) for v in x.shape)
+    if y is None:
+        y = torch.empty((N, K, H, W), dtype=torch.float32, device=x.device)
+    assert y.is_cuda and y.is_contiguous() and y.dtype == torch.float32 and tuple(y.shape) == (N, K, H, W)
+    if bias is not None:
+        assert bias.is_cuda and bias.dtype == torch.float32 and bias.numel() == K and bias.is_contiguous()
+    rc = lib.sdwino_conv3x3_f32(x.data_ptr(), wT.data_ptr(), _ptr(bias), y.data_ptr(), N, C, H, W, K, tile,
+                                workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                                _stream_ptr(stream))
+    _check(rc, "sdwino_conv3x3_f32")
     return y
 
 

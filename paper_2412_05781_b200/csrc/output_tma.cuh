@@ -24,10 +24,10 @@ constexpr uint64_t OUT_TMA_WAIT_LIMIT_NS = 2000000000ull;
 
 // tmM: fp16 [36][K][Pstride], box {256 tiles, 1 channel, 36 positions}, no swizzle (tiles and channels outside the
 // tensor read as zeros)
-template <bool EP>
+template <bool EP, typename YT = __half>
 __global__ void __launch_bounds__(OUT_TMA_THREADS, 3)
-output_transform_f4_tma_kernel(const __grid_constant__ CUtensorMap tmM, const __half* __restrict__ bias,
-                               __half* __restrict__ y, TileGeom geo, int K, long long p_begin, int steps_per_cta,
+output_transform_f4_tma_kernel(const __grid_constant__ CUtensorMap tmM, const YT* __restrict__ bias,
+                               YT* __restrict__ y, TileGeom geo, int K, long long p_begin, int steps_per_cta,
                                WtCheck chk, Epilogue ep, int* __restrict__ status_word) {
     constexpr int A = 6, M = 4;
     extern __shared__ uint8_t out_tma_smem_raw[];
@@ -102,7 +102,7 @@ output_transform_f4_tma_kernel(const __grid_constant__ CUtensorMap tmM, const __
         if (!tile_ok) continue;
         const int k = k_first + it;
         const float b = load_bias(bias, k);
-        __half* img = y + (n * K + k) * hw + pix;
+        YT* img = y + (n * K + k) * hw + pix;
         uint4 res[M];
         if constexpr (EP) {
 #pragma unroll

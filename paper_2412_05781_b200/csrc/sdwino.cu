@@ -321,19 +321,19 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
     return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
-template <int M>
-int launch_filter(const __half* w, void* wT, int K, int C, int Kb, int Cb, cudaStream_t st) {
+template <int M, typename WT>
+int launch_filter(const WT* w, void* wT, int K, int C, int Kb, int Cb, cudaStream_t st) {
     dim3 grid((Cb * 32 + 127) / 128, Kb * 16);   // a thread transforms two neighbouring input channels
     ProfScope prof(KIND_FILTER, st);
     uint32_t* header = static_cast<uint32_t*>(wT);
     __half* U = reinterpret_cast<__half*>(static_cast<uint8_t*>(wT) + WT_HEADER_BYTES);
-    const cudaError_t e = launch_pdl(filter_transform_kernel<M>, grid, dim3(128), 0, st, 0, w, header, U, K, C, Kb, Cb);
+    const cudaError_t e = launch_pdl(filter_transform_kernel<M, WT>, grid, dim3(128), 0, st, 0, w, header, U, K, C, Kb, Cb);
     g_launches.fetch_add(1);
     return e == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
 }
 
-template <int M>
-int launch_input(const __half* x, __half* V, const TileGeom& geo, int C, long long p_begin, int p_count,
+template <int M, typename XT>
+int launch_input(const XT* x, __half* V, const TileGeom& geo, int C, long long p_begin, int p_count,
                  long long Pstride, cudaStream_t st) {
     ProfScope prof(KIND_INPUT, st);
     constexpr int TPT = 8 / M;
@@ -344,16 +344,16 @@ int launch_input(const __half* x, __half* V, const TileGeom& geo, int C, long lo
             constexpr int CH = 1;   // channels per thread
             const long long threads = static_cast<long long>(p_count / TPT) * ((C + CH - 1) / CH);
             dim3 grid(static_cast<unsigned>((threads + 127) / 128));
-            e = launch_pdl(input_transform_f4_kernel<CH>, grid, dim3(128), 0, st, 0, x, V, geo, C, p_begin,
+            e = launch_pdl(input_transform_f4_kernel<CH, XT>, grid, dim3(128), 0, st, 0, x, V, geo, C, p_begin,
                            make_fastdiv(static_cast<uint32_t>(p_count / TPT)), Pstride);
         } else {
             dim3 grid(static_cast<unsigned>((units + 127) / 128));
-            e = launch_pdl(input_transform_vec_kernel<M, TPT>, grid, dim3(128), 0, st, 0, x, V, geo, C, p_begin,
+            e = launch_pdl(input_transform_vec_kernel<M, TPT, XT>, grid, dim3(128), 0, st, 0, x, V, geo, C, p_begin,
                            make_fastdiv(static_cast<uint32_t>(p_count / TPT)), Pstride);
         }
     } else {
         dim3 grid((p_count + 127) / 128, C);
-        e = launch_pdl(input_transform_kernel<M>, grid, dim3(128), 0, st, 0, x, V, geo, C, p_begin, p_count, Pstride);
+        e = launch_pdl(input_transform_kernel<M, XT>, grid, dim3(128), 0, st, 0, x, V, geo, C, p_begin, p_count, Pstride);
     }
     g_launches.fetch_add(1);
     return e == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
@@ -471,7 +471,8 @@ bool use_output_tma(const TileGeom& geo, int K, const void* y, const Epilogue& e
     return g_input_staging == 2 || p_count >= 512;
 }
 
-int launch_output_tma(const __half* Mws, const __half* bias, __half* y, const TileGeom& geo, int K, long long p_begin,
+template <typename YT>
+int launch_output_tma(const __half* Mws, const YT* bias, YT* y, const TileGeom& geo, int K, long long p_begin,
                       int p_count, long long Pstride, const WtCheck& chk, const Epilogue& ep, cudaStream_t st) {
     ProfScope prof(KIND_OUTPUT, st);
     const int sms = sm_count();
@@ -495,23 +496,30 @@ int launch_output_tma(const __half* Mws, const __half* bias, __half* y, const Ti
     if ((K + steps - 1) / steps > 65535) steps = (K + 65534) / 65535;   // grid limit; K <= 65535 * 16 was checked
     const size_t smem = static_cast<size_t>(OUT_TMA_STAGES) * OUT_TMA_STAGE_BYTES + 128;
     if (blocks >= (1ll << 31) ||
-        !ensure_dyn_smem(reinterpret_cast<const void*>(output_transform_f4_tma_kernel<false>), static_cast<int>(smem)) ||
-        !ensure_dyn_smem(reinterpret_cast<const void*>(output_transform_f4_tma_kernel<true>), static_cast<int>(smem)))
+        !ensure_dyn_smem(reinterpret_cast<const void*>(output_transform_f4_tma_kernel<false, YT>), static_cast<int>(smem)))
         return SDWINO_ERR_CUDA;
+    if constexpr (sizeof(YT) == 2) {
+        if (!ensure_dyn_smem(reinterpret_cast<const void*>(output_transform_f4_tma_kernel<true>), static_cast<int>(smem)))
+            return SDWINO_ERR_CUDA;
+    }
     dim3 grid(static_cast<unsigned>(blocks), static_cast<unsigned>((K + steps - 1) / steps));
     cudaError_t e;
-    if (ep.residual == nullptr && ep.act == 0)
-        e = launch_pdl(output_transform_f4_tma_kernel<false>, grid, dim3(OUT_TMA_THREADS), smem, st, 0, tmM, bias, y, geo, K,
+    if (ep.residual == nullptr && ep.act == 0) {
+        e = launch_pdl(output_transform_f4_tma_kernel<false, YT>, grid, dim3(OUT_TMA_THREADS), smem, st, 0, tmM, bias, y, geo, K,
                        p_begin, static_cast<int>(steps), chk, ep, status);
-    else
-        e = launch_pdl(output_transform_f4_tma_kernel<true>, grid, dim3(OUT_TMA_THREADS), smem, st, 0, tmM, bias, y, geo, K,
-                       p_begin, static_cast<int>(steps), chk, ep, status);
+    } else {
+        if constexpr (sizeof(YT) == 2)
+            e = launch_pdl(output_transform_f4_tma_kernel<true>, grid, dim3(OUT_TMA_THREADS), smem, st, 0, tmM, bias, y, geo, K,
+                           p_begin, static_cast<int>(steps), chk, ep, status);
+        else
+            return SDWINO_ERR_UNSUPPORTED;   // the fused residual / activation is part of the fp16 interface
+    }
     g_launches.fetch_add(1);
     return e == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
 }
 
-template <int M>
-int launch_output(const __half* Mws, const __half* bias, __half* y, const TileGeom& geo, int K,
+template <int M, typename YT>
+int launch_output(const __half* Mws, const YT* bias, YT* y, const TileGeom& geo, int K,
                   long long p_begin, int p_count, long long Pstride, const WtCheck& chk, const Epilogue& ep,
                   cudaStream_t st) {
     ProfScope prof(KIND_OUTPUT, st);
@@ -520,15 +528,19 @@ int launch_output(const __half* Mws, const __half* bias, __half* y, const TileGe
     const long long units = static_cast<long long>(p_count / TPT) * K;   // one thread each
     if (geo.W % 8 == 0 && aligned(y, 16) && aligned(ep.residual, 16) && units < (1ll << 31) - 128) {
         dim3 grid(static_cast<unsigned>((units + 127) / 128));
-        if (ep.residual == nullptr && ep.act == 0)
-            e = launch_pdl(output_transform_vec_kernel<M, TPT, false>, grid, dim3(128), 0, st, 0, Mws, bias, y, geo, K,
+        if (ep.residual == nullptr && ep.act == 0) {
+            e = launch_pdl(output_transform_vec_kernel<M, TPT, false, YT>, grid, dim3(128), 0, st, 0, Mws, bias, y, geo, K,
                            p_begin, make_fastdiv(static_cast<uint32_t>(p_count / TPT)), Pstride, chk, ep);
-        else
-            e = launch_pdl(output_transform_vec_kernel<M, TPT, true>, grid, dim3(128), 0, st, 0, Mws, bias, y, geo, K,
-                           p_begin, make_fastdiv(static_cast<uint32_t>(p_count / TPT)), Pstride, chk, ep);
+        } else {
+            if constexpr (sizeof(YT) == 2)
+                e = launch_pdl(output_transform_vec_kernel<M, TPT, true>, grid, dim3(128), 0, st, 0, Mws, bias, y, geo, K,
+                               p_begin, make_fastdiv(static_cast<uint32_t>(p_count / TPT)), Pstride, chk, ep);
+            else
+                return SDWINO_ERR_UNSUPPORTED;
+        }
     } else {
         dim3 grid((p_count + 127) / 128, K);
-        e = launch_pdl(output_transform_kernel<M>, grid, dim3(128), 0, st, 0, Mws, bias, y, geo, K, p_begin, p_count,
+        e = launch_pdl(output_transform_kernel<M, YT>, grid, dim3(128), 0, st, 0, Mws, bias, y, geo, K, p_begin, p_count,
                        Pstride, chk, ep);
     }
     g_launches.fetch_add(1);
@@ -711,14 +723,16 @@ int launch_gemm(const CUtensorMap& tmU, const CUtensorMap& tmV, const CUtensorMa
 
 
 int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, int C, int H, int W, int K, int tile,
-              void* ws, size_t ws_bytes, cudaStream_t st, const Epilogue& ep = Epilogue{nullptr, 0}) {
+              void* ws, size_t ws_bytes, cudaStream_t st, const Epilogue& ep = Epilogue{nullptr, 0},
+              bool io32 = false) {   // io32: x, bias and y are fp32 (the filters come from the fp32 filter transform)
     if (tile != 2 && tile != 4) {
         return (N <= 0 || C <= 0 || H <= 0 || W <= 0 || K <= 0 || !x || !wT || !y) ? SDWINO_ERR_INVALID_ARG
                                                                                      : SDWINO_ERR_UNSUPPORTED;
     }
     Plan pl;
     if (!x || !wT || !y || !make_plan(N, C, H, W, K, tile, &pl)) return SDWINO_ERR_INVALID_ARG;
-    if (!aligned(x, 2) || !aligned(y, 2) || (bias && !aligned(bias, 2)) || !aligned(wT, WS_ALIGN))
+    const size_t elem = io32 ? 4 : 2;
+    if (!aligned(x, elem) || !aligned(y, elem) || (bias && !aligned(bias, elem)) || !aligned(wT, WS_ALIGN))
         return SDWINO_ERR_MISALIGNED;
     if (!ws || ws_bytes == 0) return SDWINO_ERR_WORKSPACE;
     if (!aligned(ws, WS_ALIGN)) return SDWINO_ERR_MISALIGNED;
@@ -730,9 +744,10 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
         long long a = pl.TW, b = GEMM_BLOCK_P;
         while (b != 0) { const long long t = a % b; a = b; b = t; }
         const long long lcm = static_cast<long long>(pl.TW) / a * GEMM_BLOCK_P;
-        if (pc >= lcm && use_input_tma(g0, N, C, x, 0, lcm)) pc = pc / lcm * lcm;
+        if (pc >= lcm && !io32 && use_input_tma(g0, N, C, x, 0, lcm)) pc = pc / lcm * lcm;
     }
-    const bool plain = ep.residual == nullptr && ep.act == 0;   // the single-kernel paths end at the bias
+    // the single-kernel paths end at the bias and read and write fp16
+    const bool plain = ep.residual == nullptr && ep.act == 0 && !io32;
     if (plain && use_fused_small_k(K, W, tile, pl.P128 / 128, x, y) && !use_fused_small_c(C, tile) && !g_disable_fused)
         return launch_fused_small_k(static_cast<const __half*>(x), wT, static_cast<const __half*>(bias),
                                     static_cast<__half*>(y), pl, C, H, W, K, st);
@@ -838,7 +853,10 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
         long long remaining = pl.P128 - p0;
         const int count = static_cast<int>(remaining < pc ? remaining : pc);  // multiple of 128
         int rc;
-        if (tile == 2) rc = launch_input<2>(xh, V, geo, C, p0, count, pc, st);
+        if (io32) {
+            const float* xf = static_cast<const float*>(x);
+            rc = tile == 2 ? launch_input<2>(xf, V, geo, C, p0, count, pc, st) : launch_input<4>(xf, V, geo, C, p0, count, pc, st);
+        } else if (tile == 2) rc = launch_input<2>(xh, V, geo, C, p0, count, pc, st);
         else {
             rc = use_input_tma(geo, N, C, x, p0, count) ? launch_input_tma(xh, V, geo, N, C, p0, count, pc, st)
                                                         : SDWINO_ERR_UNSUPPORTED;
@@ -849,7 +867,13 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
         prm.num_p_tiles = (count / GEMM_BLOCK_P + p_blocks - 1) / p_blocks;
         rc = launch_gemm(tmU, tmV, tmM, prm, shape.ctas, st);
         if (rc != SDWINO_OK) return rc;
-        if (tile == 2) rc = launch_output<2>(Mws, bh, yh, geo, K, p0, count, pc, chk, ep, st);
+        if (io32) {
+            const float* bf = static_cast<const float*>(bias);
+            float* yf = static_cast<float*>(y);
+            if (tile == 2) rc = launch_output<2>(Mws, bf, yf, geo, K, p0, count, pc, chk, ep, st);
+            else if (use_output_tma(geo, K, y, ep, count)) rc = launch_output_tma(Mws, bf, yf, geo, K, p0, count, pc, chk, ep, st);
+            else rc = launch_output<4>(Mws, bf, yf, geo, K, p0, count, pc, chk, ep, st);
+        } else if (tile == 2) rc = launch_output<2>(Mws, bh, yh, geo, K, p0, count, pc, chk, ep, st);
         else if (use_output_tma(geo, K, y, ep, count)) rc = launch_output_tma(Mws, bh, yh, geo, K, p0, count, pc, chk, ep, st);
         else rc = launch_output<4>(Mws, bh, yh, geo, K, p0, count, pc, chk, ep, st);
         if (rc != SDWINO_OK) return rc;
@@ -932,6 +956,17 @@ int sdwino_filter_transform(const void* w, void* wT, int K, int C, int tile, voi
     return launch_filter<4>(static_cast<const __half*>(w), wT, K, C, Kb, Cb, st);
 }
 
+int sdwino_filter_transform_f32(const float* w, void* wT, int K, int C, int tile, void* stream) {
+    if (!w || !wT || K <= 0 || C <= 0) return SDWINO_ERR_INVALID_ARG;
+    if (tile != 2 && tile != 4) return SDWINO_ERR_UNSUPPORTED;
+    if (!aligned(w, 4) || !aligned(wT, WS_ALIGN)) return SDWINO_ERR_MISALIGNED;
+    if (static_cast<long double>(K) * C > 4.0e15L) return SDWINO_ERR_INVALID_ARG;
+    const int Kb = (K + 15) / 16, Cb = (C + 63) / 64;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (tile == 2) return launch_filter<2>(w, wT, K, C, Kb, Cb, st);
+    return launch_filter<4>(w, wT, K, C, Kb, Cb, st);
+}
+
 size_t sdwino_workspace_bytes(int N, int C, int H, int W, int K, int tile) {
     Plan pl;
     if (!make_plan(N, C, H, W, K, tile, &pl)) return 0;
@@ -967,6 +1002,12 @@ int sdwino_conv3x3_ex(const void* x, const void* wT, const void* bias, const voi
     if (residual && !aligned(residual, 2)) return SDWINO_ERR_MISALIGNED;
     return conv_impl(x, wT, bias, y, N, C, H, W, K, tile, workspace, workspace_bytes, static_cast<cudaStream_t>(stream),
                      Epilogue{static_cast<const __half*>(residual), activation});
+}
+
+int sdwino_conv3x3_f32(const float* x, const void* wT, const float* bias, float* y, int N, int C, int H, int W, int K,
+                       int tile, void* workspace, size_t workspace_bytes, void* stream) {
+    return conv_impl(x, wT, bias, y, N, C, H, W, K, tile, workspace, workspace_bytes, static_cast<cudaStream_t>(stream),
+                     Epilogue{nullptr, 0}, true);
 }
 
 int sdwino_conv3x3(const void* x, const void* wT, const void* bias, void* y, int N, int C, int H, int W, int K,

@@ -79,6 +79,17 @@ __device__ __forceinline__ float load_bias(const __half* bias, int k) {
     if (bias != nullptr) b = __half2float(bias[k]);
     return b;
 }
+__device__ __forceinline__ float load_bias(const float* bias, int k) {
+    float b = 0.f;
+    if (bias != nullptr) b = bias[k];
+    return b;
+}
+
+// The fp32 interface (x, w, bias, y in fp32): the kernels below take the element type of the tensors they read
+// from or write to the caller as a template argument.  Everything between the transforms is the same: U, V and M
+// are fp16 (the 11-bit significand of the TF32 tensor-core format), accumulation is fp32.
+__device__ __forceinline__ float to_f32(__half v) { return __half2float(v); }
+__device__ __forceinline__ float to_f32(float v) { return v; }
 
 // out[i] = sum_j coef[i][j] * in[j] with compile-time coefficients: zero terms vanish and
 // unit terms become adds once the loops are unrolled.
@@ -135,9 +146,9 @@ __device__ __forceinline__ bool wt_check(const WtCheck& c) {
 // n_tile separate 128-byte rows (the weights are the one operand that is streamed from HBM).  One thread per (k, pair of c) of the padded plane.
 // Writes all a*a positions.
 // ---------------------------------------------------------------------------------------
-template <int M>
+template <int M, typename WT = __half>
 __global__ void __launch_bounds__(128)
-filter_transform_kernel(const __half* __restrict__ w, uint32_t* __restrict__ header, __half* __restrict__ U, int K,
+filter_transform_kernel(const WT* __restrict__ w, uint32_t* __restrict__ header, __half* __restrict__ U, int K,
                         int C, int Kb, int Cb) {
     using Wm = Wino<M>;
     constexpr int A = Wm::A;
@@ -158,7 +169,7 @@ filter_transform_kernel(const __half* __restrict__ w, uint32_t* __restrict__ hea
         for (int r = 0; r < 3; ++r)
 #pragma unroll
             for (int s = 0; s < 3; ++s)
-                g[r][s] = live ? __half2float(w[(static_cast<size_t>(k) * C + c + h) * 9 + r * 3 + s]) : 0.f;
+                g[r][s] = live ? to_f32(w[(static_cast<size_t>(k) * C + c + h) * 9 + r * 3 + s]) : 0.f;
         // t = G g  (A x 3), u = t G^T (A x A)
         float t[A][3];
 #pragma unroll
@@ -229,9 +240,9 @@ __device__ __forceinline__ void decode_tile(const TileGeom& geo, long long p, lo
 // Activation preprocess.  V layout: [a*a][C][Pstride] with the chunk-local tile index
 // (p - p_begin) contiguous.  Threads past the last tile write zeros so that the GEMM reads
 // defined data.
-template <int M>
+template <int M, typename XT = __half>
 __global__ void __launch_bounds__(128)
-input_transform_kernel(const __half* __restrict__ x, __half* __restrict__ V, TileGeom geo, int C, long long p_begin,
+input_transform_kernel(const XT* __restrict__ x, __half* __restrict__ V, TileGeom geo, int C, long long p_begin,
                        int p_count, long long Pstride) {
     using Wm = Wino<M>;
     constexpr int A = Wm::A;
@@ -248,7 +259,7 @@ input_transform_kernel(const __half* __restrict__ x, __half* __restrict__ V, Til
         int tw, th;
         long long n;
         decode_tile(geo, p, n, th, tw);
-        const __half* img = x + (n * C + c) * static_cast<long long>(geo.H) * geo.W;
+        const XT* img = x + (n * C + c) * static_cast<long long>(geo.H) * geo.W;
         const int i0 = M * th - 1, j0 = M * tw - 1;
 #pragma unroll
         for (int r = 0; r < A; ++r) {
@@ -257,7 +268,7 @@ input_transform_kernel(const __half* __restrict__ x, __half* __restrict__ V, Til
 #pragma unroll
             for (int s = 0; s < A; ++s) {
                 const int j = j0 + s;
-                d[r][s] = (rin && j >= 0 && j < geo.W) ? __half2float(__ldg(img + static_cast<long long>(i) * geo.W + j))
+                d[r][s] = (rin && j >= 0 && j < geo.W) ? to_f32(__ldg(img + static_cast<long long>(i) * geo.W + j))
                                                         : 0.f;
             }
         }
@@ -302,9 +313,9 @@ __device__ __forceinline__ float epilogue_act(float v, int act) {
 }
 
 // Postprocess + bias + cast + masked store.  Mws layout: [a*a][K][Pstride]; y is NCHW.
-template <int M>
+template <int M, typename YT = __half>
 __global__ void __launch_bounds__(128)
-output_transform_kernel(const __half* __restrict__ Mws, const __half* __restrict__ bias, __half* __restrict__ y,
+output_transform_kernel(const __half* __restrict__ Mws, const YT* __restrict__ bias, YT* __restrict__ y,
                         TileGeom geo, int K, long long p_begin, int p_count, long long Pstride, WtCheck chk,
                         Epilogue ep) {
     using Wm = Wino<M>;
@@ -342,7 +353,7 @@ output_transform_kernel(const __half* __restrict__ Mws, const __half* __restrict
     long long n;
     decode_tile(geo, p, n, th, tw);
     const float b = load_bias(bias, k);
-    __half* img = y + (n * K + k) * static_cast<long long>(geo.H) * geo.W;
+    YT* img = y + (n * K + k) * static_cast<long long>(geo.H) * geo.W;
     const int i0 = M * th, j0 = M * tw;
     const bool vec_ok = ((geo.W & 1) == 0) && ((reinterpret_cast<uintptr_t>(y) & 3) == 0);
 #pragma unroll
@@ -351,6 +362,13 @@ output_transform_kernel(const __half* __restrict__ Mws, const __half* __restrict
         mat_apply<M, A>(typename Wm::At{}, t[i], o);
         const int oi = i0 + i;
         if (oi >= geo.H) continue;
+        if constexpr (sizeof(YT) == 4) {   // fp32 output: no residual, no activation, no rounding
+            float* rowf = reinterpret_cast<float*>(img) + static_cast<long long>(oi) * geo.W + j0;
+#pragma unroll
+            for (int j = 0; j < M; ++j)
+                if (j0 + j < geo.W) rowf[j] = o[j] + b;
+            continue;
+        } else {
         __half* rowp = img + static_cast<long long>(oi) * geo.W + j0;
         const __half* resp = ep.residual ? ep.residual + (rowp - y) : nullptr;
 #pragma unroll
@@ -368,6 +386,7 @@ output_transform_kernel(const __half* __restrict__ Mws, const __half* __restrict
                 if (j0 + j + 1 < geo.W) rowp[j + 1] = h1;
             }
         }
+        }   // fp16 output
     }
 }
 
@@ -430,8 +449,8 @@ __device__ __forceinline__ void at4_packed(const float2 (&m)[6], float2 (&o)[4])
 // One unit of the vector activation transform: channel c = idx / groups, TPT tiles of one tile row.  The flat
 // index over (channel, group of TPT tiles) keeps blocks full when a pass has few tiles.  Called by the kernel
 // below with one unit per thread.
-template <int M, int TPT>
-__device__ __forceinline__ void input_unit_vec(const __half* __restrict__ x, __half* __restrict__ V, const TileGeom& geo,
+template <int M, int TPT, typename XT = __half>
+__device__ __forceinline__ void input_unit_vec(const XT* __restrict__ x, __half* __restrict__ V, const TileGeom& geo,
                                                int C, long long p_begin, const FastDiv& gdiv, long long Pstride,
                                                uint32_t idx) {
     using Wm = Wino<M>;
@@ -453,21 +472,28 @@ __device__ __forceinline__ void input_unit_vec(const __half* __restrict__ x, __h
     pdl_wait();
     pdl_launch_dependents();
     if (p < geo.P) {
-        const __half* img = x + (n * C + c) * static_cast<long long>(geo.H) * geo.W;
+        const XT* img = x + (n * C + c) * static_cast<long long>(geo.H) * geo.W;
         const int i0 = M * th - 1, j0 = M * tw;
 #pragma unroll
         for (int r = 0; r < A; ++r) {
             const int i = i0 + r;
             float row[10];
             if (i >= 0 && i < geo.H) {
-                const __half* rp = img + static_cast<long long>(i) * geo.W + j0;
-                const uint4 v = __ldg(reinterpret_cast<const uint4*>(rp));
-                unpack2(v.x, row[1], row[2]);
-                unpack2(v.y, row[3], row[4]);
-                unpack2(v.z, row[5], row[6]);
-                unpack2(v.w, row[7], row[8]);
-                row[0] = j0 > 0 ? __half2float(__ldg(rp - 1)) : 0.f;
-                row[9] = j0 + 8 < geo.W ? __half2float(__ldg(rp + 8)) : 0.f;
+                const XT* rp = img + static_cast<long long>(i) * geo.W + j0;
+                if constexpr (sizeof(XT) == 4) {   // fp32 input: the eight pixels are two 16-byte loads
+                    const float4 a = __ldg(reinterpret_cast<const float4*>(rp));
+                    const float4 b = __ldg(reinterpret_cast<const float4*>(rp) + 1);
+                    row[1] = a.x; row[2] = a.y; row[3] = a.z; row[4] = a.w;
+                    row[5] = b.x; row[6] = b.y; row[7] = b.z; row[8] = b.w;
+                } else {
+                    const uint4 v = __ldg(reinterpret_cast<const uint4*>(rp));
+                    unpack2(v.x, row[1], row[2]);
+                    unpack2(v.y, row[3], row[4]);
+                    unpack2(v.z, row[5], row[6]);
+                    unpack2(v.w, row[7], row[8]);
+                }
+                row[0] = j0 > 0 ? to_f32(__ldg(rp - 1)) : 0.f;
+                row[9] = j0 + 8 < geo.W ? to_f32(__ldg(rp + 8)) : 0.f;
             } else {
 #pragma unroll
                 for (int s = 0; s < 10; ++s) row[s] = 0.f;
@@ -520,11 +546,11 @@ __device__ __forceinline__ void input_unit_vec(const __half* __restrict__ x, __h
     }   // M != 4
 }
 
-template <int M, int TPT>
+template <int M, int TPT, typename XT = __half>
 __global__ void __launch_bounds__(128)
-input_transform_vec_kernel(const __half* __restrict__ x, __half* __restrict__ V, TileGeom geo, int C,
+input_transform_vec_kernel(const XT* __restrict__ x, __half* __restrict__ V, TileGeom geo, int C,
                            long long p_begin, FastDiv gdiv, long long Pstride) {
-    input_unit_vec<M, TPT>(x, V, geo, C, p_begin, gdiv, Pstride, blockIdx.x * blockDim.x + threadIdx.x);   // < 2^31
+    input_unit_vec<M, TPT, XT>(x, V, geo, C, p_begin, gdiv, Pstride, blockIdx.x * blockDim.x + threadIdx.x);   // < 2^31
 }
 
 // F(4x4,3x3) activation transform, vector path: a thread owns 2 tiles (8 pixels of a tile row) and CH consecutive
@@ -533,8 +559,8 @@ input_transform_vec_kernel(const __half* __restrict__ x, __half* __restrict__ V,
 // permutes.  The kernel is bound by instruction issue, so this is where its time goes: 3-10 % per layer over
 // the generic vector kernel.  CH = 1 is what runs: with 2 or 4 channels per thread the per-thread set-up is
 // amortised, but the serial load -> compute chain per channel and the lower thread count cost more (measured).
-template <int CH>
-__device__ __forceinline__ void input_unit_f4(const __half* __restrict__ x, __half* __restrict__ V, const TileGeom& geo,
+template <int CH, typename XT = __half>
+__device__ __forceinline__ void input_unit_f4(const XT* __restrict__ x, __half* __restrict__ V, const TileGeom& geo,
                                               int C, long long p_begin, const FastDiv& gdiv, long long Pstride,
                                               uint32_t idx) {
     constexpr int A = 6;
@@ -547,7 +573,7 @@ __device__ __forceinline__ void input_unit_f4(const __half* __restrict__ x, __ha
     const bool valid = p < geo.P;
     int rowmask = 0;
     bool left_ok = false, right_ok = false;
-    const __half* xp = x;
+    const XT* xp = x;
     if (valid) {
         int tw, th;
         long long n;
@@ -572,6 +598,25 @@ __device__ __forceinline__ void input_unit_f4(const __half* __restrict__ x, __ha
         float2 e2[A][A];   // e2[r][nu]: rows transformed along the columns, (tile 0, tile 1)
 #pragma unroll
         for (int r = 0; r < A; ++r) {
+            float2 d[A];
+            if constexpr (sizeof(XT) == 4) {
+                // fp32 input: pixels px0..px7 = a.x .. b.w, L and R the neighbours; pairs are (tile 0, tile 1)
+                float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+                float L = 0.f, R = 0.f;
+                if ((rowmask >> r) & 1) {
+                    const XT* rp = xp + r * geo.W;
+                    a = __ldg(reinterpret_cast<const float4*>(rp));
+                    b = __ldg(reinterpret_cast<const float4*>(rp) + 1);
+                    if (left_ok) L = to_f32(__ldg(rp - 1));
+                    if (right_ok) R = to_f32(__ldg(rp + 8));
+                }
+                d[0] = make_float2(L, a.w);
+                d[1] = make_float2(a.x, b.x);
+                d[2] = make_float2(a.y, b.y);
+                d[3] = make_float2(a.z, b.z);
+                d[4] = make_float2(a.w, b.w);
+                d[5] = make_float2(b.x, R);
+            } else {
             uint4 v = make_uint4(0u, 0u, 0u, 0u);
             uint32_t lw = 0u, rw = 0u;   // aligned words before / after the segment
             if ((rowmask >> r) & 1) {
@@ -588,9 +633,9 @@ __device__ __forceinline__ void input_unit_f4(const __half* __restrict__ x, __ha
             h[3] = __byte_perm(v.y, v.w, 0x5410);   // (px2, px6)
             h[4] = __byte_perm(v.y, v.w, 0x7632);   // (px3, px7)
             h[5] = __byte_perm(v.z, rw, 0x5410);    // (px4, R)
-            float2 d[A];
 #pragma unroll
             for (int s2 = 0; s2 < A; ++s2) d[s2] = __half22float2(*reinterpret_cast<const __half2*>(&h[s2]));
+            }   // fp16 input
             bt4_packed(d, e2[r]);
         }
 #pragma unroll
@@ -608,11 +653,11 @@ __device__ __forceinline__ void input_unit_f4(const __half* __restrict__ x, __ha
     }
 }
 
-template <int CH>
+template <int CH, typename XT = __half>
 __global__ void __launch_bounds__(128, 5)
-input_transform_f4_kernel(const __half* __restrict__ x, __half* __restrict__ V, TileGeom geo, int C, long long p_begin,
+input_transform_f4_kernel(const XT* __restrict__ x, __half* __restrict__ V, TileGeom geo, int C, long long p_begin,
                           FastDiv gdiv, long long Pstride) {
-    input_unit_f4<CH>(x, V, geo, C, p_begin, gdiv, Pstride, blockIdx.x * blockDim.x + threadIdx.x);   // < 2^31
+    input_unit_f4<CH, XT>(x, V, geo, C, p_begin, gdiv, Pstride, blockIdx.x * blockDim.x + threadIdx.x);   // < 2^31
 }
 
 // Eight output pixels of one row (bias already added): residual (its eight values loaded by the caller, ahead of
@@ -640,9 +685,17 @@ __device__ __forceinline__ void store_row8(__half* rowp, float (&v)[8], const ui
     *reinterpret_cast<uint4*>(rowp) = w;
 }
 
-template <int M, int TPT, bool EP>
-__device__ __forceinline__ void output_unit_vec(const __half* __restrict__ Mws, const __half* __restrict__ bias,
-                                                __half* __restrict__ y, const TileGeom& geo, int K, long long p_begin,
+// fp32 output: eight pixels are two 16-byte stores; there is no residual, activation or rounding
+template <bool EP>
+__device__ __forceinline__ void store_row8(float* rowp, float (&v)[8], const uint4&, const Epilogue&) {
+    static_assert(!EP, "the fused residual / activation is part of the fp16 interface");
+    reinterpret_cast<float4*>(rowp)[0] = make_float4(v[0], v[1], v[2], v[3]);
+    reinterpret_cast<float4*>(rowp)[1] = make_float4(v[4], v[5], v[6], v[7]);
+}
+
+template <int M, int TPT, bool EP, typename YT = __half>
+__device__ __forceinline__ void output_unit_vec(const __half* __restrict__ Mws, const YT* __restrict__ bias,
+                                                YT* __restrict__ y, const TileGeom& geo, int K, long long p_begin,
                                                 const FastDiv& gdiv, long long Pstride, uint32_t idx, const Epilogue& ep) {
     using Wm = Wino<M>;
     constexpr int A = Wm::A;
@@ -673,7 +726,7 @@ __device__ __forceinline__ void output_unit_vec(const __half* __restrict__ Mws, 
         long long n;
         decode_tile(geo, p, n, th, tw);
         const float b = load_bias(bias, k);
-        __half* img = y + (n * K + k) * static_cast<long long>(geo.H) * geo.W;
+        YT* img = y + (n * K + k) * static_cast<long long>(geo.H) * geo.W;
         const int i0 = M * th, j0 = M * tw;
         uint4 res[M];
         if constexpr (EP) {
@@ -691,7 +744,7 @@ __device__ __forceinline__ void output_unit_vec(const __half* __restrict__ Mws, 
             at4_packed(tt[i], o);
             if (i0 + i >= geo.H) continue;
             float v[8] = {o[0].x + b, o[1].x + b, o[2].x + b, o[3].x + b, o[0].y + b, o[1].y + b, o[2].y + b, o[3].y + b};
-            __half* rowp = img + static_cast<long long>(i0 + i) * geo.W + j0;
+            YT* rowp = img + static_cast<long long>(i0 + i) * geo.W + j0;
             store_row8<EP>(rowp, v, res[i], ep);
         }
     } else {
@@ -714,7 +767,7 @@ __device__ __forceinline__ void output_unit_vec(const __half* __restrict__ Mws, 
     long long n;
     decode_tile(geo, p, n, th, tw);
     const float b = load_bias(bias, k);
-    __half* img = y + (n * K + k) * static_cast<long long>(geo.H) * geo.W;
+    YT* img = y + (n * K + k) * static_cast<long long>(geo.H) * geo.W;
     const int i0 = M * th, j0 = M * tw;
     uint4 res[M];
     if constexpr (EP) {
@@ -756,16 +809,16 @@ __device__ __forceinline__ void output_unit_vec(const __half* __restrict__ Mws, 
 }
 
 // EP = false: the plain convolution (the epilogue argument is ignored and costs no register)
-template <int M, int TPT, bool EP>
+template <int M, int TPT, bool EP, typename YT = __half>
 __global__ void __launch_bounds__(128)
-output_transform_vec_kernel(const __half* __restrict__ Mws, const __half* __restrict__ bias, __half* __restrict__ y,
+output_transform_vec_kernel(const __half* __restrict__ Mws, const YT* __restrict__ bias, YT* __restrict__ y,
                             TileGeom geo, int K, long long p_begin, FastDiv gdiv, long long Pstride, WtCheck chk,
                             Epilogue ep) {
     pdl_launch_dependents();
     const bool wt_ok = wt_check(chk);   // before the wait: see output_transform_kernel
     pdl_wait();
     if (!wt_ok) return;
-    output_unit_vec<M, TPT, EP>(Mws, bias, y, geo, K, p_begin, gdiv, Pstride, blockIdx.x * blockDim.x + threadIdx.x, ep);
+    output_unit_vec<M, TPT, EP, YT>(Mws, bias, y, geo, K, p_begin, gdiv, Pstride, blockIdx.x * blockDim.x + threadIdx.x, ep);
 }
 
 

@@ -98,16 +98,18 @@ WORKLOADS = {
 
 
 def make_inputs(layer: ConvLayer, seed: int = 0, with_bias: bool = True,
-                pin: bool = False):
-    """Return (x, w, bias) as fp16 CPU tensors drawn by the recipe in the module docstring."""
+                pin: bool = False, dtype: torch.dtype = torch.float16):
+    """Return (x, w, bias) as CPU tensors drawn by the recipe in the module docstring: fp16 by default,
+    the same draws left in fp32 with dtype=torch.float32 (inputs of the fp32 interface)."""
+    assert dtype in (torch.float16, torch.float32)
     g = torch.Generator().manual_seed(seed)
     x = torch.randn(layer.N, layer.C, layer.H, layer.W, generator=g, dtype=torch.float32)
     w = torch.randn(layer.K, layer.C, 3, 3, generator=g, dtype=torch.float32)
     w.mul_(1.0 / (9.0 * layer.C) ** 0.5)
     b: Optional[torch.Tensor] = None
     if with_bias:
-        b = torch.randn(layer.K, generator=g, dtype=torch.float32).mul_(0.02).half()
-    x, w = x.half(), w.half()
+        b = torch.randn(layer.K, generator=g, dtype=torch.float32).mul_(0.02).to(dtype)
+    x, w = x.to(dtype), w.to(dtype)
     if pin:
         x, w = x.pin_memory(), w.pin_memory()
         b = b.pin_memory() if b is not None else None

@@ -83,6 +83,15 @@ def test_argument_validation_without_gpu(binding):
     assert lib.sdwino_conv3x3_ex(p, p, None, p + 1, p, 1, 4, 8, 8, 4, 2, 1, p, 1 << 20, None) == binding.ERR_MISALIGNED
     assert lib.sdwino_conv3x3_ex(None, p, None, None, p, 1, 4, 8, 8, 4, 2, 1, p, 1 << 20, None) == binding.ERR_INVALID_ARG
     assert lib.sdwino_conv3x3_ex(p, p, None, None, p, 1, 4, 8, 8, 4, 2, 0, None, 0, None) == binding.ERR_WORKSPACE
+    # fp32 interface: the checks come before any CUDA call
+    assert lib.sdwino_filter_transform_f32(None, p, 4, 4, 2, None) == binding.ERR_INVALID_ARG
+    assert lib.sdwino_filter_transform_f32(p, p, 4, 4, 3, None) == binding.ERR_UNSUPPORTED
+    assert lib.sdwino_filter_transform_f32(p + 2, p, 4, 4, 2, None) == binding.ERR_MISALIGNED
+    assert lib.sdwino_conv3x3_f32(None, p, None, p, 1, 4, 8, 8, 4, 2, p, 1 << 20, None) == binding.ERR_INVALID_ARG
+    assert lib.sdwino_conv3x3_f32(p, p, None, p, 1, 4, 8, 8, 4, 5, p, 1 << 20, None) == binding.ERR_UNSUPPORTED
+    assert lib.sdwino_conv3x3_f32(p + 2, p, None, p, 1, 4, 8, 8, 4, 2, p, 1 << 20, None) == binding.ERR_MISALIGNED
+    assert lib.sdwino_conv3x3_f32(p, p, p + 2, p, 1, 4, 8, 8, 4, 2, p, 1 << 20, None) == binding.ERR_MISALIGNED
+    assert lib.sdwino_conv3x3_f32(p, p, None, p, 1, 4, 8, 8, 4, 2, None, 0, None) == binding.ERR_WORKSPACE
     # test hooks reject values outside their range and accept the defaults
     assert lib.sdwino_set_input_staging(3) == binding.ERR_INVALID_ARG
     assert lib.sdwino_set_input_staging(-1) == binding.ERR_INVALID_ARG
