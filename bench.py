@@ -247,16 +247,19 @@ def run_ours(args):
 
     # filter transform: once per weight, outside the timed step; timed on its own
     B.sdwino_profile_enable(True)
-    w_dev = [h[1].to(dev) for h in host]
+    io32 = args.io == "f32"       # the fp32 interface: x, w, bias, y in fp32 (the host arm below stays fp16)
+    io_bytes = 4.0 if io32 else 2.0
+    w_dev = [h[1].to(dev).float() if io32 else h[1].to(dev) for h in host]
     for _ in range(3):
-        wTs = [B.sdwino_filter_transform(wd, t) for wd, t in zip(w_dev, tiles)]
+        wTs = [(B.sdwino_filter_transform_f32 if io32 else B.sdwino_filter_transform)(wd, t) for wd, t in zip(w_dev, tiles)]
         prof = B.sdwino_profile_collect()
     ft_ms = prof["filter_transform"][0]
-    ft_bytes = sum(L.K * L.C * 18 + B.sdwino_filter_bytes(L.K, L.C, t) for L, t in zip(layers, tiles))
+    ft_bytes = sum(L.K * L.C * 9 * io_bytes + B.sdwino_filter_bytes(L.K, L.C, t) for L, t in zip(layers, tiles))
     B.sdwino_profile_enable(False)
     del w_dev
     for (x, w, b, y_h), wT in zip(host, wTs):
-        devt.append((x.to(dev), wT, b.to(dev), torch.empty(y_h.shape, dtype=torch.float16, device=dev)))
+        io_t = torch.float32 if io32 else torch.float16
+        devt.append((x.to(dev).to(io_t), wT, b.to(dev).to(io_t), torch.empty(y_h.shape, dtype=io_t, device=dev)))
     if args.epilogue != "none":
         gres = torch.Generator().manual_seed(1234)
         res_dev = [torch.randn(y_h.shape, generator=gres).half().to(dev) for (_, _, _, y_h) in host]
@@ -264,7 +267,9 @@ def run_ours(args):
 
     def run_layer(li, strm):
         L, t, (xd, wT, bd, yd) = layers[li], tiles[li], devt[li]
-        if args.epilogue == "none" or min(L.C, L.K) <= 8:     # the first and last convolution of a network have neither
+        if io32:
+            B.sdwino_conv3x3_f32(xd, wT, bd, L.K, t, ws, y=yd, stream=strm)
+        elif args.epilogue == "none" or min(L.C, L.K) <= 8:     # the first and last convolution of a network have neither
             B.sdwino_conv3x3(xd, wT, bd, L.K, t, y=yd, workspace=ws, stream=strm)
         else:
             B.sdwino_conv3x3_ex(xd, wT, bd, res_dev[li], L.K, t, act, ws, y=yd, stream=strm)
@@ -302,7 +307,7 @@ def run_ours(args):
 
     # ---- timed region: resident inputs ----
     flops_step = sum(L.direct_flops for L in layers)
-    step_bytes = sum(2.0 * L.N * (L.C + L.K) * L.H * L.W + B.sdwino_filter_bytes(L.K, L.C, t) for L, t in zip(layers, tiles))
+    step_bytes = sum(io_bytes * L.N * (L.C + L.K) * L.H * L.W + B.sdwino_filter_bytes(L.K, L.C, t) for L, t in zip(layers, tiles))
     # A step that touches less than twice the L2 would find its operands cached by the previous step: then
     # the L2 is flushed (a 256 MB buffer is written) before every step and only the steps are timed.
     flush_l2 = step_bytes < 2 * L2_BYTES
@@ -362,7 +367,7 @@ def run_ours(args):
     h2d = sum(x.numel() * 2 + b.numel() * 2 for (x, w, b, y) in host)
     d2h = sum(y.numel() * 2 for (x, w, b, y) in host)
     # what came back through the host path is what the device-resident step computed (same kernels: same bits)
-    e2e_matches = args.epilogue != "none" or all(torch.equal(y_h, yd.cpu()) for (_, _, _, y_h), (_, _, _, yd) in zip(host, devt))
+    e2e_matches = args.epilogue != "none" or io32 or all(torch.equal(y_h, yd.cpu()) for (_, _, _, y_h), (_, _, _, yd) in zip(host, devt))
     assert e2e_matches, "the host path returned something else than the device path"
 
     # ---- per-kernel and per-layer times: a second timed pass with CUDA events around every launch (recorded
@@ -425,7 +430,7 @@ def run_ours(args):
         P = L.tiles(t)
         wino_flops = 2.0 * a2 * L.K * L.C * P
         u_bytes = B.sdwino_filter_bytes(L.K, L.C, t)
-        xb, yb = 2.0 * L.N * L.C * L.H * L.W, 2.0 * L.N * L.K * L.H * L.W
+        xb, yb = io_bytes * L.N * L.C * L.H * L.W, io_bytes * L.N * L.K * L.H * L.W
         t_tensor = wino_flops / (tpeak * 1e12) * 1e6
         t_hbm = (xb + 2.0 * a2 * L.K * L.C + yb + 2 * L.K) / (hpeak * 1e9) * 1e6
         total_us = (pl["input_transform"] + pl["wino_gemm"] + pl["output_transform"] + pl["fused"]) * 1e3
@@ -530,13 +535,15 @@ def run_ours(args):
         line = {
             "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": round(ms_step, 4), "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f16", "data": "synthetic",
-            "config": {"workload": args.workload, "layers": len(layers), "layer_subset": args.layers or "all",
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32 in/out, f16 operands, f32 accumulate" if io32 else "f16",
+            "data": "synthetic",
+            "config": {"workload": args.workload, "io": args.io, "layers": len(layers), "layer_subset": args.layers or "all",
                        "batch": layers[0].N, "tile": args.tile,
                        "tile_per_layer": tiles,
                        "algorithm": ("Winograd F(2x2,3x3) or F(4x4,3x3) per layer (sdwino_choose_tile)"
                                      if args.tile == "auto" else f"Winograd F({args.tile}x{args.tile},3x3)") +
-                                    ", fp16 storage, fp32 accumulate",
+                                    (", fp32 x / w / bias / y, fp16 transformed operands, fp32 accumulate (e2e runs the fp16 interface)"
+                                     if io32 else ", fp16 storage, fp32 accumulate"),
                        "parallelism": f"replicas x{world} (no exchange step)",
                        "launch": "direct" if args.no_graph else "CUDA graph of one step, replayed",
                        "l2": ((f"flushed before every timed step (256 MB written): one step touches only {step_bytes / 1e6:.0f} MB")
@@ -575,6 +582,9 @@ def main():
     ap.add_argument("--workload", default=WORKLOAD, choices=["single", "sd15_unet", "sd_vae_512", "sd21_unet", "sdxl_1024"])
     ap.add_argument("--layers", default="", help="comma-separated layer indices of the workload (default: all)")
     ap.add_argument("--tile", default=TILE, choices=["auto", "2", "4"])
+    ap.add_argument("--io", default="f16", choices=["f16", "f32"],
+                    help="element type of x, w, bias and y in the timed step: f32 runs sdwino_conv3x3_f32 (fp16 operands, "
+                         "fp32 accumulation); the end-to-end arm stays fp16")
     ap.add_argument("--epilogue", default="none", choices=["none", "residual", "residual_silu"],
                     help="fuse y = act(conv + bias + residual) into the output transform of the timed step (sdwino_conv3x3_ex)")
     ap.add_argument("--no-graph", action="store_true", help="launch every step directly instead of replaying a CUDA graph")
