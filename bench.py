@@ -26,6 +26,14 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "direct-conv-equivalent TFLOP/s over the SD v1.5 UNet 3x3 conv sweep (2*N*K*C*H*W*9 / time)"
+_SWEEP_NAMES = {"single": "the single 320->320 at 32x32 layer", "sd15_unet": "the SD v1.5 UNet 3x3 conv sweep",
+                "sd_vae_512": "the SD VAE decoder (512x512) 3x3 conv sweep", "sd21_unet": "the SD v2.1 UNet 3x3 conv sweep",
+                "sdxl_1024": "the SDXL (1024x1024) UNet + VAE decoder 3x3 conv sweep"}
+
+
+def metric_name(workload: str) -> str:
+    """The headline metric, named for the workload that was run (the default is the SD v1.5 sweep)."""
+    return METRIC.replace("the SD v1.5 UNet 3x3 conv sweep", _SWEEP_NAMES[workload])
 UNIT = "TFLOP/s"
 WORKLOAD = "sd15_unet"
 TILE = "auto"   # per layer: what sdwino_choose_tile returns; --tile 2 / --tile 4 force one algorithm
@@ -185,7 +193,7 @@ def run_reference(args):
     val = f_tot / t_tot / 1e12
     sample = f"{nch} seeded output channels of each of the {len(layers)} layers per step (fp64 direct conv)"
     line = {
-        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+        "impl": "reference", "metric": metric_name(args.workload), "value": val, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_tot / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": args.workload, "layers": len(layers), "batch": layers[0].N, "sample": sample},
@@ -533,7 +541,7 @@ def run_ours(args):
 
     if rank == 0:
         line = {
-            "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "metric": metric_name(args.workload), "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": round(ms_step, 4), "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32 in/out, f16 operands, f32 accumulate" if io32 else "f16",
             "data": "synthetic",

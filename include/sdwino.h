@@ -125,8 +125,10 @@ int sdwino_conv3x3_ex(const void *x, const void *wT, const void *bias, const voi
  *
  * sdwino_filter_transform_f32 writes the same wT as sdwino_filter_transform (size sdwino_filter_bytes; U is
  * computed in fp32 from the fp32 weights and rounded once), so the buffer serves either convolution call.
- * sdwino_conv3x3_f32 takes its workspace explicitly (sdwino_workspace_bytes, as for the fp16 calls); layers
- * with very few channels take the general three-kernel path.  Pointers must be 4-byte aligned
+ * sdwino_conv3x3_f32 takes its workspace explicitly (sdwino_workspace_bytes, as for the fp16 calls).  The
+ * single-kernel paths of tile 2 for layers with at most 8 input or output channels serve it too (the one for
+ * few output channels rounds the pixels of x to fp16 as it loads them); with tile 4 such layers take the general
+ * three kernels.  Pointers must be 4-byte aligned
  * (SDWINO_ERR_MISALIGNED); 16-byte aligned x and y with W % 8 == 0 take the vector kernels.  Arguments, errors
  * and asynchrony otherwise as sdwino_filter_transform / sdwino_conv3x3_ws.
  */

@@ -85,10 +85,13 @@ __device__ __forceinline__ FkUnitGeo fk_decode(const TileGeom& geo, int C, long 
     return g;
 }
 
-__device__ __forceinline__ void fk_load(const __half* __restrict__ x, const TileGeom& geo, const FkUnitGeo& g, int c,
+// fp32 x (the fp32 interface): the pixels are rounded to fp16 as they are loaded, into the same packed words the
+// fp16 loads deliver; what follows is the packed fp16 arithmetic of fk_transform either way.
+template <typename XT>
+__device__ __forceinline__ void fk_load(const XT* __restrict__ x, const TileGeom& geo, const FkUnitGeo& g, int c,
                                         bool c_ok, FkRaw& raw) {
     const long long plane = static_cast<long long>(geo.H) * geo.W;
-    const __half* p0 = x + g.base + c * plane;
+    const XT* p0 = x + g.base + c * plane;
 #pragma unroll
     for (int r = 0; r < 4; ++r) {
         const bool ok = c_ok && g.valid && ((g.rows_ok >> r) & 1);
@@ -96,9 +99,17 @@ __device__ __forceinline__ void fk_load(const __half* __restrict__ x, const Tile
         uint32_t lo = 0u, hi = 0u;
         if (ok) {
             const long long off = static_cast<long long>(r) * geo.W;
+            if constexpr (sizeof(XT) == 4) {
+                const float4 a = __ldg(reinterpret_cast<const float4*>(p0 + off));
+                const float4 b = __ldg(reinterpret_cast<const float4*>(p0 + off) + 1);
+                v = make_uint4(pack2(a.x, a.y), pack2(a.z, a.w), pack2(b.x, b.y), pack2(b.z, b.w));
+                if (g.left_ok) lo = pack2(0.f, __ldg(p0 + off - 1));     // the pixel left of the segment in the high half
+                if (g.right_ok) hi = pack2(__ldg(p0 + off + 8), 0.f);    // the pixel right of it in the low half
+            } else {
             v = __ldg(reinterpret_cast<const uint4*>(p0 + off));
             if (g.left_ok) lo = __ldg(reinterpret_cast<const uint32_t*>(p0 + off - 2));
             if (g.right_ok) hi = __ldg(reinterpret_cast<const uint32_t*>(p0 + off + 8));
+            }
         }
         raw.row[r] = v;
         raw.left[r] = lo;
@@ -158,9 +169,10 @@ __device__ __forceinline__ void fk_transform_store(const FkRaw& raw, uint8_t* st
 }
 
 // Grid: x = persistent workers over the 128-tile blocks, y = chunks of 16 output channels.
+template <typename T = __half>   // element type of x, bias and y
 __global__ void __launch_bounds__(FK_THREADS, 1)
-fused_small_k_kernel(const __grid_constant__ CUtensorMap tmU, const __half* __restrict__ x,
-                     const __half* __restrict__ bias, __half* __restrict__ y, FusedKParams prm, int* status_word) {
+fused_small_k_kernel(const __grid_constant__ CUtensorMap tmU, const T* __restrict__ x,
+                     const T* __restrict__ bias, T* __restrict__ y, FusedKParams prm, int* status_word) {
     // The header may have been written by the kernel right before this one: wait for it before anything else.
     // (Uniform early return: no barrier or TMEM has been set up yet.)
     pdl_wait();
@@ -334,7 +346,7 @@ fused_small_k_kernel(const __grid_constant__ CUtensorMap tmU, const __half* __re
             long long n;
             decode_tile(prm.geo, pp, n, th, tw);
             const long long plane = static_cast<long long>(prm.geo.H) * prm.geo.W;
-            __half* out0 = y + (n * prm.K + k0) * plane + static_cast<long long>(2 * th) * prm.geo.W + 2 * tw;
+            T* out0 = y + (n * prm.K + k0) * plane + static_cast<long long>(2 * th) * prm.geo.W + 2 * tw;
             const bool row1_ok = 2 * th + 1 < prm.geo.H;
             const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                                     static_cast<uint32_t>(buf * FK_ACC_COLS);
@@ -370,9 +382,14 @@ fused_small_k_kernel(const __grid_constant__ CUtensorMap tmU, const __half* __re
                     mat_apply<2, 4>(typename Wm::At{}, t[0], o0);
                     mat_apply<2, 4>(typename Wm::At{}, t[1], o1);
                     if (valid) {
-                        __half* q = out0 + (kc + kk) * plane;
-                        *reinterpret_cast<uint32_t*>(q) = pack2(o0[0] + b, o0[1] + b);
-                        if (row1_ok) *reinterpret_cast<uint32_t*>(q + prm.geo.W) = pack2(o1[0] + b, o1[1] + b);
+                        T* q = out0 + (kc + kk) * plane;
+                        if constexpr (sizeof(T) == 4) {
+                            *reinterpret_cast<float2*>(q) = make_float2(o0[0] + b, o0[1] + b);
+                            if (row1_ok) *reinterpret_cast<float2*>(q + prm.geo.W) = make_float2(o1[0] + b, o1[1] + b);
+                        } else {
+                            *reinterpret_cast<uint32_t*>(q) = pack2(o0[0] + b, o0[1] + b);
+                            if (row1_ok) *reinterpret_cast<uint32_t*>(q + prm.geo.W) = pack2(o1[0] + b, o1[1] + b);
+                        }
                     }
                 }
             }

@@ -574,12 +574,13 @@ bool use_fused_small_k(int K, int W, int tile, long long p_tiles, const void* x,
     return tile == 2 && K <= FK_KMAX && p_tiles >= g_fk_min_p_tiles && (W % 8) == 0 && aligned(x, 16) && aligned(y, 4);
 }
 
-int launch_fused_small_k(const __half* x, const void* wT, const __half* bias, __half* y, const Plan& pl, int C, int H,
+template <typename T>
+int launch_fused_small_k(const T* x, const void* wT, const T* bias, T* y, const Plan& pl, int C, int H,
                          int W, int K, cudaStream_t st) {
     const int sms = sm_count();
     if (sms <= 0) return SDWINO_ERR_CUDA;
     int* status = status_word_ptr();
-    if (!status || !ensure_dyn_smem(reinterpret_cast<const void*>(fused_small_k_kernel), FK_DYN_SMEM)) return SDWINO_ERR_CUDA;
+    if (!status || !ensure_dyn_smem(reinterpret_cast<const void*>(fused_small_k_kernel<T>), FK_DYN_SMEM)) return SDWINO_ERR_CUDA;
     CUtensorMap tmU;
     if (!encode_filter_map(&tmU, wt_filters_of(wT), pl.Cb, pl.Kb, pl.a2, 1, 16, FK_KMAX)) return SDWINO_ERR_CUDA;
     FusedKParams prm;
@@ -592,14 +593,15 @@ int launch_fused_small_k(const __half* x, const void* wT, const __half* bias, __
     prm.num_p_tiles = static_cast<int>(pl.P128 / 128);
     const int grid_x = prm.num_p_tiles < sms ? prm.num_p_tiles : sms;
     ProfScope prof(KIND_FUSED, st);
-    const cudaError_t e = launch_pdl(fused_small_k_kernel, dim3(grid_x, (K + FK_KMAX - 1) / FK_KMAX), dim3(FK_THREADS),
+    const cudaError_t e = launch_pdl(fused_small_k_kernel<T>, dim3(grid_x, (K + FK_KMAX - 1) / FK_KMAX), dim3(FK_THREADS),
                                      static_cast<size_t>(FK_DYN_SMEM), st, 1, tmU, x, bias, y, prm, status);
     g_launches.fetch_add(1);
     return e == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
 }
 
 // F(2x2,3x3) layers with at most 8 input channels: one warp-MMA kernel (see fused_small_c_mma_kernel).
-int launch_fused_small_c_mma(const __half* x, const void* wT, const __half* bias, __half* y, const TileGeom& geo, int C,
+template <typename T>
+int launch_fused_small_c_mma(const T* x, const void* wT, const T* bias, T* y, const TileGeom& geo, int C,
                              int K, int Kb, cudaStream_t st) {
     const int sms = sm_count();
     int* status = status_word_ptr();
@@ -616,7 +618,7 @@ int launch_fused_small_c_mma(const __half* x, const void* wT, const __half* bias
     }
     dim3 grid(static_cast<unsigned>(blocks_x), static_cast<unsigned>((Kb + kb_per_block - 1) / kb_per_block));
     ProfScope prof(KIND_FUSED, st);
-    const cudaError_t e = launch_pdl(fused_small_c_mma_kernel, grid, dim3(128), 0, st, 0, x, wt_header_of(wT),
+    const cudaError_t e = launch_pdl(fused_small_c_mma_kernel<T>, grid, dim3(128), 0, st, 0, x, wt_header_of(wT),
                                      static_cast<const __half*>(wt_filters_of(wT)), bias, y, geo, C, K, Kb, kb_per_block,
                                      status);
     g_launches.fetch_add(1);
@@ -746,11 +748,23 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
         const long long lcm = static_cast<long long>(pl.TW) / a * GEMM_BLOCK_P;
         if (pc >= lcm && !io32 && use_input_tma(g0, N, C, x, 0, lcm)) pc = pc / lcm * lcm;
     }
-    // the single-kernel paths end at the bias and read and write fp16
-    const bool plain = ep.residual == nullptr && ep.act == 0 && !io32;
-    if (plain && use_fused_small_k(K, W, tile, pl.P128 / 128, x, y) && !use_fused_small_c(C, tile) && !g_disable_fused)
+    // the single-kernel paths end at the bias
+    const bool no_ep = ep.residual == nullptr && ep.act == 0;
+    const bool plain = no_ep && !io32;
+    if (no_ep && use_fused_small_k(K, W, tile, pl.P128 / 128, x, y) && !use_fused_small_c(C, tile) &&
+        (!io32 || aligned(y, 8)) && !g_disable_fused) {
+        if (io32)
+            return launch_fused_small_k(static_cast<const float*>(x), wT, static_cast<const float*>(bias),
+                                        static_cast<float*>(y), pl, C, H, W, K, st);
         return launch_fused_small_k(static_cast<const __half*>(x), wT, static_cast<const __half*>(bias),
                                     static_cast<__half*>(y), pl, C, H, W, K, st);
+    }
+    if (no_ep && io32 && tile == 2 && use_fused_small_c(C, tile) && !g_disable_fused) {
+        // the F(2x2) kernel for few input channels also serves the fp32 interface (F(4x4): the three kernels)
+        const TileGeom geo = make_geom(H, W, pl.TH, pl.TW, pl.P);
+        return launch_fused_small_c_mma(static_cast<const float*>(x), wT, static_cast<const float*>(bias),
+                                        static_cast<float*>(y), geo, C, K, pl.Kb, st);
+    }
     if (plain && use_fused_small_c(C, tile) && !g_disable_fused) {
         const TileGeom geo = make_geom(H, W, pl.TH, pl.TW, pl.P);
         const __half* xh = static_cast<const __half*>(x);

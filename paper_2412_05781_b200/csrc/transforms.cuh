@@ -977,9 +977,10 @@ __device__ __forceinline__ void mma_m16n8k8_f16f32(float (&d)[4], uint32_t a0, u
 
 // Grid: x = groups of 8 tiles, four per block (one per warp); y = chunks of `kb_per_block` blocks of 16 output
 // channels.  A warp transforms its 8 tiles once and then walks the chunk's output-channel blocks.
+template <typename T = __half>   // element type of x, bias and y
 __global__ void __launch_bounds__(128)
-fused_small_c_mma_kernel(const __half* __restrict__ x, const uint32_t* __restrict__ wt_header,
-                         const __half* __restrict__ U, const __half* __restrict__ bias, __half* __restrict__ y,
+fused_small_c_mma_kernel(const T* __restrict__ x, const uint32_t* __restrict__ wt_header,
+                         const __half* __restrict__ U, const T* __restrict__ bias, T* __restrict__ y,
                          TileGeom geo, int C, int K, int Kb, int kb_per_block, int* status_word) {
     using Wm = Wino<2>;
     pdl_launch_dependents();
@@ -1026,16 +1027,16 @@ fused_small_c_mma_kernel(const __half* __restrict__ x, const uint32_t* __restric
 #pragma unroll
                 for (int s2 = 0; s2 < 4; ++s2) d[r][s2] = 0.f;
             if (p_ok && c < C) {       // the second quad is skipped by every lane when C <= 4
-                const __half* img = x + (n * C + c) * hw;
+                const T* img = x + (n * C + c) * hw;
 #pragma unroll
                 for (int r = 0; r < 4; ++r) {
                     const int i = i0 + r;
                     if (i < 0 || i >= geo.H) continue;
-                    const __half* rowp = img + static_cast<long long>(i) * geo.W;
+                    const T* rowp = img + static_cast<long long>(i) * geo.W;
 #pragma unroll
                     for (int s2 = 0; s2 < 4; ++s2) {
                         const int j = j0 + s2;
-                        if (j >= 0 && j < geo.W) d[r][s2] = __half2float(rowp[j]);
+                        if (j >= 0 && j < geo.W) d[r][s2] = to_f32(rowp[j]);
                     }
                 }
             }
@@ -1085,9 +1086,10 @@ fused_small_c_mma_kernel(const __half* __restrict__ x, const uint32_t* __restric
             col1_ok[jt] = 2 * tw + 1 < geo.W;
         }
     }
-    const bool vec_ok = ((geo.W & 1) == 0) && ((reinterpret_cast<uintptr_t>(y) & 3) == 0);
+    // two pixels (vec_ok) or four (pair_ok) per store: the base of y must be aligned to that many elements
+    const bool vec_ok = ((geo.W & 1) == 0) && ((reinterpret_cast<uintptr_t>(y) & (2 * sizeof(T) - 1)) == 0);
     // W % 4 == 0 makes TW even, so tiles 2t and 2t+1 of a group always share a tile row
-    const bool pair_ok = ((geo.W & 3) == 0) && ((reinterpret_cast<uintptr_t>(y) & 7) == 0) && out_off[1] >= 0;
+    const bool pair_ok = ((geo.W & 3) == 0) && ((reinterpret_cast<uintptr_t>(y) & (4 * sizeof(T) - 1)) == 0) && out_off[1] >= 0;
 
     for (int kb0 = kb_begin; kb0 < kb_end; kb0 += FC_KB_CHUNK) {
     const int chunk = min(FC_KB_CHUNK, kb_end - kb0);
@@ -1132,6 +1134,32 @@ fused_small_c_mma_kernel(const __half* __restrict__ x, const uint32_t* __restric
                 row0[jt] = pack2(o0[jt][0] + b, o0[jt][1] + b);
                 row1[jt] = pack2(o1[jt][0] + b, o1[jt][1] + b);
             }
+            if constexpr (sizeof(T) == 4) {
+                // fp32 output: the same three cases with unrounded values (16-, 8- and 4-byte stores)
+                if (pair_ok) {
+                    float* q = reinterpret_cast<float*>(y) + out_off[0] + k * hw;
+                    *reinterpret_cast<float4*>(q) = make_float4(o0[0][0] + b, o0[0][1] + b, o0[1][0] + b, o0[1][1] + b);
+                    if (row1_ok[0])
+                        *reinterpret_cast<float4*>(q + geo.W) = make_float4(o1[0][0] + b, o1[0][1] + b, o1[1][0] + b, o1[1][1] + b);
+                    continue;
+                }
+#pragma unroll
+                for (int jt = 0; jt < 2; ++jt) {
+                    if (out_off[jt] < 0) continue;
+                    float* q = reinterpret_cast<float*>(y) + out_off[jt] + k * hw;
+                    if (vec_ok) {
+                        *reinterpret_cast<float2*>(q) = make_float2(o0[jt][0] + b, o0[jt][1] + b);
+                        if (row1_ok[jt]) *reinterpret_cast<float2*>(q + geo.W) = make_float2(o1[jt][0] + b, o1[jt][1] + b);
+                    } else {
+                        q[0] = o0[jt][0] + b;
+                        if (col1_ok[jt]) q[1] = o0[jt][1] + b;
+                        if (row1_ok[jt]) {
+                            q[geo.W] = o1[jt][0] + b;
+                            if (col1_ok[jt]) q[geo.W + 1] = o1[jt][1] + b;
+                        }
+                    }
+                }
+            } else {
             if (pair_ok) {
                 // the lane's two tiles are neighbours in one tile row: 4 pixels = one 8-byte store per output row,
                 // and the four lanes of an output channel complete a 32-byte sector
@@ -1156,6 +1184,7 @@ fused_small_c_mma_kernel(const __half* __restrict__ x, const uint32_t* __restric
                     }
                 }
             }
+            }   // fp16 output
         }
     }
     }   // chunks of output-channel blocks

@@ -185,3 +185,72 @@ def test_fp32_interface_sd15_layers_sampled_channels(B, idx):
     ref = oracle.direct_conv3x3(x.numpy(), w.numpy()[ks], b.numpy()[ks])
     got = y[:, ks].double().numpy()
     assert np.abs(got - ref).max() <= TOL * np.abs(ref).max()
+
+
+@pytest.mark.parametrize("shape", [(48, 3, 16, 16, 2), (128, 3, 64, 64, 1), (20, 8, 24, 40, 3), (70, 5, 40, 24, 2)])
+def test_fp32_interface_few_output_channels_fused_kernel(B, shape):
+    # F(2x2) layers with at most 8 output channels take the single tcgen05 kernel (one launch, no workspace
+    # traffic); it rounds the fp32 pixels to fp16 as it loads them.  Same result as the three-kernel path.
+    C, K, H, W, N = shape
+    layer = ConvLayer(C=C, K=K, H=H, W=W, N=N)
+    x, w, b = workloads.make_inputs(layer, seed=sum(shape), dtype=torch.float32)
+    ref = oracle.direct_conv3x3(x.numpy(), w.numpy(), b.numpy())
+    B.sdwino_set_fused_min_tiles(1)
+    try:
+        n0 = B.sdwino_launch_count()
+        y = _run32(B, layer, 2, x, w, b)
+        assert B.sdwino_launch_count() - n0 == 2          # filter transform + the fused kernel
+    finally:
+        B.sdwino_set_fused_min_tiles(0)
+    assert _rel_err(y, ref) <= TOL_F2_REGRESSION
+    B.sdwino_set_gemm_shape(1, 16)                         # forcing a GEMM shape takes the three kernels
+    try:
+        n0 = B.sdwino_launch_count()
+        y3 = _run32(B, layer, 2, x, w, b)
+        assert B.sdwino_launch_count() - n0 == 4
+    finally:
+        B.sdwino_set_gemm_shape(0, 0)
+    assert _rel_err(y3, ref) <= TOL_F2_REGRESSION
+    assert float((y - y3).abs().max()) <= 2 * TOL_F2_REGRESSION * float(np.abs(ref).max())
+    # an 8-byte aligned y is needed for the fused kernel's stores; a 4-byte aligned one takes the three kernels
+    buf = torch.empty(N * K * H * W + 1, device="cuda")
+    yv = buf[1:].view(N, K, H, W)
+    wT = B.sdwino_filter_transform_f32(w.cuda(), 2)
+    ws = B.alloc_workspace(B.sdwino_workspace_bytes(N, C, H, W, K, 2))
+    xd, bd = x.cuda(), b.cuda()
+    rc = B.lib.sdwino_conv3x3_f32(xd.data_ptr(), wT.data_ptr(), bd.data_ptr(), yv.data_ptr(), N, C, H, W, K, 2,
+                                  ws.data_ptr(), ws.numel(), None)
+    assert rc == B.OK and B.sdwino_last_device_status() == B.OK
+    assert _rel_err(yv.cpu(), ref) <= TOL_F2_REGRESSION
+
+
+@pytest.mark.parametrize("shape", [(4, 40, 16, 16, 2), (3, 17, 21, 26, 2), (8, 8, 9, 11, 1), (1, 5, 13, 2, 3), (4, 320, 64, 64, 2)])
+def test_fp32_interface_few_input_channels_fused_kernel(B, shape):
+    # F(2x2) layers with at most 8 input channels take the single warp-MMA kernel: one launch, same result as the
+    # three kernels; widths that are multiples of 4 (16-byte stores), even (8-byte) and odd (4-byte)
+    C, K, H, W, N = shape
+    layer = ConvLayer(C=C, K=K, H=H, W=W, N=N)
+    x, w, b = workloads.make_inputs(layer, seed=sum(shape), dtype=torch.float32)
+    ks = list(range(K)) if K <= 64 else sorted(np.random.default_rng(0).choice(K, 16, replace=False).tolist())
+    ref = oracle.direct_conv3x3(x.numpy(), w.numpy()[ks], b.numpy()[ks])
+    n0 = B.sdwino_launch_count()
+    y = _run32(B, layer, 2, x, w, b)
+    assert B.sdwino_launch_count() - n0 == 2              # filter transform + the fused kernel
+    assert _rel_err(y[:, ks], ref) <= TOL_F2_REGRESSION
+    B.sdwino_set_gemm_shape(1, 16)
+    try:
+        y3 = _run32(B, layer, 2, x, w, b)
+    finally:
+        B.sdwino_set_gemm_shape(0, 0)
+    assert _rel_err(y3[:, ks], ref) <= TOL_F2_REGRESSION
+    assert float((y - y3).abs().max()) <= 2 * TOL_F2_REGRESSION * float(np.abs(ref).max())
+    # y 4-byte aligned only: the scalar stores
+    buf = torch.empty(N * K * H * W + 1, device="cuda")
+    yv = buf[1:].view(N, K, H, W)
+    wT = B.sdwino_filter_transform_f32(w.cuda(), 2)
+    ws = B.alloc_workspace(B.sdwino_workspace_bytes(N, C, H, W, K, 2))
+    xd, bd = x.cuda(), b.cuda()
+    rc = B.lib.sdwino_conv3x3_f32(xd.data_ptr(), wT.data_ptr(), bd.data_ptr(), yv.data_ptr(), N, C, H, W, K, 2,
+                                  ws.data_ptr(), ws.numel(), None)
+    assert rc == B.OK and B.sdwino_last_device_status() == B.OK
+    assert torch.equal(yv.cpu(), y)
