@@ -22,6 +22,10 @@
  * device (SM count, status word, kernel attributes, copy streams of the host path, the built-in scratch of
  * sdwino_conv3x3_static) is set up on first use there, for up to 64 devices per process.  The workspace
  * registered with sdwino_set_workspace and the test hooks are per process.
+ * Threads: the filter transforms and the convolution calls that take their workspace as an argument may be
+ * called from several host threads at once, each on its own stream and workspace (the library's shared state
+ * -- the cache of tensor maps, the per-device facts, the launch counter -- is locked or atomic); functions that
+ * say "not thread-safe" below must not run beside them.
  */
 #ifndef SDWINO_H
 #define SDWINO_H

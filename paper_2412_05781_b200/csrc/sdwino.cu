@@ -82,6 +82,13 @@ constexpr size_t PASS_BUDGET = 4096ull << 20;
 constexpr size_t WS_ALIGN = 1024;
 constexpr int STATIC_MAX_DEVICES_HOST = 64;
 
+// SDWINO_ERR_CUDA, with the place and the runtime's last error on stderr when SDWINO_LOG is set
+int err_cuda(int line) {
+    if (getenv("SDWINO_LOG"))
+        fprintf(stderr, "sdwino: SDWINO_ERR_CUDA at sdwino.cu:%d (last CUDA error: %s)\n", line,
+                cudaGetErrorString(cudaPeekAtLastError()));
+    return SDWINO_ERR_CUDA;
+}
 inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
 inline long long round_up_ll(long long v, long long m) { return (v + m - 1) / m * m; }
 
@@ -128,7 +135,21 @@ long long tiles_per_pass(const Plan& pl, size_t bytes) {
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+int current_device();
+// cuTensorMapEncodeTiled is a driver call and wants a current context (CUDA_ERROR_INVALID_CONTEXT otherwise).  A
+// host thread that has made no runtime call needing one yet -- a fresh worker thread whose first convolution finds
+// everything else cached -- has none: the runtime binds the device's primary context to the thread here, once
+// per thread and device.
+void bind_context_to_thread() {
+    static thread_local int bound_dev = -1;
+    const int dev = current_device();
+    if (dev >= 0 && dev != bound_dev) {
+        cudaFree(nullptr);
+        bound_dev = dev;
+    }
+}
 EncodeTiledFn get_encode_fn() {
+    bind_context_to_thread();
     static EncodeTiledFn fn = nullptr;
     static std::once_flag once;
     std::call_once(once, [] {
@@ -186,6 +207,10 @@ bool encode_map_uncached(CUtensorMap* m, const void* base, uint64_t d0, uint64_t
                     CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS && getenv("SDWINO_LOG"))
+        fprintf(stderr, "sdwino: cuTensorMapEncodeTiled failed (%d): base %p dims %llu %llu %llu pitch %llu %llu box %u %u sw %d\n",
+                static_cast<int>(r), base, (unsigned long long)d0, (unsigned long long)d1, (unsigned long long)d2,
+                (unsigned long long)pitch0, (unsigned long long)pitch1, b0, b1, swizzle128 ? 1 : 0);
     return r == CUDA_SUCCESS;
 }
 
@@ -209,8 +234,12 @@ bool encode_filter_map(CUtensorMap* m, const void* base, uint64_t Cb, uint64_t K
     cuuint32_t estr[5] = {1, 1, 1, 1, 1};
     if (fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 5, const_cast<void*>(base), dims, strides, box, estr,
            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) {
+        if (getenv("SDWINO_LOG"))
+            fprintf(stderr, "sdwino: cuTensorMapEncodeTiled failed for the filters: base %p Cb %llu Kb %llu positions %llu box %u %u %u\n",
+                    base, (unsigned long long)Cb, (unsigned long long)Kb, (unsigned long long)npos, krows, kblocks, posbox);
         return false;
+    }
     slot.key = key;
     slot.map = *m;
     slot.used = true;
@@ -318,7 +347,11 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
     }
     cfg.attrs = attr;
     cfg.numAttrs = n;
-    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+    if (e != cudaSuccess && getenv("SDWINO_LOG"))
+        fprintf(stderr, "sdwino: kernel launch failed: %s (grid %u x %u, block %u, %zu bytes of dynamic shared memory)\n",
+                cudaGetErrorString(e), grid.x, grid.y, block.x, smem);
+    return e;
 }
 
 template <int M, typename WT>
@@ -329,7 +362,7 @@ int launch_filter(const WT* w, void* wT, int K, int C, int Kb, int Cb, cudaStrea
     __half* U = reinterpret_cast<__half*>(static_cast<uint8_t*>(wT) + WT_HEADER_BYTES);
     const cudaError_t e = launch_pdl(filter_transform_kernel<M, WT>, grid, dim3(128), 0, st, 0, w, header, U, K, C, Kb, Cb);
     g_launches.fetch_add(1);
-    return e == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
+    return e == cudaSuccess ? SDWINO_OK : err_cuda(__LINE__);
 }
 
 template <int M, typename XT>
@@ -356,7 +389,7 @@ int launch_input(const XT* x, __half* V, const TileGeom& geo, int C, long long p
         e = launch_pdl(input_transform_kernel<M, XT>, grid, dim3(128), 0, st, 0, x, V, geo, C, p_begin, p_count, Pstride);
     }
     g_launches.fetch_add(1);
-    return e == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
+    return e == cudaSuccess ? SDWINO_OK : err_cuda(__LINE__);
 }
 
 
@@ -384,7 +417,7 @@ int launch_input_tma(const __half* x, __half* V, const TileGeom& geo, int N, int
     ProfScope prof(KIND_INPUT, st);
     const int sms = sm_count();
     int* status = status_word_ptr();
-    if (sms <= 0 || !status) return SDWINO_ERR_CUDA;
+    if (sms <= 0 || !status) return err_cuda(__LINE__);
     InTmaParams q;
     q.C = C; q.TH = geo.TH; q.TW = geo.TW; q.Pstride = Pstride;
     q.p_begin = p_begin;
@@ -450,16 +483,16 @@ int launch_input_tma(const __half* x, __half* V, const TileGeom& geo, int N, int
     const long long grid_y = (csteps + steps - 1) / steps;
     if (blocks >= (1ll << 31) || grid_y > 65535) return SDWINO_ERR_UNSUPPORTED;
     CUtensorMap tmX;
-    if (!encode_image_map(&tmX, x, geo.W, geo.H, static_cast<uint64_t>(N) * C, q.bw, q.bh, q.cpb)) return SDWINO_ERR_CUDA;
+    if (!encode_image_map(&tmX, x, geo.W, geo.H, static_cast<uint64_t>(N) * C, q.bw, q.bh, q.cpb)) return err_cuda(__LINE__);
     const size_t smem = static_cast<size_t>(IN_TMA_STAGES) * q.stage_bytes + 128;
     if (smem > IN_TMA_STAGES * 32 * 1024 + 128 ||
         !ensure_dyn_smem(reinterpret_cast<const void*>(input_transform_f4_tma_kernel), IN_TMA_STAGES * 32 * 1024 + 128))
-        return SDWINO_ERR_CUDA;
+        return err_cuda(__LINE__);
     dim3 grid(static_cast<unsigned>(blocks), static_cast<unsigned>(grid_y));
     const cudaError_t e = launch_pdl(input_transform_f4_tma_kernel, grid, dim3(IN_TMA_THREADS), smem, st, 0, tmX, V, q,
                                      status);
     g_launches.fetch_add(1);
-    return e == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
+    return e == cudaSuccess ? SDWINO_OK : err_cuda(__LINE__);
 }
 
 // The TMA-staged F(4x4) output transform: see output_tma.cuh.
@@ -477,10 +510,10 @@ int launch_output_tma(const __half* Mws, const YT* bias, YT* y, const TileGeom& 
     ProfScope prof(KIND_OUTPUT, st);
     const int sms = sm_count();
     int* status = status_word_ptr();
-    if (sms <= 0 || !status) return SDWINO_ERR_CUDA;
+    if (sms <= 0 || !status) return err_cuda(__LINE__);
     CUtensorMap tmM;
     if (!encode_image_map(&tmM, Mws, static_cast<uint64_t>(Pstride), static_cast<uint64_t>(K), 36, OUT_TMA_TILES, 1, 36))
-        return SDWINO_ERR_CUDA;
+        return err_cuda(__LINE__);
     const long long blocks = (p_count + OUT_TMA_TILES - 1) / OUT_TMA_TILES;
     // channels per CTA (at most 16): three CTAs are resident per SM; the time follows the SM with the most
     // CTA-steps (one more step per CTA for the fill)
@@ -497,10 +530,10 @@ int launch_output_tma(const __half* Mws, const YT* bias, YT* y, const TileGeom& 
     const size_t smem = static_cast<size_t>(OUT_TMA_STAGES) * OUT_TMA_STAGE_BYTES + 128;
     if (blocks >= (1ll << 31) ||
         !ensure_dyn_smem(reinterpret_cast<const void*>(output_transform_f4_tma_kernel<false, YT>), static_cast<int>(smem)))
-        return SDWINO_ERR_CUDA;
+        return err_cuda(__LINE__);
     if constexpr (sizeof(YT) == 2) {
         if (!ensure_dyn_smem(reinterpret_cast<const void*>(output_transform_f4_tma_kernel<true>), static_cast<int>(smem)))
-            return SDWINO_ERR_CUDA;
+            return err_cuda(__LINE__);
     }
     dim3 grid(static_cast<unsigned>(blocks), static_cast<unsigned>((K + steps - 1) / steps));
     cudaError_t e;
@@ -515,7 +548,7 @@ int launch_output_tma(const __half* Mws, const YT* bias, YT* y, const TileGeom& 
             return SDWINO_ERR_UNSUPPORTED;   // the fused residual / activation is part of the fp16 interface
     }
     g_launches.fetch_add(1);
-    return e == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
+    return e == cudaSuccess ? SDWINO_OK : err_cuda(__LINE__);
 }
 
 template <int M, typename YT>
@@ -544,7 +577,7 @@ int launch_output(const __half* Mws, const YT* bias, YT* y, const TileGeom& geo,
                        Pstride, chk, ep);
     }
     g_launches.fetch_add(1);
-    return e == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
+    return e == cudaSuccess ? SDWINO_OK : err_cuda(__LINE__);
 }
 
 // Layers with at most 8 (tile 2) or 4 (tile 4) input channels run as one fused kernel without a workspace.
@@ -554,13 +587,13 @@ template <int M, int CP>
 int launch_fused_small_c(const __half* x, const void* wT, const __half* bias, __half* y, const TileGeom& geo, int C,
                          int K, int Kb, int Cb, cudaStream_t st) {
     int* status = status_word_ptr();
-    if (!status) return SDWINO_ERR_CUDA;
+    if (!status) return err_cuda(__LINE__);
     dim3 grid(static_cast<unsigned>((geo.P + 127) / 128), (K + FUSED_KC - 1) / FUSED_KC);
     ProfScope prof(KIND_FUSED, st);
     const cudaError_t e = launch_pdl(fused_small_c_kernel<M, CP>, grid, dim3(128), 0, st, 0, x, wt_header_of(wT),
                                      static_cast<const __half*>(wt_filters_of(wT)), bias, y, geo, C, K, Kb, Cb, status);
     g_launches.fetch_add(1);
-    return e == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
+    return e == cudaSuccess ? SDWINO_OK : err_cuda(__LINE__);
 }
 
 // Layers with at most 8 output channels run F(2x2,3x3) as one fused tensor-core kernel (no workspace traffic):
@@ -578,11 +611,11 @@ template <typename T>
 int launch_fused_small_k(const T* x, const void* wT, const T* bias, T* y, const Plan& pl, int C, int H,
                          int W, int K, cudaStream_t st) {
     const int sms = sm_count();
-    if (sms <= 0) return SDWINO_ERR_CUDA;
+    if (sms <= 0) return err_cuda(__LINE__);
     int* status = status_word_ptr();
-    if (!status || !ensure_dyn_smem(reinterpret_cast<const void*>(fused_small_k_kernel<T>), FK_DYN_SMEM)) return SDWINO_ERR_CUDA;
+    if (!status || !ensure_dyn_smem(reinterpret_cast<const void*>(fused_small_k_kernel<T>), FK_DYN_SMEM)) return err_cuda(__LINE__);
     CUtensorMap tmU;
-    if (!encode_filter_map(&tmU, wt_filters_of(wT), pl.Cb, pl.Kb, pl.a2, 1, 16, FK_KMAX)) return SDWINO_ERR_CUDA;
+    if (!encode_filter_map(&tmU, wt_filters_of(wT), pl.Cb, pl.Kb, pl.a2, 1, 16, FK_KMAX)) return err_cuda(__LINE__);
     FusedKParams prm;
     prm.wt_header = wt_header_of(wT);
     prm.geo = make_geom(H, W, pl.TH, pl.TW, pl.P);
@@ -596,7 +629,7 @@ int launch_fused_small_k(const T* x, const void* wT, const T* bias, T* y, const 
     const cudaError_t e = launch_pdl(fused_small_k_kernel<T>, dim3(grid_x, (K + FK_KMAX - 1) / FK_KMAX), dim3(FK_THREADS),
                                      static_cast<size_t>(FK_DYN_SMEM), st, 1, tmU, x, bias, y, prm, status);
     g_launches.fetch_add(1);
-    return e == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
+    return e == cudaSuccess ? SDWINO_OK : err_cuda(__LINE__);
 }
 
 // F(2x2,3x3) layers with at most 8 input channels: one warp-MMA kernel (see fused_small_c_mma_kernel).
@@ -605,7 +638,7 @@ int launch_fused_small_c_mma(const T* x, const void* wT, const T* bias, T* y, co
                              int K, int Kb, cudaStream_t st) {
     const int sms = sm_count();
     int* status = status_word_ptr();
-    if (sms <= 0 || !status) return SDWINO_ERR_CUDA;
+    if (sms <= 0 || !status) return err_cuda(__LINE__);
     const long long groups = (geo.P + 7) / 8;
     const long long blocks_x = (groups + 3) / 4;
     // The kernel is a latency chain per warp (load, transform, then per block of output channels MMAs, output
@@ -622,7 +655,7 @@ int launch_fused_small_c_mma(const T* x, const void* wT, const T* bias, T* y, co
                                      static_cast<const __half*>(wt_filters_of(wT)), bias, y, geo, C, K, Kb, kb_per_block,
                                      status);
     g_launches.fetch_add(1);
-    return e == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
+    return e == cudaSuccess ? SDWINO_OK : err_cuda(__LINE__);
 }
 
 // Shape of the GEMM launch: CTA pairs or single CTAs, and the output channels per tile (UMMA N, a
@@ -693,7 +726,7 @@ template <int CTAS, bool RES, bool DUAL = false>
 int launch_gemm_shape(const CUtensorMap& tmU, const CUtensorMap& tmV, const CUtensorMap& tmM, const GemmParams& prm,
                       int sms, int* status, cudaStream_t st) {
     using L = GemmSmemLayout;
-    if (!ensure_dyn_smem(reinterpret_cast<const void*>(wino_gemm_kernel<CTAS, RES, DUAL>), MAX_DYN_SMEM)) return SDWINO_ERR_CUDA;
+    if (!ensure_dyn_smem(reinterpret_cast<const void*>(wino_gemm_kernel<CTAS, RES, DUAL>), MAX_DYN_SMEM)) return err_cuda(__LINE__);
     const long long tiles = static_cast<long long>(prm.num_k_tiles) * prm.num_p_tiles * prm.num_pos;
     const long long workers = sms / CTAS;
     const int grid = static_cast<int>(tiles < workers ? tiles : workers) * CTAS;
@@ -708,15 +741,15 @@ int launch_gemm_shape(const CUtensorMap& tmU, const CUtensorMap& tmV, const CUte
         fprintf(stderr, "sdwino: GEMM launch failed: %s (grid %d, stages %d, n_tile %d, resident %d)\n", cudaGetErrorString(e),
                 grid, prm.stages, prm.n_tile, prm.resident);
     g_launches.fetch_add(1);
-    return e == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
+    return e == cudaSuccess ? SDWINO_OK : err_cuda(__LINE__);
 }
 
 int launch_gemm(const CUtensorMap& tmU, const CUtensorMap& tmV, const CUtensorMap& tmM, const GemmParams& prm,
                 int ctas, cudaStream_t st) {
     const int sms = sm_count();
-    if (sms <= 0) return SDWINO_ERR_CUDA;
+    if (sms <= 0) return err_cuda(__LINE__);
     int* status = status_word_ptr();
-    if (!status) return SDWINO_ERR_CUDA;
+    if (!status) return err_cuda(__LINE__);
     if (ctas == 2) return launch_gemm_shape<2, false>(tmU, tmV, tmM, prm, sms, status, st);
     if (prm.resident) return launch_gemm_shape<1, true>(tmU, tmV, tmM, prm, sms, status, st);
     if (prm.dual) return launch_gemm_shape<1, false, true>(tmU, tmV, tmM, prm, sms, status, st);
@@ -784,7 +817,7 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
     if (v_bytes + m_bytes > ws_bytes) return SDWINO_ERR_WORKSPACE;
 
     const int sms = sm_count();
-    if (sms <= 0) return SDWINO_ERR_CUDA;
+    if (sms <= 0) return err_cuda(__LINE__);
     GemmParams prm;
     prm.wt_header = wt_header_of(wT);
     prm.K = K;
@@ -855,14 +888,14 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
     if (!encode_filter_map(&tmU, wt_filters_of(wT), pl.Cb, pl.Kb, pl.a2, b_rows / 16) ||
         !encode_map(&tmV, V, pc, C, pl.a2, pc, static_cast<uint64_t>(C) * pc, 64, GEMM_BLOCK_C, true) ||
         !encode_map(&tmM, Mws, pc, K, pl.a2, pc, static_cast<uint64_t>(K) * pc, GEMM_BLOCK_P, prm.epi_rows, false))
-        return SDWINO_ERR_CUDA;
+        return err_cuda(__LINE__);
 
     const TileGeom geo = make_geom(H, W, pl.TH, pl.TW, pl.P);
     const __half* xh = static_cast<const __half*>(x);
     const __half* bh = static_cast<const __half*>(bias);
     __half* yh = static_cast<__half*>(y);
     const WtCheck chk{wt_header_of(wT), K, C, tile, status_word_ptr()};
-    if (!chk.status_word) return SDWINO_ERR_CUDA;
+    if (!chk.status_word) return err_cuda(__LINE__);
     for (long long p0 = 0; p0 < pl.P; p0 += pc) {
         long long remaining = pl.P128 - p0;
         const int count = static_cast<int>(remaining < pc ? remaining : pc);  // multiple of 128
@@ -1097,7 +1130,7 @@ int sdwino_conv3x3_host_async(const void* x_host, const void* wT, const void* bi
     if (!workspace || workspace_bytes <= staging) return SDWINO_ERR_WORKSPACE;
     if (!aligned(workspace, WS_ALIGN)) return SDWINO_ERR_MISALIGNED;
     HostPipe* hp = host_pipe();
-    if (!hp) return SDWINO_ERR_CUDA;
+    if (!hp) return err_cuda(__LINE__);
     auto up = [](size_t v) { return (v + WS_ALIGN - 1) / WS_ALIGN * WS_ALIGN; };
     const size_t xbytes = static_cast<size_t>(N) * C * H * W * sizeof(__half);
     const size_t ybytes = static_cast<size_t>(N) * K * H * W * sizeof(__half);
@@ -1124,14 +1157,14 @@ int sdwino_conv3x3_host_async(const void* x_host, const void* wT, const void* bi
                 if (cudaEventQuery(e.downloaded) != cudaSuccess &&
                     (cudaStreamWaitEvent(hp->s_in, e.computed, 0) != cudaSuccess ||
                      cudaStreamWaitEvent(st, e.downloaded, 0) != cudaSuccess))
-                    return SDWINO_ERR_CUDA;
+                    return err_cuda(__LINE__);
                 waited_same_slot = true;
             }
         } else {
             if (cudaStreamWaitEvent(hp->s_in, e.computed, 0) != cudaSuccess ||
                 cudaStreamWaitEvent(hp->s_in, e.downloaded, 0) != cudaSuccess ||
                 cudaStreamWaitEvent(st, e.downloaded, 0) != cudaSuccess)
-                return SDWINO_ERR_CUDA;
+                return err_cuda(__LINE__);
         }
     }
     if (slot < 0) slot = 0;
@@ -1141,7 +1174,7 @@ int sdwino_conv3x3_host_async(const void* x_host, const void* wT, const void* bi
     if (me.used && cudaEventQuery(me.downloaded) != cudaSuccess &&   // its download is its last operation
         (cudaStreamWaitEvent(hp->s_in, me.downloaded, 0) != cudaSuccess ||
          cudaStreamWaitEvent(st, me.downloaded, 0) != cudaSuccess))
-        return SDWINO_ERR_CUDA;
+        return err_cuda(__LINE__);
     me.used = false;
 
     uint8_t* xd = base + slot * up(xbytes);
@@ -1149,19 +1182,19 @@ int sdwino_conv3x3_host_async(const void* x_host, const void* wT, const void* bi
     uint8_t* yd = base + 2 * (up(xbytes) + up(bbytes)) + slot * up(ybytes);
     uint8_t* ws = base + staging;
     // upload on the first copy stream
-    if (cudaMemcpyAsync(xd, x_host, xbytes, cudaMemcpyHostToDevice, hp->s_in) != cudaSuccess) return SDWINO_ERR_CUDA;
+    if (cudaMemcpyAsync(xd, x_host, xbytes, cudaMemcpyHostToDevice, hp->s_in) != cudaSuccess) return err_cuda(__LINE__);
     if (bias_host && cudaMemcpyAsync(bd, bias_host, bbytes, cudaMemcpyHostToDevice, hp->s_in) != cudaSuccess)
-        return SDWINO_ERR_CUDA;
-    if (cudaEventRecord(me.uploaded, hp->s_in) != cudaSuccess) return SDWINO_ERR_CUDA;
+        return err_cuda(__LINE__);
+    if (cudaEventRecord(me.uploaded, hp->s_in) != cudaSuccess) return err_cuda(__LINE__);
     // kernels on the caller's stream
-    if (cudaStreamWaitEvent(st, me.uploaded, 0) != cudaSuccess) return SDWINO_ERR_CUDA;
+    if (cudaStreamWaitEvent(st, me.uploaded, 0) != cudaSuccess) return err_cuda(__LINE__);
     const int rc = conv_impl(xd, wT, bias_host ? bd : nullptr, yd, N, C, H, W, K, tile, ws, workspace_bytes - staging, st);
     if (rc != SDWINO_OK) return rc;
-    if (cudaEventRecord(me.computed, st) != cudaSuccess) return SDWINO_ERR_CUDA;
+    if (cudaEventRecord(me.computed, st) != cudaSuccess) return err_cuda(__LINE__);
     // download on the second copy stream
-    if (cudaStreamWaitEvent(hp->s_out, me.computed, 0) != cudaSuccess) return SDWINO_ERR_CUDA;
-    if (cudaMemcpyAsync(y_host, yd, ybytes, cudaMemcpyDeviceToHost, hp->s_out) != cudaSuccess) return SDWINO_ERR_CUDA;
-    if (cudaEventRecord(me.downloaded, hp->s_out) != cudaSuccess) return SDWINO_ERR_CUDA;
+    if (cudaStreamWaitEvent(hp->s_out, me.computed, 0) != cudaSuccess) return err_cuda(__LINE__);
+    if (cudaMemcpyAsync(y_host, yd, ybytes, cudaMemcpyDeviceToHost, hp->s_out) != cudaSuccess) return err_cuda(__LINE__);
+    if (cudaEventRecord(me.downloaded, hp->s_out) != cudaSuccess) return err_cuda(__LINE__);
     me.used = true;
     me.begin = base;
     me.end = base + workspace_bytes;
@@ -1175,12 +1208,12 @@ int sdwino_conv3x3_host_async(const void* x_host, const void* wT, const void* bi
 
 int sdwino_host_join(void* stream) {
     HostPipe* hp = host_pipe();
-    if (!hp) return SDWINO_ERR_CUDA;
+    if (!hp) return err_cuda(__LINE__);
     if (hp->calls == 0) return SDWINO_OK;
     // the download stream works in order: the newest download is the last one to finish
     const HostCall& last = hp->ring[(hp->calls - 1) % HOST_RING];
     if (last.used && cudaStreamWaitEvent(static_cast<cudaStream_t>(stream), last.downloaded, 0) != cudaSuccess)
-        return SDWINO_ERR_CUDA;
+        return err_cuda(__LINE__);
     return SDWINO_OK;
 }
 
@@ -1189,18 +1222,18 @@ int sdwino_conv3x3_host(const void* x_host, const void* wT, const void* bias_hos
     const int rc = sdwino_conv3x3_host_async(x_host, wT, bias_host, y_host, N, C, H, W, K, tile, workspace,
                                              workspace_bytes, stream);
     if (rc != SDWINO_OK) return rc;
-    if (sdwino_host_join(stream) != SDWINO_OK) return SDWINO_ERR_CUDA;
-    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return SDWINO_ERR_CUDA;
+    if (sdwino_host_join(stream) != SDWINO_OK) return err_cuda(__LINE__);
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return err_cuda(__LINE__);
     return SDWINO_OK;
 }
 
 int sdwino_last_device_status(void* stream) {
-    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return SDWINO_ERR_CUDA;
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return err_cuda(__LINE__);
     int v = 0;
-    if (cudaMemcpyFromSymbol(&v, g_status_word, sizeof(int)) != cudaSuccess) return SDWINO_ERR_CUDA;
+    if (cudaMemcpyFromSymbol(&v, g_status_word, sizeof(int)) != cudaSuccess) return err_cuda(__LINE__);
     if (v != 0) {
         int zero = 0;
-        if (cudaMemcpyToSymbol(g_status_word, &zero, sizeof(int)) != cudaSuccess) return SDWINO_ERR_CUDA;
+        if (cudaMemcpyToSymbol(g_status_word, &zero, sizeof(int)) != cudaSuccess) return err_cuda(__LINE__);
         if (getenv("SDWINO_LOG")) fprintf(stderr, "sdwino: device status word 0x%x\n", v);
     }
     return v & 0xFF;
@@ -1211,10 +1244,10 @@ unsigned long long sdwino_launch_count(void) { return g_launches.load(); }
 int sdwino_selftest_wait_timeout(unsigned long long limit_ns, void* stream) {
     if (limit_ns == 0 || limit_ns > 10000000ull) return SDWINO_ERR_INVALID_ARG;   // at most 10 ms
     int* status = nullptr;
-    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&status), g_status_word) != cudaSuccess) return SDWINO_ERR_CUDA;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&status), g_status_word) != cudaSuccess) return err_cuda(__LINE__);
     wait_timeout_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(status, limit_ns);
     g_launches.fetch_add(1);
-    return cudaGetLastError() == cudaSuccess ? SDWINO_OK : SDWINO_ERR_CUDA;
+    return cudaGetLastError() == cudaSuccess ? SDWINO_OK : err_cuda(__LINE__);
 }
 
 }  // extern "C"
@@ -1240,7 +1273,7 @@ int sdwino_conv3x3_static(const void* x, const void* wT, const void* bias, void*
     Plan pl;
     if (!x || !wT || !y || !make_plan(N, C, H, W, K, tile, &pl)) return SDWINO_ERR_INVALID_ARG;
     int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess) return SDWINO_ERR_CUDA;
+    if (cudaGetDevice(&dev) != cudaSuccess) return err_cuda(__LINE__);
     if (dev < 0 || dev >= STATIC_MAX_DEVICES) return SDWINO_ERR_UNSUPPORTED;
     void* base = nullptr;
     {
@@ -1248,7 +1281,7 @@ int sdwino_conv3x3_static(const void* x, const void* wT, const void* bias, void*
         if (!g_static_scratch_ptr[dev]) {
             // set-up, once per device, with that device current
             void* p = nullptr;
-            if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return SDWINO_ERR_CUDA;
+            if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return err_cuda(__LINE__);
             g_static_scratch_ptr[dev] = p;
         }
         base = g_static_scratch_ptr[dev];

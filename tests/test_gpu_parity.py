@@ -776,3 +776,49 @@ def test_seeded_random_layers_against_plain_kernels_and_oracle(B, shape):
     ks = sorted(rng.choice(K, min(K, 4), replace=False).tolist())
     ref = oracle.direct_conv3x3(x.numpy(), w.numpy(), b.numpy(), channels=ks)
     assert np.abs(y_auto[:, ks].cpu().double().numpy() - ref).max() <= TOL * np.abs(ref).max()
+
+
+def test_concurrent_host_threads_on_their_own_streams(B):
+    # compute calls with an explicit workspace may come from several host threads at once (ctypes releases the
+    # interpreter lock during a call): each thread has its own stream, workspace and layer; the results are the bits
+    # of the same calls made one after the other
+    import threading
+    shapes = [((72, 200, 50, 46, 2), 2), ((64, 48, 64, 64, 2), 4), ((4, 40, 16, 16, 2), 2), ((130, 257, 33, 35, 1), 4),
+              ((48, 3, 64, 64, 2), 2), ((320, 320, 32, 32, 1), 2)]
+    jobs = []
+    for i, (shape, tile) in enumerate(shapes):
+        C, K, H, W, N = shape
+        layer = ConvLayer(C=C, K=K, H=H, W=W, N=N)
+        x, w, b = workloads.make_inputs(layer, seed=40 + i)
+        wT = B.sdwino_filter_transform(w.cuda(), tile)
+        ws = B.alloc_workspace(B.sdwino_workspace_bytes(N, C, H, W, K, tile))
+        jobs.append((layer, tile, x.cuda(), wT, b.cuda(), ws))
+    torch.cuda.synchronize()
+    serial = [B.sdwino_conv3x3(xd, wT, bd, layer.K, tile, workspace=ws).clone() for layer, tile, xd, wT, bd, ws in jobs]
+    torch.cuda.synchronize()
+    results = [None] * len(jobs)
+    errors = []
+    start = threading.Barrier(len(jobs))
+
+    def work(i):
+        try:
+            layer, tile, xd, wT, bd, ws = jobs[i]
+            st = torch.cuda.Stream()
+            y = torch.empty_like(serial[i])
+            start.wait()
+            for _ in range(25):
+                B.sdwino_conv3x3(xd, wT, bd, layer.K, tile, y=y, workspace=ws, stream=st)
+            st.synchronize()
+            results[i] = y
+        except Exception as e:   # noqa: BLE001
+            errors.append((i, repr(e)))
+
+    threads = [threading.Thread(target=work, args=(i,)) for i in range(len(jobs))]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    assert B.sdwino_last_device_status() == B.OK
+    for i in range(len(jobs)):
+        assert torch.equal(results[i], serial[i]), shapes[i]
