@@ -135,21 +135,7 @@ long long tiles_per_pass(const Plan& pl, size_t bytes) {
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-int current_device();
-// cuTensorMapEncodeTiled is a driver call and wants a current context (CUDA_ERROR_INVALID_CONTEXT otherwise).  A
-// host thread that has made no runtime call needing one yet -- a fresh worker thread whose first convolution finds
-// everything else cached -- has none: the runtime binds the device's primary context to the thread here, once
-// per thread and device.
-void bind_context_to_thread() {
-    static thread_local int bound_dev = -1;
-    const int dev = current_device();
-    if (dev >= 0 && dev != bound_dev) {
-        cudaFree(nullptr);
-        bound_dev = dev;
-    }
-}
 EncodeTiledFn get_encode_fn() {
-    bind_context_to_thread();
     static EncodeTiledFn fn = nullptr;
     static std::once_flag once;
     std::call_once(once, [] {
@@ -160,6 +146,26 @@ EncodeTiledFn get_encode_fn() {
             fn = reinterpret_cast<EncodeTiledFn>(p);
     });
     return fn;
+}
+
+// cuTensorMapEncodeTiled (fp16, no interleave, 256-byte L2 promotion, no NaN fill).  It is a driver call and wants a
+// current context: a host thread that has made no runtime call needing one yet -- a fresh worker thread whose first
+// convolution finds everything else cached -- has none and gets CUDA_ERROR_INVALID_CONTEXT.  Then, and only then
+// (a thread that is capturing a stream has a context, and cudaFree is not allowed inside a capture), the runtime
+// is asked to bind the device's primary context to the thread and the call is repeated.
+CUresult encode_tiled(CUtensorMap* m, cuuint32_t rank, const void* base, const cuuint64_t* dims, const cuuint64_t* strides,
+                      const cuuint32_t* box, const cuuint32_t* estr, CUtensorMapSwizzle swizzle) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return CUDA_ERROR_NOT_INITIALIZED;
+    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, rank, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r == CUDA_ERROR_INVALID_CONTEXT) {
+        cudaFree(nullptr);
+        r = fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, rank, const_cast<void*>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    }
+    return r;
 }
 
 // fp16 tensor [d2][d1][d0] (d0 contiguous, row pitch `pitch0` elements, plane pitch `pitch1`
@@ -197,16 +203,12 @@ bool encode_map(CUtensorMap* m, const void* base, uint64_t d0, uint64_t d1, uint
 
 bool encode_map_uncached(CUtensorMap* m, const void* base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t pitch0,
                          uint64_t pitch1, uint32_t b0, uint32_t b1, bool swizzle128) {
-    EncodeTiledFn fn = get_encode_fn();
-    if (!fn) return false;
     cuuint64_t dims[3] = {d0, d1, d2};
     cuuint64_t strides[2] = {pitch0 * sizeof(__half), pitch1 * sizeof(__half)};
     cuuint32_t box[3] = {b0, b1, 1};
     cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
-                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    const CUresult r = encode_tiled(m, 3, base, dims, strides, box, estr,
+                                    swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE);
     if (r != CUDA_SUCCESS && getenv("SDWINO_LOG"))
         fprintf(stderr, "sdwino: cuTensorMapEncodeTiled failed (%d): base %p dims %llu %llu %llu pitch %llu %llu box %u %u sw %d\n",
                 static_cast<int>(r), base, (unsigned long long)d0, (unsigned long long)d1, (unsigned long long)d2,
@@ -226,15 +228,11 @@ bool encode_filter_map(CUtensorMap* m, const void* base, uint64_t Cb, uint64_t K
     MapSlot& slot = g_map_cache[h % MAP_CACHE_SLOTS];
     std::lock_guard<std::mutex> lock(g_map_mutex);
     if (slot.used && slot.key == key) { *m = slot.map; return true; }
-    EncodeTiledFn fn = get_encode_fn();
-    if (!fn) return false;
     cuuint64_t dims[5] = {64, 16, Cb, Kb, npos};
     cuuint64_t strides[4] = {128, 2048 * Kb, 2048, Kb * Cb * 2048};   // memory order [pos][Cb][Kb][16][64]
     cuuint32_t box[5] = {64, krows, 1, kblocks, posbox};
     cuuint32_t estr[5] = {1, 1, 1, 1, 1};
-    if (fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 5, const_cast<void*>(base), dims, strides, box, estr,
-           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) {
+    if (encode_tiled(m, 5, base, dims, strides, box, estr, CU_TENSOR_MAP_SWIZZLE_128B) != CUDA_SUCCESS) {
         if (getenv("SDWINO_LOG"))
             fprintf(stderr, "sdwino: cuTensorMapEncodeTiled failed for the filters: base %p Cb %llu Kb %llu positions %llu box %u %u %u\n",
                     base, (unsigned long long)Cb, (unsigned long long)Kb, (unsigned long long)npos, krows, kblocks, posbox);
@@ -303,16 +301,11 @@ bool encode_image_map(CUtensorMap* m, const void* base, uint64_t W, uint64_t H, 
     MapSlot& slot = g_map_cache[h % MAP_CACHE_SLOTS];
     std::lock_guard<std::mutex> lock(g_map_mutex);
     if (slot.used && slot.key == key) { *m = slot.map; return true; }
-    EncodeTiledFn fn = get_encode_fn();
-    if (!fn) return false;
     cuuint64_t dims[3] = {W, H, NC};
     cuuint64_t strides[2] = {W * sizeof(__half), H * W * sizeof(__half)};
     cuuint32_t box[3] = {bw, bh, cpb};
     cuuint32_t estr[3] = {1, 1, 1};
-    if (fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
-           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-        return false;
+    if (encode_tiled(m, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_SWIZZLE_NONE) != CUDA_SUCCESS) return false;
     slot.key = key;
     slot.map = *m;
     slot.used = true;

@@ -822,3 +822,32 @@ def test_concurrent_host_threads_on_their_own_streams(B):
     assert B.sdwino_last_device_status() == B.OK
     for i in range(len(jobs)):
         assert torch.equal(results[i], serial[i]), shapes[i]
+
+
+@pytest.mark.parametrize("shape,tile", [((64, 48, 64, 64, 2), 4), ((72, 200, 50, 46, 2), 2), ((4, 40, 16, 16, 2), 2),
+                                        ((48, 3, 64, 64, 8), 2)])
+def test_first_call_inside_a_stream_capture_and_graph_replay(B, shape, tile):
+    # the calls of a layer captured into a CUDA graph as the very first calls on their buffers (tensor maps not yet
+    # cached: they are encoded during the capture, which must not disturb it), then replayed on new inputs
+    C, K, H, W, N = shape
+    layer = ConvLayer(C=C, K=K, H=H, W=W, N=N)
+    x, w, b = workloads.make_inputs(layer, seed=77)
+    wT = B.sdwino_filter_transform(w.cuda(), tile)
+    ws = B.alloc_workspace(B.sdwino_workspace_bytes(N, C, H, W, K, tile) + 4096)[4096 - 1024:]   # an address no test used
+    xd, bd = torch.zeros_like(x, device="cuda"), b.cuda()
+    y = torch.empty(N, K, H, W, dtype=torch.float16, device="cuda")
+    torch.cuda.synchronize()
+    st = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=st):
+        B.sdwino_conv3x3(xd, wT, bd, K, tile, y=y, workspace=ws, stream=torch.cuda.current_stream())
+    ref = oracle.direct_conv3x3(x.numpy(), w.numpy(), b.numpy())
+    for rep in range(2):
+        y.zero_()
+        xd.copy_(x.cuda() if rep == 0 else (2 * x).cuda())
+        torch.cuda.synchronize()
+        g.replay()
+        torch.cuda.synchronize()
+        assert B.sdwino_last_device_status() == B.OK
+        want = ref if rep == 0 else 2 * (ref - b.double().numpy()[None, :, None, None]) + b.double().numpy()[None, :, None, None]
+        assert _rel_err(y.cpu(), want) <= (TOL_F2_REGRESSION if tile == 2 else TOL)
