@@ -347,9 +347,16 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
     return e;
 }
 
+// A grid of x by `rows` blocks: grid.y holds at most 65535 rows, the rest continue along grid.z (the kernels
+// number their rows blockIdx.z * gridDim.y + blockIdx.y and skip those past the end).
+inline dim3 grid_rows(unsigned x, long long rows) {
+    if (rows <= 65535) return dim3(x, static_cast<unsigned>(rows), 1);
+    return dim3(x, 65535, static_cast<unsigned>((rows + 65534) / 65535));
+}
+
 template <int M, typename WT>
 int launch_filter(const WT* w, void* wT, int K, int C, int Kb, int Cb, cudaStream_t st) {
-    dim3 grid((Cb * 32 + 127) / 128, Kb * 16);   // a thread transforms two neighbouring input channels
+    const dim3 grid = grid_rows((Cb * 32 + 127) / 128, static_cast<long long>(Kb) * 16);   // a thread transforms two neighbouring input channels
     ProfScope prof(KIND_FILTER, st);
     uint32_t* header = static_cast<uint32_t*>(wT);
     __half* U = reinterpret_cast<__half*>(static_cast<uint8_t*>(wT) + WT_HEADER_BYTES);
@@ -378,7 +385,7 @@ int launch_input(const XT* x, __half* V, const TileGeom& geo, int C, long long p
                            make_fastdiv(static_cast<uint32_t>(p_count / TPT)), Pstride);
         }
     } else {
-        dim3 grid((p_count + 127) / 128, C);
+        const dim3 grid = grid_rows((p_count + 127) / 128, C);
         e = launch_pdl(input_transform_kernel<M, XT>, grid, dim3(128), 0, st, 0, x, V, geo, C, p_begin, p_count, Pstride);
     }
     g_launches.fetch_add(1);
@@ -565,7 +572,7 @@ int launch_output(const __half* Mws, const YT* bias, YT* y, const TileGeom& geo,
                 return SDWINO_ERR_UNSUPPORTED;
         }
     } else {
-        dim3 grid((p_count + 127) / 128, K);
+        const dim3 grid = grid_rows((p_count + 127) / 128, K);
         e = launch_pdl(output_transform_kernel<M, YT>, grid, dim3(128), 0, st, 0, Mws, bias, y, geo, K, p_begin, p_count,
                        Pstride, chk, ep);
     }
@@ -581,7 +588,7 @@ int launch_fused_small_c(const __half* x, const void* wT, const __half* bias, __
                          int K, int Kb, int Cb, cudaStream_t st) {
     int* status = status_word_ptr();
     if (!status) return err_cuda(__LINE__);
-    dim3 grid(static_cast<unsigned>((geo.P + 127) / 128), (K + FUSED_KC - 1) / FUSED_KC);
+    const dim3 grid = grid_rows(static_cast<unsigned>((geo.P + 127) / 128), (K + FUSED_KC - 1) / FUSED_KC);
     ProfScope prof(KIND_FUSED, st);
     const cudaError_t e = launch_pdl(fused_small_c_kernel<M, CP>, grid, dim3(128), 0, st, 0, x, wt_header_of(wT),
                                      static_cast<const __half*>(wt_filters_of(wT)), bias, y, geo, C, K, Kb, Cb, status);

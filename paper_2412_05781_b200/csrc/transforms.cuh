@@ -154,9 +154,12 @@ filter_transform_kernel(const WT* __restrict__ w, uint32_t* __restrict__ header,
     constexpr int A = Wm::A;
     pdl_launch_dependents();
     pdl_wait();
-    const int c = (blockIdx.x * blockDim.x + threadIdx.x) * 2;   // two neighbouring input channels: 4-byte stores
-    const int k = blockIdx.y;                                    // (four per thread measured slower again)
-    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0)
+    // two neighbouring input channels per thread: 4-byte stores (four per thread measured slower again)
+    const int c = (blockIdx.x * blockDim.x + threadIdx.x) * 2;
+    // one row of blocks per output channel; more than 65535 rows continue along grid.z
+    const int k = static_cast<int>(blockIdx.z * gridDim.y + blockIdx.y);
+    if (k >= Kb * 16) return;
+    if (blockIdx.x == 0 && k == 0 && threadIdx.x == 0)
         *reinterpret_cast<uint4*>(header) = make_uint4(WT_MAGIC, static_cast<uint32_t>(K), static_cast<uint32_t>(C),
                                                        static_cast<uint32_t>(M));
     if (c >= Cb * 64) return;
@@ -251,8 +254,8 @@ input_transform_kernel(const XT* __restrict__ x, __half* __restrict__ V, TileGeo
     pdl_wait();
     pdl_launch_dependents();
     const int pl = blockIdx.x * blockDim.x + threadIdx.x;  // chunk-local tile
-    const int c = blockIdx.y;
-    if (pl >= p_count) return;
+    const int c = static_cast<int>(blockIdx.z * gridDim.y + blockIdx.y);   // grid.z continues grid.y past 65535
+    if (pl >= p_count || c >= C) return;
     const long long p = p_begin + pl;
     float d[A][A];
     if (p < geo.P) {
@@ -327,8 +330,8 @@ output_transform_kernel(const __half* __restrict__ Mws, const YT* __restrict__ b
     pdl_wait();
     if (!wt_ok) return;
     const int pl = blockIdx.x * blockDim.x + threadIdx.x;
-    const int k = blockIdx.y;
-    if (pl >= p_count) return;
+    const int k = static_cast<int>(blockIdx.z * gridDim.y + blockIdx.y);   // grid.z continues grid.y past 65535
+    if (pl >= p_count || k >= K) return;
     const long long p = p_begin + pl;
     if (p >= geo.P) return;
     const long long plane = static_cast<long long>(K) * Pstride;
@@ -845,7 +848,8 @@ fused_small_c_kernel(const __half* __restrict__ x, const uint32_t* __restrict__ 
     pdl_launch_dependents();
     pdl_wait();
     if (!wt_header_ok(wt_header, K, C, M, status_word)) return;
-    const int k0 = blockIdx.y * FUSED_KC;
+    const int k0 = static_cast<int>(blockIdx.z * gridDim.y + blockIdx.y) * FUSED_KC;   // grid.z continues grid.y
+    if (k0 >= K) return;
     // stage the filter chunk: U[pos][Cb][Kb][16][64], this layer has Cb == 1
     const size_t plane = static_cast<size_t>(Kb) * Cb * 1024;
     for (int i = threadIdx.x; i < FUSED_KC * CP * A2; i += blockDim.x) {

@@ -851,3 +851,20 @@ def test_first_call_inside_a_stream_capture_and_graph_replay(B, shape, tile):
         assert B.sdwino_last_device_status() == B.OK
         want = ref if rep == 0 else 2 * (ref - b.double().numpy()[None, :, None, None]) + b.double().numpy()[None, :, None, None]
         assert _rel_err(y.cpu(), want) <= (TOL_F2_REGRESSION if tile == 2 else TOL)
+
+
+@pytest.mark.parametrize("shape", [(1, 70000, 3, 3, 1), (70000, 1, 3, 3, 1), (16, 70000, 8, 8, 1), (70000, 16, 8, 8, 1),
+                                   (3, 5, 2, 2, 70000), (9, 9, 3, 70000, 1), (4, 70000, 5, 5, 1)])
+@pytest.mark.parametrize("tile", [2, 4])
+def test_more_than_65535_channels_images_or_columns(B, shape, tile):
+    # one dimension past the 65535 limit of grid.y / grid.z: the kernels that spend a row of blocks per channel
+    # continue along grid.z; 8 sampled output channels against the oracle
+    C, K, H, W, N = shape
+    layer = ConvLayer(C=C, K=K, H=H, W=W, N=N)
+    x, w, b = workloads.make_inputs(layer, seed=9)
+    _, _, _, y = _run(B, layer, tile, x=x, w=w, b=b)
+    ks = sorted(np.random.default_rng(1).choice(K, min(K, 8), replace=False).tolist())
+    if K > 8:
+        ks[-1] = K - 1                       # the last channel sits in the last row of blocks
+    ref = oracle.direct_conv3x3(x.numpy(), w.numpy()[ks], b.numpy()[ks])
+    assert _rel_err(y[:, ks], ref) <= (TOL_F2_REGRESSION if tile == 2 else TOL)
