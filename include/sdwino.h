@@ -140,6 +140,11 @@ int sdwino_filter_transform_f32(const float *w, void *wT, int K, int C, int tile
 int sdwino_conv3x3_f32(const float *x, const void *wT, const float *bias, float *y,
                        int N, int C, int H, int W, int K, int tile,
                        void *workspace, size_t workspace_bytes, void *stream);
+/* y = act(conv3x3(x) + bias + residual) with fp32 tensors: sdwino_conv3x3_ex for the fp32 interface (residual fp32
+ * [N][K][H][W] or NULL, may be y itself; activation SDWINO_ACT_NONE or SDWINO_ACT_SILU; nothing is rounded). */
+int sdwino_conv3x3_f32_ex(const float *x, const void *wT, const float *bias, const float *residual, float *y,
+                          int N, int C, int H, int W, int K, int tile, int activation,
+                          void *workspace, size_t workspace_bytes, void *stream);
 
 /*
  * The convolution for callers that must not allocate device memory.  (The paper has no

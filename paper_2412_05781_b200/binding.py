@@ -23,7 +23,7 @@ EXPORTS = [
     "sdwino_last_device_status", "sdwino_launch_count", "sdwino_profile_enable", "sdwino_profile_collect",
     "sdwino_profile_records", "sdwino_set_gemm_shape", "sdwino_conv3x3_static", "sdwino_set_fused_min_tiles", "sdwino_choose_tile",
     "sdwino_selftest_wait_timeout", "sdwino_conv3x3_host_async", "sdwino_host_join", "sdwino_set_input_staging", "sdwino_conv3x3_ex",
-    "sdwino_filter_transform_f32", "sdwino_conv3x3_f32",
+    "sdwino_filter_transform_f32", "sdwino_conv3x3_f32", "sdwino_conv3x3_f32_ex",
 ]
 
 KERNEL_KINDS = ("filter_transform", "input_transform", "wino_gemm", "output_transform", "fused")
@@ -66,6 +66,8 @@ def _load() -> ctypes.CDLL:
     lib.sdwino_filter_transform_f32.argtypes = [vp, vp, i, i, i, vp]
     lib.sdwino_conv3x3_f32.restype = i
     lib.sdwino_conv3x3_f32.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, vp, sz, vp]
+    lib.sdwino_conv3x3_f32_ex.restype = i
+    lib.sdwino_conv3x3_f32_ex.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, i, vp, sz, vp]
     lib.sdwino_conv3x3_host.restype = i
     lib.sdwino_conv3x3_host.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, vp, sz, vp]
     lib.sdwino_host_join.restype = i
@@ -301,6 +303,27 @@ def sdwino_conv3x3_f32(x: torch.Tensor, wT: torch.Tensor, bias: Optional[torch.T
                                 workspace.data_ptr(), workspace.numel() * workspace.element_size(),
                                 _stream_ptr(stream))
     _check(rc, "sdwino_conv3x3_f32")
+    return y
+
+
+def sdwino_conv3x3_f32_ex(x: torch.Tensor, wT: torch.Tensor, bias: Optional[torch.Tensor], residual: Optional[torch.Tensor],
+                          K: int, tile: int, activation: int, workspace: torch.Tensor, y: Optional[torch.Tensor] = None,
+                          stream=None) -> torch.Tensor:
+    """y = act(conv3x3(x) + bias + residual) with fp32 tensors (residual may be y itself)."""
+    assert x.is_cuda and x.dtype == torch.float32 and x.is_contiguous() and x.dim() == 4
+    N, C, H, W = (int(v) for v in x.shape)
+    if y is None:
+        y = torch.empty((N, K, H, W), dtype=torch.float32, device=x.device)
+    assert y.is_cuda and y.is_contiguous() and y.dtype == torch.float32 and tuple(y.shape) == (N, K, H, W)
+    if bias is not None:
+        assert bias.is_cuda and bias.dtype == torch.float32 and bias.numel() == K and bias.is_contiguous()
+    if residual is not None:
+        assert residual.is_cuda and residual.dtype == torch.float32 and residual.is_contiguous()
+        assert tuple(residual.shape) == (N, K, H, W)
+    rc = lib.sdwino_conv3x3_f32_ex(x.data_ptr(), wT.data_ptr(), _ptr(bias), _ptr(residual), y.data_ptr(), N, C, H, W, K,
+                                   tile, int(activation), workspace.data_ptr(),
+                                   workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    _check(rc, "sdwino_conv3x3_f32_ex")
     return y
 
 

@@ -104,12 +104,13 @@ output_transform_f4_tma_kernel(const __grid_constant__ CUtensorMap tmM, const YT
         const float b = load_bias(bias, k);
         YT* img = y + (n * K + k) * hw + pix;
         uint4 res[M];
-        if constexpr (EP) {
+        if constexpr (EP && sizeof(YT) == 2) {
 #pragma unroll
             for (int i = 0; i < M; ++i) {
                 res[i] = make_uint4(0u, 0u, 0u, 0u);
                 if (ep.residual && i0 + i < geo.H)
-                    res[i] = __ldg(reinterpret_cast<const uint4*>(ep.residual + (img - y) + static_cast<long long>(i) * geo.W));
+                    res[i] = __ldg(reinterpret_cast<const uint4*>(static_cast<const __half*>(ep.residual) + (img - y) +
+                                                                   static_cast<long long>(i) * geo.W));
             }
         }
 #pragma unroll
@@ -118,7 +119,7 @@ output_transform_f4_tma_kernel(const __grid_constant__ CUtensorMap tmM, const YT
             at4_packed(tt[i], o);
             if (i0 + i >= geo.H) continue;
             float v[8] = {o[0].x + b, o[1].x + b, o[2].x + b, o[3].x + b, o[0].y + b, o[1].y + b, o[2].y + b, o[3].y + b};
-            store_row8<EP>(img + static_cast<long long>(i) * geo.W, v, res[i], ep);
+            store_row8<EP>(img + static_cast<long long>(i) * geo.W, v, res[i], ep, y);
         }
     }
     if (abort_flag != 0) {

@@ -531,21 +531,16 @@ int launch_output_tma(const __half* Mws, const YT* bias, YT* y, const TileGeom& 
     if (blocks >= (1ll << 31) ||
         !ensure_dyn_smem(reinterpret_cast<const void*>(output_transform_f4_tma_kernel<false, YT>), static_cast<int>(smem)))
         return err_cuda(__LINE__);
-    if constexpr (sizeof(YT) == 2) {
-        if (!ensure_dyn_smem(reinterpret_cast<const void*>(output_transform_f4_tma_kernel<true>), static_cast<int>(smem)))
-            return err_cuda(__LINE__);
-    }
+    if (!ensure_dyn_smem(reinterpret_cast<const void*>(output_transform_f4_tma_kernel<true, YT>), static_cast<int>(smem)))
+        return err_cuda(__LINE__);
     dim3 grid(static_cast<unsigned>(blocks), static_cast<unsigned>((K + steps - 1) / steps));
     cudaError_t e;
     if (ep.residual == nullptr && ep.act == 0) {
         e = launch_pdl(output_transform_f4_tma_kernel<false, YT>, grid, dim3(OUT_TMA_THREADS), smem, st, 0, tmM, bias, y, geo, K,
                        p_begin, static_cast<int>(steps), chk, ep, status);
     } else {
-        if constexpr (sizeof(YT) == 2)
-            e = launch_pdl(output_transform_f4_tma_kernel<true>, grid, dim3(OUT_TMA_THREADS), smem, st, 0, tmM, bias, y, geo, K,
-                           p_begin, static_cast<int>(steps), chk, ep, status);
-        else
-            return SDWINO_ERR_UNSUPPORTED;   // the fused residual / activation is part of the fp16 interface
+        e = launch_pdl(output_transform_f4_tma_kernel<true, YT>, grid, dim3(OUT_TMA_THREADS), smem, st, 0, tmM, bias, y, geo, K,
+                       p_begin, static_cast<int>(steps), chk, ep, status);
     }
     g_launches.fetch_add(1);
     return e == cudaSuccess ? SDWINO_OK : err_cuda(__LINE__);
@@ -565,11 +560,8 @@ int launch_output(const __half* Mws, const YT* bias, YT* y, const TileGeom& geo,
             e = launch_pdl(output_transform_vec_kernel<M, TPT, false, YT>, grid, dim3(128), 0, st, 0, Mws, bias, y, geo, K,
                            p_begin, make_fastdiv(static_cast<uint32_t>(p_count / TPT)), Pstride, chk, ep);
         } else {
-            if constexpr (sizeof(YT) == 2)
-                e = launch_pdl(output_transform_vec_kernel<M, TPT, true>, grid, dim3(128), 0, st, 0, Mws, bias, y, geo, K,
-                               p_begin, make_fastdiv(static_cast<uint32_t>(p_count / TPT)), Pstride, chk, ep);
-            else
-                return SDWINO_ERR_UNSUPPORTED;
+            e = launch_pdl(output_transform_vec_kernel<M, TPT, true, YT>, grid, dim3(128), 0, st, 0, Mws, bias, y, geo, K,
+                           p_begin, make_fastdiv(static_cast<uint32_t>(p_count / TPT)), Pstride, chk, ep);
         }
     } else {
         const dim3 grid = grid_rows((p_count + 127) / 128, K);
@@ -1048,13 +1040,22 @@ int sdwino_conv3x3_ex(const void* x, const void* wT, const void* bias, const voi
     if (activation != SDWINO_ACT_NONE && activation != SDWINO_ACT_SILU) return SDWINO_ERR_UNSUPPORTED;
     if (residual && !aligned(residual, 2)) return SDWINO_ERR_MISALIGNED;
     return conv_impl(x, wT, bias, y, N, C, H, W, K, tile, workspace, workspace_bytes, static_cast<cudaStream_t>(stream),
-                     Epilogue{static_cast<const __half*>(residual), activation});
+                     Epilogue{residual, activation});
 }
 
 int sdwino_conv3x3_f32(const float* x, const void* wT, const float* bias, float* y, int N, int C, int H, int W, int K,
                        int tile, void* workspace, size_t workspace_bytes, void* stream) {
     return conv_impl(x, wT, bias, y, N, C, H, W, K, tile, workspace, workspace_bytes, static_cast<cudaStream_t>(stream),
                      Epilogue{nullptr, 0}, true);
+}
+
+int sdwino_conv3x3_f32_ex(const float* x, const void* wT, const float* bias, const float* residual, float* y, int N,
+                          int C, int H, int W, int K, int tile, int activation, void* workspace, size_t workspace_bytes,
+                          void* stream) {
+    if (activation != SDWINO_ACT_NONE && activation != SDWINO_ACT_SILU) return SDWINO_ERR_UNSUPPORTED;
+    if (residual && !aligned(residual, 4)) return SDWINO_ERR_MISALIGNED;
+    return conv_impl(x, wT, bias, y, N, C, H, W, K, tile, workspace, workspace_bytes, static_cast<cudaStream_t>(stream),
+                     Epilogue{residual, activation}, true);
 }
 
 int sdwino_conv3x3(const void* x, const void* wT, const void* bias, void* y, int N, int C, int H, int W, int K,

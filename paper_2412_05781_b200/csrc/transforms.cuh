@@ -308,7 +308,7 @@ input_transform_kernel(const XT* __restrict__ x, __half* __restrict__ V, TileGeo
 // passes over y that cost nothing extra here.  residual: fp16 [N][K][H][W] or null (may be y itself);
 // act: 0 none, 1 SiLU z / (1 + exp(-z)).
 struct Epilogue {
-    const __half* residual;
+    const void* residual;   // element type of y
     int act;
 };
 __device__ __forceinline__ float epilogue_act(float v, int act) {
@@ -367,13 +367,19 @@ output_transform_kernel(const __half* __restrict__ Mws, const YT* __restrict__ b
         if (oi >= geo.H) continue;
         if constexpr (sizeof(YT) == 4) {   // fp32 output: no residual, no activation, no rounding
             float* rowf = reinterpret_cast<float*>(img) + static_cast<long long>(oi) * geo.W + j0;
+            const float* resf = ep.residual ? static_cast<const float*>(ep.residual) + (rowf - reinterpret_cast<float*>(y))
+                                            : nullptr;
 #pragma unroll
             for (int j = 0; j < M; ++j)
-                if (j0 + j < geo.W) rowf[j] = o[j] + b;
+                if (j0 + j < geo.W) {
+                    float v = o[j] + b;
+                    if (resf) v += resf[j];
+                    rowf[j] = epilogue_act(v, ep.act);
+                }
             continue;
         } else {
         __half* rowp = img + static_cast<long long>(oi) * geo.W + j0;
-        const __half* resp = ep.residual ? ep.residual + (rowp - y) : nullptr;
+        const __half* resp = ep.residual ? static_cast<const __half*>(ep.residual) + (rowp - y) : nullptr;
 #pragma unroll
         for (int j = 0; j < M; j += 2) {
             float v0 = o[j] + b, v1 = o[j + 1] + b;
@@ -666,7 +672,8 @@ input_transform_f4_kernel(const XT* __restrict__ x, __half* __restrict__ V, Tile
 // Eight output pixels of one row (bias already added): residual (its eight values loaded by the caller, ahead of
 // the arithmetic), activation, one rounding, one 16-byte store.
 template <bool EP>
-__device__ __forceinline__ void store_row8(__half* rowp, float (&v)[8], const uint4& r, const Epilogue& ep) {
+__device__ __forceinline__ void store_row8(__half* rowp, float (&v)[8], const uint4& r, const Epilogue& ep,
+                                           const __half* = nullptr) {
     if constexpr (EP) {
     if (ep.residual) {
         float a, b2;
@@ -688,10 +695,23 @@ __device__ __forceinline__ void store_row8(__half* rowp, float (&v)[8], const ui
     *reinterpret_cast<uint4*>(rowp) = w;
 }
 
-// fp32 output: eight pixels are two 16-byte stores; there is no residual, activation or rounding
+// fp32 output: eight pixels are two 16-byte stores, not rounded; the residual row (same offset from ybase as rowp)
+// is loaded here
 template <bool EP>
-__device__ __forceinline__ void store_row8(float* rowp, float (&v)[8], const uint4&, const Epilogue&) {
-    static_assert(!EP, "the fused residual / activation is part of the fp16 interface");
+__device__ __forceinline__ void store_row8(float* rowp, float (&v)[8], const uint4&, const Epilogue& ep,
+                                           const float* ybase = nullptr) {
+    if constexpr (EP) {
+        if (ep.residual) {
+            const float4* rp = reinterpret_cast<const float4*>(static_cast<const float*>(ep.residual) + (rowp - ybase));
+            const float4 a = __ldg(rp), b = __ldg(rp + 1);
+            v[0] += a.x; v[1] += a.y; v[2] += a.z; v[3] += a.w;
+            v[4] += b.x; v[5] += b.y; v[6] += b.z; v[7] += b.w;
+        }
+        if (ep.act != 0) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) v[i] = epilogue_act(v[i], ep.act);
+        }
+    }
     reinterpret_cast<float4*>(rowp)[0] = make_float4(v[0], v[1], v[2], v[3]);
     reinterpret_cast<float4*>(rowp)[1] = make_float4(v[4], v[5], v[6], v[7]);
 }
@@ -732,12 +752,12 @@ __device__ __forceinline__ void output_unit_vec(const __half* __restrict__ Mws, 
         YT* img = y + (n * K + k) * static_cast<long long>(geo.H) * geo.W;
         const int i0 = M * th, j0 = M * tw;
         uint4 res[M];
-        if constexpr (EP) {
+        if constexpr (EP && sizeof(YT) == 2) {
 #pragma unroll
             for (int i = 0; i < M; ++i) {
                 res[i] = make_uint4(0u, 0u, 0u, 0u);
                 if (ep.residual && i0 + i < geo.H)
-                    res[i] = __ldg(reinterpret_cast<const uint4*>(ep.residual + (img - y) +
+                    res[i] = __ldg(reinterpret_cast<const uint4*>(static_cast<const __half*>(ep.residual) + (img - y) +
                                                                    static_cast<long long>(i0 + i) * geo.W + j0));
             }
         }
@@ -748,7 +768,7 @@ __device__ __forceinline__ void output_unit_vec(const __half* __restrict__ Mws, 
             if (i0 + i >= geo.H) continue;
             float v[8] = {o[0].x + b, o[1].x + b, o[2].x + b, o[3].x + b, o[0].y + b, o[1].y + b, o[2].y + b, o[3].y + b};
             YT* rowp = img + static_cast<long long>(i0 + i) * geo.W + j0;
-            store_row8<EP>(rowp, v, res[i], ep);
+            store_row8<EP>(rowp, v, res[i], ep, y);
         }
     } else {
     float mm[A][A][TPT];
@@ -773,12 +793,12 @@ __device__ __forceinline__ void output_unit_vec(const __half* __restrict__ Mws, 
     YT* img = y + (n * K + k) * static_cast<long long>(geo.H) * geo.W;
     const int i0 = M * th, j0 = M * tw;
     uint4 res[M];
-    if constexpr (EP) {
+    if constexpr (EP && sizeof(YT) == 2) {
 #pragma unroll
         for (int i = 0; i < M; ++i) {
             res[i] = make_uint4(0u, 0u, 0u, 0u);
             if (ep.residual && i0 + i < geo.H)
-                res[i] = __ldg(reinterpret_cast<const uint4*>(ep.residual + (img - y) +
+                res[i] = __ldg(reinterpret_cast<const uint4*>(static_cast<const __half*>(ep.residual) + (img - y) +
                                                                static_cast<long long>(i0 + i) * geo.W + j0));
         }
     }
@@ -806,7 +826,7 @@ __device__ __forceinline__ void output_unit_vec(const __half* __restrict__ Mws, 
 #pragma unroll
     for (int i = 0; i < M; ++i) {
         if (i0 + i >= geo.H) continue;
-        store_row8<EP>(img + static_cast<long long>(i0 + i) * geo.W + j0, out[i], res[i], ep);
+        store_row8<EP>(img + static_cast<long long>(i0 + i) * geo.W + j0, out[i], res[i], ep, y);
     }
     }   // M != 4
 }

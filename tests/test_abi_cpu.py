@@ -92,6 +92,9 @@ def test_argument_validation_without_gpu(binding):
     assert lib.sdwino_conv3x3_f32(p + 2, p, None, p, 1, 4, 8, 8, 4, 2, p, 1 << 20, None) == binding.ERR_MISALIGNED
     assert lib.sdwino_conv3x3_f32(p, p, p + 2, p, 1, 4, 8, 8, 4, 2, p, 1 << 20, None) == binding.ERR_MISALIGNED
     assert lib.sdwino_conv3x3_f32(p, p, None, p, 1, 4, 8, 8, 4, 2, None, 0, None) == binding.ERR_WORKSPACE
+    assert lib.sdwino_conv3x3_f32_ex(p, p, None, None, p, 1, 4, 8, 8, 4, 2, 7, p, 1 << 20, None) == binding.ERR_UNSUPPORTED
+    assert lib.sdwino_conv3x3_f32_ex(p, p, None, p + 2, p, 1, 4, 8, 8, 4, 2, 1, p, 1 << 20, None) == binding.ERR_MISALIGNED
+    assert lib.sdwino_conv3x3_f32_ex(None, p, None, None, p, 1, 4, 8, 8, 4, 2, 1, p, 1 << 20, None) == binding.ERR_INVALID_ARG
     # test hooks reject values outside their range and accept the defaults
     assert lib.sdwino_set_input_staging(3) == binding.ERR_INVALID_ARG
     assert lib.sdwino_set_input_staging(-1) == binding.ERR_INVALID_ARG

@@ -254,3 +254,43 @@ def test_fp32_interface_few_input_channels_fused_kernel(B, shape):
                                   ws.data_ptr(), ws.numel(), None)
     assert rc == B.OK and B.sdwino_last_device_status() == B.OK
     assert torch.equal(yv.cpu(), y)
+
+
+@pytest.mark.parametrize("act", ["none", "silu"])
+@pytest.mark.parametrize("shape,tile", [((32, 48, 16, 16, 2), 2), ((32, 48, 16, 16, 2), 4), ((20, 24, 9, 11, 1), 2),
+                                        ((20, 24, 9, 11, 1), 4), ((4, 40, 12, 16, 1), 2), ((40, 4, 12, 16, 2), 2),
+                                        ((64, 64, 64, 64, 1), 4), ((17, 33, 13, 24, 3), 4)])
+def test_fp32_interface_fused_residual_and_activation(B, shape, tile, act):
+    # y = act(conv + bias + residual), all fp32: vector, scalar and TMA-staged output kernels, both tiles, layers that
+    # would otherwise take a single-kernel path, the residual aliasing y
+    C, K, H, W, N = shape
+    layer = ConvLayer(C=C, K=K, H=H, W=W, N=N)
+    x, w, b = workloads.make_inputs(layer, seed=sum(shape) + tile, dtype=torch.float32)
+    g = torch.Generator().manual_seed(99)
+    res = torch.randn((N, K, H, W), generator=g)
+    name = "silu" if act == "silu" else None
+    ref = oracle.epilogue(oracle.direct_conv3x3(x.numpy(), w.numpy(), b.numpy()), res.numpy(), name)
+    wT = B.sdwino_filter_transform_f32(w.cuda(), tile)
+    ws = B.alloc_workspace(B.sdwino_workspace_bytes(N, C, H, W, K, tile))
+    flag = B.ACT_SILU if act == "silu" else B.ACT_NONE
+    xd, bd = x.cuda(), b.cuda()
+    y = B.sdwino_conv3x3_f32_ex(xd, wT, bd, res.cuda(), K, tile, flag, ws)
+    assert B.sdwino_last_device_status() == B.OK and y.dtype == torch.float32
+    assert _rel_err(y.cpu(), ref) <= TOL
+    y2 = res.cuda().clone()                                  # in place: the residual is y
+    B.sdwino_conv3x3_f32_ex(xd, wT, bd, y2, K, tile, flag, ws, y=y2)
+    assert torch.equal(y2, y)
+    y3 = B.sdwino_conv3x3_f32_ex(xd, wT, None, None, K, tile, flag, ws)      # no residual, no bias
+    ref3 = oracle.epilogue(oracle.direct_conv3x3(x.numpy(), w.numpy(), None), None, name)
+    assert _rel_err(y3.cpu(), ref3) <= TOL
+    if act == "none":
+        # the epilogue adds exactly the residual to what the three kernels of the plain call compute
+        B.sdwino_set_gemm_shape(1, 0)      # keeps the plain call off the single-kernel paths
+        try:
+            plain = B.sdwino_conv3x3_f32(xd, wT, bd, K, tile, ws)
+        finally:
+            B.sdwino_set_gemm_shape(0, 0)
+        assert torch.equal(y, plain + res.cuda())
+    with pytest.raises(B.SdwinoError) as e:
+        B.sdwino_conv3x3_f32_ex(xd, wT, bd, None, K, tile, 7, ws)
+    assert e.value.status == B.ERR_UNSUPPORTED
