@@ -270,13 +270,16 @@ def run_ours(args):
         devt.append((x.to(dev).to(io_t), wT, b.to(dev).to(io_t), torch.empty(y_h.shape, dtype=io_t, device=dev)))
     if args.epilogue != "none":
         gres = torch.Generator().manual_seed(1234)
-        res_dev = [torch.randn(y_h.shape, generator=gres).half().to(dev) for (_, _, _, y_h) in host]
+        res_dev = [torch.randn(y_h.shape, generator=gres).to(torch.float32 if io32 else torch.float16).to(dev)
+                   for (_, _, _, y_h) in host]
         act = B.ACT_SILU if args.epilogue == "residual_silu" else B.ACT_NONE
 
     def run_layer(li, strm):
         L, t, (xd, wT, bd, yd) = layers[li], tiles[li], devt[li]
-        if io32:
+        if io32 and (args.epilogue == "none" or min(L.C, L.K) <= 8):
             B.sdwino_conv3x3_f32(xd, wT, bd, L.K, t, ws, y=yd, stream=strm)
+        elif io32:
+            B.sdwino_conv3x3_f32_ex(xd, wT, bd, res_dev[li], L.K, t, act, ws, y=yd, stream=strm)
         elif args.epilogue == "none" or min(L.C, L.K) <= 8:     # the first and last convolution of a network have neither
             B.sdwino_conv3x3(xd, wT, bd, L.K, t, y=yd, workspace=ws, stream=strm)
         else:
