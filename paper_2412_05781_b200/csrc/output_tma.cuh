@@ -113,13 +113,29 @@ output_transform_f4_tma_kernel(const __grid_constant__ CUtensorMap tmM, const YT
                                                                    static_cast<long long>(i) * geo.W));
             }
         }
+        [[maybe_unused]] float4 resf[M][2];   // fp32 residual rows, loaded ahead of the second half of the transform
+        if constexpr (EP && sizeof(YT) == 4) {
+#pragma unroll
+            for (int i = 0; i < M; ++i) {
+                resf[i][0] = resf[i][1] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (ep.residual && i0 + i < geo.H) {
+                    const float4* rp = reinterpret_cast<const float4*>(static_cast<const float*>(ep.residual) + (img - y) +
+                                                                       static_cast<long long>(i) * geo.W);
+                    resf[i][0] = __ldg(rp);
+                    resf[i][1] = __ldg(rp + 1);
+                }
+            }
+        }
 #pragma unroll
         for (int i = 0; i < M; ++i) {
             float2 o[M];
             at4_packed(tt[i], o);
             if (i0 + i >= geo.H) continue;
             float v[8] = {o[0].x + b, o[1].x + b, o[2].x + b, o[3].x + b, o[0].y + b, o[1].y + b, o[2].y + b, o[3].y + b};
-            store_row8<EP>(img + static_cast<long long>(i) * geo.W, v, res[i], ep, y);
+            if constexpr (EP && sizeof(YT) == 4)
+                store_row8_f32_res(reinterpret_cast<float*>(img) + static_cast<long long>(i) * geo.W, v, resf[i], ep);
+            else
+                store_row8<EP>(img + static_cast<long long>(i) * geo.W, v, res[i], ep, y);
         }
     }
     if (abort_flag != 0) {

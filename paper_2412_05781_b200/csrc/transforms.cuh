@@ -716,6 +716,18 @@ __device__ __forceinline__ void store_row8(float* rowp, float (&v)[8], const uin
     reinterpret_cast<float4*>(rowp)[1] = make_float4(v[4], v[5], v[6], v[7]);
 }
 
+// The same with the residual row already in registers (loaded ahead of the arithmetic by the caller).
+__device__ __forceinline__ void store_row8_f32_res(float* rowp, float (&v)[8], const float4 (&rf)[2], const Epilogue& ep) {
+    v[0] += rf[0].x; v[1] += rf[0].y; v[2] += rf[0].z; v[3] += rf[0].w;
+    v[4] += rf[1].x; v[5] += rf[1].y; v[6] += rf[1].z; v[7] += rf[1].w;
+    if (ep.act != 0) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] = epilogue_act(v[i], ep.act);
+    }
+    reinterpret_cast<float4*>(rowp)[0] = make_float4(v[0], v[1], v[2], v[3]);
+    reinterpret_cast<float4*>(rowp)[1] = make_float4(v[4], v[5], v[6], v[7]);
+}
+
 template <int M, int TPT, bool EP, typename YT = __half>
 __device__ __forceinline__ void output_unit_vec(const __half* __restrict__ Mws, const YT* __restrict__ bias,
                                                 YT* __restrict__ y, const TileGeom& geo, int K, long long p_begin,
