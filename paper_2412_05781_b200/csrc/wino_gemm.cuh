@@ -93,6 +93,8 @@ struct GemmParams {
     int resident;      // 1: the filter blocks of a (position, k-tile) stay in shared memory while the CTA walks the
                        // tiles p of that pair (stages then hold V only)
     int group;         // filter-resident mode: CTAs that share out the tiles of one (position, k-tile) pair
+    int epi_alias;     // 1: no CTA has more than one tile, so the epilogue stages its rows in the (by then idle) first
+                       // pipeline stages instead of a buffer of its own, which leaves room for one more stage
     int dual;          // 1: the kernel instantiation with two blocks of 128 tiles per CTA tile (host side only)
     long long p_stride;  // tiles per pass (row pitch of V and M)
 };
@@ -128,8 +130,9 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
     const int worker = blockIdx.x / CTAS;            // index of this CTA (pair) among the persistent workers
     const int num_workers = gridDim.x / CTAS;
     uint8_t* ures_base = smem + stages * stage_bytes;
-    uint8_t* epi_base = ures_base + ures_bytes;
-    uint64_t* full_bar = reinterpret_cast<uint64_t*>(epi_base + L::epi_bytes(prm.epi_rows, prm.epi_bufs));
+    uint8_t* epi_base = prm.epi_alias ? smem : ures_base + ures_bytes;
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(ures_base + ures_bytes +
+                                                     (prm.epi_alias ? 0 : L::epi_bytes(prm.epi_rows, prm.epi_bufs)));
     uint64_t* empty_bar = full_bar + GEMM_MAX_STAGES;
     uint64_t* acc_full_bar = empty_bar + GEMM_MAX_STAGES;
     uint64_t* acc_empty_bar = acc_full_bar + 2;
