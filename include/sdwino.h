@@ -157,8 +157,9 @@ int sdwino_conv3x3_f32_ex(const float *x, const void *wT, const float *bias, con
  * holds that much memory until the process exits, and no allocation call is made on this path.
  *
  *   - Limit: a layer is accepted when one pass of 128 tiles fits, i.e. when
- *     128 * (tile+2)^2 * (C + K) * 2 bytes + 2 KiB <= SDWINO_STATIC_SCRATCH_BYTES (for tile 2,
- *     C + K <= 4095); larger layers return SDWINO_ERR_WORKSPACE.  Large images simply take more passes.
+ *     128 * (tile+2)^2 * (C + K) * 2 bytes + 2 KiB <= SDWINO_STATIC_SCRATCH_BYTES (tile 2:
+ *     C + K <= 8191; tile 4: C + K <= 3640); larger layers return SDWINO_ERR_WORKSPACE.  Large images
+ *     simply take more passes.
  *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
  *     that device current).  Make that first call outside any stream capture.
  *   - All calls share the one array and it keeps the contents of the last call.  Nothing in it has to

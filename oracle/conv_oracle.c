@@ -157,7 +157,11 @@ int oracle_winograd(const double *x, const double *w, const double *bias, double
         int th = (int)((t / TW) % TH), tw = (int)(t % TW);
         double *V = (double *)malloc(sizeof(double) * (size_t)C * aa);
         double *Mk = (double *)malloc(sizeof(double) * aa);
-        if (!V || !Mk) { err = 2; free(V); free(Mk); continue; }
+        if (!V || !Mk) {
+#pragma omp atomic write
+            err = 2;
+            free(V); free(Mk); continue;
+        }
         oracle_input_tile_transform(x, Bt, V, C, H, W, n, th, tw, m, a);
         for (int k = 0; k < K; ++k) {
             for (int e = 0; e < aa; ++e) {

@@ -8,7 +8,6 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _CSRC = os.path.join(_PKG, "csrc")
 LIB_PATH = os.path.join(_PKG, "libsdwino.so")
 _SOURCES = ["sdwino.cu"]
-_HEADERS = ["ptx.cuh", "transforms.cuh", "wino_gemm.cuh"]
 _INCLUDE = os.path.join(os.path.dirname(_PKG), "include", "sdwino.h")
 
 NVCC_FLAGS = [
@@ -21,7 +20,9 @@ def _stale() -> bool:
     if not os.path.exists(LIB_PATH):
         return True
     t = os.path.getmtime(LIB_PATH)
-    deps = [os.path.join(_CSRC, f) for f in _SOURCES + _HEADERS] + [_INCLUDE]
+    # every file under csrc/ is a dependency: sdwino.cu includes all the .cuh files
+    deps = [os.path.join(_CSRC, f) for f in sorted(os.listdir(_CSRC)) if f.endswith((".cu", ".cuh", ".h"))]
+    deps.append(_INCLUDE)
     return any(os.path.getmtime(d) > t for d in deps if os.path.exists(d))
 
 

@@ -16,6 +16,7 @@ POINT_SETS_F4 = [
     (0, 1, -1, 2, Fraction(-1, 2)),
     (0, Fraction(1, 2), Fraction(-1, 2), Fraction(3, 2), Fraction(-3, 2)),
     (0, Fraction(7, 10), Fraction(-7, 10), Fraction(7, 5), Fraction(-7, 5)),
+    (0, Fraction(3, 4), Fraction(-3, 4), Fraction(3, 2), Fraction(-3, 2)),   # the set the CUDA kernels use
 ]
 
 
