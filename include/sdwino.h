@@ -269,16 +269,20 @@ int sdwino_choose_tile(int N, int C, int H, int W, int K);
 int sdwino_set_fused_min_tiles(long long p_tiles);
 
 /*
- * Per-kernel timing for benchmarks.  While enabled, every kernel launch of the library is
- * bracketed by two CUDA events recorded on the launch's stream (this adds a little idle time
- * between kernels, so whole-call timings should be taken with profiling disabled).
+ * Timing for benchmarks.  mode 1: every kernel launch of the library is bracketed by two CUDA
+ * events recorded on the launch's stream (this adds a little idle time between kernels, so
+ * whole-call timings should be taken with profiling disabled).  mode 2: every convolution call
+ * as a whole is bracketed instead (one record of kind 5 per call; the kernels inside a call keep
+ * their overlap, so the records of a step add up to the step).  mode 0: off; other values return
+ * SDWINO_ERR_INVALID_ARG.
  * sdwino_profile_collect waits for the recorded events, adds the elapsed milliseconds and
- * the launch counts per kernel kind into the two caller arrays of 5 entries (0 filter
+ * the launch counts per kind into the two caller arrays of 6 entries (0 filter
  * transform, 1 activation transform, 2 batched GEMM, 3 output transform, 4 the single-kernel
- * paths for layers with few input or few output channels; either may be NULL)
- * and forgets the records.  Host arrays; not thread-safe against concurrent compute calls.
+ * paths for layers with few input or few output channels, 5 whole calls; either may be NULL)
+ * and forgets the records.  Host arrays.  The mode switch and the record list are safe against
+ * concurrent compute calls; the records of concurrent calls interleave.
  */
-int sdwino_profile_enable(int enable);
+int sdwino_profile_enable(int mode);
 int sdwino_profile_collect(double *ms_by_kind, unsigned long long *launches_by_kind);
 /* The same records one by one, in launch order: fills kinds[i] and ms[i] (host arrays of `capacity`
  * entries, either may be NULL; ms < 0 marks an event error) for the first `capacity` launches since

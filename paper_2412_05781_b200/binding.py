@@ -26,7 +26,7 @@ EXPORTS = [
     "sdwino_filter_transform_f32", "sdwino_conv3x3_f32", "sdwino_conv3x3_f32_ex",
 ]
 
-KERNEL_KINDS = ("filter_transform", "input_transform", "wino_gemm", "output_transform", "fused")
+KERNEL_KINDS = ("filter_transform", "input_transform", "wino_gemm", "output_transform", "fused", "layer")
 
 
 class SdwinoError(RuntimeError):
@@ -174,14 +174,16 @@ def sdwino_set_fused_min_tiles(p_tiles: int = 0) -> None:
     _check(lib.sdwino_set_fused_min_tiles(p_tiles), "sdwino_set_fused_min_tiles")
 
 
-def sdwino_profile_enable(enable: bool) -> None:
-    _check(lib.sdwino_profile_enable(1 if enable else 0), "sdwino_profile_enable")
+def sdwino_profile_enable(mode) -> None:
+    """0 / False: off; 1 / True: CUDA events around every kernel launch; 2: around every convolution call as a whole
+    (kind "layer")."""
+    _check(lib.sdwino_profile_enable(int(mode)), "sdwino_profile_enable")
 
 
 def sdwino_profile_collect():
     """-> {kernel kind: (total milliseconds, launches)} since the last collect."""
-    ms = (ctypes.c_double * 5)()
-    n = (ctypes.c_ulonglong * 5)()
+    ms = (ctypes.c_double * len(KERNEL_KINDS))()
+    n = (ctypes.c_ulonglong * len(KERNEL_KINDS))()
     _check(lib.sdwino_profile_collect(ms, n), "sdwino_profile_collect")
     return {k: (float(ms[i]), int(n[i])) for i, k in enumerate(KERNEL_KINDS)}
 

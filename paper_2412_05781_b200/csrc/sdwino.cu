@@ -29,24 +29,30 @@ __device__ int g_status_word = 0;
 
 std::atomic<unsigned long long> g_launches{0};
 std::mutex g_mutex;
-// test / tuning overrides of the GEMM launch shape (0 = choose automatically)
-int g_force_ctas = 0;
-int g_input_staging = 1;  // 0 never, 1 where it is faster, 2 wherever possible (sdwino_set_input_staging)
-bool g_disable_fused = false;  // forcing a GEMM shape also forces the GEMM path for few-channel layers
-int g_force_n_tile = 0;
+// Test / tuning overrides of the GEMM launch shape (0 = choose automatically).  Compute calls may run on several
+// host threads at once: the overrides are atomics, and a call reads each of them once.
+std::atomic<int> g_force_ctas{0};
+std::atomic<int> g_input_staging{1};  // 0 never, 1 where it is faster, 2 wherever possible (sdwino_set_input_staging)
+std::atomic<bool> g_disable_fused{false};  // forcing a GEMM shape also forces the GEMM path for few-channel layers
+std::atomic<int> g_force_n_tile{0};
 void* g_workspace = nullptr;
 size_t g_workspace_bytes = 0;
 
 // Optional per-kernel timing: when enabled every launch is bracketed by CUDA events on its stream.
-enum KernelKind { KIND_FILTER = 0, KIND_INPUT = 1, KIND_GEMM = 2, KIND_OUTPUT = 3, KIND_FUSED = 4, KIND_COUNT = 5 };
+// Mode 1 brackets every kernel, mode 2 every convolution call as a whole (KIND_LAYER: one record per call, so that
+// the kernels of a call keep their programmatic overlap and the records of a step add up to the step).
+enum KernelKind { KIND_FILTER = 0, KIND_INPUT = 1, KIND_GEMM = 2, KIND_OUTPUT = 3, KIND_FUSED = 4, KIND_LAYER = 5, KIND_COUNT = 6 };
 struct ProfRecord { int kind; cudaEvent_t beg, end; };
-bool g_profile = false;
-std::vector<ProfRecord> g_prof_records;
+std::atomic<int> g_profile{0};
+std::vector<ProfRecord> g_prof_records;   // guarded by g_mutex, like the event pool
 std::vector<cudaEvent_t> g_event_pool;
 
 cudaEvent_t prof_event() {
     cudaEvent_t e = nullptr;
-    if (!g_event_pool.empty()) { e = g_event_pool.back(); g_event_pool.pop_back(); return e; }
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        if (!g_event_pool.empty()) { e = g_event_pool.back(); g_event_pool.pop_back(); return e; }
+    }
     if (cudaEventCreate(&e) != cudaSuccess) return nullptr;
     return e;
 }
@@ -62,12 +68,17 @@ void prof_record(cudaEvent_t e, cudaStream_t st) {
 struct ProfScope {
     cudaStream_t st; int kind; cudaEvent_t beg = nullptr;
     ProfScope(int k, cudaStream_t s) : st(s), kind(k) {
-        if (g_profile) { beg = prof_event(); if (beg) prof_record(beg, st); }
+        if (g_profile.load(std::memory_order_relaxed) == (k == KIND_LAYER ? 2 : 1)) {
+            beg = prof_event();
+            if (beg) prof_record(beg, st);
+        }
     }
     ~ProfScope() {
         if (beg) {
             cudaEvent_t end = prof_event();
-            if (end) { prof_record(end, st); g_prof_records.push_back({kind, beg, end}); }
+            if (end) prof_record(end, st);
+            std::lock_guard<std::mutex> lock(g_mutex);
+            if (end) g_prof_records.push_back({kind, beg, end});
             else g_event_pool.push_back(beg);
         }
     }
@@ -594,7 +605,7 @@ int launch_fused_small_c(const __half* x, const void* wT, const __half* bias, __
 // A CTA takes 128 tiles and all input channels, so the kernel only pays off when there are enough blocks
 // of tiles to occupy the SMs (measured: 64 blocks 32 us against 48 us unfused; 16 blocks 32 us against 15 us).
 constexpr long long FK_MIN_P_TILES = 48;
-long long g_fk_min_p_tiles = FK_MIN_P_TILES;
+std::atomic<long long> g_fk_min_p_tiles{FK_MIN_P_TILES};
 bool use_fused_small_k(int K, int W, int tile, long long p_tiles, const void* x, const void* y) {
     return tile == 2 && K <= FK_KMAX && p_tiles >= g_fk_min_p_tiles && (W % 8) == 0 && aligned(x, 16) && aligned(y, 4);
 }
@@ -759,6 +770,9 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
     }
     Plan pl;
     if (!x || !wT || !y || !make_plan(N, C, H, W, K, tile, &pl)) return SDWINO_ERR_INVALID_ARG;
+    // the overrides are read once per call
+    const int force_ctas = g_force_ctas.load(), force_n_tile = g_force_n_tile.load();
+    const bool disable_fused = g_disable_fused.load();
     const size_t elem = io32 ? 4 : 2;
     if (!aligned(x, elem) || !aligned(y, elem) || (bias && !aligned(bias, elem)) || !aligned(wT, WS_ALIGN))
         return SDWINO_ERR_MISALIGNED;
@@ -766,6 +780,7 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
     if (!aligned(ws, WS_ALIGN)) return SDWINO_ERR_MISALIGNED;
     long long pc = tiles_per_pass(pl, ws_bytes);
     if (pc < GEMM_BLOCK_P) return SDWINO_ERR_WORKSPACE;
+    ProfScope layer_prof(KIND_LAYER, st);   // profile mode 2: one record for the whole call
     if (tile == 4 && pc < pl.P128) {
         // several passes: cut them at whole tile rows where that keeps the TMA-staged activation transform usable
         const TileGeom g0 = make_geom(H, W, pl.TH, pl.TW, pl.P);
@@ -778,20 +793,20 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
     const bool no_ep = ep.residual == nullptr && ep.act == 0;
     const bool plain = no_ep && !io32;
     if (no_ep && use_fused_small_k(K, W, tile, pl.P128 / 128, x, y) && !use_fused_small_c(C, tile) &&
-        (!io32 || aligned(y, 8)) && !g_disable_fused) {
+        (!io32 || aligned(y, 8)) && !disable_fused) {
         if (io32)
             return launch_fused_small_k(static_cast<const float*>(x), wT, static_cast<const float*>(bias),
                                         static_cast<float*>(y), pl, C, H, W, K, st);
         return launch_fused_small_k(static_cast<const __half*>(x), wT, static_cast<const __half*>(bias),
                                     static_cast<__half*>(y), pl, C, H, W, K, st);
     }
-    if (no_ep && io32 && tile == 2 && use_fused_small_c(C, tile) && !g_disable_fused) {
+    if (no_ep && io32 && tile == 2 && use_fused_small_c(C, tile) && !disable_fused) {
         // the F(2x2) kernel for few input channels also serves the fp32 interface (F(4x4): the three kernels)
         const TileGeom geo = make_geom(H, W, pl.TH, pl.TW, pl.P);
         return launch_fused_small_c_mma(static_cast<const float*>(x), wT, static_cast<const float*>(bias),
                                         static_cast<float*>(y), geo, C, K, pl.Kb, st);
     }
-    if (plain && use_fused_small_c(C, tile) && !g_disable_fused) {
+    if (plain && use_fused_small_c(C, tile) && !disable_fused) {
         const TileGeom geo = make_geom(H, W, pl.TH, pl.TW, pl.P);
         const __half* xh = static_cast<const __half*>(x);
         const __half* bh = static_cast<const __half*>(bias);
@@ -815,8 +830,8 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
     prm.wt_header = wt_header_of(wT);
     prm.K = K;
     prm.tile = tile;
-    GemmShape shape = choose_gemm_shape(K, C, pc / GEMM_BLOCK_P, pl.a2, sms, g_force_ctas);
-    if (g_force_n_tile >= 16 && g_force_n_tile <= GEMM_MAX_N && g_force_n_tile % 16 == 0) shape.n_tile = g_force_n_tile;
+    GemmShape shape = choose_gemm_shape(K, C, pc / GEMM_BLOCK_P, pl.a2, sms, force_ctas);
+    if (force_n_tile >= 16 && force_n_tile <= GEMM_MAX_N && force_n_tile % 16 == 0) shape.n_tile = force_n_tile;
     if (shape.ctas == 2) shape.n_tile = round_up(shape.n_tile, 32);  // each CTA of a pair loads whole 16-row blocks
     prm.n_tile = shape.n_tile;
     prm.num_k_tiles = (K + prm.n_tile - 1) / prm.n_tile;
@@ -824,7 +839,7 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
     prm.num_c_blocks = (C + GEMM_BLOCK_C - 1) / GEMM_BLOCK_C;
     prm.C = C;
     const int b_rows = prm.n_tile / shape.ctas;
-    if (g_force_n_tile != 0) shape.dual = 0;
+    if (force_n_tile != 0) shape.dual = 0;
     prm.dual = shape.dual;
     // epilogue staging: two groups of epilogue warps each take half a tile when that is a multiple of 16 channels
     const bool split = (prm.n_tile / 2) % 16 == 0;
@@ -841,7 +856,7 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
         // shapes bit for bit compare both placements.
         const long long p_blocks = shape.dual ? 2 : 1;
         const long long tiles = ((pc / GEMM_BLOCK_P + p_blocks - 1) / p_blocks) * prm.num_k_tiles * pl.a2;
-        prm.epi_alias = (shape.ctas == 1 && pc >= pl.P128 && tiles <= sms && g_force_ctas == 0 && g_force_n_tile == 0) ? 1 : 0;
+        prm.epi_alias = (shape.ctas == 1 && pc >= pl.P128 && tiles <= sms && force_ctas == 0 && force_n_tile == 0) ? 1 : 0;
     }
     prm.stages = (MAX_DYN_SMEM - GemmSmemLayout::dyn_bytes(b_rows, 0, prm.epi_rows, prm.epi_alias ? 0 : prm.epi_bufs)) /
                  (GemmSmemLayout::stage_bytes(b_rows) + (shape.dual ? GemmSmemLayout::A_BYTES : 0));
@@ -862,7 +877,7 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
         const int stages = (MAX_DYN_SMEM - GemmSmemLayout::dyn_bytes(0, 0, rows, prm.epi_bufs, ures)) / GemmSmemLayout::A_BYTES;
         // (CTA pairs gain nothing from it: with their half of a 512-channel block resident only four 16 KB stages
         // of V remain, too few bytes in flight: 512->512 at 256x256 99 against 94 us)
-        if (shape.ctas == 1 && !shape.dual && g_force_ctas == 0 && g_force_n_tile == 0 && p_tiles >= 16 && keys * p_tiles >= 4 * workers &&
+        if (shape.ctas == 1 && !shape.dual && force_ctas == 0 && force_n_tile == 0 && p_tiles >= 16 && keys * p_tiles >= 4 * workers &&
             prm.n_tile >= 224 && stages >= 4) {
             prm.resident = 1;
             // CTAs per (position, k-tile) pair.  A group walks `rounds` pairs, each CTA `run` tiles per pair,
@@ -1308,9 +1323,9 @@ int sdwino_conv3x3_static(const void* x, const void* wT, const void* bias, void*
                      static_cast<cudaStream_t>(stream));
 }
 
-int sdwino_profile_enable(int enable) {
-    std::lock_guard<std::mutex> lock(g_mutex);
-    g_profile = enable != 0;
+int sdwino_profile_enable(int mode) {
+    if (mode < 0 || mode > 2) return SDWINO_ERR_INVALID_ARG;
+    g_profile.store(mode);
     return SDWINO_OK;
 }
 

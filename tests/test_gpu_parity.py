@@ -270,17 +270,6 @@ def test_sd15_unet_layers_sampled_channels(B, idx):
     assert err <= TOL_F2_REGRESSION and edge <= TOL, (layer.name, err, edge)
 
 
-@pytest.mark.parametrize("idx", range(16))
-def test_sd15_unet_layers_with_the_chosen_tile(B, idx):
-    # the benchmark's default configuration: every layer with the algorithm sdwino_choose_tile picks for it
-    layer = workloads.sd15_unet()[idx]
-    tile = B.sdwino_choose_tile(layer.N, layer.C, layer.H, layer.W, layer.K)
-    if tile == 2:
-        pytest.skip("F(2x2) for this layer: covered by test_sd15_unet_layers_sampled_channels")
-    err, edge = _sampled_check(B, layer, 4, nch=6, seed=idx)
-    assert err <= TOL and edge <= TOL, (err, edge)
-
-
 @pytest.mark.parametrize("idx", [0, 1, 2, 5, 9])
 def test_vae_layers_sampled_channels(B, idx):
     layer = workloads.sd_vae_decoder_512()[idx]
