@@ -1,20 +1,25 @@
 #!/usr/bin/env python
-"""Benchmark of the sdwino hot path on the SD v1.5 UNet 3x3-convolution sweep.
+"""Benchmark of the sdwino hot path on the Stable Diffusion 3x3-convolution sweeps.
 
-A step is one pass over the 16 stride-1 pad-1 3x3 convolutions of the SD v1.5 UNet at 512x512
-(latent 64x64, batch 2), each run as activation transform -> batched tcgen05 GEMM -> output
-transform + bias through the C ABI.  The filter transform is the once-per-weight preprocess and
-runs before the timed region; its time is reported separately.
+A step is one pass over the stride-1 pad-1 3x3 convolutions of a workload, each run through the C ABI
+(activation transform -> batched tcgen05 GEMM -> output transform + bias, or one of the single-kernel
+paths).  The filter transform is the once-per-weight preprocess and runs before the timed region; its
+time is reported separately.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload NAME]
 
-Prints ONE JSON line (rank 0).  With --gpus N > 1 (under torchrun) every rank runs an independent
-replica of the sweep on its own GPU (the path has no exchange step); the time is the max over ranks.
+By default all five workloads are measured (single layer, SD v1.5 UNet, SD VAE decoder, SD v2.1 UNet,
+SDXL at 1024x1024) and the headline `value` sits on the largest one, `sdxl_1024`; the others are in
+`workloads`.  Prints ONE JSON line (rank 0).  With --gpus N > 1 (under torchrun) every rank runs an
+independent replica of the sweep on its own GPU (the path has no exchange step); the time is the max
+over ranks.
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
+import math
 import os
 import statistics
 import sys
@@ -25,24 +30,52 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-METRIC = "direct-conv-equivalent TFLOP/s over the SD v1.5 UNet 3x3 conv sweep (2*N*K*C*H*W*9 / time)"
+METRIC = "direct-conv-equivalent TFLOP/s over {sweep} (2*N*K*C*H*W*9 / time)"
 _SWEEP_NAMES = {"single": "the single 320->320 at 32x32 layer", "sd15_unet": "the SD v1.5 UNet 3x3 conv sweep",
                 "sd_vae_512": "the SD VAE decoder (512x512) 3x3 conv sweep", "sd21_unet": "the SD v2.1 UNet 3x3 conv sweep",
                 "sdxl_1024": "the SDXL (1024x1024) UNet + VAE decoder 3x3 conv sweep"}
+ALL_WORKLOADS = ["single", "sd15_unet", "sd_vae_512", "sd21_unet", "sdxl_1024"]
+HEADLINE = "sdxl_1024"      # the largest single-GPU configuration
 
 
 def metric_name(workload: str) -> str:
-    """The headline metric, named for the workload that was run (the default is the SD v1.5 sweep)."""
-    return METRIC.replace("the SD v1.5 UNet 3x3 conv sweep", _SWEEP_NAMES[workload])
+    return METRIC.format(sweep=_SWEEP_NAMES[workload])
+
+
 UNIT = "TFLOP/s"
-WORKLOAD = "sd15_unet"
 TILE = "auto"   # per layer: what sdwino_choose_tile returns; --tile 2 / --tile 4 force one algorithm
 L2_BYTES = 126e6
+SUSTAINED_SECONDS = 2.2
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# dram__bytes_read.sum + dram__bytes_write.sum per GEMM launch of one SD v1.5 step, from ncu captures
-# (profiles/launch_list_sd15_unet_sweep.md), by --tile.  Only valid for the default workload with all layers.
-GEMM_DRAM_BYTES_PER_LAUNCH_SD15 = {"auto": 49.89e6, "2": 40.66e6}
 PAPER_CONTEXT = {"per_layer_speedup_vs_sdcpp_m1pro": 2.76, "end_to_end_speedup_vs_sdcpp_m1pro": 4.79}
+
+# DRAM traffic of the GEMM launches of one step (ncu: dram__bytes_read.sum + dram__bytes_write.sum, summed over the
+# GEMM launches of a step and divided by their number), per workload with the per-layer tile choice.  Each entry
+# records the capture it came from and the hash of the kernel sources it was taken with; `roofline.traffic` is null,
+# with the reason, when the sources have changed since.
+GEMM_DRAM_TRAFFIC = {
+}
+
+
+def kernel_source_hash() -> str:
+    """Hash of the CUDA sources: ties a stored ncu figure to the build it was captured on."""
+    csrc = os.path.join(ROOT, "paper_2412_05781_b200", "csrc")
+    h = hashlib.sha256()
+    for name in sorted(os.listdir(csrc)):
+        if name.endswith((".cu", ".cuh")):
+            with open(os.path.join(csrc, name), "rb") as f:
+                h.update(name.encode())
+                h.update(f.read())
+    return h.hexdigest()[:12]
+
+
+def stored_traffic(workload: str, tile: str, layer_subset: str):
+    entry = GEMM_DRAM_TRAFFIC.get(workload)
+    if entry is None or tile != "auto" or layer_subset:
+        return None, "no ncu capture stored for this workload / tile / layer subset"
+    if entry["source_hash"] != kernel_source_hash():
+        return None, f"stale: the kernel sources changed since the capture ({entry['capture']})"
+    return entry["bytes_per_launch"], entry["capture"]
 
 
 def load_peaks():
@@ -98,6 +131,7 @@ class ClockSampler:
         if self.nv is not None:
             self._thread = threading.Thread(target=self._loop, daemon=True)
             self._thread.start()
+        return self
 
     def stop(self):
         self._stop.set()
@@ -155,12 +189,38 @@ def oracle_sample(layers, inputs, channels_per_layer, seed=0):
     return t, flops
 
 
-def select_layers(args):
-    """The benchmarked workload, optionally cut down to some of its layers (profiling runs)."""
+def oracle_budgeted_sample(layers, inputs, seconds: float, order_seed: int = 0, start: int = 0, max_layers=None):
+    """The oracle as it stands, on a bounded sample: it parallelises over output channels, so a sample is one seeded
+    output channel per host thread of one layer; layers are taken in a seeded order, beginning at position `start`
+    of that order, until `seconds` have been used (a layer is skipped when the rate seen so far says that it alone
+    would overrun the rest of the budget by half).  Returns (seconds, flops, names of the sampled layers)."""
+    import numpy as np
+    import oracle
+    nthreads = oracle.threads()
+    order = np.random.default_rng(order_seed).permutation(len(layers)).tolist()
+    order = order[start % len(order):] + order[:start % len(order)]
+    t_tot, f_tot, names = 0.0, 0, []
+    for li in order:
+        L = layers[li]
+        nch = min(L.K, nthreads)
+        flops = 2 * L.N * nch * L.C * L.H * L.W * 9
+        if names and f_tot > 0 and flops / (f_tot / t_tot) > 1.5 * (seconds - t_tot):
+            continue
+        t, f = oracle_sample([L], [inputs[li]], nch, seed=li)
+        t_tot += t
+        f_tot += f
+        names.append(L.name)
+        if t_tot >= seconds or (max_layers is not None and len(names) >= max_layers):
+            break
+    return t_tot, f_tot, names
+
+
+def select_layers(workload: str, layer_subset: str):
+    """A workload, optionally cut down to some of its layers (profiling runs)."""
     from paper_2412_05781_b200 import workloads
-    layers = workloads.WORKLOADS[args.workload]()
-    if args.layers:
-        layers = [layers[int(i)] for i in args.layers.split(",")]
+    layers = workloads.WORKLOADS[workload]()
+    if layer_subset:
+        layers = [layers[int(i)] for i in layer_subset.split(",")]
     return layers
 
 
@@ -173,30 +233,37 @@ def host_inputs(layers):
     return out
 
 
+def headline_of(args) -> str:
+    return HEADLINE if args.workload == "all" else args.workload
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     import oracle
-    from paper_2412_05781_b200 import workloads
     oracle.build()
-    layers = select_layers(args)
+    workload = headline_of(args)
+    layers = select_layers(workload, args.layers)
     inputs = host_inputs(layers)
-    nch = 2
-    for _ in range(args.warmup):
-        oracle_sample(layers, inputs, nch)
-    t_tot, f_tot = 0.0, 0
-    for _ in range(args.steps):
-        t, f = oracle_sample(layers, inputs, nch)
+    # A bounded sample per step: one layer (the steps walk the layers in a seeded order), one seeded output channel
+    # per host thread, which is how the oracle's loops use the cores.
+    for i in range(args.warmup):
+        oracle_budgeted_sample(layers, inputs, 1e9, start=i, max_layers=1)
+    t_tot, f_tot, seen = 0.0, 0, []
+    for i in range(args.steps):
+        t, f, names = oracle_budgeted_sample(layers, inputs, 1e9, start=args.warmup + i, max_layers=1)
         t_tot += t
         f_tot += f
+        seen += names
     val = f_tot / t_tot / 1e12
-    sample = f"{nch} seeded output channels of each of the {len(layers)} layers per step (fp64 direct conv)"
+    sample = (f"per step one layer of the {len(layers)} (seeded order, {len(set(seen))} distinct layers over the run), "
+              f"min(K, {oracle.threads()}) seeded output channels of it (fp64 direct conv)")
     line = {
-        "impl": "reference", "metric": metric_name(args.workload), "value": val, "unit": UNIT, "n_gpus": args.gpus,
+        "impl": "reference", "metric": metric_name(workload), "value": val, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_tot / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": args.workload, "layers": len(layers), "batch": layers[0].N, "sample": sample},
+        "config": {"workload": workload, "layers": len(layers), "batch": layers[0].N, "sample": sample},
         "cpu_baseline": {"value": val, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -207,71 +274,57 @@ def run_reference(args):
 # ------------------------------------------------------------------------------------------
 # our arm
 # ------------------------------------------------------------------------------------------
-def run_ours(args):
-    import torch
-    from paper_2412_05781_b200 import build_library, workloads
-    build_library()
-    from paper_2412_05781_b200 import binding as B
+class Ctx:
+    """What every workload measurement shares: the binding, the device, the timing stream, the peaks."""
+    pass
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the sdwino path has no CPU fallback")
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist_mod
-        dist_mod.init_process_group("nccl", device_id=dev)
-        dist = dist_mod
+
+def bench_workload(ctx, args, workload: str, headline: bool):
+    """Measures one workload; returns its record (see the keys at the end)."""
+    import torch
+    from paper_2412_05781_b200 import workloads
+    B, dev, stream, dist, world, rank = ctx.B, ctx.dev, ctx.stream, ctx.dist, ctx.world, ctx.rank
+    peaks, peak_kind = ctx.peaks, ctx.peak_kind
+    steps, warmup = args.steps, max(args.warmup, 3)
 
     def barrier():
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
 
-    peaks, peak_kind = load_peaks()
-    layers = select_layers(args)
+    layers = select_layers(workload, args.layers)
     tiles = [B.sdwino_choose_tile(L.N, L.C, L.H, L.W, L.K) if args.tile == "auto" else int(args.tile) for L in layers]
+    io32 = args.io == "f32"       # the fp32 interface: x, w, bias, y in fp32
+    io_bytes = 4.0 if io32 else 2.0
+    io_t = torch.float32 if io32 else torch.float16
 
     # ---- inputs: pinned host copies (for the end-to-end pass) and resident device copies ----
     host, devt = [], []
-    ws_bytes, hws_bytes = 0, 0
+    ws_bytes = 0
     for li, L in enumerate(layers):
-        x, w, b = workloads.make_inputs(L, seed=li, pin=True)
-        y_h = torch.empty(L.N, L.K, L.H, L.W, dtype=torch.float16).pin_memory()
+        x, w, b = workloads.make_inputs(L, seed=li, pin=not args.no_e2e)
+        y_h = torch.empty(L.N, L.K, L.H, L.W, dtype=torch.float16)
+        if not args.no_e2e:
+            y_h = y_h.pin_memory()
         host.append((x, w, b, y_h))
-        dims = (L.N, L.C, L.H, L.W, L.K, tiles[li])
-        ws_bytes = max(ws_bytes, B.sdwino_workspace_bytes(*dims))
-        hws_bytes = max(hws_bytes, B.sdwino_host_staging_bytes(*dims) + B.sdwino_workspace_bytes(*dims))
-    ws = B.alloc_workspace(max(ws_bytes, hws_bytes), dev)
-    # end-to-end pass: a workspace (staging + scratch) per layer, so that the copies of neighbouring layers may
-    # overlap; layers that share one are ordered copy after copy by the library
-    e2e_bytes = [B.sdwino_host_staging_bytes(L.N, L.C, L.H, L.W, L.K, t) + B.sdwino_workspace_bytes(L.N, L.C, L.H, L.W, L.K, t)
-                 for L, t in zip(layers, tiles)]
-    per_layer_ws = sum(e2e_bytes) <= (48 << 30)
-    ws_e2e = [B.alloc_workspace(nb, dev) for nb in e2e_bytes] if per_layer_ws else [ws] * len(layers)
+        ws_bytes = max(ws_bytes, B.sdwino_workspace_bytes(L.N, L.C, L.H, L.W, L.K, tiles[li]))
+    ws = B.alloc_workspace(ws_bytes, dev)
 
     # filter transform: once per weight, outside the timed step; timed on its own
-    B.sdwino_profile_enable(True)
-    io32 = args.io == "f32"       # the fp32 interface: x, w, bias, y in fp32 (the host arm below stays fp16)
-    io_bytes = 4.0 if io32 else 2.0
+    B.sdwino_profile_enable(1)
     w_dev = [h[1].to(dev).float() if io32 else h[1].to(dev) for h in host]
     for _ in range(3):
         wTs = [(B.sdwino_filter_transform_f32 if io32 else B.sdwino_filter_transform)(wd, t) for wd, t in zip(w_dev, tiles)]
         prof = B.sdwino_profile_collect()
     ft_ms = prof["filter_transform"][0]
     ft_bytes = sum(L.K * L.C * 9 * io_bytes + B.sdwino_filter_bytes(L.K, L.C, t) for L, t in zip(layers, tiles))
-    B.sdwino_profile_enable(False)
+    B.sdwino_profile_enable(0)
     del w_dev
     for (x, w, b, y_h), wT in zip(host, wTs):
-        io_t = torch.float32 if io32 else torch.float16
         devt.append((x.to(dev).to(io_t), wT, b.to(dev).to(io_t), torch.empty(y_h.shape, dtype=io_t, device=dev)))
     if args.epilogue != "none":
         gres = torch.Generator().manual_seed(1234)
-        res_dev = [torch.randn(y_h.shape, generator=gres).to(torch.float32 if io32 else torch.float16).to(dev)
-                   for (_, _, _, y_h) in host]
+        res_dev = [torch.randn(y_h.shape, generator=gres).to(io_t).to(dev) for (_, _, _, y_h) in host]
         act = B.ACT_SILU if args.epilogue == "residual_silu" else B.ACT_NONE
 
     def run_layer(li, strm):
@@ -289,13 +342,11 @@ def run_ours(args):
         for li in range(len(layers)):
             run_layer(li, torch.cuda.current_stream())
 
-    sampler = ClockSampler(visible_to_nvml_index(local_rank))
-    # the timed step is replayed from a CUDA graph captured from the same C-ABI calls, so that host launch
-    # latency (48+ launches per step) does not enter the device-resident number; --no-graph launches directly
+    # The timed step is replayed from a CUDA graph captured from the same C-ABI calls, so that host launch latency
+    # (about three launches per layer) does not enter the device-resident number; --no-graph launches directly.
     torch.cuda.synchronize()
-    stream = torch.cuda.Stream()
     with torch.cuda.stream(stream):
-        for _ in range(max(args.warmup, 3)):
+        for _ in range(warmup):
             step()
     stream.synchronize()
     l0 = B.sdwino_launch_count()
@@ -313,88 +364,129 @@ def run_ours(args):
             step()
         launches_per_step = B.sdwino_launch_count() - l0
     stream.synchronize()
-    barrier()
-    sampler.start()
 
-    # ---- timed region: resident inputs ----
+    def one_step():
+        if graph is not None:
+            graph.replay()
+        else:
+            step()
+
+    # ---- timed region: resident inputs, exactly `steps` steps, an event after every step ----
     flops_step = sum(L.direct_flops for L in layers)
     step_bytes = sum(io_bytes * L.N * (L.C + L.K) * L.H * L.W + B.sdwino_filter_bytes(L.K, L.C, t) for L, t in zip(layers, tiles))
     # A step that touches less than twice the L2 would find its operands cached by the previous step: then
     # the L2 is flushed (a 256 MB buffer is written) before every step and only the steps are timed.
     flush_l2 = step_bytes < 2 * L2_BYTES
+    sampler = ClockSampler(visible_to_nvml_index(ctx.local_rank)).start() if headline else None
     barrier()
     if not flush_l2:
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
         with torch.cuda.stream(stream):
-            e0.record(stream)
-            for _ in range(args.steps):
-                if graph is not None:
-                    graph.replay()
-                else:
-                    step()
-            e1.record(stream)
+            ev[0].record(stream)
+            for i in range(steps):
+                one_step()
+                ev[i + 1].record(stream)
         stream.synchronize()
-        ms_total = e0.elapsed_time(e1)
+        ms_total = ev[0].elapsed_time(ev[steps])
+        per_step = [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
     else:
         flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
-        pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+        pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
         with torch.cuda.stream(stream):
             for a, b_ in pairs:
                 flush_buf.fill_(1)
                 a.record(stream)
-                if graph is not None:
-                    graph.replay()
-                else:
-                    step()
+                one_step()
                 b_.record(stream)
         stream.synchronize()
-        ms_total = sum(a.elapsed_time(b_) for a, b_ in pairs)
+        per_step = [a.elapsed_time(b_) for a, b_ in pairs]
+        ms_total = sum(per_step)
         del flush_buf
     barrier()
-    launches = launches_per_step * args.steps
-    ms_step = max_over_ranks(ms_total, dist, dev) / args.steps
+    clocks = sampler.stop() if sampler is not None else None
+    ms_step = max_over_ranks(ms_total, dist, dev) / steps
     assert B.sdwino_last_device_status(stream) == B.OK, "a device-side wait timed out"
-
     value = aggregate_value(flops_step, world, ms_step)
 
-    # ---- end to end: host buffers in, host buffers out, through sdwino_conv3x3_host ----
-    e2e_steps = max(3, min(args.steps, 30))
+    # ---- sustained leg: back-to-back replays for at least two seconds, with the clocks that were seen.  For a
+    #      workload whose timed steps flush the L2 this leg does not: it is the L2-warm figure. ----
+    sustained = None
+    if not args.no_sustained:
+        n_sus = max(steps, min(200000, int(math.ceil(SUSTAINED_SECONDS * 1e3 / max(min(per_step), 1e-3)))))
+        sus_sampler = ClockSampler(visible_to_nvml_index(ctx.local_rank)).start()
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(stream):
+            s0.record(stream)
+            for _ in range(n_sus):
+                one_step()
+            s1.record(stream)
+        stream.synchronize()
+        sus_clocks = sus_sampler.stop()
+        sus_ms = max_over_ranks(s0.elapsed_time(s1), dist, dev) / n_sus
+        sustained = {"steps": n_sus, "seconds": round(sus_ms * n_sus * 1e-3, 3), "ms_per_step": round(sus_ms, 4),
+                     "value": round(aggregate_value(flops_step, world, sus_ms), 2), "unit": UNIT,
+                     "l2": "warm (no flush between steps)" if flush_l2 else "as in the timed steps",
+                     "clocks": sus_clocks,
+                     "ms_x_mhz": round(sus_ms * sus_clocks["sm_mhz"], 1) if sus_clocks.get("sm_mhz") else None}
 
-    def e2e_step():
-        for t, (x, w, b, y_h), (_, wT, _, _), wsl in zip(tiles, host, devt, ws_e2e):
-            B.sdwino_conv3x3_host(x, wT, b, y_h, t, wsl, stream=stream, wait=False)
-        B.sdwino_host_join(stream)
-        stream.synchronize()                  # y of every layer is complete in host memory
+    # ---- the same step launched directly (no graph): what a caller without graphs sees ----
+    direct_ms = None
+    if graph is not None:
+        nd = min(steps, 20)
+        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(stream):
+            step()
+            d0.record(stream)
+            for _ in range(nd):
+                step()
+            d1.record(stream)
+        stream.synchronize()
+        direct_ms = d0.elapsed_time(d1) / nd
 
-    for _ in range(3):
-        e2e_step()
-    barrier()
-    t0 = time.perf_counter()
-    for _ in range(e2e_steps):
-        e2e_step()
-    torch.cuda.synchronize()
-    e2e_s = time.perf_counter() - t0
-    e2e_value = aggregate_value(flops_step, world, max_over_ranks(e2e_s, dist, dev) / e2e_steps * 1e3)
-    h2d = sum(x.numel() * 2 + b.numel() * 2 for (x, w, b, y) in host)
-    d2h = sum(y.numel() * 2 for (x, w, b, y) in host)
-    # what came back through the host path is what the device-resident step computed (same kernels: same bits)
-    e2e_matches = args.epilogue != "none" or io32 or all(torch.equal(y_h, yd.cpu()) for (_, _, _, y_h), (_, _, _, yd) in zip(host, devt))
-    assert e2e_matches, "the host path returned something else than the device path"
+    # ---- per-layer times: the step replayed from a graph in which every convolution call (not every kernel) is
+    #      bracketed by event nodes, so the kernels of a layer keep their programmatic overlap and the layer times
+    #      add up to the step; then per-kernel times (events around every launch), used for the split of a
+    #      layer's time over its kernels. ----
+    prof_steps = max(3, min(steps, 20))
+    layer_ms = [0.0] * len(layers)
+    per_layer = [dict(input_transform=0.0, wino_gemm=0.0, output_transform=0.0, fused=0.0, launches=0) for _ in layers]
 
-    # ---- per-kernel and per-layer times: a second timed pass with CUDA events around every launch (recorded
-    #      by the library on the launch stream).  The sweeps run back to back without host syncs, so the device
-    #      stays busy and an event pair measures its kernel; the event gaps keep this pass out of `value`. ----
-    B.sdwino_profile_enable(True)
+    def profiled_pass(mode, account):
+        B.sdwino_profile_enable(mode)
+        if not args.no_graph:
+            pgraph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(pgraph, stream=stream):
+                step()
+            for _ in range(prof_steps):
+                with torch.cuda.stream(stream):
+                    pgraph.replay()
+                stream.synchronize()
+                account(B.sdwino_profile_records(keep=True))
+            B.sdwino_profile_records()
+            del pgraph
+        else:
+            for _ in range(prof_steps):
+                with torch.cuda.stream(stream):
+                    step()
+                stream.synchronize()
+                account(B.sdwino_profile_records())
+        B.sdwino_profile_enable(0)
+
+    def account_layers(recs):
+        assert len(recs) == len(layers) and all(k == "layer" and ms >= 0 for k, ms in recs)
+        for li, (_, ms) in enumerate(recs):
+            layer_ms[li] += ms / prof_steps
+
+    profiled_pass(2, account_layers)
+    B.sdwino_profile_enable(1)
     records_per_layer = []
     with torch.cuda.stream(stream):
         for li in range(len(layers)):     # learn how many launches each layer makes
             run_layer(li, stream)
             records_per_layer.append(len(B.sdwino_profile_records()))
-    prof_steps = max(3, min(args.steps, 20))
-    per_layer = [dict(input_transform=0.0, wino_gemm=0.0, output_transform=0.0, fused=0.0, launches=0)
-                 for _ in layers]
+    B.sdwino_profile_enable(0)
 
-    def account(recs):
+    def account_kernels(recs):
         assert len(recs) == sum(records_per_layer) and all(ms >= 0 for _, ms in recs)
         it = iter(recs)
         for li, nrec in enumerate(records_per_layer):
@@ -404,39 +496,19 @@ def run_ours(args):
                 if kind == "wino_gemm":
                     per_layer[li]["launches"] += 1
 
-    if graph is not None:
-        # the event records become nodes of a second graph: replaying it keeps the device busy, so an event
-        # pair measures its kernel and not the host's launch latency
-        pgraph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(pgraph, stream=stream):
-            step()
-        for _ in range(prof_steps):
-            with torch.cuda.stream(stream):
-                pgraph.replay()
-            stream.synchronize()
-            account(B.sdwino_profile_records(keep=True))
-        B.sdwino_profile_records()
-        del pgraph
-    else:
-        for _ in range(prof_steps):
-            with torch.cuda.stream(stream):
-                step()
-            stream.synchronize()
-            account(B.sdwino_profile_records())
-    B.sdwino_profile_enable(False)
-    clocks = sampler.stop()
+    profiled_pass(1, account_kernels)
 
-    def gbs_safe(nbytes, ms):
+    tpeak = peaks["bf16_tflops"]          # burst figure (the larger denominator); the sustained one is given beside it
+    tpeak_sus = peaks["bf16_tflops_sustained"]
+    hpeak = peaks["hbm_gbs"]
+
+    def gbs(nbytes, ms):
         return nbytes / (ms * 1e-3) / 1e9 if ms > 0 else 0.0
 
-    tpeak = peaks["bf16_tflops"]          # burst figure: each kernel is microseconds long and timed alone
-    hpeak = peaks["hbm_gbs"]
     layer_rows = []
     gemm_flops = gemm_ms = gemm_u_bytes = 0.0
-    in_ms = out_ms = 0.0
-    in_bytes = out_bytes = 0.0
-    fused_ms = 0.0
-    for L, t, pl in zip(layers, tiles, per_layer):
+    in_ms = out_ms = in_bytes = out_bytes = fused_ms = 0.0
+    for L, t, pl, lms in zip(layers, tiles, per_layer, layer_ms):
         a2 = (t + 2) ** 2
         P = L.tiles(t)
         wino_flops = 2.0 * a2 * L.K * L.C * P
@@ -444,50 +516,52 @@ def run_ours(args):
         xb, yb = io_bytes * L.N * L.C * L.H * L.W, io_bytes * L.N * L.K * L.H * L.W
         t_tensor = wino_flops / (tpeak * 1e12) * 1e6
         t_hbm = (xb + 2.0 * a2 * L.K * L.C + yb + 2 * L.K) / (hpeak * 1e9) * 1e6
-        total_us = (pl["input_transform"] + pl["wino_gemm"] + pl["output_transform"] + pl["fused"]) * 1e3
+        ksum = pl["input_transform"] + pl["wino_gemm"] + pl["output_transform"] + pl["fused"]
+        scale = lms / ksum if ksum > 0 else 0.0     # the kernels' event-bracketed times, scaled to the layer's time
+        k_in, k_gemm, k_out, k_fused = (pl[k] * scale for k in ("input_transform", "wino_gemm", "output_transform", "fused"))
+        total_us = lms * 1e3
         layer_rows.append({
             "layer": L.name, "tile": t, "us": round(total_us, 2),
-            "us_input": round(pl["input_transform"] * 1e3, 2), "us_gemm": round(pl["wino_gemm"] * 1e3, 2),
-            "us_output": round(pl["output_transform"] * 1e3, 2), "us_fused": round(pl["fused"] * 1e3, 2),
-            "eq_tflops": round(L.direct_flops / (total_us * 1e-6) / 1e12, 1),
+            "us_input": round(k_in * 1e3, 2), "us_gemm": round(k_gemm * 1e3, 2),
+            "us_output": round(k_out * 1e3, 2), "us_fused": round(k_fused * 1e3, 2),
+            "eq_tflops": round(L.direct_flops / (total_us * 1e-6) / 1e12, 1) if total_us > 0 else None,
             "bound": "tensor" if t_tensor >= t_hbm else "hbm",
             "roof_us": round(max(t_tensor, t_hbm), 2),
-            "frac_of_roof": round(max(t_tensor, t_hbm) / total_us, 3),
-            "gemm_tensor_frac": (round(wino_flops / (pl["wino_gemm"] * 1e-3) / 1e12 / tpeak, 3)
-                                 if pl["wino_gemm"] > 0 else None),
+            "frac_of_roof": round(max(t_tensor, t_hbm) / total_us, 3) if total_us > 0 else None,
+            "gemm_tensor_frac": (round(wino_flops / (k_gemm * 1e-3) / 1e12 / tpeak, 3) if k_gemm > 0 else None),
         })
-        if pl["wino_gemm"] > 0:                  # layers on the fused few-channel kernel have no GEMM launch
+        if pl["wino_gemm"] > 0:                  # layers on a single-kernel path have no GEMM launch
             gemm_flops += wino_flops
             gemm_u_bytes += u_bytes
-            gemm_ms += pl["wino_gemm"]
-            in_ms += pl["input_transform"]
-            out_ms += pl["output_transform"]
+            gemm_ms += k_gemm
+            in_ms += k_in
+            out_ms += k_out
             in_bytes += xb + 2.0 * a2 * L.C * P      # read x, write V
             out_bytes += 2.0 * a2 * L.K * P + yb     # read M, write y
-        fused_ms += pl["fused"]
+        fused_ms += k_fused
     gemm_launches = sum(pl["launches"] for pl in per_layer) / prof_steps
-    achieved = gemm_flops / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0   # a subset of fused-kernel layers
+    achieved = gemm_flops / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
+    traffic, traffic_note = stored_traffic(workload, args.tile, args.layers)
+    sum_layers_ms = sum(layer_ms)
     roofline = {
         "kernel": "wino_gemm_kernel", "bound": "tensor", "achieved": round(achieved, 1), "peak": tpeak,
         "unit": "TFLOP/s", "frac": round(achieved / tpeak, 4),
-        "traffic": (GEMM_DRAM_BYTES_PER_LAUNCH_SD15.get(str(args.tile))
-                    if (args.workload == WORKLOAD and not args.layers) else None),
-        "traffic_unit": "bytes per launch (ncu dram read + write, L2 left warm)",
-        "peak_source": f"{peak_kind} (cuBLAS bf16 burst; fp16 has the same nominal rate)",
+        "frac_of_sustained_peak": round(achieved / tpeak_sus, 4),
+        "traffic": traffic, "traffic_unit": "bytes per launch (ncu dram read + write, L2 left warm)",
+        "traffic_source": traffic_note,
+        "peak_source": f"{peak_kind} (cuBLAS bf16 burst {tpeak}, sustained {tpeak_sus}; fp16 has the same nominal rate)",
         "launches_per_step": gemm_launches,
         "avg_launch_us": round(gemm_ms * 1e3 / gemm_launches, 2) if gemm_launches else None,
         "algorithmic_flops_per_step": gemm_flops,
-        "share_of_step": round(gemm_ms / max(gemm_ms + in_ms + out_ms + fused_ms, 1e-12), 3),
+        "share_of_step": round(gemm_ms / sum_layers_ms, 3) if sum_layers_ms > 0 else None,
+        "sum_of_layer_times_over_step": round(sum_layers_ms / ms_step, 3),
     }
-    def gbs(nbytes, ms):
-        return nbytes / (ms * 1e-3) / 1e9 if ms > 0 else 0.0
-
     # the same launches against the other roof: the GEMM is the kernel that streams the transformed weights, and
     # on the small-image layers that stream, not the tensor pipe, is what bounds it
     roofline["weight_stream_view"] = {
         "bound": "hbm", "algorithmic_bytes_per_step": gemm_u_bytes,
-        "achieved": round(gbs_safe(gemm_u_bytes, gemm_ms), 1), "peak": hpeak, "unit": "GB/s",
-        "frac": round(gbs_safe(gemm_u_bytes, gemm_ms) / hpeak, 4)}
+        "achieved": round(gbs(gemm_u_bytes, gemm_ms), 1), "peak": hpeak, "unit": "GB/s",
+        "frac": round(gbs(gemm_u_bytes, gemm_ms) / hpeak, 4)}
     # the whole step against the per-layer roofline max(tensor time, mandatory HBM bytes / bandwidth), both at
     # the measured peaks: what an ideal implementation of each layer would need, summed over the sweep
     roof_us_sum = sum(r["roof_us"] for r in layer_rows)
@@ -495,16 +569,65 @@ def run_ours(args):
         "sum_of_layer_rooflines_us": round(roof_us_sum, 1), "step_us": round(ms_step * 1e3, 1),
         "frac": round(roof_us_sum / (ms_step * 1e3), 3),
         "hbm_bound_layers": sum(1 for r in layer_rows if r["bound"] == "hbm"), "layers": len(layer_rows)}
-
     transforms = {
-        "input_transform": {"gbs": round(gbs(in_bytes, in_ms), 1), "frac_of_hbm_peak":
-                            round(gbs(in_bytes, in_ms) / hpeak, 3), "ms_per_step": round(in_ms, 4)},
-        "output_transform": {"gbs": round(gbs(out_bytes, out_ms), 1), "frac_of_hbm_peak":
-                             round(gbs(out_bytes, out_ms) / hpeak, 3), "ms_per_step": round(out_ms, 4)},
-        "filter_transform_once_per_weight": {"ms": round(ft_ms, 4), "gbs": round(ft_bytes / (ft_ms * 1e-3) / 1e9, 1),
-                                             "frac_of_hbm_peak": round(ft_bytes / (ft_ms * 1e-3) / 1e9 / hpeak, 3)},
+        "input_transform": {"gbs": round(gbs(in_bytes, in_ms), 1), "frac_of_hbm_peak": round(gbs(in_bytes, in_ms) / hpeak, 3),
+                            "ms_per_step": round(in_ms, 4)},
+        "output_transform": {"gbs": round(gbs(out_bytes, out_ms), 1), "frac_of_hbm_peak": round(gbs(out_bytes, out_ms) / hpeak, 3),
+                             "ms_per_step": round(out_ms, 4)},
+        "single_kernel_layers_ms_per_step": round(fused_ms, 4),
+        "filter_transform_once_per_weight": {"ms": round(ft_ms, 4), "gbs": round(gbs(ft_bytes, ft_ms), 1),
+                                             "frac_of_hbm_peak": round(gbs(ft_bytes, ft_ms) / hpeak, 3)},
         "hbm_peak_gbs": hpeak, "peak_source": peak_kind,
     }
+
+    # ---- end to end: host buffers in, host buffers out, through the host entry of the C ABI (fp16 or fp32) ----
+    e2e = None
+    if not args.no_e2e:
+        host_call = B.sdwino_conv3x3_host_f32 if io32 else B.sdwino_conv3x3_host
+        staging = B.sdwino_host_staging_bytes_f32 if io32 else B.sdwino_host_staging_bytes
+        e2e_bytes = [staging(L.N, L.C, L.H, L.W, L.K, t) + B.sdwino_workspace_bytes(L.N, L.C, L.H, L.W, L.K, t)
+                     for L, t in zip(layers, tiles)]
+        per_layer_ws = sum(e2e_bytes) <= (48 << 30)
+        # a workspace (staging + scratch) per layer, so that the copies of neighbouring layers may overlap; layers
+        # that share one are ordered copy after copy by the library
+        shared = None if per_layer_ws else B.alloc_workspace(max(e2e_bytes), dev)
+        ws_e2e = [B.alloc_workspace(nb, dev) for nb in e2e_bytes] if per_layer_ws else [shared] * len(layers)
+        if io32:
+            host_io = [(x.float().pin_memory(), w, b.float().pin_memory(), torch.empty(y.shape, dtype=torch.float32).pin_memory())
+                       for (x, w, b, y) in host]
+        else:
+            host_io = host
+        e2e_steps = max(3, min(steps, 30 if flops_step < 2e12 else 10))
+
+        def e2e_step():
+            for t, (x, w, b, y_h), (_, wT, _, _), wsl in zip(tiles, host_io, devt, ws_e2e):
+                host_call(x, wT, b, y_h, t, wsl, stream=stream, wait=False)
+            B.sdwino_host_join(stream)
+            stream.synchronize()                  # y of every layer is complete in host memory
+
+        for _ in range(3):
+            e2e_step()
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            e2e_step()
+        torch.cuda.synchronize()
+        e2e_s = time.perf_counter() - t0
+        e2e_value = aggregate_value(flops_step, world, max_over_ranks(e2e_s, dist, dev) / e2e_steps * 1e3)
+        h2d = sum(x.numel() * x.element_size() + b.numel() * b.element_size() for (x, w, b, y) in host_io)
+        d2h = sum(y.numel() * y.element_size() for (x, w, b, y) in host_io)
+        # what came back through the host path is what the device-resident step computed (same kernels: same bits)
+        e2e_matches = args.epilogue != "none" or all(
+            torch.equal(y_h, yd.cpu()) for (_, _, _, y_h), (_, _, _, yd) in zip(host_io, devt))
+        assert e2e_matches, "the host path returned something else than the device path"
+        e2e = {"value": round(e2e_value, 2), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "steps": e2e_steps, "ms_per_step": round(e2e_s / e2e_steps * 1e3, 3), "matches_device_path": bool(e2e_matches),
+               "api": ("sdwino_conv3x3_host_f32_async" if io32 else "sdwino_conv3x3_host_async") +
+                      " per layer (pinned host x, bias, y; " +
+                      ("a workspace per layer: uploads and downloads overlap the neighbouring layers" if per_layer_ws
+                       else "one shared workspace: the copies of differently sized layers are ordered one after the other") +
+                      "), one join + stream synchronisation per step"}
+        del ws_e2e, shared, host_io
 
     # ---- cuDNN yardstick (not the target) ----
     cudnn = None
@@ -512,7 +635,7 @@ def run_ours(args):
         try:
             import torch.nn.functional as F
             torch.backends.cudnn.benchmark = True
-            wd = [h[1].to(dev) for h in host]
+            wd = [h[1].to(dev).to(io_t) for h in host]
             for _ in range(3):
                 for (xd, _, bd, _), w_ in zip(devt, wd):
                     F.conv2d(xd, w_, bd, padding=1)
@@ -526,82 +649,148 @@ def run_ours(args):
             torch.cuda.synchronize()
             cms = c0.elapsed_time(c1) / prof_steps
             cudnn = {"value": round(flops_step / (cms * 1e-3) / 1e12, 1), "unit": UNIT, "ms_per_step": round(cms, 4),
-                     "what": "torch.nn.functional.conv2d fp16 NCHW, cudnn.benchmark=True (yardstick only)"}
+                     "what": "torch.nn.functional.conv2d NCHW, cudnn.benchmark=True (yardstick only)"}
+            del wd
         except Exception as e:  # pragma: no cover
             cudnn = {"error": repr(e)}
 
-    # ---- oracle on the host cores (reported baseline) ----
+    # ---- oracle on the host cores (reported baseline): the headline workload at one GPU only ----
     cpu_baseline = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if headline and rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
         oracle.build()
         inputs = [(x.numpy(), w.numpy(), b.numpy()) for (x, w, b, _) in host]
-        nch = 160   # about 10-15 s of host work on the default workload
-        sec, fl = oracle_sample(layers, inputs, nch)
+        sec, fl, names = oracle_budgeted_sample(layers, inputs, 12.0)
         cpu_baseline = {"value": fl / sec / 1e12, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
-                        "sample": f"fp64 direct conv of min(K, {nch}) seeded output channels of each of the {len(layers)} "
-                                  f"layers ({fl / 1e9:.1f} GFLOP in {sec:.1f} s)"}
+                        "sample": f"fp64 direct conv of min(K, {oracle.threads()}) seeded output channels of {len(names)} of the "
+                                  f"{len(layers)} layers, taken in a seeded order until 12 s were used "
+                                  f"({fl / 1e9:.1f} GFLOP in {sec:.1f} s): " + ", ".join(names)}
 
-    if rank == 0:
+    rec = {
+        "workload": workload, "value": round(value, 2), "unit": UNIT, "ms_per_step": round(ms_step, 4),
+        "ms_per_step_min": round(min(per_step), 4), "ms_per_step_median": round(statistics.median(per_step), 4),
+        "steps": steps, "direct_launch_ms_per_step": round(direct_ms, 4) if direct_ms is not None else None,
+        "sustained": sustained, "layers_n": len(layers), "batch": layers[0].N, "tile_per_layer": tiles,
+        "launches_per_step": int(launches_per_step), "flops_per_step": flops_step,
+        "l2": ((f"flushed before every timed step (256 MB written): one step touches only {step_bytes / 1e6:.0f} MB")
+               if flush_l2 else
+               (f"no flush: one step touches {step_bytes / 1e6:.0f} MB of distinct inputs, transformed weights and outputs "
+                f"({step_bytes / L2_BYTES:.1f}x the 126 MB L2), so a layer starts with its operands cold")),
+        "e2e": e2e, "roofline": roofline, "transforms": transforms, "cudnn_yardstick": cudnn, "layers": layer_rows,
+        "clocks": clocks, "cpu_baseline": cpu_baseline,
+    }
+    del devt, host, ws, wTs, graph
+    torch.cuda.empty_cache()
+    return rec
+
+
+def run_ours(args):
+    import torch
+    from paper_2412_05781_b200 import build_library
+    build_library()
+    from paper_2412_05781_b200 import binding as B
+
+    ctx = Ctx()
+    ctx.B = B
+    ctx.world = int(os.environ.get("WORLD_SIZE", "1"))
+    ctx.rank = int(os.environ.get("RANK", "0"))
+    ctx.local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the sdwino path has no CPU fallback")
+    torch.cuda.set_device(ctx.local_rank)
+    ctx.dev = torch.device("cuda", ctx.local_rank)
+    ctx.dist = None
+    if ctx.world > 1:
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group("nccl", device_id=ctx.dev)
+        ctx.dist = dist_mod
+    ctx.peaks, ctx.peak_kind = load_peaks()
+    ctx.stream = torch.cuda.Stream()
+    B.sdwino_set_pipeline(args.pipeline, args.pipe_ring, args.pipe_lead)
+
+    head = headline_of(args)
+    names = ALL_WORKLOADS if args.workload == "all" else [args.workload]
+    records = {}
+    for name in names:
+        if name == head:
+            continue
+        records[name] = bench_workload(ctx, args, name, headline=False)
+    records[head] = bench_workload(ctx, args, head, headline=True)   # last: its clocks and CPU baseline are the line's
+    h = records[head]
+    io32 = args.io == "f32"
+
+    if ctx.rank == 0:
+        def brief(r):
+            return {k: r[k] for k in ("value", "unit", "ms_per_step", "ms_per_step_min", "ms_per_step_median", "steps",
+                                      "direct_launch_ms_per_step", "sustained", "layers_n", "batch", "tile_per_layer",
+                                      "launches_per_step", "l2", "e2e", "roofline", "transforms", "cudnn_yardstick", "layers")}
+        e2e = h["e2e"] or {"value": None, "unit": UNIT, "h2d_bytes_per_step": None, "d2h_bytes_per_step": None,
+                           "skipped": "--no-e2e"}
         line = {
-            "metric": metric_name(args.workload), "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": round(ms_step, 4), "higher_is_better": True,
+            "metric": metric_name(head), "value": h["value"], "unit": UNIT, "n_gpus": ctx.world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": h["ms_per_step"], "ms_per_step_min": h["ms_per_step_min"],
+            "ms_per_step_median": h["ms_per_step_median"], "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32 in/out, f16 operands, f32 accumulate" if io32 else "f16",
             "data": "synthetic",
-            "config": {"workload": args.workload, "io": args.io, "layers": len(layers), "layer_subset": args.layers or "all",
-                       "batch": layers[0].N, "tile": args.tile,
-                       "tile_per_layer": tiles,
+            "config": {"workload": head, "io": args.io, "layers": h["layers_n"], "layer_subset": args.layers or "all",
+                       "batch": h["batch"], "tile": args.tile, "tile_per_layer": h["tile_per_layer"],
                        "algorithm": ("Winograd F(2x2,3x3) or F(4x4,3x3) per layer (sdwino_choose_tile)"
                                      if args.tile == "auto" else f"Winograd F({args.tile}x{args.tile},3x3)") +
-                                    (", fp32 x / w / bias / y, fp16 transformed operands, fp32 accumulate (e2e runs the fp16 interface)"
+                                    (", fp32 x / w / bias / y, fp16 transformed operands, fp32 accumulate"
                                      if io32 else ", fp16 storage, fp32 accumulate"),
-                       "parallelism": f"replicas x{world} (no exchange step)",
+                       "parallelism": f"replicas x{ctx.world} (no exchange step)",
                        "launch": "direct" if args.no_graph else "CUDA graph of one step, replayed",
-                       "l2": ((f"flushed before every timed step (256 MB written): one step touches only {step_bytes / 1e6:.0f} MB")
-                              if flush_l2 else
-                              (f"no flush: one step touches {step_bytes / 1e6:.0f} MB of distinct inputs, transformed weights "
-                               f"and outputs ({step_bytes / L2_BYTES:.1f}x the 126 MB L2), so a layer starts with its operands "
-                               "cold")),
+                       "pipeline": {0: "off", 1: "where the library takes it", 2: "wherever possible"}[args.pipeline],
+                       "l2": h["l2"],
                        "filter_transform": "once per weight, before the timed region (reported separately)",
                        "epilogue": {"none": "bias", "residual": "bias + residual, fused, on the layers with more than 8 input and output channels (e2e runs the plain convolution)",
-                                    "residual_silu": "SiLU(bias + residual), fused, on the layers with more than 8 input and output channels (e2e runs the plain convolution)"}[args.epilogue]},
-            "e2e": {"value": round(e2e_value, 2), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "steps": e2e_steps, "matches_device_path": bool(e2e_matches), "api": "sdwino_conv3x3_host_async per layer (pinned host x, bias, y; " +
-                           ("a workspace per layer: uploads and downloads overlap the neighbouring layers" if per_layer_ws
-                            else "one shared workspace: the copies of differently sized layers are ordered one after the other") +
-                           "), one join + stream synchronisation per step"},
-            "gpu_launches": int(launches),
-            "clocks": clocks,
-            "roofline": roofline,
-            "transforms": transforms,
-            "cpu_baseline": cpu_baseline,
-            "cudnn_yardstick": cudnn,
-            "layers": layer_rows,
+                                    "residual_silu": "SiLU(bias + residual), fused, on the layers with more than 8 input and output channels (e2e runs the plain convolution)"}[args.epilogue],
+                       "other_workloads_in_this_line": [n for n in names if n != head]},
+            "e2e": e2e,
+            "gpu_launches": int(h["launches_per_step"] * args.steps),
+            "clocks": h["clocks"],
+            "sustained": h["sustained"],
+            "direct_launch_ms_per_step": h["direct_launch_ms_per_step"],
+            "roofline": h["roofline"],
+            "transforms": h["transforms"],
+            "cpu_baseline": h["cpu_baseline"],
+            "cudnn_yardstick": h["cudnn_yardstick"],
+            "layers": h["layers"],
+            "workloads": {n: brief(records[n]) for n in names},
+            "kernel_source_hash": kernel_source_hash(),
             "paper_context": PAPER_CONTEXT,
         }
         print(json.dumps(line), flush=True)
-    if dist is not None:
-        dist.destroy_process_group()
+    if ctx.dist is not None:
+        ctx.dist.destroy_process_group()
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
-    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default=WORKLOAD, choices=["single", "sd15_unet", "sd_vae_512", "sd21_unet", "sdxl_1024"])
+    ap.add_argument("--workload", default="all", choices=["all"] + ALL_WORKLOADS,
+                    help="all: every workload, the headline on sdxl_1024; a name: that workload alone")
     ap.add_argument("--layers", default="", help="comma-separated layer indices of the workload (default: all)")
     ap.add_argument("--tile", default=TILE, choices=["auto", "2", "4"])
     ap.add_argument("--io", default="f16", choices=["f16", "f32"],
-                    help="element type of x, w, bias and y in the timed step: f32 runs sdwino_conv3x3_f32 (fp16 operands, "
-                         "fp32 accumulation); the end-to-end arm stays fp16")
+                    help="element type of x, w, bias and y: f32 runs the fp32 interface (fp16 operands, fp32 accumulation)")
     ap.add_argument("--epilogue", default="none", choices=["none", "residual", "residual_silu"],
                     help="fuse y = act(conv + bias + residual) into the output transform of the timed step (sdwino_conv3x3_ex)")
+    ap.add_argument("--pipeline", type=int, default=1, choices=[0, 1, 2],
+                    help="the pipelined single-launch path of F(4x4): 0 never, 1 where the library takes it, 2 wherever possible")
+    ap.add_argument("--pipe-ring", type=int, default=0, help="ring length of the pipelined path in blocks of 128 tiles (0: library's choice)")
+    ap.add_argument("--pipe-lead", type=int, default=0, help="lag of its output transform in blocks (0: library's choice)")
     ap.add_argument("--no-graph", action="store_true", help="launch every step directly instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-yardstick", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer pass (profiling runs)")
+    ap.add_argument("--no-sustained", action="store_true", help="skip the two-second back-to-back leg (profiling runs)")
     args = ap.parse_args()
+    if args.layers and args.workload == "all":
+        ap.error("--layers needs a --workload")
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -200,6 +200,17 @@ int sdwino_conv3x3_host_async(const void *x_host, const void *wT, const void *bi
                               int N, int C, int H, int W, int K, int tile,
                               void *workspace, size_t workspace_bytes, void *stream);
 int sdwino_host_join(void *stream);
+/* The host-buffer entries for the fp32 interface (the model type of the "Type F32" rows of the paper's Tables 2
+ * and 3): x_host, bias_host and y_host are fp32 host arrays, wT comes from either filter transform; the staging
+ * part of the workspace is sdwino_host_staging_bytes_f32(...).  Everything else as above; the two families may be
+ * mixed on one stream and are joined by the same sdwino_host_join. */
+size_t sdwino_host_staging_bytes_f32(int N, int C, int H, int W, int K, int tile);
+int sdwino_conv3x3_host_f32(const float *x_host, const void *wT, const float *bias_host, float *y_host,
+                            int N, int C, int H, int W, int K, int tile,
+                            void *workspace, size_t workspace_bytes, void *stream);
+int sdwino_conv3x3_host_f32_async(const float *x_host, const void *wT, const float *bias_host, float *y_host,
+                                  int N, int C, int H, int W, int K, int tile,
+                                  void *workspace, size_t workspace_bytes, void *stream);
 
 /*
  * Device-side waits (on TMA / tensor-core completion barriers) are bounded; a wait that
@@ -267,6 +278,22 @@ int sdwino_choose_tile(int N, int C, int H, int W, int K);
  * Returns SDWINO_ERR_INVALID_ARG for a negative value.  Not thread-safe against concurrent compute calls.
  */
 int sdwino_set_fused_min_tiles(long long p_tiles);
+
+/*
+ * Tuning / test hook for the pipelined single-launch path of F(4x4,3x3) (Section "Techniques": the B200 counterpart
+ * of keeping the transformed data in the nearest memory and of handing work out dynamically).  Layers with
+ * thousands of tiles and filters of at most a few tens of MB run all three steps in ONE persistent, cooperative
+ * launch: V and M live in rings of a few blocks of 128 tiles that stay in L2, transform warps pull (block, channel
+ * group) items from an atomic queue while the GEMM warps of the same CTAs multiply the blocks behind them.
+ * mode 2: wherever the layer shape allows it (fp16 interface, tile 4, W % 8 == 0, 16-byte aligned x and y, more
+ * than 4 input channels, plain convolution, transformed filters of at most 40 MB); mode 0: never; mode 1 (default):
+ * where it is faster, which on the measured layers is nowhere (it moves a third of the DRAM bytes but takes 17-60 %
+ * longer than the three kernels), so today mode 1 behaves like mode 0.
+ * ring / lead: ring slots and the lag of the output transform behind the activation transform, in blocks of 128
+ * tiles; 0 = chosen by the library.  Returns SDWINO_ERR_INVALID_ARG for other values.  Results are the bits of the
+ * three-kernel path.  Safe against concurrent compute calls (a call reads the setting once).
+ */
+int sdwino_set_pipeline(int mode, int ring, int lead);
 
 /*
  * Timing for benchmarks.  mode 1: every kernel launch of the library is bracketed by two CUDA

@@ -24,6 +24,7 @@ EXPORTS = [
     "sdwino_profile_records", "sdwino_set_gemm_shape", "sdwino_conv3x3_static", "sdwino_set_fused_min_tiles", "sdwino_choose_tile",
     "sdwino_selftest_wait_timeout", "sdwino_conv3x3_host_async", "sdwino_host_join", "sdwino_set_input_staging", "sdwino_conv3x3_ex",
     "sdwino_filter_transform_f32", "sdwino_conv3x3_f32", "sdwino_conv3x3_f32_ex",
+    "sdwino_host_staging_bytes_f32", "sdwino_conv3x3_host_f32", "sdwino_conv3x3_host_f32_async", "sdwino_set_pipeline",
 ]
 
 KERNEL_KINDS = ("filter_transform", "input_transform", "wino_gemm", "output_transform", "fused", "layer")
@@ -49,7 +50,8 @@ def _load() -> ctypes.CDLL:
     lib.sdwino_filter_bytes.argtypes = [i, i, i]
     lib.sdwino_filter_transform.restype = i
     lib.sdwino_filter_transform.argtypes = [vp, vp, i, i, i, vp]
-    for name in ("sdwino_workspace_bytes", "sdwino_workspace_min_bytes", "sdwino_host_staging_bytes"):
+    for name in ("sdwino_workspace_bytes", "sdwino_workspace_min_bytes", "sdwino_host_staging_bytes",
+                 "sdwino_host_staging_bytes_f32"):
         getattr(lib, name).restype = sz
         getattr(lib, name).argtypes = [i] * 6
     lib.sdwino_set_workspace.restype = i
@@ -74,6 +76,9 @@ def _load() -> ctypes.CDLL:
     lib.sdwino_host_join.argtypes = [vp]
     lib.sdwino_conv3x3_host_async.restype = i
     lib.sdwino_conv3x3_host_async.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, vp, sz, vp]
+    for name in ("sdwino_conv3x3_host_f32", "sdwino_conv3x3_host_f32_async"):
+        getattr(lib, name).restype = i
+        getattr(lib, name).argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, vp, sz, vp]
     lib.sdwino_last_device_status.restype = i
     lib.sdwino_last_device_status.argtypes = [vp]
     lib.sdwino_launch_count.restype = ctypes.c_ulonglong
@@ -89,6 +94,8 @@ def _load() -> ctypes.CDLL:
     lib.sdwino_choose_tile.argtypes = [i, i, i, i, i]
     lib.sdwino_set_fused_min_tiles.restype = i
     lib.sdwino_set_fused_min_tiles.argtypes = [ctypes.c_longlong]
+    lib.sdwino_set_pipeline.restype = i
+    lib.sdwino_set_pipeline.argtypes = [i, i, i]
     lib.sdwino_profile_enable.restype = i
     lib.sdwino_profile_enable.argtypes = [i]
     lib.sdwino_profile_collect.restype = i
@@ -172,6 +179,12 @@ def sdwino_choose_tile(N: int, C: int, H: int, W: int, K: int) -> int:
 def sdwino_set_fused_min_tiles(p_tiles: int = 0) -> None:
     """Blocks of 128 tiles from which few-output-channel layers take the single fused kernel; 0 = default."""
     _check(lib.sdwino_set_fused_min_tiles(p_tiles), "sdwino_set_fused_min_tiles")
+
+
+def sdwino_set_pipeline(mode: int = 1, ring: int = 0, lead: int = 0) -> None:
+    """Tuning / test hook: 0 never take the pipelined single-launch path, 1 where it is faster, 2 wherever possible;
+    ring / lead in blocks of 128 tiles (0 = chosen by the library)."""
+    _check(lib.sdwino_set_pipeline(mode, ring, lead), "sdwino_set_pipeline")
 
 
 def sdwino_profile_enable(mode) -> None:
@@ -347,6 +360,10 @@ def sdwino_conv3x3_static(x: torch.Tensor, wT: torch.Tensor, bias: Optional[torc
     return y
 
 
+def sdwino_host_staging_bytes_f32(N: int, C: int, H: int, W: int, K: int, tile: int) -> int:
+    return int(lib.sdwino_host_staging_bytes_f32(N, C, H, W, K, tile))
+
+
 def sdwino_host_join(stream: Optional[torch.cuda.Stream] = None) -> None:
     """Make `stream` wait for the downloads of all earlier sdwino_conv3x3_host(..., wait=False) calls."""
     _check(lib.sdwino_host_join(_stream_ptr(stream)), "sdwino_host_join")
@@ -365,4 +382,19 @@ def sdwino_conv3x3_host(x: torch.Tensor, wT: torch.Tensor, bias: Optional[torch.
     rc = fn(x.data_ptr(), wT.data_ptr(), _ptr(bias), y.data_ptr(), N, C, H, W, K, tile,
             workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream_ptr(stream))
     _check(rc, "sdwino_conv3x3_host" if wait else "sdwino_conv3x3_host_async")
+    return y
+
+
+def sdwino_conv3x3_host_f32(x: torch.Tensor, wT: torch.Tensor, bias: Optional[torch.Tensor], y: torch.Tensor,
+                            tile: int, workspace: torch.Tensor, stream=None, wait: bool = True) -> torch.Tensor:
+    """sdwino_conv3x3_host for the fp32 interface: x, bias, y are fp32 CPU tensors; the workspace holds
+    sdwino_host_staging_bytes_f32(...) in front of the scratch."""
+    assert not x.is_cuda and not y.is_cuda and x.dtype == torch.float32 and y.dtype == torch.float32
+    assert x.is_contiguous() and y.is_contiguous() and (bias is None or bias.dtype == torch.float32)
+    N, C, H, W = (int(v) for v in x.shape)
+    K = int(y.shape[1])
+    fn = lib.sdwino_conv3x3_host_f32 if wait else lib.sdwino_conv3x3_host_f32_async
+    rc = fn(x.data_ptr(), wT.data_ptr(), _ptr(bias), y.data_ptr(), N, C, H, W, K, tile,
+            workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    _check(rc, "sdwino_conv3x3_host_f32" if wait else "sdwino_conv3x3_host_f32_async")
     return y

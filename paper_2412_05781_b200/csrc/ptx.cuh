@@ -172,6 +172,11 @@ template <int N>
 __device__ __forceinline__ void tma_store_wait_read_pending() {
     asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
 }
+// Waits until at most N of this thread's bulk groups are still in flight (complete, not just read).
+template <int N>
+__device__ __forceinline__ void tma_store_wait_pending() {
+    asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory");
+}
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 // Make generic-proxy writes to shared memory visible to the async proxy (TMA store source).
 __device__ __forceinline__ void fence_proxy_async_smem() {
@@ -366,6 +371,23 @@ __device__ __forceinline__ void umma_commit_pair(uint64_t* bar) {
             smem_u32(bar)),
         "h"(mask)
         : "memory");
+}
+
+// Orders what this thread has observed or written through the generic proxy before its later async-proxy (TMA)
+// operations, for shared and global memory alike.
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+__device__ __forceinline__ void named_barrier_sync(int id, int count) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+// Named barrier over `count` threads with an AND reduction of `pred`: every participant gets the same answer.
+__device__ __forceinline__ bool named_barrier_and(int id, int count, bool pred) {
+    uint32_t r;
+    asm volatile(
+        "{\n .reg .pred p, q;\n setp.ne.b32 q, %3, 0;\n bar.red.and.pred p, %1, %2, q;\n selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(r)
+        : "r"(id), "r"(count), "r"(static_cast<uint32_t>(pred))
+        : "memory");
+    return r != 0;
 }
 
 __device__ __forceinline__ uint32_t elect_one() {

@@ -35,6 +35,11 @@ std::atomic<int> g_force_ctas{0};
 std::atomic<int> g_input_staging{1};  // 0 never, 1 where it is faster, 2 wherever possible (sdwino_set_input_staging)
 std::atomic<bool> g_disable_fused{false};  // forcing a GEMM shape also forces the GEMM path for few-channel layers
 std::atomic<int> g_force_n_tile{0};
+// Pipelined single-launch path (see wino_gemm.cuh): 0 never, 1 where it is faster, 2 wherever it is possible (tests);
+// ring / lead in blocks of 128 tiles, 0 = chosen by the library.
+std::atomic<int> g_pipe_mode{1};
+std::atomic<int> g_pipe_ring{0};
+std::atomic<int> g_pipe_lead{0};
 void* g_workspace = nullptr;
 size_t g_workspace_bytes = 0;
 
@@ -355,6 +360,27 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
     if (e != cudaSuccess && getenv("SDWINO_LOG"))
         fprintf(stderr, "sdwino: kernel launch failed: %s (grid %u x %u, block %u, %zu bytes of dynamic shared memory)\n",
                 cudaGetErrorString(e), grid.x, grid.y, block.x, smem);
+    return e;
+}
+
+// A cooperative launch (all CTAs resident at once: the pipelined kernel's CTAs wait on one another), ordered after
+// everything before it in the stream.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_coop(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+    if (e != cudaSuccess && getenv("SDWINO_LOG"))
+        fprintf(stderr, "sdwino: cooperative launch failed: %s (grid %u, block %u, %zu bytes of dynamic shared memory)\n",
+                cudaGetErrorString(e), grid.x, block.x, smem);
     return e;
 }
 
@@ -740,7 +766,7 @@ int launch_gemm_shape(const CUtensorMap& tmU, const CUtensorMap& tmV, const CUte
                                                     prm.epi_alias ? 0 : prm.epi_bufs,
                                                     RES ? prm.num_c_blocks * L::b_bytes(prm.n_tile)
                                                         : (DUAL ? prm.stages * L::A_BYTES : 0))),
-                   st, CTAS, tmU, tmV, tmM, prm, status);
+                   st, CTAS, tmU, tmV, tmM, prm, status, PipeParams{});
     if (e != cudaSuccess && getenv("SDWINO_LOG"))
         fprintf(stderr, "sdwino: GEMM launch failed: %s (grid %d, stages %d, n_tile %d, resident %d)\n", cudaGetErrorString(e),
                 grid, prm.stages, prm.n_tile, prm.resident);
@@ -758,6 +784,169 @@ int launch_gemm(const CUtensorMap& tmU, const CUtensorMap& tmV, const CUtensorMa
     if (prm.resident) return launch_gemm_shape<1, true>(tmU, tmV, tmM, prm, sms, status, st);
     if (prm.dual) return launch_gemm_shape<1, false, true>(tmU, tmV, tmM, prm, sms, status, st);
     return launch_gemm_shape<1, false>(tmU, tmV, tmM, prm, sms, status, st);
+}
+
+
+// ---- the pipelined single-launch path for F(4x4) layers with many tiles and filters that stay in L2 ----
+// Workspace: V ring [36][C][ring * 128], M ring [36][K][ring * 128], then the counters.
+struct PipePlan {
+    int n_tile, resident, group, stages, epi_rows, epi_bufs, epi_chunks;
+    int ring, lead, nb;
+    size_t v_bytes, m_bytes, ctr_bytes;
+};
+constexpr int PIPE_CG = 20, PIPE_KG = 20;   // channels per transform item: four rounds of the team's five channel lanes
+
+bool plan_pipeline(const Plan& pl, int C, int K, int sms, int mode, PipePlan* pp) {
+    using L = GemmSmemLayout;
+    const int nb = static_cast<int>(pl.P128 / GEMM_BLOCK_P);
+    const int cblocks = (C + GEMM_BLOCK_C - 1) / GEMM_BLOCK_C;
+    const size_t u_bytes = static_cast<size_t>(pl.a2) * pl.Kb * pl.Cb * 2048;
+    if (pl.a2 != 36 || nb < 1) return false;
+    // the filters are read again for every block of tiles: they must stay in L2 beside the rings
+    if (u_bytes > (40u << 20)) return false;
+    // Measured on every long layer of the SD VAE / SDXL sweeps the pipelined launch moves a third of the DRAM bytes of
+    // the three kernels but takes 17-60 % longer (512->512 at 256x256: 204 against 170 us; 256->256 at 512x512: 408
+    // against 257 us): its ten transform warps per SM cannot hide their memory latency the way the transform kernels do
+    // with 12-20 resident warps and TMA staging, and the GEMM roles lose time to the per-tile dependency checks.  The
+    // library therefore never takes it by itself; mode 2 is for callers who trade time for DRAM traffic, and for tests.
+    if (mode == 1) return false;
+    const int smem_budget = MAX_DYN_SMEM - 1024;
+    // Filter-resident shape first: one (position, k-tile) pair per group of CTAs for the whole launch, so the filter
+    // block is loaded once per CTA; the largest n_tile whose block fits beside three or more stages of V.
+    pp->resident = 0;
+    for (int n = GEMM_MAX_N; n >= 16; n -= 16) {
+        const int ktiles = (K + n - 1) / n;
+        if (n > 16 && ktiles == (K + n - 17) / (n - 16)) continue;     // a smaller n needs as many tiles
+        const int keys = ktiles * pl.a2;
+        if (keys > sms) break;
+        const bool split = (n / 2) % 16 == 0;
+        const int grp = split ? n / 2 : n;
+        const int rows = (grp > 64 && grp % 64 == 0) ? 64 : grp;
+        const int bufs = split ? 2 : 1;
+        const int ures = cblocks * L::b_bytes(n);
+        const int stages = (smem_budget - L::dyn_bytes(0, 0, rows, bufs, ures)) / L::A_BYTES;
+        if (stages < 3) continue;
+        pp->resident = 1;
+        pp->n_tile = n;
+        pp->group = sms / keys;
+        pp->stages = stages > GEMM_MAX_STAGES ? GEMM_MAX_STAGES : stages;
+        pp->epi_rows = rows;
+        pp->epi_bufs = bufs;
+        pp->epi_chunks = grp / rows;
+        break;
+    }
+    if (!pp->resident) {
+        const GemmShape shape = choose_gemm_shape(K, C, nb >= 16 ? nb : 16, pl.a2, sms, 1);
+        pp->n_tile = shape.n_tile;
+        pp->group = 1;
+        const bool split = (pp->n_tile / 2) % 16 == 0;
+        pp->epi_rows = split ? pp->n_tile / 2 : pp->n_tile;
+        pp->epi_bufs = split ? 2 : 1;
+        pp->epi_chunks = 1;
+        pp->stages = (smem_budget - L::dyn_bytes(pp->n_tile, 0, pp->epi_rows, pp->epi_bufs)) / L::stage_bytes(pp->n_tile);
+        if (pp->stages > GEMM_MAX_STAGES) pp->stages = GEMM_MAX_STAGES;
+        if (pp->stages < 2) return false;
+    }
+    const int keys = ((K + pp->n_tile - 1) / pp->n_tile) * pl.a2;
+    const int inflight = (sms + keys - 1) / keys;          // blocks of tiles the GEMM roles work on at a time
+    int lead = g_pipe_lead.load(), ring = g_pipe_ring.load();
+    if (lead <= 0) lead = inflight + 2;
+    if (ring <= 0) ring = lead + inflight + 3;
+    if (ring > nb) ring = nb;
+    if (ring < 1) ring = 1;
+    pp->lead = lead;
+    pp->ring = ring;
+    pp->nb = nb;
+    auto up = [](size_t v) { return (v + WS_ALIGN - 1) / WS_ALIGN * WS_ALIGN; };
+    pp->v_bytes = up(static_cast<size_t>(pl.a2) * C * ring * GEMM_BLOCK_P * sizeof(__half));
+    pp->m_bytes = up(static_cast<size_t>(pl.a2) * K * ring * GEMM_BLOCK_P * sizeof(__half));
+    pp->ctr_bytes = up((3 * static_cast<size_t>(nb) + 8) * sizeof(unsigned int));
+    return true;
+}
+
+int launch_pipeline(const __half* x, const void* wT, const __half* bias, __half* y, const Plan& pl, const TileGeom& geo,
+                    int C, int K, const PipePlan& pq, void* ws, cudaStream_t st) {
+    using L = GemmSmemLayout;
+    const int sms = sm_count();
+    int* status = status_word_ptr();
+    if (sms <= 0 || !status) return err_cuda(__LINE__);
+    uint8_t* base = static_cast<uint8_t*>(ws);
+    __half* V = reinterpret_cast<__half*>(base);
+    __half* Mws = reinterpret_cast<__half*>(base + pq.v_bytes);
+    unsigned int* ctr = reinterpret_cast<unsigned int*>(base + pq.v_bytes + pq.m_bytes);
+    const long long ring_p = static_cast<long long>(pq.ring) * GEMM_BLOCK_P;
+
+    GemmParams prm;
+    prm.wt_header = wt_header_of(wT);
+    prm.K = K;
+    prm.tile = 4;
+    prm.n_tile = pq.n_tile;
+    prm.num_k_tiles = (K + pq.n_tile - 1) / pq.n_tile;
+    prm.num_p_tiles = pq.nb;
+    prm.num_pos = pl.a2;
+    prm.num_c_blocks = (C + GEMM_BLOCK_C - 1) / GEMM_BLOCK_C;
+    prm.C = C;
+    prm.stages = pq.stages;
+    prm.epi_rows = pq.epi_rows;
+    prm.epi_bufs = pq.epi_bufs;
+    prm.epi_chunks = pq.epi_chunks;
+    prm.resident = pq.resident;
+    prm.group = pq.group;
+    prm.epi_alias = 0;
+    prm.dual = 0;
+    prm.p_stride = ring_p;
+
+    PipeParams pp;
+    pp.v_ready = ctr;
+    pp.m_done = ctr + pq.nb;
+    pp.o_done = ctr + 2 * static_cast<size_t>(pq.nb);
+    pp.q_head = ctr + 3 * static_cast<size_t>(pq.nb);
+    pp.abort_word = reinterpret_cast<int*>(ctr + 3 * static_cast<size_t>(pq.nb) + 1);
+    pp.num_pblocks = pq.nb;
+    pp.ring = pq.ring;
+    pp.lead = pq.lead;
+    pp.cg = PIPE_CG;
+    pp.kg = PIPE_KG;
+    pp.it_items = (C + PIPE_CG - 1) / PIPE_CG;
+    pp.ot_items = (K + PIPE_KG - 1) / PIPE_KG;
+    pp.m_target = static_cast<unsigned int>(prm.num_k_tiles * pl.a2 * pq.epi_bufs);
+    pp.x = x;
+    pp.V = V;
+    pp.Mws = Mws;
+    pp.bias = bias;
+    pp.y = y;
+    pp.geo = geo;
+    pp.fd64 = make_fastdiv(64);
+    {
+        // blocks of tiles between two consecutive tiles of one CTA
+        const int keys = prm.num_k_tiles * pl.a2;
+        const int dist = pq.resident ? pq.group : (sms + keys - 1) / keys + 1;
+        pp.defer = pq.ring > dist + 1 ? 1 : 0;
+    }
+
+    CUtensorMap tmU, tmV, tmM;
+    if (!encode_filter_map(&tmU, wt_filters_of(wT), pl.Cb, pl.Kb, pl.a2, pq.n_tile / 16) ||
+        !encode_map(&tmV, V, ring_p, C, pl.a2, ring_p, static_cast<uint64_t>(C) * ring_p, 64, GEMM_BLOCK_C, true) ||
+        !encode_map(&tmM, Mws, ring_p, K, pl.a2, ring_p, static_cast<uint64_t>(K) * ring_p, GEMM_BLOCK_P, prm.epi_rows, false))
+        return err_cuda(__LINE__);
+    if (cudaMemsetAsync(ctr, 0, (3 * static_cast<size_t>(pq.nb) + 8) * sizeof(unsigned int), st) != cudaSuccess)
+        return err_cuda(__LINE__);
+    const size_t smem = static_cast<size_t>(
+        L::dyn_bytes(pq.resident ? 0 : pq.n_tile, pq.stages, pq.epi_rows, pq.epi_bufs,
+                     pq.resident ? prm.num_c_blocks * L::b_bytes(pq.n_tile) : 0));
+    ProfScope prof(KIND_FUSED, st);
+    cudaError_t e;
+    if (pq.resident) {
+        if (!ensure_dyn_smem(reinterpret_cast<const void*>(wino_gemm_kernel<1, true, false, true>), MAX_DYN_SMEM)) return err_cuda(__LINE__);
+        e = launch_coop(wino_gemm_kernel<1, true, false, true>, dim3(sms), dim3(PIPE_THREADS), smem, st, tmU, tmV, tmM, prm,
+                        status, pp);
+    } else {
+        if (!ensure_dyn_smem(reinterpret_cast<const void*>(wino_gemm_kernel<1, false, false, true>), MAX_DYN_SMEM)) return err_cuda(__LINE__);
+        e = launch_coop(wino_gemm_kernel<1, false, false, true>, dim3(sms), dim3(PIPE_THREADS), smem, st, tmU, tmV, tmM, prm,
+                        status, pp);
+    }
+    g_launches.fetch_add(1);
+    return e == cudaSuccess ? SDWINO_OK : err_cuda(__LINE__);
 }
 
 
@@ -813,6 +1002,19 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
         __half* yh = static_cast<__half*>(y);
         if (tile == 4) return launch_fused_small_c<4, 4>(xh, wT, bh, yh, geo, C, K, pl.Kb, pl.Cb, st);
         return launch_fused_small_c_mma(xh, wT, bh, yh, geo, C, K, pl.Kb, st);
+    }
+
+    // Long F(4x4) layers with small filters: one pipelined launch in which V and M are rings that stay in L2.
+    {
+        const int pipe_mode = g_pipe_mode.load();
+        PipePlan pq;
+        if (pipe_mode != 0 && plain && tile == 4 && force_ctas == 0 && force_n_tile == 0 && !use_fused_small_c(C, tile) &&
+            W % 8 == 0 && aligned(x, 16) && aligned(y, 16) && plan_pipeline(pl, C, K, sm_count(), pipe_mode, &pq) &&
+            pq.v_bytes + pq.m_bytes + pq.ctr_bytes <= ws_bytes) {
+            const TileGeom geo = make_geom(H, W, pl.TH, pl.TW, pl.P);
+            return launch_pipeline(static_cast<const __half*>(x), wT, static_cast<const __half*>(bias), static_cast<__half*>(y),
+                                   pl, geo, C, K, pq, ws, st);
+        }
     }
 
     // workspace: V[a2][C][pc] then M[a2][K][pc]; pc is a multiple of 128 elements, so every row starts
@@ -966,6 +1168,14 @@ int sdwino_set_input_staging(int mode) {
     return SDWINO_OK;
 }
 
+int sdwino_set_pipeline(int mode, int ring, int lead) {
+    if (mode < 0 || mode > 2 || ring < 0 || lead < 0) return SDWINO_ERR_INVALID_ARG;
+    g_pipe_mode.store(mode);
+    g_pipe_ring.store(ring);
+    g_pipe_lead.store(lead);
+    return SDWINO_OK;
+}
+
 int sdwino_choose_tile(int N, int C, int H, int W, int K) {
     if (N <= 0 || C <= 0 || H <= 0 || W <= 0 || K <= 0) return 0;
     // Layers with few input channels have a single-kernel F(2x2) path.  Otherwise F(4x4) moves 2.25 instead of 4 transform
@@ -1096,14 +1306,23 @@ int sdwino_conv3x3(const void* x, const void* wT, const void* bias, void* y, int
     return conv_impl(x, wT, bias, y, N, C, H, W, K, tile, ws, bytes, static_cast<cudaStream_t>(stream));
 }
 
-size_t sdwino_host_staging_bytes(int N, int C, int H, int W, int K, int tile) {
+namespace {
+size_t host_staging_bytes(int N, int C, int H, int W, int K, int tile, size_t elem) {
     Plan pl;
     if (!make_plan(N, C, H, W, K, tile, &pl)) return 0;
     auto up = [](size_t v) { return (v + WS_ALIGN - 1) / WS_ALIGN * WS_ALIGN; };
-    const size_t xb = up(static_cast<size_t>(N) * C * H * W * sizeof(__half));
-    const size_t yb = up(static_cast<size_t>(N) * K * H * W * sizeof(__half));
-    const size_t bb = up(static_cast<size_t>(K) * sizeof(__half));
+    const size_t xb = up(static_cast<size_t>(N) * C * H * W * elem);
+    const size_t yb = up(static_cast<size_t>(N) * K * H * W * elem);
+    const size_t bb = up(static_cast<size_t>(K) * elem);
     return 2 * (xb + bb + yb);   // two slots: uploads, kernels and downloads of consecutive calls overlap
+}
+}  // namespace
+
+size_t sdwino_host_staging_bytes(int N, int C, int H, int W, int K, int tile) {
+    return host_staging_bytes(N, C, H, W, K, tile, sizeof(__half));
+}
+size_t sdwino_host_staging_bytes_f32(int N, int C, int H, int W, int K, int tile) {
+    return host_staging_bytes(N, C, H, W, K, tile, sizeof(float));
 }
 
 namespace {
@@ -1148,20 +1367,22 @@ HostPipe* host_pipe() {
 }
 }  // namespace
 
-int sdwino_conv3x3_host_async(const void* x_host, const void* wT, const void* bias_host, void* y_host, int N, int C,
-                              int H, int W, int K, int tile, void* workspace, size_t workspace_bytes, void* stream) {
+namespace {
+int host_async_impl(const void* x_host, const void* wT, const void* bias_host, void* y_host, int N, int C,
+                    int H, int W, int K, int tile, void* workspace, size_t workspace_bytes, void* stream, bool io32) {
     if (!x_host || !y_host || !wT) return SDWINO_ERR_INVALID_ARG;
     if (tile != 2 && tile != 4) return SDWINO_ERR_UNSUPPORTED;
-    const size_t staging = sdwino_host_staging_bytes(N, C, H, W, K, tile);
+    const size_t elem = io32 ? sizeof(float) : sizeof(__half);
+    const size_t staging = host_staging_bytes(N, C, H, W, K, tile, elem);
     if (staging == 0) return SDWINO_ERR_INVALID_ARG;
     if (!workspace || workspace_bytes <= staging) return SDWINO_ERR_WORKSPACE;
     if (!aligned(workspace, WS_ALIGN)) return SDWINO_ERR_MISALIGNED;
     HostPipe* hp = host_pipe();
     if (!hp) return err_cuda(__LINE__);
     auto up = [](size_t v) { return (v + WS_ALIGN - 1) / WS_ALIGN * WS_ALIGN; };
-    const size_t xbytes = static_cast<size_t>(N) * C * H * W * sizeof(__half);
-    const size_t ybytes = static_cast<size_t>(N) * K * H * W * sizeof(__half);
-    const size_t bbytes = static_cast<size_t>(K) * sizeof(__half);
+    const size_t xbytes = static_cast<size_t>(N) * C * H * W * elem;
+    const size_t ybytes = static_cast<size_t>(N) * K * H * W * elem;
+    const size_t bbytes = static_cast<size_t>(K) * elem;
     uint8_t* base = static_cast<uint8_t*>(workspace);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
@@ -1215,7 +1436,8 @@ int sdwino_conv3x3_host_async(const void* x_host, const void* wT, const void* bi
     if (cudaEventRecord(me.uploaded, hp->s_in) != cudaSuccess) return err_cuda(__LINE__);
     // kernels on the caller's stream
     if (cudaStreamWaitEvent(st, me.uploaded, 0) != cudaSuccess) return err_cuda(__LINE__);
-    const int rc = conv_impl(xd, wT, bias_host ? bd : nullptr, yd, N, C, H, W, K, tile, ws, workspace_bytes - staging, st);
+    const int rc = conv_impl(xd, wT, bias_host ? bd : nullptr, yd, N, C, H, W, K, tile, ws, workspace_bytes - staging, st,
+                             Epilogue{nullptr, 0}, io32);
     if (rc != SDWINO_OK) return rc;
     if (cudaEventRecord(me.computed, st) != cudaSuccess) return err_cuda(__LINE__);
     // download on the second copy stream
@@ -1231,6 +1453,17 @@ int sdwino_conv3x3_host_async(const void* x_host, const void* wT, const void* bi
     me.slot = slot;
     ++hp->calls;
     return SDWINO_OK;
+}
+}  // namespace
+
+int sdwino_conv3x3_host_async(const void* x_host, const void* wT, const void* bias_host, void* y_host, int N, int C,
+                              int H, int W, int K, int tile, void* workspace, size_t workspace_bytes, void* stream) {
+    return host_async_impl(x_host, wT, bias_host, y_host, N, C, H, W, K, tile, workspace, workspace_bytes, stream, false);
+}
+
+int sdwino_conv3x3_host_f32_async(const float* x_host, const void* wT, const float* bias_host, float* y_host, int N, int C,
+                                  int H, int W, int K, int tile, void* workspace, size_t workspace_bytes, void* stream) {
+    return host_async_impl(x_host, wT, bias_host, y_host, N, C, H, W, K, tile, workspace, workspace_bytes, stream, true);
 }
 
 int sdwino_host_join(void* stream) {
@@ -1248,6 +1481,16 @@ int sdwino_conv3x3_host(const void* x_host, const void* wT, const void* bias_hos
                         int W, int K, int tile, void* workspace, size_t workspace_bytes, void* stream) {
     const int rc = sdwino_conv3x3_host_async(x_host, wT, bias_host, y_host, N, C, H, W, K, tile, workspace,
                                              workspace_bytes, stream);
+    if (rc != SDWINO_OK) return rc;
+    if (sdwino_host_join(stream) != SDWINO_OK) return err_cuda(__LINE__);
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return err_cuda(__LINE__);
+    return SDWINO_OK;
+}
+
+int sdwino_conv3x3_host_f32(const float* x_host, const void* wT, const float* bias_host, float* y_host, int N, int C,
+                            int H, int W, int K, int tile, void* workspace, size_t workspace_bytes, void* stream) {
+    const int rc = sdwino_conv3x3_host_f32_async(x_host, wT, bias_host, y_host, N, C, H, W, K, tile, workspace,
+                                                 workspace_bytes, stream);
     if (rc != SDWINO_OK) return rc;
     if (sdwino_host_join(stream) != SDWINO_OK) return err_cuda(__LINE__);
     if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return err_cuda(__LINE__);

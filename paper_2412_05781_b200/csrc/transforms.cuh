@@ -568,7 +568,9 @@ input_transform_vec_kernel(const XT* __restrict__ x, __half* __restrict__ V, Til
 // permutes.  The kernel is bound by instruction issue, so this is where its time goes: 3-10 % per layer over
 // the generic vector kernel.  CH = 1 is what runs: with 2 or 4 channels per thread the per-thread set-up is
 // amortised, but the serial load -> compute chain per channel and the lower thread count cost more (measured).
-template <int CH, typename XT = __half>
+// EARLY (fp16 input): all six row segments of a channel are loaded before the first one is used, so that a thread
+// pays one memory latency per channel instead of six: for callers that run few warps per SM.
+template <int CH, typename XT = __half, bool PDL = true, bool EARLY = false>
 __device__ __forceinline__ void input_unit_f4(const XT* __restrict__ x, __half* __restrict__ V, const TileGeom& geo,
                                               int C, long long p_begin, const FastDiv& gdiv, long long Pstride,
                                               uint32_t idx) {
@@ -601,10 +603,27 @@ __device__ __forceinline__ void input_unit_f4(const XT* __restrict__ x, __half* 
     // The index arithmetic above needs nothing from memory and runs while the preceding kernel drains.  Wait
     // first, release the GEMM second: once the GEMM runs, everything before this kernel has completed, which is
     // what lets it fetch its filters (written at the latest by the kernel before this one) early.
-    pdl_wait();
-    pdl_launch_dependents();
+    if constexpr (PDL) {   // (a caller inside a larger kernel orders its own reads)
+        pdl_wait();
+        pdl_launch_dependents();
+    }
     for (int cc = 0; cc < cend; ++cc) {
         float2 e2[A][A];   // e2[r][nu]: rows transformed along the columns, (tile 0, tile 1)
+        [[maybe_unused]] uint4 raw_v[A];
+        [[maybe_unused]] uint32_t raw_l[A], raw_r[A];
+        if constexpr (EARLY && sizeof(XT) == 2) {
+#pragma unroll
+            for (int r = 0; r < A; ++r) {
+                raw_v[r] = make_uint4(0u, 0u, 0u, 0u);
+                raw_l[r] = raw_r[r] = 0u;
+                if ((rowmask >> r) & 1) {
+                    const __half* rp = reinterpret_cast<const __half*>(xp) + r * geo.W;
+                    raw_v[r] = __ldg(reinterpret_cast<const uint4*>(rp));
+                    if (left_ok) raw_l[r] = __ldg(reinterpret_cast<const uint32_t*>(rp - 2));
+                    if (right_ok) raw_r[r] = __ldg(reinterpret_cast<const uint32_t*>(rp + 8));
+                }
+            }
+        }
 #pragma unroll
         for (int r = 0; r < A; ++r) {
             float2 d[A];
@@ -628,7 +647,9 @@ __device__ __forceinline__ void input_unit_f4(const XT* __restrict__ x, __half* 
             } else {
             uint4 v = make_uint4(0u, 0u, 0u, 0u);
             uint32_t lw = 0u, rw = 0u;   // aligned words before / after the segment
-            if ((rowmask >> r) & 1) {
+            if constexpr (EARLY) {
+                v = raw_v[r]; lw = raw_l[r]; rw = raw_r[r];
+            } else if ((rowmask >> r) & 1) {
                 const __half* rp = xp + r * geo.W;
                 v = __ldg(reinterpret_cast<const uint4*>(rp));
                 if (left_ok) lw = __ldg(reinterpret_cast<const uint32_t*>(rp - 2));
@@ -728,7 +749,9 @@ __device__ __forceinline__ void store_row8_f32_res(float* rowp, float (&v)[8], c
     reinterpret_cast<float4*>(rowp)[1] = make_float4(v[4], v[5], v[6], v[7]);
 }
 
-template <int M, int TPT, bool EP, typename YT = __half>
+// LIVE: M is being written by other SMs during this launch (the pipelined kernel): its loads then bypass L1, which
+// is not coherent across SMs and may still hold an earlier occupant of a ring slot.
+template <int M, int TPT, bool EP, typename YT = __half, bool LIVE = false>
 __device__ __forceinline__ void output_unit_vec(const __half* __restrict__ Mws, const YT* __restrict__ bias,
                                                 YT* __restrict__ y, const TileGeom& geo, int K, long long p_begin,
                                                 const FastDiv& gdiv, long long Pstride, uint32_t idx, const Epilogue& ep) {
@@ -750,7 +773,8 @@ __device__ __forceinline__ void output_unit_vec(const __half* __restrict__ Mws, 
             float2 col[A], o[M];
 #pragma unroll
             for (int r = 0; r < A; ++r) {
-                const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(src + (r * A + s) * plane));
+                const uint32_t* wp = reinterpret_cast<const uint32_t*>(src + (r * A + s) * plane);
+                const uint32_t w = LIVE ? __ldcg(wp) : __ldg(wp);
                 col[r] = __half22float2(*reinterpret_cast<const __half2*>(&w));
             }
             at4_packed(col, o);

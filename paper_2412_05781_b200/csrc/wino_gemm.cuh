@@ -41,6 +41,7 @@
 #include <cuda_fp16.h>
 
 #include "ptx.cuh"
+#include "transforms.cuh"
 
 namespace sdw {
 
@@ -53,6 +54,8 @@ constexpr int GEMM_BLOCK_P = 128;  // tiles per output tile (TMEM lanes, UMMA M)
 constexpr int GEMM_BLOCK_C = 64;   // input channels per pipeline stage (one 128-byte swizzle row of U)
 constexpr int GEMM_MAX_N = 256;    // output channels per output tile (UMMA N), multiple of 16
 constexpr int GEMM_THREADS = 320;  // warp 0 producer, warp 1 MMA, warps 2-9 epilogue (two groups of four)
+constexpr int PIPE_TRANSFORM_THREADS = 320;                            // pipelined mode: warps 10-19 run the transforms, each on its own
+constexpr int PIPE_THREADS = GEMM_THREADS + PIPE_TRANSFORM_THREADS;
 constexpr int GEMM_MAX_STAGES = 8;
 constexpr uint64_t GEMM_WAIT_LIMIT_NS = 2000000000ull;  // a wait longer than 2 s is reported, not spun on
 
@@ -60,7 +63,7 @@ struct GemmSmemLayout {
     static constexpr int A_BYTES = GEMM_BLOCK_P * GEMM_BLOCK_C * 2;          // two [64 p][64 c] boxes
     static constexpr int A_BOX_BYTES = 64 * GEMM_BLOCK_C * 2;
     static constexpr int EPI_ROW_BYTES = GEMM_BLOCK_P * 2;                   // one staged row: 128 p fp16
-    static constexpr int BAR_BYTES = (2 * GEMM_MAX_STAGES + 6) * 8 + 16;
+    static constexpr int BAR_BYTES = (2 * GEMM_MAX_STAGES + 6) * 8 + 16 + 16;   // barriers, two words, four item slots
     // `rows` = rows of U this CTA loads per stage: n_tile (single CTA) or n_tile / 2 (CTA pair)
     __host__ __device__ static constexpr int b_bytes(int rows) { return rows * GEMM_BLOCK_C * 2; }
     __host__ __device__ static constexpr int stage_bytes(int rows) {
@@ -99,17 +102,87 @@ struct GemmParams {
     long long p_stride;  // tiles per pass (row pitch of V and M)
 };
 
+// Pipelined mode (template flag PIPE): the three steps of a layer run inside ONE persistent launch.  V and M are rings
+// of `ring` blocks of 128 tiles that stay in L2; ten extra warps per CTA pull transform items -- the activation
+// transform of (block of tiles, group of input channels) and, `lead` blocks behind it, the output transform of (block,
+// group of output channels) -- from an atomic queue, while the GEMM roles walk the (block, position, k-tile) tiles in
+// block order.  Counters in global memory carry the dependencies:
+//   v_ready[b]  activation-transform items of block b completed       (the producer waits for it_items before it loads V)
+//   m_done[b]   epilogue groups that have stored their part of M of b (an output item waits for m_target; so does the
+//               activation transform of block b + ring, which overwrites the V slot of b)
+//   o_done[b]   output-transform items of block b completed           (the epilogue of block b + ring waits for ot_items
+//               before it overwrites the M slot)
+// Every item depends only on items earlier in queue order, and every role works through its list in order, so the
+// earliest unfinished item can always run: the scheme cannot deadlock as long as all CTAs are resident (the launch is
+// cooperative).  Every wait is bounded all the same and gives up through the status word and the abort word.
+struct PipeParams {
+    unsigned int* v_ready;
+    unsigned int* m_done;
+    unsigned int* o_done;
+    unsigned int* q_head;      // next transform item
+    int* abort_word;           // set by the first wait that gives up: every other wait then returns
+    int num_pblocks;           // blocks of 128 tiles in the layer
+    int ring;                  // ring slots (blocks of 128 tiles) of V and of M
+    int lead;                  // the output items of block j - lead are queued behind the activation items of block j
+    int it_items, ot_items;    // items per block: ceil(C / cg), ceil(K / kg)
+    int cg, kg;                // channels per item
+    unsigned int m_target;     // (position, k-tile) pairs x epilogue groups that store
+    const __half* x;
+    __half* V;                 // ring [pos][C][ring * 128]
+    const __half* Mws;         // ring [pos][K][ring * 128]
+    const __half* bias;
+    __half* y;
+    TileGeom geo;
+    FastDiv fd64;              // division by 64 (pairs of tiles per block)
+    int defer;                 // 1: a tile's stores are announced one tile later (needs ring > distance between a CTA's tiles)
+};
+
+__device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int* p) {
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+// Spins until *ctr >= target.  Bounded: gives up after limit_ns, or as soon as the abort word is set.
+__device__ __noinline__ bool wait_counter(const unsigned int* ctr, unsigned int target, const int* abort_word,
+                                          uint64_t limit_ns) {
+    unsigned int polls = 0;
+    uint64_t t0 = 0;
+    for (;;) {
+        unsigned int v;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ctr) : "memory");
+        if (v >= target) return true;
+        if ((++polls & 63u) == 0u) {
+            if (*reinterpret_cast<const volatile int*>(abort_word) != 0) return false;
+            const uint64_t now = global_timer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > limit_ns) return false;
+        }
+        __nanosleep(40);
+    }
+}
+// Publishes the stores made before it (by this thread, and by the threads it has synchronised with) and counts up.
+__device__ __forceinline__ void signal_counter(unsigned int* ctr) {
+    __threadfence();
+    atomicAdd(ctr, 1u);
+}
+// The same as one release operation (for a thread whose own earlier writes have already completed).
+__device__ __forceinline__ void signal_counter_release(unsigned int* ctr) {
+    asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(ctr) : "memory");
+}
+
 // tmV: fp16 [pos][C][Pstride]   box {64 p, 64 c, 1},      128B swizzle  (A operand; rows c >= C read as 0)
 // tmU: fp16 [pos][Cb][Kb][16][64] box {64 c, 16 k, 1, n_tile/16, 1}, 128B swizzle (B operand: n_tile rows of 128
 //      bytes in k order; blocks past Kb read as 0)
 // tmM: fp16 [pos][K][Pstride]   box {128 p, epi_rows k, 1}, no swizzle  (result; rows k >= K are clipped)
 // RES: the filter-resident mode, DUAL: two blocks of 128 tiles per CTA tile; separate instantiations, so that the
 // plain streaming kernel pays nothing for them.
-template <int CTAS, bool RES = false, bool DUAL = false>
-__global__ void __launch_bounds__(GEMM_THREADS, 1)
+template <int CTAS, bool RES = false, bool DUAL = false, bool PIPE = false>
+__global__ void __launch_bounds__(PIPE ? PIPE_THREADS : GEMM_THREADS, 1)
 wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant__ CUtensorMap tmV,
-                 const __grid_constant__ CUtensorMap tmM, const GemmParams prm, int* __restrict__ status_word) {
+                 const __grid_constant__ CUtensorMap tmM, const GemmParams prm, int* __restrict__ status_word,
+                 const PipeParams pp) {
     using L = GemmSmemLayout;
+    static_assert(!PIPE || (CTAS == 1 && !DUAL), "the pipelined mode runs single CTAs, one block of tiles per CTA tile");
     // The activation transform before this kernel has waited for everything before it, so the filter header is
     // final: its load is issued first and looked at after the set-up below (uniform over the CTA).
     const uint4 wt_hdr = *reinterpret_cast<const uint4*>(prm.wt_header);
@@ -140,6 +213,7 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
     uint64_t* ures_empty_bar = ures_full_bar + 1;    // the MMAs that read it have completed
     uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(ures_empty_bar + 1);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_base_slot + 1);
+    [[maybe_unused]] volatile unsigned int* item_slots = reinterpret_cast<volatile unsigned int*>(tmem_base_slot + 2);   // 4 words
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -168,6 +242,23 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
         } else {
             const int r = i / run_len;
             return (grp_id + r * num_groups) * prm.num_p_tiles + grp_lane + (i - r * run_len) * grp_size;
+        }
+    };
+
+    // tile -> (block of tiles pt, k-tile kt, position pos).  The plain list has the tiles p fastest (all CTAs at one
+    // position: its filters are small and V streams); the pipelined streaming list has them slowest, so that the
+    // CTAs move through the blocks of tiles together, behind the transform that produces them.
+    auto decode = [&](int tile, int& pt, int& kt, int& pos) {
+        if constexpr (PIPE && !RES) {
+            const int keys = prm.num_k_tiles * prm.num_pos;
+            pt = tile / keys;
+            const int key = tile - pt * keys;
+            pos = key / prm.num_k_tiles;
+            kt = key - pos * prm.num_k_tiles;
+        } else {
+            pt = tile % prm.num_p_tiles;
+            kt = (tile / prm.num_p_tiles) % prm.num_k_tiles;
+            pos = tile / (prm.num_p_tiles * prm.num_k_tiles);
         }
     };
 
@@ -221,9 +312,8 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
             uint32_t reloads = 0;
             if (my_count > 0) {
                 // the filters do not depend on the preceding kernel: the first block goes out before the wait
-                const int t0 = tile_of(0);
-                const int kt = (t0 / prm.num_p_tiles) % prm.num_k_tiles;
-                const int pos = t0 / (prm.num_p_tiles * prm.num_k_tiles);
+                int pt, kt, pos;
+                decode(tile_of(0), pt, kt, pos);
                 load_filters(pos, kt);
                 cur_key = pos * prm.num_k_tiles + kt;
             }
@@ -232,11 +322,11 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
             uint32_t phase = 0;
             uint32_t sa = smem_base, fb = full0;
             bool ok = true;
+            [[maybe_unused]] int seen_pt = -1;            // pipelined mode: the block whose counter was read ahead
+            [[maybe_unused]] unsigned int seen = 0;
             for (int i = 0; i < my_count && ok; ++i) {
-                const int tile = tile_of(i);
-                const int pt = tile % prm.num_p_tiles;
-                const int kt = (tile / prm.num_p_tiles) % prm.num_k_tiles;
-                const int pos = tile / (prm.num_p_tiles * prm.num_k_tiles);
+                int pt, kt, pos;
+                decode(tile_of(i), pt, kt, pos);
                 if (pos * prm.num_k_tiles + kt != cur_key) {
                     // the MMAs of the previous run of tiles have finished reading the resident block
                     ok = mbar_wait_bounded(ures_empty_bar, reloads & 1u, abort_flag, GEMM_WAIT_LIMIT_NS);
@@ -245,7 +335,22 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
                     load_filters(pos, kt);
                     cur_key = pos * prm.num_k_tiles + kt;
                 }
-                const int p0 = pt * GEMM_BLOCK_P;
+                int p0 = pt * GEMM_BLOCK_P;
+                if constexpr (PIPE) {
+                    // V of this block of tiles is written by the transform warps of this launch.  The counter was read
+                    // one tile ahead (the read is a round trip to L2 on this one thread's critical path).
+                    if (seen_pt != pt || seen < static_cast<unsigned int>(pp.it_items)) {
+                        ok = wait_counter(&pp.v_ready[pt], static_cast<unsigned int>(pp.it_items), pp.abort_word, GEMM_WAIT_LIMIT_NS);
+                        if (!ok) { if (*abort_flag == 0) report_timeout(status_word, 12, cta_rank); break; }
+                    }
+                    fence_proxy_async_all();
+                    p0 = (pt % pp.ring) * GEMM_BLOCK_P;
+                    if (i + 1 < my_count) {
+                        int kt1, pos1;
+                        decode(tile_of(i + 1), seen_pt, kt1, pos1);
+                        seen = ld_acquire_u32(&pp.v_ready[seen_pt]);
+                    }
+                }
                 for (int c0 = 0; c0 < prm.C; c0 += GEMM_BLOCK_C) {
                     ok = mbar_wait_bounded(&empty_bar[stage], phase ^ 1u, abort_flag, GEMM_WAIT_LIMIT_NS);
                     if (!ok) { if (*abort_flag == 0) report_timeout(status_word, 1, cta_rank); break; }
@@ -266,18 +371,19 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
             const uint32_t full0_local = smem_u32(&full_bar[0]);
             const uint32_t full0 = CTAS == 2 ? map_to_cta(full0_local, 0) : full0_local;
             uint32_t sa = smem_base, fb = full0, fb_local = full0_local;
-            // The filters do not depend on the preceding kernel (the activation transform), and the kernel
-            // before that has completed by the time this one runs (the filter transform never releases its
-            // dependents early): the filter loads of the first ring-full of stages go out before the wait, so
-            // the weight stream from HBM starts while the activation transform is still running.
-            const uint64_t u_policy = l2_policy_evict_first();
+            // The filters do not depend on the preceding kernel (the activation transform), and everything before
+            // that kernel has completed by the time this one runs: every activation transform waits for its
+            // predecessors first and releases its dependents second, whatever came before it (a filter transform
+            // releases its own dependents at once).  So the filter loads of the first ring-full of stages go out
+            // before the wait, and the weight stream from HBM starts while the activation transform is still running.
+            // (pipelined mode: the filters are read again for every block of tiles and must stay in L2)
+            const uint64_t u_policy = PIPE ? l2_policy_evict_last() : l2_policy_evict_first();
             int pre = 0;
             if constexpr (CTAS == 1) {
                 uint32_t sa_u = smem_base + a_bytes, fb_u = full0;
                 for (int i = 0; i < my_count && pre < stages; ++i) {
-                    const int tile = tile_of(i);
-                    const int kt = (tile / prm.num_p_tiles) % prm.num_k_tiles;
-                    const int pos = tile / (prm.num_p_tiles * prm.num_k_tiles);
+                    int pt, kt, pos;
+                    decode(tile_of(i), pt, kt, pos);
                     const int k0 = kt * prm.n_tile;
                     for (int c0 = 0; c0 < prm.C && pre < stages; c0 += GEMM_BLOCK_C) {
                         mbar_arrive_expect_tx_a32(fb_u, tx_bytes);
@@ -293,12 +399,27 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
             int issued = 0;
             uint32_t phase = 0;
             bool ok = true;
+            [[maybe_unused]] int seen_pt = -1;            // pipelined mode: the block whose counter was read ahead
+            [[maybe_unused]] unsigned int seen = 0;
             for (int i = 0; i < my_count && ok; ++i) {
-                const int tile = tile_of(i);
-                const int pt = tile % prm.num_p_tiles;
-                const int kt = (tile / prm.num_p_tiles) % prm.num_k_tiles;
-                const int pos = tile / (prm.num_p_tiles * prm.num_k_tiles);
-                const int p0 = (pt * CTAS * PT + static_cast<int>(cta_rank)) * GEMM_BLOCK_P;
+                int pt, kt, pos;
+                decode(tile_of(i), pt, kt, pos);
+                int p0 = (pt * CTAS * PT + static_cast<int>(cta_rank)) * GEMM_BLOCK_P;
+                if constexpr (PIPE) {
+                    // V of this block of tiles is written by the transform warps of this launch (counter read one
+                    // tile ahead, as in the filter-resident producer)
+                    if (seen_pt != pt || seen < static_cast<unsigned int>(pp.it_items)) {
+                        ok = wait_counter(&pp.v_ready[pt], static_cast<unsigned int>(pp.it_items), pp.abort_word, GEMM_WAIT_LIMIT_NS);
+                        if (!ok) { if (*abort_flag == 0) report_timeout(status_word, 12, cta_rank); break; }
+                    }
+                    fence_proxy_async_all();
+                    p0 = (pt % pp.ring) * GEMM_BLOCK_P;
+                    if (i + 1 < my_count) {
+                        int kt1, pos1;
+                        decode(tile_of(i + 1), seen_pt, kt1, pos1);
+                        seen = ld_acquire_u32(&pp.v_ready[seen_pt]);
+                    }
+                }
                 const int k0 = kt * prm.n_tile + static_cast<int>(cta_rank) * b_rows;
                 for (int c0 = 0; c0 < prm.C; c0 += GEMM_BLOCK_C) {
                     if (issued < pre) {
@@ -447,7 +568,7 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
             }
             if (!ok) *abort_flag = 1;
         }
-    } else {
+    } else if (warp < GEMM_THREADS / 32) {
         // ------------------------------ epilogue ------------------------------
         const int quarter = warp & 3;          // TMEM lanes this warp may read: 32*quarter .. +31
         pdl_wait();   // nothing is written to global memory before the predecessor has completed
@@ -459,15 +580,23 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
         const uint32_t acc_empty_addr0 = CTAS == 2 ? map_to_cta(smem_u32(&acc_empty_bar[0]), 0) : 0u;
         // one iteration per accumulator: a tile of two blocks of 128 tiles p (DUAL) fills both buffers, which are
         // drained in turn exactly as two consecutive tiles would be
+        [[maybe_unused]] int pend_pt = -1;     // pipelined mode, group_tid 0: block whose stores are to be announced
         for (int i2 = 0; i2 < my_count * PT; ++i2) {
-            const int tile = tile_of(i2 / PT);
-            const int pt = (tile % prm.num_p_tiles) * PT + (i2 % PT);
-            const int kt = (tile / prm.num_p_tiles) % prm.num_k_tiles;
-            const int pos = tile / (prm.num_p_tiles * prm.num_k_tiles);
+            int pt, kt, pos;
+            decode(tile_of(i2 / PT), pt, kt, pos);
+            pt = pt * PT + (i2 % PT);
+            // the staging buffer about to be overwritten must have been read by the group's previous TMA store
+            if (group_tid == 0) tma_store_wait_read_pending<0>();
+            [[maybe_unused]] unsigned int seen_o = 0;
+            if constexpr (PIPE) {
+                if (group_tid == 0 && pt >= pp.ring) seen_o = ld_acquire_u32(&pp.o_done[pt - pp.ring]);   // used before the store
+            }
             bool ok = mbar_wait_bounded(&acc_full_bar[buf], acc_phase, abort_flag, GEMM_WAIT_LIMIT_NS);
-            ok = __all_sync(0xffffffffu, ok);
+            // The four warps of a group give up together or not at all (a warp that left on its own would leave the
+            // other three at the group's named barrier for good); the same barrier orders the reuse of the buffer.
+            ok = named_barrier_and(1 + group, 128, ok);
             if (!ok) {
-                if (lane == 0) {
+                if (group_tid == 0) {
                     if (*abort_flag == 0) report_timeout(status_word, 4, cta_rank);
                     *abort_flag = 1;
                 }
@@ -476,7 +605,7 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
             tc_fence_after_sync();
             const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                                     static_cast<uint32_t>(buf * GEMM_MAX_N);
-            const int p0 = (pt * CTAS + static_cast<int>(cta_rank)) * GEMM_BLOCK_P + quarter * 32;
+            const int p0 = ((PIPE ? pt % pp.ring : pt * CTAS) + static_cast<int>(cta_rank)) * GEMM_BLOCK_P + quarter * 32;
             const int k0 = kt * prm.n_tile;
             const bool p_ok = p0 < prm.p_stride;   // the second CTA of the last pair may hang over the pass
             // lane = tile p, registers = output channels: staging row k receives 32 consecutive p from
@@ -487,10 +616,11 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
             const int row0 = (group * chunks + ch) * prm.epi_rows;
             if (row0 < prm.n_tile) {
                 uint8_t* stg = epi_base + group * prm.epi_rows * L::EPI_ROW_BYTES;
-                // the buffer about to be overwritten must have been read by the group's previous TMA store
-                if (group_tid == 0) tma_store_wait_read_pending<0>();
-                if (group == 0) asm volatile("bar.sync 1, 128;" ::: "memory");
-                else asm volatile("bar.sync 2, 128;" ::: "memory");
+                if (ch > 0) {   // (the first piece of a tile is ordered by the barrier after the accumulator wait)
+                    if (group_tid == 0) tma_store_wait_read_pending<0>();
+                    if (group == 0) asm volatile("bar.sync 1, 128;" ::: "memory");
+                    else asm volatile("bar.sync 2, 128;" ::: "memory");
+                }
                 __half* dst = reinterpret_cast<__half*>(stg) + quarter * 32 + lane;
                 int col = 0;
                 for (; col + 32 <= prm.epi_rows; col += 32) {
@@ -511,8 +641,47 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
                 if (group == 0) asm volatile("bar.sync 1, 128;" ::: "memory");
                 else asm volatile("bar.sync 2, 128;" ::: "memory");
                 if (group_tid == 0) {
-                    if (p_ok) tma_store_3d_hint(&tmM, stg, p0 - quarter * 32, k0 + row0, pos, l2_policy_evict_last());
+                    bool slot_free = true;
+                    if constexpr (PIPE) {
+                        // the slot of M still holds block pt - ring until its output transform has read it (the
+                        // counter was read at the start of the tile)
+                        if (ch == 0 && pt >= pp.ring) {
+                            if (seen_o < static_cast<unsigned int>(pp.ot_items))
+                                slot_free = wait_counter(&pp.o_done[pt - pp.ring], static_cast<unsigned int>(pp.ot_items),
+                                                         pp.abort_word, GEMM_WAIT_LIMIT_NS);
+                            if (!slot_free) {
+                                if (*abort_flag == 0) report_timeout(status_word, 13, cta_rank);
+                                *abort_flag = 1;
+                            }
+                            fence_proxy_async_all();
+                        }
+                    }
+                    if (p_ok && (slot_free || *abort_flag == 0))
+                        tma_store_3d_hint(&tmM, stg, p0 - quarter * 32, k0 + row0, pos, l2_policy_evict_last());
                     tma_store_commit();
+                    if constexpr (PIPE) {
+                        if (ch == chunks - 1) {
+                            if (pp.defer) {
+                                // Announce the tile BEFORE this one: its stores were issued a whole tile ago, so
+                                // waiting for all but the newest `chunks` groups returns at once.  (The host sets
+                                // `defer` only when the ring is longer than the distance between two tiles of a CTA:
+                                // otherwise the transform that feeds the next tile could be waiting for this very
+                                // announcement.)
+                                if (pend_pt >= 0) {
+                                    if (chunks == 1) tma_store_wait_pending<1>();
+                                    else if (chunks == 2) tma_store_wait_pending<2>();
+                                    else tma_store_wait_pending<4>();
+                                    fence_proxy_async_all();
+                                    signal_counter_release(&pp.m_done[pend_pt]);
+                                }
+                            } else {
+                                tma_store_wait_all();
+                                fence_proxy_async_all();
+                                signal_counter_release(&pp.m_done[pt]);
+                            }
+                            pend_pt = pt;
+                        }
+                    }
                 }
             }
             }   // chunks
@@ -526,12 +695,95 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
             buf ^= 1;
             if (buf == 0) acc_phase ^= 1u;
         }
-        if (group_tid == 0) tma_store_wait_all();
+        if (group_tid == 0) {
+            tma_store_wait_all();
+            if constexpr (PIPE) {
+                if (pp.defer && pend_pt >= 0 && *abort_flag == 0) {
+                    fence_proxy_async_all();
+                    signal_counter_release(&pp.m_done[pend_pt]);
+                }
+            }
+        }
+    } else if constexpr (PIPE) {
+        // ------------------------------ transforms (pipelined mode) ------------------------------
+        // The transform warps work as one team through the queue of transform items: one thread takes the next item
+        // and waits for what it depends on, then every thread handles one pair of tiles of one channel per round.
+        // (Warps that pull items independently of one another were built too: with ten times as many waiting
+        // parties polling the same few counters in L2 the whole launch ran 1.5-3x slower.)  Queue order, for
+        // j = 0, 1, ...: the activation-transform items of block j, then the output-transform items of block j - lead.
+        const int tt = static_cast<int>(threadIdx.x) - GEMM_THREADS;       // 0 .. 319: (channel lane, pair of tiles)
+        const unsigned int NB = static_cast<unsigned int>(pp.num_pblocks);
+        const unsigned int D = static_cast<unsigned int>(pp.lead) < NB ? static_cast<unsigned int>(pp.lead) : NB;
+        const unsigned int n_it = static_cast<unsigned int>(pp.it_items), n_ot = static_cast<unsigned int>(pp.ot_items);
+        const unsigned int head = D * n_it, per = n_it + n_ot, body = (NB - D) * per, total = NB * per;
+        const long long ring_p = static_cast<long long>(pp.ring) * GEMM_BLOCK_P;
+        const Epilogue no_ep{nullptr, 0};
+        unsigned int iter = 0;
+        int pend_kind = -1, pend_pb = 0;      // thread 0: the item just finished, announced after the team barrier
+        for (;;) {
+            __threadfence();                                   // this thread's stores of the previous item
+            named_barrier_sync(3, PIPE_TRANSFORM_THREADS);     // everyone has finished the previous item
+            if (tt == 0) {
+                if (pend_kind == 0) atomicAdd(&pp.v_ready[pend_pb], 1u);
+                else if (pend_kind == 1) atomicAdd(&pp.o_done[pend_pb], 1u);
+                const unsigned int idx = atomicAdd(pp.q_head, 1u);
+                int kind = -1;
+                unsigned int pb = 0, sub = 0;
+                if (idx < head) {
+                    kind = 0; pb = idx / n_it; sub = idx - pb * n_it;
+                } else if (idx - head < body) {
+                    const unsigned int r0 = idx - head, jj = r0 / per, r = r0 - jj * per;
+                    if (r < n_it) { kind = 0; pb = D + jj; sub = r; }
+                    else { kind = 1; pb = jj; sub = r - n_it; }
+                } else if (idx < total) {
+                    const unsigned int r0 = idx - head - body, jj = r0 / n_ot;
+                    kind = 1; pb = NB - D + jj; sub = r0 - jj * n_ot;
+                }
+                bool ok = true;
+                // an activation item overwrites the V slot of block pb - ring: its GEMM tiles must have completed
+                if (kind == 0 && pb >= static_cast<unsigned int>(pp.ring))
+                    ok = wait_counter(&pp.m_done[pb - pp.ring], pp.m_target, pp.abort_word, GEMM_WAIT_LIMIT_NS);
+                // an output item reads M of block pb: all (position, k-tile) tiles of the block must have been stored
+                if (kind == 1) ok = wait_counter(&pp.m_done[pb], pp.m_target, pp.abort_word, GEMM_WAIT_LIMIT_NS);
+                if (!ok) {
+                    if (*reinterpret_cast<volatile int*>(pp.abort_word) == 0) report_timeout(status_word, 14, 0);
+                    *reinterpret_cast<volatile int*>(pp.abort_word) = 1;
+                    kind = -1;
+                }
+                pend_kind = kind;
+                pend_pb = static_cast<int>(pb);
+                item_slots[(iter & 1u) * 2u] = static_cast<unsigned int>(kind + 1) | (sub << 2);
+                item_slots[(iter & 1u) * 2u + 1u] = pb;
+            }
+            named_barrier_sync(4, PIPE_TRANSFORM_THREADS);
+            const unsigned int w0 = item_slots[(iter & 1u) * 2u], pb = item_slots[(iter & 1u) * 2u + 1u];
+            ++iter;
+            const int kind = static_cast<int>(w0 & 3u) - 1;
+            const int sub = static_cast<int>(w0 >> 2);
+            if (kind < 0) break;
+            const long long slot_off = static_cast<long long>(pb % static_cast<unsigned int>(pp.ring)) * GEMM_BLOCK_P;
+            const long long p_begin = static_cast<long long>(pb) * GEMM_BLOCK_P;
+            const uint32_t pair = static_cast<uint32_t>(tt & 63);        // which two tiles of the block
+            if (kind == 0) {
+                const int c_end = (sub + 1) * pp.cg < prm.C ? (sub + 1) * pp.cg : prm.C;
+                for (int c = sub * pp.cg + (tt >> 6); c < c_end; c += PIPE_TRANSFORM_THREADS / 64)
+                    input_unit_f4<1, __half, false, true>(pp.x, pp.V + slot_off, pp.geo, prm.C, p_begin, pp.fd64, ring_p,
+                                                          static_cast<uint32_t>(c) * 64u + pair);
+            } else {
+                const int k_end = (sub + 1) * pp.kg < prm.K ? (sub + 1) * pp.kg : prm.K;
+                for (int k = sub * pp.kg + (tt >> 6); k < k_end; k += PIPE_TRANSFORM_THREADS / 64)
+                    output_unit_vec<4, 2, false, __half, true>(pp.Mws + slot_off, pp.bias, pp.y, pp.geo, prm.K, p_begin,
+                                                               pp.fd64, ring_p, static_cast<uint32_t>(k) * 64u + pair, no_ep);
+            }
+        }
     }
 
     __syncwarp();
     __syncthreads();
     if (*abort_flag != 0) {
+        if constexpr (PIPE) {
+            if (threadIdx.x == 0) *reinterpret_cast<volatile int*>(pp.abort_word) = 1;   // the other CTAs stop waiting
+        }
         // give copies and MMAs that may still be in flight a bounded time to land before TMEM and
         // shared memory are released
         const uint64_t t0 = global_timer_ns();
