@@ -140,6 +140,17 @@ int sdwino_filter_transform_f32(const float *w, void *wT, int K, int C, int tile
 int sdwino_conv3x3_f32(const float *x, const void *wT, const float *bias, float *y,
                        int N, int C, int H, int W, int K, int tile,
                        void *workspace, size_t workspace_bytes, void *stream);
+/* The fp32 convolution for activations of any fp32 magnitude (the "Type F32" rows of the paper's Tables 2 and 3 run
+ * fp32 models, whose activations are not bound to the fp16 range).  V and M are fp16 inside the library; this entry
+ * first finds max|x| (one extra pass over x), multiplies x by the power of two that brings that maximum near 64 on its
+ * way into V and multiplies the result by the inverse on its way out of M, so that neither overflows nor loses its
+ * small values; powers of two round nothing.  Same arguments as sdwino_conv3x3_f32; the last 1 KiB of the workspace
+ * holds the maximum (a workspace of sdwino_workspace_bytes still gives one pass).  The relative accuracy is that of
+ * sdwino_conv3x3_f32 on inputs of moderate size: 1e-2 * max|ref| as long as max|y| / max|x| stays below about 500
+ * (M must still fit fp16 after the scaling).  Layers with few channels take the three-kernel path here. */
+int sdwino_conv3x3_f32_scaled(const float *x, const void *wT, const float *bias, float *y,
+                              int N, int C, int H, int W, int K, int tile,
+                              void *workspace, size_t workspace_bytes, void *stream);
 /* y = act(conv3x3(x) + bias + residual) with fp32 tensors: sdwino_conv3x3_ex for the fp32 interface (residual fp32
  * [N][K][H][W] or NULL, may be y itself; activation SDWINO_ACT_NONE or SDWINO_ACT_SILU; nothing is rounded). */
 int sdwino_conv3x3_f32_ex(const float *x, const void *wT, const float *bias, const float *residual, float *y,

@@ -25,6 +25,7 @@ EXPORTS = [
     "sdwino_selftest_wait_timeout", "sdwino_conv3x3_host_async", "sdwino_host_join", "sdwino_set_input_staging", "sdwino_conv3x3_ex",
     "sdwino_filter_transform_f32", "sdwino_conv3x3_f32", "sdwino_conv3x3_f32_ex",
     "sdwino_host_staging_bytes_f32", "sdwino_conv3x3_host_f32", "sdwino_conv3x3_host_f32_async", "sdwino_set_pipeline",
+    "sdwino_conv3x3_f32_scaled",
 ]
 
 KERNEL_KINDS = ("filter_transform", "input_transform", "wino_gemm", "output_transform", "fused", "layer")
@@ -68,6 +69,8 @@ def _load() -> ctypes.CDLL:
     lib.sdwino_filter_transform_f32.argtypes = [vp, vp, i, i, i, vp]
     lib.sdwino_conv3x3_f32.restype = i
     lib.sdwino_conv3x3_f32.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, vp, sz, vp]
+    lib.sdwino_conv3x3_f32_scaled.restype = i
+    lib.sdwino_conv3x3_f32_scaled.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, vp, sz, vp]
     lib.sdwino_conv3x3_f32_ex.restype = i
     lib.sdwino_conv3x3_f32_ex.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, i, vp, sz, vp]
     lib.sdwino_conv3x3_host.restype = i
@@ -305,8 +308,10 @@ def sdwino_filter_transform_f32(w: torch.Tensor, tile: int, stream=None) -> torc
 
 
 def sdwino_conv3x3_f32(x: torch.Tensor, wT: torch.Tensor, bias: Optional[torch.Tensor], K: int, tile: int,
-                       workspace: torch.Tensor, y: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
-    """The convolution with fp32 x [N, C, H, W], bias [K] (or None) and y [N, K, H, W]."""
+                       workspace: torch.Tensor, y: Optional[torch.Tensor] = None, stream=None,
+                       scaled: bool = False) -> torch.Tensor:
+    """The convolution with fp32 x [N, C, H, W], bias [K] (or None) and y [N, K, H, W].  scaled=True calls
+    sdwino_conv3x3_f32_scaled: activations of any fp32 magnitude."""
     assert x.is_cuda and x.dtype == torch.float32 and x.is_contiguous() and x.dim() == 4
     N, C, H, W = (int(v) for v in x.shape)
     if y is None:
@@ -314,10 +319,10 @@ def sdwino_conv3x3_f32(x: torch.Tensor, wT: torch.Tensor, bias: Optional[torch.T
     assert y.is_cuda and y.is_contiguous() and y.dtype == torch.float32 and tuple(y.shape) == (N, K, H, W)
     if bias is not None:
         assert bias.is_cuda and bias.dtype == torch.float32 and bias.numel() == K and bias.is_contiguous()
-    rc = lib.sdwino_conv3x3_f32(x.data_ptr(), wT.data_ptr(), _ptr(bias), y.data_ptr(), N, C, H, W, K, tile,
-                                workspace.data_ptr(), workspace.numel() * workspace.element_size(),
-                                _stream_ptr(stream))
-    _check(rc, "sdwino_conv3x3_f32")
+    fn = lib.sdwino_conv3x3_f32_scaled if scaled else lib.sdwino_conv3x3_f32
+    rc = fn(x.data_ptr(), wT.data_ptr(), _ptr(bias), y.data_ptr(), N, C, H, W, K, tile,
+            workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    _check(rc, "sdwino_conv3x3_f32_scaled" if scaled else "sdwino_conv3x3_f32")
     return y
 
 

@@ -65,6 +65,8 @@ output_transform_f4_tma_kernel(const __grid_constant__ CUtensorMap tmM, const YT
     long long n = 0;
     if (tile_ok) decode_tile(geo, p, n, th, tw);
     const long long hw = static_cast<long long>(geo.H) * geo.W;
+    [[maybe_unused]] float ys = 1.f;
+    if constexpr (sizeof(YT) == 4) ys = scalbnf(1.f, range_exponent(ep.amax));   // after the wait above: the word is final
     const int i0 = M * th, j0 = M * tw;
     const long long pix = static_cast<long long>(i0) * geo.W + j0;    // first output pixel inside a channel image
 
@@ -131,6 +133,10 @@ output_transform_f4_tma_kernel(const __grid_constant__ CUtensorMap tmM, const YT
             float2 o[M];
             at4_packed(tt[i], o);
             if (i0 + i >= geo.H) continue;
+            if constexpr (sizeof(YT) == 4) {
+#pragma unroll
+                for (int j = 0; j < M; ++j) { o[j].x *= ys; o[j].y *= ys; }
+            }
             float v[8] = {o[0].x + b, o[1].x + b, o[2].x + b, o[3].x + b, o[0].y + b, o[1].y + b, o[2].y + b, o[3].y + b};
             if constexpr (EP && sizeof(YT) == 4)
                 store_row8_f32_res(reinterpret_cast<float*>(img) + static_cast<long long>(i) * geo.W, v, resf[i], ep);

@@ -404,7 +404,7 @@ int launch_filter(const WT* w, void* wT, int K, int C, int Kb, int Cb, cudaStrea
 
 template <int M, typename XT>
 int launch_input(const XT* x, __half* V, const TileGeom& geo, int C, long long p_begin, int p_count,
-                 long long Pstride, cudaStream_t st) {
+                 long long Pstride, cudaStream_t st, const float* amax = nullptr) {
     ProfScope prof(KIND_INPUT, st);
     constexpr int TPT = 8 / M;
     cudaError_t e;
@@ -415,15 +415,15 @@ int launch_input(const XT* x, __half* V, const TileGeom& geo, int C, long long p
             const long long threads = static_cast<long long>(p_count / TPT) * ((C + CH - 1) / CH);
             dim3 grid(static_cast<unsigned>((threads + 127) / 128));
             e = launch_pdl(input_transform_f4_kernel<CH, XT>, grid, dim3(128), 0, st, 0, x, V, geo, C, p_begin,
-                           make_fastdiv(static_cast<uint32_t>(p_count / TPT)), Pstride);
+                           make_fastdiv(static_cast<uint32_t>(p_count / TPT)), Pstride, amax);
         } else {
             dim3 grid(static_cast<unsigned>((units + 127) / 128));
             e = launch_pdl(input_transform_vec_kernel<M, TPT, XT>, grid, dim3(128), 0, st, 0, x, V, geo, C, p_begin,
-                           make_fastdiv(static_cast<uint32_t>(p_count / TPT)), Pstride);
+                           make_fastdiv(static_cast<uint32_t>(p_count / TPT)), Pstride, amax);
         }
     } else {
         const dim3 grid = grid_rows((p_count + 127) / 128, C);
-        e = launch_pdl(input_transform_kernel<M, XT>, grid, dim3(128), 0, st, 0, x, V, geo, C, p_begin, p_count, Pstride);
+        e = launch_pdl(input_transform_kernel<M, XT>, grid, dim3(128), 0, st, 0, x, V, geo, C, p_begin, p_count, Pstride, amax);
     }
     g_launches.fetch_add(1);
     return e == cudaSuccess ? SDWINO_OK : err_cuda(__LINE__);
@@ -951,8 +951,8 @@ int launch_pipeline(const __half* x, const void* wT, const __half* bias, __half*
 
 
 int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, int C, int H, int W, int K, int tile,
-              void* ws, size_t ws_bytes, cudaStream_t st, const Epilogue& ep = Epilogue{nullptr, 0},
-              bool io32 = false) {   // io32: x, bias and y are fp32 (the filters come from the fp32 filter transform)
+              void* ws, size_t ws_bytes, cudaStream_t st, const Epilogue& ep_in = Epilogue{nullptr, 0, nullptr},
+              bool io32 = false, bool range_safe = false) {   // io32: x, bias and y are fp32 (the filters come from the fp32 filter transform)
     if (tile != 2 && tile != 4) {
         return (N <= 0 || C <= 0 || H <= 0 || W <= 0 || K <= 0 || !x || !wT || !y) ? SDWINO_ERR_INVALID_ARG
                                                                                      : SDWINO_ERR_UNSUPPORTED;
@@ -978,8 +978,28 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
         const long long lcm = static_cast<long long>(pl.TW) / a * GEMM_BLOCK_P;
         if (pc >= lcm && !io32 && use_input_tma(g0, N, C, x, 0, lcm)) pc = pc / lcm * lcm;
     }
+    Epilogue ep = ep_in;
+    if (range_safe) {
+        // fp32 interface, range-safe call: max|x| goes into a word at the end of the workspace, which the transforms
+        // read (see range_exponent); the single-kernel paths are not taken
+        if (!io32 || ws_bytes < 2 * WS_ALIGN) return io32 ? SDWINO_ERR_WORKSPACE : SDWINO_ERR_INVALID_ARG;
+        ws_bytes -= WS_ALIGN;
+        unsigned int* word = reinterpret_cast<unsigned int*>(static_cast<uint8_t*>(ws) + ws_bytes);
+        pc = tiles_per_pass(pl, ws_bytes);
+        if (pc < GEMM_BLOCK_P) return SDWINO_ERR_WORKSPACE;
+        const long long n = static_cast<long long>(N) * C * H * W;
+        const int sms = sm_count();
+        if (sms <= 0) return err_cuda(__LINE__);
+        if (cudaMemsetAsync(word, 0, sizeof(unsigned int), st) != cudaSuccess) return err_cuda(__LINE__);
+        const long long want = (n / 4 + 255) / 256;
+        const unsigned blocks = static_cast<unsigned>(std::min<long long>(std::max<long long>(want, 1), 8ll * sms));
+        if (launch_pdl(absmax_kernel, dim3(blocks), dim3(256), 0, st, 0, static_cast<const float*>(x), n, word) != cudaSuccess)
+            return err_cuda(__LINE__);
+        g_launches.fetch_add(1);
+        ep.amax = reinterpret_cast<const float*>(word);
+    }
     // the single-kernel paths end at the bias
-    const bool no_ep = ep.residual == nullptr && ep.act == 0;
+    const bool no_ep = ep.residual == nullptr && ep.act == 0 && ep.amax == nullptr;
     const bool plain = no_ep && !io32;
     if (no_ep && use_fused_small_k(K, W, tile, pl.P128 / 128, x, y) && !use_fused_small_c(C, tile) &&
         (!io32 || aligned(y, 8)) && !disable_fused) {
@@ -1122,7 +1142,8 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
         int rc;
         if (io32) {
             const float* xf = static_cast<const float*>(x);
-            rc = tile == 2 ? launch_input<2>(xf, V, geo, C, p0, count, pc, st) : launch_input<4>(xf, V, geo, C, p0, count, pc, st);
+            rc = tile == 2 ? launch_input<2>(xf, V, geo, C, p0, count, pc, st, ep.amax)
+                           : launch_input<4>(xf, V, geo, C, p0, count, pc, st, ep.amax);
         } else if (tile == 2) rc = launch_input<2>(xh, V, geo, C, p0, count, pc, st);
         else {
             rc = use_input_tma(geo, N, C, x, p0, count) ? launch_input_tma(xh, V, geo, N, C, p0, count, pc, st)
@@ -1276,13 +1297,19 @@ int sdwino_conv3x3_ex(const void* x, const void* wT, const void* bias, const voi
     if (activation != SDWINO_ACT_NONE && activation != SDWINO_ACT_SILU) return SDWINO_ERR_UNSUPPORTED;
     if (residual && !aligned(residual, 2)) return SDWINO_ERR_MISALIGNED;
     return conv_impl(x, wT, bias, y, N, C, H, W, K, tile, workspace, workspace_bytes, static_cast<cudaStream_t>(stream),
-                     Epilogue{residual, activation});
+                     Epilogue{residual, activation, nullptr});
 }
 
 int sdwino_conv3x3_f32(const float* x, const void* wT, const float* bias, float* y, int N, int C, int H, int W, int K,
                        int tile, void* workspace, size_t workspace_bytes, void* stream) {
     return conv_impl(x, wT, bias, y, N, C, H, W, K, tile, workspace, workspace_bytes, static_cast<cudaStream_t>(stream),
-                     Epilogue{nullptr, 0}, true);
+                     Epilogue{nullptr, 0, nullptr}, true);
+}
+
+int sdwino_conv3x3_f32_scaled(const float* x, const void* wT, const float* bias, float* y, int N, int C, int H, int W,
+                              int K, int tile, void* workspace, size_t workspace_bytes, void* stream) {
+    return conv_impl(x, wT, bias, y, N, C, H, W, K, tile, workspace, workspace_bytes, static_cast<cudaStream_t>(stream),
+                     Epilogue{nullptr, 0, nullptr}, true, true);
 }
 
 int sdwino_conv3x3_f32_ex(const float* x, const void* wT, const float* bias, const float* residual, float* y, int N,
@@ -1291,7 +1318,7 @@ int sdwino_conv3x3_f32_ex(const float* x, const void* wT, const float* bias, con
     if (activation != SDWINO_ACT_NONE && activation != SDWINO_ACT_SILU) return SDWINO_ERR_UNSUPPORTED;
     if (residual && !aligned(residual, 4)) return SDWINO_ERR_MISALIGNED;
     return conv_impl(x, wT, bias, y, N, C, H, W, K, tile, workspace, workspace_bytes, static_cast<cudaStream_t>(stream),
-                     Epilogue{residual, activation}, true);
+                     Epilogue{residual, activation, nullptr}, true);
 }
 
 int sdwino_conv3x3(const void* x, const void* wT, const void* bias, void* y, int N, int C, int H, int W, int K,
@@ -1437,7 +1464,7 @@ int host_async_impl(const void* x_host, const void* wT, const void* bias_host, v
     // kernels on the caller's stream
     if (cudaStreamWaitEvent(st, me.uploaded, 0) != cudaSuccess) return err_cuda(__LINE__);
     const int rc = conv_impl(xd, wT, bias_host ? bd : nullptr, yd, N, C, H, W, K, tile, ws, workspace_bytes - staging, st,
-                             Epilogue{nullptr, 0}, io32);
+                             Epilogue{nullptr, 0, nullptr}, io32);
     if (rc != SDWINO_OK) return rc;
     if (cudaEventRecord(me.computed, st) != cudaSuccess) return err_cuda(__LINE__);
     // download on the second copy stream

@@ -91,6 +91,38 @@ __device__ __forceinline__ float load_bias(const float* bias, int k) {
 __device__ __forceinline__ float to_f32(__half v) { return __half2float(v); }
 __device__ __forceinline__ float to_f32(float v) { return v; }
 
+// Range-safe fp32 calls: x is multiplied by 2^-e on its way into V and the result by 2^e on its way out of M, with e
+// chosen from max|x| so that the scaled activations peak near 64: V and M are fp16 and would overflow (or lose their
+// small values) otherwise.  Powers of two: the scaling itself rounds nothing.
+__device__ __forceinline__ int range_exponent(const float* amax) {
+    if (amax == nullptr) return 0;
+    const float a = *amax;
+    if (!(a > 0.f) || a > 3.0e38f) return 0;
+    return ilogbf(a) - 6;
+}
+// max|x| over a tensor, as the bits of a non-negative float (which order like unsigned integers); *out starts at 0.
+__global__ void __launch_bounds__(256)
+absmax_kernel(const float* __restrict__ x, long long n, unsigned int* __restrict__ out) {
+    pdl_wait();
+    pdl_launch_dependents();
+    float m = 0.f;
+    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+    long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if ((reinterpret_cast<uintptr_t>(x) & 15) == 0) {
+        const long long n4 = n >> 2;
+        for (long long j = i; j < n4; j += stride) {
+            const float4 v = __ldg(reinterpret_cast<const float4*>(x) + j);
+            m = fmaxf(fmaxf(m, fmaxf(fabsf(v.x), fabsf(v.y))), fmaxf(fabsf(v.z), fabsf(v.w)));
+        }
+        for (long long j = (n4 << 2) + i; j < n; j += stride) m = fmaxf(m, fabsf(__ldg(x + j)));
+    } else {
+        for (long long j = i; j < n; j += stride) m = fmaxf(m, fabsf(__ldg(x + j)));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if ((threadIdx.x & 31) == 0 && m > 0.f) atomicMax(out, __float_as_uint(m));
+}
+
 // out[i] = sum_j coef[i][j] * in[j] with compile-time coefficients: zero terms vanish and
 // unit terms become adds once the loops are unrolled.
 template <int R, int Cn, typename MatT>
@@ -246,7 +278,7 @@ __device__ __forceinline__ void decode_tile(const TileGeom& geo, long long p, lo
 template <int M, typename XT = __half>
 __global__ void __launch_bounds__(128)
 input_transform_kernel(const XT* __restrict__ x, __half* __restrict__ V, TileGeom geo, int C, long long p_begin,
-                       int p_count, long long Pstride) {
+                       int p_count, long long Pstride, const float* __restrict__ amax) {
     using Wm = Wino<M>;
     constexpr int A = Wm::A;
     // Wait first, release the GEMM second: once the GEMM runs, everything before this kernel has completed,
@@ -258,6 +290,8 @@ input_transform_kernel(const XT* __restrict__ x, __half* __restrict__ V, TileGeo
     if (pl >= p_count || c >= C) return;
     const long long p = p_begin + pl;
     float d[A][A];
+    [[maybe_unused]] float xs = 1.f;
+    if constexpr (sizeof(XT) == 4) xs = scalbnf(1.f, -range_exponent(amax));
     if (p < geo.P) {
         int tw, th;
         long long n;
@@ -273,6 +307,7 @@ input_transform_kernel(const XT* __restrict__ x, __half* __restrict__ V, TileGeo
                 const int j = j0 + s;
                 d[r][s] = (rin && j >= 0 && j < geo.W) ? to_f32(__ldg(img + static_cast<long long>(i) * geo.W + j))
                                                         : 0.f;
+                if constexpr (sizeof(XT) == 4) d[r][s] *= xs;
             }
         }
     } else {
@@ -310,6 +345,7 @@ input_transform_kernel(const XT* __restrict__ x, __half* __restrict__ V, TileGeo
 struct Epilogue {
     const void* residual;   // element type of y
     int act;
+    const float* amax;      // fp32 interface, range-safe calls: device word holding max|x| (null: no scaling)
 };
 __device__ __forceinline__ float epilogue_act(float v, int act) {
     return act == 1 ? __fdividef(v, 1.f + __expf(-v)) : v;   // fast division: 2 ulp, far below the fp16 rounding that follows
@@ -356,6 +392,8 @@ output_transform_kernel(const __half* __restrict__ Mws, const YT* __restrict__ b
     long long n;
     decode_tile(geo, p, n, th, tw);
     const float b = load_bias(bias, k);
+    [[maybe_unused]] float ys = 1.f;
+    if constexpr (sizeof(YT) == 4) ys = scalbnf(1.f, range_exponent(ep.amax));
     YT* img = y + (n * K + k) * static_cast<long long>(geo.H) * geo.W;
     const int i0 = M * th, j0 = M * tw;
     const bool vec_ok = ((geo.W & 1) == 0) && ((reinterpret_cast<uintptr_t>(y) & 3) == 0);
@@ -372,7 +410,7 @@ output_transform_kernel(const __half* __restrict__ Mws, const YT* __restrict__ b
 #pragma unroll
             for (int j = 0; j < M; ++j)
                 if (j0 + j < geo.W) {
-                    float v = o[j] + b;
+                    float v = fmaf(o[j], ys, b);
                     if (resf) v += resf[j];
                     rowf[j] = epilogue_act(v, ep.act);
                 }
@@ -461,7 +499,7 @@ __device__ __forceinline__ void at4_packed(const float2 (&m)[6], float2 (&o)[4])
 template <int M, int TPT, typename XT = __half>
 __device__ __forceinline__ void input_unit_vec(const XT* __restrict__ x, __half* __restrict__ V, const TileGeom& geo,
                                                int C, long long p_begin, const FastDiv& gdiv, long long Pstride,
-                                               uint32_t idx) {
+                                               uint32_t idx, const float* __restrict__ amax = nullptr) {
     using Wm = Wino<M>;
     constexpr int A = Wm::A;
     static_assert(M * TPT == 8, "one 16-byte row segment per thread");
@@ -480,6 +518,8 @@ __device__ __forceinline__ void input_unit_vec(const XT* __restrict__ x, __half*
     // what lets it fetch its filters (written at the latest by the kernel before this one) early.
     pdl_wait();
     pdl_launch_dependents();
+    [[maybe_unused]] float xs = 1.f;
+    if constexpr (sizeof(XT) == 4) xs = scalbnf(1.f, -range_exponent(amax));
     if (p < geo.P) {
         const XT* img = x + (n * C + c) * static_cast<long long>(geo.H) * geo.W;
         const int i0 = M * th - 1, j0 = M * tw;
@@ -492,8 +532,8 @@ __device__ __forceinline__ void input_unit_vec(const XT* __restrict__ x, __half*
                 if constexpr (sizeof(XT) == 4) {   // fp32 input: the eight pixels are two 16-byte loads
                     const float4 a = __ldg(reinterpret_cast<const float4*>(rp));
                     const float4 b = __ldg(reinterpret_cast<const float4*>(rp) + 1);
-                    row[1] = a.x; row[2] = a.y; row[3] = a.z; row[4] = a.w;
-                    row[5] = b.x; row[6] = b.y; row[7] = b.z; row[8] = b.w;
+                    row[1] = a.x * xs; row[2] = a.y * xs; row[3] = a.z * xs; row[4] = a.w * xs;
+                    row[5] = b.x * xs; row[6] = b.y * xs; row[7] = b.z * xs; row[8] = b.w * xs;
                 } else {
                     const uint4 v = __ldg(reinterpret_cast<const uint4*>(rp));
                     unpack2(v.x, row[1], row[2]);
@@ -503,6 +543,7 @@ __device__ __forceinline__ void input_unit_vec(const XT* __restrict__ x, __half*
                 }
                 row[0] = j0 > 0 ? to_f32(__ldg(rp - 1)) : 0.f;
                 row[9] = j0 + 8 < geo.W ? to_f32(__ldg(rp + 8)) : 0.f;
+                if constexpr (sizeof(XT) == 4) { row[0] *= xs; row[9] *= xs; }
             } else {
 #pragma unroll
                 for (int s = 0; s < 10; ++s) row[s] = 0.f;
@@ -558,8 +599,8 @@ __device__ __forceinline__ void input_unit_vec(const XT* __restrict__ x, __half*
 template <int M, int TPT, typename XT = __half>
 __global__ void __launch_bounds__(128)
 input_transform_vec_kernel(const XT* __restrict__ x, __half* __restrict__ V, TileGeom geo, int C,
-                           long long p_begin, FastDiv gdiv, long long Pstride) {
-    input_unit_vec<M, TPT, XT>(x, V, geo, C, p_begin, gdiv, Pstride, blockIdx.x * blockDim.x + threadIdx.x);   // < 2^31
+                           long long p_begin, FastDiv gdiv, long long Pstride, const float* __restrict__ amax) {
+    input_unit_vec<M, TPT, XT>(x, V, geo, C, p_begin, gdiv, Pstride, blockIdx.x * blockDim.x + threadIdx.x, amax);   // < 2^31
 }
 
 // F(4x4,3x3) activation transform, vector path: a thread owns 2 tiles (8 pixels of a tile row) and CH consecutive
@@ -573,7 +614,7 @@ input_transform_vec_kernel(const XT* __restrict__ x, __half* __restrict__ V, Til
 template <int CH, typename XT = __half, bool PDL = true, bool EARLY = false>
 __device__ __forceinline__ void input_unit_f4(const XT* __restrict__ x, __half* __restrict__ V, const TileGeom& geo,
                                               int C, long long p_begin, const FastDiv& gdiv, long long Pstride,
-                                              uint32_t idx) {
+                                              uint32_t idx, const float* __restrict__ amax = nullptr) {
     constexpr int A = 6;
     const int cg = static_cast<int>(fast_div(idx, gdiv));          // gdiv.d = groups of 2 tiles in this pass
     const int c0 = cg * CH;
@@ -607,6 +648,8 @@ __device__ __forceinline__ void input_unit_f4(const XT* __restrict__ x, __half* 
         pdl_wait();
         pdl_launch_dependents();
     }
+    [[maybe_unused]] float xs = 1.f;
+    if constexpr (sizeof(XT) == 4) xs = scalbnf(1.f, -range_exponent(amax));
     for (int cc = 0; cc < cend; ++cc) {
         float2 e2[A][A];   // e2[r][nu]: rows transformed along the columns, (tile 0, tile 1)
         [[maybe_unused]] uint4 raw_v[A];
@@ -638,12 +681,12 @@ __device__ __forceinline__ void input_unit_f4(const XT* __restrict__ x, __half* 
                     if (left_ok) L = to_f32(__ldg(rp - 1));
                     if (right_ok) R = to_f32(__ldg(rp + 8));
                 }
-                d[0] = make_float2(L, a.w);
-                d[1] = make_float2(a.x, b.x);
-                d[2] = make_float2(a.y, b.y);
-                d[3] = make_float2(a.z, b.z);
-                d[4] = make_float2(a.w, b.w);
-                d[5] = make_float2(b.x, R);
+                d[0] = make_float2(L * xs, a.w * xs);
+                d[1] = make_float2(a.x * xs, b.x * xs);
+                d[2] = make_float2(a.y * xs, b.y * xs);
+                d[3] = make_float2(a.z * xs, b.z * xs);
+                d[4] = make_float2(a.w * xs, b.w * xs);
+                d[5] = make_float2(b.x * xs, R * xs);
             } else {
             uint4 v = make_uint4(0u, 0u, 0u, 0u);
             uint32_t lw = 0u, rw = 0u;   // aligned words before / after the segment
@@ -686,8 +729,8 @@ __device__ __forceinline__ void input_unit_f4(const XT* __restrict__ x, __half* 
 template <int CH, typename XT = __half>
 __global__ void __launch_bounds__(128, 5)
 input_transform_f4_kernel(const XT* __restrict__ x, __half* __restrict__ V, TileGeom geo, int C, long long p_begin,
-                          FastDiv gdiv, long long Pstride) {
-    input_unit_f4<CH, XT>(x, V, geo, C, p_begin, gdiv, Pstride, blockIdx.x * blockDim.x + threadIdx.x);   // < 2^31
+                          FastDiv gdiv, long long Pstride, const float* __restrict__ amax) {
+    input_unit_f4<CH, XT>(x, V, geo, C, p_begin, gdiv, Pstride, blockIdx.x * blockDim.x + threadIdx.x, amax);   // < 2^31
 }
 
 // Eight output pixels of one row (bias already added): residual (its eight values loaded by the caller, ahead of
@@ -785,6 +828,8 @@ __device__ __forceinline__ void output_unit_vec(const __half* __restrict__ Mws, 
         long long n;
         decode_tile(geo, p, n, th, tw);
         const float b = load_bias(bias, k);
+        [[maybe_unused]] float ys = 1.f;
+        if constexpr (sizeof(YT) == 4) ys = scalbnf(1.f, range_exponent(ep.amax));
         YT* img = y + (n * K + k) * static_cast<long long>(geo.H) * geo.W;
         const int i0 = M * th, j0 = M * tw;
         uint4 res[M];
@@ -802,6 +847,10 @@ __device__ __forceinline__ void output_unit_vec(const __half* __restrict__ Mws, 
             float2 o[M];
             at4_packed(tt[i], o);
             if (i0 + i >= geo.H) continue;
+            if constexpr (sizeof(YT) == 4) {
+#pragma unroll
+                for (int j = 0; j < M; ++j) { o[j].x *= ys; o[j].y *= ys; }
+            }
             float v[8] = {o[0].x + b, o[1].x + b, o[2].x + b, o[3].x + b, o[0].y + b, o[1].y + b, o[2].y + b, o[3].y + b};
             YT* rowp = img + static_cast<long long>(i0 + i) * geo.W + j0;
             store_row8<EP>(rowp, v, res[i], ep, y);
@@ -826,6 +875,8 @@ __device__ __forceinline__ void output_unit_vec(const __half* __restrict__ Mws, 
     long long n;
     decode_tile(geo, p, n, th, tw);
     const float b = load_bias(bias, k);
+    [[maybe_unused]] float ys = 1.f;
+    if constexpr (sizeof(YT) == 4) ys = scalbnf(1.f, range_exponent(ep.amax));
     YT* img = y + (n * K + k) * static_cast<long long>(geo.H) * geo.W;
     const int i0 = M * th, j0 = M * tw;
     uint4 res[M];
@@ -856,7 +907,7 @@ __device__ __forceinline__ void output_unit_vec(const __half* __restrict__ Mws, 
             float o[M];
             mat_apply<M, A>(typename Wm::At{}, tt[i], o);
 #pragma unroll
-            for (int j = 0; j < M; ++j) out[i][M * t + j] = o[j] + b;
+            for (int j = 0; j < M; ++j) out[i][M * t + j] = sizeof(YT) == 4 ? fmaf(o[j], ys, b) : o[j] + b;
         }
     }
 #pragma unroll

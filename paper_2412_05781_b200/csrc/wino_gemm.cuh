@@ -717,7 +717,7 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
         const unsigned int n_it = static_cast<unsigned int>(pp.it_items), n_ot = static_cast<unsigned int>(pp.ot_items);
         const unsigned int head = D * n_it, per = n_it + n_ot, body = (NB - D) * per, total = NB * per;
         const long long ring_p = static_cast<long long>(pp.ring) * GEMM_BLOCK_P;
-        const Epilogue no_ep{nullptr, 0};
+        const Epilogue no_ep{nullptr, 0, nullptr};
         unsigned int iter = 0;
         int pend_kind = -1, pend_pb = 0;      // thread 0: the item just finished, announced after the team barrier
         for (;;) {

@@ -294,3 +294,69 @@ def test_fp32_interface_fused_residual_and_activation(B, shape, tile, act):
     with pytest.raises(B.SdwinoError) as e:
         B.sdwino_conv3x3_f32_ex(xd, wT, bd, None, K, tile, 7, ws)
     assert e.value.status == B.ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("tile", [2, 4])
+@pytest.mark.parametrize("scale", [1.0e4, 3.0e7, 2.0e-6])
+@pytest.mark.parametrize("shape", [(64, 96, 24, 32, 2), (33, 40, 13, 17, 1), (4, 24, 16, 16, 1), (160, 8, 40, 40, 1)])
+def test_fp32_range_safe_entry_on_magnitudes_fp16_cannot_hold(B, shape, scale, tile):
+    # activations far outside (or far below) the fp16 range: V would overflow to infinity (or flush to zero) in the
+    # plain fp32 call; the range-safe call scales by a power of two around the fp16 operands
+    C, K, H, W, N = shape
+    layer = ConvLayer(C=C, K=K, H=H, W=W, N=N)
+    x, w, b = workloads.make_inputs(layer, seed=7 + C, dtype=torch.float32)
+    x = x * scale
+    b = b * scale
+    ref = oracle.direct_conv3x3(x.numpy(), w.numpy(), b.numpy())
+    wT = B.sdwino_filter_transform_f32(w.cuda(), tile)
+    ws = B.alloc_workspace(B.sdwino_workspace_bytes(N, C, H, W, K, tile))
+    y = B.sdwino_conv3x3_f32(x.cuda(), wT, b.cuda(), K, tile, workspace=ws, scaled=True)
+    assert B.sdwino_last_device_status() == B.OK
+    assert torch.isfinite(y).all()
+    assert _rel_err(y.cpu(), ref) <= (TOL_F2_REGRESSION if tile == 2 else TOL)
+    if scale >= 1.0e4 and tile == 4:
+        # where the plain call breaks down: its V exceeds the fp16 range
+        y_plain = B.sdwino_conv3x3_f32(x.cuda(), wT, b.cuda(), K, tile, workspace=ws)
+        assert B.sdwino_last_device_status() == B.OK
+        assert (not torch.isfinite(y_plain).all()) or _rel_err(y_plain.cpu(), ref) > TOL
+
+
+@pytest.mark.parametrize("tile", [2, 4])
+def test_fp32_range_safe_entry_changes_nothing_on_moderate_inputs_and_handles_zero(B, tile):
+    layer = ConvLayer(C=48, K=64, H=32, W=40, N=2)
+    x, w, b = workloads.make_inputs(layer, seed=5, dtype=torch.float32)
+    x = x * 16.0      # max|x| lands in [64, 128): the exponent is zero and the call reproduces the plain one
+    assert 64.0 <= float(x.abs().max()) < 128.0
+    wT = B.sdwino_filter_transform_f32(w.cuda(), tile)
+    ws = B.alloc_workspace(B.sdwino_workspace_bytes(layer.N, layer.C, layer.H, layer.W, layer.K, tile))
+    y_plain = B.sdwino_conv3x3_f32(x.cuda(), wT, b.cuda(), layer.K, tile, workspace=ws).clone()
+    y_safe = B.sdwino_conv3x3_f32(x.cuda(), wT, b.cuda(), layer.K, tile, workspace=ws, scaled=True)
+    assert torch.equal(y_plain, y_safe)
+    # an all-zero input has no maximum to scale by: the result is the bias
+    y0 = B.sdwino_conv3x3_f32(torch.zeros_like(x).cuda(), wT, b.cuda(), layer.K, tile, workspace=ws, scaled=True)
+    assert B.sdwino_last_device_status() == B.OK
+    assert torch.equal(y0.cpu(), b.view(1, -1, 1, 1).expand_as(y0).contiguous())
+
+
+@pytest.mark.parametrize("tile", [2, 4])
+def test_fp32_host_entry_matches_the_device_entry(B, tile):
+    layers = [ConvLayer(C=64, K=96, H=32, W=32, N=2), ConvLayer(C=20, K=24, H=17, W=23, N=1)]
+    for seed, layer in enumerate(layers):
+        x, w, b = workloads.make_inputs(layer, seed=seed, dtype=torch.float32, pin=True)
+        dims = (layer.N, layer.C, layer.H, layer.W, layer.K, tile)
+        wT = B.sdwino_filter_transform_f32(w.cuda(), tile)
+        ws = B.alloc_workspace(B.sdwino_workspace_bytes(*dims))
+        y_dev = B.sdwino_conv3x3_f32(x.cuda(), wT, b.cuda(), layer.K, tile, workspace=ws).cpu()
+        hws = B.alloc_workspace(B.sdwino_host_staging_bytes_f32(*dims) + B.sdwino_workspace_bytes(*dims))
+        assert B.sdwino_host_staging_bytes_f32(*dims) >= 2 * B.sdwino_host_staging_bytes(*dims) - 8192
+        y_host = torch.full((layer.N, layer.K, layer.H, layer.W), float("nan"), dtype=torch.float32).pin_memory()
+        B.sdwino_conv3x3_host_f32(x, wT, b, y_host, tile, hws)                       # synchronous
+        assert torch.equal(y_host, y_dev)
+        y_host.fill_(float("nan"))
+        for _ in range(3):                                                           # asynchronous, back to back
+            B.sdwino_conv3x3_host_f32(x, wT, b, y_host, tile, hws, wait=False)
+        B.sdwino_host_join()
+        torch.cuda.synchronize()
+        assert torch.equal(y_host, y_dev)
+        ref = oracle.direct_conv3x3(x.numpy(), w.numpy(), b.numpy())
+        assert _rel_err(y_host, ref) <= TOL
