@@ -57,6 +57,7 @@ def _load():
         lib.oracle_filter_transform.argtypes = [dp, dp, dp, i, i, i]
         lib.oracle_input_tile_transform.argtypes = [dp, dp, dp, i, i, i, i, i, i, i, i]
         lib.oracle_winograd.argtypes = [dp, dp, dp, dp, i, i, i, i, i, i, dp, dp, dp]
+        lib.oracle_winograd_with_filter.argtypes = [dp, dp, dp, dp, i, i, i, i, i, i, dp, dp]
         lib.oracle_threads.restype = i
         _lib = lib
     return _lib
@@ -286,4 +287,57 @@ def winograd_conv3x3(x, w, bias=None, m: int = 2, points=None):
                                  _ptr(G), _ptr(Bt), _ptr(At))
     if rc != 0:
         raise RuntimeError(f"oracle_winograd failed ({rc})")
+    return y
+
+
+# --------------------------------------------------------------------------
+# 8-bit transformed filters (the quantised operators of Section "Evaluation", "Operator Support")
+# --------------------------------------------------------------------------
+# Reading (the paper names no format): the transformed filter U is first rounded to fp16, as the fp16 path stores it;
+# then every row U[pos][k][:] (one transform position, one output channel, all input channels) gets the power-of-two
+# scale 2^e with e = floor(log2(max|U|)) - 7, so that the scaled row peaks in [128, 256), and every element is
+# rounded to the nearest FP8 E4M3 value (4 exponent bits, bias 7, 3 significand bits, subnormals below 2^-6, largest
+# finite value 448; ties to even).  The contraction uses the E4M3 values; the scale multiplies the sum over channels.
+
+E4M3_MAX = 448.0
+
+
+def round_e4m3(v):
+    """Nearest FP8 E4M3 value (ties to even, saturating at +-448) of every element of ``v``, as fp64."""
+    v = np.asarray(v, dtype=np.float64)
+    a = np.abs(v)
+    with np.errstate(divide="ignore"):
+        e = np.floor(np.log2(np.where(a > 0, a, 1.0)))
+    e = np.maximum(e, -6.0)                      # below 2^-6 the spacing stays that of the smallest normal binade
+    q = np.exp2(e - 3.0)                         # spacing: 3 significand bits
+    r = np.minimum(np.round(a / q) * q, E4M3_MAX)   # numpy rounds halves to even
+    return np.copysign(r, v)
+
+
+def quantize_filter_e4m3(U):
+    """U: transformed filter [K, C, a, a] (fp64).  Returns (Uq, e): Uq[K, C, a, a] holds the E4M3 values of the
+    scaled rows (NOT multiplied back), e[K, a, a] the exponents, so that the filter used is Uq * 2^e."""
+    U16 = np.asarray(U, dtype=np.float64).astype(np.float16).astype(np.float64)   # the fp16 path's filter
+    K, C, a, _ = U16.shape
+    amax = np.abs(U16).max(axis=1)               # [K, a, a]: over the input channels
+    e = np.zeros_like(amax)
+    nz = amax > 0
+    e[nz] = np.floor(np.log2(amax[nz])) - 7.0
+    Uq = round_e4m3(U16 / np.exp2(e)[:, None, :, :])
+    return Uq, e
+
+
+def winograd_conv3x3_q8(x, w, bias=None, m: int = 2, points=None):
+    """The Winograd convolution with the 8-bit transformed filter defined above; everything else fp64."""
+    x, w = _f64(x), _f64(w)
+    N, C, H, W = x.shape
+    K = w.shape[0]
+    b = _f64(bias) if bias is not None else None
+    Bt, G, At = _mats_f64(m, points)
+    Uq, e = quantize_filter_e4m3(filter_transform(w, m, points))
+    U = np.ascontiguousarray(Uq * np.exp2(e)[:, None, :, :])
+    y = np.full((N, K, H, W), np.nan, dtype=np.float64)
+    rc = _load().oracle_winograd_with_filter(_ptr(x), _ptr(U), _ptr(b), _ptr(y), N, C, H, W, K, m, _ptr(Bt), _ptr(At))
+    if rc != 0:
+        raise RuntimeError(f"oracle_winograd_with_filter failed ({rc})")
     return y

@@ -138,6 +138,10 @@ int oracle_input_tile_transform(const double *x, const double *Bt, double *V,
  *   (iii) Y[k]    = A^T M[k] A  (m x m) ; y = Y + b[k] where inside the image.
  * Tiles: TH = ceil(H/m), TW = ceil(W/m); outputs past the image edge are
  * computed and dropped.  At is m x a row-major. */
+static int winograd_steps_ii_iii(const double *x, const double *U, const double *bias, double *y,
+                                 int N, int C, int H, int W, int K, int m,
+                                 const double *Bt, const double *At);
+
 int oracle_winograd(const double *x, const double *w, const double *bias, double *y,
                     int N, int C, int H, int W, int K, int m,
                     const double *G, const double *Bt, const double *At)
@@ -145,10 +149,31 @@ int oracle_winograd(const double *x, const double *w, const double *bias, double
     if (!x || !w || !y || !G || !Bt || !At) return 1;
     if (N <= 0 || C <= 0 || H <= 0 || W <= 0 || K <= 0 || m <= 0) return 1;
     int a = m + 2, aa = a * a;
-    int TH = (H + m - 1) / m, TW = (W + m - 1) / m;
     double *U = (double *)malloc(sizeof(double) * (size_t)K * C * aa);
     if (!U) return 2;
     oracle_filter_transform(w, G, U, K, C, a);
+    int rc = winograd_steps_ii_iii(x, U, bias, y, N, C, H, W, K, m, Bt, At);
+    free(U);
+    return rc;
+}
+
+/* The same evaluation for a transformed filter U[K][C][a][a] handed in by the caller (a filter that was
+ * rounded or quantised after step (i)): the activation half of (i), then (ii) and (iii). */
+int oracle_winograd_with_filter(const double *x, const double *U, const double *bias, double *y,
+                                int N, int C, int H, int W, int K, int m,
+                                const double *Bt, const double *At)
+{
+    if (!x || !U || !y || !Bt || !At) return 1;
+    if (N <= 0 || C <= 0 || H <= 0 || W <= 0 || K <= 0 || m <= 0) return 1;
+    return winograd_steps_ii_iii(x, U, bias, y, N, C, H, W, K, m, Bt, At);
+}
+
+static int winograd_steps_ii_iii(const double *x, const double *U, const double *bias, double *y,
+                                 int N, int C, int H, int W, int K, int m,
+                                 const double *Bt, const double *At)
+{
+    int a = m + 2, aa = a * a;
+    int TH = (H + m - 1) / m, TW = (W + m - 1) / m;
     int err = 0;
     long long tiles = (long long)N * TH * TW;
 #pragma omp parallel for schedule(dynamic, 1)
@@ -185,6 +210,5 @@ int oracle_winograd(const double *x, const double *w, const double *bias, double
         free(V);
         free(Mk);
     }
-    free(U);
     return err;
 }
