@@ -293,38 +293,22 @@ def winograd_conv3x3(x, w, bias=None, m: int = 2, points=None):
 # --------------------------------------------------------------------------
 # 8-bit transformed filters (the quantised operators of Section "Evaluation", "Operator Support")
 # --------------------------------------------------------------------------
-# Reading (the paper names no format): the transformed filter U is first rounded to fp16, as the fp16 path stores it;
-# then every row U[pos][k][:] (one transform position, one output channel, all input channels) gets the power-of-two
-# scale 2^e with e = floor(log2(max|U|)) - 7, so that the scaled row peaks in [128, 256), and every element is
-# rounded to the nearest FP8 E4M3 value (4 exponent bits, bias 7, 3 significand bits, subnormals below 2^-6, largest
-# finite value 448; ties to even).  The contraction uses the E4M3 values; the scale multiplies the sum over channels.
+# Reading (the paper names no format; its host framework quantises weights to 8-bit integers with a scale per
+# group): the transformed filter U is first rounded to fp16, as the fp16 path stores it; then every row
+# U[pos][k][:] (one transform position, one output channel, all input channels) gets the scale s = max|U| / 127
+# and every element becomes the integer q = round(U / s) in [-127, 127] (ties to even).  The contraction runs on
+# the integers; s multiplies the sum over the channels.  The scale and the quotient are formed in fp32, the
+# precision in which the library takes this decision (both are correctly rounded IEEE operations, so that numpy's
+# float32 gives the same integers).
 
-E4M3_MAX = 448.0
-
-
-def round_e4m3(v):
-    """Nearest FP8 E4M3 value (ties to even, saturating at +-448) of every element of ``v``, as fp64."""
-    v = np.asarray(v, dtype=np.float64)
-    a = np.abs(v)
-    with np.errstate(divide="ignore"):
-        e = np.floor(np.log2(np.where(a > 0, a, 1.0)))
-    e = np.maximum(e, -6.0)                      # below 2^-6 the spacing stays that of the smallest normal binade
-    q = np.exp2(e - 3.0)                         # spacing: 3 significand bits
-    r = np.minimum(np.round(a / q) * q, E4M3_MAX)   # numpy rounds halves to even
-    return np.copysign(r, v)
-
-
-def quantize_filter_e4m3(U):
-    """U: transformed filter [K, C, a, a] (fp64).  Returns (Uq, e): Uq[K, C, a, a] holds the E4M3 values of the
-    scaled rows (NOT multiplied back), e[K, a, a] the exponents, so that the filter used is Uq * 2^e."""
-    U16 = np.asarray(U, dtype=np.float64).astype(np.float16).astype(np.float64)   # the fp16 path's filter
-    K, C, a, _ = U16.shape
-    amax = np.abs(U16).max(axis=1)               # [K, a, a]: over the input channels
-    e = np.zeros_like(amax)
-    nz = amax > 0
-    e[nz] = np.floor(np.log2(amax[nz])) - 7.0
-    Uq = round_e4m3(U16 / np.exp2(e)[:, None, :, :])
-    return Uq, e
+def quantize_filter_int8(U):
+    """U: transformed filter [K, C, a, a] (fp64).  Returns (q, s): q[K, C, a, a] integers in [-127, 127] (as fp64)
+    and the scales s[K, a, a] (fp32 values as fp64), so that the filter used is q * s."""
+    U16 = np.asarray(U, dtype=np.float64).astype(np.float16).astype(np.float32)   # the fp16 path's filter
+    amax = np.abs(U16).max(axis=1)                                                # [K, a, a]: over the input channels
+    s = np.where(amax > 0, amax / np.float32(127.0), np.float32(1.0)).astype(np.float32)
+    q = np.clip(np.rint(U16 / s[:, None, :, :]), -127.0, 127.0)                   # fp32 quotient, ties to even
+    return q.astype(np.float64), s.astype(np.float64)
 
 
 def winograd_conv3x3_q8(x, w, bias=None, m: int = 2, points=None):
@@ -334,8 +318,8 @@ def winograd_conv3x3_q8(x, w, bias=None, m: int = 2, points=None):
     K = w.shape[0]
     b = _f64(bias) if bias is not None else None
     Bt, G, At = _mats_f64(m, points)
-    Uq, e = quantize_filter_e4m3(filter_transform(w, m, points))
-    U = np.ascontiguousarray(Uq * np.exp2(e)[:, None, :, :])
+    q, s = quantize_filter_int8(filter_transform(w, m, points))
+    U = np.ascontiguousarray(q * s[:, None, :, :])
     y = np.full((N, K, H, W), np.nan, dtype=np.float64)
     rc = _load().oracle_winograd_with_filter(_ptr(x), _ptr(U), _ptr(b), _ptr(y), N, C, H, W, K, m, _ptr(Bt), _ptr(At))
     if rc != 0:
