@@ -320,6 +320,8 @@ def bench_workload(ctx, args, workload: str, headline: bool):
     ft_bytes = sum(L.K * L.C * 9 * io_bytes + B.sdwino_filter_bytes(L.K, L.C, t) for L, t in zip(layers, tiles))
     B.sdwino_profile_enable(0)
     del w_dev
+    q8 = [args.weights == "q8" and not io32 and min(L.C, L.K) > 8 for L in layers]
+    wTs = [B.sdwino_filter_quantize(wT, L.K, L.C, t) if q else wT for wT, L, t, q in zip(wTs, layers, tiles, q8)]
     for (x, w, b, y_h), wT in zip(host, wTs):
         devt.append((x.to(dev).to(io_t), wT, b.to(dev).to(io_t), torch.empty(y_h.shape, dtype=io_t, device=dev)))
     if args.epilogue != "none":
@@ -329,7 +331,9 @@ def bench_workload(ctx, args, workload: str, headline: bool):
 
     def run_layer(li, strm):
         L, t, (xd, wT, bd, yd) = layers[li], tiles[li], devt[li]
-        if io32 and (args.epilogue == "none" or min(L.C, L.K) <= 8):
+        if q8[li]:
+            B.sdwino_conv3x3_q8(xd, wT, bd, L.K, t, ws, y=yd, stream=strm)
+        elif io32 and (args.epilogue == "none" or min(L.C, L.K) <= 8):
             B.sdwino_conv3x3_f32(xd, wT, bd, L.K, t, ws, y=yd, stream=strm)
         elif io32:
             B.sdwino_conv3x3_f32_ex(xd, wT, bd, res_dev[li], L.K, t, act, ws, y=yd, stream=strm)
@@ -373,7 +377,9 @@ def bench_workload(ctx, args, workload: str, headline: bool):
 
     # ---- timed region: resident inputs, exactly `steps` steps, an event after every step ----
     flops_step = sum(L.direct_flops for L in layers)
-    step_bytes = sum(io_bytes * L.N * (L.C + L.K) * L.H * L.W + B.sdwino_filter_bytes(L.K, L.C, t) for L, t in zip(layers, tiles))
+    def filt_bytes(L, t, q):
+        return B.sdwino_filter_q8_bytes(L.K, L.C, t) if q else B.sdwino_filter_bytes(L.K, L.C, t)
+    step_bytes = sum(io_bytes * L.N * (L.C + L.K) * L.H * L.W + filt_bytes(L, t, q) for L, t, q in zip(layers, tiles, q8))
     # A step that touches less than twice the L2 would find its operands cached by the previous step: then
     # the L2 is flushed (a 256 MB buffer is written) before every step and only the steps are timed.
     flush_l2 = step_bytes < 2 * L2_BYTES
@@ -508,14 +514,14 @@ def bench_workload(ctx, args, workload: str, headline: bool):
     layer_rows = []
     gemm_flops = gemm_ms = gemm_u_bytes = 0.0
     in_ms = out_ms = in_bytes = out_bytes = fused_ms = 0.0
-    for L, t, pl, lms in zip(layers, tiles, per_layer, layer_ms):
+    for L, t, pl, lms, q in zip(layers, tiles, per_layer, layer_ms, q8):
         a2 = (t + 2) ** 2
         P = L.tiles(t)
         wino_flops = 2.0 * a2 * L.K * L.C * P
-        u_bytes = B.sdwino_filter_bytes(L.K, L.C, t)
+        u_bytes = filt_bytes(L, t, q)
         xb, yb = io_bytes * L.N * L.C * L.H * L.W, io_bytes * L.N * L.K * L.H * L.W
         t_tensor = wino_flops / (tpeak * 1e12) * 1e6
-        t_hbm = (xb + 2.0 * a2 * L.K * L.C + yb + 2 * L.K) / (hpeak * 1e9) * 1e6
+        t_hbm = (xb + (1.0 if q else 2.0) * a2 * L.K * L.C + yb + 2 * L.K) / (hpeak * 1e9) * 1e6
         ksum = pl["input_transform"] + pl["wino_gemm"] + pl["output_transform"] + pl["fused"]
         scale = lms / ksum if ksum > 0 else 0.0     # the kernels' event-bracketed times, scaled to the layer's time
         k_in, k_gemm, k_out, k_fused = (pl[k] * scale for k in ("input_transform", "wino_gemm", "output_transform", "fused"))
@@ -582,7 +588,7 @@ def bench_workload(ctx, args, workload: str, headline: bool):
 
     # ---- end to end: host buffers in, host buffers out, through the host entry of the C ABI (fp16 or fp32) ----
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and args.weights == "f16":
         host_call = B.sdwino_conv3x3_host_f32 if io32 else B.sdwino_conv3x3_host
         staging = B.sdwino_host_staging_bytes_f32 if io32 else B.sdwino_host_staging_bytes
         e2e_bytes = [staging(L.N, L.C, L.H, L.W, L.K, t) + B.sdwino_workspace_bytes(L.N, L.C, L.H, L.W, L.K, t)
@@ -740,6 +746,7 @@ def run_ours(args):
                                      if io32 else ", fp16 storage, fp32 accumulate"),
                        "parallelism": f"replicas x{ctx.world} (no exchange step)",
                        "launch": "direct" if args.no_graph else "CUDA graph of one step, replayed",
+                       "weights": args.weights,
                        "pipeline": {0: "off", 1: "where the library takes it", 2: "wherever possible"}[args.pipeline],
                        "l2": h["l2"],
                        "filter_transform": "once per weight, before the timed region (reported separately)",
@@ -779,6 +786,8 @@ def main():
                     help="element type of x, w, bias and y: f32 runs the fp32 interface (fp16 operands, fp32 accumulation)")
     ap.add_argument("--epilogue", default="none", choices=["none", "residual", "residual_silu"],
                     help="fuse y = act(conv + bias + residual) into the output transform of the timed step (sdwino_conv3x3_ex)")
+    ap.add_argument("--weights", default="f16", choices=["f16", "q8"],
+                    help="q8: 8-bit transformed filters (sdwino_conv3x3_q8) on every layer with more than 8 input and output channels")
     ap.add_argument("--pipeline", type=int, default=1, choices=[0, 1, 2],
                     help="the pipelined single-launch path of F(4x4): 0 never, 1 where the library takes it, 2 wherever possible")
     ap.add_argument("--pipe-ring", type=int, default=0, help="ring length of the pipelined path in blocks of 128 tiles (0: library's choice)")

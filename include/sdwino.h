@@ -158,6 +158,28 @@ int sdwino_conv3x3_f32_ex(const float *x, const void *wT, const float *bias, con
                           void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * 8-bit transformed filters (Section "Evaluation", "Operator Support": the quantised operators).  The filter stream
+ * bounds the layers with few tiles and many channels; storing it in 8 bits halves it.  Reading of the paper, which
+ * names no format: every row U[position][k][:] of the fp16 transformed filter becomes integers q = round(U / s) in
+ * [-127, 127] with s = max|U| / 127 over the row (both formed in fp32, ties to even); the contraction runs on the
+ * integers (exact in fp16, kind::f16 MMA, fp32 accumulation) and s multiplies the accumulator of the row.
+ *   sdwino_filter_q8_bytes      size of the 8-bit buffer (0 for invalid arguments); 1024-byte aligned like wT.
+ *   sdwino_filter_quantize      wT (made by sdwino_filter_transform[_f32] for the same K, C, tile) -> wTq; wT may
+ *                               be freed afterwards.  A wT made for other K / C / tile is reported through
+ *                               sdwino_last_device_status and nothing is written.
+ *   sdwino_conv3x3_q8           sdwino_conv3x3_ws with an 8-bit filter: fp16 x, bias, y; same workspace.  Handing it
+ *                               an fp16 wT, or an 8-bit buffer to the other entries, is caught by the header check
+ *                               (SDWINO_ERR_INVALID_ARG from sdwino_last_device_status, y untouched).
+ * Accuracy: the quantisation is part of the operator (the oracle applies the same rule); against the unquantised
+ * convolution it costs about 1 % rms with tile 2 and 3-4 % with tile 4, whose transform amplifies filter noise.
+ */
+size_t sdwino_filter_q8_bytes(int K, int C, int tile);
+int sdwino_filter_quantize(const void *wT, void *wTq, int K, int C, int tile, void *stream);
+int sdwino_conv3x3_q8(const void *x, const void *wTq, const void *bias, void *y,
+                      int N, int C, int H, int W, int K, int tile,
+                      void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * The convolution for callers that must not allocate device memory.  (The paper has no
  * counterpart; this entry point exists for the embedding of the library.)  Some callers cannot
  * call cudaMalloc or any allocator at all: code that runs inside a CUDA-graph capture or another

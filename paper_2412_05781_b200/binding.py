@@ -25,7 +25,7 @@ EXPORTS = [
     "sdwino_selftest_wait_timeout", "sdwino_conv3x3_host_async", "sdwino_host_join", "sdwino_set_input_staging", "sdwino_conv3x3_ex",
     "sdwino_filter_transform_f32", "sdwino_conv3x3_f32", "sdwino_conv3x3_f32_ex",
     "sdwino_host_staging_bytes_f32", "sdwino_conv3x3_host_f32", "sdwino_conv3x3_host_f32_async", "sdwino_set_pipeline",
-    "sdwino_conv3x3_f32_scaled",
+    "sdwino_conv3x3_f32_scaled", "sdwino_filter_q8_bytes", "sdwino_filter_quantize", "sdwino_conv3x3_q8",
 ]
 
 KERNEL_KINDS = ("filter_transform", "input_transform", "wino_gemm", "output_transform", "fused", "layer")
@@ -97,6 +97,12 @@ def _load() -> ctypes.CDLL:
     lib.sdwino_choose_tile.argtypes = [i, i, i, i, i]
     lib.sdwino_set_fused_min_tiles.restype = i
     lib.sdwino_set_fused_min_tiles.argtypes = [ctypes.c_longlong]
+    lib.sdwino_filter_q8_bytes.restype = sz
+    lib.sdwino_filter_q8_bytes.argtypes = [i, i, i]
+    lib.sdwino_filter_quantize.restype = i
+    lib.sdwino_filter_quantize.argtypes = [vp, vp, i, i, i, vp]
+    lib.sdwino_conv3x3_q8.restype = i
+    lib.sdwino_conv3x3_q8.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, vp, sz, vp]
     lib.sdwino_set_pipeline.restype = i
     lib.sdwino_set_pipeline.argtypes = [i, i, i]
     lib.sdwino_profile_enable.restype = i
@@ -402,4 +408,33 @@ def sdwino_conv3x3_host_f32(x: torch.Tensor, wT: torch.Tensor, bias: Optional[to
     rc = fn(x.data_ptr(), wT.data_ptr(), _ptr(bias), y.data_ptr(), N, C, H, W, K, tile,
             workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream_ptr(stream))
     _check(rc, "sdwino_conv3x3_host_f32" if wait else "sdwino_conv3x3_host_f32_async")
+    return y
+
+
+def sdwino_filter_q8_bytes(K: int, C: int, tile: int) -> int:
+    return int(lib.sdwino_filter_q8_bytes(K, C, tile))
+
+
+def sdwino_filter_quantize(wT: torch.Tensor, K: int, C: int, tile: int, stream=None) -> torch.Tensor:
+    """wT (fp16 transformed filter of a [K, C, 3, 3] weight) -> the 8-bit transformed filter (opaque uint8 tensor)."""
+    nbytes = int(lib.sdwino_filter_q8_bytes(K, C, tile))
+    if nbytes == 0:
+        raise SdwinoError(ERR_UNSUPPORTED if tile not in (2, 4) else ERR_INVALID_ARG, "sdwino_filter_q8_bytes")
+    wTq = alloc_workspace(nbytes, wT.device)
+    _check(lib.sdwino_filter_quantize(wT.data_ptr(), wTq.data_ptr(), K, C, tile, _stream_ptr(stream)),
+           "sdwino_filter_quantize")
+    return wTq
+
+
+def sdwino_conv3x3_q8(x: torch.Tensor, wTq: torch.Tensor, bias: Optional[torch.Tensor], K: int, tile: int,
+                      workspace: torch.Tensor, y: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """The convolution with an 8-bit transformed filter (fp16 x, bias, y)."""
+    assert x.is_cuda and x.dtype == torch.float16 and x.is_contiguous() and x.dim() == 4
+    N, C, H, W = (int(v) for v in x.shape)
+    if y is None:
+        y = torch.empty((N, K, H, W), dtype=torch.float16, device=x.device)
+    assert y.is_cuda and y.is_contiguous() and y.dtype == torch.float16 and tuple(y.shape) == (N, K, H, W)
+    rc = lib.sdwino_conv3x3_q8(x.data_ptr(), wTq.data_ptr(), _ptr(bias), y.data_ptr(), N, C, H, W, K, tile,
+                               workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    _check(rc, "sdwino_conv3x3_q8")
     return y

@@ -170,15 +170,16 @@ EncodeTiledFn get_encode_fn() {
 // (a thread that is capturing a stream has a context, and cudaFree is not allowed inside a capture), the runtime
 // is asked to bind the device's primary context to the thread and the call is repeated.
 CUresult encode_tiled(CUtensorMap* m, cuuint32_t rank, const void* base, const cuuint64_t* dims, const cuuint64_t* strides,
-                      const cuuint32_t* box, const cuuint32_t* estr, CUtensorMapSwizzle swizzle) {
+                      const cuuint32_t* box, const cuuint32_t* estr, CUtensorMapSwizzle swizzle,
+                      CUtensorMapDataType dtype = CU_TENSOR_MAP_DATA_TYPE_FLOAT16) {
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return CUDA_ERROR_NOT_INITIALIZED;
-    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, rank, const_cast<void*>(base), dims, strides, box, estr,
+    CUresult r = fn(m, dtype, rank, const_cast<void*>(base), dims, strides, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r == CUDA_ERROR_INVALID_CONTEXT) {
         cudaFree(nullptr);
-        r = fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, rank, const_cast<void*>(base), dims, strides, box, estr,
+        r = fn(m, dtype, rank, const_cast<void*>(base), dims, strides, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     }
     return r;
@@ -260,6 +261,27 @@ bool encode_filter_map(CUtensorMap* m, const void* base, uint64_t Cb, uint64_t K
     return true;
 }
 
+// The 8-bit blocked filter tensor (one byte per element, same blocking): box of `kblocks` blocks of 16 rows of 64 bytes,
+// not swizzled (the bytes are expanded to fp16 by the kernel, which places them in the swizzled operand layout itself).
+bool encode_filter_map_q8(CUtensorMap* m, const void* base, uint64_t Cb, uint64_t Kb, uint64_t npos, uint32_t kblocks) {
+    const MapKey key{base, Cb, Kb, npos, ~2ull, ~2ull, kblocks, 8, false};
+    const uint64_t h = (reinterpret_cast<uintptr_t>(base) >> 8) * 1000003u ^ Cb * 31u ^ Kb * 131u ^ (kblocks << 7) ^ 8u;
+    MapSlot& slot = g_map_cache[h % MAP_CACHE_SLOTS];
+    std::lock_guard<std::mutex> lock(g_map_mutex);
+    if (slot.used && slot.key == key) { *m = slot.map; return true; }
+    cuuint64_t dims[5] = {64, 16, Cb, Kb, npos};
+    cuuint64_t strides[4] = {64, 1024 * Kb, 1024, Kb * Cb * 1024};   // memory order [pos][Cb][Kb][16][64], bytes
+    cuuint32_t box[5] = {64, 16, 1, kblocks, 1};
+    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    if (encode_tiled(m, 5, base, dims, strides, box, estr, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_DATA_TYPE_UINT8) !=
+        CUDA_SUCCESS)
+        return false;
+    slot.key = key;
+    slot.map = *m;
+    slot.used = true;
+    return true;
+}
+
 // Per-device facts, looked up once per device (a process may drive several GPUs: everything that belongs to a
 // device -- the SM count, the address of the status word, the shared-memory limit of a kernel -- is kept per device).
 int current_device() {
@@ -304,6 +326,13 @@ bool ensure_dyn_smem(const void* kernel, int bytes) {
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return false;
     done.emplace_back(kernel, dev);
     return true;
+}
+// 8-bit filter buffer: header, the bytes, the scales (each part padded to 1 KiB)
+inline size_t q8_bytes_part(int a2, int Kb, int Cb) {
+    return (static_cast<size_t>(a2) * Kb * Cb * 1024 + WS_ALIGN - 1) / WS_ALIGN * WS_ALIGN;
+}
+inline size_t q8_scale_part(int a2, int Kb) {
+    return (static_cast<size_t>(a2) * Kb * 16 * sizeof(float) + WS_ALIGN - 1) / WS_ALIGN * WS_ALIGN;
 }
 inline const uint32_t* wt_header_of(const void* wT) { return static_cast<const uint32_t*>(wT); }
 inline const void* wt_filters_of(const void* wT) { return static_cast<const uint8_t*>(wT) + WT_HEADER_BYTES; }
@@ -751,21 +780,22 @@ GemmShape choose_gemm_shape(int K, int C, long long p_tiles128, int a2, int sms,
     return best;
 }
 
-template <int CTAS, bool RES, bool DUAL = false>
+template <int CTAS, bool RES, bool DUAL = false, bool U8 = false>
 int launch_gemm_shape(const CUtensorMap& tmU, const CUtensorMap& tmV, const CUtensorMap& tmM, const GemmParams& prm,
                       int sms, int* status, cudaStream_t st) {
     using L = GemmSmemLayout;
-    if (!ensure_dyn_smem(reinterpret_cast<const void*>(wino_gemm_kernel<CTAS, RES, DUAL>), MAX_DYN_SMEM)) return err_cuda(__LINE__);
+    if (!ensure_dyn_smem(reinterpret_cast<const void*>(wino_gemm_kernel<CTAS, RES, DUAL, false, U8>), MAX_DYN_SMEM)) return err_cuda(__LINE__);
     const long long tiles = static_cast<long long>(prm.num_k_tiles) * prm.num_p_tiles * prm.num_pos;
     const long long workers = sms / CTAS;
     const int grid = static_cast<int>(tiles < workers ? tiles : workers) * CTAS;
     ProfScope prof(KIND_GEMM, st);
     const cudaError_t e =
-        launch_pdl(wino_gemm_kernel<CTAS, RES, DUAL>, dim3(grid), dim3(GEMM_THREADS),
+        launch_pdl(wino_gemm_kernel<CTAS, RES, DUAL, false, U8>, dim3(grid), dim3(GEMM_THREADS),
                    static_cast<size_t>(L::dyn_bytes(RES ? 0 : prm.n_tile / CTAS, prm.stages, prm.epi_rows,
                                                     prm.epi_alias ? 0 : prm.epi_bufs,
                                                     RES ? prm.num_c_blocks * L::b_bytes(prm.n_tile)
-                                                        : (DUAL ? prm.stages * L::A_BYTES : 0))),
+                                                        : (DUAL ? prm.stages * L::A_BYTES
+                                                                : (U8 ? prm.raw_slots * L::raw_bytes(prm.n_tile) : 0)))),
                    st, CTAS, tmU, tmV, tmM, prm, status, PipeParams{});
     if (e != cudaSuccess && getenv("SDWINO_LOG"))
         fprintf(stderr, "sdwino: GEMM launch failed: %s (grid %d, stages %d, n_tile %d, resident %d)\n", cudaGetErrorString(e),
@@ -775,11 +805,12 @@ int launch_gemm_shape(const CUtensorMap& tmU, const CUtensorMap& tmV, const CUte
 }
 
 int launch_gemm(const CUtensorMap& tmU, const CUtensorMap& tmV, const CUtensorMap& tmM, const GemmParams& prm,
-                int ctas, cudaStream_t st) {
+                int ctas, cudaStream_t st, bool q8 = false) {
     const int sms = sm_count();
     if (sms <= 0) return err_cuda(__LINE__);
     int* status = status_word_ptr();
     if (!status) return err_cuda(__LINE__);
+    if (q8) return launch_gemm_shape<1, false, false, true>(tmU, tmV, tmM, prm, sms, status, st);
     if (ctas == 2) return launch_gemm_shape<2, false>(tmU, tmV, tmM, prm, sms, status, st);
     if (prm.resident) return launch_gemm_shape<1, true>(tmU, tmV, tmM, prm, sms, status, st);
     if (prm.dual) return launch_gemm_shape<1, false, true>(tmU, tmV, tmM, prm, sms, status, st);
@@ -895,6 +926,9 @@ int launch_pipeline(const __half* x, const void* wT, const __half* bias, __half*
     prm.epi_alias = 0;
     prm.dual = 0;
     prm.p_stride = ring_p;
+    prm.scales = nullptr;
+    prm.kpad = pl.Kb * 16;
+    prm.raw_slots = 0;
 
     PipeParams pp;
     pp.v_ready = ctr;
@@ -952,7 +986,7 @@ int launch_pipeline(const __half* x, const void* wT, const __half* bias, __half*
 
 int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, int C, int H, int W, int K, int tile,
               void* ws, size_t ws_bytes, cudaStream_t st, const Epilogue& ep_in = Epilogue{nullptr, 0, nullptr},
-              bool io32 = false, bool range_safe = false) {   // io32: x, bias and y are fp32 (the filters come from the fp32 filter transform)
+              bool io32 = false, bool range_safe = false, bool q8 = false) {   // io32: x, bias and y are fp32 (the filters come from the fp32 filter transform)
     if (tile != 2 && tile != 4) {
         return (N <= 0 || C <= 0 || H <= 0 || W <= 0 || K <= 0 || !x || !wT || !y) ? SDWINO_ERR_INVALID_ARG
                                                                                      : SDWINO_ERR_UNSUPPORTED;
@@ -999,7 +1033,8 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
         ep.amax = reinterpret_cast<const float*>(word);
     }
     // the single-kernel paths end at the bias
-    const bool no_ep = ep.residual == nullptr && ep.act == 0 && ep.amax == nullptr;
+    // (8-bit filters: only the GEMM can read them, so neither the single-kernel paths nor the pipelined launch)
+    const bool no_ep = ep.residual == nullptr && ep.act == 0 && ep.amax == nullptr && !q8;
     const bool plain = no_ep && !io32;
     if (no_ep && use_fused_small_k(K, W, tile, pl.P128 / 128, x, y) && !use_fused_small_c(C, tile) &&
         (!io32 || aligned(y, 8)) && !disable_fused) {
@@ -1051,8 +1086,13 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
     GemmParams prm;
     prm.wt_header = wt_header_of(wT);
     prm.K = K;
-    prm.tile = tile;
-    GemmShape shape = choose_gemm_shape(K, C, pc / GEMM_BLOCK_P, pl.a2, sms, force_ctas);
+    prm.tile = q8 ? (tile | static_cast<int>(WT_Q8_FLAG)) : tile;
+    prm.scales = q8 ? reinterpret_cast<const float*>(static_cast<const uint8_t*>(wT) + WT_HEADER_BYTES +
+                                                      q8_bytes_part(pl.a2, pl.Kb, pl.Cb))
+                    : nullptr;
+    prm.kpad = pl.Kb * 16;
+    GemmShape shape = choose_gemm_shape(K, C, pc / GEMM_BLOCK_P, pl.a2, sms, q8 ? 1 : force_ctas);
+    if (q8) shape.dual = 0;
     if (force_n_tile >= 16 && force_n_tile <= GEMM_MAX_N && force_n_tile % 16 == 0) shape.n_tile = force_n_tile;
     if (shape.ctas == 2) shape.n_tile = round_up(shape.n_tile, 32);  // each CTA of a pair loads whole 16-row blocks
     prm.n_tile = shape.n_tile;
@@ -1083,6 +1123,23 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
     prm.stages = (MAX_DYN_SMEM - GemmSmemLayout::dyn_bytes(b_rows, 0, prm.epi_rows, prm.epi_alias ? 0 : prm.epi_bufs)) /
                  (GemmSmemLayout::stage_bytes(b_rows) + (shape.dual ? GemmSmemLayout::A_BYTES : 0));
     if (prm.stages > GEMM_MAX_STAGES) prm.stages = GEMM_MAX_STAGES;
+    prm.raw_slots = 0;
+    if (q8) {
+        // 8-bit filters: give up one operand stage (down to three at least) for a ring of raw filter boxes, which is
+        // what keeps the weight stream from HBM deep: a raw slot is a third of an operand stage or less
+        const int room = MAX_DYN_SMEM - GemmSmemLayout::dyn_bytes(b_rows, 0, prm.epi_rows, prm.epi_alias ? 0 : prm.epi_bufs);
+        const int raw = GemmSmemLayout::raw_bytes(b_rows), stage = GemmSmemLayout::stage_bytes(b_rows);
+        int best_s = 0, best_r = 0;
+        for (int sgs = 2; sgs <= GEMM_MAX_STAGES; ++sgs) {
+            int r = (room - sgs * stage) / raw;
+            if (r > GEMM_MAX_STAGES) r = GEMM_MAX_STAGES;
+            if (r < sgs + 1) continue;                       // the raw ring leads the operand ring
+            if (sgs <= 3 || r >= 6) { best_s = sgs; best_r = r; }
+        }
+        if (best_s == 0) return SDWINO_ERR_UNSUPPORTED;
+        prm.stages = best_s;
+        prm.raw_slots = best_r;
+    }
     {
         // Filter-resident mode (see wino_gemm.cuh): single CTAs, many tiles per CTA and long runs of tiles per
         // (position, k-tile), the filter block two thirds of a stage (n_tile 224-256), and room for it beside a ring
@@ -1099,7 +1156,7 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
         const int stages = (MAX_DYN_SMEM - GemmSmemLayout::dyn_bytes(0, 0, rows, prm.epi_bufs, ures)) / GemmSmemLayout::A_BYTES;
         // (CTA pairs gain nothing from it: with their half of a 512-channel block resident only four 16 KB stages
         // of V remain, too few bytes in flight: 512->512 at 256x256 99 against 94 us)
-        if (shape.ctas == 1 && !shape.dual && force_ctas == 0 && force_n_tile == 0 && p_tiles >= 16 && keys * p_tiles >= 4 * workers &&
+        if (!q8 && shape.ctas == 1 && !shape.dual && force_ctas == 0 && force_n_tile == 0 && p_tiles >= 16 && keys * p_tiles >= 4 * workers &&
             prm.n_tile >= 224 && stages >= 4) {
             prm.resident = 1;
             // CTAs per (position, k-tile) pair.  A group walks `rounds` pairs, each CTA `run` tiles per pair,
@@ -1125,7 +1182,8 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
 
     prm.p_stride = pc;
     CUtensorMap tmU, tmV, tmM;
-    if (!encode_filter_map(&tmU, wt_filters_of(wT), pl.Cb, pl.Kb, pl.a2, b_rows / 16) ||
+    if (!(q8 ? encode_filter_map_q8(&tmU, wt_filters_of(wT), pl.Cb, pl.Kb, pl.a2, b_rows / 16)
+             : encode_filter_map(&tmU, wt_filters_of(wT), pl.Cb, pl.Kb, pl.a2, b_rows / 16)) ||
         !encode_map(&tmV, V, pc, C, pl.a2, pc, static_cast<uint64_t>(C) * pc, 64, GEMM_BLOCK_C, true) ||
         !encode_map(&tmM, Mws, pc, K, pl.a2, pc, static_cast<uint64_t>(K) * pc, GEMM_BLOCK_P, prm.epi_rows, false))
         return err_cuda(__LINE__);
@@ -1134,7 +1192,7 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
     const __half* xh = static_cast<const __half*>(x);
     const __half* bh = static_cast<const __half*>(bias);
     __half* yh = static_cast<__half*>(y);
-    const WtCheck chk{wt_header_of(wT), K, C, tile, status_word_ptr()};
+    const WtCheck chk{wt_header_of(wT), K, C, prm.tile, status_word_ptr()};
     if (!chk.status_word) return err_cuda(__LINE__);
     for (long long p0 = 0; p0 < pl.P; p0 += pc) {
         long long remaining = pl.P128 - p0;
@@ -1153,7 +1211,7 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
         if (rc != SDWINO_OK) return rc;
         const int p_blocks = shape.ctas * (shape.dual ? 2 : 1);      // blocks of 128 tiles per CTA tile / pair tile
         prm.num_p_tiles = (count / GEMM_BLOCK_P + p_blocks - 1) / p_blocks;
-        rc = launch_gemm(tmU, tmV, tmM, prm, shape.ctas, st);
+        rc = launch_gemm(tmU, tmV, tmM, prm, shape.ctas, st, q8);
         if (rc != SDWINO_OK) return rc;
         if (io32) {
             const float* bf = static_cast<const float*>(bias);
@@ -1250,6 +1308,39 @@ int sdwino_filter_transform(const void* w, void* wT, int K, int C, int tile, voi
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (tile == 2) return launch_filter<2>(static_cast<const __half*>(w), wT, K, C, Kb, Cb, st);
     return launch_filter<4>(static_cast<const __half*>(w), wT, K, C, Kb, Cb, st);
+}
+
+size_t sdwino_filter_q8_bytes(int K, int C, int tile) {
+    if (K <= 0 || C <= 0 || (tile != 2 && tile != 4)) return 0;
+    const int a2 = (tile + 2) * (tile + 2), Kb = (K + 15) / 16, Cb = (C + 63) / 64;
+    return WT_HEADER_BYTES + q8_bytes_part(a2, Kb, Cb) + q8_scale_part(a2, Kb);
+}
+
+int sdwino_filter_quantize(const void* wT, void* wTq, int K, int C, int tile, void* stream) {
+    if (!wT || !wTq || K <= 0 || C <= 0) return SDWINO_ERR_INVALID_ARG;
+    if (tile != 2 && tile != 4) return SDWINO_ERR_UNSUPPORTED;
+    if (!aligned(wT, WS_ALIGN) || !aligned(wTq, WS_ALIGN)) return SDWINO_ERR_MISALIGNED;
+    if (static_cast<long double>(K) * C > 4.0e15L) return SDWINO_ERR_INVALID_ARG;
+    const int a2 = (tile + 2) * (tile + 2), Kb = (K + 15) / 16, Cb = (C + 63) / 64;
+    if (static_cast<long long>(a2) * Kb >= (1ll << 31)) return SDWINO_ERR_INVALID_ARG;
+    int* status = status_word_ptr();
+    if (!status) return err_cuda(__LINE__);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint8_t* out = static_cast<uint8_t*>(wTq);
+    ProfScope prof(KIND_FILTER, st);
+    const cudaError_t e = launch_pdl(filter_quantize_kernel, dim3(static_cast<unsigned>(a2 * Kb)), dim3(128), 0, st, 0,
+                                     wt_header_of(wT), static_cast<const __half*>(wt_filters_of(wT)),
+                                     reinterpret_cast<uint32_t*>(out), out + WT_HEADER_BYTES,
+                                     reinterpret_cast<float*>(out + WT_HEADER_BYTES + q8_bytes_part(a2, Kb, Cb)), K, C, tile,
+                                     Kb, Cb, status);
+    g_launches.fetch_add(1);
+    return e == cudaSuccess ? SDWINO_OK : err_cuda(__LINE__);
+}
+
+int sdwino_conv3x3_q8(const void* x, const void* wTq, const void* bias, void* y, int N, int C, int H, int W, int K,
+                      int tile, void* workspace, size_t workspace_bytes, void* stream) {
+    return conv_impl(x, wTq, bias, y, N, C, H, W, K, tile, workspace, workspace_bytes, static_cast<cudaStream_t>(stream),
+                     Epilogue{nullptr, 0, nullptr}, false, false, true);
 }
 
 int sdwino_filter_transform_f32(const float* w, void* wT, int K, int C, int tile, void* stream) {

@@ -228,6 +228,59 @@ filter_transform_kernel(const WT* __restrict__ w, uint32_t* __restrict__ header,
 }
 
 // ---------------------------------------------------------------------------------------
+// 8-bit transformed filter (the quantised operators of Section "Evaluation", "Operator Support").  Input: the fp16
+// blocked filter U[a*a][Cb][Kb][16][64] made by filter_transform_kernel.  Output, same blocking: one byte q + 128 per
+// element with q = round(U / s) in [-127, 127] (fp32 quotient, ties to even) and s = max|U| / 127 taken over the row
+// U[pos][k][:] (one transform position, one output channel, all input channels); the scales follow as
+// S[a*a][Kb * 16] fp32.  The header keeps magic, K and C and marks the format in its tile word.
+// One block of 128 threads per (position, block of 16 output channels): 8 threads per row.
+// ---------------------------------------------------------------------------------------
+constexpr uint32_t WT_Q8_FLAG = 0x100u;   // or-ed into the header's tile word
+__global__ void __launch_bounds__(128)
+filter_quantize_kernel(const uint32_t* __restrict__ header16, const __half* __restrict__ U, uint32_t* __restrict__ header8,
+                       uint8_t* __restrict__ Uq, float* __restrict__ S, int K, int C, int tile, int Kb, int Cb,
+                       int* __restrict__ status_word) {
+    pdl_launch_dependents();
+    pdl_wait();
+    if (!wt_header_ok(header16, K, C, tile, status_word)) return;
+    const int pos = blockIdx.x / Kb, kb = blockIdx.x - pos * Kb;
+    const int row = threadIdx.x >> 3, sub = threadIdx.x & 7;
+    if (blockIdx.x == 0 && threadIdx.x == 0)
+        *reinterpret_cast<uint4*>(header8) = make_uint4(WT_MAGIC, static_cast<uint32_t>(K), static_cast<uint32_t>(C),
+                                                        static_cast<uint32_t>(tile) | WT_Q8_FLAG);
+    const size_t blk0 = (static_cast<size_t>(pos) * Cb * Kb + kb) * 1024 + row * 64 + sub * 8;   // cb = 0
+    const size_t cb_step = static_cast<size_t>(Kb) * 1024;
+    float amax = 0.f;
+    for (int cb = 0; cb < Cb; ++cb) {
+        const uint4 v = *reinterpret_cast<const uint4*>(U + blk0 + cb * cb_step);
+        const uint32_t wds[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&wds[i]));
+            amax = fmaxf(amax, fmaxf(fabsf(f.x), fabsf(f.y)));
+        }
+    }
+    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 4));
+    const float sc = amax > 0.f ? __fdiv_rn(amax, 127.f) : 1.f;
+    if (sub == 0) S[static_cast<size_t>(pos) * Kb * 16 + kb * 16 + row] = sc;
+    for (int cb = 0; cb < Cb; ++cb) {
+        const uint4 v = *reinterpret_cast<const uint4*>(U + blk0 + cb * cb_step);
+        const uint32_t wds[4] = {v.x, v.y, v.z, v.w};
+        uint32_t out[2] = {0u, 0u};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&wds[i]));
+            const int q0 = static_cast<int>(fminf(fmaxf(rintf(__fdiv_rn(f.x, sc)), -127.f), 127.f)) + 128;
+            const int q1 = static_cast<int>(fminf(fmaxf(rintf(__fdiv_rn(f.y, sc)), -127.f), 127.f)) + 128;
+            out[i >> 1] |= (static_cast<uint32_t>(q0) | (static_cast<uint32_t>(q1) << 8)) << ((i & 1) * 16);
+        }
+        *reinterpret_cast<uint2*>(Uq + blk0 + cb * cb_step) = make_uint2(out[0], out[1]);
+    }
+}
+
+// ---------------------------------------------------------------------------------------
 // Tile index arithmetic shared by both activation-side kernels.  Tile p (global index over
 // the whole batch) belongs to image n = p / (TH*TW), tile row th and tile column tw; its
 // input window starts at pixel (m*th - 1, m*tw - 1) and its outputs at (m*th, m*tw).

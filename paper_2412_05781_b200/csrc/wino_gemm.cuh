@@ -63,11 +63,16 @@ struct GemmSmemLayout {
     static constexpr int A_BYTES = GEMM_BLOCK_P * GEMM_BLOCK_C * 2;          // two [64 p][64 c] boxes
     static constexpr int A_BOX_BYTES = 64 * GEMM_BLOCK_C * 2;
     static constexpr int EPI_ROW_BYTES = GEMM_BLOCK_P * 2;                   // one staged row: 128 p fp16
-    static constexpr int BAR_BYTES = (2 * GEMM_MAX_STAGES + 6) * 8 + 16 + 16;   // barriers, two words, four item slots
+    static constexpr int BAR_BYTES = (4 * GEMM_MAX_STAGES + 6) * 8 + 16 + 16;   // barriers, two words, four item slots
     // `rows` = rows of U this CTA loads per stage: n_tile (single CTA) or n_tile / 2 (CTA pair)
     __host__ __device__ static constexpr int b_bytes(int rows) { return rows * GEMM_BLOCK_C * 2; }
     __host__ __device__ static constexpr int stage_bytes(int rows) {
         return (A_BYTES + b_bytes(rows) + 1023) / 1024 * 1024;
+    }
+    // 8-bit filters: a stage also holds the raw bytes of its filter box (64 per row) next to their fp16 expansion
+    __host__ __device__ static constexpr int raw_bytes(int rows) { return rows * GEMM_BLOCK_C; }
+    __host__ __device__ static constexpr int stage_bytes_u8(int rows) {
+        return (A_BYTES + b_bytes(rows) + raw_bytes(rows) + 1023) / 1024 * 1024;
     }
     // epilogue staging: `bufs` buffers of [epi_rows k][128 p] fp16
     __host__ __device__ static constexpr int epi_bytes(int epi_rows, int bufs) {
@@ -100,6 +105,9 @@ struct GemmParams {
                        // pipeline stages instead of a buffer of its own, which leaves room for one more stage
     int dual;          // 1: the kernel instantiation with two blocks of 128 tiles per CTA tile (host side only)
     long long p_stride;  // tiles per pass (row pitch of V and M)
+    const float* scales; // 8-bit filters: S[pos][kpad], the factor of every (position, output channel) row
+    int kpad;            // Kb * 16
+    int raw_slots;       // 8-bit filters: slots of the raw ring (at most GEMM_MAX_STAGES)
 };
 
 // Pipelined mode (template flag PIPE): the three steps of a layer run inside ONE persistent launch.  V and M are rings
@@ -176,13 +184,20 @@ __device__ __forceinline__ void signal_counter_release(unsigned int* ctr) {
 // tmM: fp16 [pos][K][Pstride]   box {128 p, epi_rows k, 1}, no swizzle  (result; rows k >= K are clipped)
 // RES: the filter-resident mode, DUAL: two blocks of 128 tiles per CTA tile; separate instantiations, so that the
 // plain streaming kernel pays nothing for them.
-template <int CTAS, bool RES = false, bool DUAL = false, bool PIPE = false>
+// U8: 8-bit filters (see filter_quantize_kernel).  The producer brings the bytes of a filter box into the stage's raw
+// area; the eight epilogue warps, idle during a mainloop, expand them to fp16 in the swizzled operand layout (an
+// integer of at most 127 is exact in fp16) and complete the stage's barrier; the scale of every (position, output
+// channel) row multiplies the accumulator in the epilogue.  Half the filter bytes cross HBM and L2; the contraction is
+// still kind::f16.  Meant for the weight-streaming layers (one tile per CTA): with several tiles per CTA the epilogue
+// of one tile no longer overlaps the mainloop of the next.
+template <int CTAS, bool RES = false, bool DUAL = false, bool PIPE = false, bool U8 = false>
 __global__ void __launch_bounds__(PIPE ? PIPE_THREADS : GEMM_THREADS, 1)
 wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant__ CUtensorMap tmV,
                  const __grid_constant__ CUtensorMap tmM, const GemmParams prm, int* __restrict__ status_word,
                  const PipeParams pp) {
     using L = GemmSmemLayout;
     static_assert(!PIPE || (CTAS == 1 && !DUAL), "the pipelined mode runs single CTAs, one block of tiles per CTA tile");
+    static_assert(!U8 || (CTAS == 1 && !RES && !DUAL && !PIPE), "8-bit filters: single CTAs, streaming mode");
     // The activation transform before this kernel has waited for everything before it, so the filter header is
     // final: its load is issued first and looked at after the set-up below (uniform over the CTA).
     const uint4 wt_hdr = *reinterpret_cast<const uint4*>(prm.wt_header);
@@ -196,7 +211,9 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
     constexpr int a_bytes = PT * L::A_BYTES;         // V part of a stage
     const int stage_bytes = resident ? L::A_BYTES : (PT - 1) * L::A_BYTES + L::stage_bytes(b_rows);
     const int ures_cb_bytes = L::b_bytes(prm.n_tile);                       // one 64-channel block of the resident filters
-    const int ures_bytes = resident ? prm.num_c_blocks * ures_cb_bytes : 0;
+    // 8-bit filters: the same area holds a ring of raw filter boxes (64 bytes per row), deeper than the operand ring
+    [[maybe_unused]] const int raw_slot_bytes = L::raw_bytes(b_rows);
+    const int ures_bytes = resident ? prm.num_c_blocks * ures_cb_bytes : (U8 ? prm.raw_slots * raw_slot_bytes : 0);
     const int stages = prm.stages;
     const uint32_t cta_rank = CTAS == 2 ? cluster_ctarank() : 0u;
     const bool leader = cta_rank == 0;
@@ -211,7 +228,9 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
     uint64_t* acc_empty_bar = acc_full_bar + 2;
     uint64_t* ures_full_bar = acc_empty_bar + 2;     // the resident filter block has arrived
     uint64_t* ures_empty_bar = ures_full_bar + 1;    // the MMAs that read it have completed
-    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(ures_empty_bar + 1);
+    uint64_t* raw_full_bar = ures_empty_bar + 1;     // 8-bit filters: the bytes of a raw slot have arrived
+    uint64_t* raw_empty_bar = raw_full_bar + GEMM_MAX_STAGES;   // ... and have been expanded by all eight warps
+    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(raw_empty_bar + GEMM_MAX_STAGES);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_base_slot + 1);
     [[maybe_unused]] volatile unsigned int* item_slots = reinterpret_cast<volatile unsigned int*>(tmem_base_slot + 2);   // 4 words
 
@@ -264,8 +283,12 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) {
-            mbar_init(&full_bar[s], 1);
+            mbar_init(&full_bar[s], U8 ? 9 : 1);      // 8-bit filters: the producer and the eight converting warps
             mbar_init(&empty_bar[s], 1);
+        }
+        for (int s = 0; s < GEMM_MAX_STAGES; ++s) {
+            mbar_init(&raw_full_bar[s], 1);
+            mbar_init(&raw_empty_bar[s], 8);
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(&acc_full_bar[b], 1);
@@ -362,6 +385,68 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
                     if (++stage == stages) { stage = 0; phase ^= 1u; sa = smem_base; fb = full0; }
                 }
             }
+            if (!ok) *abort_flag = 1;
+        } else if (U8 && lane == 0) {
+            // 8-bit filters.  Two streams from one thread: the raw filter boxes, which come from HBM and depend on
+            // nothing, run `lead` steps ahead of the boxes of V through a ring of their own; a step's operand stage is
+            // completed by V (this thread) and by the warps that expand the raw box into it.
+            const int R = prm.raw_slots, lead = R - 1;
+            const int spt = prm.num_c_blocks;                  // steps per tile
+            const int total = my_count * spt;
+            const uint32_t smem_base = smem_u32(smem);
+            const uint32_t raw_base = smem_u32(ures_base);
+            const uint64_t u_policy = l2_policy_evict_first();
+            bool ok = true;
+            // running state of the two streams (no division in this single-thread loop)
+            int r_slot = 0, r_cb = 0, r_tile = 0, r_kb = 0, r_pos = 0;
+            uint32_t r_par = 1;                                // parity to wait for on raw_empty: passes in the first round
+            int v_stage = 0, v_cb = 0, v_tile = 0, v_p0 = 0, v_pos = 0;
+            uint32_t v_par = 1;
+            if (total > 0) {
+                int pt, kt;
+                decode(tile_of(0), pt, kt, r_pos);
+                r_kb = (kt * prm.n_tile) >> 4;
+                v_p0 = pt * GEMM_BLOCK_P;
+                v_pos = r_pos;
+            }
+            for (int j = 0; j < total + lead && ok; ++j) {
+                if (j < total) {
+                    ok = mbar_wait_bounded(&raw_empty_bar[r_slot], r_par, abort_flag, GEMM_WAIT_LIMIT_NS);
+                    if (!ok) { if (*abort_flag == 0) report_timeout(status_word, 8, cta_rank); break; }
+                    const uint32_t rb = smem_u32(&raw_full_bar[r_slot]);
+                    mbar_arrive_expect_tx_a32(rb, static_cast<uint32_t>(raw_slot_bytes));
+                    tma_load_5d_hint_a32(raw_base + r_slot * raw_slot_bytes, &tmU, rb, r_cb, r_kb, r_pos, u_policy);
+                    if (++r_slot == R) { r_slot = 0; r_par ^= 1u; }
+                    if (++r_cb == spt) {
+                        r_cb = 0;
+                        if (++r_tile < my_count) {
+                            int pt, kt;
+                            decode(tile_of(r_tile), pt, kt, r_pos);
+                            r_kb = (kt * prm.n_tile) >> 4;
+                        }
+                    }
+                }
+                if (j >= lead) {
+                    if (j == lead) pdl_wait();                 // V is written by the preceding kernel
+                    ok = mbar_wait_bounded(&empty_bar[v_stage], v_par, abort_flag, GEMM_WAIT_LIMIT_NS);
+                    if (!ok) { if (*abort_flag == 0) report_timeout(status_word, 1, cta_rank); break; }
+                    const uint32_t fb = smem_u32(&full_bar[v_stage]);
+                    const uint32_t sa = smem_base + v_stage * stage_bytes;
+                    mbar_arrive_expect_tx_a32(fb, static_cast<uint32_t>(a_bytes));
+                    tma_load_3d_a32(sa, &tmV, fb, v_p0, v_cb * GEMM_BLOCK_C, v_pos);
+                    tma_load_3d_a32(sa + L::A_BOX_BYTES, &tmV, fb, v_p0 + 64, v_cb * GEMM_BLOCK_C, v_pos);
+                    if (++v_stage == stages) { v_stage = 0; v_par ^= 1u; }
+                    if (++v_cb == spt) {
+                        v_cb = 0;
+                        if (++v_tile < my_count) {
+                            int pt, kt;
+                            decode(tile_of(v_tile), pt, kt, v_pos);
+                            v_p0 = pt * GEMM_BLOCK_P;
+                        }
+                    }
+                }
+            }
+            if (total == 0) pdl_wait();
             if (!ok) *abort_flag = 1;
         } else if (!resident && lane == 0) {
             // the full barrier of a pair lives in the leader and counts the bytes of both CTAs
@@ -581,10 +666,69 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
         // one iteration per accumulator: a tile of two blocks of 128 tiles p (DUAL) fills both buffers, which are
         // drained in turn exactly as two consecutive tiles would be
         [[maybe_unused]] int pend_pt = -1;     // pipelined mode, group_tid 0: block whose stores are to be announced
+        [[maybe_unused]] int cv_stage = 0;     // 8-bit filters: the stage these warps expand next
+        [[maybe_unused]] uint32_t cv_phase = 0;
+        [[maybe_unused]] int cv_raw = 0;       // ... and the raw slot they read next
+        [[maybe_unused]] uint32_t cv_raw_par = 0;
         for (int i2 = 0; i2 < my_count * PT; ++i2) {
             int pt, kt, pos;
             decode(tile_of(i2 / PT), pt, kt, pos);
             pt = pt * PT + (i2 % PT);
+            if constexpr (U8) {
+                // Expand the filter bytes of every stage of this tile: thread -> (row, 16 channels) of the box; the
+                // 16 bytes become two 16-byte pieces of the row's 128 bytes, placed where the 128-byte swizzle puts
+                // them (piece j of row r at position j ^ (r & 7)).  q + 128 is a byte; 0x6400 | byte is the fp16
+                // number 1024 + byte, and subtracting 1152 leaves q exactly.
+                const int ct = static_cast<int>(threadIdx.x) - 64;       // 0 .. 255
+                const __half2 bias1152 = __half2half2(__ushort_as_half(static_cast<unsigned short>(0x6480)));
+                for (int cb = 0; cb < prm.num_c_blocks; ++cb) {
+                    // the operand stage is free once the MMAs that read its previous contents have completed, and the
+                    // raw box of this step has arrived (one lane polls, the warp follows)
+                    bool cv_ok = true;
+                    if (lane == 0) {
+                        cv_ok = mbar_wait_bounded(&empty_bar[cv_stage], cv_phase ^ 1u, abort_flag, GEMM_WAIT_LIMIT_NS) &&
+                                mbar_wait_bounded(&raw_full_bar[cv_raw], cv_raw_par, abort_flag, GEMM_WAIT_LIMIT_NS);
+                    }
+                    cv_ok = __all_sync(0xffffffffu, cv_ok);
+                    if (!cv_ok) {
+                        // This warp stops converting but does NOT leave: with the abort flag set the accumulator wait
+                        // below fails for every warp, and each group then leaves through its named barrier together.
+                        if (lane == 0) {
+                            if (*abort_flag == 0) report_timeout(status_word, 15, cta_rank);
+                            *abort_flag = 1;
+                        }
+                        break;
+                    }
+                    const uint8_t* raw = ures_base + cv_raw * raw_slot_bytes;
+                    uint8_t* bop = smem + cv_stage * stage_bytes + a_bytes;
+                    for (int idx = ct; idx < b_rows * 4; idx += 256) {
+                        const int row = idx >> 2, q = idx & 3;
+                        const uint4 v = *reinterpret_cast<const uint4*>(raw + row * GEMM_BLOCK_C + q * 16);
+                        const uint32_t wds[4] = {v.x, v.y, v.z, v.w};
+                        uint32_t h[8];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            uint32_t lo = __byte_perm(wds[i], 0x64646464u, 0x4140);   // (0x6400 | b0, 0x6400 | b1)
+                            uint32_t hi = __byte_perm(wds[i], 0x64646464u, 0x4342);   // (0x6400 | b2, 0x6400 | b3)
+                            const __half2 l2 = __hsub2(*reinterpret_cast<const __half2*>(&lo), bias1152);
+                            const __half2 h2 = __hsub2(*reinterpret_cast<const __half2*>(&hi), bias1152);
+                            h[2 * i] = *reinterpret_cast<const uint32_t*>(&l2);
+                            h[2 * i + 1] = *reinterpret_cast<const uint32_t*>(&h2);
+                        }
+                        uint8_t* rowp = bop + row * 128;
+                        *reinterpret_cast<uint4*>(rowp + (((2 * q) ^ (row & 7)) << 4)) = make_uint4(h[0], h[1], h[2], h[3]);
+                        *reinterpret_cast<uint4*>(rowp + (((2 * q + 1) ^ (row & 7)) << 4)) = make_uint4(h[4], h[5], h[6], h[7]);
+                    }
+                    fence_proxy_async_smem();      // the MMA reads the operand through the async proxy
+                    __syncwarp();
+                    if (lane == 0) {
+                        mbar_arrive(&full_bar[cv_stage]);
+                        mbar_arrive(&raw_empty_bar[cv_raw]);
+                    }
+                    if (++cv_stage == stages) { cv_stage = 0; cv_phase ^= 1u; }
+                    if (++cv_raw == prm.raw_slots) { cv_raw = 0; cv_raw_par ^= 1u; }
+                }
+            }
             // the staging buffer about to be overwritten must have been read by the group's previous TMA store
             if (group_tid == 0) tma_store_wait_read_pending<0>();
             [[maybe_unused]] unsigned int seen_o = 0;
@@ -622,20 +766,28 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
                     else asm volatile("bar.sync 2, 128;" ::: "memory");
                 }
                 __half* dst = reinterpret_cast<__half*>(stg) + quarter * 32 + lane;
+                // 8-bit filters: the factor of every output channel of this position (rows past K read padding)
+                [[maybe_unused]] const float* sc = U8 ? prm.scales + static_cast<long long>(pos) * prm.kpad + k0 + row0 : nullptr;
                 int col = 0;
                 for (; col + 32 <= prm.epi_rows; col += 32) {
                     uint32_t r[32];
                     tmem_ld_32x32_sync(t_addr + row0 + col, r);
 #pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        dst[(col + i) * GEMM_BLOCK_P] = __float2half_rn(__uint_as_float(r[i]));
+                    for (int i = 0; i < 32; ++i) {
+                        float v = __uint_as_float(r[i]);
+                        if constexpr (U8) v *= (k0 + row0 + col + i < prm.kpad) ? __ldg(sc + col + i) : 0.f;
+                        dst[(col + i) * GEMM_BLOCK_P] = __float2half_rn(v);
+                    }
                 }
                 if (col < prm.epi_rows) {
                     uint32_t r[16];
                     tmem_ld_32x16_sync(t_addr + row0 + col, r);
 #pragma unroll
-                    for (int i = 0; i < 16; ++i)
-                        dst[(col + i) * GEMM_BLOCK_P] = __float2half_rn(__uint_as_float(r[i]));
+                    for (int i = 0; i < 16; ++i) {
+                        float v = __uint_as_float(r[i]);
+                        if constexpr (U8) v *= (k0 + row0 + col + i < prm.kpad) ? __ldg(sc + col + i) : 0.f;
+                        dst[(col + i) * GEMM_BLOCK_P] = __float2half_rn(v);
+                    }
                 }
                 fence_proxy_async_smem();
                 if (group == 0) asm volatile("bar.sync 1, 128;" ::: "memory");
