@@ -54,6 +54,7 @@ def _load():
         i = ctypes.c_int
         lib.oracle_direct.argtypes = [dp, dp, dp, dp, i, i, i, i, i]
         lib.oracle_direct_channels.argtypes = [dp, dp, dp, dp, i, i, i, i, i, ip, i]
+        lib.oracle_direct_strided.argtypes = [dp, dp, dp, dp, i, i, i, i, i, i]
         lib.oracle_filter_transform.argtypes = [dp, dp, dp, i, i, i]
         lib.oracle_input_tile_transform.argtypes = [dp, dp, dp, i, i, i, i, i, i, i, i]
         lib.oracle_winograd.argtypes = [dp, dp, dp, dp, i, i, i, i, i, i, dp, dp, dp]
@@ -128,6 +129,21 @@ def direct_conv3x3(x, w, bias=None, channels=None):
             ks.ctypes.data_as(ctypes.POINTER(ctypes.c_int)), len(ks))
     if rc != 0:
         raise RuntimeError(f"oracle_direct failed ({rc})")
+    return y
+
+
+def direct_conv3x3_strided(x, w, bias=None, stride: int = 2):
+    """The 3x3 convolution with zero padding 1 sampled with a stride (the downsampling convolutions of the UNet):
+    y[n,k,i,j] = b[k] + sum_{c,u,v} xhat[n,c,s*i+u-1,s*j+v-1] * w[k,c,u,v], shape [N, K, (H-1)//s+1, (W-1)//s+1]."""
+    x, w = _f64(x), _f64(w)
+    N, C, H, W = x.shape
+    K = w.shape[0]
+    assert w.shape == (K, C, 3, 3) and stride >= 1
+    b = _f64(bias) if bias is not None else None
+    y = np.empty((N, K, (H - 1) // stride + 1, (W - 1) // stride + 1), dtype=np.float64)
+    rc = _load().oracle_direct_strided(_ptr(x), _ptr(w), _ptr(b), _ptr(y), N, C, H, W, K, stride)
+    if rc != 0:
+        raise RuntimeError(f"oracle_direct_strided failed ({rc})")
     return y
 
 

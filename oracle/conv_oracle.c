@@ -66,6 +66,34 @@ int oracle_direct_channels(const double *x, const double *w, const double *bias,
     return 0;
 }
 
+/* The same sum sampled with stride s (the downsampling convolutions of the UNet, stride 2, pad 1):
+ * y[n][k][i][j] = b[k] + sum_c sum_u sum_v xhat[n][c][s*i+u-1][s*j+v-1] * w[k][c][u][v],
+ * i < Ho = (H - 1) / s + 1, j < Wo = (W - 1) / s + 1.  y has shape [N][K][Ho][Wo]. */
+int oracle_direct_strided(const double *x, const double *w, const double *bias, double *y,
+                          int N, int C, int H, int W, int K, int s)
+{
+    if (!x || !w || !y || N <= 0 || C <= 0 || H <= 0 || W <= 0 || K <= 0 || s <= 0) return 1;
+    int Ho = (H - 1) / s + 1, Wo = (W - 1) / s + 1;
+    long long planes = (long long)N * K;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (long long pl = 0; pl < planes; ++pl) {
+        int n = (int)(pl / K), k = (int)(pl % K);
+        double *yp = y + (size_t)pl * Ho * Wo;
+        double b = bias ? bias[k] : 0.0;
+        for (int i = 0; i < Ho; ++i)
+            for (int j = 0; j < Wo; ++j) {
+                double acc = 0.0;
+                for (int c = 0; c < C; ++c)
+                    for (int u = 0; u < 3; ++u)
+                        for (int v = 0; v < 3; ++v)
+                            acc += x_at(x, C, H, W, n, c, s * i + u - 1, s * j + v - 1) *
+                                   w[IDX4(k, c, u, v, C, 3, 3)];
+                yp[(size_t)i * Wo + j] = b + acc;
+            }
+    }
+    return 0;
+}
+
 int oracle_direct(const double *x, const double *w, const double *bias, double *y,
                   int N, int C, int H, int W, int K)
 {

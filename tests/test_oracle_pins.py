@@ -333,3 +333,32 @@ def test_int8_filter_convolution_is_close_to_the_exact_one_but_not_equal():
     yq = oracle.winograd_conv3x3_q8(xs, wd, None, 2, None)
     # scale = 1/127 is not a power of two, so "exact" means: to the rounding of 127 * (1/127) in fp32
     assert np.abs(yq - oracle.direct_conv3x3(xs, wd)).max() <= 1e-6 * np.abs(xs).max() * 2
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# strided direct convolution (the downsampling convolutions)
+# ---------------------------------------------------------------------------------------------------------------
+def test_strided_direct_conv_is_the_subsampled_stride_1_result_and_matches_torch():
+    rng = np.random.default_rng(12)
+    for (N, C, K, H, W) in [(1, 1, 1, 4, 4), (2, 3, 4, 7, 10), (1, 5, 2, 8, 5), (1, 2, 3, 1, 6)]:
+        x = rng.standard_normal((N, C, H, W))
+        w = rng.standard_normal((K, C, 3, 3))
+        b = rng.standard_normal(K)
+        y1 = oracle.direct_conv3x3(x, w, b)                      # pinned above by hand values, brute force, torch, scipy
+        assert np.array_equal(oracle.direct_conv3x3_strided(x, w, b, 1), y1)
+        for s in (2, 3):
+            ys = oracle.direct_conv3x3_strided(x, w, b, s)
+            assert ys.shape == (N, K, (H - 1) // s + 1, (W - 1) // s + 1)
+            assert np.array_equal(ys, y1[:, :, ::s, ::s])         # output (i, j) of stride s is output (s i, s j) of stride 1
+            ref = torch.nn.functional.conv2d(torch.from_numpy(x), torch.from_numpy(w), torch.from_numpy(b), stride=s, padding=1)
+            assert np.abs(ys - ref.numpy()).max() <= 1e-12
+
+
+def test_strided_direct_conv_hand_worked_values():
+    # 1 x 1 x 4 x 4 input 1..16, all-ones filter, stride 2: output (i, j) sums the window centred at (2i, 2j):
+    # (0,0): rows 0-1, cols 0-1 -> 1+2+5+6 = 14; (0,1): rows 0-1, cols 1-3 -> 2+3+4+6+7+8 = 30;
+    # (1,0): rows 1-3, cols 0-1 -> 5+6+9+10+13+14 = 57; (1,1): rows 1-3, cols 1-3 -> 6+7+8+10+11+12+14+15+16 = 99
+    x = np.arange(1, 17, dtype=np.float64).reshape(1, 1, 4, 4)
+    w = np.ones((1, 1, 3, 3))
+    y = oracle.direct_conv3x3_strided(x, w, None, 2)
+    assert y.reshape(-1).tolist() == [14.0, 30.0, 57.0, 99.0]
