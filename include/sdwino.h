@@ -180,6 +180,25 @@ int sdwino_conv3x3_q8(const void *x, const void *wTq, const void *bias, void *y,
                       void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * The direct convolution, stride 1 or 2 (Abstract / Section "Techniques": the operator the paper replaces is
+ * ggml_conv_2d as a whole; the UNet's downsampling convolutions are 3x3, pad 1, stride 2, which Winograd's
+ * overlapping tiles cannot express).  It is the degenerate member of the family, F(1x1,3x3): a tile is one output
+ * pixel, the nine transform positions are the nine filter taps, and the same three steps run: the activation step
+ * gathers the nine shifted copies of x (V[tap][c][pixel]), the tcgen05 GEMM contracts the channels per tap, the output
+ * step adds the nine partial sums and the bias.  It streams 9 instead of 16 (tile 2) filter values per weight, at
+ * 2.25 times the tensor work per output pixel.
+ *   filters: sdwino_filter_bytes / sdwino_filter_transform with tile = 1 (the weights reordered tap by tap).
+ *   y: fp16 [N][K][Ho][Wo] with Ho = (H - 1) / stride + 1, Wo = (W - 1) / stride + 1; stride 1 or 2
+ *   (SDWINO_ERR_UNSUPPORTED above 2, SDWINO_ERR_INVALID_ARG below 1).  Workspace: sdwino_workspace_bytes_direct for
+ *   one pass; smaller workspaces take several passes as in sdwino_conv3x3_ws.  Other arguments and errors as
+ *   sdwino_conv3x3_ws.
+ */
+size_t sdwino_workspace_bytes_direct(int N, int C, int H, int W, int K, int stride);
+int sdwino_conv3x3_direct(const void *x, const void *wT, const void *bias, void *y,
+                          int N, int C, int H, int W, int K, int stride,
+                          void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * The convolution for callers that must not allocate device memory.  (The paper has no
  * counterpart; this entry point exists for the embedding of the library.)  Some callers cannot
  * call cudaMalloc or any allocator at all: code that runs inside a CUDA-graph capture or another

@@ -26,6 +26,7 @@ EXPORTS = [
     "sdwino_filter_transform_f32", "sdwino_conv3x3_f32", "sdwino_conv3x3_f32_ex",
     "sdwino_host_staging_bytes_f32", "sdwino_conv3x3_host_f32", "sdwino_conv3x3_host_f32_async", "sdwino_set_pipeline",
     "sdwino_conv3x3_f32_scaled", "sdwino_filter_q8_bytes", "sdwino_filter_quantize", "sdwino_conv3x3_q8",
+    "sdwino_workspace_bytes_direct", "sdwino_conv3x3_direct",
 ]
 
 KERNEL_KINDS = ("filter_transform", "input_transform", "wino_gemm", "output_transform", "fused", "layer")
@@ -103,6 +104,10 @@ def _load() -> ctypes.CDLL:
     lib.sdwino_filter_quantize.argtypes = [vp, vp, i, i, i, vp]
     lib.sdwino_conv3x3_q8.restype = i
     lib.sdwino_conv3x3_q8.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, vp, sz, vp]
+    lib.sdwino_workspace_bytes_direct.restype = sz
+    lib.sdwino_workspace_bytes_direct.argtypes = [i] * 6
+    lib.sdwino_conv3x3_direct.restype = i
+    lib.sdwino_conv3x3_direct.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, vp, sz, vp]
     lib.sdwino_set_pipeline.restype = i
     lib.sdwino_set_pipeline.argtypes = [i, i, i]
     lib.sdwino_profile_enable.restype = i
@@ -437,4 +442,23 @@ def sdwino_conv3x3_q8(x: torch.Tensor, wTq: torch.Tensor, bias: Optional[torch.T
     rc = lib.sdwino_conv3x3_q8(x.data_ptr(), wTq.data_ptr(), _ptr(bias), y.data_ptr(), N, C, H, W, K, tile,
                                workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream_ptr(stream))
     _check(rc, "sdwino_conv3x3_q8")
+    return y
+
+
+def sdwino_workspace_bytes_direct(N: int, C: int, H: int, W: int, K: int, stride: int) -> int:
+    return int(lib.sdwino_workspace_bytes_direct(N, C, H, W, K, stride))
+
+
+def sdwino_conv3x3_direct(x: torch.Tensor, wT: torch.Tensor, bias: Optional[torch.Tensor], K: int, stride: int,
+                          workspace: torch.Tensor, y: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """The direct 3x3 convolution (pad 1) with stride 1 or 2: wT from sdwino_filter_transform(w, 1)."""
+    assert x.is_cuda and x.dtype == torch.float16 and x.is_contiguous() and x.dim() == 4
+    N, C, H, W = (int(v) for v in x.shape)
+    Ho, Wo = (H - 1) // max(stride, 1) + 1, (W - 1) // max(stride, 1) + 1
+    if y is None:
+        y = torch.empty((N, K, Ho, Wo), dtype=torch.float16, device=x.device)
+    assert y.is_cuda and y.is_contiguous() and y.dtype == torch.float16 and tuple(y.shape) == (N, K, Ho, Wo)
+    rc = lib.sdwino_conv3x3_direct(x.data_ptr(), wT.data_ptr(), _ptr(bias), y.data_ptr(), N, C, H, W, K, stride,
+                                   workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    _check(rc, "sdwino_conv3x3_direct")
     return y

@@ -115,17 +115,21 @@ struct Plan {
     long long P;       // tiles in the whole batch
     long long P128;    // P rounded up to the GEMM tile
     size_t per_tile;   // workspace bytes per tile column (V + M)
+    int Ho, Wo;        // output image (equal to H, W except for the strided direct convolution)
 };
 
-bool make_plan(int N, int C, int H, int W, int K, int tile, Plan* pl) {
+// tile 2 / 4: Winograd; tile 1 with stride >= 1: the direct convolution (a tile is one output pixel)
+bool make_plan(int N, int C, int H, int W, int K, int tile, Plan* pl, int stride = 0) {
     if (N <= 0 || C <= 0 || H <= 0 || W <= 0 || K <= 0) return false;
-    if (tile != 2 && tile != 4) return false;
+    if (stride > 0 ? (tile != 1 || stride > 2) : (tile != 2 && tile != 4)) return false;
     const int a = tile + 2;
     pl->a2 = a * a;
     pl->Kb = (K + 15) / 16;
     pl->Cb = (C + 63) / 64;
-    pl->TH = (H + tile - 1) / tile;
-    pl->TW = (W + tile - 1) / tile;
+    pl->Ho = stride > 0 ? (H - 1) / stride + 1 : H;
+    pl->Wo = stride > 0 ? (W - 1) / stride + 1 : W;
+    pl->TH = stride > 0 ? pl->Ho : (H + tile - 1) / tile;
+    pl->TW = stride > 0 ? pl->Wo : (W + tile - 1) / tile;
     pl->P = static_cast<long long>(N) * pl->TH * pl->TW;
     if (pl->P >= (1ll << 31) - GEMM_BLOCK_P) return false;   // tile indices are 32-bit on the device
     pl->P128 = round_up_ll(pl->P, GEMM_BLOCK_P);
@@ -438,7 +442,10 @@ int launch_input(const XT* x, __half* V, const TileGeom& geo, int C, long long p
     constexpr int TPT = 8 / M;
     cudaError_t e;
     const long long units = static_cast<long long>(p_count / TPT) * C;   // one thread each
-    if (geo.W % 8 == 0 && aligned(x, 16) && units < (1ll << 31) - 128) {
+    if constexpr (M == 1) {
+        const dim3 grid = grid_rows((p_count + 127) / 128, C);
+        e = launch_pdl(input_transform_kernel<M, XT>, grid, dim3(128), 0, st, 0, x, V, geo, C, p_begin, p_count, Pstride, amax);
+    } else if (geo.W % 8 == 0 && aligned(x, 16) && units < (1ll << 31) - 128) {
         if constexpr (M == 4) {
             constexpr int CH = 1;   // channels per thread
             const long long threads = static_cast<long long>(p_count / TPT) * ((C + CH - 1) / CH);
@@ -620,7 +627,11 @@ int launch_output(const __half* Mws, const YT* bias, YT* y, const TileGeom& geo,
     constexpr int TPT = 8 / M;
     cudaError_t e;
     const long long units = static_cast<long long>(p_count / TPT) * K;   // one thread each
-    if (geo.W % 8 == 0 && aligned(y, 16) && aligned(ep.residual, 16) && units < (1ll << 31) - 128) {
+    if constexpr (M == 1) {
+        const dim3 grid = grid_rows((p_count + 127) / 128, K);
+        e = launch_pdl(output_transform_kernel<M, YT>, grid, dim3(128), 0, st, 0, Mws, bias, y, geo, K, p_begin, p_count,
+                       Pstride, chk, ep);
+    } else if (geo.W % 8 == 0 && aligned(y, 16) && aligned(ep.residual, 16) && units < (1ll << 31) - 128) {
         dim3 grid(static_cast<unsigned>((units + 127) / 128));
         if (ep.residual == nullptr && ep.act == 0) {
             e = launch_pdl(output_transform_vec_kernel<M, TPT, false, YT>, grid, dim3(128), 0, st, 0, Mws, bias, y, geo, K,
@@ -639,7 +650,7 @@ int launch_output(const __half* Mws, const YT* bias, YT* y, const TileGeom& geo,
 }
 
 // Layers with at most 8 (tile 2) or 4 (tile 4) input channels run as one fused kernel without a workspace.
-bool use_fused_small_c(int C, int tile) { return tile == 2 ? C <= 8 : C <= 4; }
+bool use_fused_small_c(int C, int tile) { return tile == 2 ? C <= 8 : (tile == 4 && C <= 4); }
 
 template <int M, int CP>
 int launch_fused_small_c(const __half* x, const void* wT, const __half* bias, __half* y, const TileGeom& geo, int C,
@@ -986,13 +997,15 @@ int launch_pipeline(const __half* x, const void* wT, const __half* bias, __half*
 
 int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, int C, int H, int W, int K, int tile,
               void* ws, size_t ws_bytes, cudaStream_t st, const Epilogue& ep_in = Epilogue{nullptr, 0, nullptr},
-              bool io32 = false, bool range_safe = false, bool q8 = false) {   // io32: x, bias and y are fp32 (the filters come from the fp32 filter transform)
-    if (tile != 2 && tile != 4) {
+              bool io32 = false, bool range_safe = false, bool q8 = false, int stride = 0) {
+    // io32: x, bias and y are fp32 (the filters come from the fp32 filter transform); stride > 0: the direct
+    // convolution (tile 1, fp16 interface), whose tiles are single output pixels
+    if (stride > 0 ? (tile != 1 || stride > 2 || io32 || q8) : (tile != 2 && tile != 4)) {
         return (N <= 0 || C <= 0 || H <= 0 || W <= 0 || K <= 0 || !x || !wT || !y) ? SDWINO_ERR_INVALID_ARG
                                                                                      : SDWINO_ERR_UNSUPPORTED;
     }
     Plan pl;
-    if (!x || !wT || !y || !make_plan(N, C, H, W, K, tile, &pl)) return SDWINO_ERR_INVALID_ARG;
+    if (!x || !wT || !y || !make_plan(N, C, H, W, K, tile, &pl, stride)) return SDWINO_ERR_INVALID_ARG;
     // the overrides are read once per call
     const int force_ctas = g_force_ctas.load(), force_n_tile = g_force_n_tile.load();
     const bool disable_fused = g_disable_fused.load();
@@ -1188,7 +1201,8 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
         !encode_map(&tmM, Mws, pc, K, pl.a2, pc, static_cast<uint64_t>(K) * pc, GEMM_BLOCK_P, prm.epi_rows, false))
         return err_cuda(__LINE__);
 
-    const TileGeom geo = make_geom(H, W, pl.TH, pl.TW, pl.P);
+    const TileGeom geo = make_geom(H, W, pl.TH, pl.TW, pl.P, stride > 0 ? stride : 1);
+    const TileGeom geo_out = make_geom(pl.Ho, pl.Wo, pl.TH, pl.TW, pl.P);    // differs from geo for the strided convolution
     const __half* xh = static_cast<const __half*>(x);
     const __half* bh = static_cast<const __half*>(bias);
     __half* yh = static_cast<__half*>(y);
@@ -1202,7 +1216,8 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
             const float* xf = static_cast<const float*>(x);
             rc = tile == 2 ? launch_input<2>(xf, V, geo, C, p0, count, pc, st, ep.amax)
                            : launch_input<4>(xf, V, geo, C, p0, count, pc, st, ep.amax);
-        } else if (tile == 2) rc = launch_input<2>(xh, V, geo, C, p0, count, pc, st);
+        } else if (tile == 1) rc = launch_input<1>(xh, V, geo, C, p0, count, pc, st);
+        else if (tile == 2) rc = launch_input<2>(xh, V, geo, C, p0, count, pc, st);
         else {
             rc = use_input_tma(geo, N, C, x, p0, count) ? launch_input_tma(xh, V, geo, N, C, p0, count, pc, st)
                                                         : SDWINO_ERR_UNSUPPORTED;
@@ -1219,7 +1234,8 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
             if (tile == 2) rc = launch_output<2>(Mws, bf, yf, geo, K, p0, count, pc, chk, ep, st);
             else if (use_output_tma(geo, K, y, ep, count)) rc = launch_output_tma(Mws, bf, yf, geo, K, p0, count, pc, chk, ep, st);
             else rc = launch_output<4>(Mws, bf, yf, geo, K, p0, count, pc, chk, ep, st);
-        } else if (tile == 2) rc = launch_output<2>(Mws, bh, yh, geo, K, p0, count, pc, chk, ep, st);
+        } else if (tile == 1) rc = launch_output<1>(Mws, bh, yh, geo_out, K, p0, count, pc, chk, ep, st);
+        else if (tile == 2) rc = launch_output<2>(Mws, bh, yh, geo, K, p0, count, pc, chk, ep, st);
         else if (use_output_tma(geo, K, y, ep, count)) rc = launch_output_tma(Mws, bh, yh, geo, K, p0, count, pc, chk, ep, st);
         else rc = launch_output<4>(Mws, bh, yh, geo, K, p0, count, pc, chk, ep, st);
         if (rc != SDWINO_OK) return rc;
@@ -1293,7 +1309,7 @@ const char* sdwino_status_string(int status) {
 }
 
 size_t sdwino_filter_bytes(int K, int C, int tile) {
-    if (K <= 0 || C <= 0 || (tile != 2 && tile != 4)) return 0;
+    if (K <= 0 || C <= 0 || (tile != 1 && tile != 2 && tile != 4)) return 0;
     const size_t a = tile + 2;
     const size_t bytes = a * a * static_cast<size_t>((K + 15) / 16) * ((C + 63) / 64) * 1024 * sizeof(__half);
     return WT_HEADER_BYTES + (bytes + WS_ALIGN - 1) / WS_ALIGN * WS_ALIGN;   // header + U
@@ -1301,11 +1317,12 @@ size_t sdwino_filter_bytes(int K, int C, int tile) {
 
 int sdwino_filter_transform(const void* w, void* wT, int K, int C, int tile, void* stream) {
     if (!w || !wT || K <= 0 || C <= 0) return SDWINO_ERR_INVALID_ARG;
-    if (tile != 2 && tile != 4) return SDWINO_ERR_UNSUPPORTED;
+    if (tile != 1 && tile != 2 && tile != 4) return SDWINO_ERR_UNSUPPORTED;
     if (!aligned(w, 2) || !aligned(wT, WS_ALIGN)) return SDWINO_ERR_MISALIGNED;
     if (static_cast<long double>(K) * C > 4.0e15L) return SDWINO_ERR_INVALID_ARG;
     const int Kb = (K + 15) / 16, Cb = (C + 63) / 64;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (tile == 1) return launch_filter<1>(static_cast<const __half*>(w), wT, K, C, Kb, Cb, st);
     if (tile == 2) return launch_filter<2>(static_cast<const __half*>(w), wT, K, C, Kb, Cb, st);
     return launch_filter<4>(static_cast<const __half*>(w), wT, K, C, Kb, Cb, st);
 }
@@ -1341,6 +1358,20 @@ int sdwino_conv3x3_q8(const void* x, const void* wTq, const void* bias, void* y,
                       int tile, void* workspace, size_t workspace_bytes, void* stream) {
     return conv_impl(x, wTq, bias, y, N, C, H, W, K, tile, workspace, workspace_bytes, static_cast<cudaStream_t>(stream),
                      Epilogue{nullptr, 0, nullptr}, false, false, true);
+}
+
+size_t sdwino_workspace_bytes_direct(int N, int C, int H, int W, int K, int stride) {
+    Plan pl;
+    if (stride < 1 || !make_plan(N, C, H, W, K, 1, &pl, stride)) return 0;
+    const long long pc = tiles_per_pass(pl, static_cast<size_t>(-1) / 2);
+    return static_cast<size_t>(pc) * pl.per_tile + WS_ALIGN;
+}
+
+int sdwino_conv3x3_direct(const void* x, const void* wT, const void* bias, void* y, int N, int C, int H, int W, int K,
+                          int stride, void* workspace, size_t workspace_bytes, void* stream) {
+    if (stride < 1) return SDWINO_ERR_INVALID_ARG;
+    return conv_impl(x, wT, bias, y, N, C, H, W, K, 1, workspace, workspace_bytes, static_cast<cudaStream_t>(stream),
+                     Epilogue{nullptr, 0, nullptr}, false, false, false, stride);
 }
 
 int sdwino_filter_transform_f32(const float* w, void* wT, int K, int C, int tile, void* stream) {

@@ -18,6 +18,24 @@ namespace sdw {
 
 template <int M> struct Wino;
 
+// F(1x1,3x3): the degenerate member of the family, i.e. the direct convolution.  A tile is one output pixel, the
+// nine transform positions are the nine filter taps, all three matrices are trivial (identity, identity, a row of
+// ones): the same three steps then compute y = sum over taps of (per-tap GEMM over the channels), which is the
+// convolution evaluated as nine shifted matrix products.  It also takes a stride (the input window of output pixel
+// t starts at stride * t - 1), which Winograd's overlapping tiles cannot.
+template <> struct Wino<1> {
+    static constexpr int A = 3;
+    struct Bt {
+        __host__ __device__ constexpr float operator()(int i, int j) const { return i == j ? 1.f : 0.f; }
+    };
+    struct G {
+        __host__ __device__ constexpr float operator()(int i, int j) const { return i == j ? 1.f : 0.f; }
+    };
+    struct At {
+        __host__ __device__ constexpr float operator()(int, int) const { return 1.f; }
+    };
+};
+
 template <> struct Wino<2> {
     static constexpr int A = 4;
     struct Bt {
@@ -311,9 +329,10 @@ struct TileGeom {
     int H, W, TH, TW;
     long long P;  // N*TH*TW, below 2^31
     FastDiv tw_div, th_div;
+    int stride;   // direct convolution (tile 1) only: distance of the input windows of neighbouring output pixels
 };
-inline TileGeom make_geom(int H, int W, int TH, int TW, long long P) {
-    return TileGeom{H, W, TH, TW, P, make_fastdiv(static_cast<uint32_t>(TW)), make_fastdiv(static_cast<uint32_t>(TH))};
+inline TileGeom make_geom(int H, int W, int TH, int TW, long long P, int stride = 1) {
+    return TileGeom{H, W, TH, TW, P, make_fastdiv(static_cast<uint32_t>(TW)), make_fastdiv(static_cast<uint32_t>(TH)), stride};
 }
 // tile p -> image n, tile row th, tile column tw
 __device__ __forceinline__ void decode_tile(const TileGeom& geo, long long p, long long& n, int& th, int& tw) {
@@ -350,7 +369,8 @@ input_transform_kernel(const XT* __restrict__ x, __half* __restrict__ V, TileGeo
         long long n;
         decode_tile(geo, p, n, th, tw);
         const XT* img = x + (n * C + c) * static_cast<long long>(geo.H) * geo.W;
-        const int i0 = M * th - 1, j0 = M * tw - 1;
+        const int step = M == 1 ? geo.stride : M;          // distance of neighbouring windows
+        const int i0 = step * th - 1, j0 = step * tw - 1;
 #pragma unroll
         for (int r = 0; r < A; ++r) {
             const int i = i0 + r;
@@ -471,6 +491,11 @@ output_transform_kernel(const __half* __restrict__ Mws, const YT* __restrict__ b
         } else {
         __half* rowp = img + static_cast<long long>(oi) * geo.W + j0;
         const __half* resp = ep.residual ? static_cast<const __half*>(ep.residual) + (rowp - y) : nullptr;
+        if constexpr (M == 1) {   // one output pixel per tile
+            float v0 = o[0] + b;
+            if (resp) v0 += __half2float(resp[0]);
+            rowp[0] = __float2half_rn(epilogue_act(v0, ep.act));
+        } else {
 #pragma unroll
         for (int j = 0; j < M; j += 2) {
             float v0 = o[j] + b, v1 = o[j + 1] + b;
@@ -486,6 +511,7 @@ output_transform_kernel(const __half* __restrict__ Mws, const YT* __restrict__ b
                 if (j0 + j + 1 < geo.W) rowp[j + 1] = h1;
             }
         }
+        }   // M > 1
         }   // fp16 output
     }
 }
