@@ -43,7 +43,7 @@ def metric_name(workload: str) -> str:
 
 
 UNIT = "TFLOP/s"
-TILE = "auto"   # per layer: what sdwino_choose_tile returns; --tile 2 / --tile 4 force one algorithm
+TILE = "auto"   # per layer: what sdwino_choose_algorithm returns; --tile 1 / 2 / 4 force one algorithm
 L2_BYTES = 126e6
 SUSTAINED_SECONDS = 2.2
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
@@ -293,8 +293,10 @@ def bench_workload(ctx, args, workload: str, headline: bool):
         torch.cuda.synchronize()
 
     layers = select_layers(workload, args.layers)
-    tiles = [B.sdwino_choose_tile(L.N, L.C, L.H, L.W, L.K) if args.tile == "auto" else int(args.tile) for L in layers]
+    tiles = [B.sdwino_choose_algorithm(L.N, L.C, L.H, L.W, L.K) if args.tile == "auto" else int(args.tile) for L in layers]
     io32 = args.io == "f32"       # the fp32 interface: x, w, bias, y in fp32
+    if io32 or args.weights == "q8":   # those interfaces have no direct form
+        tiles = [B.sdwino_choose_tile(L.N, L.C, L.H, L.W, L.K) if t == 1 else t for L, t in zip(layers, tiles)]
     io_bytes = 4.0 if io32 else 2.0
     io_t = torch.float32 if io32 else torch.float16
 
@@ -740,7 +742,7 @@ def run_ours(args):
             "data": "synthetic",
             "config": {"workload": head, "io": args.io, "layers": h["layers_n"], "layer_subset": args.layers or "all",
                        "batch": h["batch"], "tile": args.tile, "tile_per_layer": h["tile_per_layer"],
-                       "algorithm": ("Winograd F(2x2,3x3) or F(4x4,3x3) per layer (sdwino_choose_tile)"
+                       "algorithm": ("Winograd F(2x2,3x3) or F(4x4,3x3), or the direct form F(1x1,3x3), per layer (sdwino_choose_algorithm)"
                                      if args.tile == "auto" else f"Winograd F({args.tile}x{args.tile},3x3)") +
                                     (", fp32 x / w / bias / y, fp16 transformed operands, fp32 accumulate"
                                      if io32 else ", fp16 storage, fp32 accumulate"),
@@ -781,7 +783,7 @@ def main():
     ap.add_argument("--workload", default="all", choices=["all"] + ALL_WORKLOADS,
                     help="all: every workload, the headline on sdxl_1024; a name: that workload alone")
     ap.add_argument("--layers", default="", help="comma-separated layer indices of the workload (default: all)")
-    ap.add_argument("--tile", default=TILE, choices=["auto", "2", "4"])
+    ap.add_argument("--tile", default=TILE, choices=["auto", "1", "2", "4"])
     ap.add_argument("--io", default="f16", choices=["f16", "f32"],
                     help="element type of x, w, bias and y: f32 runs the fp32 interface (fp16 operands, fp32 accumulation)")
     ap.add_argument("--epilogue", default="none", choices=["none", "residual", "residual_silu"],

@@ -319,6 +319,11 @@ int sdwino_set_input_staging(int mode);
  * sdwino_filter_transform and sdwino_conv3x3.
  */
 int sdwino_choose_tile(int N, int C, int H, int W, int K);
+/* The same choice with the direct form (tile 1, stride 1: see sdwino_conv3x3_direct) among the candidates: returns 1,
+ * 2 or 4 (0 for invalid sizes).  The fp16 entries that take a workspace, a registered workspace, the built-in scratch
+ * or host buffers accept tile 1 and then run the direct convolution with stride 1; the fp32 and 8-bit entries do not
+ * (SDWINO_ERR_UNSUPPORTED). */
+int sdwino_choose_algorithm(int N, int C, int H, int W, int K);
 
 /*
  * Tuning and test knob.  F(2x2,3x3) layers with at most 8 output channels (the 320 -> 4 and 128 -> 3

@@ -26,7 +26,7 @@ EXPORTS = [
     "sdwino_filter_transform_f32", "sdwino_conv3x3_f32", "sdwino_conv3x3_f32_ex",
     "sdwino_host_staging_bytes_f32", "sdwino_conv3x3_host_f32", "sdwino_conv3x3_host_f32_async", "sdwino_set_pipeline",
     "sdwino_conv3x3_f32_scaled", "sdwino_filter_q8_bytes", "sdwino_filter_quantize", "sdwino_conv3x3_q8",
-    "sdwino_workspace_bytes_direct", "sdwino_conv3x3_direct",
+    "sdwino_workspace_bytes_direct", "sdwino_conv3x3_direct", "sdwino_choose_algorithm",
 ]
 
 KERNEL_KINDS = ("filter_transform", "input_transform", "wino_gemm", "output_transform", "fused", "layer")
@@ -96,6 +96,8 @@ def _load() -> ctypes.CDLL:
     lib.sdwino_selftest_wait_timeout.argtypes = [ctypes.c_ulonglong, vp]
     lib.sdwino_choose_tile.restype = i
     lib.sdwino_choose_tile.argtypes = [i, i, i, i, i]
+    lib.sdwino_choose_algorithm.restype = i
+    lib.sdwino_choose_algorithm.argtypes = [i, i, i, i, i]
     lib.sdwino_set_fused_min_tiles.restype = i
     lib.sdwino_set_fused_min_tiles.argtypes = [ctypes.c_longlong]
     lib.sdwino_filter_q8_bytes.restype = sz
@@ -190,6 +192,14 @@ def sdwino_choose_tile(N: int, C: int, H: int, W: int, K: int) -> int:
     return t
 
 
+def sdwino_choose_algorithm(N: int, C: int, H: int, W: int, K: int) -> int:
+    """1, 2 or 4: direct convolution, F(2x2) or F(4x4), whichever is expected to be fastest for this layer."""
+    t = int(lib.sdwino_choose_algorithm(N, C, H, W, K))
+    if t not in (1, 2, 4):
+        raise SdwinoError(ERR_INVALID_ARG, "sdwino_choose_algorithm")
+    return t
+
+
 def sdwino_set_fused_min_tiles(p_tiles: int = 0) -> None:
     """Blocks of 128 tiles from which few-output-channel layers take the single fused kernel; 0 = default."""
     _check(lib.sdwino_set_fused_min_tiles(p_tiles), "sdwino_set_fused_min_tiles")
@@ -241,7 +251,7 @@ def sdwino_filter_transform(w: torch.Tensor, tile: int, stream=None) -> torch.Te
     assert tuple(w.shape[2:]) == (3, 3)
     nbytes = sdwino_filter_bytes(K, C, tile)
     if nbytes == 0:
-        raise SdwinoError(ERR_UNSUPPORTED if tile not in (2, 4) else ERR_INVALID_ARG, "sdwino_filter_bytes")
+        raise SdwinoError(ERR_UNSUPPORTED if tile not in (1, 2, 4) else ERR_INVALID_ARG, "sdwino_filter_bytes")
     wT = alloc_workspace(nbytes, w.device)
     _check(lib.sdwino_filter_transform(w.data_ptr(), wT.data_ptr(), K, C, tile, _stream_ptr(stream)),
            "sdwino_filter_transform")
@@ -311,7 +321,7 @@ def sdwino_filter_transform_f32(w: torch.Tensor, tile: int, stream=None) -> torc
     assert tuple(w.shape[2:]) == (3, 3)
     nbytes = sdwino_filter_bytes(K, C, tile)
     if nbytes == 0:
-        raise SdwinoError(ERR_UNSUPPORTED if tile not in (2, 4) else ERR_INVALID_ARG, "sdwino_filter_bytes")
+        raise SdwinoError(ERR_UNSUPPORTED if tile not in (1, 2, 4) else ERR_INVALID_ARG, "sdwino_filter_bytes")
     wT = alloc_workspace(nbytes, w.device)
     _check(lib.sdwino_filter_transform_f32(w.data_ptr(), wT.data_ptr(), K, C, tile, _stream_ptr(stream)),
            "sdwino_filter_transform_f32")

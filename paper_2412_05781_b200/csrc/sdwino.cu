@@ -121,6 +121,7 @@ struct Plan {
 // tile 2 / 4: Winograd; tile 1 with stride >= 1: the direct convolution (a tile is one output pixel)
 bool make_plan(int N, int C, int H, int W, int K, int tile, Plan* pl, int stride = 0) {
     if (N <= 0 || C <= 0 || H <= 0 || W <= 0 || K <= 0) return false;
+    if (tile == 1 && stride == 0) stride = 1;      // tile 1 through the ordinary entries: the direct convolution, stride 1
     if (stride > 0 ? (tile != 1 || stride > 2) : (tile != 2 && tile != 4)) return false;
     const int a = tile + 2;
     pl->a2 = a * a;
@@ -1000,6 +1001,7 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
               bool io32 = false, bool range_safe = false, bool q8 = false, int stride = 0) {
     // io32: x, bias and y are fp32 (the filters come from the fp32 filter transform); stride > 0: the direct
     // convolution (tile 1, fp16 interface), whose tiles are single output pixels
+    if (tile == 1 && stride == 0) stride = 1;
     if (stride > 0 ? (tile != 1 || stride > 2 || io32 || q8) : (tile != 2 && tile != 4)) {
         return (N <= 0 || C <= 0 || H <= 0 || W <= 0 || K <= 0 || !x || !wT || !y) ? SDWINO_ERR_INVALID_ARG
                                                                                      : SDWINO_ERR_UNSUPPORTED;
@@ -1289,6 +1291,16 @@ int sdwino_choose_tile(int N, int C, int H, int W, int K) {
     return (20 * act >= 13 * wgt && P2 >= 256) ? 4 : 2;
 }
 
+int sdwino_choose_algorithm(int N, int C, int H, int W, int K) {
+    if (N <= 0 || C <= 0 || H <= 0 || W <= 0 || K <= 0) return 0;
+    // Layers whose whole batch is at most one block of 128 output pixels (the 8x8 layers of the UNet at batch 2):
+    // F(2x2) would fill a quarter of its block of 128 tiles and stream 16 values per weight, the direct form fills
+    // its block and streams 9.  Measured: 1280->1280 at 8x8, batch 2: 22.5 against 26.6 us, 2560->1280: 32.8 against
+    // 36.9 us; from two blocks of pixels on (12x12, 16x16) the direct form re-reads the filters per block and loses.
+    if (C > 8 && K > 8 && static_cast<long long>(N) * H * W <= GEMM_BLOCK_P) return 1;
+    return sdwino_choose_tile(N, C, H, W, K);
+}
+
 int sdwino_set_fused_min_tiles(long long p_tiles) {
     if (p_tiles < 0) return SDWINO_ERR_INVALID_ARG;
     g_fk_min_p_tiles = p_tiles == 0 ? FK_MIN_P_TILES : p_tiles;
@@ -1520,7 +1532,7 @@ namespace {
 int host_async_impl(const void* x_host, const void* wT, const void* bias_host, void* y_host, int N, int C,
                     int H, int W, int K, int tile, void* workspace, size_t workspace_bytes, void* stream, bool io32) {
     if (!x_host || !y_host || !wT) return SDWINO_ERR_INVALID_ARG;
-    if (tile != 2 && tile != 4) return SDWINO_ERR_UNSUPPORTED;
+    if (tile != 2 && tile != 4 && !(tile == 1 && !io32)) return SDWINO_ERR_UNSUPPORTED;
     const size_t elem = io32 ? sizeof(float) : sizeof(__half);
     const size_t staging = host_staging_bytes(N, C, H, W, K, tile, elem);
     if (staging == 0) return SDWINO_ERR_INVALID_ARG;
@@ -1685,7 +1697,7 @@ extern "C" {
 
 int sdwino_conv3x3_static(const void* x, const void* wT, const void* bias, void* y, int N, int C, int H, int W,
                           int K, int tile, void* stream) {
-    if (tile != 2 && tile != 4) {
+    if (tile != 1 && tile != 2 && tile != 4) {
         return (N <= 0 || C <= 0 || H <= 0 || W <= 0 || K <= 0 || !x || !wT || !y) ? SDWINO_ERR_INVALID_ARG
                                                                                      : SDWINO_ERR_UNSUPPORTED;
     }
