@@ -768,24 +768,37 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
                 __half* dst = reinterpret_cast<__half*>(stg) + quarter * 32 + lane;
                 // 8-bit filters: the factor of every output channel of this position (rows past K read padding)
                 [[maybe_unused]] const float* sc = U8 ? prm.scales + static_cast<long long>(pos) * prm.kpad + k0 + row0 : nullptr;
+                // (the scales of 16 or 32 columns are fetched as 16-byte vectors ahead of the accumulator load: one
+                // scalar load per column cost 6 us on a 25 us GEMM; kpad is a multiple of 16, so a vector is in or out)
+                auto load_scales = [&](int col, int n4, float4 (&s4)[8]) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        s4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (i < n4 && k0 + row0 + col + 4 * i < prm.kpad) s4[i] = __ldg(reinterpret_cast<const float4*>(sc + col) + i);
+                    }
+                };
                 int col = 0;
                 for (; col + 32 <= prm.epi_rows; col += 32) {
+                    [[maybe_unused]] float4 s4[8];
+                    if constexpr (U8) load_scales(col, 8, s4);
                     uint32_t r[32];
                     tmem_ld_32x32_sync(t_addr + row0 + col, r);
 #pragma unroll
                     for (int i = 0; i < 32; ++i) {
                         float v = __uint_as_float(r[i]);
-                        if constexpr (U8) v *= (k0 + row0 + col + i < prm.kpad) ? __ldg(sc + col + i) : 0.f;
+                        if constexpr (U8) v *= reinterpret_cast<const float*>(s4)[i];
                         dst[(col + i) * GEMM_BLOCK_P] = __float2half_rn(v);
                     }
                 }
                 if (col < prm.epi_rows) {
+                    [[maybe_unused]] float4 s4[8];
+                    if constexpr (U8) load_scales(col, 4, s4);
                     uint32_t r[16];
                     tmem_ld_32x16_sync(t_addr + row0 + col, r);
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
                         float v = __uint_as_float(r[i]);
-                        if constexpr (U8) v *= (k0 + row0 + col + i < prm.kpad) ? __ldg(sc + col + i) : 0.f;
+                        if constexpr (U8) v *= reinterpret_cast<const float*>(s4)[i];
                         dst[(col + i) * GEMM_BLOCK_P] = __float2half_rn(v);
                     }
                 }
