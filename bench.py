@@ -514,7 +514,7 @@ def bench_workload(ctx, args, workload: str, headline: bool):
         return nbytes / (ms * 1e-3) / 1e9 if ms > 0 else 0.0
 
     layer_rows = []
-    gemm_flops = gemm_ms = gemm_u_bytes = 0.0
+    gemm_flops = gemm_ms = gemm_u_bytes = gemm_io_bytes = 0.0
     in_ms = out_ms = in_bytes = out_bytes = fused_ms = 0.0
     for L, t, pl, lms, q in zip(layers, tiles, per_layer, layer_ms, q8):
         a2 = (t + 2) ** 2
@@ -541,6 +541,7 @@ def bench_workload(ctx, args, workload: str, headline: bool):
         if pl["wino_gemm"] > 0:                  # layers on a single-kernel path have no GEMM launch
             gemm_flops += wino_flops
             gemm_u_bytes += u_bytes
+            gemm_io_bytes += u_bytes + 2.0 * a2 * (L.C + L.K) * P      # what the unfused GEMM must move: U, V in, M out
             gemm_ms += k_gemm
             in_ms += k_in
             out_ms += k_out
@@ -570,6 +571,12 @@ def bench_workload(ctx, args, workload: str, headline: bool):
         "bound": "hbm", "algorithmic_bytes_per_step": gemm_u_bytes,
         "achieved": round(gbs(gemm_u_bytes, gemm_ms), 1), "peak": hpeak, "unit": "GB/s",
         "frac": round(gbs(gemm_u_bytes, gemm_ms) / hpeak, 4)}
+    # ... and against the bytes the GEMM kernel itself must move in the three-kernel design (U, V in, M out): on the
+    # large layers this, not the tensor pipe, is what bounds the launch (V and M do not fit in L2)
+    roofline["operand_stream_view"] = {
+        "bound": "hbm", "bytes_per_step": gemm_io_bytes, "achieved": round(gbs(gemm_io_bytes, gemm_ms), 1), "peak": hpeak,
+        "unit": "GB/s", "frac": round(gbs(gemm_io_bytes, gemm_ms) / hpeak, 4),
+        "note": "U + V + M of the GEMM launches over their time; an L2 hit counts like a DRAM access, so small layers can exceed 1"}
     # the whole step against the per-layer roofline max(tensor time, mandatory HBM bytes / bandwidth), both at
     # the measured peaks: what an ideal implementation of each layer would need, summed over the sweep
     roof_us_sum = sum(r["roof_us"] for r in layer_rows)
