@@ -54,6 +54,24 @@ def test_size_queries(binding):
     assert binding.sdwino_workspace_bytes(1, 0, 1, 1, 1, 2) == 0
     # two slots of x, bias and y, each rounded up to 1 KB
     assert binding.sdwino_host_staging_bytes(1, 4, 8, 8, 4, 2) == 1024 * 6
+    assert binding.sdwino_host_staging_bytes_f32(1, 4, 8, 8, 4, 2) == 1024 * 2 * (1 + 1 + 1)
+    assert binding.sdwino_host_staging_bytes_f32(1, 64, 8, 8, 64, 2) == 2 * (16384 + 1024 + 16384)
+    # the direct form: tile 1 = nine taps as positions; a tile is an output pixel, so stride 2 quarters the workspace
+    assert binding.sdwino_filter_bytes(320, 320, 1) == 1024 + 9 * 20 * 5 * 1024 * 2
+    assert binding.sdwino_workspace_bytes(2, 320, 64, 64, 320, 1) == 2 * 64 * 64 * 9 * 640 * 2 + 1024
+    assert binding.sdwino_workspace_bytes_direct(2, 320, 64, 64, 320, 1) == 2 * 64 * 64 * 9 * 640 * 2 + 1024
+    assert binding.sdwino_workspace_bytes_direct(2, 320, 64, 64, 320, 2) == 2 * 32 * 32 * 9 * 640 * 2 + 1024
+    assert binding.sdwino_workspace_bytes_direct(1, 4, 7, 9, 4, 2) == 128 * 9 * 8 * 2 + 1024      # 4 x 5 pixels -> one block
+    assert binding.sdwino_workspace_bytes_direct(1, 4, 8, 8, 4, 3) == 0
+    # 8-bit filters: header, one byte per element of the blocked layout, one fp32 scale per (position, padded k)
+    assert binding.sdwino_filter_q8_bytes(320, 320, 2) == 1024 + 16 * 20 * 5 * 1024 + 16 * 320 * 4
+    assert binding.sdwino_filter_q8_bytes(3, 4, 4) == 1024 + 36 * 1024 + 3072      # 36 * 16 * 4 = 2304 -> 3 KB
+    assert binding.sdwino_filter_q8_bytes(3, 4, 1) == 0
+    # the algorithm choice with the direct form among the candidates
+    assert binding.sdwino_choose_algorithm(2, 1280, 8, 8, 1280) == 1          # 128 output pixels: one block
+    assert binding.sdwino_choose_algorithm(2, 2560, 16, 16, 1280) == 2
+    assert binding.sdwino_choose_algorithm(2, 4, 8, 8, 320) == 2              # few input channels: the fused F(2x2) kernel
+    assert binding.sdwino_choose_algorithm(1, 512, 256, 256, 512) == 4
 
 
 def test_argument_validation_without_gpu(binding):
@@ -95,6 +113,28 @@ def test_argument_validation_without_gpu(binding):
     assert lib.sdwino_conv3x3_f32_ex(p, p, None, None, p, 1, 4, 8, 8, 4, 2, 7, p, 1 << 20, None) == binding.ERR_UNSUPPORTED
     assert lib.sdwino_conv3x3_f32_ex(p, p, None, p + 2, p, 1, 4, 8, 8, 4, 2, 1, p, 1 << 20, None) == binding.ERR_MISALIGNED
     assert lib.sdwino_conv3x3_f32_ex(None, p, None, None, p, 1, 4, 8, 8, 4, 2, 1, p, 1 << 20, None) == binding.ERR_INVALID_ARG
+    # the later entry points: range-safe fp32, fp32 host buffers, 8-bit filters, the direct form, the pipeline hook
+    assert lib.sdwino_conv3x3_f32_scaled(None, p, None, p, 1, 4, 8, 8, 4, 2, p, 1 << 20, None) == binding.ERR_INVALID_ARG
+    assert lib.sdwino_conv3x3_f32_scaled(p, p, None, p, 1, 4, 8, 8, 4, 5, p, 1 << 20, None) == binding.ERR_UNSUPPORTED
+    assert lib.sdwino_conv3x3_f32_scaled(p, p, None, p, 1, 4, 8, 8, 4, 2, None, 0, None) == binding.ERR_WORKSPACE
+    assert lib.sdwino_conv3x3_host_f32(None, p, None, p, 1, 4, 8, 8, 4, 2, p, 1 << 20, None) == binding.ERR_INVALID_ARG
+    assert lib.sdwino_conv3x3_host_f32(p, p, None, p, 1, 4, 8, 8, 4, 1, p, 1 << 20, None) == binding.ERR_UNSUPPORTED
+    assert lib.sdwino_conv3x3_host_f32(p, p, None, p, 1, 4, 8, 8, 4, 2, p, 1024, None) == binding.ERR_WORKSPACE
+    assert lib.sdwino_filter_quantize(None, p, 4, 4, 2, None) == binding.ERR_INVALID_ARG
+    assert lib.sdwino_filter_quantize(p, p, 4, 4, 3, None) == binding.ERR_UNSUPPORTED
+    assert lib.sdwino_filter_quantize(p, p + 16, 4, 4, 2, None) == binding.ERR_MISALIGNED
+    assert lib.sdwino_conv3x3_q8(None, p, None, p, 1, 4, 8, 8, 4, 2, p, 1 << 20, None) == binding.ERR_INVALID_ARG
+    assert lib.sdwino_conv3x3_q8(p, p, None, p, 1, 4, 8, 8, 4, 1, p, 1 << 20, None) == binding.ERR_UNSUPPORTED   # no direct form in 8 bits
+    assert lib.sdwino_conv3x3_q8(p, p, None, p, 1, 4, 8, 8, 4, 2, None, 0, None) == binding.ERR_WORKSPACE
+    assert lib.sdwino_conv3x3_direct(None, p, None, p, 1, 4, 8, 8, 4, 1, p, 1 << 20, None) == binding.ERR_INVALID_ARG
+    assert lib.sdwino_conv3x3_direct(p, p, None, p, 1, 4, 8, 8, 4, 0, p, 1 << 20, None) == binding.ERR_INVALID_ARG
+    assert lib.sdwino_conv3x3_direct(p, p, None, p, 1, 4, 8, 8, 4, 3, p, 1 << 20, None) == binding.ERR_UNSUPPORTED
+    assert lib.sdwino_conv3x3_direct(p, p, None, p, 1, 4, 8, 8, 4, 2, None, 0, None) == binding.ERR_WORKSPACE
+    assert lib.sdwino_conv3x3_f32(p, p, None, p, 1, 4, 8, 8, 4, 1, p, 1 << 20, None) == binding.ERR_UNSUPPORTED      # tile 1: fp16 entries only
+    assert lib.sdwino_set_pipeline(3, 0, 0) == binding.ERR_INVALID_ARG
+    assert lib.sdwino_set_pipeline(1, -1, 0) == binding.ERR_INVALID_ARG
+    assert lib.sdwino_set_pipeline(1, 0, 0) == binding.OK
+    assert lib.sdwino_profile_enable(3) == binding.ERR_INVALID_ARG and lib.sdwino_profile_enable(0) == binding.OK
     # test hooks reject values outside their range and accept the defaults
     assert lib.sdwino_set_input_staging(3) == binding.ERR_INVALID_ARG
     assert lib.sdwino_set_input_staging(-1) == binding.ERR_INVALID_ARG
