@@ -364,7 +364,16 @@ def bench_workload(ctx, args, workload: str, headline: bool):
         else:
             B.sdwino_conv3x3_ex(xd, wT, bd, res_dev[li], L.K, t, act, ws, y=yd, stream=strm)
 
+    # --sequence: the whole step is ONE call of the multi-layer entry (same kernels in the same order; with
+    # --prefetch-mb > 0 each layer's filters are sent towards L2 while the layer before it computes)
+    use_sequence = args.sequence and not io32 and args.epilogue == "none" and not any(q8)
+    if use_sequence:
+        seq = B.make_sequence([(xd, wT, bd, yd, L.K, t) for L, t, (xd, wT, bd, yd) in zip(layers, tiles, devt)])
+
     def step():
+        if use_sequence:
+            B.sdwino_conv3x3_sequence(seq, ws, args.prefetch_mb << 20, stream=torch.cuda.current_stream())
+            return
         for li in range(len(layers)):
             run_layer(li, torch.cuda.current_stream())
 
@@ -777,6 +786,8 @@ def run_ours(args):
                        "launch": "direct" if args.no_graph else "CUDA graph of one step, replayed",
                        "weights": args.weights,
                        "pipeline": {0: "off", 1: "where the library takes it", 2: "wherever possible"}[args.pipeline],
+                       "step_call": (f"one sdwino_conv3x3_sequence call per step, {args.prefetch_mb} MB of filters prefetched per layer"
+                                     if args.sequence else "one sdwino_conv3x3 call per layer"),
                        "l2": h["l2"],
                        "filter_transform": "once per weight, before the timed region (reported separately)",
                        "epilogue": {"none": "bias", "residual": "bias + residual, fused, on the layers with more than 8 input and output channels (e2e runs the plain convolution)",
@@ -821,6 +832,10 @@ def main():
                     help="the pipelined single-launch path of F(4x4): 0 never, 1 where the library takes it, 2 wherever possible")
     ap.add_argument("--pipe-ring", type=int, default=0, help="ring length of the pipelined path in blocks of 128 tiles (0: library's choice)")
     ap.add_argument("--pipe-lead", type=int, default=0, help="lag of its output transform in blocks (0: library's choice)")
+    ap.add_argument("--sequence", action="store_true",
+                    help="run the step as one sdwino_conv3x3_sequence call (fp16 interface, no epilogue, fp16 filters)")
+    ap.add_argument("--prefetch-mb", type=int, default=0,
+                    help="with --sequence: MB of the next layer's filters prefetched into L2 per layer (0: none)")
     ap.add_argument("--no-graph", action="store_true", help="launch every step directly instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-yardstick", action="store_true")

@@ -199,6 +199,42 @@ int sdwino_conv3x3_direct(const void *x, const void *wT, const void *bias, void 
                           void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * Several layers in one call, optionally with each layer's filters travelling to L2 while the layer before it
+ * computes (Section "Techniques", second paragraph: a core that finishes its block is handed the next one at once;
+ * here the memory system can be handed the next layer's filters, the one operand of a layer that depends on nothing
+ * before it).
+ * Layers run in order on `stream`, each exactly as sdwino_conv3x3_ws would run it (same kernels, same bits), so layer
+ * i + 1 may read what layer i wrote.  With prefetch_bytes > 0, a small kernel on a stream of the library's own (lowest
+ * priority, ordered after everything that precedes layer i in `stream`) queues L2 prefetches for up to prefetch_bytes
+ * of layer i + 1's transformed filters, the same share of every transform position; it only issues the requests and
+ * ends, nothing waits for the data, and the side stream is joined back into `stream` before the call returns, so the
+ * call can be captured into a CUDA graph.  prefetch_bytes = 0 (the recommended value): no side stream, no extra
+ * launches.  Measured on the UNet sweeps the prefetch does not pay: the GEMM already sends its first ring of filter
+ * boxes out before it waits for the activation transform, its filter stream runs at the HBM rate once started, and
+ * the early requests take bandwidth from the running layer (a sweep is 1-25 % slower with 8-128 MB prefetched per
+ * layer), so the knob is there for other parts and other layer mixes, not as a default.
+ *   layers[i]: device pointers x, wT (sdwino_filter_transform for K, C, tile), bias (or NULL), y, all fp16, and the
+ *   sizes of the layer; tile 1, 2 or 4 (sdwino_choose_algorithm).  The array itself is host memory and is only read
+ *   during the call.  workspace: device, 1024-byte aligned, shared by the layers one after the other;
+ *   sdwino_workspace_bytes_sequence gives the size at which every layer runs in one pass (0 for an invalid list).
+ * Errors: every layer is validated before the first launch (SDWINO_ERR_INVALID_ARG / _UNSUPPORTED / _MISALIGNED /
+ * _WORKSPACE as for sdwino_conv3x3_ws), so a sequence is either enqueued whole or not at all, except for
+ * SDWINO_ERR_CUDA from a launch.  Calls with prefetch_bytes > 0 from several threads are serialised while they
+ * enqueue (they share the side stream).
+ */
+typedef struct sdwino_layer {
+    const void *x;       /* device fp16 [N][C][H][W] */
+    const void *wT;      /* device, transformed filters of this layer */
+    const void *bias;    /* device fp16 [K], or NULL */
+    void *y;             /* device fp16 [N][K][H][W] */
+    int N, C, H, W, K;
+    int tile;            /* 1, 2 or 4 */
+} sdwino_layer;
+size_t sdwino_workspace_bytes_sequence(const sdwino_layer *layers, int n);
+int sdwino_conv3x3_sequence(const sdwino_layer *layers, int n, void *workspace, size_t workspace_bytes,
+                            size_t prefetch_bytes, void *stream);
+
+/*
  * The convolution for callers that must not allocate device memory.  (The paper has no
  * counterpart; this entry point exists for the embedding of the library.)  Some callers cannot
  * call cudaMalloc or any allocator at all: code that runs inside a CUDA-graph capture or another

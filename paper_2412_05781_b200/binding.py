@@ -27,7 +27,14 @@ EXPORTS = [
     "sdwino_host_staging_bytes_f32", "sdwino_conv3x3_host_f32", "sdwino_conv3x3_host_f32_async", "sdwino_set_pipeline",
     "sdwino_conv3x3_f32_scaled", "sdwino_filter_q8_bytes", "sdwino_filter_quantize", "sdwino_conv3x3_q8",
     "sdwino_workspace_bytes_direct", "sdwino_conv3x3_direct", "sdwino_choose_algorithm",
+    "sdwino_workspace_bytes_sequence", "sdwino_conv3x3_sequence",
 ]
+
+class SdwinoLayer(ctypes.Structure):
+    """struct sdwino_layer of the C ABI."""
+    _fields_ = [("x", ctypes.c_void_p), ("wT", ctypes.c_void_p), ("bias", ctypes.c_void_p), ("y", ctypes.c_void_p),
+                ("N", ctypes.c_int), ("C", ctypes.c_int), ("H", ctypes.c_int), ("W", ctypes.c_int), ("K", ctypes.c_int),
+                ("tile", ctypes.c_int)]
 
 KERNEL_KINDS = ("filter_transform", "input_transform", "wino_gemm", "output_transform", "fused", "layer")
 
@@ -116,6 +123,10 @@ def _load() -> ctypes.CDLL:
     lib.sdwino_profile_enable.argtypes = [i]
     lib.sdwino_profile_collect.restype = i
     lib.sdwino_profile_collect.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_ulonglong)]
+    lib.sdwino_workspace_bytes_sequence.restype = sz
+    lib.sdwino_workspace_bytes_sequence.argtypes = [ctypes.POINTER(SdwinoLayer), i]
+    lib.sdwino_conv3x3_sequence.restype = i
+    lib.sdwino_conv3x3_sequence.argtypes = [ctypes.POINTER(SdwinoLayer), i, vp, sz, sz, vp]
     return lib
 
 
@@ -472,3 +483,28 @@ def sdwino_conv3x3_direct(x: torch.Tensor, wT: torch.Tensor, bias: Optional[torc
                                    workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream_ptr(stream))
     _check(rc, "sdwino_conv3x3_direct")
     return y
+
+
+def make_sequence(layers) -> "ctypes.Array":
+    """An array of struct sdwino_layer from (x, wT, bias or None, y, K, tile) tuples of CUDA tensors.  The tensors must
+    stay alive while the array is used; nothing is copied."""
+    arr = (SdwinoLayer * len(layers))()
+    for d, (x, wT, bias, y, K, tile) in zip(arr, layers):
+        assert x.is_cuda and x.dtype == torch.float16 and x.is_contiguous() and x.dim() == 4
+        N, C, H, W = (int(v) for v in x.shape)
+        assert y.is_cuda and y.dtype == torch.float16 and y.is_contiguous() and tuple(y.shape) == (N, K, H, W)
+        d.x, d.wT, d.bias, d.y = x.data_ptr(), wT.data_ptr(), _ptr(bias), y.data_ptr()
+        d.N, d.C, d.H, d.W, d.K, d.tile = N, C, H, W, K, tile
+    return arr
+
+
+def sdwino_workspace_bytes_sequence(seq) -> int:
+    return int(lib.sdwino_workspace_bytes_sequence(seq, len(seq)))
+
+
+def sdwino_conv3x3_sequence(seq, workspace: torch.Tensor, prefetch_bytes: int = 0, stream=None) -> None:
+    """Runs the layers of `seq` (see make_sequence) in order on `stream`; prefetch_bytes > 0 also sends that much of each
+    layer's filters towards L2 while the layer before it computes."""
+    rc = lib.sdwino_conv3x3_sequence(seq, len(seq), workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                                     prefetch_bytes, _stream_ptr(stream))
+    _check(rc, "sdwino_conv3x3_sequence")

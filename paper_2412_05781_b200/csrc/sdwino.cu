@@ -1727,6 +1727,128 @@ int sdwino_conv3x3_static(const void* x, const void* wT, const void* bias, void*
                      static_cast<cudaStream_t>(stream));
 }
 
+}  // extern "C"
+
+namespace {
+// Issues the L2 prefetches of the first `bytes_per_pos` bytes of every transform position of a filter tensor, the
+// positions advancing together (the GEMM's CTAs work on all positions at once, each through the channel blocks in
+// order).  Nothing waits for the prefetches: the kernel ends as soon as they are queued.
+constexpr uint32_t PREFETCH_CHUNK = 4096;
+__global__ void __launch_bounds__(128) filter_prefetch_kernel(const uint8_t* __restrict__ base, size_t pos_stride,
+                                                             size_t bytes_per_pos, int num_pos) {
+    const size_t chunks_per_pos = (bytes_per_pos + PREFETCH_CHUNK - 1) / PREFETCH_CHUNK;
+    const size_t total = chunks_per_pos * static_cast<size_t>(num_pos);
+    for (size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < total;
+         i += static_cast<size_t>(gridDim.x) * blockDim.x) {
+        const size_t j = i / num_pos;
+        const size_t pos = i - j * num_pos;
+        const size_t off = j * PREFETCH_CHUNK;
+        const size_t left = bytes_per_pos - off;
+        bulk_prefetch_l2(base + pos * pos_stride + off, static_cast<uint32_t>(left < PREFETCH_CHUNK ? left : PREFETCH_CHUNK));
+    }
+}
+
+// The side stream and the events of sdwino_conv3x3_sequence, one set per device, made on first use.
+struct SequenceResources {
+    cudaStream_t side = nullptr;
+    std::vector<cudaEvent_t> events;
+};
+SequenceResources g_seq[STATIC_MAX_DEVICES_HOST];
+std::mutex g_seq_mutex;
+
+bool layer_ok(const sdwino_layer& l) {
+    return l.x && l.wT && l.y && l.N > 0 && l.C > 0 && l.H > 0 && l.W > 0 && l.K > 0;
+}
+}  // namespace
+
+extern "C" {
+
+size_t sdwino_workspace_bytes_sequence(const sdwino_layer* layers, int n) {
+    if (!layers || n <= 0) return 0;
+    size_t need = 0;
+    for (int i = 0; i < n; ++i) {
+        const sdwino_layer& l = layers[i];
+        const size_t b = sdwino_workspace_bytes(l.N, l.C, l.H, l.W, l.K, l.tile);
+        if (b == 0) return 0;
+        need = std::max(need, b);
+    }
+    return need;
+}
+
+int sdwino_conv3x3_sequence(const sdwino_layer* layers, int n, void* workspace, size_t workspace_bytes,
+                            size_t prefetch_bytes, void* stream) {
+    if (!layers || n <= 0) return SDWINO_ERR_INVALID_ARG;
+    // everything is checked before the first launch: a sequence runs whole or not at all
+    for (int i = 0; i < n; ++i) {
+        const sdwino_layer& l = layers[i];
+        if (!layer_ok(l)) return SDWINO_ERR_INVALID_ARG;
+        if (l.tile != 1 && l.tile != 2 && l.tile != 4) return SDWINO_ERR_UNSUPPORTED;
+        Plan pl;
+        if (!make_plan(l.N, l.C, l.H, l.W, l.K, l.tile, &pl)) return SDWINO_ERR_INVALID_ARG;
+        if (!aligned(l.x, 2) || !aligned(l.y, 2) || (l.bias && !aligned(l.bias, 2)) || !aligned(l.wT, WS_ALIGN))
+            return SDWINO_ERR_MISALIGNED;
+        if (!workspace || tiles_per_pass(pl, workspace_bytes) < GEMM_BLOCK_P) return SDWINO_ERR_WORKSPACE;
+    }
+    if (!aligned(workspace, WS_ALIGN)) return SDWINO_ERR_MISALIGNED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool prefetch = prefetch_bytes >= PREFETCH_CHUNK && n > 1;
+    SequenceResources* res = nullptr;
+    std::unique_lock<std::mutex> lock(g_seq_mutex, std::defer_lock);
+    if (prefetch) {
+        // one sequence at a time enqueues through the side stream (the calls only enqueue; the work itself overlaps)
+        lock.lock();
+        const int dev = current_device();
+        if (dev < 0 || dev >= STATIC_MAX_DEVICES_HOST) return err_cuda(__LINE__);
+        res = &g_seq[dev];
+        if (!res->side) {
+            int lo = 0, hi = 0;
+            if (cudaDeviceGetStreamPriorityRange(&lo, &hi) != cudaSuccess) return err_cuda(__LINE__);
+            if (cudaStreamCreateWithPriority(&res->side, cudaStreamNonBlocking, lo) != cudaSuccess) return err_cuda(__LINE__);
+        }
+        while (static_cast<int>(res->events.size()) < n + 1) {
+            cudaEvent_t e;
+            if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return err_cuda(__LINE__);
+            res->events.push_back(e);
+        }
+    }
+    bool forked = false;
+    for (int i = 0; i < n; ++i) {
+        if (prefetch && i + 1 < n) {
+            // While layer i computes, the first bytes of every position of layer i + 1's filters travel to L2:
+            // filters never depend on activations.  The side stream waits for what precedes layer i in `stream`.
+            const sdwino_layer& nx = layers[i + 1];
+            const size_t a2 = static_cast<size_t>(nx.tile + 2) * (nx.tile + 2);
+            const size_t per_pos = static_cast<size_t>((nx.K + 15) / 16) * ((nx.C + 63) / 64) * 1024 * sizeof(__half);
+            size_t want = std::min(per_pos, prefetch_bytes / a2) / PREFETCH_CHUNK * PREFETCH_CHUNK;
+            if (want * a2 >= (1u << 20)) {     // small filters are not worth a launch
+                if (cudaEventRecord(res->events[i], st) != cudaSuccess) return err_cuda(__LINE__);
+                if (cudaStreamWaitEvent(res->side, res->events[i], 0) != cudaSuccess) return err_cuda(__LINE__);
+                const size_t chunks = want / PREFETCH_CHUNK * a2;
+                const unsigned blocks = static_cast<unsigned>(std::min<size_t>((chunks + 127) / 128, 64));
+                filter_prefetch_kernel<<<blocks, 128, 0, res->side>>>(static_cast<const uint8_t*>(wt_filters_of(nx.wT)), per_pos,
+                                                                      want, static_cast<int>(a2));
+                if (cudaGetLastError() != cudaSuccess) return err_cuda(__LINE__);
+                g_launches.fetch_add(1);
+                forked = true;
+            }
+        }
+        const sdwino_layer& l = layers[i];
+        const int rc = conv_impl(l.x, l.wT, l.bias, l.y, l.N, l.C, l.H, l.W, l.K, l.tile, workspace, workspace_bytes, st);
+        if (rc != SDWINO_OK) {
+            if (forked) {   // rejoin before reporting, so that a stream capture stays valid
+                if (cudaEventRecord(res->events[n], res->side) == cudaSuccess) cudaStreamWaitEvent(st, res->events[n], 0);
+            }
+            return rc;
+        }
+    }
+    if (forked) {
+        // the side stream joins `stream` again (a no-op in time: the prefetch kernels ended long ago)
+        if (cudaEventRecord(res->events[n], res->side) != cudaSuccess) return err_cuda(__LINE__);
+        if (cudaStreamWaitEvent(st, res->events[n], 0) != cudaSuccess) return err_cuda(__LINE__);
+    }
+    return SDWINO_OK;
+}
+
 int sdwino_profile_enable(int mode) {
     if (mode < 0 || mode > 2) return SDWINO_ERR_INVALID_ARG;
     g_profile.store(mode);

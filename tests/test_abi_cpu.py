@@ -142,6 +142,41 @@ def test_argument_validation_without_gpu(binding):
     assert lib.sdwino_set_gemm_shape(0, 0) == binding.OK
 
 
+def test_sequence_entry_validates_every_layer_before_anything_runs(binding):
+    lib, Layer = binding.lib, binding.SdwinoLayer
+    buf = ctypes.create_string_buffer(4096)
+    p = (ctypes.addressof(buf) + 1023) // 1024 * 1024
+
+    def seq(*specs):
+        arr = (Layer * len(specs))()
+        for d, (x, wT, bias, y, N, C, H, W, K, tile) in zip(arr, specs):
+            d.x, d.wT, d.bias, d.y, d.N, d.C, d.H, d.W, d.K, d.tile = x, wT, bias, y, N, C, H, W, K, tile
+        return arr
+
+    good = (p, p, None, p, 1, 4, 8, 8, 4, 2)
+    big = (p, p, None, p, 2, 320, 64, 64, 320, 4)
+    # workspace of a list = the largest single-pass workspace among its layers; an invalid member makes it 0
+    assert lib.sdwino_workspace_bytes_sequence(seq(good, big), 2) == binding.sdwino_workspace_bytes(2, 320, 64, 64, 320, 4)
+    assert lib.sdwino_workspace_bytes_sequence(seq(good), 1) == binding.sdwino_workspace_bytes(1, 4, 8, 8, 4, 2)
+    assert lib.sdwino_workspace_bytes_sequence(seq(good, (p, p, None, p, 1, 4, 8, 8, 4, 3)), 2) == 0
+    assert lib.sdwino_workspace_bytes_sequence(None, 1) == 0
+    assert lib.sdwino_workspace_bytes_sequence(seq(good), 0) == 0
+    call = lib.sdwino_conv3x3_sequence
+    assert call(None, 1, p, 1 << 20, 0, None) == binding.ERR_INVALID_ARG
+    assert call(seq(good), 0, p, 1 << 20, 0, None) == binding.ERR_INVALID_ARG
+    # a fault in the LAST layer is found before the first one is launched (no GPU here: a launch would be ERR_CUDA)
+    assert call(seq(good, (None, p, None, p, 1, 4, 8, 8, 4, 2)), 2, p, 1 << 20, 0, None) == binding.ERR_INVALID_ARG
+    assert call(seq(good, (p, p, None, p, 1, 4, 8, 0, 4, 2)), 2, p, 1 << 20, 0, None) == binding.ERR_INVALID_ARG
+    assert call(seq(good, (p, p, None, p, 1, 4, 8, 8, 4, 3)), 2, p, 1 << 20, 0, None) == binding.ERR_UNSUPPORTED
+    assert call(seq(good, (p, p, None, p + 1, 1, 4, 8, 8, 4, 2)), 2, p, 1 << 20, 0, None) == binding.ERR_MISALIGNED
+    assert call(seq(good, (p, p + 16, None, p, 1, 4, 8, 8, 4, 2)), 2, p, 1 << 20, 0, None) == binding.ERR_MISALIGNED
+    assert call(seq(good, good), 2, None, 0, 0, None) == binding.ERR_WORKSPACE
+    assert call(seq(good, good), 2, p, 4096, 0, None) == binding.ERR_WORKSPACE
+    assert call(seq(good, good), 2, p + 8, 1 << 20, 0, None) == binding.ERR_MISALIGNED
+    # the struct of the binding has the layout of the header: four pointers, six ints
+    assert ctypes.sizeof(Layer) == 4 * ctypes.sizeof(ctypes.c_void_p) + 6 * ctypes.sizeof(ctypes.c_int)
+
+
 def test_missing_library_fails_loudly(monkeypatch, binding):
     import importlib
     from paper_2412_05781_b200 import build as bmod
