@@ -802,7 +802,7 @@ int launch_gemm_shape(const CUtensorMap& tmU, const CUtensorMap& tmV, const CUte
     const int grid = static_cast<int>(tiles < workers ? tiles : workers) * CTAS;
     ProfScope prof(KIND_GEMM, st);
     const cudaError_t e =
-        launch_pdl(wino_gemm_kernel<CTAS, RES, DUAL, false, U8>, dim3(grid), dim3(GEMM_THREADS),
+        launch_pdl(wino_gemm_kernel<CTAS, RES, DUAL, false, U8>, dim3(grid), dim3(GEMM_LAUNCH_THREADS),
                    static_cast<size_t>(L::dyn_bytes(RES ? 0 : prm.n_tile / CTAS, prm.stages, prm.epi_rows,
                                                     prm.epi_alias ? 0 : prm.epi_bufs,
                                                     RES ? prm.num_c_blocks * L::b_bytes(prm.n_tile)

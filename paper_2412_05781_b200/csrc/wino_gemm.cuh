@@ -54,6 +54,7 @@ constexpr int GEMM_BLOCK_P = 128;  // tiles per output tile (TMEM lanes, UMMA M)
 constexpr int GEMM_BLOCK_C = 64;   // input channels per pipeline stage (one 128-byte swizzle row of U)
 constexpr int GEMM_MAX_N = 256;    // output channels per output tile (UMMA N), multiple of 16
 constexpr int GEMM_THREADS = 320;  // warp 0 producer, warp 1 MMA, warps 2-9 epilogue (two groups of four)
+constexpr int GEMM_LAUNCH_THREADS = GEMM_THREADS + 32;   // ... and warp 10: the second producer (filters) of the streaming kernel
 constexpr int PIPE_TRANSFORM_THREADS = 320;                            // pipelined mode: warps 10-19 run the transforms, each on its own
 constexpr int PIPE_THREADS = GEMM_THREADS + PIPE_TRANSFORM_THREADS;
 constexpr int GEMM_MAX_STAGES = 8;
@@ -191,7 +192,7 @@ __device__ __forceinline__ void signal_counter_release(unsigned int* ctr) {
 // still kind::f16.  Meant for the weight-streaming layers (one tile per CTA): with several tiles per CTA the epilogue
 // of one tile no longer overlaps the mainloop of the next.
 template <int CTAS, bool RES = false, bool DUAL = false, bool PIPE = false, bool U8 = false>
-__global__ void __launch_bounds__(PIPE ? PIPE_THREADS : GEMM_THREADS, 1)
+__global__ void __launch_bounds__(PIPE ? PIPE_THREADS : GEMM_LAUNCH_THREADS, 1)
 wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant__ CUtensorMap tmV,
                  const __grid_constant__ CUtensorMap tmM, const GemmParams prm, int* __restrict__ status_word,
                  const PipeParams pp) {
@@ -207,6 +208,9 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
     static_assert(!RES || CTAS == 1, "filter-resident mode is for single CTAs");
     static_assert(!DUAL || (CTAS == 1 && !RES), "two blocks of tiles per CTA: single CTAs, streaming mode");
     constexpr bool resident = RES;
+    // Two producers (single CTAs, streaming): a thread that issues TMA loads spends about 100 ns per load on its own
+    // instruction latencies, so the boxes of V (warp 0) and the filter boxes (warp 10) go out from two warps.
+    constexpr bool SPLIT = CTAS == 1 && !RES && !PIPE && !U8;
     constexpr int PT = DUAL ? 2 : 1;                 // blocks of 128 tiles p per CTA tile (one accumulator each)
     constexpr int a_bytes = PT * L::A_BYTES;         // V part of a stage
     const int stage_bytes = resident ? L::A_BYTES : (PT - 1) * L::A_BYTES + L::stage_bytes(b_rows);
@@ -283,7 +287,7 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) {
-            mbar_init(&full_bar[s], U8 ? 9 : 1);      // 8-bit filters: the producer and the eight converting warps
+            mbar_init(&full_bar[s], U8 ? 9 : (SPLIT ? 2 : 1));   // 8-bit filters: the producer and the eight converting warps
             mbar_init(&empty_bar[s], 1);
         }
         for (int s = 0; s < GEMM_MAX_STAGES; ++s) {
@@ -464,6 +468,32 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
             // (pipelined mode: the filters are read again for every block of tiles and must stay in L2)
             const uint64_t u_policy = PIPE ? l2_policy_evict_last() : l2_policy_evict_first();
             int pre = 0;
+            if constexpr (SPLIT) {
+                // the filters are the other producer's: this one brings the boxes of V
+                pdl_wait();   // V is written by the preceding kernel
+                int stage = 0;
+                uint32_t phase = 0;
+                bool ok = true;
+                for (int i = 0; i < my_count && ok; ++i) {
+                    int pt, kt, pos;
+                    decode(tile_of(i), pt, kt, pos);
+                    const int p0 = pt * PT * GEMM_BLOCK_P;
+                    for (int c0 = 0; c0 < prm.C; c0 += GEMM_BLOCK_C) {
+                        ok = mbar_wait_bounded(&empty_bar[stage], phase ^ 1u, abort_flag, GEMM_WAIT_LIMIT_NS);
+                        if (!ok) { if (*abort_flag == 0) report_timeout(status_word, 1, cta_rank); break; }
+                        mbar_arrive_expect_tx_a32(fb, static_cast<uint32_t>(a_bytes));
+#pragma unroll
+                        for (int sub = 0; sub < PT; ++sub) {
+                            tma_load_3d_a32(sa + sub * L::A_BYTES, &tmV, fb, p0 + sub * GEMM_BLOCK_P, c0, pos);
+                            tma_load_3d_a32(sa + sub * L::A_BYTES + L::A_BOX_BYTES, &tmV, fb, p0 + sub * GEMM_BLOCK_P + 64, c0, pos);
+                        }
+                        sa += stage_bytes;
+                        fb += 8;
+                        if (++stage == stages) { stage = 0; phase ^= 1u; sa = smem_base; fb = full0; }
+                    }
+                }
+                if (!ok) *abort_flag = 1;
+            } else {
             if constexpr (CTAS == 1) {
                 uint32_t sa_u = smem_base + a_bytes, fb_u = full0;
                 for (int i = 0; i < my_count && pre < stages; ++i) {
@@ -544,6 +574,7 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
                 }
             }
             if (!ok) *abort_flag = 1;
+            }   // !SPLIT
         }
     } else if (warp == 1) {
         // ------------------------------ MMA issuer ------------------------------
@@ -868,6 +899,36 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
                     signal_counter_release(&pp.m_done[pend_pt]);
                 }
             }
+        }
+    } else if constexpr (SPLIT) {
+        // ------------------------------ second producer: the filter boxes ------------------------------
+        // The filters depend on nothing before this launch (see the comment in the first producer), so this thread
+        // never waits for the preceding kernel: the first ring-full of boxes goes out at once, the rest as stages
+        // are released.
+        if (lane == 0) {
+            const uint32_t smem_base = smem_u32(smem);
+            const uint32_t full0 = smem_u32(&full_bar[0]);
+            const uint32_t u_bytes = static_cast<uint32_t>(L::b_bytes(b_rows));
+            const uint64_t u_policy = l2_policy_evict_first();
+            uint32_t sa = smem_base + a_bytes, fb = full0;
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int i = 0; i < my_count && ok; ++i) {
+                int pt, kt, pos;
+                decode(tile_of(i), pt, kt, pos);
+                const int k0 = kt * prm.n_tile;
+                for (int c0 = 0; c0 < prm.C; c0 += GEMM_BLOCK_C) {
+                    ok = mbar_wait_bounded(&empty_bar[stage], phase ^ 1u, abort_flag, GEMM_WAIT_LIMIT_NS);
+                    if (!ok) { if (*abort_flag == 0) report_timeout(status_word, 11, cta_rank); break; }
+                    mbar_arrive_expect_tx_a32(fb, u_bytes);
+                    tma_load_5d_hint_a32(sa, &tmU, fb, c0 >> 6, k0 >> 4, pos, u_policy);
+                    sa += stage_bytes;
+                    fb += 8;
+                    if (++stage == stages) { stage = 0; phase ^= 1u; sa = smem_base + a_bytes; fb = full0; }
+                }
+            }
+            if (!ok) *abort_flag = 1;
         }
     } else if constexpr (PIPE) {
         // ------------------------------ transforms (pipelined mode) ------------------------------
