@@ -1195,6 +1195,27 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
         }
     }
 
+    if (!prm.resident && !prm.epi_alias && !q8 && force_ctas == 0 && force_n_tile == 0) {
+        // The ring is short of stages against its round trip (a stage's loads take 2-3.5 thousand cycles to arrive
+        // under load, its MMAs 300-500): an epilogue group that stages its channels 64 or 32 at a time instead of all
+        // at once leaves room for one more stage in most shapes.  Measured: CTA pairs at n_tile 256 go from five to
+        // six stages, 1280->1280 at 64x64 (batch 2) 63.8 -> 58.3 us, 512->512 at 512x512 363 -> 345 us; 16 at a time
+        // costs more in the epilogue than the stage returns (320->320 at 128x128: 28 -> 35 us).
+        const int stage = GemmSmemLayout::stage_bytes(b_rows) + (shape.dual ? GemmSmemLayout::A_BYTES : 0);
+        auto stages_for = [&](int rows) {
+            const int st = (MAX_DYN_SMEM - GemmSmemLayout::dyn_bytes(b_rows, 0, rows, prm.epi_bufs)) / stage;
+            return st > GEMM_MAX_STAGES ? GEMM_MAX_STAGES : st;
+        };
+        const int grp = prm.epi_rows;
+        int best_rows = grp, best_stages = stages_for(grp);
+        for (int rows = 64; rows >= 32; rows >>= 1) {
+            if (rows >= grp || grp % rows != 0) continue;
+            if (stages_for(rows) > best_stages) { best_stages = stages_for(rows); best_rows = rows; }
+        }
+        prm.epi_chunks = grp / best_rows;
+        prm.epi_rows = best_rows;
+        prm.stages = best_stages;
+    }
     prm.p_stride = pc;
     CUtensorMap tmU, tmV, tmM;
     if (!(q8 ? encode_filter_map_q8(&tmU, wt_filters_of(wT), pl.Cb, pl.Kb, pl.a2, b_rows / 16)

@@ -786,7 +786,7 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
             // lane = tile p, registers = output channels: staging row k receives 32 consecutive p from
             // each warp (64 contiguous bytes, no bank conflict).  Group g owns staging buffer g.
             // a group drains its channels in epi_chunks pieces of epi_rows, one TMA store each
-            const int chunks = resident ? prm.epi_chunks : 1;
+            const int chunks = prm.epi_chunks;
             for (int ch = 0; ch < chunks; ++ch) {
             const int row0 = (group * chunks + ch) * prm.epi_rows;
             if (row0 < prm.n_tile) {
