@@ -926,6 +926,9 @@ int launch_pipeline(const __half* x, const void* wT, const __half* bias, __half*
     prm.n_tile = pq.n_tile;
     prm.num_k_tiles = (K + pq.n_tile - 1) / pq.n_tile;
     prm.num_p_tiles = pq.nb;
+    prm.fd_p = make_fastdiv(static_cast<uint32_t>(prm.num_p_tiles));
+    prm.fd_k = make_fastdiv(static_cast<uint32_t>(prm.num_k_tiles));
+    prm.fd_keys = make_fastdiv(static_cast<uint32_t>(prm.num_k_tiles * pl.a2));
     prm.num_pos = pl.a2;
     prm.num_c_blocks = (C + GEMM_BLOCK_C - 1) / GEMM_BLOCK_C;
     prm.C = C;
@@ -1113,6 +1116,8 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
     prm.n_tile = shape.n_tile;
     prm.num_k_tiles = (K + prm.n_tile - 1) / prm.n_tile;
     prm.num_pos = pl.a2;
+    prm.fd_k = make_fastdiv(static_cast<uint32_t>(prm.num_k_tiles));
+    prm.fd_keys = make_fastdiv(static_cast<uint32_t>(prm.num_k_tiles * pl.a2));
     prm.num_c_blocks = (C + GEMM_BLOCK_C - 1) / GEMM_BLOCK_C;
     prm.C = C;
     const int b_rows = prm.n_tile / shape.ctas;
@@ -1249,6 +1254,7 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
         if (rc != SDWINO_OK) return rc;
         const int p_blocks = shape.ctas * (shape.dual ? 2 : 1);      // blocks of 128 tiles per CTA tile / pair tile
         prm.num_p_tiles = (count / GEMM_BLOCK_P + p_blocks - 1) / p_blocks;
+        prm.fd_p = make_fastdiv(static_cast<uint32_t>(prm.num_p_tiles));
         rc = launch_gemm(tmU, tmV, tmM, prm, shape.ctas, st, q8);
         if (rc != SDWINO_OK) return rc;
         if (io32) {

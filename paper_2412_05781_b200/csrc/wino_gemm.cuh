@@ -109,6 +109,8 @@ struct GemmParams {
     const float* scales; // 8-bit filters: S[pos][kpad], the factor of every (position, output channel) row
     int kpad;            // Kb * 16
     int raw_slots;       // 8-bit filters: slots of the raw ring (at most GEMM_MAX_STAGES)
+    FastDiv fd_p, fd_k, fd_keys;   // divisions by num_p_tiles, num_k_tiles, num_k_tiles * num_pos (the roles are single
+                                   // threads: a hardware-less integer division is a few hundred cycles of their time)
 };
 
 // Pipelined mode (template flag PIPE): the three steps of a layer run inside ONE persistent launch.  V and M are rings
@@ -274,14 +276,15 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
     auto decode = [&](int tile, int& pt, int& kt, int& pos) {
         if constexpr (PIPE && !RES) {
             const int keys = prm.num_k_tiles * prm.num_pos;
-            pt = tile / keys;
+            pt = static_cast<int>(fast_div(static_cast<uint32_t>(tile), prm.fd_keys));
             const int key = tile - pt * keys;
-            pos = key / prm.num_k_tiles;
+            pos = static_cast<int>(fast_div(static_cast<uint32_t>(key), prm.fd_k));
             kt = key - pos * prm.num_k_tiles;
         } else {
-            pt = tile % prm.num_p_tiles;
-            kt = (tile / prm.num_p_tiles) % prm.num_k_tiles;
-            pos = tile / (prm.num_p_tiles * prm.num_k_tiles);
+            const int q = static_cast<int>(fast_div(static_cast<uint32_t>(tile), prm.fd_p));
+            pt = tile - q * prm.num_p_tiles;
+            pos = static_cast<int>(fast_div(static_cast<uint32_t>(q), prm.fd_k));
+            kt = q - pos * prm.num_k_tiles;
         }
     };
 
@@ -607,7 +610,7 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
                 const int tile = tile_of(i);
                 int key = 0;
                 if (resident) {
-                    key = tile / prm.num_p_tiles;      // pos * num_k_tiles + kt
+                    key = static_cast<int>(fast_div(static_cast<uint32_t>(tile), prm.fd_p));      // pos * num_k_tiles + kt
                     if (key != cur_key) {
                         ok = mbar_wait_bounded(ures_full_bar, loads_seen & 1u, abort_flag, GEMM_WAIT_LIMIT_NS);
                         if (!ok) { if (*abort_flag == 0) report_timeout(status_word, 6, cta_rank); break; }
@@ -674,7 +677,9 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
                 else umma_commit(&acc_full_bar[buf]);
                 if constexpr (DUAL) umma_commit(&acc_full_bar[1]);
                 // the last tile of a run: once its MMAs have completed the resident filters may be replaced
-                if (resident && i + 1 < my_count && tile_of(i + 1) / prm.num_p_tiles != key) umma_commit(ures_empty_bar);
+                if (resident && i + 1 < my_count &&
+                    static_cast<int>(fast_div(static_cast<uint32_t>(tile_of(i + 1)), prm.fd_p)) != key)
+                    umma_commit(ures_empty_bar);
                 if constexpr (DUAL) {
                     acc_phase ^= 1u;          // both buffers were used: buf stays 0
                 } else {
