@@ -792,17 +792,17 @@ GemmShape choose_gemm_shape(int K, int C, long long p_tiles128, int a2, int sms,
     return best;
 }
 
-template <int CTAS, bool RES, bool DUAL = false, bool U8 = false>
+template <int CTAS, bool RES, bool DUAL = false, bool U8 = false, bool STM = true>
 int launch_gemm_shape(const CUtensorMap& tmU, const CUtensorMap& tmV, const CUtensorMap& tmM, const GemmParams& prm,
                       int sms, int* status, cudaStream_t st) {
     using L = GemmSmemLayout;
-    if (!ensure_dyn_smem(reinterpret_cast<const void*>(wino_gemm_kernel<CTAS, RES, DUAL, false, U8>), MAX_DYN_SMEM)) return err_cuda(__LINE__);
+    if (!ensure_dyn_smem(reinterpret_cast<const void*>(wino_gemm_kernel<CTAS, RES, DUAL, false, U8, STM>), MAX_DYN_SMEM)) return err_cuda(__LINE__);
     const long long tiles = static_cast<long long>(prm.num_k_tiles) * prm.num_p_tiles * prm.num_pos;
     const long long workers = sms / CTAS;
     const int grid = static_cast<int>(tiles < workers ? tiles : workers) * CTAS;
     ProfScope prof(KIND_GEMM, st);
     const cudaError_t e =
-        launch_pdl(wino_gemm_kernel<CTAS, RES, DUAL, false, U8>, dim3(grid), dim3(GEMM_LAUNCH_THREADS),
+        launch_pdl(wino_gemm_kernel<CTAS, RES, DUAL, false, U8, STM>, dim3(grid), dim3(GEMM_LAUNCH_THREADS),
                    static_cast<size_t>(L::dyn_bytes(RES ? 0 : prm.n_tile / CTAS, prm.stages, prm.epi_rows,
                                                     prm.epi_alias ? 0 : prm.epi_bufs,
                                                     RES ? prm.num_c_blocks * L::b_bytes(prm.n_tile)
@@ -822,9 +822,13 @@ int launch_gemm(const CUtensorMap& tmU, const CUtensorMap& tmV, const CUtensorMa
     if (sms <= 0) return err_cuda(__LINE__);
     int* status = status_word_ptr();
     if (!status) return err_cuda(__LINE__);
-    if (q8) return launch_gemm_shape<1, false, false, true>(tmU, tmV, tmM, prm, sms, status, st);
+    if (q8) return launch_gemm_shape<1, false, false, true, false>(tmU, tmV, tmM, prm, sms, status, st);
     if (ctas == 2) return launch_gemm_shape<2, false>(tmU, tmV, tmM, prm, sms, status, st);
     if (prm.resident) return launch_gemm_shape<1, true>(tmU, tmV, tmM, prm, sms, status, st);
+    if (!prm.epi_stm) {   // one tile per CTA: single CTAs in streaming mode
+        if (prm.dual) return launch_gemm_shape<1, false, true, false, false>(tmU, tmV, tmM, prm, sms, status, st);
+        return launch_gemm_shape<1, false, false, false, false>(tmU, tmV, tmM, prm, sms, status, st);
+    }
     if (prm.dual) return launch_gemm_shape<1, false, true>(tmU, tmV, tmM, prm, sms, status, st);
     return launch_gemm_shape<1, false>(tmU, tmV, tmM, prm, sms, status, st);
 }
@@ -944,6 +948,8 @@ int launch_pipeline(const __half* x, const void* wT, const __half* bias, __half*
     prm.scales = nullptr;
     prm.kpad = pl.Kb * 16;
     prm.raw_slots = 0;
+    prm.epi_stm = 1;
+    prm.epi_dbuf = 0;
 
     PipeParams pp;
     pp.v_ready = ctr;
@@ -976,7 +982,7 @@ int launch_pipeline(const __half* x, const void* wT, const __half* bias, __half*
     CUtensorMap tmU, tmV, tmM;
     if (!encode_filter_map(&tmU, wt_filters_of(wT), pl.Cb, pl.Kb, pl.a2, pq.n_tile / 16) ||
         !encode_map(&tmV, V, ring_p, C, pl.a2, ring_p, static_cast<uint64_t>(C) * ring_p, 64, GEMM_BLOCK_C, true) ||
-        !encode_map(&tmM, Mws, ring_p, K, pl.a2, ring_p, static_cast<uint64_t>(K) * ring_p, GEMM_BLOCK_P, prm.epi_rows, false))
+        !encode_map(&tmM, Mws, ring_p, K, pl.a2, ring_p, static_cast<uint64_t>(K) * ring_p, 64, prm.epi_rows, true))
         return err_cuda(__LINE__);
     if (cudaMemsetAsync(ctr, 0, (3 * static_cast<size_t>(pq.nb) + 8) * sizeof(unsigned int), st) != cudaSuccess)
         return err_cuda(__LINE__);
@@ -1221,12 +1227,27 @@ int conv_impl(const void* x, const void* wT, const void* bias, void* y, int N, i
         prm.epi_rows = best_rows;
         prm.stages = best_stages;
     }
+    // Epilogue staging: stmatrix into swizzled boxes where a CTA has several tiles (throughput: 3-8 % on those GEMMs),
+    // plain 2-byte stores into one box where it has one (its two TMA stores of 128-byte rows drain later at the tail
+    // of the launch: 0.5-1.5 us per layer of the SD v1.5 sweep).
+    prm.epi_dbuf = 0;
+    if (!q8 && prm.epi_chunks >= 2 && prm.epi_rows == 64) {
+        // Two buffers of 32 channels in the place of one of 64: a group then stages one piece while the TMA store still
+        // reads the other, instead of waiting 1.3-1.8 thousand cycles for it between the pieces (-1.5 to -2 % on the
+        // GEMMs with several tiles per CTA).
+        prm.epi_dbuf = 1;
+        prm.epi_rows = 32;
+        prm.epi_chunks *= 2;
+        prm.epi_bufs *= 2;
+    }
+    prm.epi_stm = (!q8 && !prm.epi_alias) ? 1 : 0;   // (an aliased staging buffer implies single CTAs in streaming mode)
     prm.p_stride = pc;
     CUtensorMap tmU, tmV, tmM;
     if (!(q8 ? encode_filter_map_q8(&tmU, wt_filters_of(wT), pl.Cb, pl.Kb, pl.a2, b_rows / 16)
              : encode_filter_map(&tmU, wt_filters_of(wT), pl.Cb, pl.Kb, pl.a2, b_rows / 16)) ||
         !encode_map(&tmV, V, pc, C, pl.a2, pc, static_cast<uint64_t>(C) * pc, 64, GEMM_BLOCK_C, true) ||
-        !encode_map(&tmM, Mws, pc, K, pl.a2, pc, static_cast<uint64_t>(K) * pc, GEMM_BLOCK_P, prm.epi_rows, false))
+        !encode_map(&tmM, Mws, pc, K, pl.a2, pc, static_cast<uint64_t>(K) * pc, prm.epi_stm ? 64 : GEMM_BLOCK_P, prm.epi_rows,
+                    prm.epi_stm != 0))
         return err_cuda(__LINE__);
 
     const TileGeom geo = make_geom(H, W, pl.TH, pl.TW, pl.P, stride > 0 ? stride : 1);

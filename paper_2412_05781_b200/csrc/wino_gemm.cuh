@@ -99,6 +99,10 @@ struct GemmParams {
     int epi_rows;      // channels staged per TMA store and epilogue group: n_tile or n_tile / 2, multiple of 16
     int epi_bufs;      // staging buffers = epilogue groups with work (1 or 2)
     int epi_chunks;    // TMA stores per group and tile: a group drains epi_rows * epi_chunks channels
+    int epi_dbuf;      // 1: a group alternates between two staging buffers of epi_rows channels, so that it rounds and
+                       // stages one piece while the TMA store still reads the other (epi_bufs then counts both)
+    int epi_stm;       // 1: staging through stmatrix into two swizzled boxes of 64 tiles (tmM has that box); 0: 2-byte
+                       // stores into one plain box of 128 tiles (launches of one tile per CTA, whose tail it shortens)
     int resident;      // 1: the filter blocks of a (position, k-tile) stay in shared memory while the CTA walks the
                        // tiles p of that pair (stages then hold V only)
     int group;         // filter-resident mode: CTAs that share out the tiles of one (position, k-tile) pair
@@ -184,7 +188,8 @@ __device__ __forceinline__ void signal_counter_release(unsigned int* ctr) {
 // tmV: fp16 [pos][C][Pstride]   box {64 p, 64 c, 1},      128B swizzle  (A operand; rows c >= C read as 0)
 // tmU: fp16 [pos][Cb][Kb][16][64] box {64 c, 16 k, 1, n_tile/16, 1}, 128B swizzle (B operand: n_tile rows of 128
 //      bytes in k order; blocks past Kb read as 0)
-// tmM: fp16 [pos][K][Pstride]   box {128 p, epi_rows k, 1}, no swizzle  (result; rows k >= K are clipped)
+// tmM: fp16 [pos][K][Pstride]   box {64 p, epi_rows k, 1}, 128B swizzle (result; rows k >= K are clipped), or, with
+//      epi_stm == 0 (one tile per CTA, 8-bit filters): box {128 p, epi_rows k, 1}, no swizzle
 // RES: the filter-resident mode, DUAL: two blocks of 128 tiles per CTA tile; separate instantiations, so that the
 // plain streaming kernel pays nothing for them.
 // U8: 8-bit filters (see filter_quantize_kernel).  The producer brings the bytes of a filter box into the stage's raw
@@ -193,7 +198,10 @@ __device__ __forceinline__ void signal_counter_release(unsigned int* ctr) {
 // channel) row multiplies the accumulator in the epilogue.  Half the filter bytes cross HBM and L2; the contraction is
 // still kind::f16.  Meant for the weight-streaming layers (one tile per CTA): with several tiles per CTA the epilogue
 // of one tile no longer overlaps the mainloop of the next.
-template <int CTAS, bool RES = false, bool DUAL = false, bool PIPE = false, bool U8 = false>
+// STM: the epilogue stages M through stmatrix into two swizzled boxes of 64 tiles (launches whose CTAs have several
+// tiles); without it, through 2-byte stores into one plain box of 128 tiles (one tile per CTA, 8-bit filters).  A
+// template flag like the others: with both forms in one kernel either was 1-3 % slower.
+template <int CTAS, bool RES = false, bool DUAL = false, bool PIPE = false, bool U8 = false, bool STM = true>
 __global__ void __launch_bounds__(PIPE ? PIPE_THREADS : GEMM_LAUNCH_THREADS, 1)
 wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant__ CUtensorMap tmV,
                  const __grid_constant__ CUtensorMap tmM, const GemmParams prm, int* __restrict__ status_word,
@@ -201,6 +209,7 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
     using L = GemmSmemLayout;
     static_assert(!PIPE || (CTAS == 1 && !DUAL), "the pipelined mode runs single CTAs, one block of tiles per CTA tile");
     static_assert(!U8 || (CTAS == 1 && !RES && !DUAL && !PIPE), "8-bit filters: single CTAs, streaming mode");
+    static_assert(!(U8 && STM), "8-bit filters use the plain staging (their scales are fetched per column)");
     // The activation transform before this kernel has waited for everything before it, so the filter header is
     // final: its load is issued first and looked at after the set-up below (uniform over the CTA).
     const uint4 wt_hdr = *reinterpret_cast<const uint4*>(prm.wt_header);
@@ -701,6 +710,7 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
         const uint32_t acc_empty_addr0 = CTAS == 2 ? map_to_cta(smem_u32(&acc_empty_bar[0]), 0) : 0u;
         // one iteration per accumulator: a tile of two blocks of 128 tiles p (DUAL) fills both buffers, which are
         // drained in turn exactly as two consecutive tiles would be
+        int stg_seq = 0;                       // pieces staged so far by this group (selects the staging buffer)
         [[maybe_unused]] int pend_pt = -1;     // pipelined mode, group_tid 0: block whose stores are to be announced
         [[maybe_unused]] int cv_stage = 0;     // 8-bit filters: the stage these warps expand next
         [[maybe_unused]] uint32_t cv_phase = 0;
@@ -765,8 +775,8 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
                     if (++cv_raw == prm.raw_slots) { cv_raw = 0; cv_raw_par ^= 1u; }
                 }
             }
-            // the staging buffer about to be overwritten must have been read by the group's previous TMA store
-            if (group_tid == 0) tma_store_wait_read_pending<0>();
+            // the staging buffer about to be overwritten must have been read by the TMA store that used it last
+            if (group_tid == 0) { if (prm.epi_dbuf) tma_store_wait_read_pending<1>(); else tma_store_wait_read_pending<0>(); }
             [[maybe_unused]] unsigned int seen_o = 0;
             if constexpr (PIPE) {
                 if (group_tid == 0 && pt >= pp.ring) seen_o = ld_acquire_u32(&pp.o_done[pt - pp.ring]);   // used before the store
@@ -795,12 +805,61 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
             for (int ch = 0; ch < chunks; ++ch) {
             const int row0 = (group * chunks + ch) * prm.epi_rows;
             if (row0 < prm.n_tile) {
-                uint8_t* stg = epi_base + group * prm.epi_rows * L::EPI_ROW_BYTES;
+                uint8_t* stg = epi_base + (prm.epi_dbuf ? group * 2 + (stg_seq & 1) : group) * prm.epi_rows * L::EPI_ROW_BYTES;
+                ++stg_seq;
                 if (ch > 0) {   // (the first piece of a tile is ordered by the barrier after the accumulator wait)
-                    if (group_tid == 0) tma_store_wait_read_pending<0>();
+                    if (group_tid == 0) { if (prm.epi_dbuf) tma_store_wait_read_pending<1>(); else tma_store_wait_read_pending<0>(); }
                     if (group == 0) asm volatile("bar.sync 1, 128;" ::: "memory");
                     else asm volatile("bar.sync 2, 128;" ::: "memory");
                 }
+                if constexpr (STM) {
+                    // The staging buffer of a group is two boxes [epi_rows k][64 p] with the 128-byte swizzle of the
+                    // TMA store.  A warp reads its 32 lanes as two halves of 16 in the fragment layout of stmatrix
+                    // (thread t: lanes t / 4 and t / 4 + 8, columns 2 (t % 4), + 1 of every 8), rounds pairs of
+                    // columns with one packed conversion and stores four transposed 8 x 8 blocks per instruction:
+                    // matrix j of an instruction = tiles p 8 (j & 1) .. + 7, channels 8 (j >> 1) .. + 7 of a 16 x 16
+                    // piece, and thread 8 j + i supplies the 16-byte row of channel i of that matrix.  The swizzle
+                    // puts the eight rows of a matrix into eight different bank groups.
+                    const uint32_t stg_a = smem_u32(stg);
+                    const uint32_t sub_bytes = static_cast<uint32_t>(prm.epi_rows) * 128u;
+                    const int mj = lane >> 3, mi = lane & 7;
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const int p_local = quarter * 32 + 16 * h + (mj & 1) * 8;
+                        const uint32_t sub = stg_a + static_cast<uint32_t>(p_local >> 6) * sub_bytes;
+                        const uint32_t pc = static_cast<uint32_t>((p_local & 63) >> 3);
+                        const uint32_t t_h = t_addr + (static_cast<uint32_t>(16 * h) << 16) + static_cast<uint32_t>(row0);
+                        auto store16 = [&](int c, const uint32_t* r) {
+                            const uint32_t krow = static_cast<uint32_t>(c + (mj >> 1) * 8 + mi);
+                            const __half2 a = __floats2half2_rn(__uint_as_float(r[0]), __uint_as_float(r[1]));
+                            const __half2 b = __floats2half2_rn(__uint_as_float(r[2]), __uint_as_float(r[3]));
+                            const __half2 c2 = __floats2half2_rn(__uint_as_float(r[4]), __uint_as_float(r[5]));
+                            const __half2 d = __floats2half2_rn(__uint_as_float(r[6]), __uint_as_float(r[7]));
+                            stmatrix_x4_trans(sub + krow * 128u + ((pc ^ (krow & 7u)) << 4),
+                                              *reinterpret_cast<const uint32_t*>(&a), *reinterpret_cast<const uint32_t*>(&b),
+                                              *reinterpret_cast<const uint32_t*>(&c2), *reinterpret_cast<const uint32_t*>(&d));
+                        };
+                        int col = 0;
+                        for (; col + 64 <= prm.epi_rows; col += 64) {
+                            uint32_t r[32];
+                            tmem_ld_16x256_sync<8>(t_h + col, r);
+#pragma unroll
+                            for (int jj = 0; jj < 4; ++jj) store16(col + 16 * jj, r + 8 * jj);
+                        }
+                        if (col + 32 <= prm.epi_rows) {
+                            uint32_t r[16];
+                            tmem_ld_16x256_sync<4>(t_h + col, r);
+                            store16(col, r);
+                            store16(col + 16, r + 8);
+                            col += 32;
+                        }
+                        if (col + 16 <= prm.epi_rows) {
+                            uint32_t r[8];
+                            tmem_ld_16x256_sync<2>(t_h + col, r);
+                            store16(col, r);
+                        }
+                    }
+                } else {
                 __half* dst = reinterpret_cast<__half*>(stg) + quarter * 32 + lane;
                 // 8-bit filters: the factor of every output channel of this position (rows past K read padding)
                 [[maybe_unused]] const float* sc = U8 ? prm.scales + static_cast<long long>(pos) * prm.kpad + k0 + row0 : nullptr;
@@ -838,6 +897,7 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
                         dst[(col + i) * GEMM_BLOCK_P] = __float2half_rn(v);
                     }
                 }
+                }   // U8: plain staging
                 fence_proxy_async_smem();
                 if (group == 0) asm volatile("bar.sync 1, 128;" ::: "memory");
                 else asm volatile("bar.sync 2, 128;" ::: "memory");
@@ -857,8 +917,15 @@ wino_gemm_kernel(const __grid_constant__ CUtensorMap tmU, const __grid_constant_
                             fence_proxy_async_all();
                         }
                     }
-                    if (p_ok && (slot_free || *abort_flag == 0))
-                        tma_store_3d_hint(&tmM, stg, p0 - quarter * 32, k0 + row0, pos, l2_policy_evict_last());
+                    if (p_ok && (slot_free || *abort_flag == 0)) {
+                        if constexpr (!STM) {
+                            tma_store_3d_hint(&tmM, stg, p0 - quarter * 32, k0 + row0, pos, l2_policy_evict_last());
+                        } else {
+                            const uint64_t pol = l2_policy_evict_last();
+                            tma_store_3d_hint(&tmM, stg, p0 - quarter * 32, k0 + row0, pos, pol);
+                            tma_store_3d_hint(&tmM, stg + prm.epi_rows * 128, p0 - quarter * 32 + 64, k0 + row0, pos, pol);
+                        }
+                    }
                     tma_store_commit();
                     if constexpr (PIPE) {
                         if (ch == chunks - 1) {
