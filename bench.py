@@ -54,23 +54,23 @@ PAPER_CONTEXT = {"per_layer_speedup_vs_sdcpp_m1pro": 2.76, "end_to_end_speedup_v
 # records the capture it came from and the hash of the kernel sources it was taken with; `roofline.traffic` is null,
 # with the reason, when the sources have changed since.
 GEMM_DRAM_TRAFFIC = {
-    "single": {"bytes_per_launch": 1935104, "launches": 1, "source_hash": "040a4471e1e1",
+    "single": {"bytes_per_launch": 2134272, "launches": 1, "source_hash": "efa84ef76a2a",
                   "capture": "ncu --metrics dram__bytes_read.sum,dram__bytes_write.sum,gpu__time_duration.sum --cache-control none "
                              "--clock-control none -k regex:wino_gemm -s 3 -c 1 python bench.py --workload single --no-cpu-baseline "
                              "--no-yardstick --no-e2e --no-sustained --no-graph --steps 2 --warmup 3 (one pass per launch; the fourth step)"},
-    "sd15_unet": {"bytes_per_launch": 45278617, "launches": 15, "source_hash": "040a4471e1e1",
+    "sd15_unet": {"bytes_per_launch": 45421380, "launches": 15, "source_hash": "efa84ef76a2a",
                   "capture": "ncu --metrics dram__bytes_read.sum,dram__bytes_write.sum,gpu__time_duration.sum --cache-control none "
                              "--clock-control none -k regex:wino_gemm -s 45 -c 15 python bench.py --workload sd15_unet --no-cpu-baseline "
                              "--no-yardstick --no-e2e --no-sustained --no-graph --steps 2 --warmup 3 (one pass per launch; the fourth step)"},
-    "sd_vae_512": {"bytes_per_launch": 275657696, "launches": 8, "source_hash": "040a4471e1e1",
+    "sd_vae_512": {"bytes_per_launch": 270605760, "launches": 8, "source_hash": "efa84ef76a2a",
                   "capture": "ncu --metrics dram__bytes_read.sum,dram__bytes_write.sum,gpu__time_duration.sum --cache-control none "
                              "--clock-control none -k regex:wino_gemm -s 24 -c 8 python bench.py --workload sd_vae_512 --no-cpu-baseline "
                              "--no-yardstick --no-e2e --no-sustained --no-graph --steps 2 --warmup 3 (one pass per launch; the fourth step)"},
-    "sd21_unet": {"bytes_per_launch": 50989243, "launches": 15, "source_hash": "040a4471e1e1",
+    "sd21_unet": {"bytes_per_launch": 51061486, "launches": 15, "source_hash": "efa84ef76a2a",
                   "capture": "ncu --metrics dram__bytes_read.sum,dram__bytes_write.sum,gpu__time_duration.sum --cache-control none "
                              "--clock-control none -k regex:wino_gemm -s 45 -c 15 python bench.py --workload sd21_unet --no-cpu-baseline "
                              "--no-yardstick --no-e2e --no-sustained --no-graph --steps 2 --warmup 3 (one pass per launch; the fourth step)"},
-    "sdxl_1024": {"bytes_per_launch": 473784620, "launches": 23, "source_hash": "040a4471e1e1",
+    "sdxl_1024": {"bytes_per_launch": 473147325, "launches": 23, "source_hash": "efa84ef76a2a",
                   "capture": "ncu --metrics dram__bytes_read.sum,dram__bytes_write.sum,gpu__time_duration.sum --cache-control none "
                              "--clock-control none -k regex:wino_gemm -s 69 -c 23 python bench.py --workload sdxl_1024 --no-cpu-baseline "
                              "--no-yardstick --no-e2e --no-sustained --no-graph --steps 2 --warmup 3 (one pass per launch; the fourth step)"},
